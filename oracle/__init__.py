@@ -1,0 +1,112 @@
+"""fp64 CPU oracle for RMSNorm / softmax / cross-entropy forward (ctypes wrapper).
+
+TEST INFRASTRUCTURE, NOT THE PRODUCT: only the test-suite, the smoke check and the
+benchmark's CPU-baseline leg may import this package.  It shares nothing with the
+CUDA library and never imports it.  All arithmetic lives in ``ak_oracle.c`` (plain C,
+double precision, the textbook definition of each op); this file only marshals numpy
+arrays.  Inputs are bf16 *bit patterns* (``uint16``); outputs are ``float64``.
+
+Ops follow Table 3 of the paper (softmax / rmsnorm / cross_ent rows) with the
+semantics of the PyTorch reference implementation the paper names as its correctness
+oracle (Section 6).  Readings the paper does not pin ("parity unpinned", PyTorch
+convention): fully -inf softmax row -> NaN; inf/NaN inputs propagate; eps = 0 with a
+zero row -> NaN; all rows ignored -> mean NaN; out-of-range target -> NaN row.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+from .build import build as _build, LIB_PATH as _LIB_PATH
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _build()  # no-op when the shared object is newer than its source
+        lib = ctypes.CDLL(_LIB_PATH)
+        i64, f32 = ctypes.c_int64, ctypes.c_float
+        p = ctypes.c_void_p
+        lib.oracle_bf16_to_f64.argtypes = [p, p, i64]
+        lib.oracle_bf16_to_f64.restype = None
+        lib.oracle_set_threads.argtypes = [ctypes.c_int]
+        lib.oracle_set_threads.restype = ctypes.c_int
+        lib.oracle_rmsnorm.argtypes = [p, p, p, i64, i64, f32]
+        lib.oracle_rmsnorm.restype = None
+        lib.oracle_softmax.argtypes = [p, p, i64, i64]
+        lib.oracle_softmax.restype = None
+        lib.oracle_xent.argtypes = [p, p, i64, p, p, p, i64, i64]
+        lib.oracle_xent.restype = None
+        _lib = lib
+    return _lib
+
+
+def _bits(a, shape=None) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    if a.dtype != np.uint16:
+        raise TypeError(f"bf16 bit patterns must be uint16, got {a.dtype}")
+    if shape is not None and a.shape != shape:
+        raise ValueError(f"expected shape {shape}, got {a.shape}")
+    return a
+
+
+def set_threads(n: int = 0) -> int:
+    """Set (n > 0) or query (n = 0) the number of row-loop threads."""
+    return int(_load().oracle_set_threads(int(n)))
+
+
+def bf16_to_f64(bits) -> np.ndarray:
+    """Exact widening of bf16 bit patterns to float64."""
+    b = _bits(bits)
+    out = np.empty(b.shape, dtype=np.float64)
+    _load().oracle_bf16_to_f64(b.ctypes.data, out.ctypes.data, b.size)
+    return out
+
+
+def rmsnorm(x_bits, w_bits, eps: float) -> np.ndarray:
+    """y[r, j] = x[r, j] * w[j] / sqrt(mean_j(x[r, :]^2) + eps), in float64.
+
+    ``eps`` is first rounded to float32 (that is what the GPU entry point receives).
+    """
+    x = _bits(x_bits)
+    if x.ndim != 2:
+        raise ValueError("x must be [rows, D]")
+    rows, D = x.shape
+    w = _bits(w_bits, (D,))
+    y = np.empty((rows, D), dtype=np.float64)
+    _load().oracle_rmsnorm(x.ctypes.data, w.ctypes.data, y.ctypes.data, rows, D,
+                           float(np.float32(eps)))
+    return y
+
+
+def softmax(x_bits) -> np.ndarray:
+    """Row-wise exp(x - max) / sum exp(x - max) over the last dim, in float64."""
+    x = _bits(x_bits)
+    if x.ndim != 2:
+        raise ValueError("x must be [rows, D]")
+    rows, D = x.shape
+    y = np.empty((rows, D), dtype=np.float64)
+    _load().oracle_softmax(x.ctypes.data, y.ctypes.data, rows, D)
+    return y
+
+
+def xent(logits_bits, targets, ignore_index: int = -100):
+    """Returns (loss_rows float64 [rows], loss_mean float, n_counted int)."""
+    x = _bits(logits_bits)
+    if x.ndim != 2:
+        raise ValueError("logits must be [rows, V]")
+    rows, V = x.shape
+    t = np.ascontiguousarray(targets)
+    if t.dtype != np.int64 or t.shape != (rows,):
+        raise TypeError("targets must be int64 [rows]")
+    loss = np.empty((rows,), dtype=np.float64)
+    mean = ctypes.c_double(float("nan"))
+    cnt = ctypes.c_int64(0)
+    _load().oracle_xent(x.ctypes.data, t.ctypes.data, int(ignore_index),
+                        loss.ctypes.data, ctypes.addressof(mean), ctypes.addressof(cnt),
+                        rows, V)
+    return loss, float(mean.value), int(cnt.value)
