@@ -1,0 +1,177 @@
+/*
+ * ak.h - C ABI of libak: row-reduction kernels for NVIDIA B200 (sm_100a).
+ *
+ * Three forward ops over contiguous row-major bf16 [rows, D] tensors:
+ *   RMSNorm            (paper Table 3, row "rmsnorm";   Table 4 rows "rmsnorm")
+ *   last-dim softmax   (paper Table 3, row "softmax";   Table 4 rows "softmax")
+ *   fused cross-entropy(paper Table 3, row "cross_ent": online log-sum-exp fused with
+ *                       the NLL gather; Table 4 rows "cross_ent")
+ * Semantics are those of the PyTorch reference ops the paper uses as its correctness
+ * oracle (Section 6): F.rms_norm, F.softmax(dim=-1), F.cross_entropy(ignore_index).
+ *
+ * Conventions for every entry point unless stated otherwise
+ *   - Pointers named *_dev / without suffix in the device entry points are DEVICE
+ *     pointers valid on the current CUDA device.  The caller owns them for the whole
+ *     asynchronous lifetime of the call; the library neither frees nor retains them.
+ *   - Tensors are dense row-major, row stride == D (or V) elements; bf16 = the upper 16
+ *     bits of an IEEE-754 binary32.  Any D >= 1 and any 2-byte-aligned bf16 pointer is
+ *     accepted; the fastest paths need 16-byte aligned base pointers and D % 8 == 0.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Device entry points only enqueue work; they never synchronise.
+ *   - The return value is an ak_status.  Arguments are validated on the host before any
+ *     launch.  Data-dependent problems (an out-of-range target) cannot be reported
+ *     synchronously and are encoded in the output (NaN); no kernel ever traps.
+ *   - rows == 0 is legal: nothing is launched (cross-entropy still writes loss_mean = NaN).
+ *   - Determinism: same inputs, shape, pointer alignment, library build and GPU model
+ *     give bit-identical outputs.  Path selection is a pure function of
+ *     (rows, D, pointer alignment); no float atomics, no order-dependent reductions.
+ *   - y may alias x exactly (in-place) for RMSNorm and softmax; partial overlap is
+ *     undefined.
+ *   - Re-entrant; safe to call concurrently on different streams.
+ */
+#ifndef AK_H_
+#define AK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    AK_OK = 0,
+    AK_ERR_NULL = 1,   /* a required pointer is NULL */
+    AK_ERR_SHAPE = 2,  /* rows < 0, D <= 0, or a size the chosen path cannot take */
+    AK_ERR_ALIGN = 3,  /* pointer not aligned to its element type (or to 16 B where a forced path needs it) */
+    AK_ERR_ARG = 4,    /* eps negative or not finite; unknown path id; bad nsplit */
+    AK_ERR_CUDA = 5,   /* a CUDA runtime call or launch failed */
+    AK_ERR_NOMEM = 6   /* scratch allocation failed or caller workspace too small */
+} ak_status;
+
+/* Path ids for the *_path entry points (testing / tuning).  0 always means "let the
+ * dispatcher choose", which is what the plain entry points do. */
+enum {
+    AK_PATH_AUTO = 0,
+    AK_PATH_WARP = 1,     /* one warp per row, row held in registers; D % 8 == 0, D <= 2048, 16 B aligned */
+    AK_PATH_CTA = 2,      /* one CTA per row, row held in registers;  D % 8 == 0, D <= 32768, 16 B aligned */
+    AK_PATH_GENERIC = 3   /* any D, any 2-byte alignment; row re-read from L1/L2, single DRAM pass */
+};
+enum {
+    AK_XENT_AUTO = 0,
+    AK_XENT_ROW = 1,      /* one CTA streams a whole row (online max / sum-exp), loss written directly */
+    AK_XENT_SPLIT = 2     /* nsplit CTAs per row write partial (max, sum-exp); a merge kernel finishes */
+};
+
+/* ---------------------------------------------------------------------------------
+ * RMSNorm forward (Table 3 "rmsnorm": warp-shuffle reduction, fast rsqrt; the weight
+ * multiply is fused into the epilogue as in Section 7.3, Tier 3).
+ *   y[r, j] = bf16_rne( x[r, j] * w[j] * rsqrt( (1/D) sum_k x[r, k]^2 + eps ) )
+ * x, y: device bf16 [rows, D]; w: device bf16 [D]; accumulation in fp32.
+ * eps must be finite and >= 0.
+ */
+int ak_rmsnorm_fwd(const void* x, const void* w, void* y,
+                   int64_t rows, int64_t D, float eps, void* cuda_stream);
+int ak_rmsnorm_fwd_path(const void* x, const void* w, void* y,
+                        int64_t rows, int64_t D, float eps, void* cuda_stream, int path);
+
+/* ---------------------------------------------------------------------------------
+ * Softmax forward over the last dimension (Table 3 "softmax").
+ *   m = max_k x[r, k];  y[r, j] = bf16_rne( exp(x[r, j] - m) / sum_k exp(x[r, k] - m) )
+ * -inf entries (a causal mask lives in the data) give exactly 0.  A row that is all
+ * -inf, or contains +inf or NaN, gives NaN (IEEE / PyTorch convention).
+ */
+int ak_softmax_fwd(const void* x, void* y, int64_t rows, int64_t D, void* cuda_stream);
+int ak_softmax_fwd_path(const void* x, void* y, int64_t rows, int64_t D,
+                        void* cuda_stream, int path);
+
+/* ---------------------------------------------------------------------------------
+ * Fused cross-entropy forward (Table 3 "cross_ent": online log-sum-exp, fused NLL).
+ *   t = targets[r]
+ *   t == ignore_index        : loss_rows[r] = 0, row not counted (its logits are not read)
+ *   t < 0 or t >= V          : loss_rows[r] = NaN, row counted (so the mean is NaN)
+ *   otherwise                : loss_rows[r] = (m - x[r, t]) + log(sum_k exp(x[r, k] - m))
+ *   loss_mean[0] = (sum of counted loss_rows, fp64, fixed order) / n_counted   (0/0 = NaN)
+ * logits: device bf16 [rows, V]; targets: device int64 [rows]; loss_rows: device fp32
+ * [rows] (required); loss_mean: device fp32 [1] or NULL (mean skipped).
+ * Rows with very long vocabularies or too few rows to fill the GPU take the split-row
+ * two-phase path, which needs rows * nsplit * 8 bytes of scratch: ak_xent_fwd obtains it
+ * with cudaMallocAsync / cudaFreeAsync on `cuda_stream` (stream-ordered; AK_ERR_NOMEM on
+ * failure); ak_xent_fwd_ws takes it from the caller instead.
+ */
+int ak_xent_fwd(const void* logits, const int64_t* targets, int64_t ignore_index,
+                float* loss_rows, float* loss_mean,
+                int64_t rows, int64_t V, void* cuda_stream);
+
+/* Bytes of scratch ak_xent_fwd_ws needs for this shape (0 when the dispatcher picks the
+ * one-CTA-per-row path).  Pure function of (rows, V). */
+size_t ak_xent_workspace_bytes(int64_t rows, int64_t V);
+
+/* Same as ak_xent_fwd but never allocates: `workspace` is a device buffer of at least
+ * ak_xent_workspace_bytes(rows, V) bytes, 8-byte aligned, owned by the caller and free
+ * to reuse once the work enqueued on `cuda_stream` has finished.  May be NULL when the
+ * required size is 0. */
+int ak_xent_fwd_ws(const void* logits, const int64_t* targets, int64_t ignore_index,
+                   float* loss_rows, float* loss_mean,
+                   int64_t rows, int64_t V, void* workspace, size_t workspace_bytes,
+                   void* cuda_stream);
+
+/* Testing / tuning variant: force the path and, for AK_XENT_SPLIT, the number of splits
+ * per row (1..64; 0 = dispatcher's choice).  Scratch is obtained as in ak_xent_fwd. */
+int ak_xent_fwd_path(const void* logits, const int64_t* targets, int64_t ignore_index,
+                     float* loss_rows, float* loss_mean,
+                     int64_t rows, int64_t V, void* cuda_stream, int path, int nsplit);
+
+/* ---------------------------------------------------------------------------------
+ * Row-sharded cross-entropy (one process per GPU, each holding a block of rows).  Per-row
+ * losses need no exchange; the scalar mean needs one: every rank computes its pair
+ * {sum of counted loss_rows (fp64, fixed order), number of counted rows (as a double)} with
+ * ak_xent_sum_count, the 16-byte pairs are all-gathered in rank order by the caller (NCCL),
+ * and ak_xent_mean_merge adds them in index order and writes sum / count (0/0 = NaN), which
+ * is bit-identical on every rank.  The paper's system is single-GPU (Section "Limitations");
+ * this is the row-shard extension of the mean in ak_xent_fwd.
+ * sum_count: device double[2]; sum_count_pairs: device double[2 * n]; loss_mean: device fp32[1].
+ */
+int ak_xent_sum_count(const float* loss_rows, const int64_t* targets, int64_t ignore_index,
+                      int64_t rows, double* sum_count, void* cuda_stream);
+int ak_xent_mean_merge(const double* sum_count_pairs, int64_t n, float* loss_mean, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------
+ * Host-buffer variants: the same ops for callers whose tensors live in HOST memory
+ * (pinned memory gives full PCIe speed; pageable works).  Each call copies its inputs to
+ * a library-owned device arena in row chunks, runs the device kernels, copies results
+ * back, and returns after everything has completed (it synchronises its own internal
+ * streams only).  Copy-in, compute and copy-out of successive chunks overlap.  The arena
+ * is cached per device and grows on demand; ak_host_arena_release frees it.  Calls are
+ * serialised by an internal lock.  All pointers here are HOST pointers.
+ */
+int ak_rmsnorm_fwd_host(const void* x_host, const void* w_host, void* y_host,
+                        int64_t rows, int64_t D, float eps);
+int ak_softmax_fwd_host(const void* x_host, void* y_host, int64_t rows, int64_t D);
+int ak_xent_fwd_host(const void* logits_host, const int64_t* targets_host, int64_t ignore_index,
+                     float* loss_rows_host, float* loss_mean_host, int64_t rows, int64_t V);
+int ak_host_arena_release(void);
+
+/* ---------------------------------------------------------------------------------
+ * Introspection.
+ */
+/* Path id the dispatcher picks for (rows, D) with fully aligned pointers (`aligned16` != 0)
+ * or not.  Pure functions; no CUDA calls. */
+int ak_rmsnorm_choose_path(int64_t rows, int64_t D, int aligned16);
+int ak_softmax_choose_path(int64_t rows, int64_t D, int aligned16);
+/* Returns AK_XENT_ROW or AK_XENT_SPLIT and stores the split count (1 for ROW). */
+int ak_xent_choose_path(int64_t rows, int64_t V, int* nsplit_out);
+
+/* Number of kernel launches this library has enqueued in this process so far. */
+int64_t ak_launch_count(void);
+
+/* Static, never-freed description of a status code. */
+const char* ak_status_string(int status);
+
+/* Library version, major * 10000 + minor * 100 + patch. */
+int ak_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AK_H_ */

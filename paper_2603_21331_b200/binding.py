@@ -1,0 +1,238 @@
+"""ctypes binding of ``libak.so``: argument marshalling only.
+
+Every op runs in the CUDA library; nothing here computes, and there is no CPU or PyTorch
+fallback: if the shared object is missing or a call fails, an exception is raised.
+
+Two layers, same names as the C ABI (``include/ak.h``):
+
+* ``lib()`` returns the ``ctypes.CDLL`` with typed entry points (``lib().ak_rmsnorm_fwd``
+  etc.), taking raw device pointers as integers.
+* ``ak_rmsnorm_fwd / ak_softmax_fwd / ak_xent_fwd`` (and ``*_host``) take torch tensors,
+  check dtype / contiguity / device, and pass ``data_ptr()`` and the current CUDA stream.
+  PyTorch is used for device memory and streams only.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libak.so")
+
+AK_OK = 0
+AK_PATH_AUTO, AK_PATH_WARP, AK_PATH_CTA, AK_PATH_GENERIC = 0, 1, 2, 3
+AK_XENT_AUTO, AK_XENT_ROW, AK_XENT_SPLIT = 0, 1, 2
+
+_i64, _f32, _int, _p, _sz = (ctypes.c_int64, ctypes.c_float, ctypes.c_int, ctypes.c_void_p,
+                             ctypes.c_size_t)
+
+# name -> (restype, argtypes); mirrors include/ak.h one to one
+SIGNATURES = {
+    "ak_rmsnorm_fwd": (_int, [_p, _p, _p, _i64, _i64, _f32, _p]),
+    "ak_rmsnorm_fwd_path": (_int, [_p, _p, _p, _i64, _i64, _f32, _p, _int]),
+    "ak_softmax_fwd": (_int, [_p, _p, _i64, _i64, _p]),
+    "ak_softmax_fwd_path": (_int, [_p, _p, _i64, _i64, _p, _int]),
+    "ak_xent_fwd": (_int, [_p, _p, _i64, _p, _p, _i64, _i64, _p]),
+    "ak_xent_workspace_bytes": (_sz, [_i64, _i64]),
+    "ak_xent_fwd_ws": (_int, [_p, _p, _i64, _p, _p, _i64, _i64, _p, _sz, _p]),
+    "ak_xent_fwd_path": (_int, [_p, _p, _i64, _p, _p, _i64, _i64, _p, _int, _int]),
+    "ak_xent_sum_count": (_int, [_p, _p, _i64, _i64, _p, _p]),
+    "ak_xent_mean_merge": (_int, [_p, _i64, _p, _p]),
+    "ak_rmsnorm_fwd_host": (_int, [_p, _p, _p, _i64, _i64, _f32]),
+    "ak_softmax_fwd_host": (_int, [_p, _p, _i64, _i64]),
+    "ak_xent_fwd_host": (_int, [_p, _p, _i64, _p, _p, _i64, _i64]),
+    "ak_host_arena_release": (_int, []),
+    "ak_rmsnorm_choose_path": (_int, [_i64, _i64, _int]),
+    "ak_softmax_choose_path": (_int, [_i64, _i64, _int]),
+    "ak_xent_choose_path": (_int, [_i64, _i64, ctypes.POINTER(_int)]),
+    "ak_launch_count": (_i64, []),
+    "ak_status_string": (ctypes.c_char_p, [_int]),
+    "ak_version": (_int, []),
+}
+
+_lib = None
+
+
+class AkError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().ak_status_string(status).decode()
+        super().__init__(f"{where} failed: status {status} ({msg})")
+
+
+def lib() -> ctypes.CDLL:
+    """Load libak.so (once).  Raises if it has not been built: there is no fallback."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2603_21331_b200.build` "
+                "(the ops have no CPU or PyTorch fallback)")
+        l = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(l, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = l
+    return _lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != AK_OK:
+        raise AkError(status, where)
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, torch.cuda.Stream):
+        return stream.cuda_stream
+    return int(stream)
+
+
+def _dev_bf16(t: torch.Tensor, name: str, ndim: int) -> None:
+    if not (t.is_cuda and t.dtype == torch.bfloat16 and t.dim() == ndim and t.is_contiguous()):
+        raise TypeError(f"{name} must be a contiguous CUDA bfloat16 tensor with {ndim} dims")
+
+
+def _host(t: torch.Tensor, name: str, dtype, ndim: int) -> None:
+    if t.is_cuda or t.dtype != dtype or t.dim() != ndim or not t.is_contiguous():
+        raise TypeError(f"{name} must be a contiguous CPU {dtype} tensor with {ndim} dims")
+
+
+# ------------------------------------------------------------------------- device tensors
+def ak_rmsnorm_fwd(x: torch.Tensor, w: torch.Tensor, y: Optional[torch.Tensor] = None,
+                   eps: float = 1e-6, stream=None, path: int = AK_PATH_AUTO) -> torch.Tensor:
+    _dev_bf16(x, "x", 2)
+    _dev_bf16(w, "w", 1)
+    rows, D = x.shape
+    if w.shape[0] != D:
+        raise ValueError("w must have D elements")
+    if y is None:
+        y = torch.empty_like(x)
+    _dev_bf16(y, "y", 2)
+    if y.shape != x.shape:
+        raise ValueError("y must have the shape of x")
+    _check(lib().ak_rmsnorm_fwd_path(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, D, eps,
+                                     _stream_ptr(stream), path), "ak_rmsnorm_fwd")
+    return y
+
+
+def ak_softmax_fwd(x: torch.Tensor, y: Optional[torch.Tensor] = None, stream=None,
+                   path: int = AK_PATH_AUTO) -> torch.Tensor:
+    _dev_bf16(x, "x", 2)
+    rows, D = x.shape
+    if y is None:
+        y = torch.empty_like(x)
+    _dev_bf16(y, "y", 2)
+    if y.shape != x.shape:
+        raise ValueError("y must have the shape of x")
+    _check(lib().ak_softmax_fwd_path(x.data_ptr(), y.data_ptr(), rows, D, _stream_ptr(stream), path),
+           "ak_softmax_fwd")
+    return y
+
+
+def ak_xent_fwd(logits: torch.Tensor, targets: torch.Tensor, ignore_index: int = -100,
+                loss_rows: Optional[torch.Tensor] = None, loss_mean: Optional[torch.Tensor] = None,
+                stream=None, path: int = AK_XENT_AUTO, nsplit: int = 0,
+                want_mean: bool = True) -> Tuple[torch.Tensor, Optional[torch.Tensor]]:
+    _dev_bf16(logits, "logits", 2)
+    rows, V = logits.shape
+    if not (targets.is_cuda and targets.dtype == torch.int64 and targets.shape == (rows,)
+            and targets.is_contiguous()):
+        raise TypeError("targets must be a contiguous CUDA int64 tensor [rows]")
+    if loss_rows is None:
+        loss_rows = torch.empty((rows,), dtype=torch.float32, device=logits.device)
+    if loss_mean is None and want_mean:
+        loss_mean = torch.empty((1,), dtype=torch.float32, device=logits.device)
+    for t, n in ((loss_rows, rows), (loss_mean, 1)):
+        if t is not None and not (t.is_cuda and t.dtype == torch.float32 and t.numel() == n
+                                  and t.is_contiguous()):
+            raise TypeError("loss buffers must be contiguous CUDA float32 tensors")
+    mean_ptr = loss_mean.data_ptr() if loss_mean is not None else None
+    _check(lib().ak_xent_fwd_path(logits.data_ptr(), targets.data_ptr(), ignore_index,
+                                  loss_rows.data_ptr(), mean_ptr, rows, V, _stream_ptr(stream),
+                                  path, nsplit), "ak_xent_fwd")
+    return loss_rows, loss_mean
+
+
+def ak_xent_workspace_bytes(rows: int, V: int) -> int:
+    return int(lib().ak_xent_workspace_bytes(rows, V))
+
+
+def ak_xent_fwd_ws(logits: torch.Tensor, targets: torch.Tensor, workspace: Optional[torch.Tensor],
+                   ignore_index: int = -100, loss_rows: Optional[torch.Tensor] = None,
+                   loss_mean: Optional[torch.Tensor] = None, stream=None):
+    _dev_bf16(logits, "logits", 2)
+    rows, V = logits.shape
+    if loss_rows is None:
+        loss_rows = torch.empty((rows,), dtype=torch.float32, device=logits.device)
+    if loss_mean is None:
+        loss_mean = torch.empty((1,), dtype=torch.float32, device=logits.device)
+    ws_ptr = workspace.data_ptr() if workspace is not None else None
+    ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    _check(lib().ak_xent_fwd_ws(logits.data_ptr(), targets.data_ptr(), ignore_index,
+                                loss_rows.data_ptr(), loss_mean.data_ptr(), rows, V, ws_ptr, ws_bytes,
+                                _stream_ptr(stream)), "ak_xent_fwd_ws")
+    return loss_rows, loss_mean
+
+
+# ------------------------------------------------------------------------- host tensors
+def ak_rmsnorm_fwd_host(x: torch.Tensor, w: torch.Tensor, y: torch.Tensor, eps: float = 1e-6) -> torch.Tensor:
+    _host(x, "x", torch.bfloat16, 2)
+    _host(w, "w", torch.bfloat16, 1)
+    _host(y, "y", torch.bfloat16, 2)
+    rows, D = x.shape
+    _check(lib().ak_rmsnorm_fwd_host(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, D, eps),
+           "ak_rmsnorm_fwd_host")
+    return y
+
+
+def ak_softmax_fwd_host(x: torch.Tensor, y: torch.Tensor) -> torch.Tensor:
+    _host(x, "x", torch.bfloat16, 2)
+    _host(y, "y", torch.bfloat16, 2)
+    rows, D = x.shape
+    _check(lib().ak_softmax_fwd_host(x.data_ptr(), y.data_ptr(), rows, D), "ak_softmax_fwd_host")
+    return y
+
+
+def ak_xent_fwd_host(logits: torch.Tensor, targets: torch.Tensor, loss_rows: torch.Tensor,
+                     loss_mean: Optional[torch.Tensor], ignore_index: int = -100):
+    _host(logits, "logits", torch.bfloat16, 2)
+    _host(targets, "targets", torch.int64, 1)
+    _host(loss_rows, "loss_rows", torch.float32, 1)
+    rows, V = logits.shape
+    mean_ptr = loss_mean.data_ptr() if loss_mean is not None else None
+    _check(lib().ak_xent_fwd_host(logits.data_ptr(), targets.data_ptr(), ignore_index,
+                                  loss_rows.data_ptr(), mean_ptr, rows, V), "ak_xent_fwd_host")
+    return loss_rows, loss_mean
+
+
+# ------------------------------------------------------------------------- introspection
+def ak_rmsnorm_choose_path(rows: int, D: int, aligned16: bool = True) -> int:
+    return int(lib().ak_rmsnorm_choose_path(rows, D, int(aligned16)))
+
+
+def ak_softmax_choose_path(rows: int, D: int, aligned16: bool = True) -> int:
+    return int(lib().ak_softmax_choose_path(rows, D, int(aligned16)))
+
+
+def ak_xent_choose_path(rows: int, V: int) -> Tuple[int, int]:
+    ns = ctypes.c_int(0)
+    path = int(lib().ak_xent_choose_path(rows, V, ctypes.byref(ns)))
+    return path, int(ns.value)
+
+
+def ak_launch_count() -> int:
+    return int(lib().ak_launch_count())
+
+
+def ak_version() -> int:
+    return int(lib().ak_version())
+
+
+def ak_status_string(status: int) -> str:
+    return lib().ak_status_string(status).decode()

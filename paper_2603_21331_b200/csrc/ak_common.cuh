@@ -1,0 +1,126 @@
+// Shared device helpers for the row-reduction kernels (sm_100a).
+// bf16 pack/unpack, streaming 16-byte loads/stores, fixed-order warp/CTA reductions.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ak.h"
+
+namespace ak {
+
+constexpr int kWarp = 32;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// ---------------------------------------------------------------- bf16 <-> fp32
+// A 32-bit word holds two bf16: element 2i in the low half, 2i+1 in the high half.
+__device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+__device__ __forceinline__ float bf16_to_float(uint16_t b) { return __uint_as_float(((uint32_t)b) << 16); }
+
+// Two floats -> packed bf16x2 with round-to-nearest-even (one cvt instruction).
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ uint16_t float_to_bf16(float v) {
+    return (uint16_t)(pack_bf16x2(v, 0.0f) & 0xffffu);
+}
+
+// Packed bf16x2 max (exact; returns the non-NaN operand when one side is NaN).
+__device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
+// ---------------------------------------------------------------- memory
+// Activations are touched exactly once: streaming (evict-first) loads and stores keep
+// them from displacing the reusable weight vector in L2/L1.
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream(uint4* p, uint4 v) { __stcs(p, v); }
+__device__ __forceinline__ uint16_t ld_stream_u16(const uint16_t* p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream_u16(uint16_t* p, uint16_t v) { __stcs(p, v); }
+
+// exp2 on the SFU (max relative error 2^-22; ex2(-inf) = 0, ex2(NaN) = NaN).
+__device__ __forceinline__ float fast_exp2(float t) {
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(t));
+    return r;
+}
+
+// ---------------------------------------------------------------- reductions
+// XOR butterflies: fp add / max are commutative, so at every level both partners compute
+// the same bits and all lanes end with one identical value; the order of operations is
+// fixed by the lane ids, hence run-to-run deterministic.
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// CTA-wide reductions with ONE barrier each.  `slots` points to 2 * 32 floats of shared
+// memory; consecutive reductions must alternate `phase` (0/1): a warp can only pass the
+// barrier of reduction k+1 after every warp has finished reading the slots of
+// reduction k, so set k%2 is free again when reduction k+2 writes it.
+template <int THREADS>
+__device__ __forceinline__ float cta_sum(float v, float* slots, int phase) {
+    constexpr int NW = THREADS / kWarp;
+    v = warp_sum(v);
+    if constexpr (NW == 1) return v;
+    float* s = slots + phase * kWarp;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) s[warp] = v;
+    __syncthreads();
+    float t = (lane < NW) ? s[lane] : 0.0f;
+    return warp_sum(t);
+}
+template <int THREADS>
+__device__ __forceinline__ float cta_max(float v, float* slots, int phase) {
+    constexpr int NW = THREADS / kWarp;
+    v = warp_max(v);
+    if constexpr (NW == 1) return v;
+    float* s = slots + phase * kWarp;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) s[warp] = v;
+    __syncthreads();
+    float t = (lane < NW) ? s[lane] : -INFINITY;
+    return warp_max(t);
+}
+
+// ---------------------------------------------------------------- host-side plumbing
+// Launch bookkeeping shared by the translation units (defined in ak_api.cu).
+void count_launch(int n = 1);
+int sm_count();  // SMs of the current device (cached per device)
+
+// Per-op host dispatchers (each defined next to its kernels).  All arguments have been
+// validated; `path` is a concrete path id or AUTO.  They return an ak_status.
+int rmsnorm_dispatch(const void* x, const void* w, void* y, int64_t rows, int64_t D, float eps,
+                     cudaStream_t st, int path);
+int softmax_dispatch(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st, int path);
+int xent_dispatch(const void* logits, const int64_t* targets, int64_t ignore_index,
+                  float* loss_rows, float* loss_mean, int64_t rows, int64_t V,
+                  void* workspace, size_t workspace_bytes, bool may_allocate,
+                  cudaStream_t st, int path, int nsplit);
+// Fixed-order fp64 mean of loss_rows over rows whose target != ignore_index (one small launch).
+int xent_mean_launch(const float* loss_rows, const int64_t* targets, int64_t ignore_index, int64_t rows,
+                     float* loss_mean, cudaStream_t st);
+int xent_sum_count_launch(const float* loss_rows, const int64_t* targets, int64_t ignore_index, int64_t rows,
+                          double* sum_count, cudaStream_t st);
+int xent_mean_merge_launch(const double* pairs, int64_t n, float* loss_mean, cudaStream_t st);
+int rmsnorm_choose(int64_t rows, int64_t D, bool aligned16);
+int softmax_choose(int64_t rows, int64_t D, bool aligned16);
+int xent_choose(int64_t rows, int64_t V, int* nsplit);
+// CTA shape of the register-resident row paths: threads per CTA and 16-byte vectors per thread.
+void cta_shape(int nvec, int* threads, int* vpt);
+
+inline bool is_aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+}  // namespace ak

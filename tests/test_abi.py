@@ -1,0 +1,121 @@
+"""CPU-only checks of the C-ABI boundary: the library loads, exports every symbol the
+header declares, the binding mirrors the header, argument validation rejects bad calls
+before any CUDA work, and the dispatcher's choices are pure functions of the shape."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2603_21331_b200 as ak
+from paper_2603_21331_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _header_functions():
+    text = open(os.path.join(ROOT, "include", "ak.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ak_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = _header_functions()
+    assert {"ak_rmsnorm_fwd", "ak_softmax_fwd", "ak_xent_fwd"} <= set(names)
+    l = ak.lib()
+    for n in names:
+        assert hasattr(l, n), f"{n} declared in ak.h but not exported"
+    assert sorted(binding.SIGNATURES) == names, "binding and header disagree"
+    assert ak.ak_version() >= 100
+
+
+def test_status_strings():
+    seen = {ak.ak_status_string(s) for s in range(7)}
+    assert len(seen) == 7 and ak.ak_status_string(0) == "ok"
+    assert ak.ak_status_string(99) == "unknown status"
+
+
+def test_validation_rejects_before_any_cuda_call():
+    l = ak.lib()
+    P = 0x1000  # fake, never dereferenced: every call below must fail validation first
+    assert l.ak_rmsnorm_fwd(None, P, P, 1, 8, 1e-6, None) == 1
+    assert l.ak_rmsnorm_fwd(P, None, P, 1, 8, 1e-6, None) == 1
+    assert l.ak_rmsnorm_fwd(P, P, None, 1, 8, 1e-6, None) == 1
+    assert l.ak_rmsnorm_fwd(P, P, P, -1, 8, 1e-6, None) == 2
+    assert l.ak_rmsnorm_fwd(P, P, P, 1, 0, 1e-6, None) == 2
+    assert l.ak_rmsnorm_fwd(P + 1, P, P, 1, 8, 1e-6, None) == 3
+    assert l.ak_rmsnorm_fwd(P, P, P, 1, 8, -1.0, None) == 4
+    assert l.ak_rmsnorm_fwd(P, P, P, 1, 8, float("nan"), None) == 4
+    assert l.ak_rmsnorm_fwd(P, P, P, 1, 8, float("inf"), None) == 4
+    assert l.ak_rmsnorm_fwd_path(P, P, P, 1, 8, 1e-6, None, 9) == 4
+    assert l.ak_rmsnorm_fwd(P, P, P, 0, 8, 1e-6, None) == 0          # rows == 0: nothing to do
+    assert l.ak_rmsnorm_fwd(P, P, P, 1 << 40, 1 << 40, 1e-6, None) == 2
+    assert l.ak_softmax_fwd(None, P, 1, 8, None) == 1
+    assert l.ak_softmax_fwd(P, P, 1, -3, None) == 2
+    assert l.ak_softmax_fwd(P, P + 1, 1, 8, None) == 3
+    assert l.ak_softmax_fwd_path(P, P, 1, 8, None, -1) == 4
+    assert l.ak_softmax_fwd(P, P, 0, 8, None) == 0
+    assert l.ak_xent_fwd(None, P, -100, P, P, 1, 8, None) == 1
+    assert l.ak_xent_fwd(P, None, -100, P, P, 1, 8, None) == 1
+    assert l.ak_xent_fwd(P, P, -100, None, P, 1, 8, None) == 1
+    assert l.ak_xent_fwd(P, P, -100, P, P, 1, 0, None) == 2
+    assert l.ak_xent_fwd(P, P + 4, -100, P, P, 1, 8, None) == 3      # int64 targets need 8 B
+    assert l.ak_xent_fwd(P, P, -100, P + 2, P, 1, 8, None) == 3      # fp32 losses need 4 B
+    assert l.ak_xent_fwd_path(P, P, -100, P, P, 1, 8, None, 5, 0) == 4
+    assert l.ak_xent_fwd_path(P, P, -100, P, P, 1, 8, None, 2, 65) == 4
+    # workspace variant: too small / missing workspace for a shape that splits
+    need = ak.ak_xent_workspace_bytes(16, 128256)
+    assert need > 0
+    assert l.ak_xent_fwd_ws(P, P, -100, P, P, 16, 128256, None, 0, None) == 1
+    assert l.ak_xent_fwd_ws(P, P, -100, P, P, 16, 128256, P, need - 1, None) == 6
+    assert l.ak_xent_fwd_ws(P, P, -100, P, P, 16, 128256, P + 4, need, None) == 3
+    # host variants validate the same way
+    assert l.ak_rmsnorm_fwd_host(None, P, P, 1, 8, 1e-6) == 1
+    assert l.ak_softmax_fwd_host(P, P, -1, 8) == 2
+    assert l.ak_xent_fwd_host(P, P + 4, -100, P, P, 1, 8) == 3
+
+
+def test_dispatch_is_a_pure_function_of_shape_and_alignment():
+    assert ak.ak_rmsnorm_choose_path(8192, 1024, True) == ak.AK_PATH_WARP
+    assert ak.ak_rmsnorm_choose_path(8192, 4096, True) == ak.AK_PATH_CTA
+    assert ak.ak_rmsnorm_choose_path(8192, 32768, True) == ak.AK_PATH_CTA
+    assert ak.ak_rmsnorm_choose_path(8192, 4099, True) == ak.AK_PATH_GENERIC
+    assert ak.ak_rmsnorm_choose_path(8192, 4096, False) == ak.AK_PATH_GENERIC
+    assert ak.ak_rmsnorm_choose_path(8192, 65536, True) == ak.AK_PATH_GENERIC
+    assert ak.ak_softmax_choose_path(16384, 512, True) == ak.AK_PATH_WARP
+    assert ak.ak_softmax_choose_path(16384, 32768, True) == ak.AK_PATH_CTA
+    assert ak.ak_softmax_choose_path(16384, 128257, True) == ak.AK_PATH_GENERIC
+    for rows, V in ((4096, 32000), (4096, 128256), (16384, 128256)):
+        assert ak.ak_xent_choose_path(rows, V) == (ak.AK_XENT_ROW, 1)
+        assert ak.ak_xent_workspace_bytes(rows, V) == 0
+    path, ns = ak.ak_xent_choose_path(16, 128256)
+    assert path == ak.AK_XENT_SPLIT and 2 <= ns <= 64
+    assert ak.ak_xent_workspace_bytes(16, 128256) == 16 * ns * 8
+    assert ak.ak_xent_choose_path(1, 128256)[1] == 15            # capped by 8192-element slices
+    assert ak.ak_xent_choose_path(16, 1000) == (ak.AK_XENT_ROW, 1)  # short rows never split
+    # repeated queries agree (no hidden state)
+    assert all(ak.ak_xent_choose_path(16, 128256) == (path, ns) for _ in range(3))
+
+
+def test_binding_refuses_cpu_tensors_instead_of_falling_back():
+    import torch
+    x = torch.zeros((2, 8), dtype=torch.bfloat16)
+    with pytest.raises(TypeError):
+        ak.ak_rmsnorm_fwd(x, torch.ones(8, dtype=torch.bfloat16))
+    with pytest.raises(TypeError):
+        ak.ak_softmax_fwd(x)
+    with pytest.raises(TypeError):
+        ak.ak_xent_fwd(x, torch.zeros(2, dtype=torch.int64))
+
+
+def test_product_does_not_import_the_checker():
+    pkg = os.path.join(ROOT, "paper_2603_21331_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in text.lower(), f"{f} mentions the checker"
+    for f in os.listdir(os.path.join(ROOT, "oracle")):
+        if f.endswith((".py", ".c")):
+            text = open(os.path.join(ROOT, "oracle", f)).read()
+            assert "paper_2603_21331_b200" not in text and "libak" not in text

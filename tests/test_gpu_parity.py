@@ -1,0 +1,303 @@
+"""GPU parity: every CUDA path against the fp64 CPU checker, element by element, on the
+same seeded bf16 bit patterns, through the C ABI (ctypes binding)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2603_21331_b200 as ak
+from paper_2603_21331_b200 import synth
+from parity import assert_bf16_close, assert_loss_close, guarded
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+WARP, CTA, GEN = ak.AK_PATH_WARP, ak.AK_PATH_CTA, ak.AK_PATH_GENERIC
+
+
+def _legal_paths(D):
+    paths = [GEN]
+    if D % 8 == 0 and D <= 32768:
+        paths.append(CTA)
+    if D % 8 == 0 and D <= 2048:
+        paths.append(WARP)
+    return paths
+
+
+# shapes: several tiles plus ragged tails, every vectors-per-thread count of both register
+# paths, non-multiples of 8, the paper's edge sizes (1023, 1537, 4097) and the benchmark's
+# (4099); rows chosen so the checker stays fast
+SHAPES = [(256, 1024), (1, 8), (3, 16), (37, 64), (129, 256), (65, 512), (33, 776), (40, 1000),
+          (33, 1280), (19, 1536), (21, 1792), (64, 2048), (17, 4096), (1, 4096), (23, 3072),
+          (9, 5120), (16, 8192), (7, 11008), (12, 16384), (5, 20480), (3, 24576), (3, 28672),
+          (6, 32768), (5, 1), (4, 7), (31, 1023), (11, 1537), (9, 4097), (13, 4099), (2, 40000),
+          (3, 128257)]
+
+
+@pytest.mark.parametrize("rows,D", SHAPES)
+def test_rmsnorm_parity_all_paths(rows, D):
+    seed = 0 if (rows, D) == (256, 1024) else synth.case_seed(2, rows * 131 + D)
+    x, w = synth.rmsnorm_inputs(rows, D, seed)
+    ref = oracle.rmsnorm(synth.to_bits(x), synth.to_bits(w), 1e-6)
+    xd, wd = x.to(DEV), w.to(DEV)
+    outs = {}
+    for path in [ak.AK_PATH_AUTO] + _legal_paths(D):
+        y, check = guarded((rows, D), torch.bfloat16, DEV)
+        ak.ak_rmsnorm_fwd(xd, wd, y, eps=1e-6, path=path)
+        torch.cuda.synchronize()
+        check()
+        assert_bf16_close(y, ref, f"rmsnorm {rows}x{D} path {path}")
+        outs[path] = y.clone()
+    auto = ak.ak_rmsnorm_choose_path(rows, D, True)
+    assert torch.equal(outs[ak.AK_PATH_AUTO].view(torch.int16), outs[auto].view(torch.int16))
+
+
+@pytest.mark.parametrize("rows,D", SHAPES)
+def test_softmax_parity_all_paths(rows, D):
+    x = synth.softmax_inputs(rows, D, synth.case_seed(3, rows * 131 + D), mask_frac=0.3)
+    ref = oracle.softmax(synth.to_bits(x))
+    xd = x.to(DEV)
+    for path in [ak.AK_PATH_AUTO] + _legal_paths(D):
+        y, check = guarded((rows, D), torch.bfloat16, DEV)
+        ak.ak_softmax_fwd(xd, y, path=path)
+        torch.cuda.synchronize()
+        check()
+        assert_bf16_close(y, ref, f"softmax {rows}x{D} path {path}")
+        neg_inf = (xd.view(torch.int16) == -128)  # 0xFF80
+        assert bool((y[neg_inf].view(torch.int16) == 0).all()), "-inf entries must give exactly +0"
+        sums = y.float().sum(dim=-1)
+        assert bool(((sums - 1).abs() <= 4e-3 + 2e-3).all())
+
+
+XENT_SHAPES = [(4, 8), (64, 1000), (33, 4099), (5, 1), (7, 9), (40, 8192), (24, 32000),
+               (12, 50304), (8, 128256), (6, 128257), (300, 2048)]
+
+
+@pytest.mark.parametrize("rows,V", XENT_SHAPES)
+def test_xent_parity_row_and_split(rows, V):
+    logits, targets = synth.xent_inputs(rows, V, synth.case_seed(4, rows * 131 + V), ignore_frac=0.2)
+    ref_rows, ref_mean, n = oracle.xent(synth.to_bits(logits), targets.numpy())
+    ld, td = logits.to(DEV), targets.to(DEV)
+    variants = [(ak.AK_XENT_AUTO, 0), (ak.AK_XENT_ROW, 0)]
+    variants += [(ak.AK_XENT_SPLIT, ns) for ns in (1, 2, 3, 7, 64)]
+    for path, ns in variants:
+        loss, check = guarded((rows,), torch.float32, DEV)
+        mean, check_mean = guarded((1,), torch.float32, DEV)
+        ak.ak_xent_fwd(ld, td, -100, loss, mean, path=path, nsplit=ns)
+        torch.cuda.synchronize()
+        check()
+        check_mean()
+        assert_loss_close(loss, ref_rows, f"xent rows {rows}x{V} path {path}/{ns}")
+        assert_loss_close(mean, np.array([ref_mean]), f"xent mean {rows}x{V} path {path}/{ns}")
+        ign = td == -100
+        assert bool((loss[ign] == 0).all())
+        assert bool((loss[~ign] >= 0).all())
+    # caller-provided workspace variant gives the same bits as the allocating entry point
+    nbytes = ak.ak_xent_workspace_bytes(rows, V)
+    ws = torch.empty((max(nbytes, 8),), dtype=torch.uint8, device=DEV)
+    l1, m1 = ak.ak_xent_fwd(ld, td)
+    l2, m2 = ak.ak_xent_fwd_ws(ld, td, ws if nbytes else None)
+    torch.cuda.synchronize()
+    assert torch.equal(l1.view(torch.int32), l2.view(torch.int32))
+    assert torch.equal(m1.view(torch.int32), m2.view(torch.int32)) or (torch.isnan(m1).all() and torch.isnan(m2).all())
+
+
+def test_xent_mean_skipped_when_null():
+    logits, targets = synth.xent_inputs(16, 512, 7)
+    loss, mean = ak.ak_xent_fwd(logits.to(DEV), targets.to(DEV), want_mean=False)
+    torch.cuda.synchronize()
+    assert mean is None and loss.shape == (16,)
+
+
+def test_xent_conventions_bad_targets_and_all_ignored():
+    logits, _ = synth.xent_inputs(6, 40, 8)
+    ld = logits.to(DEV)
+    t = torch.tensor([0, 40, -1, -100, 39, 5], dtype=torch.int64)
+    ref_rows, ref_mean, n = oracle.xent(synth.to_bits(logits), t.numpy())
+    for path, ns in ((ak.AK_XENT_ROW, 0), (ak.AK_XENT_SPLIT, 3)):
+        loss, mean = ak.ak_xent_fwd(ld, t.to(DEV), path=path, nsplit=ns)
+        torch.cuda.synchronize()
+        assert_loss_close(loss, ref_rows, "bad targets")
+        assert torch.isnan(mean).all() and np.isnan(ref_mean)
+        t_ign = torch.full((6,), -100, dtype=torch.int64, device=DEV)
+        loss, mean = ak.ak_xent_fwd(ld, t_ign, path=path, nsplit=ns)
+        torch.cuda.synchronize()
+        assert bool((loss == 0).all()) and torch.isnan(mean).all()
+        # a custom ignore_index
+        t7 = torch.tensor([7, 1, 7, 2, 3, 7], dtype=torch.int64)
+        r7, m7, _ = oracle.xent(synth.to_bits(logits), t7.numpy(), ignore_index=7)
+        loss, mean = ak.ak_xent_fwd(ld, t7.to(DEV), ignore_index=7, path=path, nsplit=ns)
+        torch.cuda.synchronize()
+        assert_loss_close(loss, r7, "ignore_index=7")
+        assert_loss_close(mean, np.array([m7]), "ignore_index=7 mean")
+    # NaN planted in an ignored row must not leak; rows = 0 gives NaN mean
+    l2 = logits.clone()
+    l2[3, 4] = float("nan")
+    loss, mean = ak.ak_xent_fwd(l2.to(DEV), torch.tensor([0, 1, 2, -100, 4, 5], device=DEV))
+    torch.cuda.synchronize()
+    assert torch.isfinite(loss).all() and torch.isfinite(mean).all()
+    empty = torch.empty((0, 40), dtype=torch.bfloat16, device=DEV)
+    loss, mean = ak.ak_xent_fwd(empty, torch.empty((0,), dtype=torch.int64, device=DEV))
+    torch.cuda.synchronize()
+    assert loss.numel() == 0 and torch.isnan(mean).all()
+
+
+def test_softmax_ieee_conventions():
+    x = torch.zeros((4, 24), dtype=torch.bfloat16)
+    x[0, :] = float("-inf")           # fully masked row -> NaN
+    x[1, 3] = float("inf")            # +inf -> NaN row
+    x[2, 5] = float("nan")            # NaN -> NaN row
+    x[3, :] = torch.arange(24) * 0.25  # ordinary row
+    ref = oracle.softmax(synth.to_bits(x))
+    for path in (WARP, CTA, GEN):
+        y = ak.ak_softmax_fwd(x.to(DEV), path=path)
+        torch.cuda.synchronize()
+        assert_bf16_close(y, ref, f"softmax conventions path {path}")
+
+
+@pytest.mark.parametrize("kind", synth.ADVERSARIAL_KINDS)
+@pytest.mark.parametrize("D", [512, 4096, 4099])
+def test_adversarial_rows_all_ops(kind, D):
+    rows = 20
+    x, hot = synth.adversarial_rows(kind, rows, D, synth.case_seed(5, D))
+    xb = synth.to_bits(x)
+    xd = x.to(DEV)
+    _, w = synth.rmsnorm_inputs(1, D, 55)
+    ref = oracle.rmsnorm(xb, synth.to_bits(w), 1e-6)
+    for path in [ak.AK_PATH_AUTO] + _legal_paths(D):
+        y = ak.ak_rmsnorm_fwd(xd, w.to(DEV), eps=1e-6, path=path)
+        assert torch.isfinite(y.float()).all()
+        assert_bf16_close(y, ref, f"rmsnorm adversarial {kind} D={D} path {path}")
+    ref = oracle.softmax(xb)
+    for path in [ak.AK_PATH_AUTO] + _legal_paths(D):
+        y = ak.ak_softmax_fwd(xd, path=path)
+        assert torch.isfinite(y.float()).all()
+        assert_bf16_close(y, ref, f"softmax adversarial {kind} D={D} path {path}")
+    t = hot.clone()
+    t[1::2] = (t[1::2] + 1) % D       # half of the rows aim beside the planted logit
+    ref_rows, ref_mean, _ = oracle.xent(xb, t.numpy())
+    for path, ns in ((ak.AK_XENT_ROW, 0), (ak.AK_XENT_SPLIT, 2), (ak.AK_XENT_SPLIT, 5)):
+        loss, mean = ak.ak_xent_fwd(xd, t.to(DEV), path=path, nsplit=ns)
+        torch.cuda.synchronize()
+        assert torch.isfinite(loss).all() and torch.isfinite(mean).all()
+        assert bool((loss >= 0).all())
+        assert_loss_close(loss, ref_rows, f"xent adversarial {kind} V={D} path {path}/{ns}")
+        assert_loss_close(mean, np.array([ref_mean]), f"xent adversarial mean {kind} V={D}")
+
+
+def test_all_equal_softmax_4099_prints_two_to_minus_12():
+    # 1/4099 rounds to 2^-12 in bf16, so an all-equal row of length 4099 is 2^-12 everywhere
+    x = torch.full((2, 4099), 3.0, dtype=torch.bfloat16, device=DEV)
+    y = ak.ak_softmax_fwd(x)
+    assert bool((y.float() == 2.0 ** -12).all())
+
+
+def test_misaligned_base_pointers_take_generic_path():
+    D, rows = 1024, 9
+    x, w = synth.rmsnorm_inputs(rows, D, 91)
+    ref = oracle.rmsnorm(synth.to_bits(x), synth.to_bits(w), 1e-6)
+    for xo, yo, wo in ((1, 1, 0), (1, 3, 0), (0, 0, 5), (3, 0, 1)):
+        xbuf = torch.zeros(rows * D + 8, dtype=torch.bfloat16, device=DEV)
+        ybuf = torch.zeros(rows * D + 8, dtype=torch.bfloat16, device=DEV)
+        wbuf = torch.zeros(D + 8, dtype=torch.bfloat16, device=DEV)
+        xv = xbuf[xo:xo + rows * D].view(rows, D)
+        yv = ybuf[yo:yo + rows * D].view(rows, D)
+        wv = wbuf[wo:wo + D]
+        xv.copy_(x)
+        wv.copy_(w)
+        ak.ak_rmsnorm_fwd(xv, wv, yv, eps=1e-6)
+        torch.cuda.synchronize()
+        assert_bf16_close(yv, ref, f"rmsnorm offsets {xo},{yo},{wo}")
+        assert bool((ybuf[:yo] == 0).all()) and bool((ybuf[yo + rows * D:] == 0).all())
+    xs = synth.softmax_inputs(rows, D, 92)
+    ref = oracle.softmax(synth.to_bits(xs))
+    for xo, yo in ((1, 1), (5, 2)):
+        xbuf = torch.zeros(rows * D + 8, dtype=torch.bfloat16, device=DEV)
+        ybuf = torch.zeros(rows * D + 8, dtype=torch.bfloat16, device=DEV)
+        xv = xbuf[xo:xo + rows * D].view(rows, D)
+        yv = ybuf[yo:yo + rows * D].view(rows, D)
+        xv.copy_(xs)
+        ak.ak_softmax_fwd(xv, yv)
+        torch.cuda.synchronize()
+        assert_bf16_close(yv, ref, f"softmax offsets {xo},{yo}")
+        assert bool((ybuf[:yo] == 0).all()) and bool((ybuf[yo + rows * D:] == 0).all())
+    logits, targets = synth.xent_inputs(rows, 1000, 93)
+    ref_rows, ref_mean, _ = oracle.xent(synth.to_bits(logits), targets.numpy())
+    lbuf = torch.zeros(rows * 1000 + 8, dtype=torch.bfloat16, device=DEV)
+    lv = lbuf[3:3 + rows * 1000].view(rows, 1000)
+    lv.copy_(logits)
+    for path, ns in ((ak.AK_XENT_ROW, 0), (ak.AK_XENT_SPLIT, 3)):
+        loss, mean = ak.ak_xent_fwd(lv, targets.to(DEV), path=path, nsplit=ns)
+        torch.cuda.synchronize()
+        assert_loss_close(loss, ref_rows, "xent offset 3")
+
+
+def test_in_place_is_allowed():
+    for D, paths in ((512, (WARP, CTA, GEN)), (4096, (CTA, GEN)), (4099, (GEN,))):
+        x, w = synth.rmsnorm_inputs(11, D, 94)
+        ref = oracle.rmsnorm(synth.to_bits(x), synth.to_bits(w), 1e-6)
+        xs = synth.softmax_inputs(11, D, 95)
+        refs = oracle.softmax(synth.to_bits(xs))
+        for path in paths:
+            xd = x.to(DEV)
+            ak.ak_rmsnorm_fwd(xd, w.to(DEV), xd, eps=1e-6, path=path)
+            assert_bf16_close(xd, ref, f"in-place rmsnorm D={D} path {path}")
+            xd = xs.to(DEV)
+            ak.ak_softmax_fwd(xd, xd, path=path)
+            assert_bf16_close(xd, refs, f"in-place softmax D={D} path {path}")
+
+
+def test_bitwise_determinism_three_runs():
+    x, w = synth.rmsnorm_inputs(4096, 4096, 96)
+    xs = synth.softmax_inputs(2048, 8192, 97)
+    logits, targets = synth.xent_inputs(512, 32000, 98)
+    xd, wd, xsd, ld, td = x.to(DEV), w.to(DEV), xs.to(DEV), logits.to(DEV), targets.to(DEV)
+    first = None
+    for _ in range(3):
+        outs = [ak.ak_rmsnorm_fwd(xd, wd).view(torch.int16).clone(),
+                ak.ak_softmax_fwd(xsd).view(torch.int16).clone()]
+        for path, ns in ((ak.AK_XENT_ROW, 0), (ak.AK_XENT_SPLIT, 4)):
+            loss, mean = ak.ak_xent_fwd(ld, td, path=path, nsplit=ns)
+            outs += [loss.view(torch.int32).clone(), mean.view(torch.int32).clone()]
+        # disturb the machine between runs
+        torch.empty(64 << 20, dtype=torch.uint8, device=DEV).fill_(1)
+        torch.cuda.synchronize()
+        if first is None:
+            first = outs
+        else:
+            for a, b in zip(first, outs):
+                assert torch.equal(a, b)
+
+
+def test_host_buffer_variants_match_device_path():
+    x, w = synth.rmsnorm_inputs(5000, 4096, 101)       # > one 16 MiB chunk, ragged last chunk
+    y_dev = ak.ak_rmsnorm_fwd(x.to(DEV), w.to(DEV)).cpu()
+    xh, yh = x.pin_memory(), torch.empty_like(x).pin_memory()
+    ak.ak_rmsnorm_fwd_host(xh, w, yh)
+    assert torch.equal(yh.view(torch.int16), y_dev.view(torch.int16))
+    xs = synth.softmax_inputs(3000, 8192, 102)
+    y_dev = ak.ak_softmax_fwd(xs.to(DEV)).cpu()
+    yh = torch.empty_like(xs)
+    ak.ak_softmax_fwd_host(xs, yh)                     # pageable memory works too
+    assert torch.equal(yh.view(torch.int16), y_dev.view(torch.int16))
+    logits, targets = synth.xent_inputs(700, 32000, 103)
+    ref_rows, ref_mean, _ = oracle.xent(synth.to_bits(logits), targets.numpy())
+    loss_h = torch.empty(700, dtype=torch.float32)
+    mean_h = torch.empty(1, dtype=torch.float32)
+    ak.ak_xent_fwd_host(logits.pin_memory(), targets, loss_h, mean_h)
+    assert_loss_close(loss_h, ref_rows, "host xent rows")
+    assert_loss_close(mean_h, np.array([ref_mean]), "host xent mean")
+    ak.lib().ak_host_arena_release()
+
+
+def test_non_default_stream_and_launch_counter():
+    x, w = synth.rmsnorm_inputs(64, 2048, 104)
+    ref = oracle.rmsnorm(synth.to_bits(x), synth.to_bits(w), 1e-6)
+    s = torch.cuda.Stream()
+    xd, wd = x.to(DEV), w.to(DEV)
+    torch.cuda.synchronize()
+    before = ak.ak_launch_count()
+    with torch.cuda.stream(s):
+        y = ak.ak_rmsnorm_fwd(xd, wd)
+    s.synchronize()
+    assert ak.ak_launch_count() == before + 1
+    assert_bf16_close(y, ref, "non-default stream")
