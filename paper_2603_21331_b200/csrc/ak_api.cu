@@ -2,6 +2,7 @@
 // host-buffer variants (chunked copy-in / compute / copy-out pipeline).
 #include <atomic>
 #include <cmath>
+#include <cstdlib>
 #include <mutex>
 
 #include "ak_common.cuh"
@@ -10,6 +11,14 @@ namespace ak {
 
 static std::atomic<int64_t> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+bool persistent_grid() {
+    static const bool on = [] {
+        const char* v = std::getenv("AK_TUNE_PERSISTENT");
+        return v != nullptr && std::atoi(v) != 0;
+    }();
+    return on;
+}
 
 int sm_count() {
     static std::mutex mu;
@@ -35,21 +44,21 @@ int check_rows_cols(int64_t rows, int64_t D) {
 }
 
 int validate_rmsnorm(const void* x, const void* w, void* y, int64_t rows, int64_t D, float eps) {
-    if (!x || !w || !y) return AK_ERR_NULL;
+    if (rows != 0 && (!x || !w || !y)) return AK_ERR_NULL;  // an empty batch may carry NULL data pointers
     if (int s = check_rows_cols(rows, D)) return s;
     if (!is_aligned(x, 2) || !is_aligned(w, 2) || !is_aligned(y, 2)) return AK_ERR_ALIGN;
     if (!(eps >= 0.0f) || !std::isfinite(eps)) return AK_ERR_ARG;
     return AK_OK;
 }
 int validate_softmax(const void* x, void* y, int64_t rows, int64_t D) {
-    if (!x || !y) return AK_ERR_NULL;
+    if (rows != 0 && (!x || !y)) return AK_ERR_NULL;
     if (int s = check_rows_cols(rows, D)) return s;
     if (!is_aligned(x, 2) || !is_aligned(y, 2)) return AK_ERR_ALIGN;
     return AK_OK;
 }
 int validate_xent(const void* logits, const int64_t* targets, float* loss_rows, float* loss_mean,
                   int64_t rows, int64_t V) {
-    if (!logits || !targets || !loss_rows) return AK_ERR_NULL;
+    if (rows != 0 && (!logits || !targets || !loss_rows)) return AK_ERR_NULL;
     if (int s = check_rows_cols(rows, V)) return s;
     if (!is_aligned(logits, 2) || !is_aligned(targets, 8) || !is_aligned(loss_rows, 4) ||
         (loss_mean && !is_aligned(loss_mean, 4)))

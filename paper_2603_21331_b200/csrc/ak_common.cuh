@@ -99,6 +99,9 @@ __device__ __forceinline__ float cta_max(float v, float* slots, int phase) {
 // Launch bookkeeping shared by the translation units (defined in ak_api.cu).
 void count_launch(int n = 1);
 int sm_count();  // SMs of the current device (cached per device)
+// Tuning knob (environment AK_TUNE_PERSISTENT, read once; default 0): 1 = register-path CTAs
+// walk rows with a grid stride on a resident-size grid, 0 = one row (warp path: 4 rows) per CTA.
+bool persistent_grid();
 
 // Per-op host dispatchers (each defined next to its kernels).  All arguments have been
 // validated; `path` is a concrete path id or AUTO.  They return an ak_status.

@@ -175,7 +175,7 @@ template <int THREADS, int VPT>
 int launch_cta(const void* x, const void* w, void* y, int64_t rows, int nvec, float inv_D, float eps,
                cudaStream_t st) {
     static const int resident = resident_ctas(rmsnorm_cta_kernel<THREADS, VPT>, THREADS);
-    const int grid = (int)(rows < resident ? rows : resident);
+    const int grid = (int)(rows < resident || !persistent_grid() ? rows : resident);
     rmsnorm_cta_kernel<THREADS, VPT><<<grid, THREADS, 0, st>>>(
         static_cast<const uint4*>(x), static_cast<const uint4*>(w), static_cast<uint4*>(y),
         rows, nvec, inv_D, eps);
@@ -213,7 +213,7 @@ int launch_warp(const void* x, const void* w, void* y, int64_t rows, int nvec, f
     static const int resident =
         resident_ctas(rmsnorm_warp_kernel<kWarpsPerCta, VPT>, kWarpsPerCta * kWarp);
     const int64_t need = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
-    const int grid = (int)(need < resident ? need : resident);
+    const int grid = (int)(need < resident || !persistent_grid() ? need : resident);
     rmsnorm_warp_kernel<kWarpsPerCta, VPT><<<grid, kWarpsPerCta * kWarp, 0, st>>>(
         static_cast<const uint4*>(x), static_cast<const uint4*>(w), static_cast<uint4*>(y),
         rows, nvec, inv_D, eps);

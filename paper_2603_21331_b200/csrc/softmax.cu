@@ -173,7 +173,7 @@ int resident_ctas(K kernel, int threads) {
 template <int THREADS, int VPT>
 int launch_cta(const void* x, void* y, int64_t rows, int nvec, cudaStream_t st) {
     static const int resident = resident_ctas(softmax_cta_kernel<THREADS, VPT>, THREADS);
-    const int grid = (int)(rows < resident ? rows : resident);
+    const int grid = (int)(rows < resident || !persistent_grid() ? rows : resident);
     softmax_cta_kernel<THREADS, VPT><<<grid, THREADS, 0, st>>>(
         static_cast<const uint4*>(x), static_cast<uint4*>(y), rows, nvec);
     count_launch();
@@ -208,7 +208,7 @@ int launch_warp(const void* x, void* y, int64_t rows, int nvec, cudaStream_t st)
     static const int resident =
         resident_ctas(softmax_warp_kernel<kWarpsPerCta, VPT>, kWarpsPerCta * kWarp);
     const int64_t need = (rows + kWarpsPerCta - 1) / kWarpsPerCta;
-    const int grid = (int)(need < resident ? need : resident);
+    const int grid = (int)(need < resident || !persistent_grid() ? need : resident);
     softmax_warp_kernel<kWarpsPerCta, VPT><<<grid, kWarpsPerCta * kWarp, 0, st>>>(
         static_cast<const uint4*>(x), static_cast<uint4*>(y), rows, nvec);
     count_launch();

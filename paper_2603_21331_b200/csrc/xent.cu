@@ -108,7 +108,11 @@ __device__ __forceinline__ void row_slice_lse(const uint16_t* __restrict__ xr, i
 __device__ __forceinline__ float finish_loss(float M, float S, float xt) {
     const float MF = fmaxf(M * kLog2e, kFloor2);
     const float err = fmaf(M, kLog2e, -MF);
-    return (M - xt) + kLn2 * (log2f(S) - err);
+    // The exact value is >= 0 (the maximum contributes 1 to the sum); the SFU's 2^-22
+    // error can leave it a few 1e-8 below.  Clamp without swallowing a NaN.
+    float lse = kLn2 * (log2f(S) - err);
+    if (lse < 0.0f) lse = 0.0f;
+    return (M - xt) + lse;
 }
 
 // ------------------------------------------------------------------ one CTA per row
