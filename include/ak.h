@@ -55,7 +55,8 @@ enum {
     AK_PATH_AUTO = 0,
     AK_PATH_WARP = 1,     /* one warp per row, row held in registers; D % 8 == 0, D <= 2048, 16 B aligned */
     AK_PATH_CTA = 2,      /* one CTA per row, row held in registers;  D % 8 == 0, D <= 32768, 16 B aligned */
-    AK_PATH_GENERIC = 3   /* any D, any 2-byte alignment; row re-read from L1/L2, single DRAM pass */
+    AK_PATH_GENERIC = 3,  /* any D, any 2-byte alignment; row re-read from L1/L2, single DRAM pass */
+    AK_PATH_SMEM = 4      /* one CTA per row, row staged in shared memory by bulk (TMA) copies; D % 8 == 0, D <= 114688, 16 B aligned */
 };
 enum {
     AK_XENT_AUTO = 0,

@@ -2,7 +2,7 @@
 forward over bf16 [rows, D] tensors, exported from the C-ABI library ``libak.so``
 (``include/ak.h``) and bound here with ctypes.  No CPU or PyTorch fallback exists."""
 from .binding import (  # noqa: F401
-    AK_OK, AK_PATH_AUTO, AK_PATH_CTA, AK_PATH_GENERIC, AK_PATH_WARP,
+    AK_OK, AK_PATH_AUTO, AK_PATH_CTA, AK_PATH_GENERIC, AK_PATH_SMEM, AK_PATH_WARP,
     AK_XENT_AUTO, AK_XENT_ROW, AK_XENT_SPLIT, AkError, LIB_PATH,
     ak_launch_count, ak_rmsnorm_choose_path, ak_rmsnorm_fwd, ak_rmsnorm_fwd_host,
     ak_softmax_choose_path, ak_softmax_fwd, ak_softmax_fwd_host, ak_status_string, ak_version,

@@ -23,7 +23,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libak.so")
 
 AK_OK = 0
-AK_PATH_AUTO, AK_PATH_WARP, AK_PATH_CTA, AK_PATH_GENERIC = 0, 1, 2, 3
+AK_PATH_AUTO, AK_PATH_WARP, AK_PATH_CTA, AK_PATH_GENERIC, AK_PATH_SMEM = 0, 1, 2, 3, 4
 AK_XENT_AUTO, AK_XENT_ROW, AK_XENT_SPLIT = 0, 1, 2
 
 _i64, _f32, _int, _p, _sz = (ctypes.c_int64, ctypes.c_float, ctypes.c_int, ctypes.c_void_p,

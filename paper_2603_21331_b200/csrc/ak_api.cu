@@ -76,7 +76,7 @@ extern "C" {
 int ak_rmsnorm_fwd_path(const void* x, const void* w, void* y, int64_t rows, int64_t D, float eps,
                         void* cuda_stream, int path) {
     if (int s = validate_rmsnorm(x, w, y, rows, D, eps)) return s;
-    if (path < AK_PATH_AUTO || path > AK_PATH_GENERIC) return AK_ERR_ARG;
+    if (path < AK_PATH_AUTO || path > AK_PATH_SMEM) return AK_ERR_ARG;
     if (rows == 0) return AK_OK;
     return rmsnorm_dispatch(x, w, y, rows, D, eps, static_cast<cudaStream_t>(cuda_stream), path);
 }
@@ -87,7 +87,7 @@ int ak_rmsnorm_fwd(const void* x, const void* w, void* y, int64_t rows, int64_t 
 
 int ak_softmax_fwd_path(const void* x, void* y, int64_t rows, int64_t D, void* cuda_stream, int path) {
     if (int s = validate_softmax(x, y, rows, D)) return s;
-    if (path < AK_PATH_AUTO || path > AK_PATH_GENERIC) return AK_ERR_ARG;
+    if (path < AK_PATH_AUTO || path > AK_PATH_SMEM) return AK_ERR_ARG;
     if (rows == 0) return AK_OK;
     return softmax_dispatch(x, y, rows, D, static_cast<cudaStream_t>(cuda_stream), path);
 }

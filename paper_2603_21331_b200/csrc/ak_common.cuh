@@ -95,6 +95,46 @@ __device__ __forceinline__ float cta_max(float v, float* slots, int phase) {
     return warp_max(t);
 }
 
+// ---------------------------------------------------------------- bulk (TMA) copies into shared memory
+// One elected thread asks the copy engine for a whole contiguous span (a row); the bytes
+// land in shared memory without passing through registers and an mbarrier counts them in.
+// Source, destination and size must be multiples of 16 bytes.  No multicast is used.
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int arrivals) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_addr(smem_dst)),
+                 "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+// Set when a bounded wait gave up (never expected; a kernel that sees it returns early and
+// leaves its outputs unwritten rather than spinning).
+static __device__ int g_wait_timeout;
+// Bounded wait for the phase with the given parity.  Returns false after ~2^20 polls.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    for (int it = 0; it < (1 << 20); ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+            : "=r"(ok)
+            : "r"(smem_addr(bar)), "r"(parity)
+            : "memory");
+        if (ok) return true;
+    }
+    atomicExch(&g_wait_timeout, 1);
+    return false;
+}
+
+// Largest row (bytes) the shared-memory-staged kernels accept: 224 KiB of dynamic shared
+// memory out of the 227 KiB a CTA may own (a few hundred bytes stay static).
+constexpr int kMaxRowSmemBytes = 224 * 1024;
+
 // ---------------------------------------------------------------- host-side plumbing
 // Launch bookkeeping shared by the translation units (defined in ak_api.cu).
 void count_launch(int n = 1);

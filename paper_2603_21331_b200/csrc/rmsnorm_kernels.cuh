@@ -1,0 +1,195 @@
+// RMSNorm forward device kernels (paper Table 3 "rmsnorm": warp-shuffle reduction + fast
+// rsqrt, weight multiply fused into the epilogue per Section 7.3 Tier 3).
+//
+//   y[r, j] = bf16_rne( x[r, j] * rsqrt(mean_k x[r, k]^2 + eps) * w[j] )
+//
+// One DRAM read and one DRAM write per element, fp32 accumulation, fixed-order reductions.
+#pragma once
+
+#include "ak_common.cuh"
+
+namespace ak {
+
+__device__ __forceinline__ float sumsq8(const uint4& v) {
+    float a0 = bf16lo(v.x), a1 = bf16hi(v.x), a2 = bf16lo(v.y), a3 = bf16hi(v.y);
+    float a4 = bf16lo(v.z), a5 = bf16hi(v.z), a6 = bf16lo(v.w), a7 = bf16hi(v.w);
+    float s0 = a0 * a0, s1 = a1 * a1;
+    s0 = fmaf(a2, a2, s0); s1 = fmaf(a3, a3, s1);
+    s0 = fmaf(a4, a4, s0); s1 = fmaf(a5, a5, s1);
+    s0 = fmaf(a6, a6, s0); s1 = fmaf(a7, a7, s1);
+    return s0 + s1;
+}
+
+__device__ __forceinline__ uint32_t scale2(uint32_t x, uint32_t w, float rstd) {
+    return pack_bf16x2(bf16lo(x) * rstd * bf16lo(w), bf16hi(x) * rstd * bf16hi(w));
+}
+__device__ __forceinline__ uint4 scale8(const uint4& x, const uint4& w, float rstd) {
+    return make_uint4(scale2(x.x, w.x, rstd), scale2(x.y, w.y, rstd),
+                      scale2(x.z, w.z, rstd), scale2(x.w, w.w, rstd));
+}
+
+// ------------------------------------------------------------------ row in registers
+// A CTA of THREADS threads is cut into THREADS / GROUP groups; one group owns one row and
+// each of its threads holds VPT 16-byte vectors of it as packed bf16 (vector i of the row
+// lives in thread i % GROUP, slot i / GROUP, so every load instruction is a contiguous
+// GROUP * 16-byte segment).  GROUP == 32 is the warp-per-row layout (no barrier at all),
+// GROUP == THREADS the CTA-per-row layout.  All of a thread's loads are issued before the
+// first use.  The weight vectors are fetched through L1 (they are shared by every row)
+// either before the reduction (W_EARLY: latency hidden behind the row loads, 4 * VPT more
+// live registers) or after it.  MINB is the launch-bounds occupancy hint that caps the
+// register count.  The grid may be smaller than the number of row slots: groups then walk
+// the rows with a grid stride.
+template <int THREADS, int GROUP, int VPT, int MINB, bool W_EARLY>
+__global__ void __launch_bounds__(THREADS, MINB)
+rmsnorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w, uint4* __restrict__ y,
+                   int64_t rows, int nvec, float inv_D, float eps) {
+    constexpr int GROUPS = THREADS / GROUP;
+    constexpr int WARPS_PER_GROUP = GROUP / kWarp;
+    static_assert(GROUP % kWarp == 0 && THREADS % GROUP == 0, "groups are whole warps");
+    __shared__ float slots[2][THREADS / kWarp];
+    const int g = threadIdx.x / GROUP;
+    const int t = threadIdx.x % GROUP;
+    const int lane = threadIdx.x & 31;
+    const int warp_in_group = t >> 5;
+
+    uint4 wv[VPT];
+    if constexpr (W_EARLY) {
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            const int i = t + k * GROUP;
+            wv[k] = (i < nvec) ? __ldg(w + i) : make_uint4(0, 0, 0, 0);
+        }
+    }
+    int phase = 0;
+    // Whole CTAs iterate together (rows beyond the end are masked, not skipped) so the
+    // barrier below is reached by every thread.
+    for (int64_t row0 = (int64_t)blockIdx.x * GROUPS; row0 < rows; row0 += (int64_t)gridDim.x * GROUPS) {
+        const int64_t row = row0 + g;
+        const bool live = row < rows;
+        const uint4* xr = x + row * nvec;
+        uint4 xv[VPT];
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            const int i = t + k * GROUP;
+            xv[k] = (live && i < nvec) ? ld_stream(xr + i) : make_uint4(0, 0, 0, 0);
+        }
+        float ss = 0.0f;
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) ss += sumsq8(xv[k]);
+        ss = warp_sum(ss);
+        if constexpr (WARPS_PER_GROUP > 1) {
+            float* s = slots[phase] + g * WARPS_PER_GROUP;
+            if (lane == 0) s[warp_in_group] = ss;
+            __syncthreads();
+            float v = (lane < WARPS_PER_GROUP) ? s[lane] : 0.0f;
+            ss = warp_sum(v);
+            phase ^= 1;
+        }
+        const float rstd = rsqrtf(fmaf(ss, inv_D, eps));
+        uint4* yr = y + row * nvec;
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            const int i = t + k * GROUP;
+            if (live && i < nvec) {
+                const uint4 wq = W_EARLY ? wv[k] : __ldg(w + i);
+                st_stream(yr + i, scale8(xv[k], wq, rstd));
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------ long rows staged in shared memory
+// One CTA per row.  One thread asks the copy engine for the whole row (bulk copies of at
+// most kBulkChunk bytes, all counted in by one mbarrier), so the bytes in flight per SM
+// are bounded by shared memory (resident CTAs x row bytes), not by registers.  The row is
+// then read twice from shared memory: sum of squares, then scale and store.  Needs
+// 16-byte aligned rows (D % 8 == 0).  Dynamic shared memory = nvec * 16 bytes.
+constexpr uint32_t kBulkChunk = 32768;
+
+template <int THREADS, int MINB>
+__global__ void __launch_bounds__(THREADS, MINB)
+rmsnorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w, uint4* __restrict__ y,
+                    int nvec, float inv_D, float eps) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    uint4* row = reinterpret_cast<uint4*>(smem_raw);
+    __shared__ uint64_t bar;
+    __shared__ float slots[2 * kWarp];
+    const int64_t r = blockIdx.x;
+    if (threadIdx.x == 0) mbar_init(&bar, 1);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const uint32_t bytes = (uint32_t)nvec * 16u;
+        mbar_expect_tx(&bar, bytes);
+        const unsigned char* src = reinterpret_cast<const unsigned char*>(x + r * nvec);
+        for (uint32_t off = 0; off < bytes; off += kBulkChunk)
+            bulk_load(smem_raw + off, src + off, min(kBulkChunk, bytes - off), &bar);
+    }
+    if (!mbar_wait(&bar, 0)) return;  // uniform: every thread waits on the same barrier
+    float ss = 0.0f;
+#pragma unroll 4
+    for (int i = threadIdx.x; i < nvec; i += THREADS) ss += sumsq8(row[i]);
+    ss = cta_sum<THREADS>(ss, slots, 0);
+    const float rstd = rsqrtf(fmaf(ss, inv_D, eps));
+    uint4* yr = y + r * nvec;
+#pragma unroll 4
+    for (int i = threadIdx.x; i < nvec; i += THREADS) st_stream(yr + i, scale8(row[i], __ldg(w + i), rstd));
+}
+
+// ------------------------------------------------------------------ generic
+// Any D and any 2-byte alignment.  Row r starts at element r*D, so its 16-byte phase
+// changes from row to row: up to 7 head elements and 7 tail elements are handled with
+// 2-byte accesses, the body with 16-byte vectors (when x and y share the phase).  The
+// second pass re-reads the row, which this CTA has just pulled through L1/L2.
+constexpr int kRmsGenericThreads = 256;
+
+__global__ void __launch_bounds__(kRmsGenericThreads)
+rmsnorm_generic_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w,
+                       uint16_t* __restrict__ y, int64_t rows, int64_t D, float inv_D, float eps) {
+    constexpr int T = kRmsGenericThreads;
+    __shared__ float slots[2 * kWarp];
+    int phase = 0;
+    for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+        const uint16_t* xr = x + row * D;
+        uint16_t* yr = y + row * D;
+        const int xph = (int)((reinterpret_cast<uintptr_t>(xr) >> 1) & 7);
+        const int yph = (int)((reinterpret_cast<uintptr_t>(yr) >> 1) & 7);
+        const bool vec_ok = (xph == yph);
+        int64_t head = vec_ok ? ((8 - xph) & 7) : D;
+        if (head > D) head = D;
+        const int64_t nbody = (D - head) >> 3;
+        const int64_t tail0 = head + (nbody << 3);
+        const uint4* xb = reinterpret_cast<const uint4*>(xr + head);
+
+        float ss = 0.0f;
+        for (int64_t i = threadIdx.x; i < nbody; i += T) ss += sumsq8(xb[i]);
+        for (int64_t j = threadIdx.x; j < head; j += T) {
+            const float v = bf16_to_float(xr[j]);
+            ss = fmaf(v, v, ss);
+        }
+        for (int64_t j = tail0 + threadIdx.x; j < D; j += T) {
+            const float v = bf16_to_float(xr[j]);
+            ss = fmaf(v, v, ss);
+        }
+        ss = cta_sum<T>(ss, slots, phase);
+        phase ^= 1;
+        const float rstd = rsqrtf(fmaf(ss, inv_D, eps));
+
+        uint4* yb = reinterpret_cast<uint4*>(yr + head);
+        for (int64_t i = threadIdx.x; i < nbody; i += T) {
+            const uint4 v = xb[i];
+            const uint16_t* wj = w + head + (i << 3);
+            uint4 wq;
+            wq.x = (uint32_t)__ldg(wj + 0) | ((uint32_t)__ldg(wj + 1) << 16);
+            wq.y = (uint32_t)__ldg(wj + 2) | ((uint32_t)__ldg(wj + 3) << 16);
+            wq.z = (uint32_t)__ldg(wj + 4) | ((uint32_t)__ldg(wj + 5) << 16);
+            wq.w = (uint32_t)__ldg(wj + 6) | ((uint32_t)__ldg(wj + 7) << 16);
+            st_stream(yb + i, scale8(v, wq, rstd));
+        }
+        for (int64_t j = threadIdx.x; j < head; j += T)
+            yr[j] = float_to_bf16(bf16_to_float(xr[j]) * rstd * bf16_to_float(__ldg(w + j)));
+        for (int64_t j = tail0 + threadIdx.x; j < D; j += T)
+            yr[j] = float_to_bf16(bf16_to_float(xr[j]) * rstd * bf16_to_float(__ldg(w + j)));
+    }
+}
+
+}  // namespace ak

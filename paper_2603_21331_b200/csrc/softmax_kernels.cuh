@@ -1,0 +1,209 @@
+// Last-dim softmax forward device kernels (paper Table 3 "softmax": warp-shuffle
+// reductions, packed 16-bit loads).
+//
+//   m = max_k x[r, k];  y[r, j] = bf16_rne( exp(x[r, j] - m) / sum_k exp(x[r, k] - m) )
+//
+// exp is evaluated as 2^(x*log2e - rn(m*log2e)) with one FMA feeding the SFU.  Rounding
+// m*log2e once scales every term of the row by the same factor, which cancels in the
+// ratio.  -inf entries give 2^(-inf) = 0 exactly; an all -inf row, +inf or NaN gives NaN
+// through inf - inf, as IEEE arithmetic on the definition would.
+#pragma once
+
+#include "ak_common.cuh"
+
+namespace ak {
+
+constexpr uint32_t kNegInf2 = 0xFF80FF80u;  // two bf16 -inf
+
+__device__ __forceinline__ uint32_t max8(const uint4& v) {
+    return bf16x2_max(bf16x2_max(v.x, v.y), bf16x2_max(v.z, v.w));
+}
+__device__ __forceinline__ float hmax_of(uint32_t m2) { return fmaxf(bf16lo(m2), bf16hi(m2)); }
+
+// e[0..7] = 2^(x*log2e - m2); returns their sum (fixed association).
+__device__ __forceinline__ float exp8(const uint4& v, float m2, float* e) {
+    e[0] = fast_exp2(fmaf(bf16lo(v.x), kLog2e, -m2));
+    e[1] = fast_exp2(fmaf(bf16hi(v.x), kLog2e, -m2));
+    e[2] = fast_exp2(fmaf(bf16lo(v.y), kLog2e, -m2));
+    e[3] = fast_exp2(fmaf(bf16hi(v.y), kLog2e, -m2));
+    e[4] = fast_exp2(fmaf(bf16lo(v.z), kLog2e, -m2));
+    e[5] = fast_exp2(fmaf(bf16hi(v.z), kLog2e, -m2));
+    e[6] = fast_exp2(fmaf(bf16lo(v.w), kLog2e, -m2));
+    e[7] = fast_exp2(fmaf(bf16hi(v.w), kLog2e, -m2));
+    return ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
+}
+__device__ __forceinline__ uint4 norm8(const float* e, float inv) {
+    return make_uint4(pack_bf16x2(e[0] * inv, e[1] * inv), pack_bf16x2(e[2] * inv, e[3] * inv),
+                      pack_bf16x2(e[4] * inv, e[5] * inv), pack_bf16x2(e[6] * inv, e[7] * inv));
+}
+
+// ------------------------------------------------------------------ row in registers
+// Same thread layout as the RMSNorm register kernel: a group of GROUP threads owns a row,
+// thread t holds vectors t, t + GROUP, ...  Two reductions per row (max, then sum).
+// RECOMPUTE == false keeps the eight exponentials of every vector in fp32 registers so
+// each is evaluated once; RECOMPUTE == true keeps only the packed inputs and evaluates the
+// exponentials a second time in the epilogue (half the registers, twice the SFU work) for
+// rows too long to hold in fp32.
+template <int THREADS, int GROUP, int VPT, int MINB, bool RECOMPUTE>
+__global__ void __launch_bounds__(THREADS, MINB)
+softmax_reg_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t rows, int nvec) {
+    constexpr int GROUPS = THREADS / GROUP;
+    constexpr int WARPS_PER_GROUP = GROUP / kWarp;
+    static_assert(GROUP % kWarp == 0 && THREADS % GROUP == 0, "groups are whole warps");
+    __shared__ float slots[2][THREADS / kWarp];
+    const int g = threadIdx.x / GROUP;
+    const int t = threadIdx.x % GROUP;
+    const int lane = threadIdx.x & 31;
+    const int warp_in_group = t >> 5;
+
+    for (int64_t row0 = (int64_t)blockIdx.x * GROUPS; row0 < rows; row0 += (int64_t)gridDim.x * GROUPS) {
+        const int64_t row = row0 + g;
+        const bool live = row < rows;
+        const uint4* xr = x + row * nvec;
+        uint4 xv[VPT];
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            const int i = t + k * GROUP;
+            xv[k] = (live && i < nvec) ? ld_stream(xr + i) : make_uint4(kNegInf2, kNegInf2, kNegInf2, kNegInf2);
+        }
+        uint32_t mx = kNegInf2;
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) mx = bf16x2_max(mx, max8(xv[k]));
+        float m = warp_max(hmax_of(mx));
+        if constexpr (WARPS_PER_GROUP > 1) {
+            float* s = slots[0] + g * WARPS_PER_GROUP;
+            if (lane == 0) s[warp_in_group] = m;
+            __syncthreads();
+            m = warp_max((lane < WARPS_PER_GROUP) ? s[lane] : -INFINITY);
+        }
+        const float m2 = m * kLog2e;
+        float e[RECOMPUTE ? 1 : VPT][8];
+        float sum = 0.0f;
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) sum += exp8(xv[k], m2, e[RECOMPUTE ? 0 : k]);
+        sum = warp_sum(sum);
+        if constexpr (WARPS_PER_GROUP > 1) {
+            float* s = slots[1] + g * WARPS_PER_GROUP;
+            if (lane == 0) s[warp_in_group] = sum;
+            __syncthreads();
+            sum = warp_sum((lane < WARPS_PER_GROUP) ? s[lane] : 0.0f);
+        }
+        const float inv = 1.0f / sum;
+        uint4* yr = y + row * nvec;
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            const int i = t + k * GROUP;
+            if constexpr (RECOMPUTE) exp8(xv[k], m2, e[0]);
+            if (live && i < nvec) st_stream(yr + i, norm8(e[RECOMPUTE ? 0 : k], inv));
+        }
+    }
+}
+
+// ------------------------------------------------------------------ long rows staged in shared memory
+// One CTA per row; the row is brought into shared memory by bulk copies counted in by one
+// mbarrier (bytes in flight bounded by shared memory, not registers), then read three
+// times from there: maximum, sum of exponentials, normalise + store.  The first KEEP
+// vectors of every thread keep their exponentials in fp32 registers between the second and
+// third pass; the rest are evaluated twice.  Needs 16-byte aligned rows (D % 8 == 0).
+// Dynamic shared memory = nvec * 16 bytes.
+constexpr uint32_t kSmBulkChunk = 32768;
+
+template <int THREADS, int MINB, int KEEP>
+__global__ void __launch_bounds__(THREADS, MINB)
+softmax_smem_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int nvec) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const uint4* row = reinterpret_cast<const uint4*>(smem_raw);
+    __shared__ uint64_t bar;
+    __shared__ float slots[2 * kWarp];
+    const int64_t r = blockIdx.x;
+    if (threadIdx.x == 0) mbar_init(&bar, 1);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const uint32_t bytes = (uint32_t)nvec * 16u;
+        mbar_expect_tx(&bar, bytes);
+        const unsigned char* src = reinterpret_cast<const unsigned char*>(x + r * nvec);
+        for (uint32_t off = 0; off < bytes; off += kSmBulkChunk)
+            bulk_load(smem_raw + off, src + off, min(kSmBulkChunk, bytes - off), &bar);
+    }
+    if (!mbar_wait(&bar, 0)) return;  // uniform: every thread waits on the same barrier
+
+    uint32_t mx = kNegInf2;
+#pragma unroll 4
+    for (int i = threadIdx.x; i < nvec; i += THREADS) mx = bf16x2_max(mx, max8(row[i]));
+    const float m = cta_max<THREADS>(hmax_of(mx), slots, 0);
+    const float m2 = m * kLog2e;
+
+    float kept[KEEP > 0 ? KEEP : 1][8];
+    float sum = 0.0f, e[8];
+#pragma unroll
+    for (int k = 0; k < KEEP; ++k) {
+        const int i = threadIdx.x + k * THREADS;
+        if (i < nvec) sum += exp8(row[i], m2, kept[k]);
+    }
+#pragma unroll 2
+    for (int i = threadIdx.x + KEEP * THREADS; i < nvec; i += THREADS) sum += exp8(row[i], m2, e);
+    sum = cta_sum<THREADS>(sum, slots, 1);
+    const float inv = 1.0f / sum;
+
+    uint4* yr = y + r * nvec;
+#pragma unroll
+    for (int k = 0; k < KEEP; ++k) {
+        const int i = threadIdx.x + k * THREADS;
+        if (i < nvec) st_stream(yr + i, norm8(kept[k], inv));
+    }
+#pragma unroll 2
+    for (int i = threadIdx.x + KEEP * THREADS; i < nvec; i += THREADS) {
+        exp8(row[i], m2, e);
+        st_stream(yr + i, norm8(e, inv));
+    }
+}
+
+// ------------------------------------------------------------------ generic
+// Any D / alignment: three passes over the row (max, sum, write); only the first comes
+// from DRAM, the other two are served by L1/L2.
+constexpr int kSmGenericThreads = 256;
+
+__global__ void __launch_bounds__(kSmGenericThreads)
+softmax_generic_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, int64_t rows, int64_t D) {
+    constexpr int T = kSmGenericThreads;
+    __shared__ float slots[2 * kWarp];
+    for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+        const uint16_t* xr = x + row * D;
+        uint16_t* yr = y + row * D;
+        const int xph = (int)((reinterpret_cast<uintptr_t>(xr) >> 1) & 7);
+        const int yph = (int)((reinterpret_cast<uintptr_t>(yr) >> 1) & 7);
+        const bool vec_ok = (xph == yph);
+        int64_t head = vec_ok ? ((8 - xph) & 7) : D;
+        if (head > D) head = D;
+        const int64_t nbody = (D - head) >> 3;
+        const int64_t tail0 = head + (nbody << 3);
+        const uint4* xb = reinterpret_cast<const uint4*>(xr + head);
+
+        uint32_t mx = kNegInf2;
+        for (int64_t i = threadIdx.x; i < nbody; i += T) mx = bf16x2_max(mx, max8(xb[i]));
+        float m = hmax_of(mx);
+        for (int64_t j = threadIdx.x; j < head; j += T) m = fmaxf(m, bf16_to_float(xr[j]));
+        for (int64_t j = tail0 + threadIdx.x; j < D; j += T) m = fmaxf(m, bf16_to_float(xr[j]));
+        m = cta_max<T>(m, slots, 0);
+        const float m2 = m * kLog2e;
+
+        float s = 0.0f, e[8];
+        for (int64_t i = threadIdx.x; i < nbody; i += T) s += exp8(xb[i], m2, e);
+        for (int64_t j = threadIdx.x; j < head; j += T) s += fast_exp2(fmaf(bf16_to_float(xr[j]), kLog2e, -m2));
+        for (int64_t j = tail0 + threadIdx.x; j < D; j += T) s += fast_exp2(fmaf(bf16_to_float(xr[j]), kLog2e, -m2));
+        s = cta_sum<T>(s, slots, 1);
+        const float inv = 1.0f / s;
+
+        uint4* yb = reinterpret_cast<uint4*>(yr + head);
+        for (int64_t i = threadIdx.x; i < nbody; i += T) {
+            exp8(xb[i], m2, e);
+            st_stream(yb + i, norm8(e, inv));
+        }
+        for (int64_t j = threadIdx.x; j < head; j += T)
+            yr[j] = float_to_bf16(fast_exp2(fmaf(bf16_to_float(xr[j]), kLog2e, -m2)) * inv);
+        for (int64_t j = tail0 + threadIdx.x; j < D; j += T)
+            yr[j] = float_to_bf16(fast_exp2(fmaf(bf16_to_float(xr[j]), kLog2e, -m2)) * inv);
+    }
+}
+
+}  // namespace ak

@@ -1,0 +1,342 @@
+// Fused cross-entropy forward device kernels (paper Table 3 "cross_ent": online log-sum-exp
+// fused with the NLL gather; a single pass over the logits).
+//
+//   loss[r] = (m - x[r, t]) + log( sum_k exp(x[r, k] - m) ),  m = max_k x[r, k]
+//
+// Each thread streams 16-byte vectors of its row (or of its slice of the row) and keeps an
+// online pair: the running maximum m (always a bf16 value) and s = sum 2^(x*log2e - mf)
+// with mf = rn(m*log2e).  Rescaling by 2^(mf_old - mf_new) happens once per batch of
+// vectors, only when the maximum moved.  Working in the rounded log2 domain is exact up to
+// one per-row constant: x*log2e - m*log2e = (x*log2e - mf) - err with
+// err = fma(m, log2e, -mf) (the rounding error of a product is representable), so
+//   log sum exp(x - m) = ln2 * (log2(s) - err).
+// The loss is assembled as (m - x_t) + that term: both parts are >= 0, and no large
+// magnitude is ever added to a small one.
+//
+// The kernel is co-bound by HBM and by the SFU: one exponential per two bytes keeps the
+// transcendental pipe ~78 % busy at 5.8 TB/s.  POLY of every 8 exponentials are therefore
+// evaluated on the FMA pipe instead (round-to-nearest range reduction + degree-4 minimax
+// polynomial, relative error 2.7e-6, the split is fixed per element so results stay
+// deterministic), and the multiply-adds and the summation use the packed f32x2 forms to
+// halve the instruction count.
+#pragma once
+
+#include "ak_common.cuh"
+
+namespace ak {
+
+constexpr uint32_t kXNegInf2 = 0xFF80FF80u;
+constexpr float kFloor2 = -1.0e30f;  // finite stand-in for "no maximum yet" in the log2 domain
+constexpr int kXentThreads = 256;
+
+// NaN-propagating packed max: a NaN logit must surface as a NaN loss.
+__device__ __forceinline__ uint32_t bf16x2_max_nan(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+__device__ __forceinline__ uint32_t xmax8(const uint4& v) {
+    return bf16x2_max_nan(bf16x2_max_nan(v.x, v.y), bf16x2_max_nan(v.z, v.w));
+}
+__device__ __forceinline__ float xhmax_of(uint32_t m2) {
+    const float a = bf16lo(m2), b = bf16hi(m2);
+    return (a != a || b != b) ? __int_as_float(0x7fc00000) : fmaxf(a, b);
+}
+
+// ---------------------------------------------------------------- packed f32x2 arithmetic
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// the two bf16 of a 32-bit word as a packed float pair (element 2i low, 2i+1 high)
+__device__ __forceinline__ f32x2 widen2(uint32_t u) { return pack2(bf16lo(u), bf16hi(u)); }
+
+// 2^t for a pair, t <= ~0, on the FMA pipe.  t is clamped at -125 (2^-125 stands in for
+// anything smaller, including 2^-inf: negligible against a sum that is >= 1), rounded to
+// the nearest integer n with the 1.5 * 2^23 trick, and 2^(t - n) comes from a degree-4
+// minimax polynomial on [-0.5, 0.5]; n is added to the exponent field.
+__device__ __forceinline__ f32x2 poly_exp2_pair(f32x2 t2) {
+    float t0, t1;
+    unpack2(t2, t0, t1);
+    const f32x2 tc = pack2(fmaxf(t0, -125.0f), fmaxf(t1, -125.0f));
+    const f32x2 magic = pack2(12582912.0f, 12582912.0f);
+    const f32x2 z = add2(tc, magic);
+    const f32x2 n = sub2(z, magic);
+    const f32x2 f = sub2(tc, n);
+    f32x2 p = pack2(0.009570079855620861f, 0.009570079855620861f);
+    p = fma2(p, f, pack2(0.05591783672571182f, 0.05591783672571182f));
+    p = fma2(p, f, pack2(0.240247443318367f, 0.240247443318367f));
+    p = fma2(p, f, pack2(0.6931217908859253f, 0.6931217908859253f));
+    p = fma2(p, f, pack2(0.9999992847442627f, 0.9999992847442627f));
+    float p0, p1, z0, z1;
+    unpack2(p, p0, p1);
+    unpack2(z, z0, z1);
+    p0 = __int_as_float(__float_as_int(p0) + (__float_as_int(z0) << 23));
+    p1 = __int_as_float(__float_as_int(p1) + (__float_as_int(z1) << 23));
+    return pack2(p0, p1);
+}
+__device__ __forceinline__ f32x2 sfu_exp2_pair(f32x2 t2) {
+    float t0, t1;
+    unpack2(t2, t0, t1);
+    return pack2(fast_exp2(t0), fast_exp2(t1));
+}
+
+// sum over the 8 elements of one vector of 2^(x*log2e - mf), as a packed pair of partial
+// sums.  The first POLY / 2 of the four pairs take the polynomial, the rest the SFU.
+template <int POLY>
+__device__ __forceinline__ f32x2 sumexp8(const uint4& v, f32x2 l2, f32x2 nmf2) {
+    static_assert(POLY % 2 == 0 && POLY >= 0 && POLY <= 8, "pairs");
+    const f32x2 t0 = fma2(widen2(v.x), l2, nmf2);
+    const f32x2 t1 = fma2(widen2(v.y), l2, nmf2);
+    const f32x2 t2 = fma2(widen2(v.z), l2, nmf2);
+    const f32x2 t3 = fma2(widen2(v.w), l2, nmf2);
+    const f32x2 e0 = (POLY >= 2) ? poly_exp2_pair(t0) : sfu_exp2_pair(t0);
+    const f32x2 e1 = (POLY >= 4) ? poly_exp2_pair(t1) : sfu_exp2_pair(t1);
+    const f32x2 e2 = (POLY >= 6) ? poly_exp2_pair(t2) : sfu_exp2_pair(t2);
+    const f32x2 e3 = (POLY >= 8) ? poly_exp2_pair(t3) : sfu_exp2_pair(t3);
+    return add2(add2(e0, e1), add2(e2, e3));
+}
+
+struct Online {
+    float m;    // running maximum (bf16-valued; -inf when nothing finite seen; NaN sticks)
+    float mf;   // max(rn(m * log2e), kFloor2)
+    f32x2 s2;   // two partial sums of 2^(x*log2e - mf)
+};
+
+__device__ __forceinline__ void raise_max(Online& o, float vm) {
+    const float vmf = fmaxf(vm * kLog2e, kFloor2);
+    if (vmf > o.mf) {
+        const float r = fast_exp2(o.mf - vmf);
+        o.s2 = fma2(o.s2, pack2(r, r), pack2(0.0f, 0.0f));
+        o.mf = vmf;
+    }
+    o.m = (vm != vm) ? vm : fmaxf(o.m, vm);  // NaN sticks (fmaxf alone would drop it)
+}
+__device__ __forceinline__ void absorb_scalar(Online& o, float v) {
+    raise_max(o, v);
+    o.s2 = add2(o.s2, pack2(fast_exp2(fmaf(v, kLog2e, -o.mf)), 0.0f));
+}
+
+// CTA-wide online (m, s) over elements [begin, end) of one row.  Returns, in every
+// thread, the maximum M and the sum S relative to MF = max(rn(M*log2e), kFloor2).
+// Uses both slot sets (max then sum).  UNROLL vectors are in flight per thread.
+template <int UNROLL, int POLY>
+__device__ __forceinline__ void row_slice_lse(const uint16_t* __restrict__ xr, int64_t begin, int64_t end,
+                                              float* slots, float& M, float& S) {
+    constexpr int T = kXentThreads;
+    Online o{-INFINITY, kFloor2, pack2(0.0f, 0.0f)};
+    const uint16_t* p = xr + begin;
+    const int64_t n = end - begin;
+    int64_t head = (8 - (int)((reinterpret_cast<uintptr_t>(p) >> 1) & 7)) & 7;
+    if (head > n) head = n;
+    const int64_t nbody = (n - head) >> 3;
+    const int64_t tail0 = head + (nbody << 3);
+    const uint4* body = reinterpret_cast<const uint4*>(p + head);
+    const f32x2 l2 = pack2(kLog2e, kLog2e);
+
+    for (int64_t base = 0; base < nbody; base += (int64_t)T * UNROLL) {
+        uint4 q[UNROLL];
+#pragma unroll
+        for (int k = 0; k < UNROLL; ++k) {
+            const int64_t i = base + threadIdx.x + (int64_t)k * T;
+            q[k] = (i < nbody) ? ld_stream(body + i) : make_uint4(kXNegInf2, kXNegInf2, kXNegInf2, kXNegInf2);
+        }
+        uint32_t mx = xmax8(q[0]);
+#pragma unroll
+        for (int k = 1; k < UNROLL; ++k) mx = bf16x2_max_nan(mx, xmax8(q[k]));
+        raise_max(o, xhmax_of(mx));
+        const f32x2 nmf2 = pack2(-o.mf, -o.mf);
+        f32x2 acc = sumexp8<POLY>(q[0], l2, nmf2);
+#pragma unroll
+        for (int k = 1; k < UNROLL; ++k) acc = add2(acc, sumexp8<POLY>(q[k], l2, nmf2));
+        o.s2 = add2(o.s2, acc);
+    }
+    if ((int64_t)threadIdx.x < head) absorb_scalar(o, bf16_to_float(ld_stream_u16(p + threadIdx.x)));
+    if (tail0 + threadIdx.x < n) absorb_scalar(o, bf16_to_float(ld_stream_u16(p + tail0 + threadIdx.x)));
+
+    // NaN must win the max: fmaxf in cta_max would drop it, so it travels as +inf plus a flag
+    const bool has_nan = (o.m != o.m) || (o.m == INFINITY);  // +inf makes inf - inf: NaN row as well
+    M = cta_max<T>(has_nan ? INFINITY : o.m, slots, 0);
+    const float MF = fmaxf(M * kLog2e, kFloor2);
+    float s0, s1;
+    unpack2(o.s2, s0, s1);
+    float s = (s0 + s1) * fast_exp2(o.mf - MF);
+    if (has_nan) s = __int_as_float(0x7fc00000);
+    S = cta_sum<T>(s, slots, 1);
+}
+
+// loss from the row's (M, S) and the target logit.
+__device__ __forceinline__ float finish_loss(float M, float S, float xt) {
+    const float MF = fmaxf(M * kLog2e, kFloor2);
+    const float err = fmaf(M, kLog2e, -MF);
+    // The exact value is >= 0 (the maximum contributes 1 to the sum); approximation error
+    // can leave it a few 1e-7 below.  Clamp without swallowing a NaN.
+    float lse = kLn2 * (log2f(S) - err);
+    if (lse < 0.0f) lse = 0.0f;
+    return (M - xt) + lse;
+}
+
+// Programmatic dependent launch: let the next kernel in the stream be scheduled while this
+// grid is still running (it waits for our completion with pdl_wait before it reads).
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// ------------------------------------------------------------------ one CTA per row
+template <int UNROLL, int POLY, int MINB = 1>
+__global__ void __launch_bounds__(kXentThreads, MINB)
+xent_row_kernel(const uint16_t* __restrict__ logits, const int64_t* __restrict__ targets,
+                int64_t ignore_index, float* __restrict__ loss_rows, int64_t V) {
+    __shared__ float slots[2 * kWarp];
+    pdl_launch_dependents();
+    const int64_t row = blockIdx.x;
+    const int64_t t = targets[row];
+    if (t == ignore_index || t < 0 || t >= V) {  // uniform across the CTA: nothing is read
+        if (threadIdx.x == 0) loss_rows[row] = (t == ignore_index) ? 0.0f : __int_as_float(0x7fc00000);
+        return;
+    }
+    const uint16_t* xr = logits + row * V;
+    // the target logit is fetched now, under the row's own traffic, not after the reduction
+    const float xt = (threadIdx.x == 0) ? bf16_to_float(xr[t]) : 0.0f;
+    float M, S;
+    row_slice_lse<UNROLL, POLY>(xr, 0, V, slots, M, S);
+    if (threadIdx.x == 0) loss_rows[row] = finish_loss(M, S, xt);
+}
+
+// ------------------------------------------------------------------ split row, phase 1
+// grid = (nsplit, rows).  Slice boundaries are multiples of 8 elements so an aligned row
+// keeps aligned slices.  partial[row * nsplit + split] = (M, S) of the slice.
+template <int UNROLL, int POLY>
+__global__ void __launch_bounds__(kXentThreads)
+xent_split_kernel(const uint16_t* __restrict__ logits, const int64_t* __restrict__ targets,
+                  int64_t ignore_index, float2* __restrict__ partial, int64_t V, int nsplit) {
+    __shared__ float slots[2 * kWarp];
+    pdl_launch_dependents();
+    const int64_t row = blockIdx.y;
+    const int sp = blockIdx.x;
+    const int64_t t = targets[row];
+    if (t == ignore_index || t < 0 || t >= V) return;
+    const int64_t groups = (V + 7) >> 3;
+    int64_t begin = ((groups * sp) / nsplit) << 3;
+    int64_t end = ((groups * (sp + 1)) / nsplit) << 3;
+    if (end > V) end = V;
+    float M, S;
+    row_slice_lse<UNROLL, POLY>(logits + row * V, begin, end, slots, M, S);
+    if (threadIdx.x == 0) partial[row * nsplit + sp] = make_float2(M, S);
+}
+
+// ------------------------------------------------------------------ finish: merge + mean
+// One CTA, launched as a programmatic dependent of the streaming kernel.  Thread i owns
+// rows i, i + T, i + 2T, ...: for the split layout it first merges the row's partials in
+// split order and writes the loss; then (if out_mean / out_pair is given) it adds its
+// rows' counted losses in fp64 in that order, and a fixed shuffle + shared-memory tree
+// adds the threads.  out_mean = sum / count (0/0 = NaN); out_pair = {sum, count}.
+constexpr int kFinishThreads = 1024;
+
+__device__ __forceinline__ double warp_sum_f64(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__global__ void __launch_bounds__(kFinishThreads)
+xent_finish_kernel(const uint16_t* __restrict__ logits, const int64_t* __restrict__ targets,
+                   int64_t ignore_index, const float2* __restrict__ partial, int nsplit,
+                   float* __restrict__ loss_rows, int64_t rows, int64_t V,
+                   float* __restrict__ out_mean, double* __restrict__ out_pair) {
+    constexpr int T = kFinishThreads;
+    __shared__ double ssum[T / kWarp];
+    __shared__ double scnt[T / kWarp];
+    pdl_wait();  // everything the streaming kernel wrote is visible from here on
+    if (nsplit > 0) {
+        for (int64_t r = threadIdx.x; r < rows; r += T) {
+            const int64_t t = targets[r];
+            float loss;
+            if (t == ignore_index) {
+                loss = 0.0f;
+            } else if (t < 0 || t >= V) {
+                loss = __int_as_float(0x7fc00000);
+            } else {
+                const float2* pr = partial + r * nsplit;
+                float M = -INFINITY;
+                for (int i = 0; i < nsplit; ++i) M = fmaxf(M, __ldcg(pr + i).x);
+                const float MF = fmaxf(M * kLog2e, kFloor2);
+                float S = 0.0f;
+                for (int i = 0; i < nsplit; ++i) {
+                    const float2 ps = __ldcg(pr + i);
+                    S += ps.y * fast_exp2(fmaxf(ps.x * kLog2e, kFloor2) - MF);
+                }
+                loss = finish_loss(M, S, bf16_to_float(logits[r * V + t]));
+            }
+            loss_rows[r] = loss;
+        }
+    }
+    if (out_mean == nullptr && out_pair == nullptr) return;
+    // Mean: batches of independent loads (a lone CTA is latency-bound, so sixteen rows are in
+    // flight per thread), added in row order per thread.  A thread re-reads only rows it
+    // wrote itself above, so program order makes them visible.
+    constexpr int B = 16;
+    double acc = 0.0, cnt = 0.0;
+    for (int64_t base = threadIdx.x; base < rows; base += (int64_t)T * B) {
+        int64_t tt[B];
+        float ll[B];
+#pragma unroll
+        for (int k = 0; k < B; ++k) {
+            const int64_t r = base + (int64_t)k * T;
+            tt[k] = (r < rows) ? targets[r] : ignore_index;
+            ll[k] = (r < rows) ? __ldcg(loss_rows + r) : 0.0f;  // L2 read: written by the grid we depend on
+        }
+#pragma unroll
+        for (int k = 0; k < B; ++k) {
+            if (tt[k] != ignore_index) {
+                acc += (double)ll[k];
+                cnt += 1.0;
+            }
+        }
+    }
+    acc = warp_sum_f64(acc);
+    cnt = warp_sum_f64(cnt);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) { ssum[warp] = acc; scnt[warp] = cnt; }
+    __syncthreads();
+    if (warp == 0) {
+        acc = warp_sum_f64(ssum[lane]);
+        cnt = warp_sum_f64(scnt[lane]);
+        if (lane == 0) {
+            if (out_mean) out_mean[0] = (cnt > 0.0) ? (float)(acc / cnt) : __int_as_float(0x7fc00000);
+            if (out_pair) { out_pair[0] = acc; out_pair[1] = cnt; }
+        }
+    }
+}
+
+// Mean over row shards: pairs[i] = {sum_i, count_i}; added in index order by one thread.
+__global__ void xent_mean_merge_kernel(const double* __restrict__ pairs, int64_t n, float* __restrict__ out_mean) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    double total = 0.0, count = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        total += pairs[2 * i];
+        count += pairs[2 * i + 1];
+    }
+    out_mean[0] = (count > 0.0) ? (float)(total / count) : __int_as_float(0x7fc00000);
+}
+
+}  // namespace ak

@@ -78,12 +78,15 @@ def test_validation_rejects_before_any_cuda_call():
 def test_dispatch_is_a_pure_function_of_shape_and_alignment():
     assert ak.ak_rmsnorm_choose_path(8192, 1024, True) == ak.AK_PATH_WARP
     assert ak.ak_rmsnorm_choose_path(8192, 4096, True) == ak.AK_PATH_CTA
-    assert ak.ak_rmsnorm_choose_path(8192, 32768, True) == ak.AK_PATH_CTA
+    assert ak.ak_rmsnorm_choose_path(8192, 16384, True) == ak.AK_PATH_CTA
+    assert ak.ak_rmsnorm_choose_path(8192, 32768, True) == ak.AK_PATH_SMEM
     assert ak.ak_rmsnorm_choose_path(8192, 4099, True) == ak.AK_PATH_GENERIC
     assert ak.ak_rmsnorm_choose_path(8192, 4096, False) == ak.AK_PATH_GENERIC
-    assert ak.ak_rmsnorm_choose_path(8192, 65536, True) == ak.AK_PATH_GENERIC
+    assert ak.ak_rmsnorm_choose_path(8192, 65536, True) == ak.AK_PATH_SMEM
+    assert ak.ak_rmsnorm_choose_path(8192, 131072, True) == ak.AK_PATH_GENERIC
     assert ak.ak_softmax_choose_path(16384, 512, True) == ak.AK_PATH_WARP
-    assert ak.ak_softmax_choose_path(16384, 32768, True) == ak.AK_PATH_CTA
+    assert ak.ak_softmax_choose_path(16384, 8192, True) == ak.AK_PATH_CTA
+    assert ak.ak_softmax_choose_path(16384, 32768, True) == ak.AK_PATH_SMEM
     assert ak.ak_softmax_choose_path(16384, 128257, True) == ak.AK_PATH_GENERIC
     for rows, V in ((4096, 32000), (4096, 128256), (16384, 128256)):
         assert ak.ak_xent_choose_path(rows, V) == (ak.AK_XENT_ROW, 1)

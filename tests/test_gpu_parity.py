@@ -11,11 +11,13 @@ from parity import assert_bf16_close, assert_loss_close, guarded
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
-WARP, CTA, GEN = ak.AK_PATH_WARP, ak.AK_PATH_CTA, ak.AK_PATH_GENERIC
+WARP, CTA, GEN, SMEM = ak.AK_PATH_WARP, ak.AK_PATH_CTA, ak.AK_PATH_GENERIC, ak.AK_PATH_SMEM
 
 
 def _legal_paths(D):
     paths = [GEN]
+    if D % 8 == 0 and D * 2 <= 224 * 1024:
+        paths.append(SMEM)
     if D % 8 == 0 and D <= 32768:
         paths.append(CTA)
     if D % 8 == 0 and D <= 2048:
@@ -29,7 +31,7 @@ def _legal_paths(D):
 SHAPES = [(256, 1024), (1, 8), (3, 16), (37, 64), (129, 256), (65, 512), (33, 776), (40, 1000),
           (33, 1280), (19, 1536), (21, 1792), (64, 2048), (17, 4096), (1, 4096), (23, 3072),
           (9, 5120), (16, 8192), (7, 11008), (12, 16384), (5, 20480), (3, 24576), (3, 28672),
-          (6, 32768), (5, 1), (4, 7), (31, 1023), (11, 1537), (9, 4097), (13, 4099), (2, 40000),
+          (6, 32768), (3, 65536), (2, 114688), (5, 1), (4, 7), (31, 1023), (11, 1537), (9, 4097), (13, 4099), (2, 40000),
           (3, 128257)]
 
 
@@ -148,7 +150,7 @@ def test_softmax_ieee_conventions():
     x[2, 5] = float("nan")            # NaN -> NaN row
     x[3, :] = torch.arange(24) * 0.25  # ordinary row
     ref = oracle.softmax(synth.to_bits(x))
-    for path in (WARP, CTA, GEN):
+    for path in (WARP, CTA, GEN, SMEM):
         y = ak.ak_softmax_fwd(x.to(DEV), path=path)
         torch.cuda.synchronize()
         assert_bf16_close(y, ref, f"softmax conventions path {path}")
@@ -232,7 +234,7 @@ def test_misaligned_base_pointers_take_generic_path():
 
 
 def test_in_place_is_allowed():
-    for D, paths in ((512, (WARP, CTA, GEN)), (4096, (CTA, GEN)), (4099, (GEN,))):
+    for D, paths in ((512, (WARP, CTA, GEN, SMEM)), (4096, (CTA, GEN, SMEM)), (4099, (GEN,)), (16384, (CTA, SMEM))):
         x, w = synth.rmsnorm_inputs(11, D, 94)
         ref = oracle.rmsnorm(synth.to_bits(x), synth.to_bits(w), 1e-6)
         xs = synth.softmax_inputs(11, D, 95)
