@@ -46,7 +46,8 @@ typedef enum {
     AK_ERR_ALIGN = 3,  /* pointer not aligned to its element type (or to 16 B where a forced path needs it) */
     AK_ERR_ARG = 4,    /* eps negative or not finite; unknown path id; bad nsplit */
     AK_ERR_CUDA = 5,   /* a CUDA runtime call or launch failed */
-    AK_ERR_NOMEM = 6   /* scratch allocation failed or caller workspace too small */
+    AK_ERR_NOMEM = 6,  /* scratch allocation failed or caller workspace too small */
+    AK_ERR_CAPACITY = 7 /* problem larger than the fixed scratch of ak_xent_fwd_static */
 } ak_status;
 
 /* Path ids for the *_path entry points (testing / tuning).  0 always means "let the
@@ -122,6 +123,31 @@ int ak_xent_fwd_ws(const void* logits, const int64_t* targets, int64_t ignore_in
 int ak_xent_fwd_path(const void* logits, const int64_t* targets, int64_t ignore_index,
                      float* loss_rows, float* loss_mean,
                      int64_t rows, int64_t V, void* cuda_stream, int path, int nsplit);
+
+/* ---------------------------------------------------------------------------------
+ * Cross-entropy forward that never allocates.  (The paper has no counterpart: this entry
+ * point exists for the library's users, not for parity with anything the paper describes.)
+ *
+ * For callers that cannot obtain device memory at call time - a process whose whole memory
+ * budget went to its own arena at start-up, a job under a hard GPU quota, a latency-critical
+ * loop that must stay out of the allocator.  Same arguments, outputs and conventions as
+ * ak_xent_fwd, computed with the split-row layout (the split count the dispatcher would pick
+ * for (rows, V)), but the per-slice scratch lives in a fixed 1 MiB array inside the library's
+ * device image: every GPU that loads the library holds that 1 MiB until the process exits, and
+ * the call performs no cudaMalloc, cudaFree or other allocating routine.
+ *   - Limit: rows <= 65535 and rows * nsplit * 8 bytes <= 1 MiB (131072 slices), otherwise
+ *     AK_ERR_CAPACITY is returned and nothing is launched.  (4096 rows of any vocabulary, or
+ *     2048 rows split 64 ways, fit.)
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress,
+ *     with that device current) and caches it; make that first call before any stream capture.
+ *   - All calls on a device share the array and inherit its previous contents.  Nothing needs
+ *     clearing (every slot read is written earlier in the same call), but calls whose kernels
+ *     overlap on the GPU (different streams) race on it: serialise them, or give each its own
+ *     buffer through ak_xent_fwd_ws.
+ */
+int ak_xent_fwd_static(const void* logits, const int64_t* targets, int64_t ignore_index,
+                       float* loss_rows, float* loss_mean,
+                       int64_t rows, int64_t V, void* cuda_stream);
 
 /* ---------------------------------------------------------------------------------
  * Row-sharded cross-entropy (one process per GPU, each holding a block of rows).  Per-row

@@ -6,5 +6,6 @@ from .binding import (  # noqa: F401
     AK_XENT_AUTO, AK_XENT_ROW, AK_XENT_SPLIT, AkError, LIB_PATH,
     ak_launch_count, ak_rmsnorm_choose_path, ak_rmsnorm_fwd, ak_rmsnorm_fwd_host,
     ak_softmax_choose_path, ak_softmax_fwd, ak_softmax_fwd_host, ak_status_string, ak_version,
-    ak_xent_choose_path, ak_xent_fwd, ak_xent_fwd_host, ak_xent_fwd_ws, ak_xent_workspace_bytes, lib,
+    ak_xent_choose_path, ak_xent_fwd, ak_xent_fwd_host, ak_xent_fwd_static, ak_xent_fwd_ws,
+    ak_xent_workspace_bytes, lib,
 )

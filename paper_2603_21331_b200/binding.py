@@ -39,6 +39,7 @@ SIGNATURES = {
     "ak_xent_workspace_bytes": (_sz, [_i64, _i64]),
     "ak_xent_fwd_ws": (_int, [_p, _p, _i64, _p, _p, _i64, _i64, _p, _sz, _p]),
     "ak_xent_fwd_path": (_int, [_p, _p, _i64, _p, _p, _i64, _i64, _p, _int, _int]),
+    "ak_xent_fwd_static": (_int, [_p, _p, _i64, _p, _p, _i64, _i64, _p]),
     "ak_xent_sum_count": (_int, [_p, _p, _i64, _i64, _p, _p]),
     "ak_xent_mean_merge": (_int, [_p, _i64, _p, _p]),
     "ak_rmsnorm_fwd_host": (_int, [_p, _p, _p, _i64, _i64, _f32]),
@@ -156,6 +157,30 @@ def ak_xent_fwd(logits: torch.Tensor, targets: torch.Tensor, ignore_index: int =
     _check(lib().ak_xent_fwd_path(logits.data_ptr(), targets.data_ptr(), ignore_index,
                                   loss_rows.data_ptr(), mean_ptr, rows, V, _stream_ptr(stream),
                                   path, nsplit), "ak_xent_fwd")
+    return loss_rows, loss_mean
+
+
+def ak_xent_fwd_static(logits: torch.Tensor, targets: torch.Tensor, ignore_index: int = -100,
+                       loss_rows: Optional[torch.Tensor] = None,
+                       loss_mean: Optional[torch.Tensor] = None, stream=None):
+    """Cross-entropy forward for callers that may not allocate device memory at call time
+    (pre-sized arenas, hard GPU quotas, allocator-free hot loops): the library's own fixed
+    1 MiB scratch is used, nothing is allocated by the call itself.  Pass ``loss_rows`` and
+    ``loss_mean`` to keep this wrapper from creating them.  Raises AkError with status 7 when
+    rows * nsplit * 8 bytes exceeds 1 MiB or rows > 65535.  Calls that overlap on the GPU
+    share the scratch and race; the first call on a device should precede any stream capture."""
+    _dev_bf16(logits, "logits", 2)
+    rows, V = logits.shape
+    if not (targets.is_cuda and targets.dtype == torch.int64 and targets.shape == (rows,)
+            and targets.is_contiguous()):
+        raise TypeError("targets must be a contiguous CUDA int64 tensor [rows]")
+    if loss_rows is None:
+        loss_rows = torch.empty((rows,), dtype=torch.float32, device=logits.device)
+    if loss_mean is None:
+        loss_mean = torch.empty((1,), dtype=torch.float32, device=logits.device)
+    _check(lib().ak_xent_fwd_static(logits.data_ptr(), targets.data_ptr(), ignore_index,
+                                    loss_rows.data_ptr(), loss_mean.data_ptr(), rows, V,
+                                    _stream_ptr(stream)), "ak_xent_fwd_static")
     return loss_rows, loss_mean
 
 

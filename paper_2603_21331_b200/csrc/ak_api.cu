@@ -165,6 +165,7 @@ const char* ak_status_string(int status) {
         case AK_ERR_ARG: return "bad scalar argument (eps, path id or nsplit)";
         case AK_ERR_CUDA: return "CUDA runtime error";
         case AK_ERR_NOMEM: return "scratch memory unavailable or workspace too small";
+        case AK_ERR_CAPACITY: return "problem exceeds the fixed scratch of the no-allocation entry point (rows * nsplit * 8 bytes > 1 MiB or rows > 65535)";
         default: return "unknown status";
     }
 }

@@ -258,7 +258,7 @@ __device__ __forceinline__ double warp_sum_f64(double v) {
     return v;
 }
 
-__global__ void __launch_bounds__(kFinishThreads)
+static __global__ void __launch_bounds__(kFinishThreads)
 xent_finish_kernel(const uint16_t* __restrict__ logits, const int64_t* __restrict__ targets,
                    int64_t ignore_index, const float2* __restrict__ partial, int nsplit,
                    float* __restrict__ loss_rows, int64_t rows, int64_t V,
@@ -329,7 +329,7 @@ xent_finish_kernel(const uint16_t* __restrict__ logits, const int64_t* __restric
 }
 
 // Mean over row shards: pairs[i] = {sum_i, count_i}; added in index order by one thread.
-__global__ void xent_mean_merge_kernel(const double* __restrict__ pairs, int64_t n, float* __restrict__ out_mean) {
+static __global__ void xent_mean_merge_kernel(const double* __restrict__ pairs, int64_t n, float* __restrict__ out_mean) {
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
     double total = 0.0, count = 0.0;
     for (int64_t i = 0; i < n; ++i) {
