@@ -180,6 +180,18 @@ int ak_xent_fwd_host(const void* logits_host, const int64_t* targets_host, int64
 int ak_host_arena_release(void);
 
 /* ---------------------------------------------------------------------------------
+ * Speed-of-light measurement aids (no op arithmetic): a streaming device-to-device copy and
+ * a streaming read, built from the same 16-byte streaming accesses and small one-shot CTAs
+ * as the row kernels, so the benchmark can report each op against the bandwidth this GPU
+ * actually delivers for 1:1 read/write traffic (RMSNorm, softmax; the paper's GB/s accounting
+ * for Table 4) and for read-only traffic (cross-entropy).  src / dst: device pointers,
+ * 16-byte aligned, `bytes` a multiple of 16; sink4: 4 writable device bytes (left untouched
+ * for ordinary data).
+ */
+int ak_sol_copy(const void* src, void* dst, size_t bytes, void* cuda_stream);
+int ak_sol_read(const void* src, size_t bytes, void* sink4, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------
  * Introspection.
  */
 /* Path id the dispatcher picks for (rows, D) with fully aligned pointers (`aligned16` != 0)

@@ -46,6 +46,8 @@ SIGNATURES = {
     "ak_softmax_fwd_host": (_int, [_p, _p, _i64, _i64]),
     "ak_xent_fwd_host": (_int, [_p, _p, _i64, _p, _p, _i64, _i64]),
     "ak_host_arena_release": (_int, []),
+    "ak_sol_copy": (_int, [_p, _p, _sz, _p]),
+    "ak_sol_read": (_int, [_p, _sz, _p, _p]),
     "ak_rmsnorm_choose_path": (_int, [_i64, _i64, _int]),
     "ak_softmax_choose_path": (_int, [_i64, _i64, _int]),
     "ak_xent_choose_path": (_int, [_i64, _i64, ctypes.POINTER(_int)]),

@@ -36,6 +36,41 @@ __device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b) {
     return r;
 }
 
+// ---------------------------------------------------------------- packed f32x2 arithmetic
+// sm_100 executes two fp32 operations per instruction on register pairs: half the issue
+// slots (and the energy that goes with them) for the conversions' consumers.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// the two bf16 of a 32-bit word as a packed float pair (element 2i low, 2i+1 high)
+__device__ __forceinline__ f32x2 widen2(uint32_t u) { return pack2(bf16lo(u), bf16hi(u)); }
+
 // ---------------------------------------------------------------- memory
 // Activations are touched exactly once: streaming (evict-first) loads and stores keep
 // them from displacing the reusable weight vector in L2/L1.
@@ -112,6 +147,9 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, 
                      smem_addr(smem_dst)),
                  "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar))
                  : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
 }
 // Set when a bounded wait gave up (never expected; a kernel that sees it returns early and
 // leaves its outputs unwritten rather than spinning).

@@ -10,22 +10,29 @@
 
 namespace ak {
 
+// Packed f32x2 arithmetic throughout: even elements accumulate in the low lane, odd ones in
+// the high lane (fixed association), one instruction per pair.
 __device__ __forceinline__ float sumsq8(const uint4& v) {
-    float a0 = bf16lo(v.x), a1 = bf16hi(v.x), a2 = bf16lo(v.y), a3 = bf16hi(v.y);
-    float a4 = bf16lo(v.z), a5 = bf16hi(v.z), a6 = bf16lo(v.w), a7 = bf16hi(v.w);
-    float s0 = a0 * a0, s1 = a1 * a1;
-    s0 = fmaf(a2, a2, s0); s1 = fmaf(a3, a3, s1);
-    s0 = fmaf(a4, a4, s0); s1 = fmaf(a5, a5, s1);
-    s0 = fmaf(a6, a6, s0); s1 = fmaf(a7, a7, s1);
-    return s0 + s1;
+    const f32x2 a = widen2(v.x), b = widen2(v.y), c = widen2(v.z), d = widen2(v.w);
+    f32x2 s = mul2(a, a);
+    s = fma2(b, b, s);
+    s = fma2(c, c, s);
+    s = fma2(d, d, s);
+    float lo, hi;
+    unpack2(s, lo, hi);
+    return lo + hi;
 }
 
-__device__ __forceinline__ uint32_t scale2(uint32_t x, uint32_t w, float rstd) {
-    return pack_bf16x2(bf16lo(x) * rstd * bf16lo(w), bf16hi(x) * rstd * bf16hi(w));
+// (x * rstd) * w per element, one rounding to bf16
+__device__ __forceinline__ uint32_t scale2(uint32_t x, uint32_t w, f32x2 rstd2) {
+    const f32x2 p = mul2(mul2(widen2(x), rstd2), widen2(w));
+    float lo, hi;
+    unpack2(p, lo, hi);
+    return pack_bf16x2(lo, hi);
 }
 __device__ __forceinline__ uint4 scale8(const uint4& x, const uint4& w, float rstd) {
-    return make_uint4(scale2(x.x, w.x, rstd), scale2(x.y, w.y, rstd),
-                      scale2(x.z, w.z, rstd), scale2(x.w, w.w, rstd));
+    const f32x2 r2 = pack2(rstd, rstd);
+    return make_uint4(scale2(x.x, w.x, r2), scale2(x.y, w.y, r2), scale2(x.z, w.z, r2), scale2(x.w, w.w, r2));
 }
 
 // ------------------------------------------------------------------ row in registers

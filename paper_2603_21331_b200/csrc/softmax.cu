@@ -85,13 +85,17 @@ int softmax_dispatch(const void* x, void* y, int64_t rows, int64_t D, cudaStream
             return launch_reg_vpt<128, 32, 1, 1>((nvec + 31) / 32, x, y, rows, nvec, st);
         case AK_PATH_CTA:
             if (D > 32768) return AK_ERR_SHAPE;
-            if (nvec <= 512) return launch_reg_vpt<128, 128, 1, 1>((nvec + 127) / 128, x, y, rows, nvec, st);
-            if (nvec <= 1024) return launch_reg_vpt<256, 256, 5, 1>((nvec + 255) / 256, x, y, rows, nvec, st);
+            // 128 threads with up to 8 vectors each (exponentials of the whole share in fp32
+            // registers, capped at 102 registers for five CTAs per SM): the best sustained shape
+            // up to D = 8192
+            if (nvec <= 1024) return launch_reg_vpt<128, 128, 1, 5>((nvec + 127) / 128, x, y, rows, nvec, st);
             if (nvec <= 2048) return launch_reg_vpt<256, 256, 1, 1>((nvec + 255) / 256, x, y, rows, nvec, st);
             return launch_reg_vpt<512, 512, 1, 1>((nvec + 511) / 512, x, y, rows, nvec, st);
         case AK_PATH_SMEM:
             if (D * 2 > kMaxRowSmemBytes) return AK_ERR_SHAPE;
-            if (nvec <= 2048) return launch_smem<256, 4>(x, y, rows, nvec, st);
+            // 256 threads keeping the first four vectors' exponentials in registers: best both in
+            // short bursts and under the power cap of a long run up to D = 32768
+            if (nvec <= 4096) return launch_smem<256, 4>(x, y, rows, nvec, st);
             return launch_smem<512, 0>(x, y, rows, nvec, st);
         case AK_PATH_GENERIC: {
             static const int resident = [] {

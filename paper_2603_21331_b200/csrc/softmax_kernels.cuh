@@ -20,21 +20,32 @@ __device__ __forceinline__ uint32_t max8(const uint4& v) {
 }
 __device__ __forceinline__ float hmax_of(uint32_t m2) { return fmaxf(bf16lo(m2), bf16hi(m2)); }
 
-// e[0..7] = 2^(x*log2e - m2); returns their sum (fixed association).
-__device__ __forceinline__ float exp8(const uint4& v, float m2, float* e) {
-    e[0] = fast_exp2(fmaf(bf16lo(v.x), kLog2e, -m2));
-    e[1] = fast_exp2(fmaf(bf16hi(v.x), kLog2e, -m2));
-    e[2] = fast_exp2(fmaf(bf16lo(v.y), kLog2e, -m2));
-    e[3] = fast_exp2(fmaf(bf16hi(v.y), kLog2e, -m2));
-    e[4] = fast_exp2(fmaf(bf16lo(v.z), kLog2e, -m2));
-    e[5] = fast_exp2(fmaf(bf16hi(v.z), kLog2e, -m2));
-    e[6] = fast_exp2(fmaf(bf16lo(v.w), kLog2e, -m2));
-    e[7] = fast_exp2(fmaf(bf16hi(v.w), kLog2e, -m2));
-    return ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
+// e[0..3] = the eight values 2^(x*log2e - m2) of one vector as four packed pairs; returns
+// their sum (fixed association: even elements in the low lane, odd in the high lane).
+// Multiply-adds, sums and the final scaling run as packed f32x2 instructions.
+__device__ __forceinline__ f32x2 exp_pair(uint32_t u, f32x2 l2, f32x2 nm2) {
+    float t0, t1;
+    unpack2(fma2(widen2(u), l2, nm2), t0, t1);
+    return pack2(fast_exp2(t0), fast_exp2(t1));
 }
-__device__ __forceinline__ uint4 norm8(const float* e, float inv) {
-    return make_uint4(pack_bf16x2(e[0] * inv, e[1] * inv), pack_bf16x2(e[2] * inv, e[3] * inv),
-                      pack_bf16x2(e[4] * inv, e[5] * inv), pack_bf16x2(e[6] * inv, e[7] * inv));
+__device__ __forceinline__ float exp8(const uint4& v, float m2, f32x2* e) {
+    const f32x2 l2 = pack2(kLog2e, kLog2e), nm2 = pack2(-m2, -m2);
+    e[0] = exp_pair(v.x, l2, nm2);
+    e[1] = exp_pair(v.y, l2, nm2);
+    e[2] = exp_pair(v.z, l2, nm2);
+    e[3] = exp_pair(v.w, l2, nm2);
+    float lo, hi;
+    unpack2(add2(add2(e[0], e[1]), add2(e[2], e[3])), lo, hi);
+    return lo + hi;
+}
+__device__ __forceinline__ uint32_t norm2(f32x2 e, f32x2 inv2) {
+    float lo, hi;
+    unpack2(mul2(e, inv2), lo, hi);
+    return pack_bf16x2(lo, hi);
+}
+__device__ __forceinline__ uint4 norm8(const f32x2* e, float inv) {
+    const f32x2 inv2 = pack2(inv, inv);
+    return make_uint4(norm2(e[0], inv2), norm2(e[1], inv2), norm2(e[2], inv2), norm2(e[3], inv2));
 }
 
 // ------------------------------------------------------------------ row in registers
@@ -77,7 +88,7 @@ softmax_reg_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t r
             m = warp_max((lane < WARPS_PER_GROUP) ? s[lane] : -INFINITY);
         }
         const float m2 = m * kLog2e;
-        float e[RECOMPUTE ? 1 : VPT][8];
+        f32x2 e[RECOMPUTE ? 1 : VPT][4];
         float sum = 0.0f;
 #pragma unroll
         for (int k = 0; k < VPT; ++k) sum += exp8(xv[k], m2, e[RECOMPUTE ? 0 : k]);
@@ -133,8 +144,9 @@ softmax_smem_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int nvec
     const float m = cta_max<THREADS>(hmax_of(mx), slots, 0);
     const float m2 = m * kLog2e;
 
-    float kept[KEEP > 0 ? KEEP : 1][8];
-    float sum = 0.0f, e[8];
+    f32x2 kept[KEEP > 0 ? KEEP : 1][4];
+    float sum = 0.0f;
+    f32x2 e[4];
 #pragma unroll
     for (int k = 0; k < KEEP; ++k) {
         const int i = threadIdx.x + k * THREADS;
@@ -187,7 +199,8 @@ softmax_generic_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y,
         m = cta_max<T>(m, slots, 0);
         const float m2 = m * kLog2e;
 
-        float s = 0.0f, e[8];
+        float s = 0.0f;
+        f32x2 e[4];
         for (int64_t i = threadIdx.x; i < nbody; i += T) s += exp8(xb[i], m2, e);
         for (int64_t j = threadIdx.x; j < head; j += T) s += fast_exp2(fmaf(bf16_to_float(xr[j]), kLog2e, -m2));
         for (int64_t j = tail0 + threadIdx.x; j < D; j += T) s += fast_exp2(fmaf(bf16_to_float(xr[j]), kLog2e, -m2));

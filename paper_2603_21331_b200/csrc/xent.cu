@@ -15,9 +15,15 @@ namespace {
 // vectors in flight per thread, exponentials per 8 evaluated on the FMA pipe
 constexpr int kUnroll = 4;
 constexpr int kPoly = 2;
-// occupancy hint: six 256-thread CTAs per SM caps the kernel at 40 registers (without it
-// the compiler spends 60+ registers on scheduling freedom and halves the CTAs in flight)
-constexpr int kMinCtas = 6;
+// Row layout: 128-thread CTAs with eight vectors in flight per thread; the occupancy hint of
+// eight CTAs per SM caps the kernel at 64 registers.  (Without a hint the compiler spends
+// registers on scheduling freedom and halves the CTAs in flight.)  Measured against 256
+// threads x 4 vectors, 64 x 8, 512 x 4 and a persistent bulk-copy ring fed by one producer
+// lane: this shape was the fastest or tied on every benchmark vocabulary; the ring lost
+// 5-8 % because the arithmetic, not the loads, needs the resident warps.
+constexpr int kRowThreads = 128;
+constexpr int kRowUnroll = 8;
+constexpr int kRowMinCtas = 8;
 
 int launch_finish(const uint16_t* logits, const int64_t* targets, int64_t ignore_index, const float2* partial,
                   int nsplit, float* loss_rows, int64_t rows, int64_t V, float* out_mean, double* out_pair,
@@ -83,7 +89,8 @@ int xent_dispatch(const void* logits, const int64_t* targets, int64_t ignore_ind
         return launch_finish(lg, targets, ignore_index, nullptr, 0, loss_rows, 0, V, loss_mean, nullptr, st, false);
     }
     if (path == AK_XENT_ROW) {
-        xent_row_kernel<kUnroll, kPoly, kMinCtas><<<(unsigned)rows, kXentThreads, 0, st>>>(lg, targets, ignore_index, loss_rows, V);
+        xent_row_kernel<kRowUnroll, kPoly, kRowMinCtas, kRowThreads><<<(unsigned)rows, kRowThreads, 0, st>>>(
+            lg, targets, ignore_index, loss_rows, V);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return AK_ERR_CUDA;
         if (loss_mean == nullptr) return AK_OK;

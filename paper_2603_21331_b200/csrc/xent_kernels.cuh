@@ -43,34 +43,6 @@ __device__ __forceinline__ float xhmax_of(uint32_t m2) {
     return (a != a || b != b) ? __int_as_float(0x7fc00000) : fmaxf(a, b);
 }
 
-// ---------------------------------------------------------------- packed f32x2 arithmetic
-typedef unsigned long long f32x2;
-__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
-    f32x2 r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack2(f32x2 v, float& lo, float& hi) {
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
-    f32x2 d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
-    f32x2 d;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
-    f32x2 d;
-    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-// the two bf16 of a 32-bit word as a packed float pair (element 2i low, 2i+1 high)
-__device__ __forceinline__ f32x2 widen2(uint32_t u) { return pack2(bf16lo(u), bf16hi(u)); }
-
 // 2^t for a pair, t <= ~0, on the FMA pipe.  t is clamped at -125 (2^-125 stands in for
 // anything smaller, including 2^-inf: negligible against a sum that is >= 1), rounded to
 // the nearest integer n with the 1.5 * 2^23 trick, and 2^(t - n) comes from a degree-4
@@ -140,10 +112,9 @@ __device__ __forceinline__ void absorb_scalar(Online& o, float v) {
 // CTA-wide online (m, s) over elements [begin, end) of one row.  Returns, in every
 // thread, the maximum M and the sum S relative to MF = max(rn(M*log2e), kFloor2).
 // Uses both slot sets (max then sum).  UNROLL vectors are in flight per thread.
-template <int UNROLL, int POLY>
+template <int UNROLL, int POLY, int T = kXentThreads>
 __device__ __forceinline__ void row_slice_lse(const uint16_t* __restrict__ xr, int64_t begin, int64_t end,
                                               float* slots, float& M, float& S) {
-    constexpr int T = kXentThreads;
     Online o{-INFINITY, kFloor2, pack2(0.0f, 0.0f)};
     const uint16_t* p = xr + begin;
     const int64_t n = end - begin;
@@ -202,8 +173,8 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // ------------------------------------------------------------------ one CTA per row
-template <int UNROLL, int POLY, int MINB = 1>
-__global__ void __launch_bounds__(kXentThreads, MINB)
+template <int UNROLL, int POLY, int MINB = 1, int T = kXentThreads>
+__global__ void __launch_bounds__(T, MINB)
 xent_row_kernel(const uint16_t* __restrict__ logits, const int64_t* __restrict__ targets,
                 int64_t ignore_index, float* __restrict__ loss_rows, int64_t V) {
     __shared__ float slots[2 * kWarp];
@@ -218,7 +189,7 @@ xent_row_kernel(const uint16_t* __restrict__ logits, const int64_t* __restrict__
     // the target logit is fetched now, under the row's own traffic, not after the reduction
     const float xt = (threadIdx.x == 0) ? bf16_to_float(xr[t]) : 0.0f;
     float M, S;
-    row_slice_lse<UNROLL, POLY>(xr, 0, V, slots, M, S);
+    row_slice_lse<UNROLL, POLY, T>(xr, 0, V, slots, M, S);
     if (threadIdx.x == 0) loss_rows[row] = finish_loss(M, S, xt);
 }
 
