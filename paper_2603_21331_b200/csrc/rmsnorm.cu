@@ -95,10 +95,10 @@ int rmsnorm_dispatch(const void* x, const void* w, void* y, int64_t rows, int64_
         case AK_PATH_CTA:
             if (D > 32768) return AK_ERR_SHAPE;
             // Shapes chosen in the sustained (power-capped) regime of a long run: 128 threads x <= 4
-            // vectors capped at 64 registers; 256 threads x <= 4 vectors capped at 51 registers
-            // (five CTAs per SM, no spill); 256 threads x <= 8 vectors capped at 85.
-            if (nvec <= 512) return launch_reg_vpt<128, 128, 8, 1>((nvec + 127) / 128, x, w, y, rows, nvec, inv_D, eps, st);
-            if (nvec <= 2048) return launch_reg_vpt<256, 256, 5, 3>((nvec + 255) / 256, x, w, y, rows, nvec, inv_D, eps, st);
+            // vectors (46 registers); 256 threads x <= 4 vectors (46 registers, five CTAs per SM);
+            // 256 threads x <= 8 vectors capped at 85 registers (62 used).
+            if (nvec <= 512) return launch_reg_vpt<128, 128, 1, 1>((nvec + 127) / 128, x, w, y, rows, nvec, inv_D, eps, st);
+            if (nvec <= 2048) return launch_reg_vpt<256, 256, 1, 3>((nvec + 255) / 256, x, w, y, rows, nvec, inv_D, eps, st);
             return launch_reg_vpt<512, 512, 1, 1>((nvec + 511) / 512, x, w, y, rows, nvec, inv_D, eps, st);
         case AK_PATH_SMEM:
             if (D * 2 > kMaxRowSmemBytes) return AK_ERR_SHAPE;
