@@ -125,13 +125,10 @@ __device__ __forceinline__ void row_slice_lse(const uint16_t* __restrict__ xr, i
     const uint4* body = reinterpret_cast<const uint4*>(p + head);
     const f32x2 l2 = pack2(kLog2e, kLog2e);
 
-    for (int64_t base = 0; base < nbody; base += (int64_t)T * UNROLL) {
-        uint4 q[UNROLL];
-#pragma unroll
-        for (int k = 0; k < UNROLL; ++k) {
-            const int64_t i = base + threadIdx.x + (int64_t)k * T;
-            q[k] = (i < nbody) ? ld_stream(body + i) : make_uint4(kXNegInf2, kXNegInf2, kXNegInf2, kXNegInf2);
-        }
+    // One batch = UNROLL vectors per thread, all loaded before the first use.  Full batches
+    // run without any per-vector bounds test (constant offsets from one moving pointer); a
+    // single masked batch finishes the slice.
+    auto absorb_batch = [&](const uint4 (&q)[UNROLL]) {
         uint32_t mx = xmax8(q[0]);
 #pragma unroll
         for (int k = 1; k < UNROLL; ++k) mx = bf16x2_max_nan(mx, xmax8(q[k]));
@@ -141,6 +138,24 @@ __device__ __forceinline__ void row_slice_lse(const uint16_t* __restrict__ xr, i
 #pragma unroll
         for (int k = 1; k < UNROLL; ++k) acc = add2(acc, sumexp8<POLY>(q[k], l2, nmf2));
         o.s2 = add2(o.s2, acc);
+    };
+    const int64_t nfull = nbody / ((int64_t)T * UNROLL);
+    const uint4* src = body + threadIdx.x;
+    for (int64_t b = 0; b < nfull; ++b, src += T * UNROLL) {
+        uint4 q[UNROLL];
+#pragma unroll
+        for (int k = 0; k < UNROLL; ++k) q[k] = ld_stream(src + k * T);
+        absorb_batch(q);
+    }
+    const int rest = (int)(nbody - nfull * T * UNROLL);  // vectors left, < T * UNROLL
+    if (rest > 0) {
+        uint4 q[UNROLL];
+#pragma unroll
+        for (int k = 0; k < UNROLL; ++k) {
+            const int i = (int)threadIdx.x + k * T;
+            q[k] = (i < rest) ? ld_stream(src + k * T) : make_uint4(kXNegInf2, kXNegInf2, kXNegInf2, kXNegInf2);
+        }
+        absorb_batch(q);
     }
     if ((int64_t)threadIdx.x < head) absorb_scalar(o, bf16_to_float(ld_stream_u16(p + threadIdx.x)));
     if (tail0 + threadIdx.x < n) absorb_scalar(o, bf16_to_float(ld_stream_u16(p + tail0 + threadIdx.x)));
