@@ -569,7 +569,7 @@ def run_sweep(ak, synth, dev, peak):
         rows_out.append({"op": op, "rows": rows, "D": D, "us_trimmed_mean": us, "us_min": us_min,
                          "us_median": us_med, "GB/s": gbs, "frac_of_8TBs": gbs / NOMINAL_HBM_GBS,
                          "frac_of_measured_copy": gbs / peak, "rows_per_s": rows / (us * 1e-6),
-                         "buffer_sets": nsets, "large_shape": one_set >= (256 << 20)})
+                         "buffer_sets": nsets, "large_shape": one_set >= (250 << 20)})
         del sets
         torch.cuda.empty_cache()
     os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)

@@ -105,6 +105,32 @@ int rmsnorm_dispatch(const void* x, const void* w, void* y, int64_t rows, int64_
             if (nvec <= 4096) return launch_smem<256>(x, w, y, rows, nvec, inv_D, eps, st);
             return launch_smem<512>(x, w, y, rows, nvec, inv_D, eps, st);
         case AK_PATH_GENERIC: {
+            // rows staged in shared memory when x and y rows share their 16-byte phase, w is
+            // 4-byte aligned and a row (plus up to 14 bytes of phase padding) fits
+            const size_t stage_bytes = (size_t)((D + 14) >> 3) * 16;
+            const bool same_phase = ((reinterpret_cast<uintptr_t>(x) ^ reinterpret_cast<uintptr_t>(y)) & 15) == 0;
+            if (same_phase && is_aligned(w, 4) && stage_bytes <= (size_t)kMaxRowSmemBytes) {
+                static const bool configured = [] {
+                    return cudaFuncSetAttribute(rmsnorm_stage_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                kMaxRowSmemBytes) == cudaSuccess &&
+                           cudaFuncSetAttribute(rmsnorm_stage_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                kMaxRowSmemBytes) == cudaSuccess &&
+                           cudaFuncSetAttribute(rmsnorm_stage_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                kMaxRowSmemBytes) == cudaSuccess;
+                }();
+                if (!configured) return AK_ERR_CUDA;
+                const uint16_t* xs = static_cast<const uint16_t*>(x);
+                const uint16_t* ws = static_cast<const uint16_t*>(w);
+                uint16_t* ys = static_cast<uint16_t*>(y);
+                if (D <= 8192)
+                    rmsnorm_stage_kernel<128><<<(unsigned)rows, 128, stage_bytes, st>>>(xs, ws, ys, D, inv_D, eps);
+                else if (D <= 32768)
+                    rmsnorm_stage_kernel<256><<<(unsigned)rows, 256, stage_bytes, st>>>(xs, ws, ys, D, inv_D, eps);
+                else
+                    rmsnorm_stage_kernel<512><<<(unsigned)rows, 512, stage_bytes, st>>>(xs, ws, ys, D, inv_D, eps);
+                count_launch();
+                return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+            }
             static const int resident = [] {
                 int per_sm = 0;
                 if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rmsnorm_generic_kernel,

@@ -182,6 +182,75 @@ rmsnorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w, ui
     for (int i = threadIdx.x; i < nvec; i += THREADS) st_stream(yr + i, scale8(row[i], __ldg(w + i), rstd));
 }
 
+// ------------------------------------------------------------------ unaligned rows staged in shared memory
+// D % 8 != 0 (or a misaligned base) makes the 16-byte phase of a row change from row to row.
+// One CTA per row copies the row into shared memory in the phase it has in global memory:
+// vector k of the staging buffer holds row elements [8k - phase, 8k - phase + 8), so every
+// fully-inside vector is one aligned 16-byte global load and, because x and y rows share the
+// phase here, one aligned 16-byte store.  The (at most two) edge vectors are filled element
+// by element, zeros standing in for the neighbours' bytes, and written back element by
+// element, so nothing outside the row is ever read or written.  Weights for an inside vector
+// start at the odd or even element 8k - phase: four 4-byte loads (phase even) or five plus
+// funnel shifts (phase odd), all L1 hits.  Needs w 4-byte aligned and the row to fit.
+// (T threads per CTA: 128 up to D = 8192, where many small CTAs per SM matter most, more above)
+
+__device__ __forceinline__ uint4 load_w_shifted(const uint16_t* __restrict__ w, int64_t j0) {
+    // j0 >= 0: first weight index of the vector; w is 4-byte aligned
+    const uint32_t* ww = reinterpret_cast<const uint32_t*>(w) + (j0 >> 1);
+    if ((j0 & 1) == 0) return make_uint4(__ldg(ww), __ldg(ww + 1), __ldg(ww + 2), __ldg(ww + 3));
+    // the fifth word would reach one element past j0 + 7 (possibly past the end of w): only
+    // its low half is needed, so fetch that half alone
+    const uint32_t a = __ldg(ww), b = __ldg(ww + 1), c = __ldg(ww + 2), d = __ldg(ww + 3);
+    const uint32_t e = (uint32_t)__ldg(w + j0 + 7);
+    return make_uint4(__funnelshift_r(a, b, 16), __funnelshift_r(b, c, 16), __funnelshift_r(c, d, 16),
+                      __funnelshift_r(d, e, 16));
+}
+
+template <int T>
+__global__ void __launch_bounds__(T)
+rmsnorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, uint16_t* __restrict__ y,
+                     int64_t D, float inv_D, float eps) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    uint4* row = reinterpret_cast<uint4*>(smem_raw);
+    uint16_t* row16 = reinterpret_cast<uint16_t*>(smem_raw);
+    __shared__ float slots[2 * kWarp];
+    const int64_t r = blockIdx.x;
+    const uint16_t* xr = x + r * D;
+    uint16_t* yr = y + r * D;
+    const int phase = (int)((reinterpret_cast<uintptr_t>(xr) >> 1) & 7);
+    const int nv = (int)((phase + D + 7) >> 3);
+    const int k_lo = phase ? 1 : 0;                      // first fully-inside vector
+    const int k_hi = ((phase + D) & 7) ? nv - 1 : nv;    // one past the last fully-inside vector
+    const uint4* xa = reinterpret_cast<const uint4*>(xr - phase);
+    uint4* ya = reinterpret_cast<uint4*>(yr - phase);
+
+    for (int k = k_lo + threadIdx.x; k < k_hi; k += T) row[k] = ld_stream(xa + k);
+    if (threadIdx.x < 16) {  // edge vectors: 8 lanes for the first, 8 for the last
+        const int k = (threadIdx.x < 8) ? 0 : nv - 1;
+        const bool edge = (threadIdx.x < 8) ? (k_lo == 1) : (k_hi == nv - 1 && !(nv == 1 && k_lo == 1));
+        if (edge) {
+            const int e = threadIdx.x & 7;
+            const int64_t j = (int64_t)k * 8 - phase + e;
+            row16[k * 8 + e] = (j >= 0 && j < D) ? ld_stream_u16(xr + j) : (uint16_t)0;
+        }
+    }
+    __syncthreads();
+    float ss = 0.0f;
+    for (int k = threadIdx.x; k < nv; k += T) ss += sumsq8(row[k]);
+    ss = cta_sum<T>(ss, slots, 0);
+    const float rstd = rsqrtf(fmaf(ss, inv_D, eps));
+    for (int k = k_lo + threadIdx.x; k < k_hi; k += T)
+        st_stream(ya + k, scale8(row[k], load_w_shifted(w, (int64_t)k * 8 - phase), rstd));
+    if (threadIdx.x < 16) {
+        const int k = (threadIdx.x < 8) ? 0 : nv - 1;
+        const bool edge = (threadIdx.x < 8) ? (k_lo == 1) : (k_hi == nv - 1 && !(nv == 1 && k_lo == 1));
+        const int e = threadIdx.x & 7;
+        const int64_t j = (int64_t)k * 8 - phase + e;
+        if (edge && j >= 0 && j < D)
+            yr[j] = float_to_bf16(bf16_to_float(row16[k * 8 + e]) * bf16_to_float(__ldg(w + j)) * rstd);
+    }
+}
+
 // ------------------------------------------------------------------ generic
 // Any D and any 2-byte alignment.  Row r starts at element r*D, so its 16-byte phase
 // changes from row to row: up to 7 head elements and 7 tail elements are handled with

@@ -170,6 +170,53 @@ softmax_smem_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int nvec
     }
 }
 
+// ------------------------------------------------------------------ unaligned rows staged in shared memory
+// Same staging as the RMSNorm kernel of that name: the row sits in shared memory in the
+// 16-byte phase it has in global memory (x and y rows share it), fully-inside vectors move
+// with aligned 16-byte loads and stores, the edge vectors element by element with -inf
+// standing in for the neighbours' bytes.  Three passes over shared memory.
+template <int T>
+__global__ void __launch_bounds__(T)
+softmax_stage_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, int64_t D) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    uint4* row = reinterpret_cast<uint4*>(smem_raw);
+    uint16_t* row16 = reinterpret_cast<uint16_t*>(smem_raw);
+    __shared__ float slots[2 * kWarp];
+    const int64_t r = blockIdx.x;
+    const uint16_t* xr = x + r * D;
+    uint16_t* yr = y + r * D;
+    const int phase = (int)((reinterpret_cast<uintptr_t>(xr) >> 1) & 7);
+    const int nv = (int)((phase + D + 7) >> 3);
+    const int k_lo = phase ? 1 : 0;
+    const int k_hi = ((phase + D) & 7) ? nv - 1 : nv;
+    const uint4* xa = reinterpret_cast<const uint4*>(xr - phase);
+    uint4* ya = reinterpret_cast<uint4*>(yr - phase);
+    const int my_edge_k = (threadIdx.x < 8) ? 0 : nv - 1;
+    const bool my_edge = (threadIdx.x < 16) &&
+                         ((threadIdx.x < 8) ? (k_lo == 1) : (k_hi == nv - 1 && !(nv == 1 && k_lo == 1)));
+    const int64_t my_j = (int64_t)my_edge_k * 8 - phase + (threadIdx.x & 7);
+
+    for (int k = k_lo + threadIdx.x; k < k_hi; k += T) row[k] = ld_stream(xa + k);
+    if (my_edge) row16[my_edge_k * 8 + (threadIdx.x & 7)] = (my_j >= 0 && my_j < D) ? ld_stream_u16(xr + my_j) : (uint16_t)0xFF80;
+    __syncthreads();
+
+    uint32_t mx = kNegInf2;
+    for (int k = threadIdx.x; k < nv; k += T) mx = bf16x2_max(mx, max8(row[k]));
+    const float m = cta_max<T>(hmax_of(mx), slots, 0);
+    const float m2 = m * kLog2e;
+    float sum = 0.0f;
+    f32x2 e[4];
+    for (int k = threadIdx.x; k < nv; k += T) sum += exp8(row[k], m2, e);
+    sum = cta_sum<T>(sum, slots, 1);
+    const float inv = 1.0f / sum;
+    for (int k = k_lo + threadIdx.x; k < k_hi; k += T) {
+        exp8(row[k], m2, e);
+        st_stream(ya + k, norm8(e, inv));
+    }
+    if (my_edge && my_j >= 0 && my_j < D)
+        yr[my_j] = float_to_bf16(fast_exp2(fmaf(bf16_to_float(row16[my_edge_k * 8 + (threadIdx.x & 7)]), kLog2e, -m2)) * inv);
+}
+
 // ------------------------------------------------------------------ generic
 // Any D / alignment: three passes over the row (max, sum, write); only the first comes
 // from DRAM, the other two are served by L1/L2.

@@ -197,7 +197,7 @@ def test_misaligned_base_pointers_take_generic_path():
     D, rows = 1024, 9
     x, w = synth.rmsnorm_inputs(rows, D, 91)
     ref = oracle.rmsnorm(synth.to_bits(x), synth.to_bits(w), 1e-6)
-    for xo, yo, wo in ((1, 1, 0), (1, 3, 0), (0, 0, 5), (3, 0, 1)):
+    for xo, yo, wo in ((1, 1, 0), (1, 3, 0), (0, 0, 5), (3, 0, 1), (2, 2, 2), (7, 7, 6), (5, 5, 0)):
         xbuf = torch.zeros(rows * D + 8, dtype=torch.bfloat16, device=DEV)
         ybuf = torch.zeros(rows * D + 8, dtype=torch.bfloat16, device=DEV)
         wbuf = torch.zeros(D + 8, dtype=torch.bfloat16, device=DEV)
