@@ -533,6 +533,60 @@ def time_op(fn_for_set, nsets, iters=200, warmup=20):
     return float(t[k:iters - k].mean()) * 1e3, float(t[0]) * 1e3, float(np.median(t)) * 1e3
 
 
+def sweep_accuracy(ak, synth, op, rows, D, bufs):
+    """Errors of the outputs of buffer set 0 against the CPU checker on a sample of rows, a
+    bitwise repeat check, and the checker's own speed on that sample (1 thread and all
+    threads), scaled to the full number of rows."""
+    import oracle
+    n = int(max(1, min(rows, 64, (1 << 22) // D)))
+    idx = np.unique(np.concatenate([[0, rows - 1], np.random.default_rng(rows + D).integers(0, rows, n)]))
+    it = torch.from_numpy(idx).to(bufs[0].device)
+    widen = lambda t: (t.cpu().view(torch.int16).numpy().view(np.uint16).astype(np.uint32) << 16
+                       ).view(np.float32).astype(np.float64)
+    cores = oracle.set_threads(0)
+
+    def timed_oracle(fn):
+        t0 = time.perf_counter()
+        ref = fn()
+        t_all = time.perf_counter() - t0
+        oracle.set_threads(1)
+        t0 = time.perf_counter()
+        fn()
+        t_one = time.perf_counter() - t0
+        oracle.set_threads(cores)
+        return ref, t_one * rows / len(idx), t_all * rows / len(idx)
+
+    if op == "rmsnorm":
+        x, w, y = bufs
+        first = y.clone()
+        ak.ak_rmsnorm_fwd(x, w, y, eps=1e-6)
+        same = torch.equal(first.view(torch.int16), y.view(torch.int16))
+        ref, t1, tn = timed_oracle(lambda: oracle.rmsnorm(synth.to_bits(x[it]), synth.to_bits(w), 1e-6))
+        got = widen(y[it])
+    elif op == "softmax":
+        x, y = bufs
+        first = y.clone()
+        ak.ak_softmax_fwd(x, y)
+        same = torch.equal(first.view(torch.int16), y.view(torch.int16))
+        ref, t1, tn = timed_oracle(lambda: oracle.softmax(synth.to_bits(x[it])))
+        got = widen(y[it])
+    else:
+        lg, tg, loss, mean, ws = bufs
+        first = loss.clone()
+        ak.ak_xent_fwd_ws(lg, tg, ws, -100, loss, mean)
+        same = torch.equal(first.view(torch.int32), loss.view(torch.int32))
+        ref, t1, tn = timed_oracle(lambda: oracle.xent(synth.to_bits(lg[it]), tg[it].cpu().numpy())[0])
+        got = loss[it].cpu().double().numpy()
+    torch.cuda.synchronize()
+    err = np.abs(got - ref)
+    rel = err / np.maximum(np.abs(ref), 1e-30)
+    return {"max_abs_err": float(err.max()), "max_rel_err_where_ref_ge_1e-3": float(rel[np.abs(ref) >= 1e-3].max()
+                                                                               if (np.abs(ref) >= 1e-3).any() else 0.0),
+            "max_err_over_tolerance": float((err / ((1.6e-2 if op != "xent" else 1e-5) * np.maximum(1.0, np.abs(ref)))).max()),
+            "bitwise_repeat": bool(same), "sampled_rows": int(len(idx)),
+            "oracle_s_1_thread_scaled": t1, "oracle_s_all_threads_scaled": tn, "oracle_threads": cores}
+
+
 def run_sweep(ak, synth, dev, peak):
     rows_out = []
     only = os.environ.get("AK_SWEEP_OPS")
@@ -566,10 +620,11 @@ def run_sweep(ak, synth, dev, peak):
             nb = algorithmic_bytes(op, rows, D, int((sets[0][1] != -100).sum()))
         us, us_min, us_med = time_op(fn, nsets)
         gbs = nb / (us * 1e-6) / 1e9
+        acc = sweep_accuracy(ak, synth, op, rows, D, sets[0])
         rows_out.append({"op": op, "rows": rows, "D": D, "us_trimmed_mean": us, "us_min": us_min,
                          "us_median": us_med, "GB/s": gbs, "frac_of_8TBs": gbs / NOMINAL_HBM_GBS,
                          "frac_of_measured_copy": gbs / peak, "rows_per_s": rows / (us * 1e-6),
-                         "buffer_sets": nsets, "large_shape": one_set >= (250 << 20)})
+                         "buffer_sets": nsets, "large_shape": one_set >= (250 << 20), **acc})
         del sets
         torch.cuda.empty_cache()
     os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
