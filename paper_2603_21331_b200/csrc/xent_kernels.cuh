@@ -109,56 +109,82 @@ __device__ __forceinline__ void absorb_scalar(Online& o, float v) {
     o.s2 = add2(o.s2, pack2(fast_exp2(fmaf(v, kLog2e, -o.mf)), 0.0f));
 }
 
-// CTA-wide online (m, s) over elements [begin, end) of one row.  Returns, in every
-// thread, the maximum M and the sum S relative to MF = max(rn(M*log2e), kFloor2).
-// Uses both slot sets (max then sum).  UNROLL vectors are in flight per thread.
-template <int UNROLL, int POLY, int T = kXentThreads>
-__device__ __forceinline__ void row_slice_lse(const uint16_t* __restrict__ xr, int64_t begin, int64_t end,
-                                              float* slots, float& M, float& S) {
-    Online o{-INFINITY, kFloor2, pack2(0.0f, 0.0f)};
-    const uint16_t* p = xr + begin;
-    const int64_t n = end - begin;
-    int64_t head = (8 - (int)((reinterpret_cast<uintptr_t>(p) >> 1) & 7)) & 7;
-    if (head > n) head = n;
-    const int64_t nbody = (n - head) >> 3;
-    const int64_t tail0 = head + (nbody << 3);
-    const uint4* body = reinterpret_cast<const uint4*>(p + head);
-    const f32x2 l2 = pack2(kLog2e, kLog2e);
-
-    // One batch = UNROLL vectors per thread, all loaded before the first use.  Full batches
-    // run without any per-vector bounds test (constant offsets from one moving pointer); a
-    // single masked batch finishes the slice.
-    auto absorb_batch = [&](const uint4 (&q)[UNROLL]) {
-        uint32_t mx = xmax8(q[0]);
+// A slice = elements [begin, end) of one row, cut into up to 7 head elements (2-byte loads
+// until the address is 16-byte aligned), nbody aligned 16-byte vectors, and up to 7 tail
+// elements.  One batch = UNROLL vectors per thread, all loaded before the first use.  Full
+// batches run without any per-vector bounds test (constant offsets from one moving pointer);
+// a single masked batch finishes the slice.
+struct Slice {
+    const uint16_t* p;
+    int64_t n, head, nbody, tail0, nfull;
+    const uint4* body;
+    int rest;  // vectors in the masked last batch, < T * UNROLL
+};
+template <int UNROLL, int T>
+__device__ __forceinline__ Slice make_slice(const uint16_t* __restrict__ xr, int64_t begin, int64_t end) {
+    Slice s;
+    s.p = xr + begin;
+    s.n = end - begin;
+    s.head = (8 - (int)((reinterpret_cast<uintptr_t>(s.p) >> 1) & 7)) & 7;
+    if (s.head > s.n) s.head = s.n;
+    s.nbody = (s.n - s.head) >> 3;
+    s.tail0 = s.head + (s.nbody << 3);
+    s.body = reinterpret_cast<const uint4*>(s.p + s.head);
+    s.nfull = s.nbody / ((int64_t)T * UNROLL);
+    s.rest = (int)(s.nbody - s.nfull * T * UNROLL);
+    return s;
+}
+// The slice's first batch (full if there is a full batch, otherwise the masked one).
+template <int UNROLL, int T>
+__device__ __forceinline__ void load_first_batch(const Slice& s, uint4 (&q)[UNROLL]) {
+    const uint4* src = s.body + threadIdx.x;
+    if (s.nfull > 0) {
 #pragma unroll
-        for (int k = 1; k < UNROLL; ++k) mx = bf16x2_max_nan(mx, xmax8(q[k]));
+        for (int k = 0; k < UNROLL; ++k) q[k] = ld_stream(src + k * T);
+    } else {
+#pragma unroll
+        for (int k = 0; k < UNROLL; ++k) {
+            const int i = (int)threadIdx.x + k * T;
+            q[k] = (i < s.rest) ? ld_stream(src + k * T) : make_uint4(kXNegInf2, kXNegInf2, kXNegInf2, kXNegInf2);
+        }
+    }
+}
+
+// CTA-wide online (m, s) over a slice whose first batch `q` is already in flight.  Returns,
+// in every thread, the maximum M and the sum S relative to MF = max(rn(M*log2e), kFloor2).
+// Uses both slot sets (max then sum).
+template <int UNROLL, int POLY, int T>
+__device__ __forceinline__ void slice_lse(const Slice& sl, uint4 (&q)[UNROLL], float* slots, float& M, float& S) {
+    Online o{-INFINITY, kFloor2, pack2(0.0f, 0.0f)};
+    const f32x2 l2 = pack2(kLog2e, kLog2e);
+    auto absorb_batch = [&](const uint4 (&v)[UNROLL]) {
+        uint32_t mx = xmax8(v[0]);
+#pragma unroll
+        for (int k = 1; k < UNROLL; ++k) mx = bf16x2_max_nan(mx, xmax8(v[k]));
         raise_max(o, xhmax_of(mx));
         const f32x2 nmf2 = pack2(-o.mf, -o.mf);
-        f32x2 acc = sumexp8<POLY>(q[0], l2, nmf2);
+        f32x2 acc = sumexp8<POLY>(v[0], l2, nmf2);
 #pragma unroll
-        for (int k = 1; k < UNROLL; ++k) acc = add2(acc, sumexp8<POLY>(q[k], l2, nmf2));
+        for (int k = 1; k < UNROLL; ++k) acc = add2(acc, sumexp8<POLY>(v[k], l2, nmf2));
         o.s2 = add2(o.s2, acc);
     };
-    const int64_t nfull = nbody / ((int64_t)T * UNROLL);
-    const uint4* src = body + threadIdx.x;
-    for (int64_t b = 0; b < nfull; ++b, src += T * UNROLL) {
-        uint4 q[UNROLL];
+    absorb_batch(q);  // batch 0 (all padding when the slice has no body)
+    const uint4* src = sl.body + threadIdx.x + T * UNROLL;
+    for (int64_t b = 1; b < sl.nfull; ++b, src += T * UNROLL) {
 #pragma unroll
         for (int k = 0; k < UNROLL; ++k) q[k] = ld_stream(src + k * T);
         absorb_batch(q);
     }
-    const int rest = (int)(nbody - nfull * T * UNROLL);  // vectors left, < T * UNROLL
-    if (rest > 0) {
-        uint4 q[UNROLL];
+    if (sl.nfull > 0 && sl.rest > 0) {
 #pragma unroll
         for (int k = 0; k < UNROLL; ++k) {
             const int i = (int)threadIdx.x + k * T;
-            q[k] = (i < rest) ? ld_stream(src + k * T) : make_uint4(kXNegInf2, kXNegInf2, kXNegInf2, kXNegInf2);
+            q[k] = (i < sl.rest) ? ld_stream(src + k * T) : make_uint4(kXNegInf2, kXNegInf2, kXNegInf2, kXNegInf2);
         }
         absorb_batch(q);
     }
-    if ((int64_t)threadIdx.x < head) absorb_scalar(o, bf16_to_float(ld_stream_u16(p + threadIdx.x)));
-    if (tail0 + threadIdx.x < n) absorb_scalar(o, bf16_to_float(ld_stream_u16(p + tail0 + threadIdx.x)));
+    if ((int64_t)threadIdx.x < sl.head) absorb_scalar(o, bf16_to_float(ld_stream_u16(sl.p + threadIdx.x)));
+    if (sl.tail0 + threadIdx.x < sl.n) absorb_scalar(o, bf16_to_float(ld_stream_u16(sl.p + sl.tail0 + threadIdx.x)));
 
     // NaN must win the max: fmaxf in cta_max would drop it, so it travels as +inf plus a flag
     const bool has_nan = (o.m != o.m) || (o.m == INFINITY);  // +inf makes inf - inf: NaN row as well
@@ -195,16 +221,21 @@ xent_row_kernel(const uint16_t* __restrict__ logits, const int64_t* __restrict__
     __shared__ float slots[2 * kWarp];
     pdl_launch_dependents();
     const int64_t row = blockIdx.x;
+    const uint16_t* xr = logits + row * V;
     const int64_t t = targets[row];
     if (t == ignore_index || t < 0 || t >= V) {  // uniform across the CTA: nothing is read
         if (threadIdx.x == 0) loss_rows[row] = (t == ignore_index) ? 0.0f : __int_as_float(0x7fc00000);
         return;
     }
-    const uint16_t* xr = logits + row * V;
+    // (Requesting the first batch before the target is known was measured: no gain, and
+    // ignored rows would be touched.)
+    const Slice sl = make_slice<UNROLL, T>(xr, 0, V);
+    uint4 q[UNROLL];
+    load_first_batch<UNROLL, T>(sl, q);
     // the target logit is fetched now, under the row's own traffic, not after the reduction
     const float xt = (threadIdx.x == 0) ? bf16_to_float(xr[t]) : 0.0f;
     float M, S;
-    row_slice_lse<UNROLL, POLY, T>(xr, 0, V, slots, M, S);
+    slice_lse<UNROLL, POLY, T>(sl, q, slots, M, S);
     if (threadIdx.x == 0) loss_rows[row] = finish_loss(M, S, xt);
 }
 
@@ -225,8 +256,11 @@ xent_split_kernel(const uint16_t* __restrict__ logits, const int64_t* __restrict
     int64_t begin = ((groups * sp) / nsplit) << 3;
     int64_t end = ((groups * (sp + 1)) / nsplit) << 3;
     if (end > V) end = V;
+    const Slice sl = make_slice<UNROLL, kXentThreads>(logits + row * V, begin, end);
+    uint4 q[UNROLL];
+    load_first_batch<UNROLL, kXentThreads>(sl, q);
     float M, S;
-    row_slice_lse<UNROLL, POLY>(logits + row * V, begin, end, slots, M, S);
+    slice_lse<UNROLL, POLY, kXentThreads>(sl, q, slots, M, S);
     if (threadIdx.x == 0) partial[row * nsplit + sp] = make_float2(M, S);
 }
 

@@ -103,6 +103,29 @@ def test_xent_parity_row_and_split(rows, V):
     assert torch.equal(m1.view(torch.int32), m2.view(torch.int32)) or (torch.isnan(m1).all() and torch.isnan(m2).all())
 
 
+@pytest.mark.parametrize("V", [1000, 32000])
+def test_xent_masked_vocabulary_and_extreme_gaps(V):
+    """-inf logits (a masked vocabulary) contribute nothing, a -inf target gives +inf, gaps far
+    beyond the polynomial's clamp (2^-125) and rows dominated by one element stay accurate."""
+    rows = 24
+    logits, targets = synth.xent_inputs(rows, V, synth.case_seed(5, V), ignore_frac=0.0)
+    g = torch.Generator().manual_seed(V)
+    masked = torch.rand((rows, V), generator=g) < 0.3
+    logits = logits.masked_fill(masked, float("-inf"))
+    logits[3, :] = -200.0                      # everything 200 below ...
+    logits[3, 17] = 50.0                       # ... one element: loss 0 on it, 250 elsewhere
+    logits[4, :] = torch.where(torch.arange(V) % 2 == 0, 0.0, -120.0).to(torch.bfloat16)
+    targets[3] = 17
+    targets[5] = int(torch.nonzero(masked[5])[0])          # target on a -inf logit -> +inf
+    ref_rows, ref_mean, _ = oracle.xent(synth.to_bits(logits), targets.numpy())
+    assert np.isinf(ref_rows[5]) and ref_rows[3] == 0.0
+    for path, ns in ((ak.AK_XENT_ROW, 0), (ak.AK_XENT_SPLIT, 3)):
+        loss, mean = ak.ak_xent_fwd(logits.to(DEV), targets.to(DEV), path=path, nsplit=ns)
+        torch.cuda.synchronize()
+        assert_loss_close(loss, ref_rows, f"masked vocabulary V={V} path {path}")
+        assert torch.isinf(mean).all() and np.isinf(ref_mean)
+
+
 def test_xent_mean_skipped_when_null():
     logits, targets = synth.xent_inputs(16, 512, 7)
     loss, mean = ak.ak_xent_fwd(logits.to(DEV), targets.to(DEV), want_mean=False)
