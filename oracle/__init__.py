@@ -37,6 +37,10 @@ def _load():
         lib.oracle_set_threads.restype = ctypes.c_int
         lib.oracle_rmsnorm.argtypes = [p, p, p, i64, i64, f32]
         lib.oracle_rmsnorm.restype = None
+        lib.oracle_layernorm.argtypes = [p, p, p, p, i64, i64, f32]
+        lib.oracle_layernorm.restype = None
+        lib.oracle_rowsum.argtypes = [p, p, i64, i64]
+        lib.oracle_rowsum.restype = None
         lib.oracle_softmax.argtypes = [p, p, i64, i64]
         lib.oracle_softmax.restype = None
         lib.oracle_xent.argtypes = [p, p, i64, p, p, p, i64, i64]
@@ -81,6 +85,32 @@ def rmsnorm(x_bits, w_bits, eps: float) -> np.ndarray:
     _load().oracle_rmsnorm(x.ctypes.data, w.ctypes.data, y.ctypes.data, rows, D,
                            float(np.float32(eps)))
     return y
+
+
+def layernorm(x_bits, gamma_bits, beta_bits, eps: float) -> np.ndarray:
+    """y[r, j] = (x[r, j] - mean_r) / sqrt(var_r + eps) * gamma[j] + beta[j] (biased variance),
+    in float64; ``eps`` is first rounded to float32."""
+    x = _bits(x_bits)
+    if x.ndim != 2:
+        raise ValueError("x must be [rows, D]")
+    rows, D = x.shape
+    g = _bits(gamma_bits, (D,))
+    b = _bits(beta_bits, (D,))
+    y = np.empty((rows, D), dtype=np.float64)
+    _load().oracle_layernorm(x.ctypes.data, g.ctypes.data, b.ctypes.data, y.ctypes.data, rows, D,
+                             float(np.float32(eps)))
+    return y
+
+
+def rowsum(x_bits) -> np.ndarray:
+    """out[r] = sum_j x[r, j], in float64."""
+    x = _bits(x_bits)
+    if x.ndim != 2:
+        raise ValueError("x must be [rows, D]")
+    rows, D = x.shape
+    out = np.empty((rows,), dtype=np.float64)
+    _load().oracle_rowsum(x.ctypes.data, out.ctypes.data, rows, D)
+    return out
 
 
 def softmax(x_bits) -> np.ndarray:

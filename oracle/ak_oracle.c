@@ -26,6 +26,9 @@
  *             t < 0 or t >= V        -> loss_r = NaN, row counted
  *             otherwise              -> loss_r = (m - x_t) + log(sum_j exp(x_j - m))
  *             loss_mean = (sum over counted rows of loss_r) / n_counted  (0/0 = NaN)
+ *   layernorm: mu = mean_j x_j ; var = mean_j (x_j - mu)^2 ;
+ *              y_j = (x_j - mu) / sqrt(var + eps) * gamma_j + beta_j   (Table 3 "layernorm")
+ *   rowsum  : out_r = sum_j x_rj                                      (Table 3 "reduce")
  *
  * Inputs are the exact bf16 bit patterns the GPU sees (uint16), widened exactly to
  * double; outputs are double and are never rounded to bf16 or fp32.
@@ -91,6 +94,47 @@ void oracle_rmsnorm(const uint16_t *x, const uint16_t *w, double *y,
         double denom = sqrt(sumsq / (double)D + eps_d);
         for (int64_t j = 0; j < D; ++j)
             yr[j] = bf16_bits_to_double(xr[j]) * bf16_bits_to_double(w[j]) / denom;
+    }
+}
+
+/* LayerNorm forward (Table 3 "layernorm": the paper's kernel is a single-pass Welford; the
+ * quantity it evaluates is the textbook one, written here as two plain passes).
+ *   mu = (1/D) sum_j x_j ;  var = (1/D) sum_j (x_j - mu)^2   (biased, as in PyTorch)
+ *   y_j = (x_j - mu) / sqrt(var + eps) * gamma_j + beta_j
+ * x: [rows, D] bf16 bits, gamma/beta: [D] bf16 bits, y: [rows, D] double. */
+void oracle_layernorm(const uint16_t *x, const uint16_t *gamma, const uint16_t *beta, double *y,
+                      int64_t rows, int64_t D, float eps)
+{
+    const double eps_d = (double)eps;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        const uint16_t *xr = x + r * D;
+        double *yr = y + r * D;
+        double sum = 0.0;
+        for (int64_t j = 0; j < D; ++j) sum += bf16_bits_to_double(xr[j]);
+        const double mu = sum / (double)D;
+        double sq = 0.0;
+        for (int64_t j = 0; j < D; ++j) {
+            double d = bf16_bits_to_double(xr[j]) - mu;
+            sq += d * d;
+        }
+        const double denom = sqrt(sq / (double)D + eps_d);
+        for (int64_t j = 0; j < D; ++j)
+            yr[j] = (bf16_bits_to_double(xr[j]) - mu) / denom * bf16_bits_to_double(gamma[j])
+                    + bf16_bits_to_double(beta[j]);
+    }
+}
+
+/* Row sum (Table 3 "reduce": hierarchical reduction of each row to one number).
+ * x: [rows, D] bf16 bits, out: [rows] double, plain left-to-right sum in double. */
+void oracle_rowsum(const uint16_t *x, double *out, int64_t rows, int64_t D)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        const uint16_t *xr = x + r * D;
+        double sum = 0.0;
+        for (int64_t j = 0; j < D; ++j) sum += bf16_bits_to_double(xr[j]);
+        out[r] = sum;
     }
 }
 

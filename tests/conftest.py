@@ -10,6 +10,12 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200); run with -m gpu")
+    # The CUDA library and the CPU checker are built in-tree on demand (both builds are
+    # no-ops when their outputs are newer than their sources); nvcc needs no GPU.
+    from paper_2603_21331_b200 import build as ak_build
+    from oracle import build as oracle_build
+    ak_build.build()
+    oracle_build.build()
 
 
 def pytest_collection_modifyitems(config, items):

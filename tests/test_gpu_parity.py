@@ -293,6 +293,38 @@ def test_bitwise_determinism_three_runs():
                 assert torch.equal(a, b)
 
 
+_DIGEST_SNIPPET = r"""
+import hashlib, sys, torch
+sys.path.insert(0, sys.argv[1])
+import paper_2603_21331_b200 as ak
+from paper_2603_21331_b200 import synth
+h = hashlib.sha256()
+x, w = synth.rmsnorm_inputs(1024, 4096, 196)
+h.update(ak.ak_rmsnorm_fwd(x.cuda(), w.cuda()).cpu().view(torch.int16).numpy().tobytes())
+xs = synth.softmax_inputs(512, 16384, 197)
+h.update(ak.ak_softmax_fwd(xs.cuda()).cpu().view(torch.int16).numpy().tobytes())
+x9, w9 = synth.rmsnorm_inputs(300, 4099, 199)
+h.update(ak.ak_rmsnorm_fwd(x9.cuda(), w9.cuda()).cpu().view(torch.int16).numpy().tobytes())
+lg, tg = synth.xent_inputs(256, 50304, 198)
+for path, ns in ((ak.AK_XENT_ROW, 0), (ak.AK_XENT_SPLIT, 5)):
+    loss, mean = ak.ak_xent_fwd(lg.cuda(), tg.cuda(), path=path, nsplit=ns)
+    h.update(loss.cpu().numpy().tobytes()); h.update(mean.cpu().numpy().tobytes())
+print(h.hexdigest())
+"""
+
+
+def test_bitwise_determinism_across_processes():
+    """Two fresh processes produce byte-identical outputs (register, shared-memory, staged and
+    both cross-entropy layouts)."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    digests = [subprocess.run([sys.executable, "-c", _DIGEST_SNIPPET, root], capture_output=True, text=True,
+                              check=True).stdout.strip() for _ in range(2)]
+    assert len(digests[0]) == 64 and digests[0] == digests[1]
+
+
 def test_host_buffer_variants_match_device_path():
     x, w = synth.rmsnorm_inputs(5000, 4096, 101)       # > one 16 MiB chunk, ragged last chunk
     y_dev = ak.ak_rmsnorm_fwd(x.to(DEV), w.to(DEV)).cpu()
