@@ -62,6 +62,10 @@ def measured_peak():
 def algorithmic_bytes(op, rows, D, n_valid=None):
     if op == "rmsnorm":
         return 4 * rows * D + 2 * D
+    if op == "layernorm":
+        return 4 * rows * D + 4 * D
+    if op == "rowsum":
+        return 2 * rows * D + 4 * rows
     if op == "softmax":
         return 4 * rows * D
     nv = rows if n_valid is None else n_valid
@@ -490,6 +494,10 @@ SWEEP = (
     + [("softmax", 16384, d) for d in (512, 1024, 2048, 4096, 8192, 32768)]
     + [("softmax", 262144, 4096), ("softmax", 16384, 4099)]
     + [("xent", 4096, v) for v in (32000, 50304, 128256, 128257)] + [("xent", 16384, 128256), ("xent", 16, 128256)]
+    + [("layernorm", 8192, 4096), ("layernorm", 4096, 5120), ("layernorm", 8192, 8192), ("layernorm", 65536, 4096),
+       ("layernorm", 4096, 32768), ("layernorm", 8192, 4099)]
+    + [("rowsum", 8192, 4096), ("rowsum", 8192, 8192), ("rowsum", 65536, 1024), ("rowsum", 65536, 8192),
+       ("rowsum", 4096, 128256), ("rowsum", 8192, 4099)]
 )
 
 
@@ -563,6 +571,21 @@ def sweep_accuracy(ak, synth, op, rows, D, bufs):
         same = torch.equal(first.view(torch.int16), y.view(torch.int16))
         ref, t1, tn = timed_oracle(lambda: oracle.rmsnorm(synth.to_bits(x[it]), synth.to_bits(w), 1e-6))
         got = widen(y[it])
+    elif op == "layernorm":
+        x, g, b, y = bufs
+        first = y.clone()
+        ak.ak_layernorm_fwd(x, g, b, y, eps=1e-5)
+        same = torch.equal(first.view(torch.int16), y.view(torch.int16))
+        ref, t1, tn = timed_oracle(lambda: oracle.layernorm(synth.to_bits(x[it]), synth.to_bits(g),
+                                                            synth.to_bits(b), 1e-5))
+        got = widen(y[it])
+    elif op == "rowsum":
+        x, out = bufs
+        first = out.clone()
+        ak.ak_rowsum_fwd(x, out)
+        same = torch.equal(first.view(torch.int32), out.view(torch.int32))
+        ref, t1, tn = timed_oracle(lambda: oracle.rowsum(synth.to_bits(x[it])))
+        got = out[it].cpu().double().numpy()
     elif op == "softmax":
         x, y = bufs
         first = y.clone()
@@ -580,6 +603,11 @@ def sweep_accuracy(ak, synth, op, rows, D, bufs):
     torch.cuda.synchronize()
     err = np.abs(got - ref)
     rel = err / np.maximum(np.abs(ref), 1e-30)
+    if op == "rowsum":   # no bf16 output: report the error relative to sum |x| (fp32 accumulation)
+        mag = np.abs(widen(x[it])).sum(axis=1)
+        return {"max_abs_err": float(err.max()), "max_err_over_sum_abs_x": float((err / np.maximum(mag, 1e-30)).max()),
+                "bitwise_repeat": bool(same), "sampled_rows": int(len(idx)),
+                "oracle_s_1_thread_scaled": t1, "oracle_s_all_threads_scaled": tn, "oracle_threads": cores}
     return {"max_abs_err": float(err.max()), "max_rel_err_where_ref_ge_1e-3": float(rel[np.abs(ref) >= 1e-3].max()
                                                                                if (np.abs(ref) >= 1e-3).any() else 0.0),
             "max_err_over_tolerance": float((err / ((1.6e-2 if op != "xent" else 1e-5) * np.maximum(1.0, np.abs(ref)))).max()),
@@ -593,13 +621,19 @@ def run_sweep(ak, synth, dev, peak):
     for op, rows, D in SWEEP:
         if only and op not in only.split(","):
             continue
-        one_set = (4 if op != "xent" else 2) * rows * D
+        one_set = (2 if op in ("xent", "rowsum") else 4) * rows * D
         nsets = int(max(1, min(64, -(-(1 << 30) // one_set))))
         sets = []
         for s in range(nsets):
             if op == "rmsnorm":
                 x, w = synth.rmsnorm_inputs(rows, D, 7000 + s, device=dev)
                 sets.append((x, w, torch.empty_like(x)))
+            elif op == "layernorm":
+                x, g, b = synth.layernorm_inputs(rows, D, 7300 + s, device=dev)
+                sets.append((x, g, b, torch.empty_like(x)))
+            elif op == "rowsum":
+                x, _, _ = synth.layernorm_inputs(rows, D, 7400 + s, device=dev)
+                sets.append((x, torch.empty((rows,), dtype=torch.float32, device=dev)))
             elif op == "softmax":
                 x = synth.softmax_inputs(rows, D, 7100 + s, device=dev)
                 sets.append((x, torch.empty_like(x)))
@@ -611,6 +645,12 @@ def run_sweep(ak, synth, dev, peak):
                              torch.empty((nws,), dtype=torch.uint8, device=dev) if nws else None))
         if op == "rmsnorm":
             fn = lambda i: ak.ak_rmsnorm_fwd(sets[i][0], sets[i][1], sets[i][2], eps=1e-6)
+            nb = algorithmic_bytes(op, rows, D)
+        elif op == "layernorm":
+            fn = lambda i: ak.ak_layernorm_fwd(sets[i][0], sets[i][1], sets[i][2], sets[i][3], eps=1e-5)
+            nb = algorithmic_bytes(op, rows, D)
+        elif op == "rowsum":
+            fn = lambda i: ak.ak_rowsum_fwd(sets[i][0], sets[i][1])
             nb = algorithmic_bytes(op, rows, D)
         elif op == "softmax":
             fn = lambda i: ak.ak_softmax_fwd(sets[i][0], sets[i][1])
@@ -649,6 +689,16 @@ def run_case(args):
         x, w = synth.rmsnorm_inputs(rows, D, 7000, device=dev)
         y = torch.empty_like(x)
         fn = lambda: ak.ak_rmsnorm_fwd(x, w, y, eps=1e-6)
+        nb = algorithmic_bytes(op, rows, D)
+    elif op == "layernorm":
+        x, g, b = synth.layernorm_inputs(rows, D, 7300, device=dev)
+        y = torch.empty_like(x)
+        fn = lambda: ak.ak_layernorm_fwd(x, g, b, y, eps=1e-5)
+        nb = algorithmic_bytes(op, rows, D)
+    elif op == "rowsum":
+        x, _, _ = synth.layernorm_inputs(rows, D, 7400, device=dev)
+        out = torch.empty((rows,), dtype=torch.float32, device=dev)
+        fn = lambda: ak.ak_rowsum_fwd(x, out)
         nb = algorithmic_bytes(op, rows, D)
     elif op == "softmax":
         x = synth.softmax_inputs(rows, D, 7100, device=dev)

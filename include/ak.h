@@ -78,6 +78,29 @@ int ak_rmsnorm_fwd_path(const void* x, const void* w, void* y,
                         int64_t rows, int64_t D, float eps, void* cuda_stream, int path);
 
 /* ---------------------------------------------------------------------------------
+ * LayerNorm forward (Table 3 "layernorm"; Table 4 rows "layernorm").
+ *   mu = (1/D) sum_k x[r, k];  var = (1/D) sum_k (x[r, k] - mu)^2   (biased)
+ *   y[r, j] = bf16_rne( (x[r, j] - mu) * rsqrt(var + eps) * gamma[j] + beta[j] )
+ * x, y: device bf16 [rows, D] (y may alias x); gamma, beta: device bf16 [D]; moments in
+ * fp32, taken in two fixed-order passes over the on-chip copy of the row (the mean as
+ * x[r,0] + mean(x - x[r,0]), so a constant row gives exactly beta).  eps finite, >= 0.
+ * Same path ids, size limits and alignment rules as RMSNorm (gamma and beta together play
+ * the part of w).  Status codes as for RMSNorm.
+ */
+int ak_layernorm_fwd(const void* x, const void* gamma, const void* beta, void* y,
+                     int64_t rows, int64_t D, float eps, void* cuda_stream);
+int ak_layernorm_fwd_path(const void* x, const void* gamma, const void* beta, void* y,
+                          int64_t rows, int64_t D, float eps, void* cuda_stream, int path);
+
+/* ---------------------------------------------------------------------------------
+ * Row-sum reduce (Table 3 "reduce").
+ *   out[r] = fp32( sum_k x[r, k] ),  fp32 accumulation in a fixed order
+ * x: device bf16 [rows, D], 2-byte aligned, any D >= 1; out: device fp32 [rows], caller
+ * owned.  One launch, no scratch.  inf/NaN propagate per IEEE-754.
+ */
+int ak_rowsum_fwd(const void* x, float* out, int64_t rows, int64_t D, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------
  * Softmax forward over the last dimension (Table 3 "softmax").
  *   m = max_k x[r, k];  y[r, j] = bf16_rne( exp(x[r, j] - m) / sum_k exp(x[r, k] - m) )
  * -inf entries (a causal mask lives in the data) give exactly 0.  A row that is all
@@ -197,6 +220,7 @@ int ak_sol_read(const void* src, size_t bytes, void* sink4, void* cuda_stream);
 /* Path id the dispatcher picks for (rows, D) with fully aligned pointers (`aligned16` != 0)
  * or not.  Pure functions; no CUDA calls. */
 int ak_rmsnorm_choose_path(int64_t rows, int64_t D, int aligned16);
+int ak_layernorm_choose_path(int64_t rows, int64_t D, int aligned16);
 int ak_softmax_choose_path(int64_t rows, int64_t D, int aligned16);
 /* Returns AK_XENT_ROW or AK_XENT_SPLIT and stores the split count (1 for ROW). */
 int ak_xent_choose_path(int64_t rows, int64_t V, int* nsplit_out);

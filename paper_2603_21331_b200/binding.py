@@ -33,6 +33,9 @@ _i64, _f32, _int, _p, _sz = (ctypes.c_int64, ctypes.c_float, ctypes.c_int, ctype
 SIGNATURES = {
     "ak_rmsnorm_fwd": (_int, [_p, _p, _p, _i64, _i64, _f32, _p]),
     "ak_rmsnorm_fwd_path": (_int, [_p, _p, _p, _i64, _i64, _f32, _p, _int]),
+    "ak_layernorm_fwd": (_int, [_p, _p, _p, _p, _i64, _i64, _f32, _p]),
+    "ak_layernorm_fwd_path": (_int, [_p, _p, _p, _p, _i64, _i64, _f32, _p, _int]),
+    "ak_rowsum_fwd": (_int, [_p, _p, _i64, _i64, _p]),
     "ak_softmax_fwd": (_int, [_p, _p, _i64, _i64, _p]),
     "ak_softmax_fwd_path": (_int, [_p, _p, _i64, _i64, _p, _int]),
     "ak_xent_fwd": (_int, [_p, _p, _i64, _p, _p, _i64, _i64, _p]),
@@ -49,6 +52,7 @@ SIGNATURES = {
     "ak_sol_copy": (_int, [_p, _p, _sz, _p]),
     "ak_sol_read": (_int, [_p, _sz, _p, _p]),
     "ak_rmsnorm_choose_path": (_int, [_i64, _i64, _int]),
+    "ak_layernorm_choose_path": (_int, [_i64, _i64, _int]),
     "ak_softmax_choose_path": (_int, [_i64, _i64, _int]),
     "ak_xent_choose_path": (_int, [_i64, _i64, ctypes.POINTER(_int)]),
     "ak_launch_count": (_i64, []),
@@ -122,6 +126,36 @@ def ak_rmsnorm_fwd(x: torch.Tensor, w: torch.Tensor, y: Optional[torch.Tensor] =
     _check(lib().ak_rmsnorm_fwd_path(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, D, eps,
                                      _stream_ptr(stream), path), "ak_rmsnorm_fwd")
     return y
+
+
+def ak_layernorm_fwd(x: torch.Tensor, gamma: torch.Tensor, beta: torch.Tensor,
+                     y: Optional[torch.Tensor] = None, eps: float = 1e-5, stream=None,
+                     path: int = AK_PATH_AUTO) -> torch.Tensor:
+    _dev_bf16(x, "x", 2)
+    _dev_bf16(gamma, "gamma", 1)
+    _dev_bf16(beta, "beta", 1)
+    rows, D = x.shape
+    if gamma.shape[0] != D or beta.shape[0] != D:
+        raise ValueError("gamma and beta must have D elements")
+    if y is None:
+        y = torch.empty_like(x)
+    _dev_bf16(y, "y", 2)
+    if y.shape != x.shape:
+        raise ValueError("y must have the shape of x")
+    _check(lib().ak_layernorm_fwd_path(x.data_ptr(), gamma.data_ptr(), beta.data_ptr(), y.data_ptr(),
+                                       rows, D, eps, _stream_ptr(stream), path), "ak_layernorm_fwd")
+    return y
+
+
+def ak_rowsum_fwd(x: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    _dev_bf16(x, "x", 2)
+    rows, D = x.shape
+    if out is None:
+        out = torch.empty((rows,), dtype=torch.float32, device=x.device)
+    if not (out.is_cuda and out.dtype == torch.float32 and out.shape == (rows,) and out.is_contiguous()):
+        raise TypeError("out must be a contiguous CUDA float32 tensor [rows]")
+    _check(lib().ak_rowsum_fwd(x.data_ptr(), out.data_ptr(), rows, D, _stream_ptr(stream)), "ak_rowsum_fwd")
+    return out
 
 
 def ak_softmax_fwd(x: torch.Tensor, y: Optional[torch.Tensor] = None, stream=None,
@@ -241,6 +275,10 @@ def ak_xent_fwd_host(logits: torch.Tensor, targets: torch.Tensor, loss_rows: tor
 # ------------------------------------------------------------------------- introspection
 def ak_rmsnorm_choose_path(rows: int, D: int, aligned16: bool = True) -> int:
     return int(lib().ak_rmsnorm_choose_path(rows, D, int(aligned16)))
+
+
+def ak_layernorm_choose_path(rows: int, D: int, aligned16: bool = True) -> int:
+    return int(lib().ak_layernorm_choose_path(rows, D, int(aligned16)))
 
 
 def ak_softmax_choose_path(rows: int, D: int, aligned16: bool = True) -> int:

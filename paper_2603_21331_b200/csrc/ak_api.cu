@@ -85,6 +85,28 @@ int ak_rmsnorm_fwd(const void* x, const void* w, void* y, int64_t rows, int64_t 
     return ak_rmsnorm_fwd_path(x, w, y, rows, D, eps, cuda_stream, AK_PATH_AUTO);
 }
 
+int ak_layernorm_fwd_path(const void* x, const void* gamma, const void* beta, void* y, int64_t rows, int64_t D,
+                          float eps, void* cuda_stream, int path) {
+    if (int s = validate_rmsnorm(x, gamma, y, rows, D, eps)) return s;
+    if (rows != 0 && !beta) return AK_ERR_NULL;
+    if (!is_aligned(beta, 2)) return AK_ERR_ALIGN;
+    if (path < AK_PATH_AUTO || path > AK_PATH_SMEM) return AK_ERR_ARG;
+    if (rows == 0) return AK_OK;
+    return layernorm_dispatch(x, gamma, beta, y, rows, D, eps, static_cast<cudaStream_t>(cuda_stream), path);
+}
+int ak_layernorm_fwd(const void* x, const void* gamma, const void* beta, void* y, int64_t rows, int64_t D,
+                     float eps, void* cuda_stream) {
+    return ak_layernorm_fwd_path(x, gamma, beta, y, rows, D, eps, cuda_stream, AK_PATH_AUTO);
+}
+
+int ak_rowsum_fwd(const void* x, float* out, int64_t rows, int64_t D, void* cuda_stream) {
+    if (rows != 0 && (!x || !out)) return AK_ERR_NULL;
+    if (int s = check_rows_cols(rows, D)) return s;
+    if (!is_aligned(x, 2) || !is_aligned(out, 4)) return AK_ERR_ALIGN;
+    if (rows == 0) return AK_OK;
+    return rowsum_dispatch(x, out, rows, D, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int ak_softmax_fwd_path(const void* x, void* y, int64_t rows, int64_t D, void* cuda_stream, int path) {
     if (int s = validate_softmax(x, y, rows, D)) return s;
     if (path < AK_PATH_AUTO || path > AK_PATH_SMEM) return AK_ERR_ARG;
@@ -148,6 +170,9 @@ int ak_xent_mean_merge(const double* sum_count_pairs, int64_t n, float* loss_mea
 
 int ak_rmsnorm_choose_path(int64_t rows, int64_t D, int aligned16) {
     return rmsnorm_choose(rows, D, aligned16 != 0);
+}
+int ak_layernorm_choose_path(int64_t rows, int64_t D, int aligned16) {
+    return layernorm_choose(rows, D, aligned16 != 0);
 }
 int ak_softmax_choose_path(int64_t rows, int64_t D, int aligned16) {
     return softmax_choose(rows, D, aligned16 != 0);

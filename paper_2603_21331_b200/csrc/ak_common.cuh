@@ -196,6 +196,10 @@ int xent_mean_launch(const float* loss_rows, const int64_t* targets, int64_t ign
 int xent_sum_count_launch(const float* loss_rows, const int64_t* targets, int64_t ignore_index, int64_t rows,
                           double* sum_count, cudaStream_t st);
 int xent_mean_merge_launch(const double* pairs, int64_t n, float* loss_mean, cudaStream_t st);
+int layernorm_dispatch(const void* x, const void* gamma, const void* beta, void* y, int64_t rows, int64_t D,
+                       float eps, cudaStream_t st, int path);
+int layernorm_choose(int64_t rows, int64_t D, bool aligned16);
+int rowsum_dispatch(const void* x, float* out, int64_t rows, int64_t D, cudaStream_t st);
 int rmsnorm_choose(int64_t rows, int64_t D, bool aligned16);
 int softmax_choose(int64_t rows, int64_t D, bool aligned16);
 int xent_choose(int64_t rows, int64_t V, int* nsplit);

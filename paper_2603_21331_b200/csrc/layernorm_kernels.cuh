@@ -1,0 +1,269 @@
+// LayerNorm forward device kernels (paper Table 3 "layernorm"; Table 4 rows "layernorm").
+//
+//   mu = mean_k x[r, k];  var = mean_k (x[r, k] - mu)^2  (biased);
+//   y[r, j] = bf16_rne( (x[r, j] - mu) * rsqrt(var + eps) * gamma[j] + beta[j] )
+//
+// The paper's kernel is a single-pass Welford.  Here the row already sits in registers (or
+// shared memory) after its one trip from HBM, so the moments are taken in two exact-order
+// passes over that copy, which is both simpler and more accurate: first the mean, computed
+// as K + mean(x - K) with K the row's first element (for a constant row every difference is
+// exactly zero and mu == K exactly; in general the partial sums stay small, so fp32 does not
+// lose the low bits of large activations), then the sum of squared deviations from mu.
+// One DRAM read and one DRAM write per element.  Differences x - K and x - mu come straight
+// from the packed bf16 halves with the mixed-precision subtract (no widening instruction).
+#pragma once
+
+#include "ak_common.cuh"
+
+namespace ak {
+
+__device__ __forceinline__ void ln_halves(uint32_t u, uint16_t& lo, uint16_t& hi) {
+    asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(u));
+}
+// x - c with x a bf16 half: exact operand, one rounding
+__device__ __forceinline__ float sub_bf16(uint16_t x, float c) {
+    float d;
+    asm("sub.rn.f32.bf16 %0, %1, %2;" : "=f"(d) : "h"(x), "f"(c));
+    return d;
+}
+__device__ __forceinline__ f32x2 dev2(uint32_t u, float c) {
+    uint16_t lo, hi;
+    ln_halves(u, lo, hi);
+    return pack2(sub_bf16(lo, c), sub_bf16(hi, c));
+}
+// sum over the 8 elements of (x - c)
+__device__ __forceinline__ float sumdev8(const uint4& v, float c) {
+    float lo, hi;
+    unpack2(add2(add2(dev2(v.x, c), dev2(v.y, c)), add2(dev2(v.z, c), dev2(v.w, c))), lo, hi);
+    return lo + hi;
+}
+// sum over the 8 elements of (x - c)^2
+__device__ __forceinline__ float sqdev8(const uint4& v, float c) {
+    const f32x2 a = dev2(v.x, c), b = dev2(v.y, c), d = dev2(v.z, c), e = dev2(v.w, c);
+    f32x2 s = mul2(a, a);
+    s = fma2(b, b, s);
+    s = fma2(d, d, s);
+    s = fma2(e, e, s);
+    float lo, hi;
+    unpack2(s, lo, hi);
+    return lo + hi;
+}
+// ((x - mu) * rstd) * gamma + beta for one packed pair, rounded once to bf16
+__device__ __forceinline__ uint32_t ln_out2(uint32_t x, uint32_t g, uint32_t b, float mu, f32x2 rstd2) {
+    const f32x2 t = fma2(mul2(dev2(x, mu), rstd2), widen2(g), widen2(b));
+    float lo, hi;
+    unpack2(t, lo, hi);
+    return pack_bf16x2(lo, hi);
+}
+__device__ __forceinline__ uint4 ln_out8(const uint4& x, const uint4& g, const uint4& b, float mu, float rstd) {
+    const f32x2 r2 = pack2(rstd, rstd);
+    return make_uint4(ln_out2(x.x, g.x, b.x, mu, r2), ln_out2(x.y, g.y, b.y, mu, r2),
+                      ln_out2(x.z, g.z, b.z, mu, r2), ln_out2(x.w, g.w, b.w, mu, r2));
+}
+__device__ __forceinline__ float ln_out1(uint16_t x, uint16_t g, uint16_t b, float mu, float rstd) {
+    return fmaf(sub_bf16(x, mu) * rstd, bf16_to_float(g), bf16_to_float(b));
+}
+
+// ------------------------------------------------------------------ row in registers
+// Same thread layout as the RMSNorm register kernel (a group of GROUP threads owns a row,
+// thread t holds vectors t, t + GROUP, ...), two reductions per row.  Padding slots hold
+// copies of K so they add exactly zero to the first sum and are excluded from the second.
+template <int THREADS, int GROUP, int VPT, int MINB>
+__global__ void __launch_bounds__(THREADS, MINB)
+layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamma, const uint4* __restrict__ beta,
+                     uint4* __restrict__ y, int64_t rows, int nvec, float inv_D, float eps) {
+    constexpr int GROUPS = THREADS / GROUP;
+    constexpr int WARPS_PER_GROUP = GROUP / kWarp;
+    static_assert(GROUP % kWarp == 0 && THREADS % GROUP == 0, "groups are whole warps");
+    __shared__ float slots[2][THREADS / kWarp];
+    const int g = threadIdx.x / GROUP;
+    const int t = threadIdx.x % GROUP;
+    const int lane = threadIdx.x & 31;
+    const int warp_in_group = t >> 5;
+
+    for (int64_t row0 = (int64_t)blockIdx.x * GROUPS; row0 < rows; row0 += (int64_t)gridDim.x * GROUPS) {
+        const int64_t row = row0 + g;
+        const bool live = row < rows;
+        const uint4* xr = x + row * nvec;
+        const float K = live ? bf16_to_float(__ldg(reinterpret_cast<const uint16_t*>(xr))) : 0.0f;
+        uint4 xv[VPT];
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            const int i = t + k * GROUP;
+            if (live && i < nvec) xv[k] = ld_stream(xr + i);
+        }
+        float s1 = 0.0f;
+#pragma unroll
+        for (int k = 0; k < VPT; ++k)
+            if (live && t + k * GROUP < nvec) s1 += sumdev8(xv[k], K);
+        s1 = warp_sum(s1);
+        if constexpr (WARPS_PER_GROUP > 1) {
+            float* s = slots[0] + g * WARPS_PER_GROUP;
+            if (lane == 0) s[warp_in_group] = s1;
+            __syncthreads();
+            s1 = warp_sum((lane < WARPS_PER_GROUP) ? s[lane] : 0.0f);
+        }
+        const float mu = fmaf(s1, inv_D, K);
+        float s2 = 0.0f;
+#pragma unroll
+        for (int k = 0; k < VPT; ++k)
+            if (live && t + k * GROUP < nvec) s2 += sqdev8(xv[k], mu);
+        s2 = warp_sum(s2);
+        if constexpr (WARPS_PER_GROUP > 1) {
+            float* s = slots[1] + g * WARPS_PER_GROUP;
+            if (lane == 0) s[warp_in_group] = s2;
+            __syncthreads();
+            s2 = warp_sum((lane < WARPS_PER_GROUP) ? s[lane] : 0.0f);
+        }
+        const float rstd = rsqrtf(fmaf(s2, inv_D, eps));
+        uint4* yr = y + row * nvec;
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            const int i = t + k * GROUP;
+            if (live && i < nvec) st_stream(yr + i, ln_out8(xv[k], __ldg(gamma + i), __ldg(beta + i), mu, rstd));
+        }
+    }
+}
+
+// ------------------------------------------------------------------ long rows staged in shared memory
+// One CTA per row; the row is brought into shared memory by bulk (TMA) copies counted in by
+// one mbarrier, then read three times from there.  Needs 16-byte aligned rows (D % 8 == 0).
+// Dynamic shared memory = nvec * 16 bytes.
+constexpr uint32_t kLnBulkChunk = 32768;
+
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS, 1)
+layernorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamma, const uint4* __restrict__ beta,
+                      uint4* __restrict__ y, int nvec, float inv_D, float eps) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const uint4* row = reinterpret_cast<const uint4*>(smem_raw);
+    __shared__ uint64_t bar;
+    __shared__ float slots[2 * kWarp];
+    const int64_t r = blockIdx.x;
+    if (threadIdx.x == 0) mbar_init(&bar, 1);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const uint32_t bytes = (uint32_t)nvec * 16u;
+        mbar_expect_tx(&bar, bytes);
+        const unsigned char* src = reinterpret_cast<const unsigned char*>(x + r * nvec);
+        for (uint32_t off = 0; off < bytes; off += kLnBulkChunk)
+            bulk_load(smem_raw + off, src + off, min(kLnBulkChunk, bytes - off), &bar);
+    }
+    if (!mbar_wait(&bar, 0)) return;  // uniform: every thread waits on the same barrier
+    const float K = bf16_to_float(reinterpret_cast<const uint16_t*>(smem_raw)[0]);
+    float s1 = 0.0f;
+#pragma unroll 4
+    for (int i = threadIdx.x; i < nvec; i += THREADS) s1 += sumdev8(row[i], K);
+    s1 = cta_sum<THREADS>(s1, slots, 0);
+    const float mu = fmaf(s1, inv_D, K);
+    float s2 = 0.0f;
+#pragma unroll 4
+    for (int i = threadIdx.x; i < nvec; i += THREADS) s2 += sqdev8(row[i], mu);
+    s2 = cta_sum<THREADS>(s2, slots, 1);
+    const float rstd = rsqrtf(fmaf(s2, inv_D, eps));
+    uint4* yr = y + r * nvec;
+#pragma unroll 2
+    for (int i = threadIdx.x; i < nvec; i += THREADS)
+        st_stream(yr + i, ln_out8(row[i], __ldg(gamma + i), __ldg(beta + i), mu, rstd));
+}
+
+// ------------------------------------------------------------------ unaligned rows staged in shared memory
+// D % 8 != 0 (or a misaligned base): one CTA per row copies the row into shared memory in the
+// 16-byte phase it has in global memory, so interior vectors are aligned 16-byte loads and
+// (x and y rows sharing the phase) aligned 16-byte stores; the at most two edge vectors are
+// handled element by element by 16 threads, so nothing outside the row is read or written and
+// the padding never enters a sum.  gamma and beta for an interior vector start at element
+// 8k - phase: 4-byte loads plus funnel shifts.  Needs gamma and beta 4-byte aligned.
+__device__ __forceinline__ uint4 ln_load_shifted(const uint16_t* __restrict__ p, int64_t j0) {
+    const uint32_t* pw = reinterpret_cast<const uint32_t*>(p) + (j0 >> 1);
+    if ((j0 & 1) == 0) return make_uint4(__ldg(pw), __ldg(pw + 1), __ldg(pw + 2), __ldg(pw + 3));
+    // odd start: the fifth word would reach past element j0 + 7; fetch only its low half
+    const uint32_t a = __ldg(pw), b = __ldg(pw + 1), c = __ldg(pw + 2), d = __ldg(pw + 3);
+    const uint32_t e = (uint32_t)__ldg(p + j0 + 7);
+    return make_uint4(__funnelshift_r(a, b, 16), __funnelshift_r(b, c, 16), __funnelshift_r(c, d, 16),
+                      __funnelshift_r(d, e, 16));
+}
+
+template <int T>
+__global__ void __launch_bounds__(T)
+layernorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ gamma,
+                       const uint16_t* __restrict__ beta, uint16_t* __restrict__ y, int64_t D, float inv_D,
+                       float eps) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    uint4* row = reinterpret_cast<uint4*>(smem_raw);
+    uint16_t* row16 = reinterpret_cast<uint16_t*>(smem_raw);
+    __shared__ float slots[2 * kWarp];
+    const int64_t r = blockIdx.x;
+    const uint16_t* xr = x + r * D;
+    uint16_t* yr = y + r * D;
+    const int phase = (int)((reinterpret_cast<uintptr_t>(xr) >> 1) & 7);
+    const int nv = (int)((phase + D + 7) >> 3);
+    const int k_lo = phase ? 1 : 0;                      // first fully-inside vector
+    const int k_hi = ((phase + D) & 7) ? nv - 1 : nv;    // one past the last fully-inside vector
+    const uint4* xa = reinterpret_cast<const uint4*>(xr - phase);
+    uint4* ya = reinterpret_cast<uint4*>(yr - phase);
+
+    // edge element owned by this thread (threads 0..7: first vector, 8..15: last vector)
+    const int ek = (threadIdx.x < 8) ? 0 : nv - 1;
+    const bool is_edge_vec = (threadIdx.x < 8) ? (k_lo == 1) : (k_hi == nv - 1 && !(nv == 1 && k_lo == 1));
+    const int64_t ej = (int64_t)ek * 8 - phase + (threadIdx.x & 7);
+    const bool edge = threadIdx.x < 16 && is_edge_vec && ej >= 0 && ej < D;
+
+    for (int k = k_lo + threadIdx.x; k < k_hi; k += T) row[k] = ld_stream(xa + k);
+    if (edge) row16[ek * 8 + (threadIdx.x & 7)] = ld_stream_u16(xr + ej);
+    __syncthreads();
+    const float K = bf16_to_float(row16[phase]);
+    float s1 = 0.0f;
+    for (int k = k_lo + threadIdx.x; k < k_hi; k += T) s1 += sumdev8(row[k], K);
+    if (edge) s1 += sub_bf16(row16[ek * 8 + (threadIdx.x & 7)], K);
+    s1 = cta_sum<T>(s1, slots, 0);
+    const float mu = fmaf(s1, inv_D, K);
+    float s2 = 0.0f;
+    for (int k = k_lo + threadIdx.x; k < k_hi; k += T) s2 += sqdev8(row[k], mu);
+    if (edge) {
+        const float d = sub_bf16(row16[ek * 8 + (threadIdx.x & 7)], mu);
+        s2 = fmaf(d, d, s2);
+    }
+    s2 = cta_sum<T>(s2, slots, 1);
+    const float rstd = rsqrtf(fmaf(s2, inv_D, eps));
+    for (int k = k_lo + threadIdx.x; k < k_hi; k += T) {
+        const int64_t j0 = (int64_t)k * 8 - phase;
+        st_stream(ya + k, ln_out8(row[k], ln_load_shifted(gamma, j0), ln_load_shifted(beta, j0), mu, rstd));
+    }
+    if (edge)
+        yr[ej] = float_to_bf16(ln_out1(row16[ek * 8 + (threadIdx.x & 7)], __ldg(gamma + ej), __ldg(beta + ej), mu, rstd));
+}
+
+// ------------------------------------------------------------------ generic
+// Any D and any 2-byte alignment: element-wise 2-byte accesses, three passes over the row
+// (the second and third are served by L1/L2).  The slow, always-correct fallback; aligned
+// shapes never reach it.
+constexpr int kLnGenericThreads = 256;
+
+__global__ void __launch_bounds__(kLnGenericThreads)
+layernorm_generic_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ gamma,
+                         const uint16_t* __restrict__ beta, uint16_t* __restrict__ y, int64_t rows, int64_t D,
+                         float inv_D, float eps) {
+    constexpr int T = kLnGenericThreads;
+    __shared__ float slots[2 * kWarp];
+    for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+        const uint16_t* xr = x + row * D;
+        uint16_t* yr = y + row * D;
+        const float K = bf16_to_float(xr[0]);
+        float s1 = 0.0f;
+        for (int64_t j = threadIdx.x; j < D; j += T) s1 += sub_bf16(xr[j], K);
+        s1 = cta_sum<T>(s1, slots, 0);
+        const float mu = fmaf(s1, inv_D, K);
+        float s2 = 0.0f;
+        for (int64_t j = threadIdx.x; j < D; j += T) {
+            const float d = sub_bf16(xr[j], mu);
+            s2 = fmaf(d, d, s2);
+        }
+        s2 = cta_sum<T>(s2, slots, 1);
+        const float rstd = rsqrtf(fmaf(s2, inv_D, eps));
+        for (int64_t j = threadIdx.x; j < D; j += T)
+            yr[j] = float_to_bf16(ln_out1(xr[j], __ldg(gamma + j), __ldg(beta + j), mu, rstd));
+    }
+}
+
+}  // namespace ak

@@ -50,6 +50,21 @@ def test_validation_rejects_before_any_cuda_call():
     assert l.ak_rmsnorm_fwd_path(P, P, P, 1, 8, 1e-6, None, 9) == 4
     assert l.ak_rmsnorm_fwd(P, P, P, 0, 8, 1e-6, None) == 0          # rows == 0: nothing to do
     assert l.ak_rmsnorm_fwd(P, P, P, 1 << 40, 1 << 40, 1e-6, None) == 2
+    assert l.ak_layernorm_fwd(None, P, P, P, 1, 8, 1e-5, None) == 1
+    assert l.ak_layernorm_fwd(P, None, P, P, 1, 8, 1e-5, None) == 1
+    assert l.ak_layernorm_fwd(P, P, None, P, 1, 8, 1e-5, None) == 1
+    assert l.ak_layernorm_fwd(P, P, P, None, 1, 8, 1e-5, None) == 1
+    assert l.ak_layernorm_fwd(P, P, P, P, 1, 0, 1e-5, None) == 2
+    assert l.ak_layernorm_fwd(P, P, P + 1, P, 1, 8, 1e-5, None) == 3
+    assert l.ak_layernorm_fwd(P, P, P, P, 1, 8, -1e-5, None) == 4
+    assert l.ak_layernorm_fwd_path(P, P, P, P, 1, 8, 1e-5, None, 5) == 4
+    assert l.ak_layernorm_fwd(P, P, P, P, 0, 8, 1e-5, None) == 0
+    assert l.ak_rowsum_fwd(None, P, 1, 8, None) == 1
+    assert l.ak_rowsum_fwd(P, None, 1, 8, None) == 1
+    assert l.ak_rowsum_fwd(P, P, 1, 0, None) == 2
+    assert l.ak_rowsum_fwd(P + 1, P, 1, 8, None) == 3
+    assert l.ak_rowsum_fwd(P, P + 2, 1, 8, None) == 3                # fp32 sums need 4 B
+    assert l.ak_rowsum_fwd(P, P, 0, 8, None) == 0
     assert l.ak_softmax_fwd(None, P, 1, 8, None) == 1
     assert l.ak_softmax_fwd(P, P, 1, -3, None) == 2
     assert l.ak_softmax_fwd(P, P + 1, 1, 8, None) == 3
