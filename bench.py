@@ -496,7 +496,7 @@ SWEEP = (
     + [("xent", 4096, v) for v in (32000, 50304, 128256, 128257)] + [("xent", 16384, 128256), ("xent", 16, 128256)]
     + [("layernorm", 8192, 4096), ("layernorm", 4096, 5120), ("layernorm", 8192, 8192), ("layernorm", 65536, 4096),
        ("layernorm", 4096, 32768), ("layernorm", 8192, 4099)]
-    + [("rowsum", 8192, 4096), ("rowsum", 8192, 8192), ("rowsum", 65536, 1024), ("rowsum", 65536, 8192),
+    + [("rowsum", 8192, 4096), ("rowsum", 16384, 4096), ("rowsum", 8192, 8192), ("rowsum", 65536, 1024), ("rowsum", 65536, 8192),
        ("rowsum", 4096, 128256), ("rowsum", 8192, 4099)]
 )
 

@@ -21,18 +21,20 @@ int launch_reg(const void* x, const void* g, const void* b, void* y, int64_t row
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
-template <int THREADS, int GROUP, int MINB_LO, int MINB_HI>
+// vectors per thread 1..8 for a fixed (THREADS, GROUP); the minimum-CTAs-per-SM hint (a register
+// cap) is given per vector count: M14 for 1..4 vectors, M56 for 5..6, M7 and M8 for 7 and 8
+template <int THREADS, int GROUP, int M14, int M56, int M7, int M8>
 int launch_reg_vpt(int vpt, const void* x, const void* g, const void* b, void* y, int64_t rows, int nvec,
                    float inv_D, float eps, cudaStream_t st) {
     switch (vpt) {
-        case 1: return launch_reg<THREADS, GROUP, 1, MINB_LO>(x, g, b, y, rows, nvec, inv_D, eps, st);
-        case 2: return launch_reg<THREADS, GROUP, 2, MINB_LO>(x, g, b, y, rows, nvec, inv_D, eps, st);
-        case 3: return launch_reg<THREADS, GROUP, 3, MINB_LO>(x, g, b, y, rows, nvec, inv_D, eps, st);
-        case 4: return launch_reg<THREADS, GROUP, 4, MINB_LO>(x, g, b, y, rows, nvec, inv_D, eps, st);
-        case 5: return launch_reg<THREADS, GROUP, 5, MINB_HI>(x, g, b, y, rows, nvec, inv_D, eps, st);
-        case 6: return launch_reg<THREADS, GROUP, 6, MINB_HI>(x, g, b, y, rows, nvec, inv_D, eps, st);
-        case 7: return launch_reg<THREADS, GROUP, 7, MINB_HI>(x, g, b, y, rows, nvec, inv_D, eps, st);
-        case 8: return launch_reg<THREADS, GROUP, 8, MINB_HI>(x, g, b, y, rows, nvec, inv_D, eps, st);
+        case 1: return launch_reg<THREADS, GROUP, 1, M14>(x, g, b, y, rows, nvec, inv_D, eps, st);
+        case 2: return launch_reg<THREADS, GROUP, 2, M14>(x, g, b, y, rows, nvec, inv_D, eps, st);
+        case 3: return launch_reg<THREADS, GROUP, 3, M14>(x, g, b, y, rows, nvec, inv_D, eps, st);
+        case 4: return launch_reg<THREADS, GROUP, 4, M14>(x, g, b, y, rows, nvec, inv_D, eps, st);
+        case 5: return launch_reg<THREADS, GROUP, 5, M56>(x, g, b, y, rows, nvec, inv_D, eps, st);
+        case 6: return launch_reg<THREADS, GROUP, 6, M56>(x, g, b, y, rows, nvec, inv_D, eps, st);
+        case 7: return launch_reg<THREADS, GROUP, 7, M7>(x, g, b, y, rows, nvec, inv_D, eps, st);
+        case 8: return launch_reg<THREADS, GROUP, 8, M8>(x, g, b, y, rows, nvec, inv_D, eps, st);
         default: return AK_ERR_SHAPE;
     }
 }
@@ -88,18 +90,21 @@ int layernorm_dispatch(const void* x, const void* gamma, const void* beta, void*
     if (rows > 2147483647LL) return AK_ERR_SHAPE;  // grid.x limit of the one-row-per-CTA layouts
     const int nvec = (int)(D >> 3);
     switch (path) {
+        // Launch shapes and register caps below were picked by timing each candidate in the
+        // sustained (power-capped) regime of a long run.
         case AK_PATH_WARP:
             if (D > 2048) return AK_ERR_SHAPE;
-            if (nvec <= 128)
-                return launch_reg_vpt<256, 32, 4, 1>((nvec + 31) / 32, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
-            return launch_reg_vpt<128, 32, 1, 1>((nvec + 31) / 32, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
+            if (nvec <= 128)   // a warp per row, 8 rows per CTA, 46 registers
+                return launch_reg_vpt<256, 32, 5, 1, 1, 1>((nvec + 31) / 32, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
+            // two warps per row, 4 rows per CTA
+            return launch_reg_vpt<256, 64, 5, 1, 1, 1>((nvec + 63) / 64, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
         case AK_PATH_CTA:
             if (D > 32768) return AK_ERR_SHAPE;
-            if (nvec <= 512)
-                return launch_reg_vpt<128, 128, 1, 1>((nvec + 127) / 128, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
+            if (nvec <= 1024)  // 128 threads x up to 8 vectors: many small CTAs per SM
+                return launch_reg_vpt<128, 128, 10, 8, 6, 8>((nvec + 127) / 128, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
             if (nvec <= 2048)
-                return launch_reg_vpt<256, 256, 1, 3>((nvec + 255) / 256, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
-            return launch_reg_vpt<512, 512, 1, 1>((nvec + 511) / 512, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
+                return launch_reg_vpt<256, 256, 5, 4, 4, 4>((nvec + 255) / 256, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
+            return launch_reg_vpt<512, 512, 1, 2, 2, 2>((nvec + 511) / 512, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
         case AK_PATH_SMEM:
             if (D * 2 > kMaxRowSmemBytes) return AK_ERR_SHAPE;
             if (nvec <= 4096) return launch_smem<256>(x, gamma, beta, y, rows, nvec, inv_D, eps, st);
