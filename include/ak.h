@@ -59,6 +59,12 @@ enum {
     AK_PATH_GENERIC = 3,  /* any D, any 2-byte alignment; row re-read from L1/L2, single DRAM pass */
     AK_PATH_SMEM = 4      /* one CTA per row, row staged in shared memory by bulk (TMA) copies; D % 8 == 0, D <= 114688, 16 B aligned */
 };
+/* Element types of the *_dt entry points.  The plain entry points are bf16. */
+enum {
+    AK_DTYPE_BF16 = 0,
+    AK_DTYPE_F16 = 1,     /* IEEE binary16 */
+    AK_DTYPE_F32 = 2
+};
 enum {
     AK_XENT_AUTO = 0,
     AK_XENT_ROW = 1,      /* one CTA streams a whole row (online max / sum-exp), loss written directly */
@@ -76,6 +82,29 @@ int ak_rmsnorm_fwd(const void* x, const void* w, void* y,
                    int64_t rows, int64_t D, float eps, void* cuda_stream);
 int ak_rmsnorm_fwd_path(const void* x, const void* w, void* y,
                         int64_t rows, int64_t D, float eps, void* cuda_stream, int path);
+
+/* ---------------------------------------------------------------------------------
+ * Element-type variants of the three ops (the paper measures in FP16 and its benchmark
+ * harness sweeps FP16 / BF16 / FP32: Section 6 and the Table 4 caption).  Same definitions
+ * as the bf16 entry points; `dtype` (AK_DTYPE_*) is the type of x, w, y / logits; losses
+ * stay fp32; accumulation is fp32; outputs are rounded once, to nearest even (fp32
+ * outputs carry the fp32 arithmetic's own rounding).  Pointers must be aligned to the
+ * element size; the fast paths need 16-byte aligned bases and rows that are a multiple of
+ * 16 bytes (D % 8 == 0 for 16-bit types, D % 4 == 0 for fp32); the path limits of AK_PATH_*
+ * scale with the row's BYTES (4 KiB / 64 KiB / 224 KiB).  fp16 outputs beyond 65504
+ * become inf, as the type dictates.  `path` (and `nsplit`) as in the *_path entry points;
+ * 0 = automatic.  An unknown dtype gives AK_ERR_ARG.
+ */
+int ak_rmsnorm_fwd_dt(const void* x, const void* w, void* y, int64_t rows, int64_t D, float eps,
+                      int dtype, void* cuda_stream, int path);
+int ak_softmax_fwd_dt(const void* x, void* y, int64_t rows, int64_t D,
+                      int dtype, void* cuda_stream, int path);
+int ak_xent_fwd_dt(const void* logits, const int64_t* targets, int64_t ignore_index,
+                   float* loss_rows, float* loss_mean, int64_t rows, int64_t V,
+                   int dtype, void* cuda_stream, int path, int nsplit);
+/* Path the dispatcher picks for op (0 = RMSNorm, 1 = softmax) at this shape, alignment and
+ * element type; -1 for an unknown op or dtype.  Pure function; no CUDA calls. */
+int ak_choose_path_dt(int op, int64_t rows, int64_t D, int aligned16, int dtype);
 
 /* ---------------------------------------------------------------------------------
  * LayerNorm forward (Table 3 "layernorm"; Table 4 rows "layernorm").

@@ -1,4 +1,4 @@
-"""fp64 CPU oracle for RMSNorm / softmax / cross-entropy forward (ctypes wrapper).
+"""fp64 CPU oracle for RMSNorm / LayerNorm / softmax / cross-entropy forward and row-sum (ctypes wrapper).
 
 TEST INFRASTRUCTURE, NOT THE PRODUCT: only the test-suite, the smoke check and the
 benchmark's CPU-baseline leg may import this package.  It shares nothing with the
@@ -6,11 +6,11 @@ CUDA library and never imports it.  All arithmetic lives in ``ak_oracle.c`` (pla
 double precision, the textbook definition of each op); this file only marshals numpy
 arrays.  Inputs are bf16 *bit patterns* (``uint16``); outputs are ``float64``.
 
-Ops follow Table 3 of the paper (softmax / rmsnorm / cross_ent rows) with the
+Ops follow Table 3 of the paper (softmax / rmsnorm / layernorm / cross_ent / reduce rows) with the
 semantics of the PyTorch reference implementation the paper names as its correctness
 oracle (Section 6).  Readings the paper does not pin ("parity unpinned", PyTorch
 convention): fully -inf softmax row -> NaN; inf/NaN inputs propagate; eps = 0 with a
-zero row -> NaN; all rows ignored -> mean NaN; out-of-range target -> NaN row.
+zero row -> NaN; inf/NaN in a LayerNorm row -> NaN row; all rows ignored -> mean NaN; out-of-range target -> NaN row.
 """
 from __future__ import annotations
 
@@ -35,6 +35,14 @@ def _load():
         lib.oracle_bf16_to_f64.restype = None
         lib.oracle_set_threads.argtypes = [ctypes.c_int]
         lib.oracle_set_threads.restype = ctypes.c_int
+        lib.oracle_f16_to_f64.argtypes = [p, p, i64]
+        lib.oracle_f16_to_f64.restype = None
+        lib.oracle_rmsnorm_dt.argtypes = [p, p, p, i64, i64, f32, ctypes.c_int]
+        lib.oracle_rmsnorm_dt.restype = None
+        lib.oracle_softmax_dt.argtypes = [p, p, i64, i64, ctypes.c_int]
+        lib.oracle_softmax_dt.restype = None
+        lib.oracle_xent_dt.argtypes = [p, p, i64, p, p, p, i64, i64, ctypes.c_int]
+        lib.oracle_xent_dt.restype = None
         lib.oracle_rmsnorm.argtypes = [p, p, p, i64, i64, f32]
         lib.oracle_rmsnorm.restype = None
         lib.oracle_layernorm.argtypes = [p, p, p, p, i64, i64, f32]
@@ -58,6 +66,20 @@ def _bits(a, shape=None) -> np.ndarray:
     return a
 
 
+DTYPES = {"bf16": 0, "f16": 1, "f32": 2}
+
+
+def _elems(a, dtype: str, shape=None) -> np.ndarray:
+    """Input array of element type ``dtype``: uint16 bit patterns for bf16 / f16, float32 for f32."""
+    a = np.ascontiguousarray(a)
+    want = np.float32 if dtype == "f32" else np.uint16
+    if a.dtype != want:
+        raise TypeError(f"{dtype} inputs must be {np.dtype(want)}, got {a.dtype}")
+    if shape is not None and a.shape != shape:
+        raise ValueError(f"expected shape {shape}, got {a.shape}")
+    return a
+
+
 def set_threads(n: int = 0) -> int:
     """Set (n > 0) or query (n = 0) the number of row-loop threads."""
     return int(_load().oracle_set_threads(int(n)))
@@ -69,6 +91,54 @@ def bf16_to_f64(bits) -> np.ndarray:
     out = np.empty(b.shape, dtype=np.float64)
     _load().oracle_bf16_to_f64(b.ctypes.data, out.ctypes.data, b.size)
     return out
+
+
+def f16_to_f64(bits) -> np.ndarray:
+    """Exact widening of IEEE binary16 bit patterns to float64."""
+    b = _bits(bits)
+    out = np.empty(b.shape, dtype=np.float64)
+    _load().oracle_f16_to_f64(b.ctypes.data, out.ctypes.data, b.size)
+    return out
+
+
+def rmsnorm_dt(x, w, eps: float, dtype: str) -> np.ndarray:
+    """RMSNorm on inputs of element type ``dtype`` ("bf16", "f16": uint16 bits; "f32": float32)."""
+    x = _elems(x, dtype)
+    if x.ndim != 2:
+        raise ValueError("x must be [rows, D]")
+    rows, D = x.shape
+    w = _elems(w, dtype, (D,))
+    y = np.empty((rows, D), dtype=np.float64)
+    _load().oracle_rmsnorm_dt(x.ctypes.data, w.ctypes.data, y.ctypes.data, rows, D,
+                              float(np.float32(eps)), DTYPES[dtype])
+    return y
+
+
+def softmax_dt(x, dtype: str) -> np.ndarray:
+    x = _elems(x, dtype)
+    if x.ndim != 2:
+        raise ValueError("x must be [rows, D]")
+    rows, D = x.shape
+    y = np.empty((rows, D), dtype=np.float64)
+    _load().oracle_softmax_dt(x.ctypes.data, y.ctypes.data, rows, D, DTYPES[dtype])
+    return y
+
+
+def xent_dt(logits, targets, dtype: str, ignore_index: int = -100):
+    """Returns (loss_rows float64 [rows], loss_mean float, n_counted int)."""
+    x = _elems(logits, dtype)
+    if x.ndim != 2:
+        raise ValueError("logits must be [rows, V]")
+    rows, V = x.shape
+    t = np.ascontiguousarray(targets)
+    if t.dtype != np.int64 or t.shape != (rows,):
+        raise TypeError("targets must be int64 [rows]")
+    loss = np.empty((rows,), dtype=np.float64)
+    mean = ctypes.c_double(float("nan"))
+    cnt = ctypes.c_int64(0)
+    _load().oracle_xent_dt(x.ctypes.data, t.ctypes.data, int(ignore_index), loss.ctypes.data,
+                           ctypes.addressof(mean), ctypes.addressof(cnt), rows, V, DTYPES[dtype])
+    return loss, float(mean.value), int(cnt.value)
 
 
 def rmsnorm(x_bits, w_bits, eps: float) -> np.ndarray:

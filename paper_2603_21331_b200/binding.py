@@ -25,6 +25,8 @@ LIB_PATH = os.path.join(_HERE, "libak.so")
 AK_OK = 0
 AK_PATH_AUTO, AK_PATH_WARP, AK_PATH_CTA, AK_PATH_GENERIC, AK_PATH_SMEM = 0, 1, 2, 3, 4
 AK_XENT_AUTO, AK_XENT_ROW, AK_XENT_SPLIT = 0, 1, 2
+AK_DTYPE_BF16, AK_DTYPE_F16, AK_DTYPE_F32 = 0, 1, 2
+_DTYPES = {torch.bfloat16: AK_DTYPE_BF16, torch.float16: AK_DTYPE_F16, torch.float32: AK_DTYPE_F32}
 
 _i64, _f32, _int, _p, _sz = (ctypes.c_int64, ctypes.c_float, ctypes.c_int, ctypes.c_void_p,
                              ctypes.c_size_t)
@@ -33,6 +35,10 @@ _i64, _f32, _int, _p, _sz = (ctypes.c_int64, ctypes.c_float, ctypes.c_int, ctype
 SIGNATURES = {
     "ak_rmsnorm_fwd": (_int, [_p, _p, _p, _i64, _i64, _f32, _p]),
     "ak_rmsnorm_fwd_path": (_int, [_p, _p, _p, _i64, _i64, _f32, _p, _int]),
+    "ak_rmsnorm_fwd_dt": (_int, [_p, _p, _p, _i64, _i64, _f32, _int, _p, _int]),
+    "ak_softmax_fwd_dt": (_int, [_p, _p, _i64, _i64, _int, _p, _int]),
+    "ak_xent_fwd_dt": (_int, [_p, _p, _i64, _p, _p, _i64, _i64, _int, _p, _int, _int]),
+    "ak_choose_path_dt": (_int, [_int, _i64, _i64, _int, _int]),
     "ak_layernorm_fwd": (_int, [_p, _p, _p, _p, _i64, _i64, _f32, _p]),
     "ak_layernorm_fwd_path": (_int, [_p, _p, _p, _p, _i64, _i64, _f32, _p, _int]),
     "ak_rowsum_fwd": (_int, [_p, _p, _i64, _i64, _p]),
@@ -126,6 +132,68 @@ def ak_rmsnorm_fwd(x: torch.Tensor, w: torch.Tensor, y: Optional[torch.Tensor] =
     _check(lib().ak_rmsnorm_fwd_path(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, D, eps,
                                      _stream_ptr(stream), path), "ak_rmsnorm_fwd")
     return y
+
+
+def _dev_dt(t: torch.Tensor, name: str, ndim: int, dtype=None) -> int:
+    want = t.dtype if dtype is None else dtype
+    if want not in _DTYPES or not (t.is_cuda and t.dtype == want and t.dim() == ndim and t.is_contiguous()):
+        raise TypeError(f"{name} must be a contiguous CUDA bf16 / fp16 / fp32 tensor with {ndim} dims"
+                        + ("" if dtype is None else f" of dtype {dtype}"))
+    return _DTYPES[want]
+
+
+def ak_rmsnorm_fwd_dt(x: torch.Tensor, w: torch.Tensor, y: Optional[torch.Tensor] = None,
+                      eps: float = 1e-6, stream=None, path: int = AK_PATH_AUTO) -> torch.Tensor:
+    """RMSNorm in the element type of x (bf16, fp16 or fp32); w and y share it."""
+    dt = _dev_dt(x, "x", 2)
+    _dev_dt(w, "w", 1, x.dtype)
+    rows, D = x.shape
+    if w.shape[0] != D:
+        raise ValueError("w must have D elements")
+    if y is None:
+        y = torch.empty_like(x)
+    _dev_dt(y, "y", 2, x.dtype)
+    if y.shape != x.shape:
+        raise ValueError("y must have the shape of x")
+    _check(lib().ak_rmsnorm_fwd_dt(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, D, eps, dt,
+                                   _stream_ptr(stream), path), "ak_rmsnorm_fwd_dt")
+    return y
+
+
+def ak_softmax_fwd_dt(x: torch.Tensor, y: Optional[torch.Tensor] = None, stream=None,
+                      path: int = AK_PATH_AUTO) -> torch.Tensor:
+    """Softmax over the last dim in the element type of x (bf16, fp16 or fp32)."""
+    dt = _dev_dt(x, "x", 2)
+    rows, D = x.shape
+    if y is None:
+        y = torch.empty_like(x)
+    _dev_dt(y, "y", 2, x.dtype)
+    if y.shape != x.shape:
+        raise ValueError("y must have the shape of x")
+    _check(lib().ak_softmax_fwd_dt(x.data_ptr(), y.data_ptr(), rows, D, dt, _stream_ptr(stream), path),
+           "ak_softmax_fwd_dt")
+    return y
+
+
+def ak_xent_fwd_dt(logits: torch.Tensor, targets: torch.Tensor, ignore_index: int = -100,
+                   stream=None, path: int = AK_XENT_AUTO, nsplit: int = 0,
+                   want_mean: bool = True) -> Tuple[torch.Tensor, Optional[torch.Tensor]]:
+    """Cross-entropy on logits of type bf16, fp16 or fp32; losses are fp32."""
+    dt = _dev_dt(logits, "logits", 2)
+    rows, V = logits.shape
+    if not (targets.is_cuda and targets.dtype == torch.int64 and targets.shape == (rows,)
+            and targets.is_contiguous()):
+        raise TypeError("targets must be a contiguous CUDA int64 tensor [rows]")
+    loss_rows = torch.empty((rows,), dtype=torch.float32, device=logits.device)
+    loss_mean = torch.empty((1,), dtype=torch.float32, device=logits.device) if want_mean else None
+    _check(lib().ak_xent_fwd_dt(logits.data_ptr(), targets.data_ptr(), ignore_index, loss_rows.data_ptr(),
+                                loss_mean.data_ptr() if want_mean else None, rows, V, dt,
+                                _stream_ptr(stream), path, nsplit), "ak_xent_fwd_dt")
+    return loss_rows, loss_mean
+
+
+def ak_choose_path_dt(op: str, rows: int, D: int, dtype: torch.dtype, aligned16: bool = True) -> int:
+    return int(lib().ak_choose_path_dt({"rmsnorm": 0, "softmax": 1}[op], rows, D, int(aligned16), _DTYPES[dtype]))
 
 
 def ak_layernorm_fwd(x: torch.Tensor, gamma: torch.Tensor, beta: torch.Tensor,

@@ -43,24 +43,26 @@ int check_rows_cols(int64_t rows, int64_t D) {
     return AK_OK;
 }
 
-int validate_rmsnorm(const void* x, const void* w, void* y, int64_t rows, int64_t D, float eps) {
+bool known_dtype(int dtype) { return dtype == AK_DTYPE_BF16 || dtype == AK_DTYPE_F16 || dtype == AK_DTYPE_F32; }
+
+int validate_rmsnorm(const void* x, const void* w, void* y, int64_t rows, int64_t D, float eps, size_t esize = 2) {
     if (rows != 0 && (!x || !w || !y)) return AK_ERR_NULL;  // an empty batch may carry NULL data pointers
     if (int s = check_rows_cols(rows, D)) return s;
-    if (!is_aligned(x, 2) || !is_aligned(w, 2) || !is_aligned(y, 2)) return AK_ERR_ALIGN;
+    if (!is_aligned(x, esize) || !is_aligned(w, esize) || !is_aligned(y, esize)) return AK_ERR_ALIGN;
     if (!(eps >= 0.0f) || !std::isfinite(eps)) return AK_ERR_ARG;
     return AK_OK;
 }
-int validate_softmax(const void* x, void* y, int64_t rows, int64_t D) {
+int validate_softmax(const void* x, void* y, int64_t rows, int64_t D, size_t esize = 2) {
     if (rows != 0 && (!x || !y)) return AK_ERR_NULL;
     if (int s = check_rows_cols(rows, D)) return s;
-    if (!is_aligned(x, 2) || !is_aligned(y, 2)) return AK_ERR_ALIGN;
+    if (!is_aligned(x, esize) || !is_aligned(y, esize)) return AK_ERR_ALIGN;
     return AK_OK;
 }
 int validate_xent(const void* logits, const int64_t* targets, float* loss_rows, float* loss_mean,
-                  int64_t rows, int64_t V) {
+                  int64_t rows, int64_t V, size_t esize = 2) {
     if (rows != 0 && (!logits || !targets || !loss_rows)) return AK_ERR_NULL;
     if (int s = check_rows_cols(rows, V)) return s;
-    if (!is_aligned(logits, 2) || !is_aligned(targets, 8) || !is_aligned(loss_rows, 4) ||
+    if (!is_aligned(logits, esize) || !is_aligned(targets, 8) || !is_aligned(loss_rows, 4) ||
         (loss_mean && !is_aligned(loss_mean, 4)))
         return AK_ERR_ALIGN;
     return AK_OK;
@@ -83,6 +85,36 @@ int ak_rmsnorm_fwd_path(const void* x, const void* w, void* y, int64_t rows, int
 int ak_rmsnorm_fwd(const void* x, const void* w, void* y, int64_t rows, int64_t D, float eps,
                    void* cuda_stream) {
     return ak_rmsnorm_fwd_path(x, w, y, rows, D, eps, cuda_stream, AK_PATH_AUTO);
+}
+
+int ak_rmsnorm_fwd_dt(const void* x, const void* w, void* y, int64_t rows, int64_t D, float eps, int dtype,
+                      void* cuda_stream, int path) {
+    if (!known_dtype(dtype)) return AK_ERR_ARG;
+    if (int s = validate_rmsnorm(x, w, y, rows, D, eps, (size_t)dtype_bytes(dtype))) return s;
+    if (path < AK_PATH_AUTO || path > AK_PATH_SMEM) return AK_ERR_ARG;
+    if (rows == 0) return AK_OK;
+    return rmsnorm_dispatch(x, w, y, rows, D, eps, static_cast<cudaStream_t>(cuda_stream), path, dtype);
+}
+int ak_softmax_fwd_dt(const void* x, void* y, int64_t rows, int64_t D, int dtype, void* cuda_stream, int path) {
+    if (!known_dtype(dtype)) return AK_ERR_ARG;
+    if (int s = validate_softmax(x, y, rows, D, (size_t)dtype_bytes(dtype))) return s;
+    if (path < AK_PATH_AUTO || path > AK_PATH_SMEM) return AK_ERR_ARG;
+    if (rows == 0) return AK_OK;
+    return softmax_dispatch(x, y, rows, D, static_cast<cudaStream_t>(cuda_stream), path, dtype);
+}
+int ak_xent_fwd_dt(const void* logits, const int64_t* targets, int64_t ignore_index, float* loss_rows,
+                   float* loss_mean, int64_t rows, int64_t V, int dtype, void* cuda_stream, int path, int nsplit) {
+    if (!known_dtype(dtype)) return AK_ERR_ARG;
+    if (int s = validate_xent(logits, targets, loss_rows, loss_mean, rows, V, (size_t)dtype_bytes(dtype))) return s;
+    if (path < AK_XENT_AUTO || path > AK_XENT_SPLIT || nsplit < 0 || nsplit > 64) return AK_ERR_ARG;
+    return xent_dispatch(logits, targets, ignore_index, loss_rows, loss_mean, rows, V, nullptr, 0, true,
+                         static_cast<cudaStream_t>(cuda_stream), path, nsplit, dtype);
+}
+int ak_choose_path_dt(int op, int64_t rows, int64_t D, int aligned16, int dtype) {
+    if (!known_dtype(dtype)) return -1;
+    if (op == 0) return rmsnorm_choose(rows, D, aligned16 != 0, dtype);
+    if (op == 1) return softmax_choose(rows, D, aligned16 != 0, dtype);
+    return -1;
 }
 
 int ak_layernorm_fwd_path(const void* x, const void* gamma, const void* beta, void* y, int64_t rows, int64_t D,
@@ -187,7 +219,7 @@ const char* ak_status_string(int status) {
         case AK_ERR_NULL: return "a required pointer is NULL";
         case AK_ERR_SHAPE: return "bad shape (rows < 0, D <= 0, or size not supported by the requested path)";
         case AK_ERR_ALIGN: return "pointer not sufficiently aligned";
-        case AK_ERR_ARG: return "bad scalar argument (eps, path id or nsplit)";
+        case AK_ERR_ARG: return "bad scalar argument (eps, path id, nsplit or dtype)";
         case AK_ERR_CUDA: return "CUDA runtime error";
         case AK_ERR_NOMEM: return "scratch memory unavailable or workspace too small";
         case AK_ERR_CAPACITY: return "problem exceeds the fixed scratch of the no-allocation entry point (rows * nsplit * 8 bytes > 1 MiB or rows > 65535)";

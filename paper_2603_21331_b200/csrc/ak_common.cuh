@@ -71,6 +71,76 @@ __device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
 // the two bf16 of a 32-bit word as a packed float pair (element 2i low, 2i+1 high)
 __device__ __forceinline__ f32x2 widen2(uint32_t u) { return pack2(bf16lo(u), bf16hi(u)); }
 
+// ---------------------------------------------------------------- element types
+// The kernels are written once over 16-byte vectors and take the element type as a template
+// parameter (an ak_dtype value): bf16 and fp16 put 8 elements in a vector (pairs packed in
+// 32-bit words, element 2i in the low half), fp32 puts 4.  Elem<DT> holds what differs for the
+// 16-bit types: widening (exact), rounding (nearest-even), the packed max and the packed -inf.
+template <int DT> struct Elem;
+template <> struct Elem<AK_DTYPE_BF16> {
+    static constexpr int kBytes = 2, kPerVec = 8;
+    static constexpr uint32_t kNegInf2 = 0xFF80FF80u;
+    static constexpr uint16_t kNegInf = 0xFF80;
+    static __device__ __forceinline__ float lo(uint32_t u) { return bf16lo(u); }
+    static __device__ __forceinline__ float hi(uint32_t u) { return bf16hi(u); }
+    static __device__ __forceinline__ float to_float(uint16_t b) { return bf16_to_float(b); }
+    static __device__ __forceinline__ uint32_t pack(float l, float h) { return pack_bf16x2(l, h); }
+    static __device__ __forceinline__ uint16_t from_float(float v) { return float_to_bf16(v); }
+    static __device__ __forceinline__ uint32_t max2(uint32_t a, uint32_t b) { return bf16x2_max(a, b); }
+    static __device__ __forceinline__ uint32_t max2_nan(uint32_t a, uint32_t b) {
+        uint32_t r;
+        asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+        return r;
+    }
+    static __device__ __forceinline__ float fma_h(uint16_t a, uint16_t b, float c) {  // a*b exact, + c, one rounding
+        float d;
+        asm("fma.rn.f32.bf16 %0, %1, %2, %3;" : "=f"(d) : "h"(a), "h"(b), "f"(c));
+        return d;
+    }
+};
+template <> struct Elem<AK_DTYPE_F16> {
+    static constexpr int kBytes = 2, kPerVec = 8;
+    static constexpr uint32_t kNegInf2 = 0xFC00FC00u;
+    static constexpr uint16_t kNegInf = 0xFC00;
+    static __device__ __forceinline__ float to_float(uint16_t b) {
+        float f;
+        asm("cvt.f32.f16 %0, %1;" : "=f"(f) : "h"(b));
+        return f;
+    }
+    static __device__ __forceinline__ float lo(uint32_t u) { return to_float((uint16_t)(u & 0xffffu)); }
+    static __device__ __forceinline__ float hi(uint32_t u) { return to_float((uint16_t)(u >> 16)); }
+    static __device__ __forceinline__ uint32_t pack(float l, float h) {
+        uint32_t r;
+        asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(h), "f"(l));
+        return r;
+    }
+    static __device__ __forceinline__ uint16_t from_float(float v) {
+        uint16_t r;
+        asm("cvt.rn.f16.f32 %0, %1;" : "=h"(r) : "f"(v));
+        return r;
+    }
+    static __device__ __forceinline__ uint32_t max2(uint32_t a, uint32_t b) {
+        uint32_t r;
+        asm("max.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+        return r;
+    }
+    static __device__ __forceinline__ uint32_t max2_nan(uint32_t a, uint32_t b) {
+        uint32_t r;
+        asm("max.NaN.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+        return r;
+    }
+    static __device__ __forceinline__ float fma_h(uint16_t a, uint16_t b, float c) {  // 11-bit x 11-bit: exact product
+        float d;
+        asm("fma.rn.f32.f16 %0, %1, %2, %3;" : "=f"(d) : "h"(a), "h"(b), "f"(c));
+        return d;
+    }
+};
+template <> struct Elem<AK_DTYPE_F32> {
+    static constexpr int kBytes = 4, kPerVec = 4;
+};
+template <int DT>
+__device__ __forceinline__ f32x2 widen2_t(uint32_t u) { return pack2(Elem<DT>::lo(u), Elem<DT>::hi(u)); }
+
 // ---------------------------------------------------------------- memory
 // Activations are touched exactly once: streaming (evict-first) loads and stores keep
 // them from displacing the reusable weight vector in L2/L1.
@@ -184,12 +254,13 @@ bool persistent_grid();
 // Per-op host dispatchers (each defined next to its kernels).  All arguments have been
 // validated; `path` is a concrete path id or AUTO.  They return an ak_status.
 int rmsnorm_dispatch(const void* x, const void* w, void* y, int64_t rows, int64_t D, float eps,
-                     cudaStream_t st, int path);
-int softmax_dispatch(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st, int path);
+                     cudaStream_t st, int path, int dtype = AK_DTYPE_BF16);
+int softmax_dispatch(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st, int path,
+                     int dtype = AK_DTYPE_BF16);
 int xent_dispatch(const void* logits, const int64_t* targets, int64_t ignore_index,
                   float* loss_rows, float* loss_mean, int64_t rows, int64_t V,
                   void* workspace, size_t workspace_bytes, bool may_allocate,
-                  cudaStream_t st, int path, int nsplit);
+                  cudaStream_t st, int path, int nsplit, int dtype = AK_DTYPE_BF16);
 // Fixed-order fp64 mean of loss_rows over rows whose target != ignore_index (one small launch).
 int xent_mean_launch(const float* loss_rows, const int64_t* targets, int64_t ignore_index, int64_t rows,
                      float* loss_mean, cudaStream_t st);
@@ -200,12 +271,13 @@ int layernorm_dispatch(const void* x, const void* gamma, const void* beta, void*
                        float eps, cudaStream_t st, int path);
 int layernorm_choose(int64_t rows, int64_t D, bool aligned16);
 int rowsum_dispatch(const void* x, float* out, int64_t rows, int64_t D, cudaStream_t st);
-int rmsnorm_choose(int64_t rows, int64_t D, bool aligned16);
-int softmax_choose(int64_t rows, int64_t D, bool aligned16);
+int rmsnorm_choose(int64_t rows, int64_t D, bool aligned16, int dtype = AK_DTYPE_BF16);
+int softmax_choose(int64_t rows, int64_t D, bool aligned16, int dtype = AK_DTYPE_BF16);
 int xent_choose(int64_t rows, int64_t V, int* nsplit);
 // CTA shape of the register-resident row paths: threads per CTA and 16-byte vectors per thread.
 void cta_shape(int nvec, int* threads, int* vpt);
 
+inline int dtype_bytes(int dtype) { return dtype == AK_DTYPE_F32 ? 4 : 2; }
 inline bool is_aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
 }  // namespace ak

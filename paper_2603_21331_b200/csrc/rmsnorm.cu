@@ -11,7 +11,7 @@
 namespace ak {
 namespace {
 
-template <int THREADS, int GROUP, int VPT, int MINB>
+template <int DT, int THREADS, int GROUP, int VPT, int MINB>
 int launch_reg(const void* x, const void* w, void* y, int64_t rows, int nvec, float inv_D, float eps,
                cudaStream_t st) {
     constexpr int GROUPS = THREADS / GROUP;
@@ -21,46 +21,46 @@ int launch_reg(const void* x, const void* w, void* y, int64_t rows, int nvec, fl
         static const int resident = [] {
             int per_sm = 0;
             if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-                    &per_sm, rmsnorm_reg_kernel<THREADS, GROUP, VPT, MINB, false>, THREADS, 0) != cudaSuccess ||
+                    &per_sm, rmsnorm_reg_kernel<THREADS, GROUP, VPT, MINB, false, DT>, THREADS, 0) != cudaSuccess ||
                 per_sm < 1)
                 per_sm = 1;
             return per_sm * sm_count();
         }();
         if (grid > resident) grid = resident;
     }
-    rmsnorm_reg_kernel<THREADS, GROUP, VPT, MINB, false><<<(unsigned)grid, THREADS, 0, st>>>(
+    rmsnorm_reg_kernel<THREADS, GROUP, VPT, MINB, false, DT><<<(unsigned)grid, THREADS, 0, st>>>(
         static_cast<const uint4*>(x), static_cast<const uint4*>(w), static_cast<uint4*>(y), rows, nvec, inv_D, eps);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
 // vectors per thread 1..MAXV for a fixed (THREADS, GROUP)
-template <int THREADS, int GROUP, int MINB_LO, int MINB_HI>
+template <int DT, int THREADS, int GROUP, int MINB_LO, int MINB_HI>
 int launch_reg_vpt(int vpt, const void* x, const void* w, void* y, int64_t rows, int nvec, float inv_D,
                    float eps, cudaStream_t st) {
     switch (vpt) {
-        case 1: return launch_reg<THREADS, GROUP, 1, MINB_LO>(x, w, y, rows, nvec, inv_D, eps, st);
-        case 2: return launch_reg<THREADS, GROUP, 2, MINB_LO>(x, w, y, rows, nvec, inv_D, eps, st);
-        case 3: return launch_reg<THREADS, GROUP, 3, MINB_LO>(x, w, y, rows, nvec, inv_D, eps, st);
-        case 4: return launch_reg<THREADS, GROUP, 4, MINB_LO>(x, w, y, rows, nvec, inv_D, eps, st);
-        case 5: return launch_reg<THREADS, GROUP, 5, MINB_HI>(x, w, y, rows, nvec, inv_D, eps, st);
-        case 6: return launch_reg<THREADS, GROUP, 6, MINB_HI>(x, w, y, rows, nvec, inv_D, eps, st);
-        case 7: return launch_reg<THREADS, GROUP, 7, MINB_HI>(x, w, y, rows, nvec, inv_D, eps, st);
-        case 8: return launch_reg<THREADS, GROUP, 8, MINB_HI>(x, w, y, rows, nvec, inv_D, eps, st);
+        case 1: return launch_reg<DT, THREADS, GROUP, 1, MINB_LO>(x, w, y, rows, nvec, inv_D, eps, st);
+        case 2: return launch_reg<DT, THREADS, GROUP, 2, MINB_LO>(x, w, y, rows, nvec, inv_D, eps, st);
+        case 3: return launch_reg<DT, THREADS, GROUP, 3, MINB_LO>(x, w, y, rows, nvec, inv_D, eps, st);
+        case 4: return launch_reg<DT, THREADS, GROUP, 4, MINB_LO>(x, w, y, rows, nvec, inv_D, eps, st);
+        case 5: return launch_reg<DT, THREADS, GROUP, 5, MINB_HI>(x, w, y, rows, nvec, inv_D, eps, st);
+        case 6: return launch_reg<DT, THREADS, GROUP, 6, MINB_HI>(x, w, y, rows, nvec, inv_D, eps, st);
+        case 7: return launch_reg<DT, THREADS, GROUP, 7, MINB_HI>(x, w, y, rows, nvec, inv_D, eps, st);
+        case 8: return launch_reg<DT, THREADS, GROUP, 8, MINB_HI>(x, w, y, rows, nvec, inv_D, eps, st);
         default: return AK_ERR_SHAPE;
     }
 }
 
-template <int THREADS>
+template <int DT, int THREADS>
 int launch_smem(const void* x, const void* w, void* y, int64_t rows, int nvec, float inv_D, float eps,
                 cudaStream_t st) {
     const size_t smem = (size_t)nvec * 16;
     static const bool configured = [] {
-        return cudaFuncSetAttribute(rmsnorm_smem_kernel<THREADS, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        return cudaFuncSetAttribute(rmsnorm_smem_kernel<THREADS, 1, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     kMaxRowSmemBytes) == cudaSuccess;
     }();
     if (!configured) return AK_ERR_CUDA;
-    rmsnorm_smem_kernel<THREADS, 1><<<(unsigned)rows, THREADS, smem, st>>>(
+    rmsnorm_smem_kernel<THREADS, 1, DT><<<(unsigned)rows, THREADS, smem, st>>>(
         static_cast<const uint4*>(x), static_cast<const uint4*>(w), static_cast<uint4*>(y), nvec, inv_D, eps);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
@@ -68,85 +68,115 @@ int launch_smem(const void* x, const void* w, void* y, int64_t rows, int nvec, f
 
 }  // namespace
 
-int rmsnorm_choose(int64_t rows, int64_t D, bool aligned16) {
+int rmsnorm_choose(int64_t rows, int64_t D, bool aligned16, int dtype) {
     (void)rows;
-    if (!aligned16 || (D & 7) != 0 || D * 2 > kMaxRowSmemBytes) return AK_PATH_GENERIC;
-    if (D <= 2048) return AK_PATH_WARP;
-    if (D <= 16384) return AK_PATH_CTA;
+    const int64_t bytes = D * dtype_bytes(dtype);   // row bytes decide the layout
+    if (!aligned16 || (bytes & 15) != 0 || bytes > kMaxRowSmemBytes) return AK_PATH_GENERIC;
+    if (bytes <= 4096) return AK_PATH_WARP;
+    if (bytes <= 32768) return AK_PATH_CTA;
     return AK_PATH_SMEM;
 }
 
-int rmsnorm_dispatch(const void* x, const void* w, void* y, int64_t rows, int64_t D, float eps,
-                     cudaStream_t st, int path) {
+namespace {
+
+template <int DT>
+int dispatch_t(const void* x, const void* w, void* y, int64_t rows, int64_t D, float eps, cudaStream_t st, int path) {
+    constexpr int kBytes = Elem<DT>::kBytes;
+    const int64_t row_bytes = D * kBytes;
     const bool aligned16 = is_aligned(x, 16) && is_aligned(y, 16) && is_aligned(w, 16);
-    if (path == AK_PATH_AUTO) path = rmsnorm_choose(rows, D, aligned16);
+    if (path == AK_PATH_AUTO) path = rmsnorm_choose(rows, D, aligned16, DT);
     const float inv_D = 1.0f / (float)D;
     if (path != AK_PATH_GENERIC) {
-        if ((D & 7) != 0) return AK_ERR_SHAPE;
+        if ((row_bytes & 15) != 0) return AK_ERR_SHAPE;
         if (!aligned16) return AK_ERR_ALIGN;
     }
     if (rows > 2147483647LL) return AK_ERR_SHAPE;  // grid.x limit of the one-row-per-CTA layouts
-    const int nvec = (int)(D >> 3);
+    const int nvec = (int)(row_bytes >> 4);
     switch (path) {
         case AK_PATH_WARP:
-            if (D > 2048) return AK_ERR_SHAPE;
-            if (nvec <= 128) return launch_reg_vpt<256, 32, 4, 1>((nvec + 31) / 32, x, w, y, rows, nvec, inv_D, eps, st);
-            return launch_reg_vpt<128, 32, 1, 1>((nvec + 31) / 32, x, w, y, rows, nvec, inv_D, eps, st);
+            if (row_bytes > 4096) return AK_ERR_SHAPE;
+            if (nvec <= 128) return launch_reg_vpt<DT, 256, 32, 4, 1>((nvec + 31) / 32, x, w, y, rows, nvec, inv_D, eps, st);
+            return launch_reg_vpt<DT, 128, 32, 1, 1>((nvec + 31) / 32, x, w, y, rows, nvec, inv_D, eps, st);
         case AK_PATH_CTA:
-            if (D > 32768) return AK_ERR_SHAPE;
+            if (row_bytes > 65536) return AK_ERR_SHAPE;
             // Shapes chosen in the sustained (power-capped) regime of a long run: 128 threads x <= 4
             // vectors (46 registers); 256 threads x <= 4 vectors (46 registers, five CTAs per SM);
             // 256 threads x <= 8 vectors capped at 85 registers (62 used).
-            if (nvec <= 512) return launch_reg_vpt<128, 128, 1, 1>((nvec + 127) / 128, x, w, y, rows, nvec, inv_D, eps, st);
-            if (nvec <= 2048) return launch_reg_vpt<256, 256, 1, 3>((nvec + 255) / 256, x, w, y, rows, nvec, inv_D, eps, st);
-            return launch_reg_vpt<512, 512, 1, 1>((nvec + 511) / 512, x, w, y, rows, nvec, inv_D, eps, st);
+            if (nvec <= 512) return launch_reg_vpt<DT, 128, 128, 1, 1>((nvec + 127) / 128, x, w, y, rows, nvec, inv_D, eps, st);
+            if (nvec <= 2048) return launch_reg_vpt<DT, 256, 256, 1, 3>((nvec + 255) / 256, x, w, y, rows, nvec, inv_D, eps, st);
+            return launch_reg_vpt<DT, 512, 512, 1, 1>((nvec + 511) / 512, x, w, y, rows, nvec, inv_D, eps, st);
         case AK_PATH_SMEM:
-            if (D * 2 > kMaxRowSmemBytes) return AK_ERR_SHAPE;
-            if (nvec <= 4096) return launch_smem<256>(x, w, y, rows, nvec, inv_D, eps, st);
-            return launch_smem<512>(x, w, y, rows, nvec, inv_D, eps, st);
+            if (row_bytes > kMaxRowSmemBytes) return AK_ERR_SHAPE;
+            if (nvec <= 4096) return launch_smem<DT, 256>(x, w, y, rows, nvec, inv_D, eps, st);
+            return launch_smem<DT, 512>(x, w, y, rows, nvec, inv_D, eps, st);
         case AK_PATH_GENERIC: {
-            // rows staged in shared memory when x and y rows share their 16-byte phase, w is
-            // 4-byte aligned and a row (plus up to 14 bytes of phase padding) fits
-            const size_t stage_bytes = (size_t)((D + 14) >> 3) * 16;
-            const bool same_phase = ((reinterpret_cast<uintptr_t>(x) ^ reinterpret_cast<uintptr_t>(y)) & 15) == 0;
-            if (same_phase && is_aligned(w, 4) && stage_bytes <= (size_t)kMaxRowSmemBytes) {
-                static const bool configured = [] {
-                    return cudaFuncSetAttribute(rmsnorm_stage_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                kMaxRowSmemBytes) == cudaSuccess &&
-                           cudaFuncSetAttribute(rmsnorm_stage_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                kMaxRowSmemBytes) == cudaSuccess &&
-                           cudaFuncSetAttribute(rmsnorm_stage_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                kMaxRowSmemBytes) == cudaSuccess;
+            if constexpr (DT == AK_DTYPE_F32) {
+                static const int resident32 = [] {
+                    int per_sm = 0;
+                    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rmsnorm_generic32_kernel,
+                                                                      kRmsGenericThreads, 0) != cudaSuccess || per_sm < 1)
+                        per_sm = 1;
+                    return per_sm * sm_count();
                 }();
-                if (!configured) return AK_ERR_CUDA;
+                const int grid = (int)(rows < resident32 ? rows : resident32);
+                rmsnorm_generic32_kernel<<<grid, kRmsGenericThreads, 0, st>>>(
+                    static_cast<const float*>(x), static_cast<const float*>(w), static_cast<float*>(y), rows, D, inv_D, eps);
+                count_launch();
+                return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+            } else {
+                // rows staged in shared memory when x and y rows share their 16-byte phase, w is
+                // 4-byte aligned and a row (plus up to 14 bytes of phase padding) fits
+                const size_t stage_bytes = (size_t)((D + 14) >> 3) * 16;
+                const bool same_phase = ((reinterpret_cast<uintptr_t>(x) ^ reinterpret_cast<uintptr_t>(y)) & 15) == 0;
                 const uint16_t* xs = static_cast<const uint16_t*>(x);
                 const uint16_t* ws = static_cast<const uint16_t*>(w);
                 uint16_t* ys = static_cast<uint16_t*>(y);
-                if (D <= 8192)
-                    rmsnorm_stage_kernel<128><<<(unsigned)rows, 128, stage_bytes, st>>>(xs, ws, ys, D, inv_D, eps);
-                else if (D <= 32768)
-                    rmsnorm_stage_kernel<256><<<(unsigned)rows, 256, stage_bytes, st>>>(xs, ws, ys, D, inv_D, eps);
-                else
-                    rmsnorm_stage_kernel<512><<<(unsigned)rows, 512, stage_bytes, st>>>(xs, ws, ys, D, inv_D, eps);
+                if (same_phase && is_aligned(w, 4) && stage_bytes <= (size_t)kMaxRowSmemBytes) {
+                    static const bool configured = [] {
+                        return cudaFuncSetAttribute(rmsnorm_stage_kernel<128, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                    kMaxRowSmemBytes) == cudaSuccess &&
+                               cudaFuncSetAttribute(rmsnorm_stage_kernel<256, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                    kMaxRowSmemBytes) == cudaSuccess &&
+                               cudaFuncSetAttribute(rmsnorm_stage_kernel<512, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                    kMaxRowSmemBytes) == cudaSuccess;
+                    }();
+                    if (!configured) return AK_ERR_CUDA;
+                    if (D <= 8192)
+                        rmsnorm_stage_kernel<128, DT><<<(unsigned)rows, 128, stage_bytes, st>>>(xs, ws, ys, D, inv_D, eps);
+                    else if (D <= 32768)
+                        rmsnorm_stage_kernel<256, DT><<<(unsigned)rows, 256, stage_bytes, st>>>(xs, ws, ys, D, inv_D, eps);
+                    else
+                        rmsnorm_stage_kernel<512, DT><<<(unsigned)rows, 512, stage_bytes, st>>>(xs, ws, ys, D, inv_D, eps);
+                    count_launch();
+                    return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+                }
+                static const int resident = [] {
+                    int per_sm = 0;
+                    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rmsnorm_generic_kernel<DT>,
+                                                                      kRmsGenericThreads, 0) != cudaSuccess || per_sm < 1)
+                        per_sm = 1;
+                    return per_sm * sm_count();
+                }();
+                const int grid = (int)(rows < resident ? rows : resident);
+                rmsnorm_generic_kernel<DT><<<grid, kRmsGenericThreads, 0, st>>>(xs, ws, ys, rows, D, inv_D, eps);
                 count_launch();
                 return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
             }
-            static const int resident = [] {
-                int per_sm = 0;
-                if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rmsnorm_generic_kernel,
-                                                                  kRmsGenericThreads, 0) != cudaSuccess || per_sm < 1)
-                    per_sm = 1;
-                return per_sm * sm_count();
-            }();
-            const int grid = (int)(rows < resident ? rows : resident);
-            rmsnorm_generic_kernel<<<grid, kRmsGenericThreads, 0, st>>>(
-                static_cast<const uint16_t*>(x), static_cast<const uint16_t*>(w), static_cast<uint16_t*>(y),
-                rows, D, inv_D, eps);
-            count_launch();
-            return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
         }
         default:
             return AK_ERR_ARG;
+    }
+}
+
+}  // namespace
+
+int rmsnorm_dispatch(const void* x, const void* w, void* y, int64_t rows, int64_t D, float eps,
+                     cudaStream_t st, int path, int dtype) {
+    switch (dtype) {
+        case AK_DTYPE_BF16: return dispatch_t<AK_DTYPE_BF16>(x, w, y, rows, D, eps, st, path);
+        case AK_DTYPE_F16: return dispatch_t<AK_DTYPE_F16>(x, w, y, rows, D, eps, st, path);
+        case AK_DTYPE_F32: return dispatch_t<AK_DTYPE_F32>(x, w, y, rows, D, eps, st, path);
+        default: return AK_ERR_ARG;
     }
 }
 

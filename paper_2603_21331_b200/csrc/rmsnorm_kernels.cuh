@@ -1,79 +1,69 @@
 // RMSNorm forward device kernels (paper Table 3 "rmsnorm": warp-shuffle reduction + fast
 // rsqrt, weight multiply fused into the epilogue per Section 7.3 Tier 3).
 //
-//   y[r, j] = bf16_rne( x[r, j] * rsqrt(mean_k x[r, k]^2 + eps) * w[j] )
+//   y[r, j] = rne( x[r, j] * rsqrt(mean_k x[r, k]^2 + eps) * w[j] )
 //
 // One DRAM read and one DRAM write per element, fp32 accumulation, fixed-order reductions.
+// Every kernel takes the element type DT (bf16, fp16 or fp32) as a template parameter; sizes
+// are counted in 16-byte vectors (8 or 4 elements).  The phase-staged and the multi-pass
+// kernels address 2-byte elements and serve the 16-bit types; fp32 rows that are not 16-byte
+// aligned go to rmsnorm_generic32_kernel.
 #pragma once
 
 #include "ak_common.cuh"
 
 namespace ak {
 
-// AK_RMS_MIXED = 1 (default) uses the mixed-precision multiply-adds; 0 keeps the packed
-// f32x2 formulation (kept for A/B measurements: 2 % slower sustained, 14 more registers).
-#ifndef AK_RMS_MIXED
-#define AK_RMS_MIXED 1
-#endif
-#if AK_RMS_MIXED
-// Mixed-precision forms (sm_100): the multiply-add reads its bf16 operands straight from
-// the two halves of a packed word and accumulates in fp32, so no widening instruction is
-// spent.  x*x + s and x*w are exact products (8-bit x 8-bit significands) with one rounding.
+// Vector helpers, one 16-byte vector at a time, per element type.
+//
+// 16-bit types use the mixed-precision forms (sm_100): the multiply-add reads its bf16 / fp16
+// operands straight from the two halves of a packed word and accumulates in fp32, so no
+// widening instruction is spent.  x*x + s and x*w are exact products (8-bit x 8-bit or
+// 11-bit x 11-bit significands) with one rounding.  (The packed f32x2 formulation measured 2 %
+// slower sustained with 14 more registers.)
 __device__ __forceinline__ void halves(uint32_t u, uint16_t& lo, uint16_t& hi) {
     asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(u));
 }
-__device__ __forceinline__ float fma_bf16(uint16_t a, uint16_t b, float c) {
-    float d;
-    asm("fma.rn.f32.bf16 %0, %1, %2, %3;" : "=f"(d) : "h"(a), "h"(b), "f"(c));
-    return d;
+template <int DT>
+__device__ __forceinline__ float sumsq_v(const uint4& v) {
+    if constexpr (DT == AK_DTYPE_F32) {
+        const float a = __uint_as_float(v.x), b = __uint_as_float(v.y), c = __uint_as_float(v.z), d = __uint_as_float(v.w);
+        return fmaf(c, c, a * a) + fmaf(d, d, b * b);
+    } else {
+        using E = Elem<DT>;
+        uint16_t a0, a1, a2, a3, a4, a5, a6, a7;
+        halves(v.x, a0, a1); halves(v.y, a2, a3); halves(v.z, a4, a5); halves(v.w, a6, a7);
+        float s0 = E::fma_h(a0, a0, 0.0f), s1 = E::fma_h(a1, a1, 0.0f);
+        s0 = E::fma_h(a2, a2, s0); s1 = E::fma_h(a3, a3, s1);
+        s0 = E::fma_h(a4, a4, s0); s1 = E::fma_h(a5, a5, s1);
+        s0 = E::fma_h(a6, a6, s0); s1 = E::fma_h(a7, a7, s1);
+        return s0 + s1;
+    }
 }
-__device__ __forceinline__ float sumsq8(const uint4& v) {
-    uint16_t a0, a1, a2, a3, a4, a5, a6, a7;
-    halves(v.x, a0, a1); halves(v.y, a2, a3); halves(v.z, a4, a5); halves(v.w, a6, a7);
-    float s0 = fma_bf16(a0, a0, 0.0f), s1 = fma_bf16(a1, a1, 0.0f);
-    s0 = fma_bf16(a2, a2, s0); s1 = fma_bf16(a3, a3, s1);
-    s0 = fma_bf16(a4, a4, s0); s1 = fma_bf16(a5, a5, s1);
-    s0 = fma_bf16(a6, a6, s0); s1 = fma_bf16(a7, a7, s1);
-    return s0 + s1;
-}
+template <int DT>
 __device__ __forceinline__ uint32_t scale2(uint32_t x, uint32_t w, f32x2 rstd2) {
+    using E = Elem<DT>;
     uint16_t x0, x1, w0, w1;
     halves(x, x0, x1); halves(w, w0, w1);
-    const f32x2 p = mul2(pack2(fma_bf16(x0, w0, 0.0f), fma_bf16(x1, w1, 0.0f)), rstd2);
+    const f32x2 p = mul2(pack2(E::fma_h(x0, w0, 0.0f), E::fma_h(x1, w1, 0.0f)), rstd2);
     float lo, hi;
     unpack2(p, lo, hi);
-    return pack_bf16x2(lo, hi);
+    return E::pack(lo, hi);
 }
-__device__ __forceinline__ uint4 scale8(const uint4& x, const uint4& w, float rstd) {
-    const f32x2 r2 = pack2(rstd, rstd);
-    return make_uint4(scale2(x.x, w.x, r2), scale2(x.y, w.y, r2), scale2(x.z, w.z, r2), scale2(x.w, w.w, r2));
+// (x * w) * rstd per element, one rounding to the output type (fp32: (x * rstd) * w)
+template <int DT>
+__device__ __forceinline__ uint4 scale_v(const uint4& x, const uint4& w, float rstd) {
+    if constexpr (DT == AK_DTYPE_F32) {
+        return make_uint4(__float_as_uint(__uint_as_float(x.x) * rstd * __uint_as_float(w.x)),
+                          __float_as_uint(__uint_as_float(x.y) * rstd * __uint_as_float(w.y)),
+                          __float_as_uint(__uint_as_float(x.z) * rstd * __uint_as_float(w.z)),
+                          __float_as_uint(__uint_as_float(x.w) * rstd * __uint_as_float(w.w)));
+    } else {
+        const f32x2 r2 = pack2(rstd, rstd);
+        return make_uint4(scale2<DT>(x.x, w.x, r2), scale2<DT>(x.y, w.y, r2), scale2<DT>(x.z, w.z, r2),
+                          scale2<DT>(x.w, w.w, r2));
+    }
 }
-#else
-// Packed f32x2 arithmetic throughout: even elements accumulate in the low lane, odd ones in
-// the high lane (fixed association), one instruction per pair.
-__device__ __forceinline__ float sumsq8(const uint4& v) {
-    const f32x2 a = widen2(v.x), b = widen2(v.y), c = widen2(v.z), d = widen2(v.w);
-    f32x2 s = mul2(a, a);
-    s = fma2(b, b, s);
-    s = fma2(c, c, s);
-    s = fma2(d, d, s);
-    float lo, hi;
-    unpack2(s, lo, hi);
-    return lo + hi;
-}
-
-// (x * rstd) * w per element, one rounding to bf16
-__device__ __forceinline__ uint32_t scale2(uint32_t x, uint32_t w, f32x2 rstd2) {
-    const f32x2 p = mul2(mul2(widen2(x), rstd2), widen2(w));
-    float lo, hi;
-    unpack2(p, lo, hi);
-    return pack_bf16x2(lo, hi);
-}
-__device__ __forceinline__ uint4 scale8(const uint4& x, const uint4& w, float rstd) {
-    const f32x2 r2 = pack2(rstd, rstd);
-    return make_uint4(scale2(x.x, w.x, r2), scale2(x.y, w.y, r2), scale2(x.z, w.z, r2), scale2(x.w, w.w, r2));
-}
-#endif
 
 // ------------------------------------------------------------------ row in registers
 // A CTA of THREADS threads is cut into THREADS / GROUP groups; one group owns one row and
@@ -86,7 +76,7 @@ __device__ __forceinline__ uint4 scale8(const uint4& x, const uint4& w, float rs
 // live registers) or after it.  MINB is the launch-bounds occupancy hint that caps the
 // register count.  The grid may be smaller than the number of row slots: groups then walk
 // the rows with a grid stride.
-template <int THREADS, int GROUP, int VPT, int MINB, bool W_EARLY>
+template <int THREADS, int GROUP, int VPT, int MINB, bool W_EARLY, int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(THREADS, MINB)
 rmsnorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w, uint4* __restrict__ y,
                    int64_t rows, int nvec, float inv_D, float eps) {
@@ -122,7 +112,7 @@ rmsnorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w, uin
         }
         float ss = 0.0f;
 #pragma unroll
-        for (int k = 0; k < VPT; ++k) ss += sumsq8(xv[k]);
+        for (int k = 0; k < VPT; ++k) ss += sumsq_v<DT>(xv[k]);
         ss = warp_sum(ss);
         if constexpr (WARPS_PER_GROUP > 1) {
             float* s = slots[phase] + g * WARPS_PER_GROUP;
@@ -139,7 +129,7 @@ rmsnorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w, uin
             const int i = t + k * GROUP;
             if (live && i < nvec) {
                 const uint4 wq = W_EARLY ? wv[k] : __ldg(w + i);
-                st_stream(yr + i, scale8(xv[k], wq, rstd));
+                st_stream(yr + i, scale_v<DT>(xv[k], wq, rstd));
             }
         }
     }
@@ -153,7 +143,7 @@ rmsnorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w, uin
 // 16-byte aligned rows (D % 8 == 0).  Dynamic shared memory = nvec * 16 bytes.
 constexpr uint32_t kBulkChunk = 32768;
 
-template <int THREADS, int MINB>
+template <int THREADS, int MINB, int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(THREADS, MINB)
 rmsnorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w, uint4* __restrict__ y,
                     int nvec, float inv_D, float eps) {
@@ -174,12 +164,12 @@ rmsnorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w, ui
     if (!mbar_wait(&bar, 0)) return;  // uniform: every thread waits on the same barrier
     float ss = 0.0f;
 #pragma unroll 4
-    for (int i = threadIdx.x; i < nvec; i += THREADS) ss += sumsq8(row[i]);
+    for (int i = threadIdx.x; i < nvec; i += THREADS) ss += sumsq_v<DT>(row[i]);
     ss = cta_sum<THREADS>(ss, slots, 0);
     const float rstd = rsqrtf(fmaf(ss, inv_D, eps));
     uint4* yr = y + r * nvec;
 #pragma unroll 4
-    for (int i = threadIdx.x; i < nvec; i += THREADS) st_stream(yr + i, scale8(row[i], __ldg(w + i), rstd));
+    for (int i = threadIdx.x; i < nvec; i += THREADS) st_stream(yr + i, scale_v<DT>(row[i], __ldg(w + i), rstd));
 }
 
 // ------------------------------------------------------------------ unaligned rows staged in shared memory
@@ -206,7 +196,7 @@ __device__ __forceinline__ uint4 load_w_shifted(const uint16_t* __restrict__ w, 
                       __funnelshift_r(d, e, 16));
 }
 
-template <int T>
+template <int T, int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(T)
 rmsnorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, uint16_t* __restrict__ y,
                      int64_t D, float inv_D, float eps) {
@@ -236,18 +226,18 @@ rmsnorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict_
     }
     __syncthreads();
     float ss = 0.0f;
-    for (int k = threadIdx.x; k < nv; k += T) ss += sumsq8(row[k]);
+    for (int k = threadIdx.x; k < nv; k += T) ss += sumsq_v<DT>(row[k]);
     ss = cta_sum<T>(ss, slots, 0);
     const float rstd = rsqrtf(fmaf(ss, inv_D, eps));
     for (int k = k_lo + threadIdx.x; k < k_hi; k += T)
-        st_stream(ya + k, scale8(row[k], load_w_shifted(w, (int64_t)k * 8 - phase), rstd));
+        st_stream(ya + k, scale_v<DT>(row[k], load_w_shifted(w, (int64_t)k * 8 - phase), rstd));
     if (threadIdx.x < 16) {
         const int k = (threadIdx.x < 8) ? 0 : nv - 1;
         const bool edge = (threadIdx.x < 8) ? (k_lo == 1) : (k_hi == nv - 1 && !(nv == 1 && k_lo == 1));
         const int e = threadIdx.x & 7;
         const int64_t j = (int64_t)k * 8 - phase + e;
         if (edge && j >= 0 && j < D)
-            yr[j] = float_to_bf16(bf16_to_float(row16[k * 8 + e]) * bf16_to_float(__ldg(w + j)) * rstd);
+            yr[j] = Elem<DT>::from_float(Elem<DT>::to_float(row16[k * 8 + e]) * Elem<DT>::to_float(__ldg(w + j)) * rstd);
     }
 }
 
@@ -258,6 +248,7 @@ rmsnorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict_
 // second pass re-reads the row, which this CTA has just pulled through L1/L2.
 constexpr int kRmsGenericThreads = 256;
 
+template <int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(kRmsGenericThreads)
 rmsnorm_generic_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w,
                        uint16_t* __restrict__ y, int64_t rows, int64_t D, float inv_D, float eps) {
@@ -277,13 +268,13 @@ rmsnorm_generic_kernel(const uint16_t* __restrict__ x, const uint16_t* __restric
         const uint4* xb = reinterpret_cast<const uint4*>(xr + head);
 
         float ss = 0.0f;
-        for (int64_t i = threadIdx.x; i < nbody; i += T) ss += sumsq8(xb[i]);
+        for (int64_t i = threadIdx.x; i < nbody; i += T) ss += sumsq_v<DT>(xb[i]);
         for (int64_t j = threadIdx.x; j < head; j += T) {
-            const float v = bf16_to_float(xr[j]);
+            const float v = Elem<DT>::to_float(xr[j]);
             ss = fmaf(v, v, ss);
         }
         for (int64_t j = tail0 + threadIdx.x; j < D; j += T) {
-            const float v = bf16_to_float(xr[j]);
+            const float v = Elem<DT>::to_float(xr[j]);
             ss = fmaf(v, v, ss);
         }
         ss = cta_sum<T>(ss, slots, phase);
@@ -299,12 +290,38 @@ rmsnorm_generic_kernel(const uint16_t* __restrict__ x, const uint16_t* __restric
             wq.y = (uint32_t)__ldg(wj + 2) | ((uint32_t)__ldg(wj + 3) << 16);
             wq.z = (uint32_t)__ldg(wj + 4) | ((uint32_t)__ldg(wj + 5) << 16);
             wq.w = (uint32_t)__ldg(wj + 6) | ((uint32_t)__ldg(wj + 7) << 16);
-            st_stream(yb + i, scale8(v, wq, rstd));
+            st_stream(yb + i, scale_v<DT>(v, wq, rstd));
         }
         for (int64_t j = threadIdx.x; j < head; j += T)
-            yr[j] = float_to_bf16(bf16_to_float(xr[j]) * rstd * bf16_to_float(__ldg(w + j)));
+            yr[j] = Elem<DT>::from_float(Elem<DT>::to_float(xr[j]) * rstd * Elem<DT>::to_float(__ldg(w + j)));
         for (int64_t j = tail0 + threadIdx.x; j < D; j += T)
-            yr[j] = float_to_bf16(bf16_to_float(xr[j]) * rstd * bf16_to_float(__ldg(w + j)));
+            yr[j] = Elem<DT>::from_float(Elem<DT>::to_float(xr[j]) * rstd * Elem<DT>::to_float(__ldg(w + j)));
+    }
+}
+
+// fp32 rows with no 16-byte alignment (D % 4 != 0 or a misaligned base): element-wise, two
+// passes, the second from L1/L2.
+__global__ void __launch_bounds__(kRmsGenericThreads)
+rmsnorm_generic32_kernel(const float* __restrict__ x, const float* __restrict__ w, float* __restrict__ y,
+                         int64_t rows, int64_t D, float inv_D, float eps) {
+    constexpr int T = kRmsGenericThreads;
+    __shared__ float slots[2 * kWarp];
+    int phase = 0;
+    for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+        const float* xr = x + row * D;
+        float* yr = y + row * D;
+        float s0 = 0.0f, s1 = 0.0f;
+        int64_t j = threadIdx.x;
+        for (; j + T < D; j += 2 * T) {
+            const float a = xr[j], b = xr[j + T];
+            s0 = fmaf(a, a, s0);
+            s1 = fmaf(b, b, s1);
+        }
+        if (j < D) s0 = fmaf(xr[j], xr[j], s0);
+        const float ss = cta_sum<T>(s0 + s1, slots, phase);
+        phase ^= 1;
+        const float rstd = rsqrtf(fmaf(ss, inv_D, eps));
+        for (int64_t k = threadIdx.x; k < D; k += T) yr[k] = xr[k] * rstd * __ldg(w + k);
     }
 }
 

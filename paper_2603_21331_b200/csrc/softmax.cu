@@ -1,15 +1,16 @@
 // Last-dim softmax forward: host dispatch.  Kernels live in softmax_kernels.cuh.
 //
 // Launch shapes come from CUDA-graph timed sweeps on B200 (see rmsnorm.cu for the
-// reasoning): one row per warp up to D = 2048, one row per CTA in registers up to
-// D = 8192 (exponentials kept in fp32, register cap chosen for five CTAs per SM), rows
-// beyond that staged in shared memory by the copy engine.
+// reasoning): one row per warp up to 4 KiB rows, one row per CTA in registers up to
+// 16 KiB rows (exponentials kept in fp32, register cap chosen for five CTAs per SM), rows
+// beyond that staged in shared memory by the copy engine.  The thresholds are in row bytes,
+// so they hold for every element type.
 #include "softmax_kernels.cuh"
 
 namespace ak {
 namespace {
 
-template <int THREADS, int GROUP, int VPT, int MINB>
+template <int DT, int THREADS, int GROUP, int VPT, int MINB>
 int launch_reg(const void* x, void* y, int64_t rows, int nvec, cudaStream_t st) {
     constexpr int GROUPS = THREADS / GROUP;
     const int64_t need = (rows + GROUPS - 1) / GROUPS;
@@ -18,126 +19,146 @@ int launch_reg(const void* x, void* y, int64_t rows, int nvec, cudaStream_t st) 
         static const int resident = [] {
             int per_sm = 0;
             if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-                    &per_sm, softmax_reg_kernel<THREADS, GROUP, VPT, MINB, false>, THREADS, 0) != cudaSuccess ||
+                    &per_sm, softmax_reg_kernel<THREADS, GROUP, VPT, MINB, false, DT>, THREADS, 0) != cudaSuccess ||
                 per_sm < 1)
                 per_sm = 1;
             return per_sm * sm_count();
         }();
         if (grid > resident) grid = resident;
     }
-    softmax_reg_kernel<THREADS, GROUP, VPT, MINB, false><<<(unsigned)grid, THREADS, 0, st>>>(
+    softmax_reg_kernel<THREADS, GROUP, VPT, MINB, false, DT><<<(unsigned)grid, THREADS, 0, st>>>(
         static_cast<const uint4*>(x), static_cast<uint4*>(y), rows, nvec);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
-template <int THREADS, int GROUP, int MINB_LO, int MINB_HI>
+template <int DT, int THREADS, int GROUP, int MINB_LO, int MINB_HI>
 int launch_reg_vpt(int vpt, const void* x, void* y, int64_t rows, int nvec, cudaStream_t st) {
     switch (vpt) {
-        case 1: return launch_reg<THREADS, GROUP, 1, MINB_LO>(x, y, rows, nvec, st);
-        case 2: return launch_reg<THREADS, GROUP, 2, MINB_LO>(x, y, rows, nvec, st);
-        case 3: return launch_reg<THREADS, GROUP, 3, MINB_LO>(x, y, rows, nvec, st);
-        case 4: return launch_reg<THREADS, GROUP, 4, MINB_LO>(x, y, rows, nvec, st);
-        case 5: return launch_reg<THREADS, GROUP, 5, MINB_HI>(x, y, rows, nvec, st);
-        case 6: return launch_reg<THREADS, GROUP, 6, MINB_HI>(x, y, rows, nvec, st);
-        case 7: return launch_reg<THREADS, GROUP, 7, MINB_HI>(x, y, rows, nvec, st);
-        case 8: return launch_reg<THREADS, GROUP, 8, MINB_HI>(x, y, rows, nvec, st);
+        case 1: return launch_reg<DT, THREADS, GROUP, 1, MINB_LO>(x, y, rows, nvec, st);
+        case 2: return launch_reg<DT, THREADS, GROUP, 2, MINB_LO>(x, y, rows, nvec, st);
+        case 3: return launch_reg<DT, THREADS, GROUP, 3, MINB_LO>(x, y, rows, nvec, st);
+        case 4: return launch_reg<DT, THREADS, GROUP, 4, MINB_LO>(x, y, rows, nvec, st);
+        case 5: return launch_reg<DT, THREADS, GROUP, 5, MINB_HI>(x, y, rows, nvec, st);
+        case 6: return launch_reg<DT, THREADS, GROUP, 6, MINB_HI>(x, y, rows, nvec, st);
+        case 7: return launch_reg<DT, THREADS, GROUP, 7, MINB_HI>(x, y, rows, nvec, st);
+        case 8: return launch_reg<DT, THREADS, GROUP, 8, MINB_HI>(x, y, rows, nvec, st);
         default: return AK_ERR_SHAPE;
     }
 }
 
-template <int THREADS, int KEEP>
+template <int DT, int THREADS, int KEEP>
 int launch_smem(const void* x, void* y, int64_t rows, int nvec, cudaStream_t st) {
     const size_t smem = (size_t)nvec * 16;
     static const bool configured = [] {
-        return cudaFuncSetAttribute(softmax_smem_kernel<THREADS, 1, KEEP>,
+        return cudaFuncSetAttribute(softmax_smem_kernel<THREADS, 1, KEEP, DT>,
                                     cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxRowSmemBytes) == cudaSuccess;
     }();
     if (!configured) return AK_ERR_CUDA;
-    softmax_smem_kernel<THREADS, 1, KEEP><<<(unsigned)rows, THREADS, smem, st>>>(
+    softmax_smem_kernel<THREADS, 1, KEEP, DT><<<(unsigned)rows, THREADS, smem, st>>>(
         static_cast<const uint4*>(x), static_cast<uint4*>(y), nvec);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
-}  // namespace
-
-int softmax_choose(int64_t rows, int64_t D, bool aligned16) {
-    (void)rows;
-    if (!aligned16 || (D & 7) != 0 || D * 2 > kMaxRowSmemBytes) return AK_PATH_GENERIC;
-    if (D <= 2048) return AK_PATH_WARP;
-    if (D <= 8192) return AK_PATH_CTA;
-    return AK_PATH_SMEM;
+template <int DT, int T>
+int launch_stage(const uint16_t* x, uint16_t* y, int64_t rows, int64_t D, size_t stage_bytes, cudaStream_t st) {
+    static const bool configured = [] {
+        return cudaFuncSetAttribute(softmax_stage_kernel<T, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    kMaxRowSmemBytes) == cudaSuccess;
+    }();
+    if (!configured) return AK_ERR_CUDA;
+    softmax_stage_kernel<T, DT><<<(unsigned)rows, T, stage_bytes, st>>>(x, y, D);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
-int softmax_dispatch(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st, int path) {
+template <typename K>
+int resident_ctas(K kernel, int threads) {
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, 0) != cudaSuccess || per_sm < 1)
+        per_sm = 1;
+    return per_sm * sm_count();
+}
+
+template <int DT>
+int dispatch_t(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st, int path) {
+    const int64_t row_bytes = D * Elem<DT>::kBytes;
     const bool aligned16 = is_aligned(x, 16) && is_aligned(y, 16);
-    if (path == AK_PATH_AUTO) path = softmax_choose(rows, D, aligned16);
+    if (path == AK_PATH_AUTO) path = softmax_choose(rows, D, aligned16, DT);
     if (path != AK_PATH_GENERIC) {
-        if ((D & 7) != 0) return AK_ERR_SHAPE;
+        if ((row_bytes & 15) != 0) return AK_ERR_SHAPE;
         if (!aligned16) return AK_ERR_ALIGN;
     }
     if (rows > 2147483647LL) return AK_ERR_SHAPE;  // grid.x limit of the one-row-per-CTA layouts
-    const int nvec = (int)(D >> 3);
+    const int nvec = (int)(row_bytes >> 4);
     switch (path) {
         case AK_PATH_WARP:
-            if (D > 2048) return AK_ERR_SHAPE;
-            return launch_reg_vpt<128, 32, 1, 1>((nvec + 31) / 32, x, y, rows, nvec, st);
+            if (row_bytes > 4096) return AK_ERR_SHAPE;
+            return launch_reg_vpt<DT, 128, 32, 1, 1>((nvec + 31) / 32, x, y, rows, nvec, st);
         case AK_PATH_CTA:
-            if (D > 32768) return AK_ERR_SHAPE;
+            if (row_bytes > 65536) return AK_ERR_SHAPE;
             // 128 threads with up to 8 vectors each (exponentials of the whole share in fp32
             // registers, capped at 102 registers for five CTAs per SM): the best sustained shape
-            // up to D = 8192
-            if (nvec <= 1024) return launch_reg_vpt<128, 128, 1, 5>((nvec + 127) / 128, x, y, rows, nvec, st);
-            if (nvec <= 2048) return launch_reg_vpt<256, 256, 1, 1>((nvec + 255) / 256, x, y, rows, nvec, st);
-            return launch_reg_vpt<512, 512, 1, 1>((nvec + 511) / 512, x, y, rows, nvec, st);
+            // up to 16 KiB rows
+            if (nvec <= 1024) return launch_reg_vpt<DT, 128, 128, 1, 5>((nvec + 127) / 128, x, y, rows, nvec, st);
+            if (nvec <= 2048) return launch_reg_vpt<DT, 256, 256, 1, 1>((nvec + 255) / 256, x, y, rows, nvec, st);
+            return launch_reg_vpt<DT, 512, 512, 1, 1>((nvec + 511) / 512, x, y, rows, nvec, st);
         case AK_PATH_SMEM:
-            if (D * 2 > kMaxRowSmemBytes) return AK_ERR_SHAPE;
+            if (row_bytes > kMaxRowSmemBytes) return AK_ERR_SHAPE;
             // 256 threads keeping the first four vectors' exponentials in registers: best both in
-            // short bursts and under the power cap of a long run up to D = 32768
-            if (nvec <= 4096) return launch_smem<256, 4>(x, y, rows, nvec, st);
-            return launch_smem<512, 0>(x, y, rows, nvec, st);
+            // short bursts and under the power cap of a long run up to 64 KiB rows
+            if (nvec <= 4096) return launch_smem<DT, 256, 4>(x, y, rows, nvec, st);
+            return launch_smem<DT, 512, 0>(x, y, rows, nvec, st);
         case AK_PATH_GENERIC: {
-            // rows staged in shared memory when x and y rows share their 16-byte phase and a row
-            // (plus up to 14 bytes of phase padding) fits
-            const size_t stage_bytes = (size_t)((D + 14) >> 3) * 16;
-            const bool same_phase = ((reinterpret_cast<uintptr_t>(x) ^ reinterpret_cast<uintptr_t>(y)) & 15) == 0;
-            if (same_phase && stage_bytes <= (size_t)kMaxRowSmemBytes) {
-                static const bool configured = [] {
-                    return cudaFuncSetAttribute(softmax_stage_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                kMaxRowSmemBytes) == cudaSuccess &&
-                           cudaFuncSetAttribute(softmax_stage_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                kMaxRowSmemBytes) == cudaSuccess &&
-                           cudaFuncSetAttribute(softmax_stage_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                kMaxRowSmemBytes) == cudaSuccess;
-                }();
-                if (!configured) return AK_ERR_CUDA;
+            if constexpr (DT == AK_DTYPE_F32) {
+                static const int resident = resident_ctas(softmax_generic32_kernel, kSmGenericThreads);
+                const int grid = (int)(rows < resident ? rows : resident);
+                softmax_generic32_kernel<<<grid, kSmGenericThreads, 0, st>>>(
+                    static_cast<const float*>(x), static_cast<float*>(y), rows, D);
+                count_launch();
+                return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+            } else {
+                // rows staged in shared memory when x and y rows share their 16-byte phase and a
+                // row (plus up to 14 bytes of phase padding) fits
+                const size_t stage_bytes = (size_t)((D + 14) >> 3) * 16;
+                const bool same_phase = ((reinterpret_cast<uintptr_t>(x) ^ reinterpret_cast<uintptr_t>(y)) & 15) == 0;
                 const uint16_t* xs = static_cast<const uint16_t*>(x);
                 uint16_t* ys = static_cast<uint16_t*>(y);
-                if (D <= 8192)
-                    softmax_stage_kernel<128><<<(unsigned)rows, 128, stage_bytes, st>>>(xs, ys, D);
-                else if (D <= 32768)
-                    softmax_stage_kernel<256><<<(unsigned)rows, 256, stage_bytes, st>>>(xs, ys, D);
-                else
-                    softmax_stage_kernel<512><<<(unsigned)rows, 512, stage_bytes, st>>>(xs, ys, D);
+                if (same_phase && stage_bytes <= (size_t)kMaxRowSmemBytes) {
+                    if (D <= 8192) return launch_stage<DT, 128>(xs, ys, rows, D, stage_bytes, st);
+                    if (D <= 32768) return launch_stage<DT, 256>(xs, ys, rows, D, stage_bytes, st);
+                    return launch_stage<DT, 512>(xs, ys, rows, D, stage_bytes, st);
+                }
+                static const int resident = resident_ctas(softmax_generic_kernel<DT>, kSmGenericThreads);
+                const int grid = (int)(rows < resident ? rows : resident);
+                softmax_generic_kernel<DT><<<grid, kSmGenericThreads, 0, st>>>(xs, ys, rows, D);
                 count_launch();
                 return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
             }
-            static const int resident = [] {
-                int per_sm = 0;
-                if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, softmax_generic_kernel,
-                                                                  kSmGenericThreads, 0) != cudaSuccess || per_sm < 1)
-                    per_sm = 1;
-                return per_sm * sm_count();
-            }();
-            const int grid = (int)(rows < resident ? rows : resident);
-            softmax_generic_kernel<<<grid, kSmGenericThreads, 0, st>>>(
-                static_cast<const uint16_t*>(x), static_cast<uint16_t*>(y), rows, D);
-            count_launch();
-            return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
         }
         default:
             return AK_ERR_ARG;
+    }
+}
+
+}  // namespace
+
+int softmax_choose(int64_t rows, int64_t D, bool aligned16, int dtype) {
+    (void)rows;
+    const int64_t bytes = D * dtype_bytes(dtype);
+    if (!aligned16 || (bytes & 15) != 0 || bytes > kMaxRowSmemBytes) return AK_PATH_GENERIC;
+    if (bytes <= 4096) return AK_PATH_WARP;
+    if (bytes <= 16384) return AK_PATH_CTA;
+    return AK_PATH_SMEM;
+}
+
+int softmax_dispatch(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st, int path, int dtype) {
+    switch (dtype) {
+        case AK_DTYPE_BF16: return dispatch_t<AK_DTYPE_BF16>(x, y, rows, D, st, path);
+        case AK_DTYPE_F16: return dispatch_t<AK_DTYPE_F16>(x, y, rows, D, st, path);
+        case AK_DTYPE_F32: return dispatch_t<AK_DTYPE_F32>(x, y, rows, D, st, path);
+        default: return AK_ERR_ARG;
     }
 }
 

@@ -1,7 +1,11 @@
 // Last-dim softmax forward device kernels (paper Table 3 "softmax": warp-shuffle
 // reductions, packed 16-bit loads).
 //
-//   m = max_k x[r, k];  y[r, j] = bf16_rne( exp(x[r, j] - m) / sum_k exp(x[r, k] - m) )
+//   m = max_k x[r, k];  y[r, j] = rne( exp(x[r, j] - m) / sum_k exp(x[r, k] - m) )
+//
+// Every kernel takes the element type DT (bf16, fp16 or fp32) as a template parameter; sizes
+// are counted in 16-byte vectors.  The phase-staged and multi-pass kernels address 2-byte
+// elements (16-bit types); unaligned fp32 rows go to softmax_generic32_kernel.
 //
 // exp is evaluated as 2^(x*log2e - rn(m*log2e)) with one FMA feeding the SFU.  Rounding
 // m*log2e once scales every term of the row by the same factor, which cancels in the
@@ -13,40 +17,79 @@
 
 namespace ak {
 
-constexpr uint32_t kNegInf2 = 0xFF80FF80u;  // two bf16 -inf
-
-__device__ __forceinline__ uint32_t max8(const uint4& v) {
-    return bf16x2_max(bf16x2_max(v.x, v.y), bf16x2_max(v.z, v.w));
+// Vector helpers per element type DT (16-byte vectors: 8 bf16 / fp16 or 4 fp32 elements).
+// The running maximum travels as one 32-bit word: a packed pair for the 16-bit types (the
+// packed max instruction is exact), the float's bits for fp32.
+template <int DT>
+__device__ __forceinline__ constexpr uint32_t neg_inf_word() {
+    if constexpr (DT == AK_DTYPE_F32) return 0xFF800000u; else return Elem<DT>::kNegInf2;
 }
-__device__ __forceinline__ float hmax_of(uint32_t m2) { return fmaxf(bf16lo(m2), bf16hi(m2)); }
+template <int DT>
+__device__ __forceinline__ uint32_t max_w(uint32_t a, uint32_t b) {   // drops a NaN operand
+    if constexpr (DT == AK_DTYPE_F32) return __float_as_uint(fmaxf(__uint_as_float(a), __uint_as_float(b)));
+    else return Elem<DT>::max2(a, b);
+}
+template <int DT>
+__device__ __forceinline__ uint32_t max_v(const uint4& v) {
+    return max_w<DT>(max_w<DT>(v.x, v.y), max_w<DT>(v.z, v.w));
+}
+template <int DT>
+__device__ __forceinline__ float hmax_of(uint32_t m) {
+    if constexpr (DT == AK_DTYPE_F32) return __uint_as_float(m);
+    else return fmaxf(Elem<DT>::lo(m), Elem<DT>::hi(m));
+}
+template <int DT>
+__device__ __forceinline__ uint4 neg_inf_vec() {
+    return make_uint4(neg_inf_word<DT>(), neg_inf_word<DT>(), neg_inf_word<DT>(), neg_inf_word<DT>());
+}
 
-// e[0..3] = the eight values 2^(x*log2e - m2) of one vector as four packed pairs; returns
-// their sum (fixed association: even elements in the low lane, odd in the high lane).
-// Multiply-adds, sums and the final scaling run as packed f32x2 instructions.
-__device__ __forceinline__ f32x2 exp_pair(uint32_t u, f32x2 l2, f32x2 nm2) {
+// e[..] = the values 2^(x*log2e - m2) of one vector as packed pairs (four pairs for the 16-bit
+// types, two for fp32); returns their sum (fixed association: even elements in the low lane,
+// odd in the high lane).  Multiply-adds, sums and the final scaling run as packed f32x2
+// instructions.
+__device__ __forceinline__ f32x2 exp_of_pair(f32x2 x2, f32x2 l2, f32x2 nm2) {
     float t0, t1;
-    unpack2(fma2(widen2(u), l2, nm2), t0, t1);
+    unpack2(fma2(x2, l2, nm2), t0, t1);
     return pack2(fast_exp2(t0), fast_exp2(t1));
 }
-__device__ __forceinline__ float exp8(const uint4& v, float m2, f32x2* e) {
+template <int DT>
+__device__ __forceinline__ float exp_v(const uint4& v, float m2, f32x2* e) {
     const f32x2 l2 = pack2(kLog2e, kLog2e), nm2 = pack2(-m2, -m2);
-    e[0] = exp_pair(v.x, l2, nm2);
-    e[1] = exp_pair(v.y, l2, nm2);
-    e[2] = exp_pair(v.z, l2, nm2);
-    e[3] = exp_pair(v.w, l2, nm2);
     float lo, hi;
-    unpack2(add2(add2(e[0], e[1]), add2(e[2], e[3])), lo, hi);
+    if constexpr (DT == AK_DTYPE_F32) {
+        e[0] = exp_of_pair(pack2(__uint_as_float(v.x), __uint_as_float(v.y)), l2, nm2);
+        e[1] = exp_of_pair(pack2(__uint_as_float(v.z), __uint_as_float(v.w)), l2, nm2);
+        unpack2(add2(e[0], e[1]), lo, hi);
+    } else {
+        e[0] = exp_of_pair(widen2_t<DT>(v.x), l2, nm2);
+        e[1] = exp_of_pair(widen2_t<DT>(v.y), l2, nm2);
+        e[2] = exp_of_pair(widen2_t<DT>(v.z), l2, nm2);
+        e[3] = exp_of_pair(widen2_t<DT>(v.w), l2, nm2);
+        unpack2(add2(add2(e[0], e[1]), add2(e[2], e[3])), lo, hi);
+    }
     return lo + hi;
 }
-__device__ __forceinline__ uint32_t norm2(f32x2 e, f32x2 inv2) {
-    float lo, hi;
-    unpack2(mul2(e, inv2), lo, hi);
-    return pack_bf16x2(lo, hi);
-}
-__device__ __forceinline__ uint4 norm8(const f32x2* e, float inv) {
+template <int DT>
+__device__ __forceinline__ uint4 norm_v(const f32x2* e, float inv) {
     const f32x2 inv2 = pack2(inv, inv);
-    return make_uint4(norm2(e[0], inv2), norm2(e[1], inv2), norm2(e[2], inv2), norm2(e[3], inv2));
+    if constexpr (DT == AK_DTYPE_F32) {
+        float a, b, c, d;
+        unpack2(mul2(e[0], inv2), a, b);
+        unpack2(mul2(e[1], inv2), c, d);
+        return make_uint4(__float_as_uint(a), __float_as_uint(b), __float_as_uint(c), __float_as_uint(d));
+    } else {
+        uint32_t o[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float lo, hi;
+            unpack2(mul2(e[i], inv2), lo, hi);
+            o[i] = Elem<DT>::pack(lo, hi);
+        }
+        return make_uint4(o[0], o[1], o[2], o[3]);
+    }
 }
+// exponentials kept per vector: four pairs (16-bit types) or two (fp32)
+template <int DT> constexpr int kExpPairs = (DT == AK_DTYPE_F32) ? 2 : 4;
 
 // ------------------------------------------------------------------ row in registers
 // Same thread layout as the RMSNorm register kernel: a group of GROUP threads owns a row,
@@ -55,7 +98,7 @@ __device__ __forceinline__ uint4 norm8(const f32x2* e, float inv) {
 // each is evaluated once; RECOMPUTE == true keeps only the packed inputs and evaluates the
 // exponentials a second time in the epilogue (half the registers, twice the SFU work) for
 // rows too long to hold in fp32.
-template <int THREADS, int GROUP, int VPT, int MINB, bool RECOMPUTE>
+template <int THREADS, int GROUP, int VPT, int MINB, bool RECOMPUTE, int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(THREADS, MINB)
 softmax_reg_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t rows, int nvec) {
     constexpr int GROUPS = THREADS / GROUP;
@@ -75,12 +118,12 @@ softmax_reg_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t r
 #pragma unroll
         for (int k = 0; k < VPT; ++k) {
             const int i = t + k * GROUP;
-            xv[k] = (live && i < nvec) ? ld_stream(xr + i) : make_uint4(kNegInf2, kNegInf2, kNegInf2, kNegInf2);
+            xv[k] = (live && i < nvec) ? ld_stream(xr + i) : neg_inf_vec<DT>();
         }
-        uint32_t mx = kNegInf2;
+        uint32_t mx = neg_inf_word<DT>();
 #pragma unroll
-        for (int k = 0; k < VPT; ++k) mx = bf16x2_max(mx, max8(xv[k]));
-        float m = warp_max(hmax_of(mx));
+        for (int k = 0; k < VPT; ++k) mx = max_w<DT>(mx, max_v<DT>(xv[k]));
+        float m = warp_max(hmax_of<DT>(mx));
         if constexpr (WARPS_PER_GROUP > 1) {
             float* s = slots[0] + g * WARPS_PER_GROUP;
             if (lane == 0) s[warp_in_group] = m;
@@ -88,10 +131,10 @@ softmax_reg_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t r
             m = warp_max((lane < WARPS_PER_GROUP) ? s[lane] : -INFINITY);
         }
         const float m2 = m * kLog2e;
-        f32x2 e[RECOMPUTE ? 1 : VPT][4];
+        f32x2 e[RECOMPUTE ? 1 : VPT][kExpPairs<DT>];
         float sum = 0.0f;
 #pragma unroll
-        for (int k = 0; k < VPT; ++k) sum += exp8(xv[k], m2, e[RECOMPUTE ? 0 : k]);
+        for (int k = 0; k < VPT; ++k) sum += exp_v<DT>(xv[k], m2, e[RECOMPUTE ? 0 : k]);
         sum = warp_sum(sum);
         if constexpr (WARPS_PER_GROUP > 1) {
             float* s = slots[1] + g * WARPS_PER_GROUP;
@@ -104,8 +147,8 @@ softmax_reg_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t r
 #pragma unroll
         for (int k = 0; k < VPT; ++k) {
             const int i = t + k * GROUP;
-            if constexpr (RECOMPUTE) exp8(xv[k], m2, e[0]);
-            if (live && i < nvec) st_stream(yr + i, norm8(e[RECOMPUTE ? 0 : k], inv));
+            if constexpr (RECOMPUTE) exp_v<DT>(xv[k], m2, e[0]);
+            if (live && i < nvec) st_stream(yr + i, norm_v<DT>(e[RECOMPUTE ? 0 : k], inv));
         }
     }
 }
@@ -119,7 +162,7 @@ softmax_reg_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t r
 // Dynamic shared memory = nvec * 16 bytes.
 constexpr uint32_t kSmBulkChunk = 32768;
 
-template <int THREADS, int MINB, int KEEP>
+template <int THREADS, int MINB, int KEEP, int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(THREADS, MINB)
 softmax_smem_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int nvec) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -138,22 +181,22 @@ softmax_smem_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int nvec
     }
     if (!mbar_wait(&bar, 0)) return;  // uniform: every thread waits on the same barrier
 
-    uint32_t mx = kNegInf2;
+    uint32_t mx = neg_inf_word<DT>();
 #pragma unroll 4
-    for (int i = threadIdx.x; i < nvec; i += THREADS) mx = bf16x2_max(mx, max8(row[i]));
-    const float m = cta_max<THREADS>(hmax_of(mx), slots, 0);
+    for (int i = threadIdx.x; i < nvec; i += THREADS) mx = max_w<DT>(mx, max_v<DT>(row[i]));
+    const float m = cta_max<THREADS>(hmax_of<DT>(mx), slots, 0);
     const float m2 = m * kLog2e;
 
-    f32x2 kept[KEEP > 0 ? KEEP : 1][4];
+    f32x2 kept[KEEP > 0 ? KEEP : 1][kExpPairs<DT>];
     float sum = 0.0f;
-    f32x2 e[4];
+    f32x2 e[kExpPairs<DT>];
 #pragma unroll
     for (int k = 0; k < KEEP; ++k) {
         const int i = threadIdx.x + k * THREADS;
-        if (i < nvec) sum += exp8(row[i], m2, kept[k]);
+        if (i < nvec) sum += exp_v<DT>(row[i], m2, kept[k]);
     }
 #pragma unroll 2
-    for (int i = threadIdx.x + KEEP * THREADS; i < nvec; i += THREADS) sum += exp8(row[i], m2, e);
+    for (int i = threadIdx.x + KEEP * THREADS; i < nvec; i += THREADS) sum += exp_v<DT>(row[i], m2, e);
     sum = cta_sum<THREADS>(sum, slots, 1);
     const float inv = 1.0f / sum;
 
@@ -161,12 +204,12 @@ softmax_smem_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int nvec
 #pragma unroll
     for (int k = 0; k < KEEP; ++k) {
         const int i = threadIdx.x + k * THREADS;
-        if (i < nvec) st_stream(yr + i, norm8(kept[k], inv));
+        if (i < nvec) st_stream(yr + i, norm_v<DT>(kept[k], inv));
     }
 #pragma unroll 2
     for (int i = threadIdx.x + KEEP * THREADS; i < nvec; i += THREADS) {
-        exp8(row[i], m2, e);
-        st_stream(yr + i, norm8(e, inv));
+        exp_v<DT>(row[i], m2, e);
+        st_stream(yr + i, norm_v<DT>(e, inv));
     }
 }
 
@@ -175,7 +218,7 @@ softmax_smem_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int nvec
 // 16-byte phase it has in global memory (x and y rows share it), fully-inside vectors move
 // with aligned 16-byte loads and stores, the edge vectors element by element with -inf
 // standing in for the neighbours' bytes.  Three passes over shared memory.
-template <int T>
+template <int T, int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(T)
 softmax_stage_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, int64_t D) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -197,24 +240,24 @@ softmax_stage_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, i
     const int64_t my_j = (int64_t)my_edge_k * 8 - phase + (threadIdx.x & 7);
 
     for (int k = k_lo + threadIdx.x; k < k_hi; k += T) row[k] = ld_stream(xa + k);
-    if (my_edge) row16[my_edge_k * 8 + (threadIdx.x & 7)] = (my_j >= 0 && my_j < D) ? ld_stream_u16(xr + my_j) : (uint16_t)0xFF80;
+    if (my_edge) row16[my_edge_k * 8 + (threadIdx.x & 7)] = (my_j >= 0 && my_j < D) ? ld_stream_u16(xr + my_j) : Elem<DT>::kNegInf;
     __syncthreads();
 
-    uint32_t mx = kNegInf2;
-    for (int k = threadIdx.x; k < nv; k += T) mx = bf16x2_max(mx, max8(row[k]));
-    const float m = cta_max<T>(hmax_of(mx), slots, 0);
+    uint32_t mx = neg_inf_word<DT>();
+    for (int k = threadIdx.x; k < nv; k += T) mx = max_w<DT>(mx, max_v<DT>(row[k]));
+    const float m = cta_max<T>(hmax_of<DT>(mx), slots, 0);
     const float m2 = m * kLog2e;
     float sum = 0.0f;
-    f32x2 e[4];
-    for (int k = threadIdx.x; k < nv; k += T) sum += exp8(row[k], m2, e);
+    f32x2 e[kExpPairs<DT>];
+    for (int k = threadIdx.x; k < nv; k += T) sum += exp_v<DT>(row[k], m2, e);
     sum = cta_sum<T>(sum, slots, 1);
     const float inv = 1.0f / sum;
     for (int k = k_lo + threadIdx.x; k < k_hi; k += T) {
-        exp8(row[k], m2, e);
-        st_stream(ya + k, norm8(e, inv));
+        exp_v<DT>(row[k], m2, e);
+        st_stream(ya + k, norm_v<DT>(e, inv));
     }
     if (my_edge && my_j >= 0 && my_j < D)
-        yr[my_j] = float_to_bf16(fast_exp2(fmaf(bf16_to_float(row16[my_edge_k * 8 + (threadIdx.x & 7)]), kLog2e, -m2)) * inv);
+        yr[my_j] = Elem<DT>::from_float(fast_exp2(fmaf(Elem<DT>::to_float(row16[my_edge_k * 8 + (threadIdx.x & 7)]), kLog2e, -m2)) * inv);
 }
 
 // ------------------------------------------------------------------ generic
@@ -222,6 +265,7 @@ softmax_stage_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, i
 // from DRAM, the other two are served by L1/L2.
 constexpr int kSmGenericThreads = 256;
 
+template <int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(kSmGenericThreads)
 softmax_generic_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, int64_t rows, int64_t D) {
     constexpr int T = kSmGenericThreads;
@@ -238,31 +282,51 @@ softmax_generic_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y,
         const int64_t tail0 = head + (nbody << 3);
         const uint4* xb = reinterpret_cast<const uint4*>(xr + head);
 
-        uint32_t mx = kNegInf2;
-        for (int64_t i = threadIdx.x; i < nbody; i += T) mx = bf16x2_max(mx, max8(xb[i]));
-        float m = hmax_of(mx);
-        for (int64_t j = threadIdx.x; j < head; j += T) m = fmaxf(m, bf16_to_float(xr[j]));
-        for (int64_t j = tail0 + threadIdx.x; j < D; j += T) m = fmaxf(m, bf16_to_float(xr[j]));
+        uint32_t mx = neg_inf_word<DT>();
+        for (int64_t i = threadIdx.x; i < nbody; i += T) mx = max_w<DT>(mx, max_v<DT>(xb[i]));
+        float m = hmax_of<DT>(mx);
+        for (int64_t j = threadIdx.x; j < head; j += T) m = fmaxf(m, Elem<DT>::to_float(xr[j]));
+        for (int64_t j = tail0 + threadIdx.x; j < D; j += T) m = fmaxf(m, Elem<DT>::to_float(xr[j]));
         m = cta_max<T>(m, slots, 0);
         const float m2 = m * kLog2e;
 
         float s = 0.0f;
-        f32x2 e[4];
-        for (int64_t i = threadIdx.x; i < nbody; i += T) s += exp8(xb[i], m2, e);
-        for (int64_t j = threadIdx.x; j < head; j += T) s += fast_exp2(fmaf(bf16_to_float(xr[j]), kLog2e, -m2));
-        for (int64_t j = tail0 + threadIdx.x; j < D; j += T) s += fast_exp2(fmaf(bf16_to_float(xr[j]), kLog2e, -m2));
+        f32x2 e[kExpPairs<DT>];
+        for (int64_t i = threadIdx.x; i < nbody; i += T) s += exp_v<DT>(xb[i], m2, e);
+        for (int64_t j = threadIdx.x; j < head; j += T) s += fast_exp2(fmaf(Elem<DT>::to_float(xr[j]), kLog2e, -m2));
+        for (int64_t j = tail0 + threadIdx.x; j < D; j += T) s += fast_exp2(fmaf(Elem<DT>::to_float(xr[j]), kLog2e, -m2));
         s = cta_sum<T>(s, slots, 1);
         const float inv = 1.0f / s;
 
         uint4* yb = reinterpret_cast<uint4*>(yr + head);
         for (int64_t i = threadIdx.x; i < nbody; i += T) {
-            exp8(xb[i], m2, e);
-            st_stream(yb + i, norm8(e, inv));
+            exp_v<DT>(xb[i], m2, e);
+            st_stream(yb + i, norm_v<DT>(e, inv));
         }
         for (int64_t j = threadIdx.x; j < head; j += T)
-            yr[j] = float_to_bf16(fast_exp2(fmaf(bf16_to_float(xr[j]), kLog2e, -m2)) * inv);
+            yr[j] = Elem<DT>::from_float(fast_exp2(fmaf(Elem<DT>::to_float(xr[j]), kLog2e, -m2)) * inv);
         for (int64_t j = tail0 + threadIdx.x; j < D; j += T)
-            yr[j] = float_to_bf16(fast_exp2(fmaf(bf16_to_float(xr[j]), kLog2e, -m2)) * inv);
+            yr[j] = Elem<DT>::from_float(fast_exp2(fmaf(Elem<DT>::to_float(xr[j]), kLog2e, -m2)) * inv);
+    }
+}
+
+// fp32 rows with no 16-byte alignment: element-wise, three passes (the last two from L1/L2).
+__global__ void __launch_bounds__(kSmGenericThreads)
+softmax_generic32_kernel(const float* __restrict__ x, float* __restrict__ y, int64_t rows, int64_t D) {
+    constexpr int T = kSmGenericThreads;
+    __shared__ float slots[2 * kWarp];
+    for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+        const float* xr = x + row * D;
+        float* yr = y + row * D;
+        float m = -INFINITY;
+        for (int64_t j = threadIdx.x; j < D; j += T) m = fmaxf(m, xr[j]);
+        m = cta_max<T>(m, slots, 0);
+        const float m2 = m * kLog2e;
+        float s = 0.0f;
+        for (int64_t j = threadIdx.x; j < D; j += T) s += fast_exp2(fmaf(xr[j], kLog2e, -m2));
+        s = cta_sum<T>(s, slots, 1);
+        const float inv = 1.0f / s;
+        for (int64_t j = threadIdx.x; j < D; j += T) yr[j] = fast_exp2(fmaf(xr[j], kLog2e, -m2)) * inv;
     }
 }
 

@@ -25,7 +25,8 @@ constexpr int kRowThreads = 128;
 constexpr int kRowUnroll = 8;
 constexpr int kRowMinCtas = 8;
 
-int launch_finish(const uint16_t* logits, const int64_t* targets, int64_t ignore_index, const float2* partial,
+template <int DT>
+int launch_finish(const typename XElem<DT>::type* logits, const int64_t* targets, int64_t ignore_index, const float2* partial,
                   int nsplit, float* loss_rows, int64_t rows, int64_t V, float* out_mean, double* out_pair,
                   cudaStream_t st, bool dependent) {
     cudaLaunchConfig_t cfg = {};
@@ -38,7 +39,7 @@ int launch_finish(const uint16_t* logits, const int64_t* targets, int64_t ignore
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = dependent ? 1 : 0;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, xent_finish_kernel, logits, targets, ignore_index, partial, nsplit,
+    cudaError_t e = cudaLaunchKernelEx(&cfg, xent_finish_kernel<DT>, logits, targets, ignore_index, partial, nsplit,
                                        loss_rows, rows, V, out_mean, out_pair);
     count_launch();
     return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
@@ -63,10 +64,14 @@ int xent_choose(int64_t rows, int64_t V, int* nsplit) {
     return ns > 1 ? AK_XENT_SPLIT : AK_XENT_ROW;
 }
 
-int xent_dispatch(const void* logits, const int64_t* targets, int64_t ignore_index,
-                  float* loss_rows, float* loss_mean, int64_t rows, int64_t V,
-                  void* workspace, size_t workspace_bytes, bool may_allocate,
-                  cudaStream_t st, int path, int nsplit) {
+namespace {
+
+template <int DT>
+int dispatch_t(const void* logits, const int64_t* targets, int64_t ignore_index,
+               float* loss_rows, float* loss_mean, int64_t rows, int64_t V,
+               void* workspace, size_t workspace_bytes, bool may_allocate,
+               cudaStream_t st, int path, int nsplit) {
+    using elem_t = typename XElem<DT>::type;
     int auto_ns = 1;
     const int auto_path = xent_choose(rows, V, &auto_ns);
     if (path == AK_XENT_AUTO) {
@@ -81,20 +86,20 @@ int xent_dispatch(const void* logits, const int64_t* targets, int64_t ignore_ind
         return AK_ERR_ARG;
     }
     if (rows > 2147483647LL) return AK_ERR_SHAPE;  // grid.x limit
-    const uint16_t* lg = static_cast<const uint16_t*>(logits);
+    const elem_t* lg = static_cast<const elem_t*>(logits);
 
     if (rows == 0) {
         // nothing to stream; the mean of an empty batch is NaN
         if (loss_mean == nullptr) return AK_OK;
-        return launch_finish(lg, targets, ignore_index, nullptr, 0, loss_rows, 0, V, loss_mean, nullptr, st, false);
+        return launch_finish<DT>(lg, targets, ignore_index, nullptr, 0, loss_rows, 0, V, loss_mean, nullptr, st, false);
     }
     if (path == AK_XENT_ROW) {
-        xent_row_kernel<kRowUnroll, kPoly, kRowMinCtas, kRowThreads><<<(unsigned)rows, kRowThreads, 0, st>>>(
+        xent_row_kernel<kRowUnroll, kPoly, kRowMinCtas, kRowThreads, DT><<<(unsigned)rows, kRowThreads, 0, st>>>(
             lg, targets, ignore_index, loss_rows, V);
         count_launch();
         if (cudaGetLastError() != cudaSuccess) return AK_ERR_CUDA;
         if (loss_mean == nullptr) return AK_OK;
-        return launch_finish(lg, targets, ignore_index, nullptr, 0, loss_rows, rows, V, loss_mean, nullptr, st, true);
+        return launch_finish<DT>(lg, targets, ignore_index, nullptr, 0, loss_rows, rows, V, loss_mean, nullptr, st, true);
     }
     if (rows > 65535) return AK_ERR_SHAPE;  // grid.y limit; the dispatcher never splits that many rows
     const size_t need = (size_t)rows * (size_t)nsplit * sizeof(float2);
@@ -110,26 +115,47 @@ int xent_dispatch(const void* logits, const int64_t* targets, int64_t ignore_ind
         partial = static_cast<float2*>(p);
         own = true;
     }
-    xent_split_kernel<kUnroll, kPoly><<<dim3((unsigned)nsplit, (unsigned)rows), kXentThreads, 0, st>>>(
+    xent_split_kernel<kUnroll, kPoly, DT><<<dim3((unsigned)nsplit, (unsigned)rows), kXentThreads, 0, st>>>(
         lg, targets, ignore_index, partial, V, nsplit);
     count_launch();
     int status = cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
     if (status == AK_OK)
-        status = launch_finish(lg, targets, ignore_index, partial, nsplit, loss_rows, rows, V, loss_mean, nullptr, st, true);
+        status = launch_finish<DT>(lg, targets, ignore_index, partial, nsplit, loss_rows, rows, V, loss_mean, nullptr, st, true);
     if (own) cudaFreeAsync(partial, st);
     return status;
 }
 
+}  // namespace
+
+int xent_dispatch(const void* logits, const int64_t* targets, int64_t ignore_index,
+                  float* loss_rows, float* loss_mean, int64_t rows, int64_t V,
+                  void* workspace, size_t workspace_bytes, bool may_allocate,
+                  cudaStream_t st, int path, int nsplit, int dtype) {
+    switch (dtype) {
+        case AK_DTYPE_BF16:
+            return dispatch_t<AK_DTYPE_BF16>(logits, targets, ignore_index, loss_rows, loss_mean, rows, V, workspace,
+                                             workspace_bytes, may_allocate, st, path, nsplit);
+        case AK_DTYPE_F16:
+            return dispatch_t<AK_DTYPE_F16>(logits, targets, ignore_index, loss_rows, loss_mean, rows, V, workspace,
+                                            workspace_bytes, may_allocate, st, path, nsplit);
+        case AK_DTYPE_F32:
+            return dispatch_t<AK_DTYPE_F32>(logits, targets, ignore_index, loss_rows, loss_mean, rows, V, workspace,
+                                            workspace_bytes, may_allocate, st, path, nsplit);
+        default:
+            return AK_ERR_ARG;
+    }
+}
+
 int xent_mean_launch(const float* loss_rows, const int64_t* targets, int64_t ignore_index, int64_t rows,
                      float* loss_mean, cudaStream_t st) {
-    return launch_finish(nullptr, targets, ignore_index, nullptr, 0, const_cast<float*>(loss_rows), rows, 0,
-                         loss_mean, nullptr, st, false);
+    return launch_finish<AK_DTYPE_BF16>(nullptr, targets, ignore_index, nullptr, 0, const_cast<float*>(loss_rows), rows,
+                                        0, loss_mean, nullptr, st, false);
 }
 
 int xent_sum_count_launch(const float* loss_rows, const int64_t* targets, int64_t ignore_index, int64_t rows,
                           double* sum_count, cudaStream_t st) {
-    return launch_finish(nullptr, targets, ignore_index, nullptr, 0, const_cast<float*>(loss_rows), rows, 0,
-                         nullptr, sum_count, st, false);
+    return launch_finish<AK_DTYPE_BF16>(nullptr, targets, ignore_index, nullptr, 0, const_cast<float*>(loss_rows), rows,
+                                        0, nullptr, sum_count, st, false);
 }
 
 int xent_mean_merge_launch(const double* pairs, int64_t n, float* loss_mean, cudaStream_t st) {

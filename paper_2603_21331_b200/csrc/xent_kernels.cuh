@@ -3,8 +3,10 @@
 //
 //   loss[r] = (m - x[r, t]) + log( sum_k exp(x[r, k] - m) ),  m = max_k x[r, k]
 //
+// Kernels take the element type DT of the logits (bf16, fp16 or fp32) as a template parameter.
+//
 // Each thread streams 16-byte vectors of its row (or of its slice of the row) and keeps an
-// online pair: the running maximum m (always a bf16 value) and s = sum 2^(x*log2e - mf)
+// online pair: the running maximum m (always a value of the element type) and s = sum 2^(x*log2e - mf)
 // with mf = rn(m*log2e).  Rescaling by 2^(mf_old - mf_new) happens once per batch of
 // vectors, only when the maximum moved.  Working in the rounded log2 domain is exact up to
 // one per-row constant: x*log2e - m*log2e = (x*log2e - mf) - err with
@@ -25,22 +27,53 @@
 
 namespace ak {
 
-constexpr uint32_t kXNegInf2 = 0xFF80FF80u;
 constexpr float kFloor2 = -1.0e30f;  // finite stand-in for "no maximum yet" in the log2 domain
 constexpr int kXentThreads = 256;
 
-// NaN-propagating packed max: a NaN logit must surface as a NaN loss.
-__device__ __forceinline__ uint32_t bf16x2_max_nan(uint32_t a, uint32_t b) {
-    uint32_t r;
-    asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
-    return r;
+// Per element type DT: the storage type of one element, the -inf padding word, and the
+// NaN-propagating maximum of a 16-byte vector (a NaN logit must surface as a NaN loss).  The
+// running maximum of a batch travels as one 32-bit word (a packed pair for the 16-bit types,
+// the float's bits for fp32).
+template <int DT> struct XElem { using type = uint16_t; };
+template <> struct XElem<AK_DTYPE_F32> { using type = float; };
+template <int DT>
+__device__ __forceinline__ constexpr uint32_t xneg_inf_word() {
+    if constexpr (DT == AK_DTYPE_F32) return 0xFF800000u; else return Elem<DT>::kNegInf2;
 }
-__device__ __forceinline__ uint32_t xmax8(const uint4& v) {
-    return bf16x2_max_nan(bf16x2_max_nan(v.x, v.y), bf16x2_max_nan(v.z, v.w));
+template <int DT>
+__device__ __forceinline__ uint4 xneg_inf_vec() {
+    return make_uint4(xneg_inf_word<DT>(), xneg_inf_word<DT>(), xneg_inf_word<DT>(), xneg_inf_word<DT>());
 }
+template <int DT>
+__device__ __forceinline__ uint32_t xmax_w(uint32_t a, uint32_t b) {
+    if constexpr (DT == AK_DTYPE_F32) {
+        uint32_t r;
+        asm("max.NaN.f32 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+        return r;
+    } else {
+        return Elem<DT>::max2_nan(a, b);
+    }
+}
+template <int DT>
+__device__ __forceinline__ uint32_t xmax_v(const uint4& v) {
+    return xmax_w<DT>(xmax_w<DT>(v.x, v.y), xmax_w<DT>(v.z, v.w));
+}
+template <int DT>
 __device__ __forceinline__ float xhmax_of(uint32_t m2) {
-    const float a = bf16lo(m2), b = bf16hi(m2);
-    return (a != a || b != b) ? __int_as_float(0x7fc00000) : fmaxf(a, b);
+    if constexpr (DT == AK_DTYPE_F32) {
+        return __uint_as_float(m2);
+    } else {
+        const float a = Elem<DT>::lo(m2), b = Elem<DT>::hi(m2);
+        return (a != a || b != b) ? __int_as_float(0x7fc00000) : fmaxf(a, b);
+    }
+}
+template <int DT>
+__device__ __forceinline__ float xload(const typename XElem<DT>::type* p) {   // one element, streaming
+    if constexpr (DT == AK_DTYPE_F32) return __ldcs(p); else return Elem<DT>::to_float(ld_stream_u16(p));
+}
+template <int DT>
+__device__ __forceinline__ float xread(const typename XElem<DT>::type* p) {   // one element, cached
+    if constexpr (DT == AK_DTYPE_F32) return *p; else return Elem<DT>::to_float(*p);
 }
 
 // 2^t for a pair, t <= ~0, on the FMA pipe.  t is clamped at -125 (2^-125 stands in for
@@ -73,20 +106,30 @@ __device__ __forceinline__ f32x2 sfu_exp2_pair(f32x2 t2) {
     return pack2(fast_exp2(t0), fast_exp2(t1));
 }
 
-// sum over the 8 elements of one vector of 2^(x*log2e - mf), as a packed pair of partial
-// sums.  The first POLY / 2 of the four pairs take the polynomial, the rest the SFU.
-template <int POLY>
-__device__ __forceinline__ f32x2 sumexp8(const uint4& v, f32x2 l2, f32x2 nmf2) {
+// sum over the elements of one vector of 2^(x*log2e - mf), as a packed pair of partial sums.
+// 16-bit types: four pairs, the first POLY / 2 of them take the polynomial, the rest the SFU.
+// fp32: two pairs and half as many exponentials per byte, so the SFU keeps up: pair k takes
+// the polynomial only if POLY >= 4 * (k + 1).
+template <int POLY, int DT>
+__device__ __forceinline__ f32x2 sumexp_v(const uint4& v, f32x2 l2, f32x2 nmf2) {
     static_assert(POLY % 2 == 0 && POLY >= 0 && POLY <= 8, "pairs");
-    const f32x2 t0 = fma2(widen2(v.x), l2, nmf2);
-    const f32x2 t1 = fma2(widen2(v.y), l2, nmf2);
-    const f32x2 t2 = fma2(widen2(v.z), l2, nmf2);
-    const f32x2 t3 = fma2(widen2(v.w), l2, nmf2);
-    const f32x2 e0 = (POLY >= 2) ? poly_exp2_pair(t0) : sfu_exp2_pair(t0);
-    const f32x2 e1 = (POLY >= 4) ? poly_exp2_pair(t1) : sfu_exp2_pair(t1);
-    const f32x2 e2 = (POLY >= 6) ? poly_exp2_pair(t2) : sfu_exp2_pair(t2);
-    const f32x2 e3 = (POLY >= 8) ? poly_exp2_pair(t3) : sfu_exp2_pair(t3);
-    return add2(add2(e0, e1), add2(e2, e3));
+    if constexpr (DT == AK_DTYPE_F32) {
+        const f32x2 t0 = fma2(pack2(__uint_as_float(v.x), __uint_as_float(v.y)), l2, nmf2);
+        const f32x2 t1 = fma2(pack2(__uint_as_float(v.z), __uint_as_float(v.w)), l2, nmf2);
+        const f32x2 e0 = (POLY >= 4) ? poly_exp2_pair(t0) : sfu_exp2_pair(t0);
+        const f32x2 e1 = (POLY >= 8) ? poly_exp2_pair(t1) : sfu_exp2_pair(t1);
+        return add2(e0, e1);
+    } else {
+        const f32x2 t0 = fma2(widen2_t<DT>(v.x), l2, nmf2);
+        const f32x2 t1 = fma2(widen2_t<DT>(v.y), l2, nmf2);
+        const f32x2 t2 = fma2(widen2_t<DT>(v.z), l2, nmf2);
+        const f32x2 t3 = fma2(widen2_t<DT>(v.w), l2, nmf2);
+        const f32x2 e0 = (POLY >= 2) ? poly_exp2_pair(t0) : sfu_exp2_pair(t0);
+        const f32x2 e1 = (POLY >= 4) ? poly_exp2_pair(t1) : sfu_exp2_pair(t1);
+        const f32x2 e2 = (POLY >= 6) ? poly_exp2_pair(t2) : sfu_exp2_pair(t2);
+        const f32x2 e3 = (POLY >= 8) ? poly_exp2_pair(t3) : sfu_exp2_pair(t3);
+        return add2(add2(e0, e1), add2(e2, e3));
+    }
 }
 
 struct Online {
@@ -109,34 +152,37 @@ __device__ __forceinline__ void absorb_scalar(Online& o, float v) {
     o.s2 = add2(o.s2, pack2(fast_exp2(fmaf(v, kLog2e, -o.mf)), 0.0f));
 }
 
-// A slice = elements [begin, end) of one row, cut into up to 7 head elements (2-byte loads
-// until the address is 16-byte aligned), nbody aligned 16-byte vectors, and up to 7 tail
-// elements.  One batch = UNROLL vectors per thread, all loaded before the first use.  Full
-// batches run without any per-vector bounds test (constant offsets from one moving pointer);
-// a single masked batch finishes the slice.
+// A slice = elements [begin, end) of one row, cut into up to kPerVec - 1 head elements (single
+// loads until the address is 16-byte aligned), nbody aligned 16-byte vectors, and up to
+// kPerVec - 1 tail elements.  One batch = UNROLL vectors per thread, all loaded before the
+// first use.  Full batches run without any per-vector bounds test (constant offsets from one
+// moving pointer); a single masked batch finishes the slice.
+template <int DT>
 struct Slice {
-    const uint16_t* p;
+    const typename XElem<DT>::type* p;
     int64_t n, head, nbody, tail0, nfull;
     const uint4* body;
     int rest;  // vectors in the masked last batch, < T * UNROLL
 };
-template <int UNROLL, int T>
-__device__ __forceinline__ Slice make_slice(const uint16_t* __restrict__ xr, int64_t begin, int64_t end) {
-    Slice s;
+template <int UNROLL, int T, int DT>
+__device__ __forceinline__ Slice<DT> make_slice(const typename XElem<DT>::type* __restrict__ xr, int64_t begin, int64_t end) {
+    constexpr int PV = Elem<DT>::kPerVec;
+    constexpr int LOG_PV = (PV == 8) ? 3 : 2, LOG_BYTES = (Elem<DT>::kBytes == 2) ? 1 : 2;
+    Slice<DT> s;
     s.p = xr + begin;
     s.n = end - begin;
-    s.head = (8 - (int)((reinterpret_cast<uintptr_t>(s.p) >> 1) & 7)) & 7;
+    s.head = (PV - (int)((reinterpret_cast<uintptr_t>(s.p) >> LOG_BYTES) & (PV - 1))) & (PV - 1);
     if (s.head > s.n) s.head = s.n;
-    s.nbody = (s.n - s.head) >> 3;
-    s.tail0 = s.head + (s.nbody << 3);
+    s.nbody = (s.n - s.head) >> LOG_PV;
+    s.tail0 = s.head + (s.nbody << LOG_PV);
     s.body = reinterpret_cast<const uint4*>(s.p + s.head);
     s.nfull = s.nbody / ((int64_t)T * UNROLL);
     s.rest = (int)(s.nbody - s.nfull * T * UNROLL);
     return s;
 }
 // The slice's first batch (full if there is a full batch, otherwise the masked one).
-template <int UNROLL, int T>
-__device__ __forceinline__ void load_first_batch(const Slice& s, uint4 (&q)[UNROLL]) {
+template <int UNROLL, int T, int DT>
+__device__ __forceinline__ void load_first_batch(const Slice<DT>& s, uint4 (&q)[UNROLL]) {
     const uint4* src = s.body + threadIdx.x;
     if (s.nfull > 0) {
 #pragma unroll
@@ -145,7 +191,7 @@ __device__ __forceinline__ void load_first_batch(const Slice& s, uint4 (&q)[UNRO
 #pragma unroll
         for (int k = 0; k < UNROLL; ++k) {
             const int i = (int)threadIdx.x + k * T;
-            q[k] = (i < s.rest) ? ld_stream(src + k * T) : make_uint4(kXNegInf2, kXNegInf2, kXNegInf2, kXNegInf2);
+            q[k] = (i < s.rest) ? ld_stream(src + k * T) : xneg_inf_vec<DT>();
         }
     }
 }
@@ -153,19 +199,19 @@ __device__ __forceinline__ void load_first_batch(const Slice& s, uint4 (&q)[UNRO
 // CTA-wide online (m, s) over a slice whose first batch `q` is already in flight.  Returns,
 // in every thread, the maximum M and the sum S relative to MF = max(rn(M*log2e), kFloor2).
 // Uses both slot sets (max then sum).
-template <int UNROLL, int POLY, int T>
-__device__ __forceinline__ void slice_lse(const Slice& sl, uint4 (&q)[UNROLL], float* slots, float& M, float& S) {
+template <int UNROLL, int POLY, int T, int DT>
+__device__ __forceinline__ void slice_lse(const Slice<DT>& sl, uint4 (&q)[UNROLL], float* slots, float& M, float& S) {
     Online o{-INFINITY, kFloor2, pack2(0.0f, 0.0f)};
     const f32x2 l2 = pack2(kLog2e, kLog2e);
     auto absorb_batch = [&](const uint4 (&v)[UNROLL]) {
-        uint32_t mx = xmax8(v[0]);
+        uint32_t mx = xmax_v<DT>(v[0]);
 #pragma unroll
-        for (int k = 1; k < UNROLL; ++k) mx = bf16x2_max_nan(mx, xmax8(v[k]));
-        raise_max(o, xhmax_of(mx));
+        for (int k = 1; k < UNROLL; ++k) mx = xmax_w<DT>(mx, xmax_v<DT>(v[k]));
+        raise_max(o, xhmax_of<DT>(mx));
         const f32x2 nmf2 = pack2(-o.mf, -o.mf);
-        f32x2 acc = sumexp8<POLY>(v[0], l2, nmf2);
+        f32x2 acc = sumexp_v<POLY, DT>(v[0], l2, nmf2);
 #pragma unroll
-        for (int k = 1; k < UNROLL; ++k) acc = add2(acc, sumexp8<POLY>(v[k], l2, nmf2));
+        for (int k = 1; k < UNROLL; ++k) acc = add2(acc, sumexp_v<POLY, DT>(v[k], l2, nmf2));
         o.s2 = add2(o.s2, acc);
     };
     absorb_batch(q);  // batch 0 (all padding when the slice has no body)
@@ -179,12 +225,12 @@ __device__ __forceinline__ void slice_lse(const Slice& sl, uint4 (&q)[UNROLL], f
 #pragma unroll
         for (int k = 0; k < UNROLL; ++k) {
             const int i = (int)threadIdx.x + k * T;
-            q[k] = (i < sl.rest) ? ld_stream(src + k * T) : make_uint4(kXNegInf2, kXNegInf2, kXNegInf2, kXNegInf2);
+            q[k] = (i < sl.rest) ? ld_stream(src + k * T) : xneg_inf_vec<DT>();
         }
         absorb_batch(q);
     }
-    if ((int64_t)threadIdx.x < sl.head) absorb_scalar(o, bf16_to_float(ld_stream_u16(sl.p + threadIdx.x)));
-    if (sl.tail0 + threadIdx.x < sl.n) absorb_scalar(o, bf16_to_float(ld_stream_u16(sl.p + sl.tail0 + threadIdx.x)));
+    if ((int64_t)threadIdx.x < sl.head) absorb_scalar(o, xload<DT>(sl.p + threadIdx.x));
+    if (sl.tail0 + threadIdx.x < sl.n) absorb_scalar(o, xload<DT>(sl.p + sl.tail0 + threadIdx.x));
 
     // NaN must win the max: fmaxf in cta_max would drop it, so it travels as +inf plus a flag
     const bool has_nan = (o.m != o.m) || (o.m == INFINITY);  // +inf makes inf - inf: NaN row as well
@@ -214,14 +260,14 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // ------------------------------------------------------------------ one CTA per row
-template <int UNROLL, int POLY, int MINB = 1, int T = kXentThreads>
+template <int UNROLL, int POLY, int MINB = 1, int T = kXentThreads, int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(T, MINB)
-xent_row_kernel(const uint16_t* __restrict__ logits, const int64_t* __restrict__ targets,
+xent_row_kernel(const typename XElem<DT>::type* __restrict__ logits, const int64_t* __restrict__ targets,
                 int64_t ignore_index, float* __restrict__ loss_rows, int64_t V) {
     __shared__ float slots[2 * kWarp];
     pdl_launch_dependents();
     const int64_t row = blockIdx.x;
-    const uint16_t* xr = logits + row * V;
+    const typename XElem<DT>::type* xr = logits + row * V;
     const int64_t t = targets[row];
     if (t == ignore_index || t < 0 || t >= V) {  // uniform across the CTA: nothing is read
         if (threadIdx.x == 0) loss_rows[row] = (t == ignore_index) ? 0.0f : __int_as_float(0x7fc00000);
@@ -229,22 +275,22 @@ xent_row_kernel(const uint16_t* __restrict__ logits, const int64_t* __restrict__
     }
     // (Requesting the first batch before the target is known was measured: no gain, and
     // ignored rows would be touched.)
-    const Slice sl = make_slice<UNROLL, T>(xr, 0, V);
+    const Slice<DT> sl = make_slice<UNROLL, T, DT>(xr, 0, V);
     uint4 q[UNROLL];
-    load_first_batch<UNROLL, T>(sl, q);
+    load_first_batch<UNROLL, T, DT>(sl, q);
     // the target logit is fetched now, under the row's own traffic, not after the reduction
-    const float xt = (threadIdx.x == 0) ? bf16_to_float(xr[t]) : 0.0f;
+    const float xt = (threadIdx.x == 0) ? xread<DT>(xr + t) : 0.0f;
     float M, S;
-    slice_lse<UNROLL, POLY, T>(sl, q, slots, M, S);
+    slice_lse<UNROLL, POLY, T, DT>(sl, q, slots, M, S);
     if (threadIdx.x == 0) loss_rows[row] = finish_loss(M, S, xt);
 }
 
 // ------------------------------------------------------------------ split row, phase 1
 // grid = (nsplit, rows).  Slice boundaries are multiples of 8 elements so an aligned row
 // keeps aligned slices.  partial[row * nsplit + split] = (M, S) of the slice.
-template <int UNROLL, int POLY>
+template <int UNROLL, int POLY, int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(kXentThreads)
-xent_split_kernel(const uint16_t* __restrict__ logits, const int64_t* __restrict__ targets,
+xent_split_kernel(const typename XElem<DT>::type* __restrict__ logits, const int64_t* __restrict__ targets,
                   int64_t ignore_index, float2* __restrict__ partial, int64_t V, int nsplit) {
     __shared__ float slots[2 * kWarp];
     pdl_launch_dependents();
@@ -256,11 +302,11 @@ xent_split_kernel(const uint16_t* __restrict__ logits, const int64_t* __restrict
     int64_t begin = ((groups * sp) / nsplit) << 3;
     int64_t end = ((groups * (sp + 1)) / nsplit) << 3;
     if (end > V) end = V;
-    const Slice sl = make_slice<UNROLL, kXentThreads>(logits + row * V, begin, end);
+    const Slice<DT> sl = make_slice<UNROLL, kXentThreads, DT>(logits + row * V, begin, end);
     uint4 q[UNROLL];
-    load_first_batch<UNROLL, kXentThreads>(sl, q);
+    load_first_batch<UNROLL, kXentThreads, DT>(sl, q);
     float M, S;
-    slice_lse<UNROLL, POLY, kXentThreads>(sl, q, slots, M, S);
+    slice_lse<UNROLL, POLY, kXentThreads, DT>(sl, q, slots, M, S);
     if (threadIdx.x == 0) partial[row * nsplit + sp] = make_float2(M, S);
 }
 
@@ -278,8 +324,9 @@ __device__ __forceinline__ double warp_sum_f64(double v) {
     return v;
 }
 
-static __global__ void __launch_bounds__(kFinishThreads)
-xent_finish_kernel(const uint16_t* __restrict__ logits, const int64_t* __restrict__ targets,
+template <int DT = AK_DTYPE_BF16>
+__global__ void __launch_bounds__(kFinishThreads)
+xent_finish_kernel(const typename XElem<DT>::type* __restrict__ logits, const int64_t* __restrict__ targets,
                    int64_t ignore_index, const float2* __restrict__ partial, int nsplit,
                    float* __restrict__ loss_rows, int64_t rows, int64_t V,
                    float* __restrict__ out_mean, double* __restrict__ out_pair) {
@@ -305,7 +352,7 @@ xent_finish_kernel(const uint16_t* __restrict__ logits, const int64_t* __restric
                     const float2 ps = __ldcg(pr + i);
                     S += ps.y * fast_exp2(fmaxf(ps.x * kLog2e, kFloor2) - MF);
                 }
-                loss = finish_loss(M, S, bf16_to_float(logits[r * V + t]));
+                loss = finish_loss(M, S, xread<DT>(logits + r * V + t));
             }
             loss_rows[r] = loss;
         }

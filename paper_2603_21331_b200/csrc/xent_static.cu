@@ -82,7 +82,7 @@ extern "C" int ak_xent_fwd_static(const void* logits, const int64_t* targets, in
         return AK_OK;
     }
     // merge the slices in split order, write the losses, then the fixed-order mean
-    xent_finish_kernel<<<1, kFinishThreads, 0, st>>>(lg, targets, ignore_index, scratch, rows > 0 ? nsplit : 0,
+    xent_finish_kernel<AK_DTYPE_BF16><<<1, kFinishThreads, 0, st>>>(lg, targets, ignore_index, scratch, rows > 0 ? nsplit : 0,
                                                     loss_rows, rows, V, loss_mean, nullptr);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;

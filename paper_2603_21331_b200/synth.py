@@ -35,8 +35,8 @@ def _gen(seed: int, device) -> torch.Generator:
 
 
 def _normal_bf16(rows: int, cols: int, std: float, mean: float, g: torch.Generator,
-                 device) -> torch.Tensor:
-    out = torch.empty((rows, cols), dtype=torch.bfloat16, device=device)
+                 device, dtype=torch.bfloat16) -> torch.Tensor:
+    out = torch.empty((rows, cols), dtype=dtype, device=device)
     step = max(1, _CHUNK_ELEMS // max(1, cols))
     for r0 in range(0, rows, step):
         r1 = min(rows, r0 + step)
@@ -56,17 +56,31 @@ def to_bits(t: torch.Tensor) -> np.ndarray:
     return t.detach().contiguous().cpu().view(torch.int16).numpy().view(np.uint16)
 
 
+def to_elems(t: torch.Tensor) -> np.ndarray:
+    """Tensor of any supported element type -> the array the CPU checker's *_dt functions take:
+    uint16 bit patterns for bf16 / fp16, float32 values for fp32."""
+    t = t.detach().contiguous().cpu()
+    if t.dtype in (torch.bfloat16, torch.float16):
+        return t.view(torch.int16).numpy().view(np.uint16)
+    if t.dtype == torch.float32:
+        return t.numpy()
+    raise TypeError("expected a bfloat16, float16 or float32 tensor")
+
+
+DTYPE_NAMES = {torch.bfloat16: "bf16", torch.float16: "f16", torch.float32: "f32"}
+
+
 def from_bits(bits: np.ndarray, device="cpu") -> torch.Tensor:
     """numpy uint16 bit patterns -> bf16 tensor on ``device``."""
     a = np.ascontiguousarray(bits, dtype=np.uint16)
     return torch.from_numpy(a.view(np.int16).copy()).view(torch.bfloat16).to(device)
 
 
-def rmsnorm_inputs(rows: int, D: int, seed: int, device="cpu"):
-    """(x bf16 [rows, D], w bf16 [D])."""
+def rmsnorm_inputs(rows: int, D: int, seed: int, device="cpu", dtype=torch.bfloat16):
+    """(x [rows, D], w [D]) of element type ``dtype`` (float32 draws rounded once to it)."""
     g = _gen(seed, device)
-    x = _normal_bf16(rows, D, 1.0, 0.0, g, device)
-    w = _normal_bf16(1, D, 0.1, 1.0, g, device).reshape(D)
+    x = _normal_bf16(rows, D, 1.0, 0.0, g, device, dtype)
+    w = _normal_bf16(1, D, 0.1, 1.0, g, device, dtype).reshape(D)
     return x, w
 
 
@@ -80,10 +94,11 @@ def layernorm_inputs(rows: int, D: int, seed: int, device="cpu"):
     return x, gamma, beta
 
 
-def softmax_inputs(rows: int, D: int, seed: int, device="cpu", mask_frac: float = 0.1):
-    """x bf16 [rows, D] with ~mask_frac of the rows causal-masked by trailing -inf."""
+def softmax_inputs(rows: int, D: int, seed: int, device="cpu", mask_frac: float = 0.1,
+                   dtype=torch.bfloat16):
+    """x [rows, D] with ~mask_frac of the rows causal-masked by trailing -inf."""
     g = _gen(seed, device)
-    x = _normal_bf16(rows, D, 4.0, 0.0, g, device)
+    x = _normal_bf16(rows, D, 4.0, 0.0, g, device, dtype)
     masked = torch.rand((rows,), device=device, generator=g) < mask_frac
     k = torch.randint(0, D, (rows,), device=device, generator=g)  # {0..D-1}
     k = torch.where(masked, k, torch.zeros_like(k))
@@ -97,10 +112,10 @@ def softmax_inputs(rows: int, D: int, seed: int, device="cpu", mask_frac: float 
 
 
 def xent_inputs(rows: int, V: int, seed: int, device="cpu", ignore_frac: float = 0.05,
-                ignore_index: int = IGNORE_INDEX):
-    """(logits bf16 [rows, V], targets int64 [rows])."""
+                ignore_index: int = IGNORE_INDEX, dtype=torch.bfloat16):
+    """(logits [rows, V] of element type ``dtype``, targets int64 [rows])."""
     g = _gen(seed, device)
-    logits = _normal_bf16(rows, V, 2.0, 0.0, g, device)
+    logits = _normal_bf16(rows, V, 2.0, 0.0, g, device, dtype)
     targets = torch.randint(0, V, (rows,), dtype=torch.int64, device=device, generator=g)
     ign = torch.rand((rows,), device=device, generator=g) < ignore_frac
     targets = torch.where(ign, torch.full_like(targets, ignore_index), targets)

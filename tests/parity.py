@@ -45,6 +45,37 @@ def assert_bf16_close(gpu: torch.Tensor, ref: np.ndarray, what: str = "", tight:
     return worst
 
 
+# fp16 / fp32 outputs (derived from the arithmetic, the benchmark's bar being stated for bf16
+# only): main bound = two units in the last place of the type relative to max(1, |ref|) for
+# fp16 (2 * 2^-11), 1e-5 for fp32 (fp32 accumulation, rsqrt / ex2 approximations of ~2^-22 and
+# the rounding of x*log2e at |x - m| up to ~100); tight bound = one rounding to nearest plus
+# the fp32 evaluation error, relative to |ref|, plus the type's subnormal quantum.
+DT_TOL = {torch.float16: 1.0e-3, torch.float32: 1.0e-5}
+DT_TIGHT = {torch.float16: (2.0 ** -11 * 1.02 + 4e-6, 2.0 ** -24), torch.float32: (1.0e-5, 1e-37)}
+
+
+def assert_close_dt(gpu: torch.Tensor, ref: np.ndarray, what: str = "", tight: bool = True):
+    """Element-wise comparison of a bf16 / fp16 / fp32 GPU output with the fp64 reference."""
+    if gpu.dtype == torch.bfloat16:
+        return assert_bf16_close(gpu, ref, what, tight)
+    got = gpu.detach().cpu().double().numpy().reshape(ref.shape)
+    nan_ref = np.isnan(ref)
+    assert np.array_equal(np.isnan(got), nan_ref), f"{what}: NaN pattern differs"
+    inf_ref = np.isinf(ref)
+    assert np.array_equal(np.isinf(got), inf_ref), f"{what}: inf pattern differs"
+    assert np.array_equal(got[inf_ref], ref[inf_ref]), f"{what}: inf sign differs"
+    fin = ~(nan_ref | inf_ref)
+    err = np.abs(got[fin] - ref[fin])
+    bound = DT_TOL[gpu.dtype] * np.maximum(1.0, np.abs(ref[fin]))
+    worst = float(np.max(err / bound)) if err.size else 0.0
+    assert worst <= 1.0, f"{what}: max err/bound = {worst:.3f}"
+    if tight and err.size:
+        rel, quantum = DT_TIGHT[gpu.dtype]
+        worst_t = float(np.max(err / (rel * np.abs(ref[fin]) + quantum)))
+        assert worst_t <= 1.0, f"{what}: exceeds one-rounding bound by {worst_t:.3f}x"
+    return worst
+
+
 def assert_loss_close(gpu: torch.Tensor, ref: np.ndarray, what: str = ""):
     got = gpu.detach().cpu().double().numpy().reshape(ref.shape)
     nan_ref = np.isnan(ref)
