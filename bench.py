@@ -498,7 +498,12 @@ SWEEP = (
        ("layernorm", 4096, 32768), ("layernorm", 8192, 4099)]
     + [("rowsum", 8192, 4096), ("rowsum", 16384, 4096), ("rowsum", 8192, 8192), ("rowsum", 65536, 1024), ("rowsum", 65536, 8192),
        ("rowsum", 4096, 128256), ("rowsum", 8192, 4099)]
+    # element-type variants ("op.f16" / "op.f32"): the paper's Table 4 shapes were measured in FP16
+    + [("rmsnorm.f16", 8192, 4096), ("rmsnorm.f16", 8192, 8192), ("rmsnorm.f32", 8192, 8192),
+       ("softmax.f16", 16384, 4096), ("softmax.f16", 16384, 8192), ("softmax.f32", 16384, 8192),
+       ("xent.f16", 4096, 50304), ("xent.f16", 4096, 128256), ("xent.f32", 4096, 50304)]
 )
+SWEEP_DTYPES = {"f16": torch.float16, "f32": torch.float32}
 
 
 def time_op(fn_for_set, nsets, iters=200, warmup=20):
@@ -564,6 +569,36 @@ def sweep_accuracy(ak, synth, op, rows, D, bufs):
         oracle.set_threads(cores)
         return ref, t_one * rows / len(idx), t_all * rows / len(idx)
 
+    if "." in op:
+        base, dts = op.split(".")
+        tol = {"f16": 1e-3, "f32": 1e-5}[dts] if base != "xent" else 1e-5
+        if base == "rmsnorm":
+            x, w, y = bufs
+            first = y.clone()
+            ak.ak_rmsnorm_fwd_dt(x, w, y, eps=1e-6)
+            same = torch.equal(first.view(torch.uint8), y.view(torch.uint8))
+            ref, t1, tn = timed_oracle(lambda: oracle.rmsnorm_dt(synth.to_elems(x[it]), synth.to_elems(w), 1e-6, dts))
+            got = y[it].cpu().double().numpy()
+        elif base == "softmax":
+            x, y = bufs
+            first = y.clone()
+            ak.ak_softmax_fwd_dt(x, y)
+            same = torch.equal(first.view(torch.uint8), y.view(torch.uint8))
+            ref, t1, tn = timed_oracle(lambda: oracle.softmax_dt(synth.to_elems(x[it]), dts))
+            got = y[it].cpu().double().numpy()
+        else:
+            lg, tg = bufs
+            first, _ = ak.ak_xent_fwd_dt(lg, tg)
+            loss, _ = ak.ak_xent_fwd_dt(lg, tg)
+            same = torch.equal(first.view(torch.int32), loss.view(torch.int32))
+            ref, t1, tn = timed_oracle(lambda: oracle.xent_dt(synth.to_elems(lg[it]), tg[it].cpu().numpy(), dts)[0])
+            got = loss[it].cpu().double().numpy()
+        torch.cuda.synchronize()
+        err = np.abs(got - ref)
+        return {"max_abs_err": float(err.max()),
+                "max_err_over_tolerance": float((err / (tol * np.maximum(1.0, np.abs(ref)))).max()),
+                "bitwise_repeat": bool(same), "sampled_rows": int(len(idx)),
+                "oracle_s_1_thread_scaled": t1, "oracle_s_all_threads_scaled": tn, "oracle_threads": cores}
     if op == "rmsnorm":
         x, w, y = bufs
         first = y.clone()
@@ -619,13 +654,25 @@ def run_sweep(ak, synth, dev, peak):
     rows_out = []
     only = os.environ.get("AK_SWEEP_OPS")
     for op, rows, D in SWEEP:
-        if only and op not in only.split(","):
+        if only and op not in only.split(",") and not ("." in op and "dtypes" in only.split(",")):
             continue
-        one_set = (2 if op in ("xent", "rowsum") else 4) * rows * D
+        base, _, dts = op.partition(".")
+        esize = 4 if dts == "f32" else 2
+        one_set = (1 if base in ("xent", "rowsum") else 2) * esize * rows * D
         nsets = int(max(1, min(64, -(-(1 << 30) // one_set))))
         sets = []
         for s in range(nsets):
-            if op == "rmsnorm":
+            if dts:
+                tdt = SWEEP_DTYPES[dts]
+                if base == "rmsnorm":
+                    x, w = synth.rmsnorm_inputs(rows, D, 7500 + s, device=dev, dtype=tdt)
+                    sets.append((x, w, torch.empty_like(x)))
+                elif base == "softmax":
+                    x = synth.softmax_inputs(rows, D, 7600 + s, device=dev, dtype=tdt)
+                    sets.append((x, torch.empty_like(x)))
+                else:
+                    sets.append(synth.xent_inputs(rows, D, 7700 + s, device=dev, dtype=tdt))
+            elif op == "rmsnorm":
                 x, w = synth.rmsnorm_inputs(rows, D, 7000 + s, device=dev)
                 sets.append((x, w, torch.empty_like(x)))
             elif op == "layernorm":
@@ -643,7 +690,19 @@ def run_sweep(ak, synth, dev, peak):
                 sets.append((lg, tg, torch.empty((rows,), dtype=torch.float32, device=dev),
                              torch.empty((1,), dtype=torch.float32, device=dev),
                              torch.empty((nws,), dtype=torch.uint8, device=dev) if nws else None))
-        if op == "rmsnorm":
+        if dts:
+            scale = esize // 2   # algorithmic_bytes counts 2-byte elements
+            if base == "rmsnorm":
+                fn = lambda i: ak.ak_rmsnorm_fwd_dt(sets[i][0], sets[i][1], sets[i][2], eps=1e-6)
+                nb = algorithmic_bytes(base, rows, D) * scale
+            elif base == "softmax":
+                fn = lambda i: ak.ak_softmax_fwd_dt(sets[i][0], sets[i][1])
+                nb = algorithmic_bytes(base, rows, D) * scale
+            else:
+                fn = lambda i: ak.ak_xent_fwd_dt(sets[i][0], sets[i][1])
+                nv = int((sets[0][1] != -100).sum())
+                nb = 2 * scale * D * nv + 12 * rows + 4
+        elif op == "rmsnorm":
             fn = lambda i: ak.ak_rmsnorm_fwd(sets[i][0], sets[i][1], sets[i][2], eps=1e-6)
             nb = algorithmic_bytes(op, rows, D)
         elif op == "layernorm":
@@ -671,7 +730,7 @@ def run_sweep(ak, synth, dev, peak):
     with open(os.path.join(ROOT, "gpurun_out", "sweep.json"), "w") as f:
         json.dump(rows_out, f, indent=1)
     for r in rows_out:
-        print(f"# {r['op']:8s} {r['rows']:7d} x {r['D']:6d}  {r['us_trimmed_mean']:9.1f} us  "
+        print(f"# {r['op']:11s} {r['rows']:7d} x {r['D']:6d}  {r['us_trimmed_mean']:9.1f} us  "
               f"{r['GB/s']:7.0f} GB/s  {100 * r['frac_of_8TBs']:5.1f}% of 8TB/s  "
               f"{100 * r['frac_of_measured_copy']:5.1f}% of copy", file=sys.stderr)
 
