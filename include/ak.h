@@ -102,6 +102,34 @@ int ak_softmax_fwd_dt(const void* x, void* y, int64_t rows, int64_t D,
 int ak_xent_fwd_dt(const void* logits, const int64_t* targets, int64_t ignore_index,
                    float* loss_rows, float* loss_mean, int64_t rows, int64_t V,
                    int dtype, void* cuda_stream, int path, int nsplit);
+/* ---------------------------------------------------------------------------------
+ * Vocabulary-parallel cross-entropy (the fused cross_ent of Table 3 with the vocabulary
+ * dimension sharded over ranks, as in tensor-parallel language-model heads).  Rank k holds
+ * logits_shard: device [rows, V_local] of `dtype`, the columns
+ * [vocab_start, vocab_start + V_local) of the full [rows, V_total] logits; targets index the
+ * FULL vocabulary and are the same on every rank.
+ *   1. ak_xent_vp_partial on every rank: writes `partial` = rows * (nsplit + 1) pairs of fp32
+ *      (ak_xent_vp_partial_bytes): per row, nsplit online (max, sum-exp) pairs of the shard's
+ *      slices, then (x[r, t], 1) if this shard owns column t, else (0, 0).  Rows whose target
+ *      is ignore_index or outside [0, V_total) are neither read nor written.
+ *   2. the caller all-gathers the partial buffers in rank order into [nranks][rows][nsplit+1]
+ *      pairs (16 * (nsplit + 1) bytes per row and rank; the only exchange).
+ *   3. ak_xent_vp_merge on every rank: merges in (rank, slice) order and writes loss_rows
+ *      [rows] and, if not NULL, loss_mean [1], with the conventions of ak_xent_fwd; identical
+ *      bits on all ranks.  A valid target owned by no shard or by several gives NaN.
+ * nsplit (1..64) must be the same on all ranks; ak_xent_vp_nsplit gives the dispatcher's
+ * choice for (rows, V_local) (1 when rows alone fill the GPU).  All buffers are caller-owned;
+ * nothing is allocated; each call enqueues one or two kernels on `cuda_stream`.
+ */
+int ak_xent_vp_nsplit(int64_t rows, int64_t V_local);
+size_t ak_xent_vp_partial_bytes(int64_t rows, int nsplit);
+int ak_xent_vp_partial(const void* logits_shard, const int64_t* targets, int64_t ignore_index,
+                       int64_t vocab_start, int64_t V_total, void* partial,
+                       int64_t rows, int64_t V_local, int nsplit, int dtype, void* cuda_stream);
+int ak_xent_vp_merge(const void* partials, int nranks, int nsplit, const int64_t* targets,
+                     int64_t ignore_index, int64_t V_total, float* loss_rows, float* loss_mean,
+                     int64_t rows, void* cuda_stream);
+
 /* Path the dispatcher picks for op (0 = RMSNorm, 1 = softmax) at this shape, alignment and
  * element type; -1 for an unknown op or dtype.  Pure function; no CUDA calls. */
 int ak_choose_path_dt(int op, int64_t rows, int64_t D, int aligned16, int dtype);

@@ -39,6 +39,10 @@ SIGNATURES = {
     "ak_softmax_fwd_dt": (_int, [_p, _p, _i64, _i64, _int, _p, _int]),
     "ak_xent_fwd_dt": (_int, [_p, _p, _i64, _p, _p, _i64, _i64, _int, _p, _int, _int]),
     "ak_choose_path_dt": (_int, [_int, _i64, _i64, _int, _int]),
+    "ak_xent_vp_nsplit": (_int, [_i64, _i64]),
+    "ak_xent_vp_partial_bytes": (_sz, [_i64, _int]),
+    "ak_xent_vp_partial": (_int, [_p, _p, _i64, _i64, _i64, _p, _i64, _i64, _int, _int, _p]),
+    "ak_xent_vp_merge": (_int, [_p, _int, _int, _p, _i64, _i64, _p, _p, _i64, _p]),
     "ak_layernorm_fwd": (_int, [_p, _p, _p, _p, _i64, _i64, _f32, _p]),
     "ak_layernorm_fwd_path": (_int, [_p, _p, _p, _p, _i64, _i64, _f32, _p, _int]),
     "ak_rowsum_fwd": (_int, [_p, _p, _i64, _i64, _p]),
@@ -189,6 +193,53 @@ def ak_xent_fwd_dt(logits: torch.Tensor, targets: torch.Tensor, ignore_index: in
     _check(lib().ak_xent_fwd_dt(logits.data_ptr(), targets.data_ptr(), ignore_index, loss_rows.data_ptr(),
                                 loss_mean.data_ptr() if want_mean else None, rows, V, dt,
                                 _stream_ptr(stream), path, nsplit), "ak_xent_fwd_dt")
+    return loss_rows, loss_mean
+
+
+def ak_xent_vp_nsplit(rows: int, V_local: int) -> int:
+    return int(lib().ak_xent_vp_nsplit(rows, V_local))
+
+
+def ak_xent_vp_partial(logits_shard: torch.Tensor, targets: torch.Tensor, vocab_start: int, V_total: int,
+                       nsplit: int = 0, ignore_index: int = -100, partial: Optional[torch.Tensor] = None,
+                       stream=None) -> torch.Tensor:
+    """Phase 1 of the vocabulary-parallel cross-entropy on this rank's [rows, V_local] shard.
+    Returns the partial buffer: float32 [rows, nsplit + 1, 2]."""
+    dt = _dev_dt(logits_shard, "logits_shard", 2)
+    rows, V_local = logits_shard.shape
+    if not (targets.is_cuda and targets.dtype == torch.int64 and targets.shape == (rows,)
+            and targets.is_contiguous()):
+        raise TypeError("targets must be a contiguous CUDA int64 tensor [rows]")
+    if nsplit == 0:
+        nsplit = ak_xent_vp_nsplit(rows, V_local)
+    if partial is None:
+        # zero-filled so that the entries of unread rows are defined bytes for the exchange
+        partial = torch.zeros((rows, nsplit + 1, 2), dtype=torch.float32, device=logits_shard.device)
+    if not (partial.is_cuda and partial.dtype == torch.float32 and partial.shape == (rows, nsplit + 1, 2)
+            and partial.is_contiguous()):
+        raise TypeError("partial must be a contiguous CUDA float32 tensor [rows, nsplit + 1, 2]")
+    _check(lib().ak_xent_vp_partial(logits_shard.data_ptr(), targets.data_ptr(), ignore_index, vocab_start,
+                                    V_total, partial.data_ptr(), rows, V_local, nsplit, dt,
+                                    _stream_ptr(stream)), "ak_xent_vp_partial")
+    return partial
+
+
+def ak_xent_vp_merge(partials: torch.Tensor, targets: torch.Tensor, V_total: int, ignore_index: int = -100,
+                     want_mean: bool = True, stream=None) -> Tuple[torch.Tensor, Optional[torch.Tensor]]:
+    """Phase 2: ``partials`` = float32 [nranks, rows, nsplit + 1, 2] (all ranks' buffers in rank
+    order).  Returns (loss_rows fp32 [rows], loss_mean fp32 [1] or None)."""
+    if not (partials.is_cuda and partials.dtype == torch.float32 and partials.dim() == 4
+            and partials.shape[3] == 2 and partials.is_contiguous()):
+        raise TypeError("partials must be a contiguous CUDA float32 tensor [nranks, rows, nsplit + 1, 2]")
+    nranks, rows, ns1, _ = partials.shape
+    if not (targets.is_cuda and targets.dtype == torch.int64 and targets.shape == (rows,)
+            and targets.is_contiguous()):
+        raise TypeError("targets must be a contiguous CUDA int64 tensor [rows]")
+    loss_rows = torch.empty((rows,), dtype=torch.float32, device=partials.device)
+    loss_mean = torch.empty((1,), dtype=torch.float32, device=partials.device) if want_mean else None
+    _check(lib().ak_xent_vp_merge(partials.data_ptr(), nranks, ns1 - 1, targets.data_ptr(), ignore_index,
+                                  V_total, loss_rows.data_ptr(), loss_mean.data_ptr() if want_mean else None,
+                                  rows, _stream_ptr(stream)), "ak_xent_vp_merge")
     return loss_rows, loss_mean
 
 

@@ -110,6 +110,43 @@ int ak_xent_fwd_dt(const void* logits, const int64_t* targets, int64_t ignore_in
     return xent_dispatch(logits, targets, ignore_index, loss_rows, loss_mean, rows, V, nullptr, 0, true,
                          static_cast<cudaStream_t>(cuda_stream), path, nsplit, dtype);
 }
+int ak_xent_vp_nsplit(int64_t rows, int64_t V_local) {
+    int ns = 1;
+    if (rows > 0 && V_local > 0) xent_choose(rows, V_local, &ns);
+    return ns;
+}
+size_t ak_xent_vp_partial_bytes(int64_t rows, int nsplit) {
+    if (rows <= 0 || nsplit < 1) return 0;
+    return (size_t)rows * (size_t)(nsplit + 1) * sizeof(float2);
+}
+int ak_xent_vp_partial(const void* logits_shard, const int64_t* targets, int64_t ignore_index,
+                       int64_t vocab_start, int64_t V_total, void* partial, int64_t rows, int64_t V_local,
+                       int nsplit, int dtype, void* cuda_stream) {
+    if (!known_dtype(dtype)) return AK_ERR_ARG;
+    if (rows != 0 && (!logits_shard || !targets || !partial)) return AK_ERR_NULL;
+    if (int s = check_rows_cols(rows, V_local)) return s;
+    if (vocab_start < 0 || V_total < V_local || vocab_start > V_total - V_local) return AK_ERR_SHAPE;
+    if (!is_aligned(logits_shard, (size_t)dtype_bytes(dtype)) || !is_aligned(targets, 8) || !is_aligned(partial, 8))
+        return AK_ERR_ALIGN;
+    if (nsplit < 1 || nsplit > 64) return AK_ERR_ARG;
+    if (rows > 2147483647LL) return AK_ERR_SHAPE;
+    if (rows == 0) return AK_OK;
+    return xent_vp_partial_launch(logits_shard, targets, ignore_index, vocab_start, V_total, partial, rows, V_local,
+                                  nsplit, dtype, static_cast<cudaStream_t>(cuda_stream));
+}
+int ak_xent_vp_merge(const void* partials, int nranks, int nsplit, const int64_t* targets, int64_t ignore_index,
+                     int64_t V_total, float* loss_rows, float* loss_mean, int64_t rows, void* cuda_stream) {
+    if (rows != 0 && (!partials || !targets || !loss_rows)) return AK_ERR_NULL;
+    if (rows < 0 || V_total <= 0) return AK_ERR_SHAPE;
+    if (nranks < 1 || nranks > 4096 || nsplit < 1 || nsplit > 64) return AK_ERR_ARG;
+    if (!is_aligned(partials, 8) || !is_aligned(targets, 8) || !is_aligned(loss_rows, 4) ||
+        (loss_mean && !is_aligned(loss_mean, 4)))
+        return AK_ERR_ALIGN;
+    if (rows > 2147483647LL * 128) return AK_ERR_SHAPE;
+    return xent_vp_merge_launch(partials, nranks, nsplit, targets, ignore_index, V_total, loss_rows, loss_mean, rows,
+                                static_cast<cudaStream_t>(cuda_stream));
+}
+
 int ak_choose_path_dt(int op, int64_t rows, int64_t D, int aligned16, int dtype) {
     if (!known_dtype(dtype)) return -1;
     if (op == 0) return rmsnorm_choose(rows, D, aligned16 != 0, dtype);

@@ -266,6 +266,12 @@ int xent_mean_launch(const float* loss_rows, const int64_t* targets, int64_t ign
                      float* loss_mean, cudaStream_t st);
 int xent_sum_count_launch(const float* loss_rows, const int64_t* targets, int64_t ignore_index, int64_t rows,
                           double* sum_count, cudaStream_t st);
+// Vocabulary-parallel cross-entropy (defined in xent_vp.cu).
+int xent_vp_partial_launch(const void* logits, const int64_t* targets, int64_t ignore_index, int64_t vocab_start,
+                           int64_t V_total, void* part, int64_t rows, int64_t V_local, int nsplit, int dtype,
+                           cudaStream_t st);
+int xent_vp_merge_launch(const void* parts, int nranks, int nsplit, const int64_t* targets, int64_t ignore_index,
+                         int64_t V_total, float* loss_rows, float* loss_mean, int64_t rows, cudaStream_t st);
 int xent_mean_merge_launch(const double* pairs, int64_t n, float* loss_mean, cudaStream_t st);
 int layernorm_dispatch(const void* x, const void* gamma, const void* beta, void* y, int64_t rows, int64_t D,
                        float eps, cudaStream_t st, int path);

@@ -1,0 +1,139 @@
+// Vocabulary-parallel cross-entropy: the logits' last dimension is sharded over ranks
+// (tensor parallelism), rank k holding columns [vocab_start_k, vocab_start_k + V_local_k).
+//
+//   phase 1 (every rank, its own shard)  ak_xent_vp_partial: per row, nsplit slices' online
+//           (max, sum-exp) pairs and the target logit if this shard owns the target column
+//   exchange                             one all-gather of rows * (nsplit + 1) * 8 bytes per rank
+//   phase 2 (every rank, identical bits) ak_xent_vp_merge: merge all ranks' pairs in
+//           (rank, slice) order, add the owner's target logit, then the fixed-order mean
+//
+// This is the split-row layout of the single-GPU kernel with the slices living on different
+// GPUs: the same slice_lse, the same merge arithmetic, the same loss assembly.  The exchange
+// is 16 bytes per row against 2 * V_local bytes per row of local streaming (1 : 16000 at
+// V_local = 128k), so it is latency-bound and there is no tile whose transfer could overlap
+// the math; it goes through the communication library as one small collective.
+#include "xent_kernels.cuh"
+
+namespace ak {
+namespace {
+
+// grid = (rows, nsplit).  part[row * (nsplit + 1) + s] = (M, S) of slice s of this shard;
+// part[row * (nsplit + 1) + nsplit] = (x_t, 1) if the shard owns column t, else (0, 0).
+// Rows whose target is ignore_index or outside [0, V_total) are not read and their entries
+// are not written (the merge never looks at them).
+template <int UNROLL, int POLY, int MINB, int T, int DT>
+__global__ void __launch_bounds__(T, MINB)
+xent_vp_partial_kernel(const typename XElem<DT>::type* __restrict__ logits, const int64_t* __restrict__ targets,
+                       int64_t ignore_index, int64_t vocab_start, int64_t V_total, float2* __restrict__ part,
+                       int64_t V_local, int nsplit) {
+    __shared__ float slots[2 * kWarp];
+    const int64_t row = blockIdx.x;
+    const int sp = blockIdx.y;
+    const int64_t t = targets[row];
+    if (t == ignore_index || t < 0 || t >= V_total) return;
+    const typename XElem<DT>::type* xr = logits + row * V_local;
+    const int64_t groups = (V_local + 7) >> 3;
+    int64_t begin = ((groups * sp) / nsplit) << 3;
+    int64_t end = ((groups * (sp + 1)) / nsplit) << 3;
+    if (end > V_local) end = V_local;
+    const Slice<DT> sl = make_slice<UNROLL, T, DT>(xr, begin, end);
+    uint4 q[UNROLL];
+    load_first_batch<UNROLL, T, DT>(sl, q);
+    float2 mine = make_float2(0.0f, 0.0f);
+    if (sp == 0 && threadIdx.x == 0) {
+        const int64_t tl = t - vocab_start;
+        if (tl >= 0 && tl < V_local) mine = make_float2(xread<DT>(xr + tl), 1.0f);
+    }
+    float M, S;
+    slice_lse<UNROLL, POLY, T, DT>(sl, q, slots, M, S);
+    if (threadIdx.x == 0) {
+        float2* pr = part + row * (nsplit + 1);
+        pr[sp] = make_float2(M, S);
+        if (sp == 0) pr[nsplit] = mine;
+    }
+}
+
+// One thread per row: all ranks' slices in (rank, slice) order, exactly the arithmetic of the
+// single-GPU split merge.  parts = [nranks][rows][nsplit + 1] pairs.
+constexpr int kVpMergeThreads = 128;
+__global__ void __launch_bounds__(kVpMergeThreads)
+xent_vp_merge_kernel(const float2* __restrict__ parts, int nranks, int nsplit, const int64_t* __restrict__ targets,
+                     int64_t ignore_index, int64_t V_total, float* __restrict__ loss_rows, int64_t rows) {
+    const int64_t r = (int64_t)blockIdx.x * kVpMergeThreads + threadIdx.x;
+    if (r >= rows) return;
+    const int64_t t = targets[r];
+    float loss;
+    if (t == ignore_index) {
+        loss = 0.0f;
+    } else if (t < 0 || t >= V_total) {
+        loss = __int_as_float(0x7fc00000);
+    } else {
+        const int64_t stride = (int64_t)rows * (nsplit + 1);
+        const float2* pr = parts + r * (nsplit + 1);
+        float M = -INFINITY;
+        for (int k = 0; k < nranks; ++k)
+            for (int i = 0; i < nsplit; ++i) M = fmaxf(M, __ldg(pr + k * stride + i).x);
+        const float MF = fmaxf(M * kLog2e, kFloor2);
+        float S = 0.0f, xt = 0.0f, owners = 0.0f;
+        for (int k = 0; k < nranks; ++k) {
+            for (int i = 0; i < nsplit; ++i) {
+                const float2 ps = __ldg(pr + k * stride + i);
+                S += ps.y * fast_exp2(fmaxf(ps.x * kLog2e, kFloor2) - MF);
+            }
+            const float2 own = __ldg(pr + k * stride + nsplit);
+            if (own.y != 0.0f) { xt = own.x; owners += 1.0f; }
+        }
+        // exactly one shard owns a valid target when the shards tile [0, V_total)
+        loss = (owners == 1.0f) ? finish_loss(M, S, xt) : __int_as_float(0x7fc00000);
+    }
+    loss_rows[r] = loss;
+}
+
+template <int DT>
+int partial_t(const void* logits, const int64_t* targets, int64_t ignore_index, int64_t vocab_start, int64_t V_total,
+              float2* part, int64_t rows, int64_t V_local, int nsplit, cudaStream_t st) {
+    using elem_t = typename XElem<DT>::type;
+    const elem_t* lg = static_cast<const elem_t*>(logits);
+    const dim3 grid((unsigned)rows, (unsigned)nsplit);
+    if (nsplit == 1)   // the single-GPU row layout: 128 threads x 8 vectors, 64 registers
+        xent_vp_partial_kernel<8, 2, 8, 128, DT><<<grid, 128, 0, st>>>(lg, targets, ignore_index, vocab_start, V_total,
+                                                                      part, V_local, nsplit);
+    else
+        xent_vp_partial_kernel<4, 2, 1, kXentThreads, DT><<<grid, kXentThreads, 0, st>>>(
+            lg, targets, ignore_index, vocab_start, V_total, part, V_local, nsplit);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+}
+
+}  // namespace
+
+int xent_vp_partial_launch(const void* logits, const int64_t* targets, int64_t ignore_index, int64_t vocab_start,
+                           int64_t V_total, void* part, int64_t rows, int64_t V_local, int nsplit, int dtype,
+                           cudaStream_t st) {
+    float2* p = static_cast<float2*>(part);
+    switch (dtype) {
+        case AK_DTYPE_BF16:
+            return partial_t<AK_DTYPE_BF16>(logits, targets, ignore_index, vocab_start, V_total, p, rows, V_local, nsplit, st);
+        case AK_DTYPE_F16:
+            return partial_t<AK_DTYPE_F16>(logits, targets, ignore_index, vocab_start, V_total, p, rows, V_local, nsplit, st);
+        case AK_DTYPE_F32:
+            return partial_t<AK_DTYPE_F32>(logits, targets, ignore_index, vocab_start, V_total, p, rows, V_local, nsplit, st);
+        default:
+            return AK_ERR_ARG;
+    }
+}
+
+int xent_vp_merge_launch(const void* parts, int nranks, int nsplit, const int64_t* targets, int64_t ignore_index,
+                         int64_t V_total, float* loss_rows, float* loss_mean, int64_t rows, cudaStream_t st) {
+    if (rows > 0) {
+        const unsigned grid = (unsigned)((rows + kVpMergeThreads - 1) / kVpMergeThreads);
+        xent_vp_merge_kernel<<<grid, kVpMergeThreads, 0, st>>>(static_cast<const float2*>(parts), nranks, nsplit, targets,
+                                                              ignore_index, V_total, loss_rows, rows);
+        count_launch();
+        if (cudaGetLastError() != cudaSuccess) return AK_ERR_CUDA;
+    }
+    if (loss_mean == nullptr) return AK_OK;
+    return xent_mean_launch(loss_rows, targets, ignore_index, rows, loss_mean, st);
+}
+
+}  // namespace ak

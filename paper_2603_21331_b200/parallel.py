@@ -44,6 +44,46 @@ def merge_pairs_host(pairs: torch.Tensor) -> float:
     return total / count if count > 0 else float("nan")
 
 
+def shard_vocab(V: int, rank: int, world: int) -> Tuple[int, int]:
+    """Contiguous block [begin, end) of the vocabulary owned by ``rank``.  Block starts are
+    multiples of 8 columns (16-byte aligned shards for the 16-bit types); the last rank takes
+    the remainder."""
+    if world < 1 or not (0 <= rank < world) or V < 0:
+        raise ValueError("bad shard request")
+    per = -(-V // world)
+    per = -(-per // 8) * 8
+    begin = min(V, rank * per)
+    return begin, min(V, begin + per)
+
+
+def gather_partials(partial: torch.Tensor, group=None) -> torch.Tensor:
+    """All-gather the per-rank partial buffers [rows, nsplit + 1, 2] -> [world, rows, nsplit + 1, 2]
+    in rank order (the only exchange of the vocabulary-parallel cross-entropy)."""
+    if partial.dtype != torch.float32 or partial.dim() != 3 or partial.shape[2] != 2:
+        raise TypeError("partial must be a float32 tensor [rows, nsplit + 1, 2]")
+    world = dist.get_world_size(group)
+    out = torch.empty((world,) + tuple(partial.shape), dtype=torch.float32, device=partial.device)
+    dist.all_gather_into_tensor(out.view(-1), partial.contiguous().view(-1), group=group)
+    return out
+
+
+def vocab_parallel_xent(logits_shard: torch.Tensor, targets: torch.Tensor, vocab_start: int, V_total: int,
+                        ignore_index: int = -100, group=None, stream=None, nsplit: int = 0):
+    """Cross-entropy of [rows, V_total] logits whose columns are sharded over the ranks of
+    ``group``: this rank passes its [rows, V_local] block and its first column.  Returns
+    (loss_rows, loss_mean), bit-identical on every rank.  ``nsplit`` must agree across ranks;
+    0 derives it from (rows, largest shard), which is the same everywhere for block shards."""
+    from . import binding
+    rows, V_local = logits_shard.shape
+    if nsplit == 0:
+        world = dist.get_world_size(group)
+        nsplit = binding.ak_xent_vp_nsplit(rows, shard_vocab(V_total, 0, world)[1])
+    part = binding.ak_xent_vp_partial(logits_shard, targets, vocab_start, V_total, nsplit, ignore_index,
+                                      stream=stream)
+    parts = gather_partials(part, group)
+    return binding.ak_xent_vp_merge(parts, targets, V_total, ignore_index, stream=stream)
+
+
 def global_xent_mean(loss_rows: torch.Tensor, targets: torch.Tensor, ignore_index: int = -100,
                      group=None, stream=None) -> torch.Tensor:
     """Mean cross-entropy over all ranks' rows (device tensors; kernels from libak)."""

@@ -65,6 +65,31 @@ def test_validation_rejects_before_any_cuda_call():
     assert l.ak_rowsum_fwd(P + 1, P, 1, 8, None) == 3
     assert l.ak_rowsum_fwd(P, P + 2, 1, 8, None) == 3                # fp32 sums need 4 B
     assert l.ak_rowsum_fwd(P, P, 0, 8, None) == 0
+    # element-type variants: unknown dtype, fp32 alignment
+    assert l.ak_rmsnorm_fwd_dt(P, P, P, 1, 8, 1e-6, 7, None, 0) == 4
+    assert l.ak_rmsnorm_fwd_dt(P + 2, P, P, 1, 8, 1e-6, 2, None, 0) == 3     # fp32 needs 4 B
+    assert l.ak_softmax_fwd_dt(P, P + 2, 1, 8, 2, None, 0) == 3
+    assert l.ak_softmax_fwd_dt(P, P, 1, 8, -1, None, 0) == 4
+    assert l.ak_xent_fwd_dt(P + 2, P, -100, P, P, 1, 8, 2, None, 0, 0) == 3
+    assert l.ak_xent_fwd_dt(P, P, -100, P, P, 1, 8, 3, None, 0, 0) == 4
+    assert l.ak_choose_path_dt(0, 8192, 4096, 1, 2) == ak.AK_PATH_CTA       # 16 KiB fp32 rows
+    assert l.ak_choose_path_dt(0, 8192, 1024, 1, 2) == ak.AK_PATH_WARP
+    assert l.ak_choose_path_dt(0, 8192, 1022, 1, 2) == ak.AK_PATH_GENERIC   # 4088 B: not a multiple of 16
+    assert l.ak_choose_path_dt(1, 8192, 8192, 1, 2) == ak.AK_PATH_SMEM      # 32 KiB fp32 softmax rows
+    assert l.ak_choose_path_dt(1, 8192, 8192, 1, 1) == ak.AK_PATH_CTA
+    assert l.ak_choose_path_dt(2, 1, 8, 1, 0) == -1 and l.ak_choose_path_dt(0, 1, 8, 1, 9) == -1
+    # vocabulary-parallel cross-entropy
+    assert l.ak_xent_vp_partial_bytes(10, 3) == 10 * 4 * 8 and l.ak_xent_vp_partial_bytes(0, 3) == 0
+    assert l.ak_xent_vp_nsplit(4096, 16032) == 1 and l.ak_xent_vp_nsplit(16, 16032) == 1
+    assert l.ak_xent_vp_nsplit(16, 64128) == 7
+    assert l.ak_xent_vp_partial(None, P, -100, 0, 64, P, 1, 32, 1, 0, None) == 1
+    assert l.ak_xent_vp_partial(P, P, -100, 40, 64, P, 1, 32, 1, 0, None) == 2   # shard sticks out of the vocabulary
+    assert l.ak_xent_vp_partial(P, P, -100, 0, 64, P, 1, 0, 1, 0, None) == 2     # empty shard
+    assert l.ak_xent_vp_partial(P, P, -100, 0, 64, P, 1, 32, 0, 0, None) == 4
+    assert l.ak_xent_vp_partial(P, P, -100, 0, 64, P + 4, 1, 32, 1, 0, None) == 3
+    assert l.ak_xent_vp_merge(None, 2, 1, P, -100, 64, P, P, 1, None) == 1
+    assert l.ak_xent_vp_merge(P, 0, 1, P, -100, 64, P, P, 1, None) == 4
+    assert l.ak_xent_vp_merge(P, 2, 65, P, -100, 64, P, P, 1, None) == 4
     assert l.ak_softmax_fwd(None, P, 1, 8, None) == 1
     assert l.ak_softmax_fwd(P, P, 1, -3, None) == 2
     assert l.ak_softmax_fwd(P, P + 1, 1, 8, None) == 3

@@ -66,3 +66,40 @@ def test_merge_pairs_host_conventions():
     assert np.isnan(parallel.merge_pairs_host(torch.zeros((2, 2), dtype=torch.float64)))
     p = torch.tensor([[3.0, 2.0], [0.0, 0.0], [9.0, 2.0]], dtype=torch.float64)
     assert parallel.merge_pairs_host(p) == 3.0
+
+
+def _vp_worker(rank, world, port, out_dir):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        rows, nsplit = 5, 3
+        # a recognisable partial buffer: value encodes (rank, row, slot, component)
+        part = torch.arange(rows * (nsplit + 1) * 2, dtype=torch.float32).view(rows, nsplit + 1, 2) + 1000.0 * rank
+        parts = parallel.gather_partials(part)
+        assert parts.shape == (world, rows, nsplit + 1, 2)
+        for k in range(world):
+            assert torch.equal(parts[k], part - 1000.0 * rank + 1000.0 * k)   # rank order, layout kept
+        np.save(os.path.join(out_dir, f"parts{rank}.npy"), parts.numpy())
+    finally:
+        dist.destroy_process_group()
+
+
+def test_vocab_parallel_exchange_two_ranks(tmp_path):
+    """The one exchange of the vocabulary-parallel cross-entropy: every rank ends with all
+    ranks' partial buffers, in rank order, bit-identical everywhere."""
+    world = 2
+    mp.spawn(_vp_worker, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    a, b = (np.load(tmp_path / f"parts{r}.npy") for r in range(world))
+    assert np.array_equal(a, b)
+
+
+def test_shard_vocab_tiles_the_vocabulary_with_aligned_starts():
+    for V in (1, 9, 1000, 4099, 32000, 128256, 128257):
+        for world in (1, 2, 3, 8):
+            spans = [parallel.shard_vocab(V, r, world) for r in range(world)]
+            assert spans[0][0] == 0 and spans[-1][1] == V
+            assert all(spans[i][1] == spans[i + 1][0] for i in range(world - 1))
+            assert all(b % 8 == 0 or b == V for b, _ in spans)
+    with pytest.raises(ValueError):
+        parallel.shard_vocab(8, 3, 2)
