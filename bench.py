@@ -488,7 +488,7 @@ def run_ours(args, rank, world, local_rank):
 
 
 # --------------------------------------------------------------------------- per-shape sweep
-SWEEP = (
+SWEEP = list(
     [("rmsnorm", 8192, d) for d in (1024, 2048, 4096, 8192, 16384)]
     + [("rmsnorm", r, 4096) for r in (1, 17, 65536, 262144)] + [("rmsnorm", 8192, 4099)]
     + [("softmax", 16384, d) for d in (512, 1024, 2048, 4096, 8192, 32768)]
@@ -504,6 +504,9 @@ SWEEP = (
        ("xent.f16", 4096, 50304), ("xent.f16", 4096, 128256), ("xent.f32", 4096, 50304)]
 )
 SWEEP_DTYPES = {"f16": torch.float16, "f32": torch.float32}
+# vocabulary-parallel cross-entropy as one of 8 ranks sees it: its [rows, V/8] shard -> partial
+# kernel, then the merge over 8 ranks' partial buffers (the 7 others' stand-ins are copies)
+SWEEP += [("xent_vp8", 4096, 128256 // 8), ("xent_vp8", 16384, 128256 // 8)]
 
 
 def time_op(fn_for_set, nsets, iters=200, warmup=20):
@@ -569,6 +572,26 @@ def sweep_accuracy(ak, synth, op, rows, D, bufs):
         oracle.set_threads(cores)
         return ref, t_one * rows / len(idx), t_all * rows / len(idx)
 
+    if op == "xent_vp8":
+        lg, tg, parts = bufs
+        V = 8 * D
+        tgt = torch.where(tg == -100, tg, tg % D)   # keep the targets inside this shard
+        part = ak.ak_xent_vp_partial(lg, tgt, 0, V, 1)
+        # the other seven shards: all-(-inf) columns contribute (max, sum) = (-inf, 0)
+        stack = torch.zeros((8,) + tuple(part.shape), dtype=torch.float32, device=part.device)
+        stack[:, :, 0, 0] = float("-inf")
+        stack[0] = part
+        loss, _ = ak.ak_xent_vp_merge(stack, tgt, V)
+        again, _ = ak.ak_xent_vp_merge(stack, tgt, V)
+        same = torch.equal(loss.view(torch.int32), again.view(torch.int32))
+        ref, t1, tn = timed_oracle(lambda: oracle.xent(synth.to_bits(lg[it]), tgt[it].cpu().numpy())[0])
+        got = loss[it].cpu().double().numpy()
+        torch.cuda.synchronize()
+        err = np.abs(got - ref)
+        return {"max_abs_err": float(err.max()),
+                "max_err_over_tolerance": float((err / (1e-5 * np.maximum(1.0, np.abs(ref)))).max()),
+                "bitwise_repeat": bool(same), "sampled_rows": int(len(idx)),
+                "oracle_s_1_thread_scaled": t1, "oracle_s_all_threads_scaled": tn, "oracle_threads": cores}
     if "." in op:
         base, dts = op.split(".")
         tol = {"f16": 1e-3, "f32": 1e-5}[dts] if base != "xent" else 1e-5
@@ -658,11 +681,14 @@ def run_sweep(ak, synth, dev, peak):
             continue
         base, _, dts = op.partition(".")
         esize = 4 if dts == "f32" else 2
-        one_set = (1 if base in ("xent", "rowsum") else 2) * esize * rows * D
+        one_set = (1 if base in ("xent", "rowsum", "xent_vp8") else 2) * esize * rows * D
         nsets = int(max(1, min(64, -(-(1 << 30) // one_set))))
         sets = []
         for s in range(nsets):
-            if dts:
+            if op == "xent_vp8":
+                lg, tg = synth.xent_inputs(rows, D, 7800 + s, device=dev)
+                sets.append((lg, tg, torch.zeros((8, rows, 2, 2), dtype=torch.float32, device=dev)))
+            elif dts:
                 tdt = SWEEP_DTYPES[dts]
                 if base == "rmsnorm":
                     x, w = synth.rmsnorm_inputs(rows, D, 7500 + s, device=dev, dtype=tdt)
@@ -690,7 +716,14 @@ def run_sweep(ak, synth, dev, peak):
                 sets.append((lg, tg, torch.empty((rows,), dtype=torch.float32, device=dev),
                              torch.empty((1,), dtype=torch.float32, device=dev),
                              torch.empty((nws,), dtype=torch.uint8, device=dev) if nws else None))
-        if dts:
+        if op == "xent_vp8":
+            def fn(i):
+                lg, tg, parts = sets[i]
+                ak.ak_xent_vp_partial(lg, tg, 0, 8 * D, 1, partial=parts[0])
+                ak.ak_xent_vp_merge(parts, tg, 8 * D)
+            nv = int((sets[0][1] != -100).sum())
+            nb = 2 * D * nv + 8 * rows + (8 + 1) * 16 * rows + 12 * rows + 4
+        elif dts:
             scale = esize // 2   # algorithmic_bytes counts 2-byte elements
             if base == "rmsnorm":
                 fn = lambda i: ak.ak_rmsnorm_fwd_dt(sets[i][0], sets[i][1], sets[i][2], eps=1e-6)

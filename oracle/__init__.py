@@ -43,6 +43,8 @@ def _load():
         lib.oracle_softmax_dt.restype = None
         lib.oracle_xent_dt.argtypes = [p, p, i64, p, p, p, i64, i64, ctypes.c_int]
         lib.oracle_xent_dt.restype = None
+        lib.oracle_rope.argtypes = [p, p, i64, i64, i64, f32, i64, ctypes.c_int]
+        lib.oracle_rope.restype = None
         lib.oracle_rmsnorm.argtypes = [p, p, p, i64, i64, f32]
         lib.oracle_rmsnorm.restype = None
         lib.oracle_layernorm.argtypes = [p, p, p, p, i64, i64, f32]
@@ -139,6 +141,20 @@ def xent_dt(logits, targets, dtype: str, ignore_index: int = -100):
     _load().oracle_xent_dt(x.ctypes.data, t.ctypes.data, int(ignore_index), loss.ctypes.data,
                            ctypes.addressof(mean), ctypes.addressof(cnt), rows, V, DTYPES[dtype])
     return loss, float(mean.value), int(cnt.value)
+
+
+def rope(x, dtype: str, base: float = 10000.0, pos_offset: int = 0) -> np.ndarray:
+    """Interleaved rotary embedding of x [n_seq, S, Dh] (element type ``dtype``): the pair
+    (2i, 2i+1) at sequence index s is rotated by (pos_offset + s) * base^(-2i/Dh).  float64 out;
+    ``base`` is first rounded to float32."""
+    x = _elems(x, dtype)
+    if x.ndim != 3 or x.shape[2] % 2:
+        raise ValueError("x must be [n_seq, S, Dh] with even Dh")
+    n_seq, S, Dh = x.shape
+    y = np.empty((n_seq, S, Dh), dtype=np.float64)
+    _load().oracle_rope(x.ctypes.data, y.ctypes.data, n_seq, S, Dh, float(np.float32(base)),
+                        int(pos_offset), DTYPES[dtype])
+    return y
 
 
 def rmsnorm(x_bits, w_bits, eps: float) -> np.ndarray:

@@ -29,6 +29,7 @@
  *   layernorm: mu = mean_j x_j ; var = mean_j (x_j - mu)^2 ;
  *              y_j = (x_j - mu) / sqrt(var + eps) * gamma_j + beta_j   (Table 3 "layernorm")
  *   rowsum  : out_r = sum_j x_rj                                      (Table 3 "reduce")
+ *   rope    : pair (2i, 2i+1) at position p rotated by p * base^(-2i/Dh)   (Table 3 "rotary_emb")
  *
  * Inputs are the exact bit patterns the GPU sees (bf16 or fp16 as uint16, or fp32),
  * widened exactly to double; outputs are double and are never rounded.  The *_dt functions
@@ -170,6 +171,34 @@ void oracle_rowsum(const uint16_t *x, double *out, int64_t rows, int64_t D)
         double sum = 0.0;
         for (int64_t j = 0; j < D; ++j) sum += bf16_bits_to_double(xr[j]);
         out[r] = sum;
+    }
+}
+
+/* Rotary position embedding forward (Table 3 "rotary_emb": interleaved rotation; Table 4
+ * rows "rotary", shape batch x heads x sequence x head_dim).  x: [n_seq, S, Dh] elements of
+ * `dtype` (n_seq = batch * heads); the head vector at sequence index s has position
+ * p = pos_offset + s, and its pair i = elements (2i, 2i + 1) is rotated by the angle
+ *   theta = p * base^(-2i / Dh):
+ *   y[2i]     = x[2i] cos(theta) - x[2i + 1] sin(theta)
+ *   y[2i + 1] = x[2i] sin(theta) + x[2i + 1] cos(theta)
+ * `base` arrives as the float the GPU entry point receives and is widened.  Dh must be even. */
+void oracle_rope(const void *x, double *y, int64_t n_seq, int64_t S, int64_t Dh,
+                 float base, int64_t pos_offset, int dtype)
+{
+    const double base_d = (double)base;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < n_seq * S; ++r) {
+        const int64_t s = r % S;
+        const double p = (double)(pos_offset + s);
+        const char *xr = (const char *)x + r * Dh * elem_bytes(dtype);
+        double *yr = y + r * Dh;
+        for (int64_t i = 0; i < Dh / 2; ++i) {
+            const double theta = p * pow(base_d, -2.0 * (double)i / (double)Dh);
+            const double c = cos(theta), sn = sin(theta);
+            const double a = load_elem(xr, 2 * i, dtype), b = load_elem(xr, 2 * i + 1, dtype);
+            yr[2 * i] = a * c - b * sn;
+            yr[2 * i + 1] = a * sn + b * c;
+        }
     }
 }
 

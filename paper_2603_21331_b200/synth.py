@@ -94,6 +94,12 @@ def layernorm_inputs(rows: int, D: int, seed: int, device="cpu"):
     return x, gamma, beta
 
 
+def rope_inputs(n_seq: int, S: int, Dh: int, seed: int, device="cpu", dtype=torch.bfloat16):
+    """x [n_seq, S, Dh] ~ N(0, 1): query / key head vectors before the rotation."""
+    g = _gen(seed, device)
+    return _normal_bf16(n_seq * S, Dh, 1.0, 0.0, g, device, dtype).view(n_seq, S, Dh)
+
+
 def softmax_inputs(rows: int, D: int, seed: int, device="cpu", mask_frac: float = 0.1,
                    dtype=torch.bfloat16):
     """x [rows, D] with ~mask_frac of the rows causal-masked by trailing -inf."""

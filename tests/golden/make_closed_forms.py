@@ -10,7 +10,7 @@ Run:  python tests/golden/make_closed_forms.py
 """
 import os
 
-from mpmath import mp, mpf, exp, log, sqrt
+from mpmath import mp, mpf, exp, log, sqrt, cos, sin
 
 mp.dps = 40
 HERE = os.path.dirname(os.path.abspath(__file__))
@@ -60,6 +60,17 @@ add("bf16_of_65000", bf16_round(mpf(65000)), "nearest bf16 to 65000")
 # one dominant logit: gap 20 over V-1 = 7 others -> loss at the hot index = log1p(7 e^-20)
 add("xent_hot_gap20_V8", log(1 + 7 * exp(-20)), "log(1 + 7 e^-20)")
 add("xent_cold_gap20_V8", 20 + log(1 + 7 * exp(-20)), "20 + log(1 + 7 e^-20)")
+
+# rotary embedding (Table 3 "rotary_emb"): pair 0 turns by the position itself (base^0 = 1);
+# with Dh = 4 and base = 10000 pair 1 turns by p * 10000^(-1/2) = p / 100
+for p_ in (1, 2, 3, 2047):
+    add(f"cos_{p_}", cos(mpf(p_)), f"rope pair 0 at position {p_}: (1,0) -> (cos, sin)")
+    add(f"sin_{p_}", sin(mpf(p_)), f"rope pair 0 at position {p_}")
+    add(f"cos_{p_}_over_100", cos(mpf(p_) / 100), f"rope Dh=4 base=1e4 pair 1 at position {p_}")
+    add(f"sin_{p_}_over_100", sin(mpf(p_) / 100), f"rope Dh=4 base=1e4 pair 1 at position {p_}")
+# Dh = 128, base = 10000, pair 32: exponent -64/128 = -1/2 again; pair 16: 10000^(-1/4) = 1/10
+add("cos_7_over_10", cos(mpf(7) / 10), "rope Dh=128 pair 16 at position 7: angle 7 * 10000^(-1/4)")
+add("sin_7_over_10", sin(mpf(7) / 10), "rope Dh=128 pair 16 at position 7")
 
 with open(os.path.join(HERE, "closed_forms.txt"), "w") as f:
     f.write("# name value  # derivation (closed forms, 40-digit mpmath; see make_closed_forms.py)\n")
