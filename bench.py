@@ -507,6 +507,10 @@ SWEEP_DTYPES = {"f16": torch.float16, "f32": torch.float32}
 # vocabulary-parallel cross-entropy as one of 8 ranks sees it: its [rows, V/8] shard -> partial
 # kernel, then the merge over 8 ranks' partial buffers (the 7 others' stand-ins are copies)
 SWEEP += [("xent_vp8", 4096, 128256 // 8), ("xent_vp8", 16384, 128256 // 8)]
+# rotary embedding, the paper's Table 4 shapes 2 x 32 x {2k, 4k} x 128 (rows = 64 sequences x S)
+SWEEP += [("rope.f16", 64 * 2048, 128), ("rope.f16", 64 * 4096, 128), ("rope.bf16", 64 * 4096, 128),
+          ("rope.f32", 64 * 4096, 128), ("rope.bf16", 64 * 16384, 128)]
+SWEEP_DTYPES["bf16"] = torch.bfloat16
 
 
 def time_op(fn_for_set, nsets, iters=200, warmup=20):
@@ -572,6 +576,29 @@ def sweep_accuracy(ak, synth, op, rows, D, bufs):
         oracle.set_threads(cores)
         return ref, t_one * rows / len(idx), t_all * rows / len(idx)
 
+    if op.startswith("rope."):
+        dts = op.split(".")[1]
+        x, y = bufs
+        first = y.clone()
+        ak.ak_rope_fwd(x, y)
+        same = torch.equal(first.view(torch.uint8), y.view(torch.uint8))
+        S = x.shape[1]
+        pos = np.sort(np.unique(np.concatenate([[0, S - 1], np.random.default_rng(S).integers(0, S, 14)])))
+        refs, t1, tn, gots = [], 0.0, 0.0, []
+        for p in pos:   # one position of every sequence at a time: the checker gets [64, 1, Dh] at offset p
+            xs = x[:, int(p):int(p) + 1].contiguous()
+            ref, a, b = timed_oracle(lambda: oracle.rope(synth.to_elems(xs), dts, pos_offset=int(p)))
+            refs.append(ref); t1 += a; tn += b
+            gots.append(y[:, int(p):int(p) + 1].cpu().double().numpy())
+        ref, got = np.concatenate(refs, axis=1), np.concatenate(gots, axis=1)
+        err = np.abs(got - ref)
+        tol = {"bf16": 1.6e-2, "f16": 1e-3, "f32": 1e-5}[dts]
+        scale = rows / (64.0 * len(pos)) * len(idx) / rows   # timed_oracle scaled by rows / len(idx)
+        return {"max_abs_err": float(err.max()),
+                "max_err_over_tolerance": float((err / (tol * np.maximum(1.0, np.abs(ref)))).max()),
+                "bitwise_repeat": bool(same), "sampled_rows": int(64 * len(pos)),
+                "oracle_s_1_thread_scaled": t1 * scale, "oracle_s_all_threads_scaled": tn * scale,
+                "oracle_threads": cores}
     if op == "xent_vp8":
         lg, tg, parts = bufs
         V = 8 * D
@@ -685,7 +712,10 @@ def run_sweep(ak, synth, dev, peak):
         nsets = int(max(1, min(64, -(-(1 << 30) // one_set))))
         sets = []
         for s in range(nsets):
-            if op == "xent_vp8":
+            if base == "rope":
+                x = synth.rope_inputs(64, rows // 64, D, 7900 + s, device=dev, dtype=SWEEP_DTYPES[dts])
+                sets.append((x, torch.empty_like(x)))
+            elif op == "xent_vp8":
                 lg, tg = synth.xent_inputs(rows, D, 7800 + s, device=dev)
                 sets.append((lg, tg, torch.zeros((8, rows, 2, 2), dtype=torch.float32, device=dev)))
             elif dts:
@@ -716,7 +746,10 @@ def run_sweep(ak, synth, dev, peak):
                 sets.append((lg, tg, torch.empty((rows,), dtype=torch.float32, device=dev),
                              torch.empty((1,), dtype=torch.float32, device=dev),
                              torch.empty((nws,), dtype=torch.uint8, device=dev) if nws else None))
-        if op == "xent_vp8":
+        if base == "rope":
+            fn = lambda i: ak.ak_rope_fwd(sets[i][0], sets[i][1])
+            nb = 2 * esize * rows * D
+        elif op == "xent_vp8":
             def fn(i):
                 lg, tg, parts = sets[i]
                 ak.ak_xent_vp_partial(lg, tg, 0, 8 * D, 1, partial=parts[0])

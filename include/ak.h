@@ -103,6 +103,23 @@ int ak_xent_fwd_dt(const void* logits, const int64_t* targets, int64_t ignore_in
                    float* loss_rows, float* loss_mean, int64_t rows, int64_t V,
                    int dtype, void* cuda_stream, int path, int nsplit);
 /* ---------------------------------------------------------------------------------
+ * Rotary position embedding forward (Table 3 "rotary_emb": interleaved rotation; Table 4
+ * rows "rotary": batch x heads x sequence x head_dim).
+ *   x, y: device [n_seq, S, Dh] of `dtype`, n_seq = batch * heads, dense; y may alias x.
+ *   The head vector at sequence index s has position p = pos_offset + s; its pair
+ *   i = elements (2i, 2i + 1) turns by theta = p * base^(-2i / Dh):
+ *     y[2i]     = rne( x[2i] cos(theta) - x[2i + 1] sin(theta) )
+ *     y[2i + 1] = rne( x[2i] sin(theta) + x[2i + 1] cos(theta) )
+ * Dh even, 2 <= Dh <= 512 (else AK_ERR_SHAPE); base finite and > 0 (typically 10000);
+ * 0 <= pos_offset < 2^52.  Frequencies are formed in double on the host, angles reduced in
+ * double on the device, so cos / sin are right to fp32 rounding at any position; products
+ * and sums in fp32.  Fast path: 16-byte aligned x and y and Dh a multiple of the elements in
+ * 16 bytes; anything else takes an element-wise kernel.  One launch, no scratch.
+ */
+int ak_rope_fwd(const void* x, void* y, int64_t n_seq, int64_t S, int64_t Dh, float base,
+                int64_t pos_offset, int dtype, void* cuda_stream);
+
+/* ---------------------------------------------------------------------------------
  * Vocabulary-parallel cross-entropy (the fused cross_ent of Table 3 with the vocabulary
  * dimension sharded over ranks, as in tensor-parallel language-model heads).  Rank k holds
  * logits_shard: device [rows, V_local] of `dtype`, the columns

@@ -39,6 +39,7 @@ SIGNATURES = {
     "ak_softmax_fwd_dt": (_int, [_p, _p, _i64, _i64, _int, _p, _int]),
     "ak_xent_fwd_dt": (_int, [_p, _p, _i64, _p, _p, _i64, _i64, _int, _p, _int, _int]),
     "ak_choose_path_dt": (_int, [_int, _i64, _i64, _int, _int]),
+    "ak_rope_fwd": (_int, [_p, _p, _i64, _i64, _i64, _f32, _i64, _int, _p]),
     "ak_xent_vp_nsplit": (_int, [_i64, _i64]),
     "ak_xent_vp_partial_bytes": (_sz, [_i64, _int]),
     "ak_xent_vp_partial": (_int, [_p, _p, _i64, _i64, _i64, _p, _i64, _i64, _int, _int, _p]),
@@ -194,6 +195,21 @@ def ak_xent_fwd_dt(logits: torch.Tensor, targets: torch.Tensor, ignore_index: in
                                 loss_mean.data_ptr() if want_mean else None, rows, V, dt,
                                 _stream_ptr(stream), path, nsplit), "ak_xent_fwd_dt")
     return loss_rows, loss_mean
+
+
+def ak_rope_fwd(x: torch.Tensor, y: Optional[torch.Tensor] = None, base: float = 10000.0,
+                pos_offset: int = 0, stream=None) -> torch.Tensor:
+    """Interleaved rotary embedding of x [n_seq, S, Dh] (bf16, fp16 or fp32); y may be x."""
+    dt = _dev_dt(x, "x", 3)
+    n_seq, S, Dh = x.shape
+    if y is None:
+        y = torch.empty_like(x)
+    _dev_dt(y, "y", 3, x.dtype)
+    if y.shape != x.shape:
+        raise ValueError("y must have the shape of x")
+    _check(lib().ak_rope_fwd(x.data_ptr(), y.data_ptr(), n_seq, S, Dh, base, pos_offset, dt,
+                             _stream_ptr(stream)), "ak_rope_fwd")
+    return y
 
 
 def ak_xent_vp_nsplit(rows: int, V_local: int) -> int:

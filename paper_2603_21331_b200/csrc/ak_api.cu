@@ -110,6 +110,20 @@ int ak_xent_fwd_dt(const void* logits, const int64_t* targets, int64_t ignore_in
     return xent_dispatch(logits, targets, ignore_index, loss_rows, loss_mean, rows, V, nullptr, 0, true,
                          static_cast<cudaStream_t>(cuda_stream), path, nsplit, dtype);
 }
+int ak_rope_fwd(const void* x, void* y, int64_t n_seq, int64_t S, int64_t Dh, float base, int64_t pos_offset,
+                int dtype, void* cuda_stream) {
+    if (!known_dtype(dtype)) return AK_ERR_ARG;
+    if (n_seq < 0 || S < 0 || Dh <= 0 || (Dh & 1) || Dh > 512) return AK_ERR_SHAPE;
+    if (n_seq != 0 && S != 0 && (!x || !y)) return AK_ERR_NULL;
+    if (n_seq > 0 && S > 0 && (S > (int64_t)0x7fffffffffffLL / Dh || n_seq > (int64_t)0x7fffffffffffLL / (S * Dh)))
+        return AK_ERR_SHAPE;
+    if (!is_aligned(x, (size_t)dtype_bytes(dtype)) || !is_aligned(y, (size_t)dtype_bytes(dtype))) return AK_ERR_ALIGN;
+    if (!(base > 0.0f) || !std::isfinite(base)) return AK_ERR_ARG;
+    if (pos_offset < 0 || pos_offset > ((int64_t)1 << 52) - S) return AK_ERR_ARG;
+    if (n_seq == 0 || S == 0) return AK_OK;
+    return rope_dispatch(x, y, n_seq, S, Dh, base, pos_offset, dtype, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int ak_xent_vp_nsplit(int64_t rows, int64_t V_local) {
     int ns = 1;
     if (rows > 0 && V_local > 0) xent_choose(rows, V_local, &ns);
@@ -256,7 +270,7 @@ const char* ak_status_string(int status) {
         case AK_ERR_NULL: return "a required pointer is NULL";
         case AK_ERR_SHAPE: return "bad shape (rows < 0, D <= 0, or size not supported by the requested path)";
         case AK_ERR_ALIGN: return "pointer not sufficiently aligned";
-        case AK_ERR_ARG: return "bad scalar argument (eps, path id, nsplit or dtype)";
+        case AK_ERR_ARG: return "bad scalar argument (eps, base, position offset, path id, nsplit or dtype)";
         case AK_ERR_CUDA: return "CUDA runtime error";
         case AK_ERR_NOMEM: return "scratch memory unavailable or workspace too small";
         case AK_ERR_CAPACITY: return "problem exceeds the fixed scratch of the no-allocation entry point (rows * nsplit * 8 bytes > 1 MiB or rows > 65535)";

@@ -276,6 +276,8 @@ int xent_mean_merge_launch(const double* pairs, int64_t n, float* loss_mean, cud
 int layernorm_dispatch(const void* x, const void* gamma, const void* beta, void* y, int64_t rows, int64_t D,
                        float eps, cudaStream_t st, int path);
 int layernorm_choose(int64_t rows, int64_t D, bool aligned16);
+int rope_dispatch(const void* x, void* y, int64_t n_seq, int64_t S, int64_t Dh, float base, int64_t pos_offset,
+                  int dtype, cudaStream_t st);
 int rowsum_dispatch(const void* x, float* out, int64_t rows, int64_t D, cudaStream_t st);
 int rmsnorm_choose(int64_t rows, int64_t D, bool aligned16, int dtype = AK_DTYPE_BF16);
 int softmax_choose(int64_t rows, int64_t D, bool aligned16, int dtype = AK_DTYPE_BF16);
