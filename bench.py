@@ -46,7 +46,7 @@ FALLBACK_HBM_GBS = 6650.0
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel
 # (cross-entropy row kernel at [4096, 128256]): the [2048, 128256] capture summarised in
 # profiles/kernels_ncu_set_full.md, 498.8 MB read + 7.3 MB written, scaled by rows (x2).
-NCU_TRAFFIC_BYTES_DOMINANT = {"xent": 1012253184}
+NCU_TRAFFIC_BYTES_DOMINANT = {"xent": 1006287872}
 
 
 def measured_peak():
@@ -810,15 +810,20 @@ def run_case(args):
     rows, D = int(rows), int(D)
     dev = "cuda:0"
     torch.cuda.set_device(0)
-    if op == "rmsnorm":
+    if op == "rope":   # rows = 64 sequences x S positions, D = head dimension, fp16 as in the paper
+        x = synth.rope_inputs(64, rows // 64, D, 7900, device=dev, dtype=torch.float16)
+        y = torch.empty_like(x)
+        fn = lambda: ak.ak_rope_fwd(x, y)
+        nb = 4 * rows * D
+    elif op == "rmsnorm":
         x, w = synth.rmsnorm_inputs(rows, D, 7000, device=dev)
         y = torch.empty_like(x)
         fn = lambda: ak.ak_rmsnorm_fwd(x, w, y, eps=1e-6)
         nb = algorithmic_bytes(op, rows, D)
     elif op == "layernorm":
-        x, g, b = synth.layernorm_inputs(rows, D, 7300, device=dev)
+        x, gamma, beta = synth.layernorm_inputs(rows, D, 7300, device=dev)
         y = torch.empty_like(x)
-        fn = lambda: ak.ak_layernorm_fwd(x, g, b, y, eps=1e-5)
+        fn = lambda: ak.ak_layernorm_fwd(x, gamma, beta, y, eps=1e-5)
         nb = algorithmic_bytes(op, rows, D)
     elif op == "rowsum":
         x, _, _ = synth.layernorm_inputs(rows, D, 7400, device=dev)
