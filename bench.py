@@ -45,7 +45,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel
 # (cross-entropy row kernel at [4096, 128256]): the [2048, 128256] capture summarised in
-# profiles/kernels_ncu_set_full.md, 498.8 MB read + 7.3 MB written, scaled by rows (x2).
+# profiles/kernels_ncu_set_full.md, 498.7 MB read + 4.4 MB written, scaled by rows (x2).
 NCU_TRAFFIC_BYTES_DOMINANT = {"xent": 1006287872}
 
 
