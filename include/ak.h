@@ -1,11 +1,14 @@
 /*
  * ak.h - C ABI of libak: row-reduction kernels for NVIDIA B200 (sm_100a).
  *
- * Three forward ops over contiguous row-major bf16 [rows, D] tensors:
+ * Forward ops over contiguous row-major bf16 [rows, D] tensors:
  *   RMSNorm            (paper Table 3, row "rmsnorm";   Table 4 rows "rmsnorm")
  *   last-dim softmax   (paper Table 3, row "softmax";   Table 4 rows "softmax")
  *   fused cross-entropy(paper Table 3, row "cross_ent": online log-sum-exp fused with
  *                       the NLL gather; Table 4 rows "cross_ent")
+ * and, built on the same skeletons: LayerNorm ("layernorm"), row-sum ("reduce"), rotary
+ * embedding ("rotary_emb"), fp16 / fp32 variants of the first three (*_dt) and the
+ * vocabulary-parallel form of the cross-entropy (ak_xent_vp_*).
  * Semantics are those of the PyTorch reference ops the paper uses as its correctness
  * oracle (Section 6): F.rms_norm, F.softmax(dim=-1), F.cross_entropy(ignore_index).
  *
