@@ -99,3 +99,128 @@ def test_xent_full_size(rows, V):
         assert abs(mean.item() - (math.log(V) + 2.0)) < 0.2   # E[loss] for N(0, 2^2) logits
     del logits
     _free()
+
+
+@pytest.mark.parametrize("rows,D", [(8192, 4096), (4096, 5120), (8192, 8192), (65536, 4096), (4096, 32768),
+                                    (8192, 4099)])
+def test_layernorm_full_size(rows, D):
+    x, g, b = synth.layernorm_inputs(rows, D, synth.case_seed(6, D + rows), device=DEV)
+    y = ak.ak_layernorm_fwd(x, g, b, eps=1e-5)
+    y2 = ak.ak_layernorm_fwd(x, g, b, eps=1e-5)
+    torch.cuda.synchronize()
+    assert torch.equal(y.view(torch.int16), y2.view(torch.int16))
+    del y2
+    idx = _sample_rows(rows, seed=D)
+    it = torch.from_numpy(idx).to(DEV)
+    ref = oracle.layernorm(synth.to_bits(x[it]), synth.to_bits(g), synth.to_bits(b), 1e-5)
+    assert_bf16_close(y[it], ref, f"layernorm {rows}x{D} sampled rows", tight=False)
+    # property: (y - beta) / gamma has zero mean and unit variance in every row
+    for r0 in range(0, rows, 16384):
+        z = (y[r0:r0 + 16384].float() - b.float()[None, :]) / g.float()[None, :]
+        assert torch.isfinite(z).all()
+        assert bool((z.mean(dim=-1).abs() < 2e-2).all())
+        assert bool((((z * z).mean(dim=-1)) - 1).abs().max() < 3e-2)
+    del x, y
+    _free()
+
+
+@pytest.mark.parametrize("rows,D", [(16384, 4096), (8192, 8192), (65536, 1024), (65536, 8192), (4096, 128256),
+                                    (8192, 4099)])
+def test_rowsum_full_size(rows, D):
+    x, _, _ = synth.layernorm_inputs(rows, D, synth.case_seed(8, D + rows), device=DEV)
+    s = ak.ak_rowsum_fwd(x)
+    s2 = ak.ak_rowsum_fwd(x)
+    torch.cuda.synchronize()
+    assert torch.equal(s.view(torch.int32), s2.view(torch.int32))
+    idx = _sample_rows(rows, seed=D)
+    it = torch.from_numpy(idx).to(DEV)
+    xb = synth.to_bits(x[it])
+    ref = oracle.rowsum(xb)
+    mag = np.abs(oracle.bf16_to_f64(xb)).sum(axis=1)
+    err = np.abs(s[it].cpu().double().numpy() - ref)
+    assert float(np.max(err / (1e-6 * mag + 2.0 ** -24 * np.abs(ref)))) <= 1.0
+    # property at any size: agrees with a float64 sum done by another library on the device
+    for r0 in range(0, rows, 8192):
+        want = x[r0:r0 + 8192].double().sum(dim=-1)
+        absx = x[r0:r0 + 8192].double().abs().sum(dim=-1)
+        assert bool(((s[r0:r0 + 8192].double() - want).abs() <= 1e-6 * absx + 1e-6 * want.abs()).all())
+    del x
+    _free()
+
+
+@pytest.mark.parametrize("dtype,S", [(torch.float16, 2048), (torch.float16, 4096), (torch.bfloat16, 4096),
+                                     (torch.float32, 4096)])
+def test_rope_full_size(dtype, S):
+    n_seq, Dh = 64, 128                                    # 2 x 32 heads, the benchmark's layout
+    x = synth.rope_inputs(n_seq, S, Dh, synth.case_seed(18, S), device=DEV, dtype=dtype)
+    y = ak.ak_rope_fwd(x)
+    y2 = ak.ak_rope_fwd(x)
+    torch.cuda.synchronize()
+    assert torch.equal(y.view(torch.uint8), y2.view(torch.uint8))
+    del y2
+    name = synth.DTYPE_NAMES[dtype]
+    tol = {torch.bfloat16: 1.6e-2, torch.float16: 1e-3, torch.float32: 1e-5}[dtype]
+    for p in (0, 1, S // 2, S - 1, 777):                   # sampled positions, every sequence
+        ref = oracle.rope(synth.to_elems(x[:, p:p + 1].contiguous()), name, pos_offset=p)
+        got = y[:, p:p + 1].cpu().double().numpy()
+        assert float(np.max(np.abs(got - ref) / (tol * np.maximum(1.0, np.abs(ref))))) <= 1.0
+    # property at any size: a rotation keeps the length of every pair
+    xf, yf = x.float(), y.float()
+    n_in = xf[..., 0::2] ** 2 + xf[..., 1::2] ** 2
+    n_out = yf[..., 0::2] ** 2 + yf[..., 1::2] ** 2
+    rel = {torch.bfloat16: 2e-2, torch.float16: 3e-3, torch.float32: 1e-5}[dtype]
+    assert bool(((n_out - n_in).abs() <= rel * n_in + 1e-6).all())
+    del x, y
+    _free()
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.float32])
+def test_dtype_variants_full_size(dtype):
+    name = synth.DTYPE_NAMES[dtype]
+    from parity import assert_close_dt
+    x, w = synth.rmsnorm_inputs(8192, 8192, synth.case_seed(12, 1), device=DEV, dtype=dtype)
+    y = ak.ak_rmsnorm_fwd_dt(x, w)
+    it = torch.from_numpy(_sample_rows(8192, seed=1)).to(DEV)
+    assert_close_dt(y[it], oracle.rmsnorm_dt(synth.to_elems(x[it]), synth.to_elems(w), 1e-6, name), f"rmsnorm {name} full")
+    del x, y
+    _free()
+    xs = synth.softmax_inputs(16384, 8192, synth.case_seed(13, 1), device=DEV, dtype=dtype)
+    y = ak.ak_softmax_fwd_dt(xs)
+    it = torch.from_numpy(_sample_rows(16384, seed=2)).to(DEV)
+    assert_close_dt(y[it], oracle.softmax_dt(synth.to_elems(xs[it]), name), f"softmax {name} full")
+    assert bool(((y.float().sum(dim=-1) - 1).abs() < 2e-3).all())
+    del xs, y
+    _free()
+    V = 128256 if dtype == torch.float16 else 50304
+    lg, tg = synth.xent_inputs(4096, V, synth.case_seed(14, 1), device=DEV, dtype=dtype)
+    loss, mean = ak.ak_xent_fwd_dt(lg, tg)
+    idx = _sample_rows(4096, seed=3)
+    it = torch.from_numpy(idx).to(DEV)
+    ref_rows, _, _ = oracle.xent_dt(synth.to_elems(lg[it]), tg[it].cpu().numpy(), name)
+    assert_loss_close(loss[it], ref_rows, f"xent {name} full")
+    valid = tg != -100
+    want_mean = loss[valid].double().sum().item() / int(valid.sum())
+    assert abs(mean.item() - want_mean) <= 1e-6 * want_mean
+    del lg
+    _free()
+
+
+def test_vocab_parallel_full_size_eight_ranks():
+    from paper_2603_21331_b200 import parallel
+    rows, V, world = 4096, 128256, 8
+    lg, tg = synth.xent_inputs(rows, V, synth.case_seed(16, 1), device=DEV)
+    parts = []
+    for rank in range(world):
+        b, e = parallel.shard_vocab(V, rank, world)
+        parts.append(ak.ak_xent_vp_partial(lg[:, b:e].contiguous(), tg, b, V, 1))
+    loss, mean = ak.ak_xent_vp_merge(torch.stack(parts).contiguous(), tg, V)
+    idx = _sample_rows(rows, seed=4)
+    it = torch.from_numpy(idx).to(DEV)
+    ref_rows, _, _ = oracle.xent(synth.to_bits(lg[it]), tg[it].cpu().numpy())
+    assert_loss_close(loss[it], ref_rows, "vocabulary-parallel xent, 8 shards, sampled rows")
+    # and against the single-GPU kernel on the unsharded logits: same loss up to the merge's rounding
+    single, smean = ak.ak_xent_fwd(lg, tg)
+    assert bool(((loss - single).abs() <= 2e-6 * single.abs().clamp(min=1.0)).all())
+    assert abs(mean.item() - smean.item()) <= 2e-6 * abs(smean.item())
+    del lg
+    _free()
