@@ -317,6 +317,8 @@ def run_ours(args, rank, world, local_rank):
     use_graph = world == 1 and not os.environ.get("AK_BENCH_EAGER")
     launches0 = ak.ak_launch_count()
     step()
+    if world > 1:
+        global_mean()
     torch.cuda.synchronize()
     kernels_per_step = ak.ak_launch_count() - launches0
     graph = None

@@ -47,7 +47,7 @@ typedef enum {
     AK_ERR_NULL = 1,   /* a required pointer is NULL */
     AK_ERR_SHAPE = 2,  /* rows < 0, D <= 0, or a size the chosen path cannot take */
     AK_ERR_ALIGN = 3,  /* pointer not aligned to its element type (or to 16 B where a forced path needs it) */
-    AK_ERR_ARG = 4,    /* eps negative or not finite; unknown path id; bad nsplit */
+    AK_ERR_ARG = 4,    /* eps negative or not finite; bad base or position offset; unknown path id or dtype; bad nsplit */
     AK_ERR_CUDA = 5,   /* a CUDA runtime call or launch failed */
     AK_ERR_NOMEM = 6,  /* scratch allocation failed or caller workspace too small */
     AK_ERR_CAPACITY = 7 /* problem larger than the fixed scratch of ak_xent_fwd_static */
@@ -57,10 +57,12 @@ typedef enum {
  * dispatcher choose", which is what the plain entry points do. */
 enum {
     AK_PATH_AUTO = 0,
-    AK_PATH_WARP = 1,     /* one warp per row, row held in registers; D % 8 == 0, D <= 2048, 16 B aligned */
-    AK_PATH_CTA = 2,      /* one CTA per row, row held in registers;  D % 8 == 0, D <= 32768, 16 B aligned */
-    AK_PATH_GENERIC = 3,  /* any D, any 2-byte alignment; row re-read from L1/L2, single DRAM pass */
-    AK_PATH_SMEM = 4      /* one CTA per row, row staged in shared memory by bulk (TMA) copies; D % 8 == 0, D <= 114688, 16 B aligned */
+    /* Size limits are in row BYTES (bf16: D = bytes / 2); the register and shared-memory paths
+     * need 16-byte aligned pointers and rows that are a multiple of 16 bytes. */
+    AK_PATH_WARP = 1,     /* one (or two) warps per row, row held in registers; rows <= 4 KiB (bf16 D <= 2048) */
+    AK_PATH_CTA = 2,      /* one CTA per row, row held in registers; rows <= 64 KiB (bf16 D <= 32768) */
+    AK_PATH_GENERIC = 3,  /* any D, any element alignment; row staged in shared memory in its 16-byte phase or re-read from L1/L2, single DRAM pass */
+    AK_PATH_SMEM = 4      /* one CTA per row, row staged in shared memory by bulk (TMA) copies; rows <= 224 KiB (bf16 D <= 114688) */
 };
 /* Element types of the *_dt entry points.  The plain entry points are bf16. */
 enum {

@@ -7,7 +7,8 @@ Two layers, same names as the C ABI (``include/ak.h``):
 
 * ``lib()`` returns the ``ctypes.CDLL`` with typed entry points (``lib().ak_rmsnorm_fwd``
   etc.), taking raw device pointers as integers.
-* ``ak_rmsnorm_fwd / ak_softmax_fwd / ak_xent_fwd`` (and ``*_host``) take torch tensors,
+* ``ak_rmsnorm_fwd / ak_softmax_fwd / ak_xent_fwd`` (and ``*_host``, ``*_dt``,
+  ``ak_layernorm_fwd``, ``ak_rowsum_fwd``, ``ak_rope_fwd``, ``ak_xent_vp_*``) take torch tensors,
   check dtype / contiguity / device, and pass ``data_ptr()`` and the current CUDA stream.
   PyTorch is used for device memory and streams only.
 """
