@@ -68,6 +68,31 @@ int launch_stage(const uint16_t* x, const uint16_t* g, const uint16_t* b, uint16
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
+template <int THREADS, int VPT, int MINB>
+int launch_regp(const uint16_t* x, const uint16_t* g, const uint16_t* b, uint16_t* y, int64_t rows, int64_t D,
+                float inv_D, float eps, cudaStream_t st) {
+    layernorm_regp_kernel<THREADS, VPT, MINB><<<(unsigned)rows, THREADS, 0, st>>>(x, g, b, y, D, inv_D, eps);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+}
+// unaligned rows held in registers: vectors per thread 1..8 for a CTA of THREADS threads
+// (register caps: M14 for 1..5 vectors, M58 for 6..8)
+template <int THREADS, int M14, int M58>
+int launch_regp_vpt(int vpt, const uint16_t* x, const uint16_t* g, const uint16_t* b, uint16_t* y, int64_t rows,
+                    int64_t D, float inv_D, float eps, cudaStream_t st) {
+    switch (vpt) {
+        case 1: return launch_regp<THREADS, 1, M14>(x, g, b, y, rows, D, inv_D, eps, st);
+        case 2: return launch_regp<THREADS, 2, M14>(x, g, b, y, rows, D, inv_D, eps, st);
+        case 3: return launch_regp<THREADS, 3, M14>(x, g, b, y, rows, D, inv_D, eps, st);
+        case 4: return launch_regp<THREADS, 4, M14>(x, g, b, y, rows, D, inv_D, eps, st);
+        case 5: return launch_regp<THREADS, 5, M14>(x, g, b, y, rows, D, inv_D, eps, st);
+        case 6: return launch_regp<THREADS, 6, M58>(x, g, b, y, rows, D, inv_D, eps, st);
+        case 7: return launch_regp<THREADS, 7, M58>(x, g, b, y, rows, D, inv_D, eps, st);
+        case 8: return launch_regp<THREADS, 8, M58>(x, g, b, y, rows, D, inv_D, eps, st);
+        default: return AK_ERR_SHAPE;
+    }
+}
+
 }  // namespace
 
 int layernorm_choose(int64_t rows, int64_t D, bool aligned16) {
@@ -116,6 +141,10 @@ int layernorm_dispatch(const void* x, const void* gamma, const void* beta, void*
             const uint16_t* gs = static_cast<const uint16_t*>(gamma);
             const uint16_t* bs = static_cast<const uint16_t*>(beta);
             uint16_t* ys = static_cast<uint16_t*>(y);
+            // rows of up to 1024 covering vectors stay in the registers of a 128-thread CTA
+            const int64_t max_nv = (D + 14) >> 3;   // vectors covering the row at the worst phase
+            if (same_phase && is_aligned(gamma, 4) && is_aligned(beta, 4) && max_nv <= 1024)
+                return launch_regp_vpt<128, 10, 6>((int)((max_nv + 127) / 128), xs, gs, bs, ys, rows, D, inv_D, eps, st);
             if (same_phase && is_aligned(gamma, 4) && is_aligned(beta, 4) && stage_bytes <= (size_t)kMaxRowSmemBytes) {
                 if (D <= 8192) return launch_stage<128>(xs, gs, bs, ys, rows, D, stage_bytes, inv_D, eps, st);
                 if (D <= 32768) return launch_stage<256>(xs, gs, bs, ys, rows, D, stage_bytes, inv_D, eps, st);

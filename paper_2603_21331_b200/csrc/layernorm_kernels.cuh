@@ -234,6 +234,63 @@ layernorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restric
         yr[ej] = float_to_bf16(ln_out1(row16[ek * 8 + (threadIdx.x & 7)], __ldg(gamma + ej), __ldg(beta + ej), mu, rstd));
 }
 
+// ------------------------------------------------------------------ unaligned rows in registers
+// The phase layout of layernorm_stage_kernel without the trip through shared memory, for rows
+// short enough to sit in registers: interior vectors are loaded before the first use, the edge
+// elements are single values in sixteen threads.  Needs x and y rows in the same phase, gamma
+// and beta 4-byte aligned and at most THREADS * VPT covering vectors.
+template <int THREADS, int VPT, int MINB>
+__global__ void __launch_bounds__(THREADS, MINB)
+layernorm_regp_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ gamma,
+                      const uint16_t* __restrict__ beta, uint16_t* __restrict__ y, int64_t D, float inv_D, float eps) {
+    __shared__ float slots[2 * kWarp];
+    const int64_t r = blockIdx.x;
+    const uint16_t* xr = x + r * D;
+    uint16_t* yr = y + r * D;
+    // interior vectors k_lo .. k_hi - 1 live in registers (slot i of thread t holds vector
+    // k_lo + t + i * THREADS); the up to 14 edge elements belong to threads 0..15, one each
+    const int phase = (int)((reinterpret_cast<uintptr_t>(xr) >> 1) & 7);
+    const int nv = (int)((phase + D + 7) >> 3);
+    const int k_lo = phase ? 1 : 0;
+    const int k_hi = ((phase + D) & 7) ? nv - 1 : nv;
+    const uint4* xa = reinterpret_cast<const uint4*>(xr - phase);
+    uint4* ya = reinterpret_cast<uint4*>(yr - phase);
+    const int ek = (threadIdx.x < 8) ? 0 : nv - 1;
+    const bool evec = (threadIdx.x < 8) ? (k_lo == 1) : (k_hi == nv - 1 && !(nv == 1 && k_lo == 1));
+    const int64_t ej = (int64_t)ek * 8 - phase + (threadIdx.x & 7);
+    const bool edge = threadIdx.x < 16 && evec && ej >= 0 && ej < D;
+    const float K = bf16_to_float(__ldg(xr));
+    uint4 xv[VPT];
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int k = k_lo + threadIdx.x + i * THREADS;
+        if (k < k_hi) xv[i] = ld_stream(xa + k);
+    }
+    const uint16_t xe = edge ? ld_stream_u16(xr + ej) : (uint16_t)0;
+    float s1 = edge ? sub_bf16(xe, K) : 0.0f;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i)
+        if (k_lo + (int)threadIdx.x + i * THREADS < k_hi) s1 += sumdev8(xv[i], K);
+    s1 = cta_sum<THREADS>(s1, slots, 0);
+    const float mu = fmaf(s1, inv_D, K);
+    const float de = edge ? sub_bf16(xe, mu) : 0.0f;
+    float s2 = de * de;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i)
+        if (k_lo + (int)threadIdx.x + i * THREADS < k_hi) s2 += sqdev8(xv[i], mu);
+    s2 = cta_sum<THREADS>(s2, slots, 1);
+    const float rstd = rsqrtf(fmaf(s2, inv_D, eps));
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int k = k_lo + threadIdx.x + i * THREADS;
+        if (k < k_hi) {
+            const int64_t j0 = (int64_t)k * 8 - phase;
+            st_stream(ya + k, ln_out8(xv[i], ln_load_shifted(gamma, j0), ln_load_shifted(beta, j0), mu, rstd));
+        }
+    }
+    if (edge) yr[ej] = float_to_bf16(ln_out1(xe, __ldg(gamma + ej), __ldg(beta + ej), mu, rstd));
+}
+
 // ------------------------------------------------------------------ generic
 // Any D and any 2-byte alignment: element-wise 2-byte accesses, three passes over the row
 // (the second and third are served by L1/L2).  The slow, always-correct fallback; aligned

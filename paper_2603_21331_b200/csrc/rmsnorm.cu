@@ -66,6 +66,30 @@ int launch_smem(const void* x, const void* w, void* y, int64_t rows, int nvec, f
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
+// unaligned rows held in registers: vectors per thread 1..8 for a CTA of THREADS threads
+template <int DT, int THREADS, int VPT>
+int launch_regp(const uint16_t* x, const uint16_t* w, uint16_t* y, int64_t rows, int64_t D, float inv_D, float eps,
+                cudaStream_t st) {
+    rmsnorm_regp_kernel<THREADS, VPT, DT><<<(unsigned)rows, THREADS, 0, st>>>(x, w, y, D, inv_D, eps);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+}
+template <int DT, int THREADS>
+int launch_regp_vpt(int vpt, const uint16_t* x, const uint16_t* w, uint16_t* y, int64_t rows, int64_t D, float inv_D,
+                    float eps, cudaStream_t st) {
+    switch (vpt) {
+        case 1: return launch_regp<DT, THREADS, 1>(x, w, y, rows, D, inv_D, eps, st);
+        case 2: return launch_regp<DT, THREADS, 2>(x, w, y, rows, D, inv_D, eps, st);
+        case 3: return launch_regp<DT, THREADS, 3>(x, w, y, rows, D, inv_D, eps, st);
+        case 4: return launch_regp<DT, THREADS, 4>(x, w, y, rows, D, inv_D, eps, st);
+        case 5: return launch_regp<DT, THREADS, 5>(x, w, y, rows, D, inv_D, eps, st);
+        case 6: return launch_regp<DT, THREADS, 6>(x, w, y, rows, D, inv_D, eps, st);
+        case 7: return launch_regp<DT, THREADS, 7>(x, w, y, rows, D, inv_D, eps, st);
+        case 8: return launch_regp<DT, THREADS, 8>(x, w, y, rows, D, inv_D, eps, st);
+        default: return AK_ERR_SHAPE;
+    }
+}
+
 }  // namespace
 
 int rmsnorm_choose(int64_t rows, int64_t D, bool aligned16, int dtype) {
@@ -131,6 +155,10 @@ int dispatch_t(const void* x, const void* w, void* y, int64_t rows, int64_t D, f
                 const uint16_t* xs = static_cast<const uint16_t*>(x);
                 const uint16_t* ws = static_cast<const uint16_t*>(w);
                 uint16_t* ys = static_cast<uint16_t*>(y);
+                // rows of up to 1024 covering vectors stay in the registers of a 128-thread CTA
+                const int64_t max_nv = (D + 14) >> 3;   // vectors covering the row at the worst phase
+                if (same_phase && is_aligned(w, 4) && max_nv <= 1024)
+                    return launch_regp_vpt<DT, 128>((int)((max_nv + 127) / 128), xs, ws, ys, rows, D, inv_D, eps, st);
                 if (same_phase && is_aligned(w, 4) && stage_bytes <= (size_t)kMaxRowSmemBytes) {
                     static const bool configured = [] {
                         return cudaFuncSetAttribute(rmsnorm_stage_kernel<128, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,

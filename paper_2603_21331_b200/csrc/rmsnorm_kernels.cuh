@@ -241,6 +241,51 @@ rmsnorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict_
     }
 }
 
+// ------------------------------------------------------------------ unaligned rows in registers
+// The phase layout of rmsnorm_stage_kernel without the trip through shared memory, for rows
+// short enough to sit in registers: every interior vector is loaded before the first use and
+// the edge elements are single values in sixteen threads, outside the unrolled slots.  Needs x
+// and y rows in the same phase, w 4-byte aligned and at most THREADS * VPT covering vectors.
+template <int THREADS, int VPT, int DT>
+__global__ void __launch_bounds__(THREADS)
+rmsnorm_regp_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, uint16_t* __restrict__ y,
+                    int64_t D, float inv_D, float eps) {
+    __shared__ float slots[2 * kWarp];
+    const int64_t r = blockIdx.x;
+    const uint16_t* xr = x + r * D;
+    uint16_t* yr = y + r * D;
+    // interior vectors k_lo .. k_hi - 1 live in registers (slot i of thread t holds vector
+    // k_lo + t + i * THREADS); the up to 14 edge elements belong to threads 0..15, one each
+    const int phase = (int)((reinterpret_cast<uintptr_t>(xr) >> 1) & 7);
+    const int nv = (int)((phase + D + 7) >> 3);
+    const int k_lo = phase ? 1 : 0;
+    const int k_hi = ((phase + D) & 7) ? nv - 1 : nv;
+    const uint4* xa = reinterpret_cast<const uint4*>(xr - phase);
+    uint4* ya = reinterpret_cast<uint4*>(yr - phase);
+    const int ek = (threadIdx.x < 8) ? 0 : nv - 1;
+    const bool evec = (threadIdx.x < 8) ? (k_lo == 1) : (k_hi == nv - 1 && !(nv == 1 && k_lo == 1));
+    const int64_t ej = (int64_t)ek * 8 - phase + (threadIdx.x & 7);
+    const bool edge = threadIdx.x < 16 && evec && ej >= 0 && ej < D;
+    uint4 xv[VPT];
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int k = k_lo + threadIdx.x + i * THREADS;
+        xv[i] = (k < k_hi) ? ld_stream(xa + k) : make_uint4(0, 0, 0, 0);
+    }
+    const float xe = edge ? Elem<DT>::to_float(ld_stream_u16(xr + ej)) : 0.0f;
+    float ss = xe * xe;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) ss += sumsq_v<DT>(xv[i]);
+    ss = cta_sum<THREADS>(ss, slots, 0);
+    const float rstd = rsqrtf(fmaf(ss, inv_D, eps));
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int k = k_lo + threadIdx.x + i * THREADS;
+        if (k < k_hi) st_stream(ya + k, scale_v<DT>(xv[i], load_w_shifted(w, (int64_t)k * 8 - phase), rstd));
+    }
+    if (edge) yr[ej] = Elem<DT>::from_float(xe * Elem<DT>::to_float(__ldg(w + ej)) * rstd);
+}
+
 // ------------------------------------------------------------------ generic
 // Any D and any 2-byte alignment.  Row r starts at element r*D, so its 16-byte phase
 // changes from row to row: up to 7 head elements and 7 tail elements are handled with

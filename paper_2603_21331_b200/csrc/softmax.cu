@@ -73,6 +73,28 @@ int launch_stage(const uint16_t* x, uint16_t* y, int64_t rows, int64_t D, size_t
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
+template <int DT, int THREADS, int VPT, int MINB>
+int launch_regp(const uint16_t* x, uint16_t* y, int64_t rows, int64_t D, cudaStream_t st) {
+    softmax_regp_kernel<THREADS, VPT, MINB, DT><<<(unsigned)rows, THREADS, 0, st>>>(x, y, D);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+}
+// unaligned rows held in registers: vectors per thread 1..8 for a CTA of THREADS threads
+template <int DT, int THREADS, int MINB>
+int launch_regp_vpt(int vpt, const uint16_t* x, uint16_t* y, int64_t rows, int64_t D, cudaStream_t st) {
+    switch (vpt) {
+        case 1: return launch_regp<DT, THREADS, 1, 1>(x, y, rows, D, st);
+        case 2: return launch_regp<DT, THREADS, 2, 1>(x, y, rows, D, st);
+        case 3: return launch_regp<DT, THREADS, 3, 1>(x, y, rows, D, st);
+        case 4: return launch_regp<DT, THREADS, 4, 1>(x, y, rows, D, st);
+        case 5: return launch_regp<DT, THREADS, 5, MINB>(x, y, rows, D, st);
+        case 6: return launch_regp<DT, THREADS, 6, MINB>(x, y, rows, D, st);
+        case 7: return launch_regp<DT, THREADS, 7, MINB>(x, y, rows, D, st);
+        case 8: return launch_regp<DT, THREADS, 8, MINB>(x, y, rows, D, st);
+        default: return AK_ERR_SHAPE;
+    }
+}
+
 template <typename K>
 int resident_ctas(K kernel, int threads) {
     int per_sm = 0;
@@ -125,6 +147,10 @@ int dispatch_t(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st,
                 const bool same_phase = ((reinterpret_cast<uintptr_t>(x) ^ reinterpret_cast<uintptr_t>(y)) & 15) == 0;
                 const uint16_t* xs = static_cast<const uint16_t*>(x);
                 uint16_t* ys = static_cast<uint16_t*>(y);
+                // rows of up to 1024 covering vectors stay in the registers of a 128-thread CTA
+                const int64_t max_nv = (D + 14) >> 3;   // vectors covering the row at the worst phase
+                if (same_phase && max_nv <= 1024)
+                    return launch_regp_vpt<DT, 128, 5>((int)((max_nv + 127) / 128), xs, ys, rows, D, st);
                 if (same_phase && stage_bytes <= (size_t)kMaxRowSmemBytes) {
                     if (D <= 8192) return launch_stage<DT, 128>(xs, ys, rows, D, stage_bytes, st);
                     if (D <= 32768) return launch_stage<DT, 256>(xs, ys, rows, D, stage_bytes, st);

@@ -260,6 +260,57 @@ softmax_stage_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, i
         yr[my_j] = Elem<DT>::from_float(fast_exp2(fmaf(Elem<DT>::to_float(row16[my_edge_k * 8 + (threadIdx.x & 7)]), kLog2e, -m2)) * inv);
 }
 
+// ------------------------------------------------------------------ unaligned rows in registers
+// The phase layout of softmax_stage_kernel without the trip through shared memory, for rows
+// short enough to sit in registers (exponentials kept in fp32): interior vectors are loaded
+// before the first use, the edge elements are single values in sixteen threads.  Needs x and y
+// rows in the same phase and at most THREADS * VPT covering vectors.
+template <int THREADS, int VPT, int MINB, int DT>
+__global__ void __launch_bounds__(THREADS, MINB)
+softmax_regp_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, int64_t D) {
+    __shared__ float slots[2 * kWarp];
+    const int64_t r = blockIdx.x;
+    const uint16_t* xr = x + r * D;
+    uint16_t* yr = y + r * D;
+    // interior vectors k_lo .. k_hi - 1 live in registers (slot i of thread t holds vector
+    // k_lo + t + i * THREADS); the up to 14 edge elements belong to threads 0..15, one each
+    const int phase = (int)((reinterpret_cast<uintptr_t>(xr) >> 1) & 7);
+    const int nv = (int)((phase + D + 7) >> 3);
+    const int k_lo = phase ? 1 : 0;
+    const int k_hi = ((phase + D) & 7) ? nv - 1 : nv;
+    const uint4* xa = reinterpret_cast<const uint4*>(xr - phase);
+    uint4* ya = reinterpret_cast<uint4*>(yr - phase);
+    const int ek = (threadIdx.x < 8) ? 0 : nv - 1;
+    const bool evec = (threadIdx.x < 8) ? (k_lo == 1) : (k_hi == nv - 1 && !(nv == 1 && k_lo == 1));
+    const int64_t ej = (int64_t)ek * 8 - phase + (threadIdx.x & 7);
+    const bool edge = threadIdx.x < 16 && evec && ej >= 0 && ej < D;
+    uint4 xv[VPT];
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int k = k_lo + threadIdx.x + i * THREADS;
+        xv[i] = (k < k_hi) ? ld_stream(xa + k) : neg_inf_vec<DT>();
+    }
+    const float xe = edge ? Elem<DT>::to_float(ld_stream_u16(xr + ej)) : -INFINITY;
+    uint32_t mx = neg_inf_word<DT>();
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) mx = max_w<DT>(mx, max_v<DT>(xv[i]));
+    const float m = cta_max<THREADS>(fmaxf(hmax_of<DT>(mx), xe), slots, 0);
+    const float m2 = m * kLog2e;
+    f32x2 e[VPT][4];
+    const float ee = fast_exp2(fmaf(xe, kLog2e, -m2));   // 0 for the threads without an edge element
+    float sum = ee;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) sum += exp_v<DT>(xv[i], m2, e[i]);
+    sum = cta_sum<THREADS>(sum, slots, 1);
+    const float inv = 1.0f / sum;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+        const int k = k_lo + threadIdx.x + i * THREADS;
+        if (k < k_hi) st_stream(ya + k, norm_v<DT>(e[i], inv));
+    }
+    if (edge) yr[ej] = Elem<DT>::from_float(ee * inv);
+}
+
 // ------------------------------------------------------------------ generic
 // Any D / alignment: three passes over the row (max, sum, write); only the first comes
 // from DRAM, the other two are served by L1/L2.
