@@ -135,3 +135,47 @@ def test_fuzz_rope():
         torch.cuda.synchronize()
         assert_close_dt(yv, ref, f"rope {NAME[dtype]} {n_seq}x{S}x{Dh} off {off} pos {pos}", tight=False)
         assert _guards_untouched(ybuf, off, x.numel(), 7.0)
+
+
+def test_two_streams_and_graph_replay():
+    """Re-entrancy: the same ops enqueued on two streams at once (disjoint buffers) give the
+    results of the serial calls; and a captured graph holding one call of every op replays to
+    the same bits."""
+    x, w = synth.rmsnorm_inputs(2048, 4096, 601, device=DEV)
+    xs = synth.softmax_inputs(1024, 8192, 602, device=DEV)
+    lg, tg = synth.xent_inputs(2048, 32000, 603, device=DEV)
+    xl, g, b = synth.layernorm_inputs(2048, 4096, 604, device=DEV)
+    xr = synth.rope_inputs(16, 512, 128, 605, device=DEV, dtype=torch.float16)
+
+    def run_all(stream=None):
+        loss, mean = ak.ak_xent_fwd(lg, tg, stream=stream)
+        return [ak.ak_rmsnorm_fwd(x, w, stream=stream), ak.ak_softmax_fwd(xs, stream=stream), loss, mean,
+                ak.ak_layernorm_fwd(xl, g, b, stream=stream), ak.ak_rowsum_fwd(xl, stream=stream),
+                ak.ak_rope_fwd(xr, stream=stream)]
+
+    serial = [t.clone() for t in run_all()]
+    torch.cuda.synchronize()
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    with torch.cuda.stream(s1):
+        a = run_all(s1)
+    with torch.cuda.stream(s2):
+        c = run_all(s2)
+    torch.cuda.synchronize()
+    for ref, u, v in zip(serial, a, c):
+        assert torch.equal(ref.view(torch.uint8), u.view(torch.uint8))
+        assert torch.equal(ref.view(torch.uint8), v.view(torch.uint8))
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        run_all()                                   # warm-up outside the capture
+        with torch.cuda.graph(graph, stream=side):
+            outs = run_all()
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(2):
+        for t in outs:
+            t.view(torch.uint8).zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        for ref, u in zip(serial, outs):
+            assert torch.equal(ref.view(torch.uint8), u.view(torch.uint8))
