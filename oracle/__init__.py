@@ -43,6 +43,10 @@ def _load():
         lib.oracle_softmax_dt.restype = None
         lib.oracle_xent_dt.argtypes = [p, p, i64, p, p, p, i64, i64, ctypes.c_int]
         lib.oracle_xent_dt.restype = None
+        lib.oracle_layernorm_dt.argtypes = [p, p, p, p, i64, i64, f32, ctypes.c_int]
+        lib.oracle_layernorm_dt.restype = None
+        lib.oracle_rowsum_dt.argtypes = [p, p, i64, i64, ctypes.c_int]
+        lib.oracle_rowsum_dt.restype = None
         lib.oracle_rope.argtypes = [p, p, i64, i64, i64, f32, i64, ctypes.c_int]
         lib.oracle_rope.restype = None
         lib.oracle_rmsnorm.argtypes = [p, p, p, i64, i64, f32]
@@ -141,6 +145,31 @@ def xent_dt(logits, targets, dtype: str, ignore_index: int = -100):
     _load().oracle_xent_dt(x.ctypes.data, t.ctypes.data, int(ignore_index), loss.ctypes.data,
                            ctypes.addressof(mean), ctypes.addressof(cnt), rows, V, DTYPES[dtype])
     return loss, float(mean.value), int(cnt.value)
+
+
+def layernorm_dt(x, gamma, beta, eps: float, dtype: str) -> np.ndarray:
+    """LayerNorm on inputs of element type ``dtype`` (see :func:`layernorm`)."""
+    x = _elems(x, dtype)
+    if x.ndim != 2:
+        raise ValueError("x must be [rows, D]")
+    rows, D = x.shape
+    g = _elems(gamma, dtype, (D,))
+    b = _elems(beta, dtype, (D,))
+    y = np.empty((rows, D), dtype=np.float64)
+    _load().oracle_layernorm_dt(x.ctypes.data, g.ctypes.data, b.ctypes.data, y.ctypes.data, rows, D,
+                                float(np.float32(eps)), DTYPES[dtype])
+    return y
+
+
+def rowsum_dt(x, dtype: str) -> np.ndarray:
+    """out[r] = sum_j x[r, j] for inputs of element type ``dtype``, in float64."""
+    x = _elems(x, dtype)
+    if x.ndim != 2:
+        raise ValueError("x must be [rows, D]")
+    rows, D = x.shape
+    out = np.empty((rows,), dtype=np.float64)
+    _load().oracle_rowsum_dt(x.ctypes.data, out.ctypes.data, rows, D, DTYPES[dtype])
+    return out
 
 
 def rope(x, dtype: str, base: float = 10000.0, pos_offset: int = 0) -> np.ndarray:

@@ -138,40 +138,49 @@ void oracle_rmsnorm(const uint16_t *x, const uint16_t *w, double *y,
  *   mu = (1/D) sum_j x_j ;  var = (1/D) sum_j (x_j - mu)^2   (biased, as in PyTorch)
  *   y_j = (x_j - mu) / sqrt(var + eps) * gamma_j + beta_j
  * x: [rows, D] bf16 bits, gamma/beta: [D] bf16 bits, y: [rows, D] double. */
-void oracle_layernorm(const uint16_t *x, const uint16_t *gamma, const uint16_t *beta, double *y,
-                      int64_t rows, int64_t D, float eps)
+void oracle_layernorm_dt(const void *x, const void *gamma, const void *beta, double *y,
+                         int64_t rows, int64_t D, float eps, int dtype)
 {
     const double eps_d = (double)eps;
 #pragma omp parallel for schedule(static)
     for (int64_t r = 0; r < rows; ++r) {
-        const uint16_t *xr = x + r * D;
+        const char *xr = (const char *)x + r * D * elem_bytes(dtype);
         double *yr = y + r * D;
         double sum = 0.0;
-        for (int64_t j = 0; j < D; ++j) sum += bf16_bits_to_double(xr[j]);
+        for (int64_t j = 0; j < D; ++j) sum += load_elem(xr, j, dtype);
         const double mu = sum / (double)D;
         double sq = 0.0;
         for (int64_t j = 0; j < D; ++j) {
-            double d = bf16_bits_to_double(xr[j]) - mu;
+            double d = load_elem(xr, j, dtype) - mu;
             sq += d * d;
         }
         const double denom = sqrt(sq / (double)D + eps_d);
         for (int64_t j = 0; j < D; ++j)
-            yr[j] = (bf16_bits_to_double(xr[j]) - mu) / denom * bf16_bits_to_double(gamma[j])
-                    + bf16_bits_to_double(beta[j]);
+            yr[j] = (load_elem(xr, j, dtype) - mu) / denom * load_elem(gamma, j, dtype)
+                    + load_elem(beta, j, dtype);
     }
+}
+void oracle_layernorm(const uint16_t *x, const uint16_t *gamma, const uint16_t *beta, double *y,
+                      int64_t rows, int64_t D, float eps)
+{
+    oracle_layernorm_dt(x, gamma, beta, y, rows, D, eps, ORACLE_BF16);
 }
 
 /* Row sum (Table 3 "reduce": hierarchical reduction of each row to one number).
  * x: [rows, D] bf16 bits, out: [rows] double, plain left-to-right sum in double. */
-void oracle_rowsum(const uint16_t *x, double *out, int64_t rows, int64_t D)
+void oracle_rowsum_dt(const void *x, double *out, int64_t rows, int64_t D, int dtype)
 {
 #pragma omp parallel for schedule(static)
     for (int64_t r = 0; r < rows; ++r) {
-        const uint16_t *xr = x + r * D;
+        const char *xr = (const char *)x + r * D * elem_bytes(dtype);
         double sum = 0.0;
-        for (int64_t j = 0; j < D; ++j) sum += bf16_bits_to_double(xr[j]);
+        for (int64_t j = 0; j < D; ++j) sum += load_elem(xr, j, dtype);
         out[r] = sum;
     }
+}
+void oracle_rowsum(const uint16_t *x, double *out, int64_t rows, int64_t D)
+{
+    oracle_rowsum_dt(x, out, rows, D, ORACLE_BF16);
 }
 
 /* Rotary position embedding forward (Table 3 "rotary_emb": interleaved rotation; Table 4

@@ -84,13 +84,13 @@ def rmsnorm_inputs(rows: int, D: int, seed: int, device="cpu", dtype=torch.bfloa
     return x, w
 
 
-def layernorm_inputs(rows: int, D: int, seed: int, device="cpu"):
+def layernorm_inputs(rows: int, D: int, seed: int, device="cpu", dtype=torch.bfloat16):
     """(x bf16 [rows, D] ~ N(0.5, 1.5^2), gamma bf16 [D] = 1 + 0.1 N(0,1), beta bf16 [D] = 0.1 N(0,1)).
     The non-zero mean makes the centring matter."""
     g = _gen(seed, device)
-    x = _normal_bf16(rows, D, 1.5, 0.5, g, device)
-    gamma = _normal_bf16(1, D, 0.1, 1.0, g, device).reshape(D)
-    beta = _normal_bf16(1, D, 0.1, 0.0, g, device).reshape(D)
+    x = _normal_bf16(rows, D, 1.5, 0.5, g, device, dtype)
+    gamma = _normal_bf16(1, D, 0.1, 1.0, g, device, dtype).reshape(D)
+    beta = _normal_bf16(1, D, 0.1, 0.0, g, device, dtype).reshape(D)
     return x, gamma, beta
 
 

@@ -54,6 +54,33 @@ def test_dt_functions_agree_with_the_pinned_bf16_functions_on_shared_values():
         assert np.array_equal(lr, base_x[0]) and lm == base_x[1] and n == base_x[2] == 5
 
 
+def test_layernorm_and_rowsum_dt_agree_with_the_pinned_bf16_functions_and_torch():
+    rng = np.random.default_rng(6)
+    x = rng.integers(-128, 129, size=(5, 41)) / 8.0
+    g = rng.integers(4, 13, size=41) / 8.0
+    b = rng.integers(-8, 9, size=41) / 8.0
+    base_l = oracle.layernorm(bits(x), bits(g), bits(b), 1e-5)
+    base_s = oracle.rowsum(bits(x))
+    for dt in ("bf16", "f16", "f32"):
+        assert np.array_equal(oracle.layernorm_dt(_as(dt, x), _as(dt, g), _as(dt, b), 1e-5, dt), base_l)
+        assert np.array_equal(oracle.rowsum_dt(_as(dt, x), dt), base_s)
+    # values only fp16 / fp32 hold: a row of c and c + 2^-10 alternating has mean c + 2^-11,
+    # deviations +-2^-11, variance 2^-22: y = +-1 / sqrt(1 + eps / 2^-22) exactly in closed form
+    eps32 = float(np.float32(1e-5))
+    for dt in ("f16", "f32"):
+        row = np.where(np.arange(64) % 2 == 0, 1.0, 1.0 + 2.0 ** -10)[None, :]
+        y = oracle.layernorm_dt(_as(dt, row), _as(dt, np.ones(64)), _as(dt, np.zeros(64)), 1e-5, dt)
+        want = np.where(np.arange(64) % 2 == 0, -1.0, 1.0) * 2.0 ** -11 / math.sqrt(2.0 ** -22 + eps32)
+        assert np.allclose(y[0], want, rtol=1e-12)
+        assert oracle.rowsum_dt(_as(dt, row), dt)[0] == 64 + 32 * 2.0 ** -10
+    for dt, tdt in (("f16", torch.float16), ("f32", torch.float32)):
+        x, g, b = synth.layernorm_inputs(9, 1537, seed=84, dtype=tdt)
+        got = oracle.layernorm_dt(synth.to_elems(x), synth.to_elems(g), synth.to_elems(b), 1e-5, dt)
+        want = F.layer_norm(x.double(), (1537,), g.double(), b.double(), float(np.float32(1e-5))).numpy()
+        assert np.allclose(got, want, rtol=1e-11, atol=1e-12)
+        assert np.allclose(oracle.rowsum_dt(synth.to_elems(x), dt), x.double().sum(dim=-1).numpy(), rtol=1e-13)
+
+
 def test_dt_closed_forms_on_values_only_wider_types_hold():
     # c = 1 + 2^-10 (fp16, fp32) and 1 + 2^-20 (fp32 only): constant rows
     eps32 = float(np.float32(1e-6))
