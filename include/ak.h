@@ -107,6 +107,12 @@ int ak_softmax_fwd_dt(const void* x, void* y, int64_t rows, int64_t D,
 int ak_xent_fwd_dt(const void* logits, const int64_t* targets, int64_t ignore_index,
                    float* loss_rows, float* loss_mean, int64_t rows, int64_t V,
                    int dtype, void* cuda_stream, int path, int nsplit);
+/* LayerNorm and row-sum in the element type `dtype` (x, gamma, beta, y; the sums stay fp32);
+ * same rules as the *_dt entry points above. */
+int ak_layernorm_fwd_dt(const void* x, const void* gamma, const void* beta, void* y,
+                        int64_t rows, int64_t D, float eps, int dtype, void* cuda_stream, int path);
+int ak_rowsum_fwd_dt(const void* x, float* out, int64_t rows, int64_t D, int dtype, void* cuda_stream);
+
 /* ---------------------------------------------------------------------------------
  * Rotary position embedding forward (Table 3 "rotary_emb": interleaved rotation; Table 4
  * rows "rotary": batch x heads x sequence x head_dim).
@@ -152,7 +158,7 @@ int ak_xent_vp_merge(const void* partials, int nranks, int nsplit, const int64_t
                      int64_t ignore_index, int64_t V_total, float* loss_rows, float* loss_mean,
                      int64_t rows, void* cuda_stream);
 
-/* Path the dispatcher picks for op (0 = RMSNorm, 1 = softmax) at this shape, alignment and
+/* Path the dispatcher picks for op (0 = RMSNorm, 1 = softmax, 2 = LayerNorm) at this shape, alignment and
  * element type; -1 for an unknown op or dtype.  Pure function; no CUDA calls. */
 int ak_choose_path_dt(int op, int64_t rows, int64_t D, int aligned16, int dtype);
 

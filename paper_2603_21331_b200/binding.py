@@ -40,6 +40,8 @@ SIGNATURES = {
     "ak_softmax_fwd_dt": (_int, [_p, _p, _i64, _i64, _int, _p, _int]),
     "ak_xent_fwd_dt": (_int, [_p, _p, _i64, _p, _p, _i64, _i64, _int, _p, _int, _int]),
     "ak_choose_path_dt": (_int, [_int, _i64, _i64, _int, _int]),
+    "ak_layernorm_fwd_dt": (_int, [_p, _p, _p, _p, _i64, _i64, _f32, _int, _p, _int]),
+    "ak_rowsum_fwd_dt": (_int, [_p, _p, _i64, _i64, _int, _p]),
     "ak_rope_fwd": (_int, [_p, _p, _i64, _i64, _i64, _f32, _i64, _int, _p]),
     "ak_xent_vp_nsplit": (_int, [_i64, _i64]),
     "ak_xent_vp_partial_bytes": (_sz, [_i64, _int]),
@@ -198,6 +200,39 @@ def ak_xent_fwd_dt(logits: torch.Tensor, targets: torch.Tensor, ignore_index: in
     return loss_rows, loss_mean
 
 
+def ak_layernorm_fwd_dt(x: torch.Tensor, gamma: torch.Tensor, beta: torch.Tensor,
+                        y: Optional[torch.Tensor] = None, eps: float = 1e-5, stream=None,
+                        path: int = AK_PATH_AUTO) -> torch.Tensor:
+    """LayerNorm in the element type of x (bf16, fp16 or fp32); gamma, beta and y share it."""
+    dt = _dev_dt(x, "x", 2)
+    _dev_dt(gamma, "gamma", 1, x.dtype)
+    _dev_dt(beta, "beta", 1, x.dtype)
+    rows, D = x.shape
+    if gamma.shape[0] != D or beta.shape[0] != D:
+        raise ValueError("gamma and beta must have D elements")
+    if y is None:
+        y = torch.empty_like(x)
+    _dev_dt(y, "y", 2, x.dtype)
+    if y.shape != x.shape:
+        raise ValueError("y must have the shape of x")
+    _check(lib().ak_layernorm_fwd_dt(x.data_ptr(), gamma.data_ptr(), beta.data_ptr(), y.data_ptr(), rows, D,
+                                     eps, dt, _stream_ptr(stream), path), "ak_layernorm_fwd_dt")
+    return y
+
+
+def ak_rowsum_fwd_dt(x: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Row sums (fp32) of x in bf16, fp16 or fp32."""
+    dt = _dev_dt(x, "x", 2)
+    rows, D = x.shape
+    if out is None:
+        out = torch.empty((rows,), dtype=torch.float32, device=x.device)
+    if not (out.is_cuda and out.dtype == torch.float32 and out.shape == (rows,) and out.is_contiguous()):
+        raise TypeError("out must be a contiguous CUDA float32 tensor [rows]")
+    _check(lib().ak_rowsum_fwd_dt(x.data_ptr(), out.data_ptr(), rows, D, dt, _stream_ptr(stream)),
+           "ak_rowsum_fwd_dt")
+    return out
+
+
 def ak_rope_fwd(x: torch.Tensor, y: Optional[torch.Tensor] = None, base: float = 10000.0,
                 pos_offset: int = 0, stream=None) -> torch.Tensor:
     """Interleaved rotary embedding of x [n_seq, S, Dh] (bf16, fp16 or fp32); y may be x."""
@@ -261,7 +296,7 @@ def ak_xent_vp_merge(partials: torch.Tensor, targets: torch.Tensor, V_total: int
 
 
 def ak_choose_path_dt(op: str, rows: int, D: int, dtype: torch.dtype, aligned16: bool = True) -> int:
-    return int(lib().ak_choose_path_dt({"rmsnorm": 0, "softmax": 1}[op], rows, D, int(aligned16), _DTYPES[dtype]))
+    return int(lib().ak_choose_path_dt({"rmsnorm": 0, "softmax": 1, "layernorm": 2}[op], rows, D, int(aligned16), _DTYPES[dtype]))
 
 
 def ak_layernorm_fwd(x: torch.Tensor, gamma: torch.Tensor, beta: torch.Tensor,

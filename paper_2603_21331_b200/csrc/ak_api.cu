@@ -110,6 +110,25 @@ int ak_xent_fwd_dt(const void* logits, const int64_t* targets, int64_t ignore_in
     return xent_dispatch(logits, targets, ignore_index, loss_rows, loss_mean, rows, V, nullptr, 0, true,
                          static_cast<cudaStream_t>(cuda_stream), path, nsplit, dtype);
 }
+int ak_layernorm_fwd_dt(const void* x, const void* gamma, const void* beta, void* y, int64_t rows, int64_t D,
+                        float eps, int dtype, void* cuda_stream, int path) {
+    if (!known_dtype(dtype)) return AK_ERR_ARG;
+    const size_t es = (size_t)dtype_bytes(dtype);
+    if (int s = validate_rmsnorm(x, gamma, y, rows, D, eps, es)) return s;
+    if (rows != 0 && !beta) return AK_ERR_NULL;
+    if (!is_aligned(beta, es)) return AK_ERR_ALIGN;
+    if (path < AK_PATH_AUTO || path > AK_PATH_SMEM) return AK_ERR_ARG;
+    if (rows == 0) return AK_OK;
+    return layernorm_dispatch(x, gamma, beta, y, rows, D, eps, static_cast<cudaStream_t>(cuda_stream), path, dtype);
+}
+int ak_rowsum_fwd_dt(const void* x, float* out, int64_t rows, int64_t D, int dtype, void* cuda_stream) {
+    if (!known_dtype(dtype)) return AK_ERR_ARG;
+    if (rows != 0 && (!x || !out)) return AK_ERR_NULL;
+    if (int s = check_rows_cols(rows, D)) return s;
+    if (!is_aligned(x, (size_t)dtype_bytes(dtype)) || !is_aligned(out, 4)) return AK_ERR_ALIGN;
+    if (rows == 0) return AK_OK;
+    return rowsum_dispatch(x, out, rows, D, static_cast<cudaStream_t>(cuda_stream), dtype);
+}
 int ak_rope_fwd(const void* x, void* y, int64_t n_seq, int64_t S, int64_t Dh, float base, int64_t pos_offset,
                 int dtype, void* cuda_stream) {
     if (!known_dtype(dtype)) return AK_ERR_ARG;
@@ -165,6 +184,7 @@ int ak_choose_path_dt(int op, int64_t rows, int64_t D, int aligned16, int dtype)
     if (!known_dtype(dtype)) return -1;
     if (op == 0) return rmsnorm_choose(rows, D, aligned16 != 0, dtype);
     if (op == 1) return softmax_choose(rows, D, aligned16 != 0, dtype);
+    if (op == 2) return layernorm_choose(rows, D, aligned16 != 0, dtype);
     return -1;
 }
 

@@ -274,11 +274,11 @@ int xent_vp_merge_launch(const void* parts, int nranks, int nsplit, const int64_
                          int64_t V_total, float* loss_rows, float* loss_mean, int64_t rows, cudaStream_t st);
 int xent_mean_merge_launch(const double* pairs, int64_t n, float* loss_mean, cudaStream_t st);
 int layernorm_dispatch(const void* x, const void* gamma, const void* beta, void* y, int64_t rows, int64_t D,
-                       float eps, cudaStream_t st, int path);
-int layernorm_choose(int64_t rows, int64_t D, bool aligned16);
+                       float eps, cudaStream_t st, int path, int dtype = AK_DTYPE_BF16);
+int layernorm_choose(int64_t rows, int64_t D, bool aligned16, int dtype = AK_DTYPE_BF16);
 int rope_dispatch(const void* x, void* y, int64_t n_seq, int64_t S, int64_t Dh, float base, int64_t pos_offset,
                   int dtype, cudaStream_t st);
-int rowsum_dispatch(const void* x, float* out, int64_t rows, int64_t D, cudaStream_t st);
+int rowsum_dispatch(const void* x, float* out, int64_t rows, int64_t D, cudaStream_t st, int dtype = AK_DTYPE_BF16);
 int rmsnorm_choose(int64_t rows, int64_t D, bool aligned16, int dtype = AK_DTYPE_BF16);
 int softmax_choose(int64_t rows, int64_t D, bool aligned16, int dtype = AK_DTYPE_BF16);
 int xent_choose(int64_t rows, int64_t V, int* nsplit);

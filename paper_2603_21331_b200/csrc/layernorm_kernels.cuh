@@ -1,7 +1,7 @@
 // LayerNorm forward device kernels (paper Table 3 "layernorm"; Table 4 rows "layernorm").
 //
 //   mu = mean_k x[r, k];  var = mean_k (x[r, k] - mu)^2  (biased);
-//   y[r, j] = bf16_rne( (x[r, j] - mu) * rsqrt(var + eps) * gamma[j] + beta[j] )
+//   y[r, j] = rne( (x[r, j] - mu) * rsqrt(var + eps) * gamma[j] + beta[j] )
 //
 // The paper's kernel is a single-pass Welford.  Here the row already sits in registers (or
 // shared memory) after its one trip from HBM, so the moments are taken in two exact-order
@@ -10,65 +10,106 @@
 // exactly zero and mu == K exactly; in general the partial sums stay small, so fp32 does not
 // lose the low bits of large activations), then the sum of squared deviations from mu.
 // One DRAM read and one DRAM write per element.  Differences x - K and x - mu come straight
-// from the packed bf16 halves with the mixed-precision subtract (no widening instruction).
+// from the packed 16-bit halves with the mixed-precision subtract (no widening instruction).
+// Kernels take the element type DT (bf16, fp16, fp32) as a template parameter; the phase-staged
+// and multi-pass kernels serve the 16-bit types, unaligned fp32 rows go to
+// layernorm_generic32_kernel.
 #pragma once
 
 #include "ak_common.cuh"
 
 namespace ak {
 
+// Vector helpers per element type DT (16-byte vectors: 8 bf16 / fp16 or 4 fp32 elements).
 __device__ __forceinline__ void ln_halves(uint32_t u, uint16_t& lo, uint16_t& hi) {
     asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(u));
 }
-// x - c with x a bf16 half: exact operand, one rounding
-__device__ __forceinline__ float sub_bf16(uint16_t x, float c) {
+// x - c with x a 16-bit element: exact operand, one rounding
+template <int DT>
+__device__ __forceinline__ float sub_h(uint16_t x, float c) {
     float d;
-    asm("sub.rn.f32.bf16 %0, %1, %2;" : "=f"(d) : "h"(x), "f"(c));
+    if constexpr (DT == AK_DTYPE_F16) asm("sub.rn.f32.f16 %0, %1, %2;" : "=f"(d) : "h"(x), "f"(c));
+    else asm("sub.rn.f32.bf16 %0, %1, %2;" : "=f"(d) : "h"(x), "f"(c));
     return d;
 }
+template <int DT>
 __device__ __forceinline__ f32x2 dev2(uint32_t u, float c) {
     uint16_t lo, hi;
     ln_halves(u, lo, hi);
-    return pack2(sub_bf16(lo, c), sub_bf16(hi, c));
+    return pack2(sub_h<DT>(lo, c), sub_h<DT>(hi, c));
 }
-// sum over the 8 elements of (x - c)
-__device__ __forceinline__ float sumdev8(const uint4& v, float c) {
+// sum over the elements of (x - c)
+template <int DT>
+__device__ __forceinline__ float sumdev_v(const uint4& v, float c) {
     float lo, hi;
-    unpack2(add2(add2(dev2(v.x, c), dev2(v.y, c)), add2(dev2(v.z, c), dev2(v.w, c))), lo, hi);
+    if constexpr (DT == AK_DTYPE_F32) {
+        const f32x2 c2 = pack2(c, c);
+        unpack2(add2(sub2(pack2(__uint_as_float(v.x), __uint_as_float(v.y)), c2),
+                     sub2(pack2(__uint_as_float(v.z), __uint_as_float(v.w)), c2)), lo, hi);
+    } else {
+        unpack2(add2(add2(dev2<DT>(v.x, c), dev2<DT>(v.y, c)), add2(dev2<DT>(v.z, c), dev2<DT>(v.w, c))), lo, hi);
+    }
     return lo + hi;
 }
-// sum over the 8 elements of (x - c)^2
-__device__ __forceinline__ float sqdev8(const uint4& v, float c) {
-    const f32x2 a = dev2(v.x, c), b = dev2(v.y, c), d = dev2(v.z, c), e = dev2(v.w, c);
-    f32x2 s = mul2(a, a);
-    s = fma2(b, b, s);
-    s = fma2(d, d, s);
-    s = fma2(e, e, s);
+// sum over the elements of (x - c)^2
+template <int DT>
+__device__ __forceinline__ float sqdev_v(const uint4& v, float c) {
     float lo, hi;
-    unpack2(s, lo, hi);
+    if constexpr (DT == AK_DTYPE_F32) {
+        const f32x2 c2 = pack2(c, c);
+        const f32x2 a = sub2(pack2(__uint_as_float(v.x), __uint_as_float(v.y)), c2);
+        const f32x2 b = sub2(pack2(__uint_as_float(v.z), __uint_as_float(v.w)), c2);
+        unpack2(fma2(b, b, mul2(a, a)), lo, hi);
+    } else {
+        const f32x2 a = dev2<DT>(v.x, c), b = dev2<DT>(v.y, c), d = dev2<DT>(v.z, c), e = dev2<DT>(v.w, c);
+        f32x2 s = mul2(a, a);
+        s = fma2(b, b, s);
+        s = fma2(d, d, s);
+        s = fma2(e, e, s);
+        unpack2(s, lo, hi);
+    }
     return lo + hi;
 }
-// ((x - mu) * rstd) * gamma + beta for one packed pair, rounded once to bf16
+// ((x - mu) * rstd) * gamma + beta per element, rounded once to the output type
+template <int DT>
 __device__ __forceinline__ uint32_t ln_out2(uint32_t x, uint32_t g, uint32_t b, float mu, f32x2 rstd2) {
-    const f32x2 t = fma2(mul2(dev2(x, mu), rstd2), widen2(g), widen2(b));
+    const f32x2 t = fma2(mul2(dev2<DT>(x, mu), rstd2), widen2_t<DT>(g), widen2_t<DT>(b));
     float lo, hi;
     unpack2(t, lo, hi);
-    return pack_bf16x2(lo, hi);
+    return Elem<DT>::pack(lo, hi);
 }
-__device__ __forceinline__ uint4 ln_out8(const uint4& x, const uint4& g, const uint4& b, float mu, float rstd) {
+template <int DT>
+__device__ __forceinline__ uint4 ln_out_v(const uint4& x, const uint4& g, const uint4& b, float mu, float rstd) {
     const f32x2 r2 = pack2(rstd, rstd);
-    return make_uint4(ln_out2(x.x, g.x, b.x, mu, r2), ln_out2(x.y, g.y, b.y, mu, r2),
-                      ln_out2(x.z, g.z, b.z, mu, r2), ln_out2(x.w, g.w, b.w, mu, r2));
+    if constexpr (DT == AK_DTYPE_F32) {
+        const f32x2 m2 = pack2(mu, mu);
+        float o0, o1, o2, o3;
+        unpack2(fma2(mul2(sub2(pack2(__uint_as_float(x.x), __uint_as_float(x.y)), m2), r2),
+                     pack2(__uint_as_float(g.x), __uint_as_float(g.y)), pack2(__uint_as_float(b.x), __uint_as_float(b.y))), o0, o1);
+        unpack2(fma2(mul2(sub2(pack2(__uint_as_float(x.z), __uint_as_float(x.w)), m2), r2),
+                     pack2(__uint_as_float(g.z), __uint_as_float(g.w)), pack2(__uint_as_float(b.z), __uint_as_float(b.w))), o2, o3);
+        return make_uint4(__float_as_uint(o0), __float_as_uint(o1), __float_as_uint(o2), __float_as_uint(o3));
+    } else {
+        return make_uint4(ln_out2<DT>(x.x, g.x, b.x, mu, r2), ln_out2<DT>(x.y, g.y, b.y, mu, r2),
+                          ln_out2<DT>(x.z, g.z, b.z, mu, r2), ln_out2<DT>(x.w, g.w, b.w, mu, r2));
+    }
 }
+template <int DT>
 __device__ __forceinline__ float ln_out1(uint16_t x, uint16_t g, uint16_t b, float mu, float rstd) {
-    return fmaf(sub_bf16(x, mu) * rstd, bf16_to_float(g), bf16_to_float(b));
+    return fmaf(sub_h<DT>(x, mu) * rstd, Elem<DT>::to_float(g), Elem<DT>::to_float(b));
+}
+// first element of a row (any element type), the shift K of the mean
+template <int DT>
+__device__ __forceinline__ float first_elem(const void* row) {
+    if constexpr (DT == AK_DTYPE_F32) return __ldg(static_cast<const float*>(row));
+    else return Elem<DT>::to_float(__ldg(static_cast<const uint16_t*>(row)));
 }
 
 // ------------------------------------------------------------------ row in registers
 // Same thread layout as the RMSNorm register kernel (a group of GROUP threads owns a row,
 // thread t holds vectors t, t + GROUP, ...), two reductions per row.  Padding slots hold
 // copies of K so they add exactly zero to the first sum and are excluded from the second.
-template <int THREADS, int GROUP, int VPT, int MINB>
+template <int THREADS, int GROUP, int VPT, int MINB, int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(THREADS, MINB)
 layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamma, const uint4* __restrict__ beta,
                      uint4* __restrict__ y, int64_t rows, int nvec, float inv_D, float eps) {
@@ -85,7 +126,7 @@ layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamm
         const int64_t row = row0 + g;
         const bool live = row < rows;
         const uint4* xr = x + row * nvec;
-        const float K = live ? bf16_to_float(__ldg(reinterpret_cast<const uint16_t*>(xr))) : 0.0f;
+        const float K = live ? first_elem<DT>(xr) : 0.0f;
         uint4 xv[VPT];
 #pragma unroll
         for (int k = 0; k < VPT; ++k) {
@@ -95,7 +136,7 @@ layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamm
         float s1 = 0.0f;
 #pragma unroll
         for (int k = 0; k < VPT; ++k)
-            if (live && t + k * GROUP < nvec) s1 += sumdev8(xv[k], K);
+            if (live && t + k * GROUP < nvec) s1 += sumdev_v<DT>(xv[k], K);
         s1 = warp_sum(s1);
         if constexpr (WARPS_PER_GROUP > 1) {
             float* s = slots[0] + g * WARPS_PER_GROUP;
@@ -107,7 +148,7 @@ layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamm
         float s2 = 0.0f;
 #pragma unroll
         for (int k = 0; k < VPT; ++k)
-            if (live && t + k * GROUP < nvec) s2 += sqdev8(xv[k], mu);
+            if (live && t + k * GROUP < nvec) s2 += sqdev_v<DT>(xv[k], mu);
         s2 = warp_sum(s2);
         if constexpr (WARPS_PER_GROUP > 1) {
             float* s = slots[1] + g * WARPS_PER_GROUP;
@@ -120,7 +161,7 @@ layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamm
 #pragma unroll
         for (int k = 0; k < VPT; ++k) {
             const int i = t + k * GROUP;
-            if (live && i < nvec) st_stream(yr + i, ln_out8(xv[k], __ldg(gamma + i), __ldg(beta + i), mu, rstd));
+            if (live && i < nvec) st_stream(yr + i, ln_out_v<DT>(xv[k], __ldg(gamma + i), __ldg(beta + i), mu, rstd));
         }
     }
 }
@@ -131,7 +172,7 @@ layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamm
 // Dynamic shared memory = nvec * 16 bytes.
 constexpr uint32_t kLnBulkChunk = 32768;
 
-template <int THREADS>
+template <int THREADS, int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(THREADS, 1)
 layernorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamma, const uint4* __restrict__ beta,
                       uint4* __restrict__ y, int nvec, float inv_D, float eps) {
@@ -150,21 +191,23 @@ layernorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gam
             bulk_load(smem_raw + off, src + off, min(kLnBulkChunk, bytes - off), &bar);
     }
     if (!mbar_wait(&bar, 0)) return;  // uniform: every thread waits on the same barrier
-    const float K = bf16_to_float(reinterpret_cast<const uint16_t*>(smem_raw)[0]);
+    float K;
+    if constexpr (DT == AK_DTYPE_F32) K = reinterpret_cast<const float*>(smem_raw)[0];
+    else K = Elem<DT>::to_float(reinterpret_cast<const uint16_t*>(smem_raw)[0]);
     float s1 = 0.0f;
 #pragma unroll 4
-    for (int i = threadIdx.x; i < nvec; i += THREADS) s1 += sumdev8(row[i], K);
+    for (int i = threadIdx.x; i < nvec; i += THREADS) s1 += sumdev_v<DT>(row[i], K);
     s1 = cta_sum<THREADS>(s1, slots, 0);
     const float mu = fmaf(s1, inv_D, K);
     float s2 = 0.0f;
 #pragma unroll 4
-    for (int i = threadIdx.x; i < nvec; i += THREADS) s2 += sqdev8(row[i], mu);
+    for (int i = threadIdx.x; i < nvec; i += THREADS) s2 += sqdev_v<DT>(row[i], mu);
     s2 = cta_sum<THREADS>(s2, slots, 1);
     const float rstd = rsqrtf(fmaf(s2, inv_D, eps));
     uint4* yr = y + r * nvec;
 #pragma unroll 2
     for (int i = threadIdx.x; i < nvec; i += THREADS)
-        st_stream(yr + i, ln_out8(row[i], __ldg(gamma + i), __ldg(beta + i), mu, rstd));
+        st_stream(yr + i, ln_out_v<DT>(row[i], __ldg(gamma + i), __ldg(beta + i), mu, rstd));
 }
 
 // ------------------------------------------------------------------ unaligned rows staged in shared memory
@@ -184,7 +227,7 @@ __device__ __forceinline__ uint4 ln_load_shifted(const uint16_t* __restrict__ p,
                       __funnelshift_r(d, e, 16));
 }
 
-template <int T>
+template <int T, int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(T)
 layernorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ gamma,
                        const uint16_t* __restrict__ beta, uint16_t* __restrict__ y, int64_t D, float inv_D,
@@ -212,26 +255,26 @@ layernorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restric
     for (int k = k_lo + threadIdx.x; k < k_hi; k += T) row[k] = ld_stream(xa + k);
     if (edge) row16[ek * 8 + (threadIdx.x & 7)] = ld_stream_u16(xr + ej);
     __syncthreads();
-    const float K = bf16_to_float(row16[phase]);
+    const float K = Elem<DT>::to_float(row16[phase]);
     float s1 = 0.0f;
-    for (int k = k_lo + threadIdx.x; k < k_hi; k += T) s1 += sumdev8(row[k], K);
-    if (edge) s1 += sub_bf16(row16[ek * 8 + (threadIdx.x & 7)], K);
+    for (int k = k_lo + threadIdx.x; k < k_hi; k += T) s1 += sumdev_v<DT>(row[k], K);
+    if (edge) s1 += sub_h<DT>(row16[ek * 8 + (threadIdx.x & 7)], K);
     s1 = cta_sum<T>(s1, slots, 0);
     const float mu = fmaf(s1, inv_D, K);
     float s2 = 0.0f;
-    for (int k = k_lo + threadIdx.x; k < k_hi; k += T) s2 += sqdev8(row[k], mu);
+    for (int k = k_lo + threadIdx.x; k < k_hi; k += T) s2 += sqdev_v<DT>(row[k], mu);
     if (edge) {
-        const float d = sub_bf16(row16[ek * 8 + (threadIdx.x & 7)], mu);
+        const float d = sub_h<DT>(row16[ek * 8 + (threadIdx.x & 7)], mu);
         s2 = fmaf(d, d, s2);
     }
     s2 = cta_sum<T>(s2, slots, 1);
     const float rstd = rsqrtf(fmaf(s2, inv_D, eps));
     for (int k = k_lo + threadIdx.x; k < k_hi; k += T) {
         const int64_t j0 = (int64_t)k * 8 - phase;
-        st_stream(ya + k, ln_out8(row[k], ln_load_shifted(gamma, j0), ln_load_shifted(beta, j0), mu, rstd));
+        st_stream(ya + k, ln_out_v<DT>(row[k], ln_load_shifted(gamma, j0), ln_load_shifted(beta, j0), mu, rstd));
     }
     if (edge)
-        yr[ej] = float_to_bf16(ln_out1(row16[ek * 8 + (threadIdx.x & 7)], __ldg(gamma + ej), __ldg(beta + ej), mu, rstd));
+        yr[ej] = Elem<DT>::from_float(ln_out1<DT>(row16[ek * 8 + (threadIdx.x & 7)], __ldg(gamma + ej), __ldg(beta + ej), mu, rstd));
 }
 
 // ------------------------------------------------------------------ unaligned rows in registers
@@ -239,7 +282,7 @@ layernorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restric
 // short enough to sit in registers: interior vectors are loaded before the first use, the edge
 // elements are single values in sixteen threads.  Needs x and y rows in the same phase, gamma
 // and beta 4-byte aligned and at most THREADS * VPT covering vectors.
-template <int THREADS, int VPT, int MINB>
+template <int THREADS, int VPT, int MINB, int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(THREADS, MINB)
 layernorm_regp_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ gamma,
                       const uint16_t* __restrict__ beta, uint16_t* __restrict__ y, int64_t D, float inv_D, float eps) {
@@ -259,7 +302,7 @@ layernorm_regp_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict
     const bool evec = (threadIdx.x < 8) ? (k_lo == 1) : (k_hi == nv - 1 && !(nv == 1 && k_lo == 1));
     const int64_t ej = (int64_t)ek * 8 - phase + (threadIdx.x & 7);
     const bool edge = threadIdx.x < 16 && evec && ej >= 0 && ej < D;
-    const float K = bf16_to_float(__ldg(xr));
+    const float K = Elem<DT>::to_float(__ldg(xr));
     uint4 xv[VPT];
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
@@ -267,17 +310,17 @@ layernorm_regp_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict
         if (k < k_hi) xv[i] = ld_stream(xa + k);
     }
     const uint16_t xe = edge ? ld_stream_u16(xr + ej) : (uint16_t)0;
-    float s1 = edge ? sub_bf16(xe, K) : 0.0f;
+    float s1 = edge ? sub_h<DT>(xe, K) : 0.0f;
 #pragma unroll
     for (int i = 0; i < VPT; ++i)
-        if (k_lo + (int)threadIdx.x + i * THREADS < k_hi) s1 += sumdev8(xv[i], K);
+        if (k_lo + (int)threadIdx.x + i * THREADS < k_hi) s1 += sumdev_v<DT>(xv[i], K);
     s1 = cta_sum<THREADS>(s1, slots, 0);
     const float mu = fmaf(s1, inv_D, K);
-    const float de = edge ? sub_bf16(xe, mu) : 0.0f;
+    const float de = edge ? sub_h<DT>(xe, mu) : 0.0f;
     float s2 = de * de;
 #pragma unroll
     for (int i = 0; i < VPT; ++i)
-        if (k_lo + (int)threadIdx.x + i * THREADS < k_hi) s2 += sqdev8(xv[i], mu);
+        if (k_lo + (int)threadIdx.x + i * THREADS < k_hi) s2 += sqdev_v<DT>(xv[i], mu);
     s2 = cta_sum<THREADS>(s2, slots, 1);
     const float rstd = rsqrtf(fmaf(s2, inv_D, eps));
 #pragma unroll
@@ -285,10 +328,10 @@ layernorm_regp_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict
         const int k = k_lo + threadIdx.x + i * THREADS;
         if (k < k_hi) {
             const int64_t j0 = (int64_t)k * 8 - phase;
-            st_stream(ya + k, ln_out8(xv[i], ln_load_shifted(gamma, j0), ln_load_shifted(beta, j0), mu, rstd));
+            st_stream(ya + k, ln_out_v<DT>(xv[i], ln_load_shifted(gamma, j0), ln_load_shifted(beta, j0), mu, rstd));
         }
     }
-    if (edge) yr[ej] = float_to_bf16(ln_out1(xe, __ldg(gamma + ej), __ldg(beta + ej), mu, rstd));
+    if (edge) yr[ej] = Elem<DT>::from_float(ln_out1<DT>(xe, __ldg(gamma + ej), __ldg(beta + ej), mu, rstd));
 }
 
 // ------------------------------------------------------------------ generic
@@ -297,6 +340,7 @@ layernorm_regp_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict
 // shapes never reach it.
 constexpr int kLnGenericThreads = 256;
 
+template <int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(kLnGenericThreads)
 layernorm_generic_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ gamma,
                          const uint16_t* __restrict__ beta, uint16_t* __restrict__ y, int64_t rows, int64_t D,
@@ -306,20 +350,45 @@ layernorm_generic_kernel(const uint16_t* __restrict__ x, const uint16_t* __restr
     for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
         const uint16_t* xr = x + row * D;
         uint16_t* yr = y + row * D;
-        const float K = bf16_to_float(xr[0]);
+        const float K = Elem<DT>::to_float(xr[0]);
         float s1 = 0.0f;
-        for (int64_t j = threadIdx.x; j < D; j += T) s1 += sub_bf16(xr[j], K);
+        for (int64_t j = threadIdx.x; j < D; j += T) s1 += sub_h<DT>(xr[j], K);
         s1 = cta_sum<T>(s1, slots, 0);
         const float mu = fmaf(s1, inv_D, K);
         float s2 = 0.0f;
         for (int64_t j = threadIdx.x; j < D; j += T) {
-            const float d = sub_bf16(xr[j], mu);
+            const float d = sub_h<DT>(xr[j], mu);
             s2 = fmaf(d, d, s2);
         }
         s2 = cta_sum<T>(s2, slots, 1);
         const float rstd = rsqrtf(fmaf(s2, inv_D, eps));
         for (int64_t j = threadIdx.x; j < D; j += T)
-            yr[j] = float_to_bf16(ln_out1(xr[j], __ldg(gamma + j), __ldg(beta + j), mu, rstd));
+            yr[j] = Elem<DT>::from_float(ln_out1<DT>(xr[j], __ldg(gamma + j), __ldg(beta + j), mu, rstd));
+    }
+}
+
+// fp32 rows with no 16-byte alignment: element-wise, three passes (the last two from L1/L2).
+__global__ void __launch_bounds__(kLnGenericThreads)
+layernorm_generic32_kernel(const float* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
+                           float* __restrict__ y, int64_t rows, int64_t D, float inv_D, float eps) {
+    constexpr int T = kLnGenericThreads;
+    __shared__ float slots[2 * kWarp];
+    for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+        const float* xr = x + row * D;
+        float* yr = y + row * D;
+        const float K = xr[0];
+        float s1 = 0.0f;
+        for (int64_t j = threadIdx.x; j < D; j += T) s1 += xr[j] - K;
+        s1 = cta_sum<T>(s1, slots, 0);
+        const float mu = fmaf(s1, inv_D, K);
+        float s2 = 0.0f;
+        for (int64_t j = threadIdx.x; j < D; j += T) {
+            const float d = xr[j] - mu;
+            s2 = fmaf(d, d, s2);
+        }
+        s2 = cta_sum<T>(s2, slots, 1);
+        const float rstd = rsqrtf(fmaf(s2, inv_D, eps));
+        for (int64_t j = threadIdx.x; j < D; j += T) yr[j] = fmaf((xr[j] - mu) * rstd, __ldg(gamma + j), __ldg(beta + j));
     }
 }
 

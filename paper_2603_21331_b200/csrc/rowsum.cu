@@ -1,41 +1,61 @@
-// Row-sum reduce (paper Table 3 "reduce"): out[r] = sum_j x[r, j], bf16 in, fp32 accumulate
-// and out.  Read-only streaming: 2 bytes per element from HBM, 4 bytes per row back.
+// Row-sum reduce (paper Table 3 "reduce"): out[r] = sum_j x[r, j], bf16 / fp16 / fp32 in, fp32
+// accumulate and out.  Read-only streaming: one read of every element, 4 bytes per row back.
 //
-// A group of GROUP threads owns a row.  Rows need no alignment beyond 2 bytes: up to 7 head
-// elements bring the row to a 16-byte boundary, the body is read as 16-byte vectors (UNROLL
-// independent loads in flight per thread) and up to 7 tail elements finish it.  Every thread
-// keeps eight lane accumulators fed straight from the bf16 halves by the mixed-precision add;
-// the combine order (lanes pairwise, XOR butterfly over the warp, then over the group's warps)
-// is fixed, so results are bitwise reproducible.
+// A group of GROUP threads owns a row.  Rows need no alignment beyond the element's own: a few
+// head elements bring the row to a 16-byte boundary, the body is read as 16-byte vectors
+// (UNROLL independent loads in flight per thread) and a few tail elements finish it.  Every
+// thread keeps eight lane accumulators (16-bit types: fed straight from the packed halves by
+// the mixed-precision add; fp32: four of them, one per vector lane); the combine order (lanes
+// pairwise, XOR butterfly over the warp, then over the group's warps) is fixed, so results
+// are bitwise reproducible.
 #include "ak_common.cuh"
 
 namespace ak {
 namespace {
 
-__device__ __forceinline__ float add_bf16(uint16_t x, float c) {
+template <int DT>
+__device__ __forceinline__ float add_h(uint16_t x, float c) {   // x + c, x a 16-bit element (exact operand)
     float d;
-    asm("add.rn.f32.bf16 %0, %1, %2;" : "=f"(d) : "h"(x), "f"(c));
+    if constexpr (DT == AK_DTYPE_F16) asm("add.rn.f32.f16 %0, %1, %2;" : "=f"(d) : "h"(x), "f"(c));
+    else asm("add.rn.f32.bf16 %0, %1, %2;" : "=f"(d) : "h"(x), "f"(c));
     return d;
 }
+template <int DT>
 __device__ __forceinline__ void acc_pair(uint32_t u, float& a, float& b) {
     uint16_t lo, hi;
     asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(u));
-    a = add_bf16(lo, a);
-    b = add_bf16(hi, b);
+    a = add_h<DT>(lo, a);
+    b = add_h<DT>(hi, b);
 }
-__device__ __forceinline__ void acc8(const uint4& v, float (&a)[8]) {
-    acc_pair(v.x, a[0], a[1]);
-    acc_pair(v.y, a[2], a[3]);
-    acc_pair(v.z, a[4], a[5]);
-    acc_pair(v.w, a[6], a[7]);
+template <int DT>
+__device__ __forceinline__ void acc_v(const uint4& v, float (&a)[8]) {
+    if constexpr (DT == AK_DTYPE_F32) {
+        a[0] += __uint_as_float(v.x);
+        a[1] += __uint_as_float(v.y);
+        a[2] += __uint_as_float(v.z);
+        a[3] += __uint_as_float(v.w);
+    } else {
+        acc_pair<DT>(v.x, a[0], a[1]);
+        acc_pair<DT>(v.y, a[2], a[3]);
+        acc_pair<DT>(v.z, a[4], a[5]);
+        acc_pair<DT>(v.w, a[6], a[7]);
+    }
+}
+template <int DT> struct RsElem { using type = uint16_t; };
+template <> struct RsElem<AK_DTYPE_F32> { using type = float; };
+template <int DT>
+__device__ __forceinline__ float load_one(const typename RsElem<DT>::type* p) {
+    if constexpr (DT == AK_DTYPE_F32) return __ldcs(p); else return Elem<DT>::to_float(ld_stream_u16(p));
 }
 
-template <int THREADS, int GROUP, int UNROLL, int MINB>
+template <int THREADS, int GROUP, int UNROLL, int MINB, int DT>
 __global__ void __launch_bounds__(THREADS, MINB)
-rowsum_kernel(const uint16_t* __restrict__ x, float* __restrict__ out, int64_t rows, int64_t D) {
+rowsum_kernel(const typename RsElem<DT>::type* __restrict__ x, float* __restrict__ out, int64_t rows, int64_t D) {
     constexpr int GROUPS = THREADS / GROUP;
     constexpr int WARPS_PER_GROUP = GROUP / kWarp;
+    constexpr int PV = Elem<DT>::kPerVec, LOG_PV = (PV == 8) ? 3 : 2, LOG_BYTES = (Elem<DT>::kBytes == 2) ? 1 : 2;
     static_assert(GROUP % kWarp == 0 && THREADS % GROUP == 0, "groups are whole warps");
+    static_assert(GROUP >= PV, "head and tail elements take one thread each");
     __shared__ float slots[THREADS / kWarp];
     const int g = threadIdx.x / GROUP;
     const int t = threadIdx.x % GROUP;
@@ -45,12 +65,12 @@ rowsum_kernel(const uint16_t* __restrict__ x, float* __restrict__ out, int64_t r
 
     float a[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
     if (live) {
-        const uint16_t* xr = x + row * D;
-        const int phase = (int)((reinterpret_cast<uintptr_t>(xr) >> 1) & 7);
-        int64_t head = (8 - phase) & 7;
+        const typename RsElem<DT>::type* xr = x + row * D;
+        const int phase = (int)((reinterpret_cast<uintptr_t>(xr) >> LOG_BYTES) & (PV - 1));
+        int64_t head = (PV - phase) & (PV - 1);
         if (head > D) head = D;
-        const int64_t nbody = (D - head) >> 3;
-        const int64_t tail0 = head + (nbody << 3);
+        const int64_t nbody = (D - head) >> LOG_PV;
+        const int64_t tail0 = head + (nbody << LOG_PV);
         const uint4* xb = reinterpret_cast<const uint4*>(xr + head);
         int64_t i = t;
         for (; i + (int64_t)(UNROLL - 1) * GROUP < nbody; i += (int64_t)UNROLL * GROUP) {
@@ -58,11 +78,11 @@ rowsum_kernel(const uint16_t* __restrict__ x, float* __restrict__ out, int64_t r
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) v[u] = ld_stream(xb + i + (int64_t)u * GROUP);
 #pragma unroll
-            for (int u = 0; u < UNROLL; ++u) acc8(v[u], a);
+            for (int u = 0; u < UNROLL; ++u) acc_v<DT>(v[u], a);
         }
-        for (; i < nbody; i += GROUP) acc8(ld_stream(xb + i), a);
-        if (t < head) a[0] = add_bf16(ld_stream_u16(xr + t), a[0]);
-        if (tail0 + t < D) a[1] = add_bf16(ld_stream_u16(xr + tail0 + t), a[1]);
+        for (; i < nbody; i += GROUP) acc_v<DT>(ld_stream(xb + i), a);
+        if (t < head) a[0] += load_one<DT>(xr + t);
+        if (tail0 + t < D) a[1] += load_one<DT>(xr + tail0 + t);
     }
     float s = ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
     s = warp_sum(s);
@@ -75,23 +95,34 @@ rowsum_kernel(const uint16_t* __restrict__ x, float* __restrict__ out, int64_t r
     if (live && t == 0) out[row] = s;
 }
 
-template <int THREADS, int GROUP, int UNROLL, int MINB>
+template <int DT, int THREADS, int GROUP, int UNROLL, int MINB>
 int launch(const void* x, float* out, int64_t rows, int64_t D, cudaStream_t st) {
     constexpr int GROUPS = THREADS / GROUP;
     const int64_t grid = (rows + GROUPS - 1) / GROUPS;
     if (grid > 2147483647LL) return AK_ERR_SHAPE;
-    rowsum_kernel<THREADS, GROUP, UNROLL, MINB><<<(unsigned)grid, THREADS, 0, st>>>(
-        static_cast<const uint16_t*>(x), out, rows, D);
+    rowsum_kernel<THREADS, GROUP, UNROLL, MINB, DT><<<(unsigned)grid, THREADS, 0, st>>>(
+        static_cast<const typename RsElem<DT>::type*>(x), out, rows, D);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
+template <int DT>
+int dispatch_t(const void* x, float* out, int64_t rows, int64_t D, cudaStream_t st) {
+    const int64_t row_bytes = D * Elem<DT>::kBytes;
+    if (row_bytes <= 2048) return launch<DT, 256, 32, 4, 4>(x, out, rows, D, st);    // a warp per row
+    if (row_bytes <= 32768) return launch<DT, 128, 128, 4, 8>(x, out, rows, D, st);  // a 128-thread CTA per row
+    return launch<DT, 256, 256, 8, 4>(x, out, rows, D, st);
+}
+
 }  // namespace
 
-int rowsum_dispatch(const void* x, float* out, int64_t rows, int64_t D, cudaStream_t st) {
-    if (D <= 1024) return launch<256, 32, 4, 4>(x, out, rows, D, st);    // a warp per row
-    if (D <= 16384) return launch<128, 128, 4, 8>(x, out, rows, D, st);  // a 128-thread CTA per row
-    return launch<256, 256, 8, 4>(x, out, rows, D, st);
+int rowsum_dispatch(const void* x, float* out, int64_t rows, int64_t D, cudaStream_t st, int dtype) {
+    switch (dtype) {
+        case AK_DTYPE_BF16: return dispatch_t<AK_DTYPE_BF16>(x, out, rows, D, st);
+        case AK_DTYPE_F16: return dispatch_t<AK_DTYPE_F16>(x, out, rows, D, st);
+        case AK_DTYPE_F32: return dispatch_t<AK_DTYPE_F32>(x, out, rows, D, st);
+        default: return AK_ERR_ARG;
+    }
 }
 
 }  // namespace ak

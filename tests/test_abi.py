@@ -77,7 +77,11 @@ def test_validation_rejects_before_any_cuda_call():
     assert l.ak_choose_path_dt(0, 8192, 1022, 1, 2) == ak.AK_PATH_GENERIC   # 4088 B: not a multiple of 16
     assert l.ak_choose_path_dt(1, 8192, 8192, 1, 2) == ak.AK_PATH_SMEM      # 32 KiB fp32 softmax rows
     assert l.ak_choose_path_dt(1, 8192, 8192, 1, 1) == ak.AK_PATH_CTA
-    assert l.ak_choose_path_dt(2, 1, 8, 1, 0) == -1 and l.ak_choose_path_dt(0, 1, 8, 1, 9) == -1
+    assert l.ak_choose_path_dt(3, 1, 8, 1, 0) == -1 and l.ak_choose_path_dt(0, 1, 8, 1, 9) == -1
+    assert l.ak_choose_path_dt(2, 8192, 4096, 1, 2) == ak.AK_PATH_CTA and l.ak_choose_path_dt(2, 8192, 4096, 1, 0) == ak.AK_PATH_CTA
+    assert l.ak_layernorm_fwd_dt(P, P, P + 2, P, 1, 8, 1e-5, 2, None, 0) == 3
+    assert l.ak_layernorm_fwd_dt(P, P, P, P, 1, 8, 1e-5, 5, None, 0) == 4
+    assert l.ak_rowsum_fwd_dt(P + 2, P, 1, 8, 2, None) == 3 and l.ak_rowsum_fwd_dt(P, P, 1, 8, 4, None) == 4
     # vocabulary-parallel cross-entropy
     assert l.ak_xent_vp_partial_bytes(10, 3) == 10 * 4 * 8 and l.ak_xent_vp_partial_bytes(0, 3) == 0
     assert l.ak_xent_vp_nsplit(4096, 16032) == 1 and l.ak_xent_vp_nsplit(16, 16032) == 1

@@ -214,3 +214,100 @@ def test_bf16_through_the_dt_entry_points_is_bit_identical():
     a, am = ak.ak_xent_fwd(lg, tg)
     b, bm = ak.ak_xent_fwd_dt(lg, tg)
     assert torch.equal(a.view(torch.int32), b.view(torch.int32)) and torch.equal(am.view(torch.int32), bm.view(torch.int32))
+
+
+# ------------------------------------------------------------------ LayerNorm and row-sum in fp16 / fp32
+def _assert_ln_close_dt(y, ref, b, what):
+    """Main bar of the element type, plus one rounding relative to |z * gamma| + |beta| (the
+    output may cancel) and the fp32 error of the mean."""
+    assert_close_dt(y, ref, what, tight=False)
+    got = y.detach().cpu().double().numpy().reshape(ref.shape)
+    beta = np.broadcast_to(b.double().numpy()[None, :], ref.shape)
+    rnd = {torch.float16: 2.0 ** -11 * 1.02, torch.float32: 2.0 ** -23}[y.dtype]
+    bound = rnd * np.abs(ref) + 4e-6 * (np.abs(ref - beta) + np.abs(beta)) + 2e-6
+    fin = np.isfinite(ref)
+    worst = float(np.max(np.abs(got - ref)[fin] / bound[fin])) if fin.any() else 0.0
+    assert worst <= 1.0, f"{what}: exceeds one-rounding bound by {worst:.3f}x"
+
+
+@pytest.mark.parametrize("dtype", DTS)
+@pytest.mark.parametrize("rows,D", SHAPES + [(5, 4), (7, 12), (9, 1028), (3, 57344)])
+def test_layernorm_dt_parity_all_paths(rows, D, dtype):
+    x, g, b = synth.layernorm_inputs(rows, D, synth.case_seed(19, rows * 131 + D), dtype=dtype)
+    ref = oracle.layernorm_dt(synth.to_elems(x), synth.to_elems(g), synth.to_elems(b), 1e-5, NAME[dtype])
+    xd, gd, bd = x.to(DEV), g.to(DEV), b.to(DEV)
+    outs = {}
+    for path in [ak.AK_PATH_AUTO] + _legal_paths(D, dtype):
+        y, check = guarded((rows, D), dtype, DEV)
+        ak.ak_layernorm_fwd_dt(xd, gd, bd, y, eps=1e-5, path=path)
+        torch.cuda.synchronize()
+        check()
+        _assert_ln_close_dt(y, ref, b, f"layernorm {NAME[dtype]} {rows}x{D} path {path}")
+        outs[path] = y.clone()
+    auto = ak.ak_choose_path_dt("layernorm", rows, D, dtype)
+    assert torch.equal(outs[ak.AK_PATH_AUTO].view(torch.uint8), outs[auto].view(torch.uint8))
+
+
+@pytest.mark.parametrize("dtype", DTS)
+@pytest.mark.parametrize("rows,D", SHAPES + [(1000, 128), (300, 1025), (5, 4), (7, 13)])
+def test_rowsum_dt_parity_and_exact_integers(rows, D, dtype):
+    x, _, _ = synth.layernorm_inputs(rows, D, synth.case_seed(20, rows * 131 + D), dtype=dtype)
+    out, check = guarded((rows,), torch.float32, DEV)
+    ak.ak_rowsum_fwd_dt(x.to(DEV), out)
+    torch.cuda.synchronize()
+    check()
+    ref = oracle.rowsum_dt(synth.to_elems(x), NAME[dtype])
+    mag = x.double().abs().sum(dim=-1).numpy()
+    err = np.abs(out.cpu().double().numpy() - ref)
+    assert float(np.max(err / (1e-6 * mag + 2.0 ** -24 * np.abs(ref) + 1e-45))) <= 1.0
+    # integer entries: every fp32 partial sum is exact whatever the tree, at every base offset
+    gen = torch.Generator().manual_seed(D)
+    xi = torch.randint(-8, 9, (min(rows, 13), D), generator=gen).to(dtype)
+    refi = oracle.rowsum_dt(synth.to_elems(xi), NAME[dtype])
+    per16 = 16 // xi.element_size()
+    for off in range(per16):
+        buf = torch.full((xi.numel() + 16,), 3.0, dtype=dtype, device=DEV)
+        xv = buf[off:off + xi.numel()].view(xi.shape)
+        xv.copy_(xi)
+        assert np.array_equal(ak.ak_rowsum_fwd_dt(xv).cpu().double().numpy(), refi), f"offset {off}"
+
+
+@pytest.mark.parametrize("dtype", DTS)
+def test_layernorm_dt_adversarial_misaligned_in_place(dtype):
+    for kind in synth.ADVERSARIAL_KINDS:
+        for D in (512, 4099):
+            xb, _ = synth.adversarial_rows(kind, 20, D, synth.case_seed(21, D))
+            x = xb.to(dtype)
+            _, g, b = synth.layernorm_inputs(1, D, 156, dtype=dtype)
+            ref = oracle.layernorm_dt(synth.to_elems(x), synth.to_elems(g), synth.to_elems(b), 1e-5, NAME[dtype])
+            for path in [ak.AK_PATH_AUTO] + _legal_paths(D, dtype):
+                y = ak.ak_layernorm_fwd_dt(x.to(DEV), g.to(DEV), b.to(DEV), eps=1e-5, path=path)
+                assert torch.isfinite(y.float()).all()
+                _assert_ln_close_dt(y, ref, b, f"layernorm {NAME[dtype]} adversarial {kind} D={D} path {path}")
+                if kind in ("big_equal", "all_equal"):
+                    assert torch.equal(y.cpu(), b[None, :].expand(20, D))     # constant rows give beta exactly
+    rows, D = 9, 1537
+    x, g, b = synth.layernorm_inputs(rows, D, 391, dtype=dtype)
+    ref = oracle.layernorm_dt(synth.to_elems(x), synth.to_elems(g), synth.to_elems(b), 1e-5, NAME[dtype])
+    per16 = 16 // x.element_size()
+    for xo, yo, go, bo in ((1, 1, 0, 0), (1, 3, 0, 0), (0, 0, 1, 0), (2, 2, 2, 2), (per16 - 1, per16 - 1, 2, 0), (0, 0, 0, 0)):
+        xbuf = torch.zeros(rows * D + 8, dtype=dtype, device=DEV)
+        ybuf = torch.zeros(rows * D + 8, dtype=dtype, device=DEV)
+        gbuf = torch.zeros(D + 8, dtype=dtype, device=DEV)
+        bbuf = torch.zeros(D + 8, dtype=dtype, device=DEV)
+        xv, yv = xbuf[xo:xo + rows * D].view(rows, D), ybuf[yo:yo + rows * D].view(rows, D)
+        gv, bv = gbuf[go:go + D], bbuf[bo:bo + D]
+        xv.copy_(x); gv.copy_(g); bv.copy_(b)
+        ak.ak_layernorm_fwd_dt(xv, gv, bv, yv, eps=1e-5)
+        torch.cuda.synchronize()
+        _assert_ln_close_dt(yv, ref, b, f"layernorm {NAME[dtype]} offsets {xo},{yo},{go},{bo}")
+        assert bool((ybuf[:yo] == 0).all()) and bool((ybuf[yo + rows * D:] == 0).all())
+    xd = x.to(DEV)
+    ak.ak_layernorm_fwd_dt(xd, g.to(DEV), b.to(DEV), xd, eps=1e-5)
+    _assert_ln_close_dt(xd, ref, b, f"layernorm {NAME[dtype]} in place")
+
+
+def test_layernorm_rowsum_bf16_through_the_dt_entry_points_is_bit_identical():
+    x, g, b = synth.layernorm_inputs(300, 4096, 392, device=DEV)
+    assert torch.equal(ak.ak_layernorm_fwd(x, g, b).view(torch.int16), ak.ak_layernorm_fwd_dt(x, g, b).view(torch.int16))
+    assert torch.equal(ak.ak_rowsum_fwd(x).view(torch.int32), ak.ak_rowsum_fwd_dt(x).view(torch.int32))
