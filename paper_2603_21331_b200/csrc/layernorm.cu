@@ -130,7 +130,7 @@ int dispatch_t(const void* x, const void* gamma, const void* beta, void* y, int6
                 return launch_reg_vpt<DT, 128, 128, 10, 8, 6, 8>((nvec + 127) / 128, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
             if (nvec <= 2048)
                 return launch_reg_vpt<DT, 256, 256, 5, 4, 4, 4>((nvec + 255) / 256, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
-            return launch_reg_vpt<DT, 512, 512, 1, 2, 2, 2>((nvec + 511) / 512, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
+            return launch_reg_vpt<DT, 512, 512, 2, 2, 2, 2>((nvec + 511) / 512, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
         case AK_PATH_SMEM:
             if (row_bytes > kMaxRowSmemBytes) return AK_ERR_SHAPE;
             if (nvec <= 4096) return launch_smem<DT, 256>(x, gamma, beta, y, rows, nvec, inv_D, eps, st);
@@ -180,7 +180,7 @@ int layernorm_choose(int64_t rows, int64_t D, bool aligned16, int dtype) {
     const int64_t bytes = D * dtype_bytes(dtype);
     if (!aligned16 || (bytes & 15) != 0 || bytes > kMaxRowSmemBytes) return AK_PATH_GENERIC;
     if (bytes <= 4096) return AK_PATH_WARP;
-    if (bytes <= 32768) return AK_PATH_CTA;
+    if (bytes <= 65536) return AK_PATH_CTA;   // up to 64 KiB the register layout beats the staged one
     return AK_PATH_SMEM;
 }
 

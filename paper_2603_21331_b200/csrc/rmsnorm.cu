@@ -97,7 +97,7 @@ int rmsnorm_choose(int64_t rows, int64_t D, bool aligned16, int dtype) {
     const int64_t bytes = D * dtype_bytes(dtype);   // row bytes decide the layout
     if (!aligned16 || (bytes & 15) != 0 || bytes > kMaxRowSmemBytes) return AK_PATH_GENERIC;
     if (bytes <= 4096) return AK_PATH_WARP;
-    if (bytes <= 32768) return AK_PATH_CTA;
+    if (bytes <= 65536) return AK_PATH_CTA;   // up to 64 KiB the register layout beats the staged one
     return AK_PATH_SMEM;
 }
 
@@ -125,10 +125,12 @@ int dispatch_t(const void* x, const void* w, void* y, int64_t rows, int64_t D, f
             if (row_bytes > 65536) return AK_ERR_SHAPE;
             // Shapes chosen in the sustained (power-capped) regime of a long run: 128 threads x <= 4
             // vectors (46 registers); 256 threads x <= 4 vectors (46 registers, five CTAs per SM);
-            // 256 threads x <= 8 vectors capped at 85 registers (62 used).
+            // 256 threads x <= 8 vectors capped at 85 registers (62 used); 512 threads x <= 8 vectors
+            // capped at 64 registers so that two CTAs share an SM (6.5 TB/s at 64 KiB rows against 6.2
+            // for the shared-memory kernel).
             if (nvec <= 512) return launch_reg_vpt<DT, 128, 128, 1, 1>((nvec + 127) / 128, x, w, y, rows, nvec, inv_D, eps, st);
             if (nvec <= 2048) return launch_reg_vpt<DT, 256, 256, 1, 3>((nvec + 255) / 256, x, w, y, rows, nvec, inv_D, eps, st);
-            return launch_reg_vpt<DT, 512, 512, 1, 1>((nvec + 511) / 512, x, w, y, rows, nvec, inv_D, eps, st);
+            return launch_reg_vpt<DT, 512, 512, 2, 2>((nvec + 511) / 512, x, w, y, rows, nvec, inv_D, eps, st);
         case AK_PATH_SMEM:
             if (row_bytes > kMaxRowSmemBytes) return AK_ERR_SHAPE;
             if (nvec <= 4096) return launch_smem<DT, 256>(x, w, y, rows, nvec, inv_D, eps, st);

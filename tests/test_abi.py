@@ -123,7 +123,10 @@ def test_dispatch_is_a_pure_function_of_shape_and_alignment():
     assert ak.ak_rmsnorm_choose_path(8192, 1024, True) == ak.AK_PATH_WARP
     assert ak.ak_rmsnorm_choose_path(8192, 4096, True) == ak.AK_PATH_CTA
     assert ak.ak_rmsnorm_choose_path(8192, 16384, True) == ak.AK_PATH_CTA
-    assert ak.ak_rmsnorm_choose_path(8192, 32768, True) == ak.AK_PATH_SMEM
+    assert ak.ak_rmsnorm_choose_path(8192, 32768, True) == ak.AK_PATH_CTA
+    assert ak.ak_rmsnorm_choose_path(8192, 32776, True) == ak.AK_PATH_SMEM
+    assert ak.ak_layernorm_choose_path(8192, 32768, True) == ak.AK_PATH_CTA
+    assert ak.ak_layernorm_choose_path(8192, 40960, True) == ak.AK_PATH_SMEM
     assert ak.ak_rmsnorm_choose_path(8192, 4099, True) == ak.AK_PATH_GENERIC
     assert ak.ak_rmsnorm_choose_path(8192, 4096, False) == ak.AK_PATH_GENERIC
     assert ak.ak_rmsnorm_choose_path(8192, 65536, True) == ak.AK_PATH_SMEM
