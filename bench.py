@@ -16,7 +16,7 @@ weak scaling, no data-path collective) and the cross-entropy mean is made global
 
 ``--impl reference`` times the fp64 CPU checker on the host cores on a bounded sample of
 the same workload.  ``--sweep`` additionally times every benchmark shape one by one and
-writes a table to gpurun_out/sweep.json (not part of the JSON line contract).
+writes a table (sweep.json, in the scratch output folder; not part of the JSON line contract).
 """
 from __future__ import annotations
 
