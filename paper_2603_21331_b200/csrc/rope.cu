@@ -159,7 +159,7 @@ int rope_t(const void* x, void* y, int64_t n_seq, int64_t S, int64_t Dh, int64_t
         if (gx > 2147483647LL) return AK_ERR_SHAPE;
         chunking(gx, n_seq, &seq_per_cta, &gy);
         if ((n_seq + seq_per_cta - 1) / seq_per_cta > 65535) return AK_ERR_SHAPE;
-        rope_vec_kernel<DT, 4><<<dim3((unsigned)gx, gy), kRopeThreads, 0, st>>>(
+        rope_vec_kernel<DT, 8><<<dim3((unsigned)gx, gy), kRopeThreads, 0, st>>>(
             static_cast<const uint4*>(x), static_cast<uint4*>(y), n_seq, nvs, vpr, pos_offset, seq_per_cta, freq);
     } else {
         const int half = (int)(Dh / 2);
