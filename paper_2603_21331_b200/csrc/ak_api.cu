@@ -12,14 +12,6 @@ namespace ak {
 static std::atomic<int64_t> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
-bool persistent_grid() {
-    static const bool on = [] {
-        const char* v = std::getenv("AK_TUNE_PERSISTENT");
-        return v != nullptr && std::atoi(v) != 0;
-    }();
-    return on;
-}
-
 int sm_count() {
     static std::mutex mu;
     static int cached[64] = {0};

@@ -247,9 +247,6 @@ constexpr int kMaxRowSmemBytes = 224 * 1024;
 // Launch bookkeeping shared by the translation units (defined in ak_api.cu).
 void count_launch(int n = 1);
 int sm_count();  // SMs of the current device (cached per device)
-// Tuning knob (environment AK_TUNE_PERSISTENT, read once; default 0): 1 = register-path CTAs
-// walk rows with a grid stride on a resident-size grid, 0 = one row (warp path: 4 rows) per CTA.
-bool persistent_grid();
 
 // Per-op host dispatchers (each defined next to its kernels).  All arguments have been
 // validated; `path` is a concrete path id or AUTO.  They return an ak_status.
@@ -282,8 +279,6 @@ int rowsum_dispatch(const void* x, float* out, int64_t rows, int64_t D, cudaStre
 int rmsnorm_choose(int64_t rows, int64_t D, bool aligned16, int dtype = AK_DTYPE_BF16);
 int softmax_choose(int64_t rows, int64_t D, bool aligned16, int dtype = AK_DTYPE_BF16);
 int xent_choose(int64_t rows, int64_t V, int* nsplit);
-// CTA shape of the register-resident row paths: threads per CTA and 16-byte vectors per thread.
-void cta_shape(int nvec, int* threads, int* vpt);
 
 inline int dtype_bytes(int dtype) { return dtype == AK_DTYPE_F32 ? 4 : 2; }
 inline bool is_aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }

@@ -15,19 +15,7 @@ template <int DT, int THREADS, int GROUP, int VPT, int MINB>
 int launch_reg(const void* x, const void* w, void* y, int64_t rows, int nvec, float inv_D, float eps,
                cudaStream_t st) {
     constexpr int GROUPS = THREADS / GROUP;
-    const int64_t need = (rows + GROUPS - 1) / GROUPS;
-    int64_t grid = need;
-    if (persistent_grid()) {
-        static const int resident = [] {
-            int per_sm = 0;
-            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-                    &per_sm, rmsnorm_reg_kernel<THREADS, GROUP, VPT, MINB, false, DT>, THREADS, 0) != cudaSuccess ||
-                per_sm < 1)
-                per_sm = 1;
-            return per_sm * sm_count();
-        }();
-        if (grid > resident) grid = resident;
-    }
+    const int64_t grid = (rows + GROUPS - 1) / GROUPS;
     rmsnorm_reg_kernel<THREADS, GROUP, VPT, MINB, false, DT><<<(unsigned)grid, THREADS, 0, st>>>(
         static_cast<const uint4*>(x), static_cast<const uint4*>(w), static_cast<uint4*>(y), rows, nvec, inv_D, eps);
     count_launch();
