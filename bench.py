@@ -505,7 +505,7 @@ SWEEP = list(
     + [("layernorm", 8192, 4096), ("layernorm", 4096, 5120), ("layernorm", 8192, 8192), ("layernorm", 65536, 4096),
        ("layernorm", 4096, 32768), ("layernorm", 8192, 4099)]
     + [("rowsum", 8192, 4096), ("rowsum", 16384, 4096), ("rowsum", 8192, 8192), ("rowsum", 65536, 1024), ("rowsum", 65536, 8192),
-       ("rowsum", 4096, 128256), ("rowsum", 8192, 4099)]
+       ("rowsum", 4096, 128256), ("rowsum", 8192, 4099), ("rowsum", 16, 128256), ("rowsum", 1, 1 << 24)]
     # element-type variants ("op.f16" / "op.f32"): the paper's Table 4 shapes were measured in FP16
     + [("rmsnorm.f16", 8192, 4096), ("rmsnorm.f16", 8192, 8192), ("rmsnorm.f32", 8192, 8192),
        ("softmax.f16", 16384, 4096), ("softmax.f16", 16384, 8192), ("softmax.f32", 16384, 8192),

@@ -181,7 +181,10 @@ int ak_layernorm_fwd_path(const void* x, const void* gamma, const void* beta, vo
  * Row-sum reduce (Table 3 "reduce").
  *   out[r] = fp32( sum_k x[r, k] ),  fp32 accumulation in a fixed order
  * x: device bf16 [rows, D], 2-byte aligned, any D >= 1; out: device fp32 [rows], caller
- * owned.  One launch, no scratch.  inf/NaN propagate per IEEE-754.
+ * owned.  One launch and no scratch, except for a few long rows (rows < 592 and D >= 16384; a
+ * vector sum is rows == 1): then nsplit CTAs per row write partial sums and a second launch
+ * adds them in a fixed order, with rows * nsplit * 4 bytes of stream-ordered scratch obtained
+ * and released on `cuda_stream` (AK_ERR_NOMEM if that fails).  inf/NaN propagate per IEEE-754.
  */
 int ak_rowsum_fwd(const void* x, float* out, int64_t rows, int64_t D, void* cuda_stream);
 

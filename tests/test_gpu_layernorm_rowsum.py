@@ -215,3 +215,28 @@ def test_rowsum_ieee_conventions():
     x[3, 2] = float("-inf")
     out = ak.ak_rowsum_fwd(x.to(DEV)).cpu().numpy()
     assert out[0] == np.inf and out[1] == -np.inf and np.isnan(out[2]) and np.isnan(out[3])
+
+
+@pytest.mark.parametrize("rows,D", [(1, 1 << 24), (1, (1 << 22) + 3), (4, 262144 + 5), (100, 65536), (591, 16384),
+                                    (592, 16384), (1, 16383), (1, 16384)])
+def test_rowsum_few_long_rows_and_vector_sum(rows, D):
+    # a handful of long rows (a vector sum is rows == 1) take the split layout: partial sums by
+    # many CTAs, then a fixed-order second launch
+    x, _, _ = synth.layernorm_inputs(rows, D, synth.case_seed(22, rows + D), device=DEV)
+    out, check = guarded((rows,), torch.float32, DEV)
+    ak.ak_rowsum_fwd(x, out)
+    again = ak.ak_rowsum_fwd(x)
+    torch.cuda.synchronize()
+    check()
+    assert torch.equal(out.view(torch.int32), again.view(torch.int32))
+    xb = synth.to_bits(x)
+    _assert_rowsum_close(out, xb, f"rowsum split {rows}x{D}")
+    # small integers: exact whatever the tree and the slicing, also from an odd base offset
+    gen = torch.Generator().manual_seed(D)
+    xi = torch.randint(-4, 5, (rows, D), generator=gen).to(torch.bfloat16)
+    ref = oracle.rowsum(synth.to_bits(xi))
+    for off in (0, 3):
+        buf = torch.full((rows * D + 16,), 3.0, dtype=torch.bfloat16, device=DEV)
+        xv = buf[off:off + rows * D].view(rows, D)
+        xv.copy_(xi)
+        assert np.array_equal(ak.ak_rowsum_fwd(xv).cpu().double().numpy(), ref), f"offset {off}"
