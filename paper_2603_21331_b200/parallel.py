@@ -34,16 +34,6 @@ def gather_pairs(local_pair: torch.Tensor, group=None) -> torch.Tensor:
     return out
 
 
-def merge_pairs_host(pairs: torch.Tensor) -> float:
-    """Rank-order merge of gathered pairs on the host (CPU tensors): the same arithmetic,
-    in the same order, as the library's merge kernel.  Used where no GPU is involved."""
-    total, count = 0.0, 0.0
-    for s, c in pairs.double().cpu().tolist():
-        total += s
-        count += c
-    return total / count if count > 0 else float("nan")
-
-
 def shard_vocab(V: int, rank: int, world: int) -> Tuple[int, int]:
     """Contiguous block [begin, end) of the vocabulary owned by ``rank``.  Block starts are
     multiples of 8 columns (16-byte aligned shards for the 16-bit types); the last rank takes

