@@ -477,10 +477,8 @@ def run_ours(args, rank, world, local_rank):
     if rank == 0 and world == 1:
         out["widened_rows"] = [
             {"op": r["op"], "rows": r["rows"], "D": r["D"], "us": round(r["us_trimmed_mean"], 2),
-             "GB/s": round(r["GB/s"], 1), "frac_of_measured_peak": round(r["GB/s"] / peak, 4),
-             "max_err_over_tolerance": r.get("max_err_over_tolerance"),
-             "max_err_over_sum_abs_x": r.get("max_err_over_sum_abs_x"), "bitwise_repeat": r["bitwise_repeat"]}
-            for r in run_sweep(ak, synth, dev, peak, shapes=WIDENED, iters=60, write=False)]
+             "GB/s": round(r["GB/s"], 1), "frac_of_measured_peak": round(r["GB/s"] / peak, 4)}
+            for r in run_sweep(ak, synth, dev, peak, shapes=WIDENED, iters=60, write=False, accuracy=False)]
         out["cpu_baseline"] = cpu_baseline_leg()
     elif rank == 0:
         out["cpu_baseline"] = None
@@ -715,7 +713,7 @@ WIDENED = [("layernorm", 8192, 4096), ("rowsum", 16384, 4096), ("rope.f16", 64 *
            ("rmsnorm.f16", 8192, 8192), ("xent_vp8", 4096, 128256 // 8)]
 
 
-def run_sweep(ak, synth, dev, peak, shapes=None, iters=200, write=True):
+def run_sweep(ak, synth, dev, peak, shapes=None, iters=200, write=True, accuracy=True):
     rows_out = []
     only = os.environ.get("AK_SWEEP_OPS") if shapes is None else None
     for op, rows, D in (SWEEP if shapes is None else shapes):
@@ -800,7 +798,8 @@ def run_sweep(ak, synth, dev, peak, shapes=None, iters=200, write=True):
             nb = algorithmic_bytes(op, rows, D, int((sets[0][1] != -100).sum()))
         us, us_min, us_med = time_op(fn, nsets, iters=iters)
         gbs = nb / (us * 1e-6) / 1e9
-        acc = sweep_accuracy(ak, synth, op, rows, D, sets[0])
+        # errors against the CPU checker and its timing belong to the per-shape CPU-baseline report
+        acc = sweep_accuracy(ak, synth, op, rows, D, sets[0]) if accuracy else {}
         rows_out.append({"op": op, "rows": rows, "D": D, "us_trimmed_mean": us, "us_min": us_min,
                          "us_median": us_med, "GB/s": gbs, "frac_of_8TBs": gbs / NOMINAL_HBM_GBS,
                          "frac_of_measured_copy": gbs / peak, "rows_per_s": rows / (us * 1e-6),
