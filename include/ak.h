@@ -24,6 +24,10 @@
  *   - The return value is an ak_status.  Arguments are validated on the host before any
  *     launch.  Data-dependent problems (an out-of-range target) cannot be reported
  *     synchronously and are encoded in the output (NaN); no kernel ever traps.
+ *   - Stream-ordered scratch, where an entry point says it uses some, comes from a CUDA
+ *     memory pool of the library's own (one per device, created at first use, keeps up to
+ *     256 MiB cached between calls) through cudaMallocFromPoolAsync / cudaFreeAsync on the
+ *     call's stream; such calls may be captured in CUDA graphs.
  *   - rows == 0 is legal: nothing is launched (cross-entropy still writes loss_mean = NaN).
  *   - Determinism: same inputs, shape, pointer alignment, library build and GPU model
  *     give bit-identical outputs.  Path selection is a pure function of
@@ -170,7 +174,12 @@ int ak_choose_path_dt(int op, int64_t rows, int64_t D, int aligned16, int dtype)
  * fp32, taken in two fixed-order passes over the on-chip copy of the row (the mean as
  * x[r,0] + mean(x - x[r,0]), so a constant row gives exactly beta).  eps finite, >= 0.
  * Same path ids, size limits and alignment rules as RMSNorm (gamma and beta together play
- * the part of w).  Status codes as for RMSNorm.
+ * the part of w).  Status codes as for RMSNorm.  One launch and no scratch, except for 1024 or
+ * more rows that are not 16-byte aligned and short enough for registers (D <= about 32750):
+ * then a small kernel first writes gamma and beta in all eight 2-byte shifts to
+ * about 32 * D bytes of stream-ordered scratch obtained and released on `cuda_stream`, and
+ * the row kernel runs as its programmatic dependent; if the scratch cannot be had the
+ * single-launch kernel runs instead (same results).
  */
 int ak_layernorm_fwd(const void* x, const void* gamma, const void* beta, void* y,
                      int64_t rows, int64_t D, float eps, void* cuda_stream);
@@ -208,9 +217,9 @@ int ak_softmax_fwd_path(const void* x, void* y, int64_t rows, int64_t D,
  * logits: device bf16 [rows, V]; targets: device int64 [rows]; loss_rows: device fp32
  * [rows] (required); loss_mean: device fp32 [1] or NULL (mean skipped).
  * Rows with very long vocabularies or too few rows to fill the GPU take the split-row
- * two-phase path, which needs rows * nsplit * 8 bytes of scratch: ak_xent_fwd obtains it
- * with cudaMallocAsync / cudaFreeAsync on `cuda_stream` (stream-ordered; AK_ERR_NOMEM on
- * failure); ak_xent_fwd_ws takes it from the caller instead.
+ * two-phase path, which needs rows * nsplit * 8 bytes of scratch: ak_xent_fwd obtains and
+ * releases it stream-ordered on `cuda_stream` (AK_ERR_NOMEM on failure); ak_xent_fwd_ws takes
+ * it from the caller instead.
  */
 int ak_xent_fwd(const void* logits, const int64_t* targets, int64_t ignore_index,
                 float* loss_rows, float* loss_mean,

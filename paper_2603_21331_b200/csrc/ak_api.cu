@@ -12,6 +12,40 @@ namespace ak {
 static std::atomic<int64_t> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+// Stream-ordered scratch comes from a memory pool of the library's own, one per device, that
+// keeps up to 256 MiB cached between calls.  (The device's default pool releases everything at
+// the next synchronisation unless the application raised its threshold; each call after a
+// synchronise would then pay for a fresh physical allocation, hundreds of microseconds.)
+cudaError_t scratch_alloc(void** p, size_t bytes, cudaStream_t st) {
+    static std::mutex mu;
+    static cudaMemPool_t pools[64] = {};
+    static bool tried[64] = {};
+    int dev = 0;
+    cudaMemPool_t pool = nullptr;
+    if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64) {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!tried[dev]) {
+            tried[dev] = true;
+            cudaMemPoolProps props = {};
+            props.allocType = cudaMemAllocationTypePinned;
+            props.handleTypes = cudaMemHandleTypeNone;
+            props.location.type = cudaMemLocationTypeDevice;
+            props.location.id = dev;
+            cudaMemPool_t created = nullptr;
+            if (cudaMemPoolCreate(&created, &props) == cudaSuccess) {
+                uint64_t keep = 256ull << 20;
+                cudaMemPoolSetAttribute(created, cudaMemPoolAttrReleaseThreshold, &keep);
+                pools[dev] = created;
+            } else {
+                (void)cudaGetLastError();
+            }
+        }
+        pool = pools[dev];
+    }
+    if (pool != nullptr) return cudaMallocFromPoolAsync(p, bytes, pool, st);
+    return cudaMallocAsync(p, bytes, st);
+}
+
 int sm_count() {
     static std::mutex mu;
     static int cached[64] = {0};

@@ -246,6 +246,8 @@ constexpr int kMaxRowSmemBytes = 224 * 1024;
 // ---------------------------------------------------------------- host-side plumbing
 // Launch bookkeeping shared by the translation units (defined in ak_api.cu).
 void count_launch(int n = 1);
+// cudaMallocAsync from the library's own pool (free with cudaFreeAsync on the same stream)
+cudaError_t scratch_alloc(void** p, size_t bytes, cudaStream_t st);
 int sm_count();  // SMs of the current device (cached per device)
 
 // Per-op host dispatchers (each defined next to its kernels).  All arguments have been
@@ -282,5 +284,60 @@ int xent_choose(int64_t rows, int64_t V, int* nsplit);
 
 inline int dtype_bytes(int dtype) { return dtype == AK_DTYPE_F32 ? 4 : 2; }
 inline bool is_aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+// Programmatic dependent launch: let the next kernel in the stream be scheduled while this
+// grid is still running (it waits for our completion with pdl_wait before it reads).
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// ------------------------------------------------------------------ pre-shifted parameter vectors
+// Rows of 2-byte elements that do not start on a 16-byte boundary are processed in their own
+// phase (phase p = the row start's element offset inside its 16-byte group): vector k of such a
+// row holds elements 8k - p .. 8k - p + 7.  Per-column parameters (the RMSNorm weight, the
+// LayerNorm gamma and beta) are needed in the same shifted layout.  Rather than assembling them
+// from 4-byte loads and funnel shifts for every output vector of every row, this kernel writes
+// all eight shifts once per launch:
+//     tab[(o * 8 + p) * nvp + k] = elements 8k - p .. 8k - p + 7 of parameter vector o
+// (zero outside [0, D)), nvp = (D + 14) / 8 vectors; the row kernels, launched as programmatic
+// dependents, read them with one 16-byte load each after pdl_wait.  p1 may be null (one vector).
+constexpr int kShiftThreads = 128;
+template <int UNUSED = 0>
+__global__ void __launch_bounds__(kShiftThreads)
+shift_params_kernel(const uint16_t* __restrict__ p0, const uint16_t* __restrict__ p1, int64_t D, int nvp,
+                    uint4* __restrict__ tab) {
+    pdl_launch_dependents();
+    const int idx = blockIdx.x * kShiftThreads + threadIdx.x;
+    const int total = (p1 ? 16 : 8) * nvp;
+    if (idx >= total) return;
+    const int k = idx % nvp;
+    const int p = (idx / nvp) & 7;
+    const uint16_t* src = (idx >= 8 * nvp) ? p1 : p0;
+    uint32_t w[4];
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+        const int64_t j = (int64_t)k * 8 - p + 2 * h;
+        const uint32_t lo = (j >= 0 && j < D) ? (uint32_t)__ldg(src + j) : 0u;
+        const uint32_t hi = (j + 1 >= 0 && j + 1 < D) ? (uint32_t)__ldg(src + j + 1) : 0u;
+        w[h] = lo | (hi << 16);
+    }
+    tab[idx] = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// Launch `kernel` as a programmatic dependent of the work before it in the stream.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
 
 }  // namespace ak

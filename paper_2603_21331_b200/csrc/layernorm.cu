@@ -69,10 +69,35 @@ int launch_stage(const uint16_t* x, const uint16_t* g, const uint16_t* b, uint16
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
+constexpr int64_t kShiftMinRows = 1024;
+
 template <int DT, int THREADS, int VPT, int MINB>
 int launch_regp(const uint16_t* x, const uint16_t* g, const uint16_t* b, uint16_t* y, int64_t rows, int64_t D,
                 float inv_D, float eps, cudaStream_t st) {
-    layernorm_regp_kernel<THREADS, VPT, MINB, DT><<<(unsigned)rows, THREADS, 0, st>>>(x, g, b, y, D, inv_D, eps);
+    // From kShiftMinRows rows on, gamma and beta are shifted once per launch into a table (16 x
+    // the row's vectors, stream-ordered scratch) instead of once per output vector.
+    const int nvp = (int)((D + 14) >> 3);
+    void* tab = nullptr;
+    if (rows >= kShiftMinRows) {
+        if (scratch_alloc(&tab, (size_t)16 * nvp * sizeof(uint4), st) != cudaSuccess) {
+            (void)cudaGetLastError();
+            tab = nullptr;
+        }
+    }
+    if (tab != nullptr) {
+        shift_params_kernel<<<(16 * nvp + kShiftThreads - 1) / kShiftThreads, kShiftThreads, 0, st>>>(
+            g, b, D, nvp, static_cast<uint4*>(tab));
+        count_launch();
+        cudaError_t e = cudaGetLastError();
+        if (e == cudaSuccess)
+            e = launch_dependent(layernorm_regp_kernel<THREADS, VPT, MINB, DT, true>, dim3((unsigned)rows), dim3(THREADS),
+                                 0, st, x, g, b, y, D, inv_D, eps, static_cast<const uint4*>(tab), nvp);
+        count_launch();
+        cudaFreeAsync(tab, st);
+        return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+    }
+    layernorm_regp_kernel<THREADS, VPT, MINB, DT, false><<<(unsigned)rows, THREADS, 0, st>>>(x, g, b, y, D, inv_D, eps,
+                                                                                            nullptr, 0);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
@@ -152,10 +177,14 @@ int dispatch_t(const void* x, const void* gamma, const void* beta, void* y, int6
                 const uint16_t* gs = static_cast<const uint16_t*>(gamma);
                 const uint16_t* bs = static_cast<const uint16_t*>(beta);
                 uint16_t* ys = static_cast<uint16_t*>(y);
-                // rows of up to 1024 covering vectors stay in the registers of a 128-thread CTA
+                // rows of up to 1024 covering vectors stay in the registers of a 128-thread CTA ...
                 const int64_t max_nv = (D + 14) >> 3;   // vectors covering the row at the worst phase
                 if (same_phase && params4 && max_nv <= 1024)
                     return launch_regp_vpt<DT, 128, 10, 6>((int)((max_nv + 127) / 128), xs, gs, bs, ys, rows, D, inv_D, eps, st);
+                if (same_phase && params4 && max_nv <= 2048)   // ... or of a 256-thread CTA up to 2048
+                    return launch_regp_vpt<DT, 256, 5, 3>((int)((max_nv + 255) / 256), xs, gs, bs, ys, rows, D, inv_D, eps, st);
+                if (same_phase && params4 && max_nv <= 4096)   // ... 512 threads up to 4096
+                    return launch_regp_vpt<DT, 512, 2, 2>((int)((max_nv + 511) / 512), xs, gs, bs, ys, rows, D, inv_D, eps, st);
                 if (same_phase && params4 && stage_bytes <= (size_t)kMaxRowSmemBytes) {
                     if (D <= 8192) return launch_stage<DT, 128>(xs, gs, bs, ys, rows, D, stage_bytes, inv_D, eps, st);
                     if (D <= 32768) return launch_stage<DT, 256>(xs, gs, bs, ys, rows, D, stage_bytes, inv_D, eps, st);

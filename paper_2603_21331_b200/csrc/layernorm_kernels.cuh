@@ -281,11 +281,15 @@ layernorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restric
 // The phase layout of layernorm_stage_kernel without the trip through shared memory, for rows
 // short enough to sit in registers: interior vectors are loaded before the first use, the edge
 // elements are single values in sixteen threads.  Needs x and y rows in the same phase, gamma
-// and beta 4-byte aligned and at most THREADS * VPT covering vectors.
-template <int THREADS, int VPT, int MINB, int DT = AK_DTYPE_BF16>
+// and beta 4-byte aligned and at most THREADS * VPT covering vectors.  TAB: gamma and beta of the
+// interior vectors come pre-shifted from the table of shift_params_kernel (this kernel then runs
+// as its programmatic dependent: the statistics need no parameters, so only the output phase
+// waits for the table).
+template <int THREADS, int VPT, int MINB, int DT = AK_DTYPE_BF16, bool TAB = false>
 __global__ void __launch_bounds__(THREADS, MINB)
 layernorm_regp_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ gamma,
-                      const uint16_t* __restrict__ beta, uint16_t* __restrict__ y, int64_t D, float inv_D, float eps) {
+                      const uint16_t* __restrict__ beta, uint16_t* __restrict__ y, int64_t D, float inv_D, float eps,
+                      const uint4* tab, int nvp) {
     __shared__ float slots[2 * kWarp];
     const int64_t r = blockIdx.x;
     const uint16_t* xr = x + r * D;
@@ -323,12 +327,23 @@ layernorm_regp_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict
         if (k_lo + (int)threadIdx.x + i * THREADS < k_hi) s2 += sqdev_v<DT>(xv[i], mu);
     s2 = cta_sum<THREADS>(s2, slots, 1);
     const float rstd = rsqrtf(fmaf(s2, inv_D, eps));
+    if constexpr (TAB) {
+        pdl_wait();   // the table is complete and visible; plain loads (cached in L1), not the read-only path
+        const uint4* gt = tab + (size_t)phase * nvp;
+        const uint4* bt = tab + (size_t)(8 + phase) * nvp;
 #pragma unroll
-    for (int i = 0; i < VPT; ++i) {
-        const int k = k_lo + threadIdx.x + i * THREADS;
-        if (k < k_hi) {
-            const int64_t j0 = (int64_t)k * 8 - phase;
-            st_stream(ya + k, ln_out_v<DT>(xv[i], ln_load_shifted(gamma, j0), ln_load_shifted(beta, j0), mu, rstd));
+        for (int i = 0; i < VPT; ++i) {
+            const int k = k_lo + threadIdx.x + i * THREADS;
+            if (k < k_hi) st_stream(ya + k, ln_out_v<DT>(xv[i], gt[k], bt[k], mu, rstd));
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int k = k_lo + threadIdx.x + i * THREADS;
+            if (k < k_hi) {
+                const int64_t j0 = (int64_t)k * 8 - phase;
+                st_stream(ya + k, ln_out_v<DT>(xv[i], ln_load_shifted(gamma, j0), ln_load_shifted(beta, j0), mu, rstd));
+            }
         }
     }
     if (edge) yr[ej] = Elem<DT>::from_float(ln_out1<DT>(xe, __ldg(gamma + ej), __ldg(beta + ej), mu, rstd));

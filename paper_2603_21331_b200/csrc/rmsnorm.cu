@@ -145,10 +145,14 @@ int dispatch_t(const void* x, const void* w, void* y, int64_t rows, int64_t D, f
                 const uint16_t* xs = static_cast<const uint16_t*>(x);
                 const uint16_t* ws = static_cast<const uint16_t*>(w);
                 uint16_t* ys = static_cast<uint16_t*>(y);
-                // rows of up to 1024 covering vectors stay in the registers of a 128-thread CTA
+                // rows of up to 1024 covering vectors stay in the registers of a 128-thread CTA ...
                 const int64_t max_nv = (D + 14) >> 3;   // vectors covering the row at the worst phase
                 if (same_phase && is_aligned(w, 4) && max_nv <= 1024)
                     return launch_regp_vpt<DT, 128>((int)((max_nv + 127) / 128), xs, ws, ys, rows, D, inv_D, eps, st);
+                if (same_phase && is_aligned(w, 4) && max_nv <= 2048)   // ... or of a 256-thread CTA up to 2048
+                    return launch_regp_vpt<DT, 256>((int)((max_nv + 255) / 256), xs, ws, ys, rows, D, inv_D, eps, st);
+                if (same_phase && is_aligned(w, 4) && max_nv <= 4096)   // ... 512 threads up to 4096
+                    return launch_regp_vpt<DT, 512>((int)((max_nv + 511) / 512), xs, ws, ys, rows, D, inv_D, eps, st);
                 if (same_phase && is_aligned(w, 4) && stage_bytes <= (size_t)kMaxRowSmemBytes) {
                     static const bool configured = [] {
                         return cudaFuncSetAttribute(rmsnorm_stage_kernel<128, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,

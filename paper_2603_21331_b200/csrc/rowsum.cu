@@ -153,7 +153,7 @@ template <int DT>
 int launch_split(const void* x, float* out, int64_t rows, int64_t D, int nsplit, cudaStream_t st) {
     if (rows > 65535) return AK_ERR_SHAPE;   // grid.y; the split is only chosen for a few rows
     float* partial = nullptr;
-    if (cudaMallocAsync(reinterpret_cast<void**>(&partial), (size_t)rows * nsplit * sizeof(float), st) != cudaSuccess) {
+    if (scratch_alloc(reinterpret_cast<void**>(&partial), (size_t)rows * nsplit * sizeof(float), st) != cudaSuccess) {
         (void)cudaGetLastError();
         return AK_ERR_NOMEM;
     }

@@ -108,7 +108,7 @@ int dispatch_t(const void* logits, const int64_t* targets, int64_t ignore_index,
     if (partial == nullptr || workspace_bytes < need) {
         if (!may_allocate) return AK_ERR_NOMEM;
         void* p = nullptr;
-        if (cudaMallocAsync(&p, need, st) != cudaSuccess) {
+        if (scratch_alloc(&p, need, st) != cudaSuccess) {
             (void)cudaGetLastError();
             return AK_ERR_NOMEM;
         }

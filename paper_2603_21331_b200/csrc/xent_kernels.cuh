@@ -254,11 +254,6 @@ __device__ __forceinline__ float finish_loss(float M, float S, float xt) {
     return (M - xt) + lse;
 }
 
-// Programmatic dependent launch: let the next kernel in the stream be scheduled while this
-// grid is still running (it waits for our completion with pdl_wait before it reads).
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
 // ------------------------------------------------------------------ one CTA per row
 template <int UNROLL, int POLY, int MINB = 1, int T = kXentThreads, int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(T, MINB)

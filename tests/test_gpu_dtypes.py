@@ -307,6 +307,17 @@ def test_layernorm_dt_adversarial_misaligned_in_place(dtype):
     _assert_ln_close_dt(xd, ref, b, f"layernorm {NAME[dtype]} in place")
 
 
+def test_layernorm_fp16_unaligned_rows_with_the_shift_table():
+    rows, D = 1200, 2051
+    x, g, b = synth.layernorm_inputs(rows, D, 393, dtype=torch.float16)
+    ref = oracle.layernorm_dt(synth.to_elems(x), synth.to_elems(g), synth.to_elems(b), 1e-5, "f16")
+    n0 = ak.ak_launch_count()
+    y = ak.ak_layernorm_fwd_dt(x.to(DEV), g.to(DEV), b.to(DEV), eps=1e-5)
+    torch.cuda.synchronize()
+    assert ak.ak_launch_count() - n0 == 2
+    _assert_ln_close_dt(y, ref, b, "layernorm f16 1200x2051 (shift table)")
+
+
 def test_layernorm_rowsum_bf16_through_the_dt_entry_points_is_bit_identical():
     x, g, b = synth.layernorm_inputs(300, 4096, 392, device=DEV)
     assert torch.equal(ak.ak_layernorm_fwd(x, g, b).view(torch.int16), ak.ak_layernorm_fwd_dt(x, g, b).view(torch.int16))

@@ -117,6 +117,45 @@ def test_layernorm_misaligned_base_pointers():
             assert bool((ybuf[:yo] == 0).all()) and bool((ybuf[yo + rows * D:] == 0).all())
 
 
+@pytest.mark.parametrize("rows,D,xo", [(1024, 1027, 0), (1500, 4099, 0), (1100, 2051, 3), (1024, 8190, 1),
+                                       (1030, 16379, 0), (1025, 32754, 5)])
+def test_layernorm_unaligned_rows_with_the_shift_table(rows, D, xo):
+    """From 1024 rows on, unaligned rows that fit in registers read gamma and beta from a table of
+    all eight shifts written by a small kernel in front.  Parity on such launches, and the same
+    bits as the launch without the table (fewer rows) gives for the rows they share."""
+    x, g, b = synth.layernorm_inputs(rows, D, synth.case_seed(8, rows + D))
+    xb, gb, bb = synth.to_bits(x), synth.to_bits(g), synth.to_bits(b)
+    ref = oracle.layernorm(xb, gb, bb, EPS)
+    xbuf = torch.zeros(rows * D + 8, dtype=torch.bfloat16, device=DEV)
+    ybuf = torch.zeros(rows * D + 8, dtype=torch.bfloat16, device=DEV)
+    xv = xbuf[xo:xo + rows * D].view(rows, D)
+    yv = ybuf[xo:xo + rows * D].view(rows, D)
+    xv.copy_(x)
+    gd, bd = g.to(DEV), b.to(DEV)
+    n0 = ak.ak_launch_count()
+    ak.ak_layernorm_fwd(xv, gd, bd, yv, eps=EPS)
+    torch.cuda.synchronize()
+    assert ak.ak_launch_count() - n0 == 2          # the table kernel and the row kernel
+    _assert_ln_close(yv, ref, xb, gb, bb, f"layernorm {rows}x{D} offset {xo} (shift table)")
+    assert bool((ybuf[:xo] == 0).all()) and bool((ybuf[xo + rows * D:] == 0).all())
+    few = 1000
+    y2buf = torch.zeros(few * D + 8, dtype=torch.bfloat16, device=DEV)
+    y2 = y2buf[xo:xo + few * D].view(few, D)
+    n0 = ak.ak_launch_count()
+    ak.ak_layernorm_fwd(xv[:few], gd, bd, y2, eps=EPS)
+    torch.cuda.synchronize()
+    assert ak.ak_launch_count() - n0 == 1
+    assert torch.equal(y2.view(torch.int16), yv[:few].view(torch.int16))
+    # new parameters at the same addresses: the next launch must not see the old table
+    gd.mul_(-0.5)
+    bd.add_(1.0)
+    ref2 = oracle.layernorm(xb, synth.to_bits(gd.cpu()), synth.to_bits(bd.cpu()), EPS)
+    ak.ak_layernorm_fwd(xv, gd, bd, yv, eps=EPS)
+    torch.cuda.synchronize()
+    _assert_ln_close(yv, ref2, xb, synth.to_bits(gd.cpu()), synth.to_bits(bd.cpu()),
+                     f"layernorm {rows}x{D} offset {xo} (shift table, new parameters)")
+
+
 def test_layernorm_in_place_and_empty():
     for D, paths in ((512, _legal_paths(512)), (4096, _legal_paths(4096)), (4099, _legal_paths(4099)),
                      (16384, _legal_paths(16384))):

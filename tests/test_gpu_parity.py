@@ -32,7 +32,9 @@ SHAPES = [(256, 1024), (1, 8), (3, 16), (37, 64), (129, 256), (65, 512), (33, 77
           (33, 1280), (19, 1536), (21, 1792), (64, 2048), (17, 4096), (1, 4096), (23, 3072),
           (9, 5120), (16, 8192), (7, 11008), (12, 16384), (5, 20480), (3, 24576), (3, 28672),
           (6, 32768), (3, 65536), (2, 114688), (5, 1), (4, 7), (31, 1023), (11, 1537), (9, 4097), (13, 4099), (2, 40000),
-          (3, 128257)]
+          (3, 128257),
+          # unaligned rows in the registers of 256- and 512-thread CTAs, and just past them
+          (10, 8190), (6, 10247), (5, 12290), (4, 16379), (3, 24571), (3, 32754), (2, 32771)]
 
 
 @pytest.mark.parametrize("rows,D", SHAPES)
