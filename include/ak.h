@@ -174,9 +174,9 @@ int ak_choose_path_dt(int op, int64_t rows, int64_t D, int aligned16, int dtype)
  * fp32, taken in two fixed-order passes over the on-chip copy of the row (the mean as
  * x[r,0] + mean(x - x[r,0]), so a constant row gives exactly beta).  eps finite, >= 0.
  * Same path ids, size limits and alignment rules as RMSNorm (gamma and beta together play
- * the part of w).  Status codes as for RMSNorm.  One launch and no scratch, except for 1024 or
- * more rows that are not 16-byte aligned and short enough for registers (D <= about 32750):
- * then a small kernel first writes gamma and beta in all eight 2-byte shifts to
+ * the part of w).  Status codes as for RMSNorm.  One launch and no scratch, except for many
+ * rows that are not 16-byte aligned (1024 or more of D <= about 32750, 256 or more longer ones
+ * that fit in shared memory): then a small kernel first writes gamma and beta in all eight 2-byte shifts to
  * about 32 * D bytes of stream-ordered scratch obtained and released on `cuda_stream`, and
  * the row kernel runs as its programmatic dependent; if the scratch cannot be had the
  * single-launch kernel runs instead (same results).

@@ -239,6 +239,29 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     return false;
 }
 
+// Bring the fully-inside vectors k_lo .. k_hi - 1 of a phase-staged row (16-byte aligned in
+// global and in shared memory) into the staging buffer with bulk copies of at most kStageChunk
+// bytes, all counted in by one mbarrier.  Every thread of the CTA calls this (it contains a
+// barrier); the caller fills the edge vectors, calls __syncthreads and then mbar_wait(bar, 0).
+constexpr uint32_t kStageChunk = 32768;
+__device__ __forceinline__ void stage_interior_bulk(unsigned char* smem_raw, const uint4* xa, int k_lo, int k_hi,
+                                                    uint64_t* bar) {
+    if (threadIdx.x == 0) mbar_init(bar, 1);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (k_hi > k_lo) {
+            const uint32_t bytes = (uint32_t)(k_hi - k_lo) * 16u;
+            mbar_expect_tx(bar, bytes);
+            const unsigned char* src = reinterpret_cast<const unsigned char*>(xa + k_lo);
+            unsigned char* dst = smem_raw + (size_t)k_lo * 16;
+            for (uint32_t off = 0; off < bytes; off += kStageChunk)
+                bulk_load(dst + off, src + off, min(kStageChunk, bytes - off), bar);
+        } else {
+            mbar_arrive(bar);
+        }
+    }
+}
+
 // Largest row (bytes) the shared-memory-staged kernels accept: 224 KiB of dynamic shared
 // memory out of the 227 KiB a CTA may own (a few hundred bytes stay static).
 constexpr int kMaxRowSmemBytes = 224 * 1024;

@@ -56,44 +56,65 @@ int launch_smem(const void* x, const void* g, const void* b, void* y, int64_t ro
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
+// Rows that are not 16-byte aligned need gamma and beta shifted to the row's phase.  From
+// `min_rows` rows on they are shifted once per launch, for all eight phases, into a table in
+// stream-ordered scratch (16 x the row's vectors) instead of once per output vector; the row
+// kernel then runs as the programmatic dependent of the kernel that writes the table.  Returns
+// null (and launches nothing) for fewer rows or when the scratch cannot be had.
+const uint4* shift_table(const uint16_t* g, const uint16_t* b, int64_t rows, int64_t D, int64_t min_rows,
+                         cudaStream_t st, int* nvp_out) {
+    const int nvp = (int)((D + 14) >> 3);
+    *nvp_out = nvp;
+    if (rows < min_rows) return nullptr;
+    void* tab = nullptr;
+    if (scratch_alloc(&tab, (size_t)16 * nvp * sizeof(uint4), st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return nullptr;
+    }
+    shift_params_kernel<<<(16 * nvp + kShiftThreads - 1) / kShiftThreads, kShiftThreads, 0, st>>>(
+        g, b, D, nvp, static_cast<uint4*>(tab));
+    count_launch();
+    if (cudaGetLastError() != cudaSuccess) {
+        cudaFreeAsync(tab, st);
+        return nullptr;
+    }
+    return static_cast<const uint4*>(tab);
+}
+constexpr int64_t kShiftMinRowsRegs = 1024;    // rows of up to 64 KiB in registers
+constexpr int64_t kShiftMinRowsStaged = 256;   // longer rows staged in shared memory
+
 template <int DT, int T>
 int launch_stage(const uint16_t* x, const uint16_t* g, const uint16_t* b, uint16_t* y, int64_t rows, int64_t D,
                  size_t stage_bytes, float inv_D, float eps, cudaStream_t st) {
     static const bool configured = [] {
-        return cudaFuncSetAttribute(layernorm_stage_kernel<T, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        return cudaFuncSetAttribute(layernorm_stage_kernel<T, DT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    kMaxRowSmemBytes) == cudaSuccess &&
+               cudaFuncSetAttribute(layernorm_stage_kernel<T, DT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     kMaxRowSmemBytes) == cudaSuccess;
     }();
     if (!configured) return AK_ERR_CUDA;
-    layernorm_stage_kernel<T, DT><<<(unsigned)rows, T, stage_bytes, st>>>(x, g, b, y, D, inv_D, eps);
+    int nvp = 0;
+    if (const uint4* tab = shift_table(g, b, rows, D, kShiftMinRowsStaged, st, &nvp)) {
+        const cudaError_t e = launch_dependent(layernorm_stage_kernel<T, DT, true>, dim3((unsigned)rows), dim3(T),
+                                               stage_bytes, st, x, g, b, y, D, inv_D, eps, tab, nvp);
+        count_launch();
+        cudaFreeAsync(const_cast<uint4*>(tab), st);
+        return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+    }
+    layernorm_stage_kernel<T, DT, false><<<(unsigned)rows, T, stage_bytes, st>>>(x, g, b, y, D, inv_D, eps, nullptr, 0);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
-constexpr int64_t kShiftMinRows = 1024;
-
 template <int DT, int THREADS, int VPT, int MINB>
 int launch_regp(const uint16_t* x, const uint16_t* g, const uint16_t* b, uint16_t* y, int64_t rows, int64_t D,
                 float inv_D, float eps, cudaStream_t st) {
-    // From kShiftMinRows rows on, gamma and beta are shifted once per launch into a table (16 x
-    // the row's vectors, stream-ordered scratch) instead of once per output vector.
-    const int nvp = (int)((D + 14) >> 3);
-    void* tab = nullptr;
-    if (rows >= kShiftMinRows) {
-        if (scratch_alloc(&tab, (size_t)16 * nvp * sizeof(uint4), st) != cudaSuccess) {
-            (void)cudaGetLastError();
-            tab = nullptr;
-        }
-    }
-    if (tab != nullptr) {
-        shift_params_kernel<<<(16 * nvp + kShiftThreads - 1) / kShiftThreads, kShiftThreads, 0, st>>>(
-            g, b, D, nvp, static_cast<uint4*>(tab));
+    int nvp = 0;
+    if (const uint4* tab = shift_table(g, b, rows, D, kShiftMinRowsRegs, st, &nvp)) {
+        const cudaError_t e = launch_dependent(layernorm_regp_kernel<THREADS, VPT, MINB, DT, true>, dim3((unsigned)rows),
+                                               dim3(THREADS), 0, st, x, g, b, y, D, inv_D, eps, tab, nvp);
         count_launch();
-        cudaError_t e = cudaGetLastError();
-        if (e == cudaSuccess)
-            e = launch_dependent(layernorm_regp_kernel<THREADS, VPT, MINB, DT, true>, dim3((unsigned)rows), dim3(THREADS),
-                                 0, st, x, g, b, y, D, inv_D, eps, static_cast<const uint4*>(tab), nvp);
-        count_launch();
-        cudaFreeAsync(tab, st);
+        cudaFreeAsync(const_cast<uint4*>(tab), st);
         return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
     }
     layernorm_regp_kernel<THREADS, VPT, MINB, DT, false><<<(unsigned)rows, THREADS, 0, st>>>(x, g, b, y, D, inv_D, eps,

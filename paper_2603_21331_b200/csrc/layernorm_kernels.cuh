@@ -227,14 +227,17 @@ __device__ __forceinline__ uint4 ln_load_shifted(const uint16_t* __restrict__ p,
                       __funnelshift_r(d, e, 16));
 }
 
-template <int T, int DT = AK_DTYPE_BF16>
+// TAB: gamma and beta of the inside vectors come pre-shifted from the table of shift_params_kernel,
+// whose programmatic dependent this kernel then is (only the output phase waits for the table).
+template <int T, int DT = AK_DTYPE_BF16, bool TAB = false>
 __global__ void __launch_bounds__(T)
 layernorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ gamma,
                        const uint16_t* __restrict__ beta, uint16_t* __restrict__ y, int64_t D, float inv_D,
-                       float eps) {
+                       float eps, const uint4* tab, int nvp) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     uint4* row = reinterpret_cast<uint4*>(smem_raw);
     uint16_t* row16 = reinterpret_cast<uint16_t*>(smem_raw);
+    __shared__ uint64_t bar;
     __shared__ float slots[2 * kWarp];
     const int64_t r = blockIdx.x;
     const uint16_t* xr = x + r * D;
@@ -252,9 +255,10 @@ layernorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restric
     const int64_t ej = (int64_t)ek * 8 - phase + (threadIdx.x & 7);
     const bool edge = threadIdx.x < 16 && is_edge_vec && ej >= 0 && ej < D;
 
-    for (int k = k_lo + threadIdx.x; k < k_hi; k += T) row[k] = ld_stream(xa + k);
+    stage_interior_bulk(smem_raw, xa, k_lo, k_hi, &bar);   // the copy engine brings the inside vectors
     if (edge) row16[ek * 8 + (threadIdx.x & 7)] = ld_stream_u16(xr + ej);
     __syncthreads();
+    if (!mbar_wait(&bar, 0)) return;  // uniform: every thread waits on the same barrier
     const float K = Elem<DT>::to_float(row16[phase]);
     float s1 = 0.0f;
     for (int k = k_lo + threadIdx.x; k < k_hi; k += T) s1 += sumdev_v<DT>(row[k], K);
@@ -269,9 +273,18 @@ layernorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restric
     }
     s2 = cta_sum<T>(s2, slots, 1);
     const float rstd = rsqrtf(fmaf(s2, inv_D, eps));
-    for (int k = k_lo + threadIdx.x; k < k_hi; k += T) {
-        const int64_t j0 = (int64_t)k * 8 - phase;
-        st_stream(ya + k, ln_out_v<DT>(row[k], ln_load_shifted(gamma, j0), ln_load_shifted(beta, j0), mu, rstd));
+    if constexpr (TAB) {
+        pdl_wait();   // the table is complete and visible; plain loads (cached in L1), not the read-only path
+        const uint4* gt = tab + (size_t)phase * nvp;
+        const uint4* bt = tab + (size_t)(8 + phase) * nvp;
+#pragma unroll 2
+        for (int k = k_lo + threadIdx.x; k < k_hi; k += T)
+            st_stream(ya + k, ln_out_v<DT>(row[k], gt[k], bt[k], mu, rstd));
+    } else {
+        for (int k = k_lo + threadIdx.x; k < k_hi; k += T) {
+            const int64_t j0 = (int64_t)k * 8 - phase;
+            st_stream(ya + k, ln_out_v<DT>(row[k], ln_load_shifted(gamma, j0), ln_load_shifted(beta, j0), mu, rstd));
+        }
     }
     if (edge)
         yr[ej] = Elem<DT>::from_float(ln_out1<DT>(row16[ek * 8 + (threadIdx.x & 7)], __ldg(gamma + ej), __ldg(beta + ej), mu, rstd));

@@ -175,9 +175,9 @@ rmsnorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w, ui
 // ------------------------------------------------------------------ unaligned rows staged in shared memory
 // D % 8 != 0 (or a misaligned base) makes the 16-byte phase of a row change from row to row.
 // One CTA per row copies the row into shared memory in the phase it has in global memory:
-// vector k of the staging buffer holds row elements [8k - phase, 8k - phase + 8), so every
-// fully-inside vector is one aligned 16-byte global load and, because x and y rows share the
-// phase here, one aligned 16-byte store.  The (at most two) edge vectors are filled element
+// vector k of the staging buffer holds row elements [8k - phase, 8k - phase + 8), so the run of
+// fully-inside vectors is 16-byte aligned on both sides and arrives by bulk (TMA) copies, and,
+// because x and y rows share the phase here, every one of them leaves by an aligned 16-byte store.  The (at most two) edge vectors are filled element
 // by element, zeros standing in for the neighbours' bytes, and written back element by
 // element, so nothing outside the row is ever read or written.  Weights for an inside vector
 // start at the odd or even element 8k - phase: four 4-byte loads (phase even) or five plus
@@ -203,6 +203,7 @@ rmsnorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict_
     extern __shared__ __align__(128) unsigned char smem_raw[];
     uint4* row = reinterpret_cast<uint4*>(smem_raw);
     uint16_t* row16 = reinterpret_cast<uint16_t*>(smem_raw);
+    __shared__ uint64_t bar;
     __shared__ float slots[2 * kWarp];
     const int64_t r = blockIdx.x;
     const uint16_t* xr = x + r * D;
@@ -214,7 +215,9 @@ rmsnorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict_
     const uint4* xa = reinterpret_cast<const uint4*>(xr - phase);
     uint4* ya = reinterpret_cast<uint4*>(yr - phase);
 
-    for (int k = k_lo + threadIdx.x; k < k_hi; k += T) row[k] = ld_stream(xa + k);
+    // the fully-inside vectors are 16-byte aligned on both sides: the copy engine brings them in
+    // while sixteen threads fill the edge vectors
+    stage_interior_bulk(smem_raw, xa, k_lo, k_hi, &bar);
     if (threadIdx.x < 16) {  // edge vectors: 8 lanes for the first, 8 for the last
         const int k = (threadIdx.x < 8) ? 0 : nv - 1;
         const bool edge = (threadIdx.x < 8) ? (k_lo == 1) : (k_hi == nv - 1 && !(nv == 1 && k_lo == 1));
@@ -225,6 +228,7 @@ rmsnorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict_
         }
     }
     __syncthreads();
+    if (!mbar_wait(&bar, 0)) return;  // uniform: every thread waits on the same barrier
     float ss = 0.0f;
     for (int k = threadIdx.x; k < nv; k += T) ss += sumsq_v<DT>(row[k]);
     ss = cta_sum<T>(ss, slots, 0);

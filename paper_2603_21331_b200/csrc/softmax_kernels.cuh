@@ -224,6 +224,7 @@ softmax_stage_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, i
     extern __shared__ __align__(128) unsigned char smem_raw[];
     uint4* row = reinterpret_cast<uint4*>(smem_raw);
     uint16_t* row16 = reinterpret_cast<uint16_t*>(smem_raw);
+    __shared__ uint64_t bar;
     __shared__ float slots[2 * kWarp];
     const int64_t r = blockIdx.x;
     const uint16_t* xr = x + r * D;
@@ -239,9 +240,10 @@ softmax_stage_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, i
                          ((threadIdx.x < 8) ? (k_lo == 1) : (k_hi == nv - 1 && !(nv == 1 && k_lo == 1)));
     const int64_t my_j = (int64_t)my_edge_k * 8 - phase + (threadIdx.x & 7);
 
-    for (int k = k_lo + threadIdx.x; k < k_hi; k += T) row[k] = ld_stream(xa + k);
+    stage_interior_bulk(smem_raw, xa, k_lo, k_hi, &bar);   // the copy engine brings the inside vectors
     if (my_edge) row16[my_edge_k * 8 + (threadIdx.x & 7)] = (my_j >= 0 && my_j < D) ? ld_stream_u16(xr + my_j) : Elem<DT>::kNegInf;
     __syncthreads();
+    if (!mbar_wait(&bar, 0)) return;  // uniform: every thread waits on the same barrier
 
     uint32_t mx = neg_inf_word<DT>();
     for (int k = threadIdx.x; k < nv; k += T) mx = max_w<DT>(mx, max_v<DT>(row[k]));

@@ -117,12 +117,13 @@ def test_layernorm_misaligned_base_pointers():
             assert bool((ybuf[:yo] == 0).all()) and bool((ybuf[yo + rows * D:] == 0).all())
 
 
-@pytest.mark.parametrize("rows,D,xo", [(1024, 1027, 0), (1500, 4099, 0), (1100, 2051, 3), (1024, 8190, 1),
-                                       (1030, 16379, 0), (1025, 32754, 5)])
-def test_layernorm_unaligned_rows_with_the_shift_table(rows, D, xo):
-    """From 1024 rows on, unaligned rows that fit in registers read gamma and beta from a table of
-    all eight shifts written by a small kernel in front.  Parity on such launches, and the same
-    bits as the launch without the table (fewer rows) gives for the rows they share."""
+@pytest.mark.parametrize("rows,D,xo,few", [(1024, 1027, 0, 1000), (1500, 4099, 0, 1000), (1100, 2051, 3, 1000),
+                                           (1024, 8190, 1, 1000), (1030, 16379, 0, 1000), (1025, 32754, 5, 1000),
+                                           (256, 32771, 0, 200), (300, 40001, 3, 255), (260, 65539, 1, 100)])
+def test_layernorm_unaligned_rows_with_the_shift_table(rows, D, xo, few):
+    """From 1024 rows on (256 for rows staged in shared memory), unaligned rows read gamma and beta
+    from a table of all eight shifts written by a small kernel in front.  Parity on such launches,
+    and the same bits as the launch without the table (fewer rows) gives for the rows they share."""
     x, g, b = synth.layernorm_inputs(rows, D, synth.case_seed(8, rows + D))
     xb, gb, bb = synth.to_bits(x), synth.to_bits(g), synth.to_bits(b)
     ref = oracle.layernorm(xb, gb, bb, EPS)
@@ -138,7 +139,6 @@ def test_layernorm_unaligned_rows_with_the_shift_table(rows, D, xo):
     assert ak.ak_launch_count() - n0 == 2          # the table kernel and the row kernel
     _assert_ln_close(yv, ref, xb, gb, bb, f"layernorm {rows}x{D} offset {xo} (shift table)")
     assert bool((ybuf[:xo] == 0).all()) and bool((ybuf[xo + rows * D:] == 0).all())
-    few = 1000
     y2buf = torch.zeros(few * D + 8, dtype=torch.bfloat16, device=DEV)
     y2 = y2buf[xo:xo + few * D].view(few, D)
     n0 = ak.ak_launch_count()
