@@ -118,7 +118,7 @@ def test_layernorm_misaligned_base_pointers():
 
 
 @pytest.mark.parametrize("rows,D,xo,few", [(1024, 1027, 0, 1000), (1500, 4099, 0, 1000), (1100, 2051, 3, 1000),
-                                           (1024, 8190, 1, 1000), (1030, 16379, 0, 1000), (1025, 32754, 5, 1000),
+                                           (1024, 8190, 1, 200), (1030, 16379, 0, 255), (1025, 32754, 5, 1000),
                                            (256, 32771, 0, 200), (300, 40001, 3, 255), (260, 65539, 1, 100)])
 def test_layernorm_unaligned_rows_with_the_shift_table(rows, D, xo, few):
     """From 1024 rows on (256 for rows staged in shared memory), unaligned rows read gamma and beta
