@@ -24,7 +24,14 @@ cudaError_t scratch_alloc(void** p, size_t bytes, cudaStream_t st) {
     cudaMemPool_t pool = nullptr;
     if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64) {
         std::lock_guard<std::mutex> lock(mu);
-        if (!tried[dev]) {
+        // the pool is not created while `st` is being captured (creating one is no stream
+        // operation and could invalidate the capture); such a call uses the default pool
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (!tried[dev] && cudaStreamIsCapturing(st, &cap) != cudaSuccess) {
+            (void)cudaGetLastError();
+            cap = cudaStreamCaptureStatusActive;
+        }
+        if (!tried[dev] && cap == cudaStreamCaptureStatusNone) {
             tried[dev] = true;
             cudaMemPoolProps props = {};
             props.allocType = cudaMemAllocationTypePinned;

@@ -181,3 +181,42 @@ def test_two_streams_and_graph_replay():
         torch.cuda.synchronize()
         for ref, u in zip(serial, outs):
             assert torch.equal(ref.view(torch.uint8), u.view(torch.uint8))
+
+
+def test_first_call_inside_a_stream_capture():
+    """A process whose very first library call happens inside a CUDA-graph capture (nothing
+    warmed up, no scratch pool yet): the ops that take stream-ordered scratch capture, replay and
+    match the eager results taken afterwards."""
+    import subprocess
+    import sys
+    code = r"""
+import torch
+import paper_2603_21331_b200 as ak
+from paper_2603_21331_b200 import synth
+dev = "cuda"
+xu, gu, bu = synth.layernorm_inputs(1500, 2051, 606, device=dev)
+xl, _, _ = synth.layernorm_inputs(16, 65536, 607, device=dev)
+lg, tg = synth.xent_inputs(16, 65536, 608, device=dev)
+torch.cuda.synchronize()
+side = torch.cuda.Stream()
+side.wait_stream(torch.cuda.current_stream())
+graph = torch.cuda.CUDAGraph()
+with torch.cuda.stream(side):
+    with torch.cuda.graph(graph, stream=side):
+        loss, mean = ak.ak_xent_fwd(lg, tg)
+        outs = [ak.ak_layernorm_fwd(xu, gu, bu), ak.ak_rowsum_fwd(xl), loss, mean]
+torch.cuda.current_stream().wait_stream(side)
+graph.replay()
+torch.cuda.synchronize()
+got = [t.clone() for t in outs]
+loss, mean = ak.ak_xent_fwd(lg, tg)
+eager = [ak.ak_layernorm_fwd(xu, gu, bu), ak.ak_rowsum_fwd(xl), loss, mean]
+torch.cuda.synchronize()
+for a, b in zip(got, eager):
+    assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
+print("capture-first ok")
+"""
+    import os
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-c", code], cwd=root, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0 and "capture-first ok" in r.stdout, r.stdout[-2000:] + r.stderr[-4000:]
