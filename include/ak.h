@@ -66,7 +66,8 @@ enum {
     AK_PATH_WARP = 1,     /* one (or two) warps per row, row held in registers; rows <= 4 KiB (bf16 D <= 2048) */
     AK_PATH_CTA = 2,      /* one CTA per row, row held in registers; rows <= 64 KiB (bf16 D <= 32768) */
     AK_PATH_GENERIC = 3,  /* any D, any element alignment; row staged in shared memory in its 16-byte phase or re-read from L1/L2, single DRAM pass */
-    AK_PATH_SMEM = 4      /* one CTA per row, row staged in shared memory by bulk (TMA) copies; rows <= 224 KiB (bf16 D <= 114688) */
+    AK_PATH_SMEM = 4,     /* one CTA per row, row staged in shared memory by bulk (TMA) copies; rows <= 224 KiB (bf16 D <= 114688) */
+    AK_PATH_CLUSTER = 5   /* a thread-block cluster of 2, 4 or 8 CTAs per row, each staging a slice in its shared memory, partial results exchanged through distributed shared memory; rows of 32 bytes .. 1792 KiB (bf16 D <= 917504); chosen for rows longer than 224 KiB and when one CTA per row would leave SMs idle */
 };
 /* Element types of the *_dt entry points.  The plain entry points are bf16. */
 enum {

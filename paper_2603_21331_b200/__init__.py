@@ -3,7 +3,7 @@ cross-entropy and row-sum forward over bf16 [rows, D] tensors, exported from the
 library ``libak.so`` (``include/ak.h``) and bound here with ctypes.  No CPU or PyTorch
 fallback exists."""
 from .binding import (  # noqa: F401
-    AK_OK, AK_PATH_AUTO, AK_PATH_CTA, AK_PATH_GENERIC, AK_PATH_SMEM, AK_PATH_WARP,
+    AK_OK, AK_PATH_AUTO, AK_PATH_CLUSTER, AK_PATH_CTA, AK_PATH_GENERIC, AK_PATH_SMEM, AK_PATH_WARP,
     AK_XENT_AUTO, AK_XENT_ROW, AK_XENT_SPLIT, AkError, LIB_PATH,
     AK_DTYPE_BF16, AK_DTYPE_F16, AK_DTYPE_F32, ak_choose_path_dt, ak_rmsnorm_fwd_dt, ak_softmax_fwd_dt,
     ak_xent_fwd_dt, ak_launch_count, ak_layernorm_choose_path, ak_layernorm_fwd, ak_layernorm_fwd_dt, ak_rowsum_fwd_dt, ak_rmsnorm_choose_path,

@@ -24,7 +24,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libak.so")
 
 AK_OK = 0
-AK_PATH_AUTO, AK_PATH_WARP, AK_PATH_CTA, AK_PATH_GENERIC, AK_PATH_SMEM = 0, 1, 2, 3, 4
+AK_PATH_AUTO, AK_PATH_WARP, AK_PATH_CTA, AK_PATH_GENERIC, AK_PATH_SMEM, AK_PATH_CLUSTER = 0, 1, 2, 3, 4, 5
 AK_XENT_AUTO, AK_XENT_ROW, AK_XENT_SPLIT = 0, 1, 2
 AK_DTYPE_BF16, AK_DTYPE_F16, AK_DTYPE_F32 = 0, 1, 2
 _DTYPES = {torch.bfloat16: AK_DTYPE_BF16, torch.float16: AK_DTYPE_F16, torch.float32: AK_DTYPE_F32}

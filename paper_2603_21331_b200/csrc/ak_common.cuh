@@ -262,6 +262,60 @@ __device__ __forceinline__ void stage_interior_bulk(unsigned char* smem_raw, con
     }
 }
 
+// ---------------------------------------------------------------- thread-block clusters
+// A row split over the C CTAs of a cluster (C = 2, 4 or 8): every CTA stages its slice in its own
+// shared memory, reduces it, and the per-CTA results meet through distributed shared memory.
+// An exchange is a mailbox: `box` (C floats) plus an mbarrier in every CTA, armed once for
+// C x 4 bytes.  CTA `rank` posts its value v (uniform over its threads) to slot `rank` of the box
+// of EVERY CTA of the cluster with asynchronous remote stores that count their bytes in on the
+// RECEIVER's mbarrier; each CTA then waits on its own barrier only.  No cluster-wide barrier or
+// fence is on the path (a release / acquire cluster barrier per exchange stalled every warp on
+// the fence: about a fifth of the kernel's time).  Every CTA combines box[0 .. C-1] in rank
+// order, so all of them hold the same bits.  A mailbox serves one exchange per kernel.
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// The one cluster barrier of these kernels says "every CTA of the cluster runs and has armed its
+// mailboxes" (the mbarrier initialisation is published by fence.mbarrier_init.release.cluster in
+// mbar_init); it orders no other memory, so the arrival is relaxed, and it is split so that the
+// row's load and first pass run between arrival and wait.
+__device__ __forceinline__ void cluster_arrive_relaxed() {
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.aligned;" ::: "memory"); }
+// by one thread, before the CTA's cluster_arrive_relaxed
+__device__ __forceinline__ void mailbox_arm(uint64_t* xbar, int C) {
+    mbar_init(xbar, 1);
+    mbar_expect_tx(xbar, (uint32_t)C * 4u);
+}
+// by every thread of every CTA of the cluster; returns false if the bounded wait gave up
+__device__ __forceinline__ bool mailbox_exchange(float v, float* box, uint64_t* xbar, int C, uint32_t rank) {
+    if ((int)threadIdx.x < C) {
+        uint32_t rbox, rbar;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbox) : "r"(smem_addr(box + rank)), "r"(threadIdx.x));
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(smem_addr(xbar)), "r"(threadIdx.x));
+        asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(rbox),
+                     "r"(__float_as_uint(v)), "r"(rbar)
+                     : "memory");
+    }
+    return mbar_wait(xbar, 0);
+}
+// One thread starts the bulk copies of a contiguous, 16-byte aligned span into shared memory
+// (nothing to copy: a plain arrival, so the wait still completes).  The mbarrier must be
+// initialised and that made visible (a CTA barrier) before.
+__device__ __forceinline__ void bulk_load_span(unsigned char* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar) {
+    if (bytes == 0) {
+        mbar_arrive(bar);
+        return;
+    }
+    mbar_expect_tx(bar, bytes);
+    const unsigned char* src = static_cast<const unsigned char*>(gmem_src);
+    for (uint32_t off = 0; off < bytes; off += kStageChunk) bulk_load(smem_dst + off, src + off, min(kStageChunk, bytes - off), bar);
+}
+constexpr int kMaxCluster = 8;   // portable cluster size limit
+
 // Largest row (bytes) the shared-memory-staged kernels accept: 224 KiB of dynamic shared
 // memory out of the 227 KiB a CTA may own (a few hundred bytes stay static).
 constexpr int kMaxRowSmemBytes = 224 * 1024;
@@ -271,6 +325,11 @@ constexpr int kMaxRowSmemBytes = 224 * 1024;
 void count_launch(int n = 1);
 // cudaMallocAsync from the library's own pool (free with cudaFreeAsync on the same stream)
 cudaError_t scratch_alloc(void** p, size_t bytes, cudaStream_t st);
+// CTAs per row of the cluster layout for aligned rows of `row_bytes` bytes: 1 = keep one CTA per
+// row (or the row does not fit eight slices); otherwise 2, 4 or 8.  Pure function of its arguments.
+int cluster_ctas(int64_t rows, int64_t row_bytes, int64_t split_from);
+constexpr int64_t kClusterFromNorm = 65536 + 16;   // RMSNorm, LayerNorm: rows longer than the 64 KiB the register path takes
+constexpr int64_t kClusterFromSoftmax = 65536;     // softmax: from 64 KiB rows on
 int sm_count();  // SMs of the current device (cached per device)
 
 // Per-op host dispatchers (each defined next to its kernels).  All arguments have been
@@ -344,6 +403,25 @@ shift_params_kernel(const uint16_t* __restrict__ p0, const uint16_t* __restrict_
         w[h] = lo | (hi << 16);
     }
     tab[idx] = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// Launch `kernel` in thread-block clusters of C CTAs along x (grid a multiple of C).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_cluster(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, int C,
+                                  cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)C;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
 // Launch `kernel` as a programmatic dependent of the work before it in the stream.

@@ -56,6 +56,23 @@ int launch_smem(const void* x, const void* g, const void* b, void* y, int64_t ro
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
+// a cluster of C CTAs per row (C from cluster_ctas, at least 2)
+template <int DT, int THREADS>
+int launch_cluster_rows(const void* x, const void* g, const void* b, void* y, int64_t rows, int nvec, int C, float inv_D,
+                        float eps, cudaStream_t st) {
+    static const bool configured = [] {
+        return cudaFuncSetAttribute(layernorm_cluster_kernel<THREADS, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    kMaxRowSmemBytes) == cudaSuccess;
+    }();
+    if (!configured) return AK_ERR_CUDA;
+    const size_t smem = (size_t)((nvec + C - 1) / C) * 16;
+    const cudaError_t e = launch_cluster(layernorm_cluster_kernel<THREADS, DT>, (unsigned)(rows * C), THREADS, smem, C, st,
+                                         static_cast<const uint4*>(x), static_cast<const uint4*>(g),
+                                         static_cast<const uint4*>(b), static_cast<uint4*>(y), nvec, C, inv_D, eps);
+    count_launch();
+    return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+}
+
 // Rows that are not 16-byte aligned need gamma and beta shifted to the row's phase.  From
 // `min_rows` rows on they are shifted once per launch, for all eight phases, into a table in
 // stream-ordered scratch (16 x the row's vectors) instead of once per output vector; the row
@@ -181,6 +198,14 @@ int dispatch_t(const void* x, const void* gamma, const void* beta, void* y, int6
             if (row_bytes > kMaxRowSmemBytes) return AK_ERR_SHAPE;
             if (nvec <= 4096) return launch_smem<DT, 256>(x, gamma, beta, y, rows, nvec, inv_D, eps, st);
             return launch_smem<DT, 512>(x, gamma, beta, y, rows, nvec, inv_D, eps, st);
+        case AK_PATH_CLUSTER: {
+            int C = cluster_ctas(rows, row_bytes, kClusterFromNorm);
+            if (C < 2) C = 2;   // forced by the caller
+            if (nvec < C || row_bytes > (int64_t)C * kMaxRowSmemBytes || rows * C > 2147483647LL) return AK_ERR_SHAPE;
+            if ((nvec + C - 1) / C <= 4096)
+                return launch_cluster_rows<DT, 256>(x, gamma, beta, y, rows, nvec, C, inv_D, eps, st);
+            return launch_cluster_rows<DT, 512>(x, gamma, beta, y, rows, nvec, C, inv_D, eps, st);
+        }
         case AK_PATH_GENERIC: {
             if constexpr (DT == AK_DTYPE_F32) {
                 static const int resident = resident_ctas(layernorm_generic32_kernel, kLnGenericThreads);
@@ -226,9 +251,10 @@ int dispatch_t(const void* x, const void* gamma, const void* beta, void* y, int6
 }  // namespace
 
 int layernorm_choose(int64_t rows, int64_t D, bool aligned16, int dtype) {
-    (void)rows;
     const int64_t bytes = D * dtype_bytes(dtype);
-    if (!aligned16 || (bytes & 15) != 0 || bytes > kMaxRowSmemBytes) return AK_PATH_GENERIC;
+    if (!aligned16 || (bytes & 15) != 0) return AK_PATH_GENERIC;
+    if (cluster_ctas(rows, bytes, kClusterFromNorm) > 1) return AK_PATH_CLUSTER;
+    if (bytes > kMaxRowSmemBytes) return AK_PATH_GENERIC;
     if (bytes <= 4096) return AK_PATH_WARP;
     if (bytes <= 65536) return AK_PATH_CTA;   // up to 64 KiB the register layout beats the staged one
     return AK_PATH_SMEM;

@@ -210,6 +210,66 @@ layernorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gam
         st_stream(yr + i, ln_out_v<DT>(row[i], __ldg(gamma + i), __ldg(beta + i), mu, rstd));
 }
 
+// ------------------------------------------------------------------ rows split over a cluster
+// C CTAs of a thread-block cluster share one row (few rows still fill the GPU; rows of up to
+// C x 224 KiB are done in one pass over DRAM).  CTA c stages vectors
+// [nvec * c / C, nvec * (c + 1) / C) in its shared memory by bulk copies; the slice sums of
+// x - K (K = the row's first element, read by every CTA) and then of (x - mu)^2 meet through
+// distributed shared memory and are added in rank order in every CTA.  grid = rows * C,
+// cluster = C.  Dynamic shared memory = ceil(nvec / C) * 16 bytes.
+template <int THREADS, int DT = AK_DTYPE_BF16>
+__global__ void __launch_bounds__(THREADS)
+layernorm_cluster_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamma, const uint4* __restrict__ beta,
+                         uint4* __restrict__ y, int nvec, int C, float inv_D, float eps) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const uint4* row = reinterpret_cast<const uint4*>(smem_raw);
+    __shared__ uint64_t bar;
+    __shared__ float slots[2 * kWarp];
+    __shared__ float box1[kMaxCluster], box2[kMaxCluster];
+    __shared__ uint64_t xbar1, xbar2;
+    const uint32_t c = cluster_rank();
+    const int64_t r = blockIdx.x / C;
+    const int v0 = (int)((int64_t)nvec * c / C);
+    const int n = (int)((int64_t)nvec * (c + 1) / C) - v0;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        mailbox_arm(&xbar1, C);
+        mailbox_arm(&xbar2, C);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) bulk_load_span(smem_raw, x + r * nvec + v0, (uint32_t)n * 16u, &bar);
+    const uint32_t first = __ldg(reinterpret_cast<const uint32_t*>(x + r * nvec));
+    float K;
+    if constexpr (DT == AK_DTYPE_F32) K = __uint_as_float(first);
+    else K = Elem<DT>::to_float((uint16_t)(first & 0xffffu));
+    cluster_arrive_relaxed();
+    // a wait that gave up (never expected) contributes nothing and writes nothing, but still posts
+    int nn = mbar_wait(&bar, 0) ? n : 0;
+    float s1 = 0.0f;
+#pragma unroll 4
+    for (int i = threadIdx.x; i < nn; i += THREADS) s1 += sumdev_v<DT>(row[i], K);
+    s1 = cta_sum<THREADS>(s1, slots, 0);
+    cluster_wait();   // every CTA of the cluster runs, its mailboxes armed, before anything is posted to it
+    if (!mailbox_exchange(s1, box1, &xbar1, C, c)) nn = 0;
+    float t1 = 0.0f;
+    for (int i = 0; i < C; ++i) t1 += box1[i];
+    const float mu = fmaf(t1, inv_D, K);
+    float s2 = 0.0f;
+#pragma unroll 4
+    for (int i = threadIdx.x; i < nn; i += THREADS) s2 += sqdev_v<DT>(row[i], mu);
+    s2 = cta_sum<THREADS>(s2, slots, 1);
+    if (!mailbox_exchange(s2, box2, &xbar2, C, c)) nn = 0;
+    float t2 = 0.0f;
+    for (int i = 0; i < C; ++i) t2 += box2[i];
+    const float rstd = rsqrtf(fmaf(t2, inv_D, eps));
+    uint4* yr = y + r * nvec + v0;
+    const uint4* gr = gamma + v0;
+    const uint4* br = beta + v0;
+#pragma unroll 2
+    for (int i = threadIdx.x; i < nn; i += THREADS)
+        st_stream(yr + i, ln_out_v<DT>(row[i], __ldg(gr + i), __ldg(br + i), mu, rstd));
+}
+
 // ------------------------------------------------------------------ unaligned rows staged in shared memory
 // D % 8 != 0 (or a misaligned base): one CTA per row copies the row into shared memory in the
 // 16-byte phase it has in global memory, so interior vectors are aligned 16-byte loads and

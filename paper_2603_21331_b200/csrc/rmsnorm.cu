@@ -54,6 +54,23 @@ int launch_smem(const void* x, const void* w, void* y, int64_t rows, int nvec, f
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
+// a cluster of C CTAs per row (C from cluster_ctas, at least 2)
+template <int DT, int THREADS>
+int launch_cluster_rows(const void* x, const void* w, void* y, int64_t rows, int nvec, int C, float inv_D, float eps,
+                        cudaStream_t st) {
+    static const bool configured = [] {
+        return cudaFuncSetAttribute(rmsnorm_cluster_kernel<THREADS, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    kMaxRowSmemBytes) == cudaSuccess;
+    }();
+    if (!configured) return AK_ERR_CUDA;
+    const size_t smem = (size_t)((nvec + C - 1) / C) * 16;
+    const cudaError_t e = launch_cluster(rmsnorm_cluster_kernel<THREADS, DT>, (unsigned)(rows * C), THREADS, smem, C, st,
+                                         static_cast<const uint4*>(x), static_cast<const uint4*>(w),
+                                         static_cast<uint4*>(y), nvec, C, inv_D, eps);
+    count_launch();
+    return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+}
+
 // unaligned rows held in registers: vectors per thread 1..8 for a CTA of THREADS threads
 template <int DT, int THREADS, int VPT>
 int launch_regp(const uint16_t* x, const uint16_t* w, uint16_t* y, int64_t rows, int64_t D, float inv_D, float eps,
@@ -81,9 +98,10 @@ int launch_regp_vpt(int vpt, const uint16_t* x, const uint16_t* w, uint16_t* y, 
 }  // namespace
 
 int rmsnorm_choose(int64_t rows, int64_t D, bool aligned16, int dtype) {
-    (void)rows;
     const int64_t bytes = D * dtype_bytes(dtype);   // row bytes decide the layout
-    if (!aligned16 || (bytes & 15) != 0 || bytes > kMaxRowSmemBytes) return AK_PATH_GENERIC;
+    if (!aligned16 || (bytes & 15) != 0) return AK_PATH_GENERIC;
+    if (cluster_ctas(rows, bytes, kClusterFromNorm) > 1) return AK_PATH_CLUSTER;
+    if (bytes > kMaxRowSmemBytes) return AK_PATH_GENERIC;
     if (bytes <= 4096) return AK_PATH_WARP;
     if (bytes <= 65536) return AK_PATH_CTA;   // up to 64 KiB the register layout beats the staged one
     return AK_PATH_SMEM;
@@ -123,6 +141,13 @@ int dispatch_t(const void* x, const void* w, void* y, int64_t rows, int64_t D, f
             if (row_bytes > kMaxRowSmemBytes) return AK_ERR_SHAPE;
             if (nvec <= 4096) return launch_smem<DT, 256>(x, w, y, rows, nvec, inv_D, eps, st);
             return launch_smem<DT, 512>(x, w, y, rows, nvec, inv_D, eps, st);
+        case AK_PATH_CLUSTER: {
+            int C = cluster_ctas(rows, row_bytes, kClusterFromNorm);
+            if (C < 2) C = 2;   // forced by the caller
+            if (nvec < C || row_bytes > (int64_t)C * kMaxRowSmemBytes || rows * C > 2147483647LL) return AK_ERR_SHAPE;
+            if ((nvec + C - 1) / C <= 4096) return launch_cluster_rows<DT, 256>(x, w, y, rows, nvec, C, inv_D, eps, st);
+            return launch_cluster_rows<DT, 512>(x, w, y, rows, nvec, C, inv_D, eps, st);
+        }
         case AK_PATH_GENERIC: {
             if constexpr (DT == AK_DTYPE_F32) {
                 static const int resident32 = [] {

@@ -172,6 +172,51 @@ rmsnorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w, ui
     for (int i = threadIdx.x; i < nvec; i += THREADS) st_stream(yr + i, scale_v<DT>(row[i], __ldg(w + i), rstd));
 }
 
+// ------------------------------------------------------------------ rows split over a cluster
+// C CTAs of a thread-block cluster share one row: few rows then still fill the GPU, and rows of
+// up to C x 224 KiB are normalised in one pass over DRAM.  CTA c stages vectors
+// [nvec * c / C, nvec * (c + 1) / C) in its shared memory by bulk copies, sums its squares, and
+// the C partial sums meet through distributed shared memory (a mailbox exchange; added in rank
+// order in every CTA, so all hold the same bits).  grid = rows * C, cluster = C.  Dynamic shared memory = the
+// largest slice, ceil(nvec / C) * 16 bytes.
+template <int THREADS, int DT = AK_DTYPE_BF16>
+__global__ void __launch_bounds__(THREADS)
+rmsnorm_cluster_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w, uint4* __restrict__ y,
+                       int nvec, int C, float inv_D, float eps) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const uint4* row = reinterpret_cast<const uint4*>(smem_raw);
+    __shared__ uint64_t bar;
+    __shared__ float slots[2 * kWarp];
+    __shared__ float box[kMaxCluster];
+    __shared__ uint64_t xbar;
+    const uint32_t c = cluster_rank();
+    const int64_t r = blockIdx.x / C;
+    const int v0 = (int)((int64_t)nvec * c / C);
+    const int n = (int)((int64_t)nvec * (c + 1) / C) - v0;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        mailbox_arm(&xbar, C);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) bulk_load_span(smem_raw, x + r * nvec + v0, (uint32_t)n * 16u, &bar);
+    cluster_arrive_relaxed();
+    // a wait that gave up (never expected) contributes nothing and writes nothing, but still posts
+    int nn = mbar_wait(&bar, 0) ? n : 0;
+    float ss = 0.0f;
+#pragma unroll 4
+    for (int i = threadIdx.x; i < nn; i += THREADS) ss += sumsq_v<DT>(row[i]);
+    ss = cta_sum<THREADS>(ss, slots, 0);
+    cluster_wait();   // every CTA of the cluster runs, its mailboxes armed, before anything is posted to it
+    if (!mailbox_exchange(ss, box, &xbar, C, c)) nn = 0;
+    float tot = 0.0f;
+    for (int i = 0; i < C; ++i) tot += box[i];
+    const float rstd = rsqrtf(fmaf(tot, inv_D, eps));
+    uint4* yr = y + r * nvec + v0;
+    const uint4* wr = w + v0;
+#pragma unroll 4
+    for (int i = threadIdx.x; i < nn; i += THREADS) st_stream(yr + i, scale_v<DT>(row[i], __ldg(wr + i), rstd));
+}
+
 // ------------------------------------------------------------------ unaligned rows staged in shared memory
 // D % 8 != 0 (or a misaligned base) makes the 16-byte phase of a row change from row to row.
 // One CTA per row copies the row into shared memory in the phase it has in global memory:

@@ -67,6 +67,21 @@ int launch_regp(const uint16_t* x, uint16_t* y, int64_t rows, int64_t D, cudaStr
     count_launch();
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
+// a cluster of C CTAs per row (C from cluster_ctas, at least 2)
+template <int DT, int THREADS, int KEEP>
+int launch_cluster_rows(const void* x, void* y, int64_t rows, int nvec, int C, cudaStream_t st) {
+    static const bool configured = [] {
+        return cudaFuncSetAttribute(softmax_cluster_kernel<THREADS, KEEP, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    kMaxRowSmemBytes) == cudaSuccess;
+    }();
+    if (!configured) return AK_ERR_CUDA;
+    const size_t smem = (size_t)((nvec + C - 1) / C) * 16;
+    const cudaError_t e = launch_cluster(softmax_cluster_kernel<THREADS, KEEP, DT>, (unsigned)(rows * C), THREADS, smem, C, st,
+                                         static_cast<const uint4*>(x), static_cast<uint4*>(y), nvec, C);
+    count_launch();
+    return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+}
+
 // unaligned rows held in registers: vectors per thread 1..8 for a CTA of THREADS threads
 template <int DT, int THREADS, int MINB>
 int launch_regp_vpt(int vpt, const uint16_t* x, uint16_t* y, int64_t rows, int64_t D, cudaStream_t st) {
@@ -120,6 +135,13 @@ int dispatch_t(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st,
             // short bursts and under the power cap of a long run up to 64 KiB rows
             if (nvec <= 4096) return launch_smem<DT, 256, 4>(x, y, rows, nvec, st);
             return launch_smem<DT, 512, 0>(x, y, rows, nvec, st);
+        case AK_PATH_CLUSTER: {
+            int C = cluster_ctas(rows, row_bytes, kClusterFromSoftmax);
+            if (C < 2) C = 2;   // forced by the caller
+            if (nvec < C || row_bytes > (int64_t)C * kMaxRowSmemBytes || rows * C > 2147483647LL) return AK_ERR_SHAPE;
+            if ((nvec + C - 1) / C <= 4096) return launch_cluster_rows<DT, 256, 4>(x, y, rows, nvec, C, st);
+            return launch_cluster_rows<DT, 512, 0>(x, y, rows, nvec, C, st);
+        }
         case AK_PATH_GENERIC: {
             if constexpr (DT == AK_DTYPE_F32) {
                 static const int resident = resident_ctas(softmax_generic32_kernel, kSmGenericThreads);
@@ -160,9 +182,10 @@ int dispatch_t(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st,
 }  // namespace
 
 int softmax_choose(int64_t rows, int64_t D, bool aligned16, int dtype) {
-    (void)rows;
     const int64_t bytes = D * dtype_bytes(dtype);
-    if (!aligned16 || (bytes & 15) != 0 || bytes > kMaxRowSmemBytes) return AK_PATH_GENERIC;
+    if (!aligned16 || (bytes & 15) != 0) return AK_PATH_GENERIC;
+    if (cluster_ctas(rows, bytes, kClusterFromSoftmax) > 1) return AK_PATH_CLUSTER;
+    if (bytes > kMaxRowSmemBytes) return AK_PATH_GENERIC;
     if (bytes <= 4096) return AK_PATH_WARP;
     if (bytes <= 16384) return AK_PATH_CTA;
     return AK_PATH_SMEM;

@@ -213,6 +213,76 @@ softmax_smem_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int nvec
     }
 }
 
+// ------------------------------------------------------------------ rows split over a cluster
+// C CTAs of a thread-block cluster share one row (few rows still fill the GPU; rows of up to
+// C x 224 KiB, a 128K vocabulary among them, are done in one pass over DRAM).  CTA c stages
+// vectors [nvec * c / C, nvec * (c + 1) / C) in its shared memory by bulk copies; the slice
+// maxima and then the slice sums meet through distributed shared memory and are combined in
+// rank order in every CTA.  The first KEEP vectors of a thread keep their exponentials in
+// registers.  grid = rows * C, cluster = C.  Dynamic shared memory = ceil(nvec / C) * 16 bytes.
+template <int THREADS, int KEEP, int DT = AK_DTYPE_BF16>
+__global__ void __launch_bounds__(THREADS)
+softmax_cluster_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int nvec, int C) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const uint4* row = reinterpret_cast<const uint4*>(smem_raw);
+    __shared__ uint64_t bar;
+    __shared__ float slots[2 * kWarp];
+    __shared__ float box_m[kMaxCluster], box_s[kMaxCluster];
+    __shared__ uint64_t xbar_m, xbar_s;
+    const uint32_t c = cluster_rank();
+    const int64_t r = blockIdx.x / C;
+    const int v0 = (int)((int64_t)nvec * c / C);
+    const int n = (int)((int64_t)nvec * (c + 1) / C) - v0;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        mailbox_arm(&xbar_m, C);
+        mailbox_arm(&xbar_s, C);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) bulk_load_span(smem_raw, x + r * nvec + v0, (uint32_t)n * 16u, &bar);
+    cluster_arrive_relaxed();
+    // a wait that gave up (never expected) contributes nothing and writes nothing, but still posts
+    int nn = mbar_wait(&bar, 0) ? n : 0;
+
+    uint32_t mx = neg_inf_word<DT>();
+#pragma unroll 4
+    for (int i = threadIdx.x; i < nn; i += THREADS) mx = max_w<DT>(mx, max_v<DT>(row[i]));
+    const float m_cta = cta_max<THREADS>(hmax_of<DT>(mx), slots, 0);
+    cluster_wait();   // every CTA of the cluster runs, its mailboxes armed, before anything is posted to it
+    if (!mailbox_exchange(m_cta, box_m, &xbar_m, C, c)) nn = 0;
+    float m = box_m[0];
+    for (int i = 1; i < C; ++i) m = fmaxf(m, box_m[i]);
+    const float m2 = m * kLog2e;
+
+    f32x2 kept[KEEP > 0 ? KEEP : 1][kExpPairs<DT>];
+    float sum = 0.0f;
+    f32x2 e[kExpPairs<DT>];
+#pragma unroll
+    for (int k = 0; k < KEEP; ++k) {
+        const int i = threadIdx.x + k * THREADS;
+        if (i < nn) sum += exp_v<DT>(row[i], m2, kept[k]);
+    }
+#pragma unroll 2
+    for (int i = threadIdx.x + KEEP * THREADS; i < nn; i += THREADS) sum += exp_v<DT>(row[i], m2, e);
+    sum = cta_sum<THREADS>(sum, slots, 1);
+    if (!mailbox_exchange(sum, box_s, &xbar_s, C, c)) nn = 0;
+    float tot = 0.0f;
+    for (int i = 0; i < C; ++i) tot += box_s[i];
+    const float inv = 1.0f / tot;
+
+    uint4* yr = y + r * nvec + v0;
+#pragma unroll
+    for (int k = 0; k < KEEP; ++k) {
+        const int i = threadIdx.x + k * THREADS;
+        if (i < nn) st_stream(yr + i, norm_v<DT>(kept[k], inv));
+    }
+#pragma unroll 2
+    for (int i = threadIdx.x + KEEP * THREADS; i < nn; i += THREADS) {
+        exp_v<DT>(row[i], m2, e);
+        st_stream(yr + i, norm_v<DT>(e, inv));
+    }
+}
+
 // ------------------------------------------------------------------ unaligned rows staged in shared memory
 // Same staging as the RMSNorm kernel of that name: the row sits in shared memory in the
 // 16-byte phase it has in global memory (x and y rows share it), fully-inside vectors move

@@ -57,7 +57,8 @@ def test_validation_rejects_before_any_cuda_call():
     assert l.ak_layernorm_fwd(P, P, P, P, 1, 0, 1e-5, None) == 2
     assert l.ak_layernorm_fwd(P, P, P + 1, P, 1, 8, 1e-5, None) == 3
     assert l.ak_layernorm_fwd(P, P, P, P, 1, 8, -1e-5, None) == 4
-    assert l.ak_layernorm_fwd_path(P, P, P, P, 1, 8, 1e-5, None, 5) == 4
+    assert l.ak_layernorm_fwd_path(P, P, P, P, 1, 8, 1e-5, None, 6) == 4
+    assert l.ak_layernorm_fwd_path(P, P, P, P, 1, 8, 1e-5, None, 5) == 2          # a cluster needs two vectors per row
     assert l.ak_layernorm_fwd(P, P, P, P, 0, 8, 1e-5, None) == 0
     assert l.ak_rowsum_fwd(None, P, 1, 8, None) == 1
     assert l.ak_rowsum_fwd(P, None, 1, 8, None) == 1
@@ -124,16 +125,23 @@ def test_dispatch_is_a_pure_function_of_shape_and_alignment():
     assert ak.ak_rmsnorm_choose_path(8192, 4096, True) == ak.AK_PATH_CTA
     assert ak.ak_rmsnorm_choose_path(8192, 16384, True) == ak.AK_PATH_CTA
     assert ak.ak_rmsnorm_choose_path(8192, 32768, True) == ak.AK_PATH_CTA
-    assert ak.ak_rmsnorm_choose_path(8192, 32776, True) == ak.AK_PATH_SMEM
+    assert ak.ak_rmsnorm_choose_path(8192, 32776, True) == ak.AK_PATH_CLUSTER    # longer than 64 KiB: split over a cluster
     assert ak.ak_layernorm_choose_path(8192, 32768, True) == ak.AK_PATH_CTA
-    assert ak.ak_layernorm_choose_path(8192, 40960, True) == ak.AK_PATH_SMEM
+    assert ak.ak_layernorm_choose_path(8192, 40960, True) == ak.AK_PATH_CLUSTER
     assert ak.ak_rmsnorm_choose_path(8192, 4099, True) == ak.AK_PATH_GENERIC
     assert ak.ak_rmsnorm_choose_path(8192, 4096, False) == ak.AK_PATH_GENERIC
-    assert ak.ak_rmsnorm_choose_path(8192, 65536, True) == ak.AK_PATH_SMEM
-    assert ak.ak_rmsnorm_choose_path(8192, 131072, True) == ak.AK_PATH_GENERIC
+    assert ak.ak_rmsnorm_choose_path(8192, 65536, True) == ak.AK_PATH_CLUSTER
+    assert ak.ak_rmsnorm_choose_path(8192, 131072, True) == ak.AK_PATH_CLUSTER   # 256 KiB rows: four to eight CTAs' shared memory
+    assert ak.ak_rmsnorm_choose_path(8192, 917504, True) == ak.AK_PATH_CLUSTER   # 8 x 224 KiB, the longest
+    assert ak.ak_rmsnorm_choose_path(8192, 917512, True) == ak.AK_PATH_GENERIC
+    assert ak.ak_rmsnorm_choose_path(64, 16384, True) == ak.AK_PATH_CLUSTER      # few rows of 32 KiB or more
+    assert ak.ak_rmsnorm_choose_path(65, 16384, True) == ak.AK_PATH_CTA
+    assert ak.ak_rmsnorm_choose_path(64, 8192, True) == ak.AK_PATH_CTA
+    assert ak.ak_softmax_choose_path(16384, 16384, True) == ak.AK_PATH_SMEM
+    assert ak.ak_softmax_choose_path(16, 128256, True) == ak.AK_PATH_CLUSTER
     assert ak.ak_softmax_choose_path(16384, 512, True) == ak.AK_PATH_WARP
     assert ak.ak_softmax_choose_path(16384, 8192, True) == ak.AK_PATH_CTA
-    assert ak.ak_softmax_choose_path(16384, 32768, True) == ak.AK_PATH_SMEM
+    assert ak.ak_softmax_choose_path(16384, 32768, True) == ak.AK_PATH_CLUSTER   # 64 KiB rows and longer
     assert ak.ak_softmax_choose_path(16384, 128257, True) == ak.AK_PATH_GENERIC
     for rows, V in ((4096, 32000), (4096, 128256), (16384, 128256)):
         assert ak.ak_xent_choose_path(rows, V) == (ak.AK_XENT_ROW, 1)

@@ -19,6 +19,8 @@ NAME = synth.DTYPE_NAMES
 def _legal_paths(D, dtype):
     nbytes = D * torch.empty((), dtype=dtype).element_size()
     paths = [ak.AK_PATH_GENERIC]
+    if nbytes % 16 == 0 and nbytes >= 32 and nbytes <= 8 * 224 * 1024:
+        paths.append(ak.AK_PATH_CLUSTER)
     if nbytes % 16 == 0 and nbytes <= 224 * 1024:
         paths.append(ak.AK_PATH_SMEM)
     if nbytes % 16 == 0 and nbytes <= 65536:

@@ -12,10 +12,13 @@ from parity import assert_bf16_close, assert_loss_close, guarded
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
 WARP, CTA, GEN, SMEM = ak.AK_PATH_WARP, ak.AK_PATH_CTA, ak.AK_PATH_GENERIC, ak.AK_PATH_SMEM
+CLUSTER = ak.AK_PATH_CLUSTER
 
 
 def _legal_paths(D):
     paths = [GEN]
+    if D % 8 == 0 and D >= 16 and D * 2 <= 8 * 224 * 1024:
+        paths.append(CLUSTER)
     if D % 8 == 0 and D * 2 <= 224 * 1024:
         paths.append(SMEM)
     if D % 8 == 0 and D <= 32768:
