@@ -199,7 +199,7 @@ int dispatch_t(const void* x, const void* gamma, const void* beta, void* y, int6
             if (nvec <= 4096) return launch_smem<DT, 256>(x, gamma, beta, y, rows, nvec, inv_D, eps, st);
             return launch_smem<DT, 512>(x, gamma, beta, y, rows, nvec, inv_D, eps, st);
         case AK_PATH_CLUSTER: {
-            int C = cluster_ctas(rows, row_bytes, kClusterFromNorm);
+            int C = cluster_ctas(rows, row_bytes, kClusterFrom);
             if (C < 2) C = 2;   // forced by the caller
             if (nvec < C || row_bytes > (int64_t)C * kMaxRowSmemBytes || rows * C > 2147483647LL) return AK_ERR_SHAPE;
             if ((nvec + C - 1) / C <= 4096)
@@ -253,7 +253,7 @@ int dispatch_t(const void* x, const void* gamma, const void* beta, void* y, int6
 int layernorm_choose(int64_t rows, int64_t D, bool aligned16, int dtype) {
     const int64_t bytes = D * dtype_bytes(dtype);
     if (!aligned16 || (bytes & 15) != 0) return AK_PATH_GENERIC;
-    if (cluster_ctas(rows, bytes, kClusterFromNorm) > 1) return AK_PATH_CLUSTER;
+    if (cluster_ctas(rows, bytes, kClusterFrom) > 1) return AK_PATH_CLUSTER;
     if (bytes > kMaxRowSmemBytes) return AK_PATH_GENERIC;
     if (bytes <= 4096) return AK_PATH_WARP;
     if (bytes <= 65536) return AK_PATH_CTA;   // up to 64 KiB the register layout beats the staged one

@@ -136,7 +136,7 @@ int dispatch_t(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st,
             if (nvec <= 4096) return launch_smem<DT, 256, 4>(x, y, rows, nvec, st);
             return launch_smem<DT, 512, 0>(x, y, rows, nvec, st);
         case AK_PATH_CLUSTER: {
-            int C = cluster_ctas(rows, row_bytes, kClusterFromSoftmax);
+            int C = cluster_ctas(rows, row_bytes, kClusterFrom);
             if (C < 2) C = 2;   // forced by the caller
             if (nvec < C || row_bytes > (int64_t)C * kMaxRowSmemBytes || rows * C > 2147483647LL) return AK_ERR_SHAPE;
             if ((nvec + C - 1) / C <= 4096) return launch_cluster_rows<DT, 256, 4>(x, y, rows, nvec, C, st);
@@ -184,7 +184,7 @@ int dispatch_t(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st,
 int softmax_choose(int64_t rows, int64_t D, bool aligned16, int dtype) {
     const int64_t bytes = D * dtype_bytes(dtype);
     if (!aligned16 || (bytes & 15) != 0) return AK_PATH_GENERIC;
-    if (cluster_ctas(rows, bytes, kClusterFromSoftmax) > 1) return AK_PATH_CLUSTER;
+    if (cluster_ctas(rows, bytes, kClusterFrom) > 1) return AK_PATH_CLUSTER;
     if (bytes > kMaxRowSmemBytes) return AK_PATH_GENERIC;
     if (bytes <= 4096) return AK_PATH_WARP;
     if (bytes <= 16384) return AK_PATH_CTA;

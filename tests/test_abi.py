@@ -141,7 +141,8 @@ def test_dispatch_is_a_pure_function_of_shape_and_alignment():
     assert ak.ak_softmax_choose_path(16, 128256, True) == ak.AK_PATH_CLUSTER
     assert ak.ak_softmax_choose_path(16384, 512, True) == ak.AK_PATH_WARP
     assert ak.ak_softmax_choose_path(16384, 8192, True) == ak.AK_PATH_CTA
-    assert ak.ak_softmax_choose_path(16384, 32768, True) == ak.AK_PATH_CLUSTER   # 64 KiB rows and longer
+    assert ak.ak_softmax_choose_path(16384, 32768, True) == ak.AK_PATH_SMEM
+    assert ak.ak_softmax_choose_path(16384, 32776, True) == ak.AK_PATH_CLUSTER   # longer than 64 KiB
     assert ak.ak_softmax_choose_path(16384, 128257, True) == ak.AK_PATH_GENERIC
     for rows, V in ((4096, 32000), (4096, 128256), (16384, 128256)):
         assert ak.ak_xent_choose_path(rows, V) == (ak.AK_XENT_ROW, 1)

@@ -31,7 +31,8 @@ def _free():
 
 
 @pytest.mark.parametrize("rows,D", [(8192, 1024), (8192, 2048), (8192, 4096), (8192, 8192),
-                                    (8192, 16384), (65536, 4096), (262144, 4096), (8192, 4099)])
+                                    (8192, 16384), (65536, 4096), (262144, 4096), (8192, 4099),
+                                    (4096, 65536), (2048, 128256), (16, 128256), (512, 262144)])
 def test_rmsnorm_full_size(rows, D):
     x, w = synth.rmsnorm_inputs(rows, D, synth.case_seed(2, D + rows), device=DEV)
     y = ak.ak_rmsnorm_fwd(x, w, eps=1e-6)
@@ -54,7 +55,8 @@ def test_rmsnorm_full_size(rows, D):
 
 
 @pytest.mark.parametrize("rows,D", [(16384, 512), (16384, 1024), (16384, 2048), (16384, 4096),
-                                    (16384, 8192), (16384, 32768), (262144, 4096), (4096, 4099)])
+                                    (16384, 8192), (16384, 32768), (262144, 4096), (4096, 4099),
+                                    (4096, 65536), (4096, 128256), (16, 128256), (1, 128256), (512, 262144)])
 def test_softmax_full_size(rows, D):
     x = synth.softmax_inputs(rows, D, synth.case_seed(3, D + rows), device=DEV)
     y = ak.ak_softmax_fwd(x)
@@ -102,7 +104,7 @@ def test_xent_full_size(rows, V):
 
 
 @pytest.mark.parametrize("rows,D", [(8192, 4096), (4096, 5120), (8192, 8192), (65536, 4096), (4096, 32768),
-                                    (8192, 4099)])
+                                    (8192, 4099), (4096, 65536), (2048, 128256), (16, 128256), (512, 262144)])
 def test_layernorm_full_size(rows, D):
     x, g, b = synth.layernorm_inputs(rows, D, synth.case_seed(6, D + rows), device=DEV)
     y = ak.ak_layernorm_fwd(x, g, b, eps=1e-5)

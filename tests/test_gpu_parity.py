@@ -363,3 +363,59 @@ def test_non_default_stream_and_launch_counter():
     s.synchronize()
     assert ak.ak_launch_count() == before + 1
     assert_bf16_close(y, ref, "non-default stream")
+
+
+@pytest.mark.parametrize("rows,D", [(1, 16), (3, 24), (5, 4104), (64, 16384), (65, 16384), (7, 131072), (2, 458752),
+                                    (1, 917504), (3, 128256), (9, 65544)])
+def test_cluster_path_slices_and_limits(rows, D):
+    """Rows split over a thread-block cluster: slices of unequal length (D / 8 not a multiple of
+    the cluster size), the shortest legal rows (two vectors), rows far beyond one CTA's shared
+    memory up to the 8 x 224 KiB limit, and both sides of the few-rows rule.  All three ops, forced
+    and as the dispatcher's own choice; -inf and identical-value rows included."""
+    x, w = synth.rmsnorm_inputs(rows, D, synth.case_seed(9, rows * 131 + D))
+    if rows > 1:
+        x[0, : D // 2] = float("-inf")      # whole slices of -inf (softmax); replaced by -3 for the norms
+    xs = x.clone()
+    xr = torch.nan_to_num(x, neginf=-3.0)
+    _, g, b = synth.layernorm_inputs(1, D, 77)
+    ref_r = oracle.rmsnorm(synth.to_bits(xr), synth.to_bits(w), 1e-6)
+    ref_s = oracle.softmax(synth.to_bits(xs))
+    ref_l = oracle.layernorm(synth.to_bits(xr), synth.to_bits(g), synth.to_bits(b), 1e-5)
+    for path in (CLUSTER, ak.AK_PATH_AUTO):
+        y, check = guarded((rows, D), torch.bfloat16, DEV)
+        ak.ak_rmsnorm_fwd(xr.to(DEV), w.to(DEV), y, eps=1e-6, path=path)
+        torch.cuda.synchronize()
+        check()
+        assert_bf16_close(y, ref_r, f"rmsnorm cluster {rows}x{D} path {path}")
+        y, check = guarded((rows, D), torch.bfloat16, DEV)
+        ak.ak_softmax_fwd(xs.to(DEV), y, path=path)
+        torch.cuda.synchronize()
+        check()
+        assert_bf16_close(y, ref_s, f"softmax cluster {rows}x{D} path {path}")
+        y, check = guarded((rows, D), torch.bfloat16, DEV)
+        ak.ak_layernorm_fwd(xr.to(DEV), g.to(DEV), b.to(DEV), y, eps=1e-5, path=path)
+        torch.cuda.synchronize()
+        check()
+        # z * gamma + beta may cancel, so only the benchmark's bar applies here (the one-rounding
+        # bound relative to |z * gamma| + |beta| is checked in the LayerNorm tests proper)
+        assert_bf16_close(y, ref_l, f"layernorm cluster {rows}x{D} path {path}", tight=False)
+    if D * 2 > 8 * 224 * 1024:
+        return
+    want = CLUSTER if (D * 2 > 65536 or (rows <= 64 and D * 2 >= 32768)) else None
+    if want is not None:
+        assert ak.ak_rmsnorm_choose_path(rows, D, True) == want
+        assert ak.ak_softmax_choose_path(rows, D, True) == want
+
+
+def test_cluster_path_rejects_rows_it_cannot_hold():
+    x = torch.zeros((1, 8), dtype=torch.bfloat16, device=DEV)           # one vector: nothing to split
+    w = torch.ones((8,), dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(ak.AkError):
+        ak.ak_rmsnorm_fwd(x, w, path=CLUSTER)
+    big = torch.zeros((1, 917512), dtype=torch.bfloat16, device=DEV)    # one vector beyond 8 x 224 KiB
+    with pytest.raises(ak.AkError):
+        ak.ak_softmax_fwd(big, path=CLUSTER)
+    y = ak.ak_softmax_fwd(big)                                          # the dispatcher falls back to the multi-pass kernel
+    torch.cuda.synchronize()
+    v = y.float()
+    assert bool((v == v[0, 0]).all()) and abs(float(v[0, 0]) * 917512 - 1.0) < 2.0 ** -8
