@@ -148,12 +148,16 @@ def test_two_streams_and_graph_replay():
     xr = synth.rope_inputs(16, 512, 128, 605, device=DEV, dtype=torch.float16)
     # unaligned rows, enough of them for the shifted-parameter table (scratch + dependent launch)
     xu, gu, bu = synth.layernorm_inputs(1500, 2051, 606, device=DEV)
+    # rows split over thread-block clusters (a few long rows; rows beyond one CTA's shared memory)
+    xc = synth.softmax_inputs(8, 131072, 609, device=DEV)
+    xk, wk = synth.rmsnorm_inputs(300, 128256, 610, device=DEV)
 
     def run_all(stream=None):
         loss, mean = ak.ak_xent_fwd(lg, tg, stream=stream)
         return [ak.ak_rmsnorm_fwd(x, w, stream=stream), ak.ak_softmax_fwd(xs, stream=stream), loss, mean,
                 ak.ak_layernorm_fwd(xl, g, b, stream=stream), ak.ak_rowsum_fwd(xl, stream=stream),
-                ak.ak_rope_fwd(xr, stream=stream), ak.ak_layernorm_fwd(xu, gu, bu, stream=stream)]
+                ak.ak_rope_fwd(xr, stream=stream), ak.ak_layernorm_fwd(xu, gu, bu, stream=stream),
+                ak.ak_softmax_fwd(xc, stream=stream), ak.ak_rmsnorm_fwd(xk, wk, stream=stream)]
 
     serial = [t.clone() for t in run_all()]
     torch.cuda.synchronize()
