@@ -72,6 +72,18 @@ rope_vec_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t n_se
     if (v >= nvs) return;
     const int64_t s = v / vpr;
     const int j = (int)(v - s * vpr);
+    int64_t n = (int64_t)blockIdx.y * seq_per_cta;
+    int64_t n_end = n + seq_per_cta;
+    if (n_end > n_seq) n_end = n_seq;
+    const uint4* xp = x + n * nvs + v;
+    uint4* yp = y + n * nvs + v;
+    // the first batch of loads is in flight while the sines and cosines are evaluated
+    uint4 q[UNROLL];
+    const bool full_first = n + UNROLL <= n_end;
+    if (full_first) {
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) q[u] = ld_stream(xp + u * nvs);
+    }
     const double pos = (double)(pos_offset + s);
     f32x2 cc[PPV], ns[PPV];
 #pragma unroll
@@ -81,13 +93,12 @@ rope_vec_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t n_se
         cc[k] = pack2(c, c);
         ns[k] = pack2(-sn, sn);
     }
-    int64_t n = (int64_t)blockIdx.y * seq_per_cta;
-    int64_t n_end = n + seq_per_cta;
-    if (n_end > n_seq) n_end = n_seq;
-    const uint4* xp = x + n * nvs + v;
-    uint4* yp = y + n * nvs + v;
+    if (full_first) {
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) st_stream(yp + u * nvs, rotate_vec<DT>(q[u], cc, ns));
+        n += UNROLL, xp += UNROLL * nvs, yp += UNROLL * nvs;
+    }
     for (; n + UNROLL <= n_end; n += UNROLL, xp += UNROLL * nvs, yp += UNROLL * nvs) {
-        uint4 q[UNROLL];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) q[u] = ld_stream(xp + u * nvs);
 #pragma unroll
@@ -130,11 +141,12 @@ rope_pair_kernel(const void* __restrict__ xv, void* __restrict__ yv, int64_t n_s
 }
 
 // Sequences are cut into chunks (grid.y) so that the grid fills the GPU (about 32 CTAs of 128
-// threads per SM in total), but a chunk keeps at least sixteen sequences where it can, so the
-// trigonometry stays amortised.  (Timed on B200 for 296 .. 4736 CTAs and 4 / 16 sequences:
-// within 10 % of each other; this choice was best or tied on every shape.)
+// threads per SM in total), but a chunk keeps at least eight sequences where it can (one full
+// batch of loads, in flight while the trigonometry runs), so the trigonometry stays amortised.
+// (Timed on B200 for 296 .. 4736 CTAs and 4 / 8 / 16 sequences: within 10 % of each other; this
+// choice was best or tied on every shape.)
 void chunking(int64_t gx, int64_t n_seq, int* seq_per_cta, unsigned* gy) {
-    constexpr int64_t target = 148 * 32, minseq = 16;
+    constexpr int64_t target = 148 * 32, minseq = 8;
     int64_t want = (target + gx - 1) / gx;
     int64_t most = n_seq / minseq > 1 ? n_seq / minseq : 1;
     if (want > most) want = most;
