@@ -2,8 +2,9 @@
 //
 // Same dispatch structure as RMSNorm (the op moves the same bytes: one read of x, one write
 // of y, gamma and beta from L1/L2): a warp (or two) per row for short rows, a CTA per row with
-// the row in registers up to 32 KiB, the row staged in shared memory by bulk copies beyond,
-// and the phase kernels for rows that are not 16-byte aligned.  Thresholds are in row bytes,
+// the row in registers up to 64 KiB, longer rows (and a few long rows) split over a thread-block
+// cluster whose CTAs stage their slices in shared memory by bulk copies, and the phase kernels
+// for rows that are not 16-byte aligned.  Thresholds are in row bytes,
 // so they hold for every element type.
 #include "layernorm_kernels.cuh"
 

@@ -4,8 +4,9 @@
 // threads per CTA, threads per row, vectors per thread and register caps): what decides
 // the bandwidth is how many bytes each SM keeps in flight, i.e. resident CTAs x bytes per
 // CTA, so weights are fetched late (fewer live registers, more CTAs), one row (or one row
-// per warp) per CTA beats grid-stride persistence, and rows beyond 32 KiB are staged in
-// shared memory by the copy engine instead of registers.
+// per warp) per CTA beats grid-stride persistence, and rows beyond 64 KiB are split over a
+// thread-block cluster whose CTAs stage slices of at most 32 KiB in shared memory by the copy
+// engine (as are a few long rows, which one CTA each would not spread over the GPU).
 #include "rmsnorm_kernels.cuh"
 
 namespace ak {

@@ -3,8 +3,9 @@
 // Launch shapes come from CUDA-graph timed sweeps on B200 (see rmsnorm.cu for the
 // reasoning): one row per warp up to 4 KiB rows, one row per CTA in registers up to
 // 16 KiB rows (exponentials kept in fp32, register cap chosen for five CTAs per SM), rows
-// beyond that staged in shared memory by the copy engine.  The thresholds are in row bytes,
-// so they hold for every element type.
+// up to 64 KiB staged in shared memory by the copy engine, longer rows (and a few long rows)
+// split over a thread-block cluster.  The thresholds are in row bytes, so they hold for every
+// element type.
 #include "softmax_kernels.cuh"
 
 namespace ak {
