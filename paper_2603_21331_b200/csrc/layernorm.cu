@@ -11,12 +11,18 @@
 namespace ak {
 namespace {
 
-template <int DT, int THREADS, int GROUP, int VPT, int MINB>
+// A launch of at most this many rows and bytes does not fill the GPU and is latency-bound: gamma
+// and beta are then requested together with the row instead of after the reductions, without a
+// register cap (1 x 1024 .. 512 x 4096: 5-32 % faster, e.g. 8 x 8192 4.3 -> 3.0 us; beyond 4 MiB
+// the uncapped registers cost occupancy: 1024 x 8192 8.1 -> 13.3 us, so those keep the late fetch).
+constexpr int64_t kEarlyParamRows = 1024, kEarlyParamBytes = 4 << 20;
+
+template <int DT, int THREADS, int GROUP, int VPT, int MINB, bool PE = false>
 int launch_reg(const void* x, const void* g, const void* b, void* y, int64_t rows, int nvec, float inv_D,
                float eps, cudaStream_t st) {
     constexpr int GROUPS = THREADS / GROUP;
     const int64_t grid = (rows + GROUPS - 1) / GROUPS;
-    layernorm_reg_kernel<THREADS, GROUP, VPT, MINB, DT><<<(unsigned)grid, THREADS, 0, st>>>(
+    layernorm_reg_kernel<THREADS, GROUP, VPT, MINB, DT, PE><<<(unsigned)grid, THREADS, 0, st>>>(
         static_cast<const uint4*>(x), static_cast<const uint4*>(g), static_cast<const uint4*>(b),
         static_cast<uint4*>(y), rows, nvec, inv_D, eps);
     count_launch();
@@ -25,18 +31,18 @@ int launch_reg(const void* x, const void* g, const void* b, void* y, int64_t row
 
 // vectors per thread 1..8 for a fixed (THREADS, GROUP); the minimum-CTAs-per-SM hint (a register
 // cap) is given per vector count: M14 for 1..4 vectors, M56 for 5..6, M7 and M8 for 7 and 8
-template <int DT, int THREADS, int GROUP, int M14, int M56, int M7, int M8>
+template <int DT, int THREADS, int GROUP, int M14, int M56, int M7, int M8, bool PE = false>
 int launch_reg_vpt(int vpt, const void* x, const void* g, const void* b, void* y, int64_t rows, int nvec,
                    float inv_D, float eps, cudaStream_t st) {
     switch (vpt) {
-        case 1: return launch_reg<DT, THREADS, GROUP, 1, M14>(x, g, b, y, rows, nvec, inv_D, eps, st);
-        case 2: return launch_reg<DT, THREADS, GROUP, 2, M14>(x, g, b, y, rows, nvec, inv_D, eps, st);
-        case 3: return launch_reg<DT, THREADS, GROUP, 3, M14>(x, g, b, y, rows, nvec, inv_D, eps, st);
-        case 4: return launch_reg<DT, THREADS, GROUP, 4, M14>(x, g, b, y, rows, nvec, inv_D, eps, st);
-        case 5: return launch_reg<DT, THREADS, GROUP, 5, M56>(x, g, b, y, rows, nvec, inv_D, eps, st);
-        case 6: return launch_reg<DT, THREADS, GROUP, 6, M56>(x, g, b, y, rows, nvec, inv_D, eps, st);
-        case 7: return launch_reg<DT, THREADS, GROUP, 7, M7>(x, g, b, y, rows, nvec, inv_D, eps, st);
-        case 8: return launch_reg<DT, THREADS, GROUP, 8, M8>(x, g, b, y, rows, nvec, inv_D, eps, st);
+        case 1: return launch_reg<DT, THREADS, GROUP, 1, M14, PE>(x, g, b, y, rows, nvec, inv_D, eps, st);
+        case 2: return launch_reg<DT, THREADS, GROUP, 2, M14, PE>(x, g, b, y, rows, nvec, inv_D, eps, st);
+        case 3: return launch_reg<DT, THREADS, GROUP, 3, M14, PE>(x, g, b, y, rows, nvec, inv_D, eps, st);
+        case 4: return launch_reg<DT, THREADS, GROUP, 4, M14, PE>(x, g, b, y, rows, nvec, inv_D, eps, st);
+        case 5: return launch_reg<DT, THREADS, GROUP, 5, M56, PE>(x, g, b, y, rows, nvec, inv_D, eps, st);
+        case 6: return launch_reg<DT, THREADS, GROUP, 6, M56, PE>(x, g, b, y, rows, nvec, inv_D, eps, st);
+        case 7: return launch_reg<DT, THREADS, GROUP, 7, M7, PE>(x, g, b, y, rows, nvec, inv_D, eps, st);
+        case 8: return launch_reg<DT, THREADS, GROUP, 8, M8, PE>(x, g, b, y, rows, nvec, inv_D, eps, st);
         default: return AK_ERR_SHAPE;
     }
 }
@@ -184,12 +190,20 @@ int dispatch_t(const void* x, const void* gamma, const void* beta, void* y, int6
         // sustained (power-capped) regime of a long run.
         case AK_PATH_WARP:
             if (row_bytes > 4096) return AK_ERR_SHAPE;
+            if (rows <= kEarlyParamRows && rows * row_bytes <= kEarlyParamBytes) {
+                if (nvec <= 128) return launch_reg_vpt<DT, 256, 32, 1, 1, 1, 1, true>((nvec + 31) / 32, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
+                return launch_reg_vpt<DT, 256, 64, 1, 1, 1, 1, true>((nvec + 63) / 64, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
+            }
             if (nvec <= 128)   // a warp per row, 8 rows per CTA, 46 registers
                 return launch_reg_vpt<DT, 256, 32, 5, 1, 1, 1>((nvec + 31) / 32, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
             // two warps per row, 4 rows per CTA
             return launch_reg_vpt<DT, 256, 64, 5, 1, 1, 1>((nvec + 63) / 64, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
         case AK_PATH_CTA:
             if (row_bytes > 65536) return AK_ERR_SHAPE;
+            if (rows <= kEarlyParamRows && rows * row_bytes <= kEarlyParamBytes) {
+                if (nvec <= 1024) return launch_reg_vpt<DT, 128, 128, 1, 1, 1, 1, true>((nvec + 127) / 128, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
+                if (nvec <= 2048) return launch_reg_vpt<DT, 256, 256, 1, 1, 1, 1, true>((nvec + 255) / 256, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
+            }
             if (nvec <= 1024)  // 128 threads x up to 8 vectors: many small CTAs per SM
                 return launch_reg_vpt<DT, 128, 128, 10, 8, 6, 8>((nvec + 127) / 128, x, gamma, beta, y, rows, nvec, inv_D, eps, st);
             if (nvec <= 2048)

@@ -109,7 +109,9 @@ __device__ __forceinline__ float first_elem(const void* row) {
 // Same thread layout as the RMSNorm register kernel (a group of GROUP threads owns a row,
 // thread t holds vectors t, t + GROUP, ...), two reductions per row.  Padding slots hold
 // copies of K so they add exactly zero to the first sum and are excluded from the second.
-template <int THREADS, int GROUP, int VPT, int MINB, int DT = AK_DTYPE_BF16>
+// P_EARLY: gamma and beta are requested together with the row instead of after the reductions
+// (8 * VPT more live registers; for launches too small to fill the GPU, where latency counts).
+template <int THREADS, int GROUP, int VPT, int MINB, int DT = AK_DTYPE_BF16, bool P_EARLY = false>
 __global__ void __launch_bounds__(THREADS, MINB)
 layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamma, const uint4* __restrict__ beta,
                      uint4* __restrict__ y, int64_t rows, int nvec, float inv_D, float eps) {
@@ -122,6 +124,17 @@ layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamm
     const int lane = threadIdx.x & 31;
     const int warp_in_group = t >> 5;
 
+    uint4 gv[P_EARLY ? VPT : 1], bv[P_EARLY ? VPT : 1];
+    if constexpr (P_EARLY) {
+#pragma unroll
+        for (int k = 0; k < VPT; ++k) {
+            const int i = t + k * GROUP;
+            if (i < nvec) {
+                gv[k] = __ldg(gamma + i);
+                bv[k] = __ldg(beta + i);
+            }
+        }
+    }
     for (int64_t row0 = (int64_t)blockIdx.x * GROUPS; row0 < rows; row0 += (int64_t)gridDim.x * GROUPS) {
         const int64_t row = row0 + g;
         const bool live = row < rows;
@@ -161,7 +174,10 @@ layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamm
 #pragma unroll
         for (int k = 0; k < VPT; ++k) {
             const int i = t + k * GROUP;
-            if (live && i < nvec) st_stream(yr + i, ln_out_v<DT>(xv[k], __ldg(gamma + i), __ldg(beta + i), mu, rstd));
+            if (live && i < nvec) {
+                if constexpr (P_EARLY) st_stream(yr + i, ln_out_v<DT>(xv[k], gv[k], bv[k], mu, rstd));
+                else st_stream(yr + i, ln_out_v<DT>(xv[k], __ldg(gamma + i), __ldg(beta + i), mu, rstd));
+            }
         }
     }
 }

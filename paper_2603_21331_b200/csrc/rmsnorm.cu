@@ -12,30 +12,36 @@
 namespace ak {
 namespace {
 
-template <int DT, int THREADS, int GROUP, int VPT, int MINB>
+// A launch of at most this many rows and bytes does not fill the GPU and is latency-bound: the
+// weights are then requested together with the row instead of after the reduction (no register
+// cap to keep: 1 x 1024 .. 1024 x 4096 run 5-47 % faster, e.g. 8 x 2048 3.2 -> 1.7 us; from 2048
+// rows or 8 MiB on the late fetch with its tighter register budget is as fast or faster).
+constexpr int64_t kEarlyWeightRows = 1024, kEarlyWeightBytes = 8 << 20;
+
+template <int DT, int THREADS, int GROUP, int VPT, int MINB, bool WE = false>
 int launch_reg(const void* x, const void* w, void* y, int64_t rows, int nvec, float inv_D, float eps,
                cudaStream_t st) {
     constexpr int GROUPS = THREADS / GROUP;
     const int64_t grid = (rows + GROUPS - 1) / GROUPS;
-    rmsnorm_reg_kernel<THREADS, GROUP, VPT, MINB, false, DT><<<(unsigned)grid, THREADS, 0, st>>>(
+    rmsnorm_reg_kernel<THREADS, GROUP, VPT, MINB, WE, DT><<<(unsigned)grid, THREADS, 0, st>>>(
         static_cast<const uint4*>(x), static_cast<const uint4*>(w), static_cast<uint4*>(y), rows, nvec, inv_D, eps);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
 // vectors per thread 1..MAXV for a fixed (THREADS, GROUP)
-template <int DT, int THREADS, int GROUP, int MINB_LO, int MINB_HI>
+template <int DT, int THREADS, int GROUP, int MINB_LO, int MINB_HI, bool WE = false>
 int launch_reg_vpt(int vpt, const void* x, const void* w, void* y, int64_t rows, int nvec, float inv_D,
                    float eps, cudaStream_t st) {
     switch (vpt) {
-        case 1: return launch_reg<DT, THREADS, GROUP, 1, MINB_LO>(x, w, y, rows, nvec, inv_D, eps, st);
-        case 2: return launch_reg<DT, THREADS, GROUP, 2, MINB_LO>(x, w, y, rows, nvec, inv_D, eps, st);
-        case 3: return launch_reg<DT, THREADS, GROUP, 3, MINB_LO>(x, w, y, rows, nvec, inv_D, eps, st);
-        case 4: return launch_reg<DT, THREADS, GROUP, 4, MINB_LO>(x, w, y, rows, nvec, inv_D, eps, st);
-        case 5: return launch_reg<DT, THREADS, GROUP, 5, MINB_HI>(x, w, y, rows, nvec, inv_D, eps, st);
-        case 6: return launch_reg<DT, THREADS, GROUP, 6, MINB_HI>(x, w, y, rows, nvec, inv_D, eps, st);
-        case 7: return launch_reg<DT, THREADS, GROUP, 7, MINB_HI>(x, w, y, rows, nvec, inv_D, eps, st);
-        case 8: return launch_reg<DT, THREADS, GROUP, 8, MINB_HI>(x, w, y, rows, nvec, inv_D, eps, st);
+        case 1: return launch_reg<DT, THREADS, GROUP, 1, MINB_LO, WE>(x, w, y, rows, nvec, inv_D, eps, st);
+        case 2: return launch_reg<DT, THREADS, GROUP, 2, MINB_LO, WE>(x, w, y, rows, nvec, inv_D, eps, st);
+        case 3: return launch_reg<DT, THREADS, GROUP, 3, MINB_LO, WE>(x, w, y, rows, nvec, inv_D, eps, st);
+        case 4: return launch_reg<DT, THREADS, GROUP, 4, MINB_LO, WE>(x, w, y, rows, nvec, inv_D, eps, st);
+        case 5: return launch_reg<DT, THREADS, GROUP, 5, MINB_HI, WE>(x, w, y, rows, nvec, inv_D, eps, st);
+        case 6: return launch_reg<DT, THREADS, GROUP, 6, MINB_HI, WE>(x, w, y, rows, nvec, inv_D, eps, st);
+        case 7: return launch_reg<DT, THREADS, GROUP, 7, MINB_HI, WE>(x, w, y, rows, nvec, inv_D, eps, st);
+        case 8: return launch_reg<DT, THREADS, GROUP, 8, MINB_HI, WE>(x, w, y, rows, nvec, inv_D, eps, st);
         default: return AK_ERR_SHAPE;
     }
 }
@@ -126,6 +132,10 @@ int dispatch_t(const void* x, const void* w, void* y, int64_t rows, int64_t D, f
     switch (path) {
         case AK_PATH_WARP:
             if (row_bytes > 4096) return AK_ERR_SHAPE;
+            if (rows <= kEarlyWeightRows && rows * row_bytes <= kEarlyWeightBytes) {
+                if (nvec <= 128) return launch_reg_vpt<DT, 256, 32, 4, 1, true>((nvec + 31) / 32, x, w, y, rows, nvec, inv_D, eps, st);
+                return launch_reg_vpt<DT, 128, 32, 1, 1, true>((nvec + 31) / 32, x, w, y, rows, nvec, inv_D, eps, st);
+            }
             if (nvec <= 128) return launch_reg_vpt<DT, 256, 32, 4, 1>((nvec + 31) / 32, x, w, y, rows, nvec, inv_D, eps, st);
             return launch_reg_vpt<DT, 128, 32, 1, 1>((nvec + 31) / 32, x, w, y, rows, nvec, inv_D, eps, st);
         case AK_PATH_CTA:
@@ -135,6 +145,10 @@ int dispatch_t(const void* x, const void* w, void* y, int64_t rows, int64_t D, f
             // 256 threads x <= 8 vectors capped at 85 registers (62 used); 512 threads x <= 8 vectors
             // capped at 64 registers so that two CTAs share an SM (6.5 TB/s at 64 KiB rows against 6.2
             // for the shared-memory kernel).
+            if (rows <= kEarlyWeightRows && rows * row_bytes <= kEarlyWeightBytes) {
+                if (nvec <= 512) return launch_reg_vpt<DT, 128, 128, 1, 1, true>((nvec + 127) / 128, x, w, y, rows, nvec, inv_D, eps, st);
+                if (nvec <= 2048) return launch_reg_vpt<DT, 256, 256, 1, 1, true>((nvec + 255) / 256, x, w, y, rows, nvec, inv_D, eps, st);
+            }
             if (nvec <= 512) return launch_reg_vpt<DT, 128, 128, 1, 1>((nvec + 127) / 128, x, w, y, rows, nvec, inv_D, eps, st);
             if (nvec <= 2048) return launch_reg_vpt<DT, 256, 256, 1, 3>((nvec + 255) / 256, x, w, y, rows, nvec, inv_D, eps, st);
             return launch_reg_vpt<DT, 512, 512, 2, 2>((nvec + 511) / 512, x, w, y, rows, nvec, inv_D, eps, st);

@@ -419,3 +419,22 @@ def test_cluster_path_rejects_rows_it_cannot_hold():
     torch.cuda.synchronize()
     v = y.float()
     assert bool((v == v[0, 0]).all()) and abs(float(v[0, 0]) * 917512 - 1.0) < 2.0 ** -8
+
+
+@pytest.mark.parametrize("D", [1024, 2048, 4096, 8192])
+def test_small_launches_fetch_parameters_early_with_the_same_bits(D):
+    """Launches too small to fill the GPU request w (gamma, beta) together with the row instead of
+    after the reductions; that changes when the loads are issued, not the arithmetic: the rows a
+    small and a large launch share come out bit for bit the same."""
+    big, small = 3000, 24
+    x, w = synth.rmsnorm_inputs(big, D, synth.case_seed(11, D), device=DEV)
+    _, g, b = synth.layernorm_inputs(1, D, 78, device=DEV)
+    y_big = ak.ak_rmsnorm_fwd(x, w)
+    y_small = ak.ak_rmsnorm_fwd(x[:small].contiguous(), w)
+    l_big = ak.ak_layernorm_fwd(x, g, b)
+    l_small = ak.ak_layernorm_fwd(x[:small].contiguous(), g, b)
+    torch.cuda.synchronize()
+    assert torch.equal(y_big[:small].view(torch.int16), y_small.view(torch.int16))
+    assert torch.equal(l_big[:small].view(torch.int16), l_small.view(torch.int16))
+    ref = oracle.rmsnorm(synth.to_bits(x[:small].cpu()), synth.to_bits(w.cpu()), 1e-6)
+    assert_bf16_close(y_small, ref, f"rmsnorm {small}x{D} (early weights)")
