@@ -712,7 +712,9 @@ def sweep_accuracy(ak, synth, op, rows, D, bufs):
 # reduce 16384 x 4096, rotary 2 x 32 x 2k x 128 in FP16), an FP16 variant, and the vocabulary-parallel
 # cross-entropy as one of eight ranks runs it: timed briefly in every default run ("widened_rows").
 WIDENED = [("layernorm", 8192, 4096), ("rowsum", 16384, 4096), ("rope.f16", 64 * 2048, 128),
-           ("rmsnorm.f16", 8192, 8192), ("xent_vp8", 4096, 128256 // 8)]
+           ("rmsnorm.f16", 8192, 8192), ("xent_vp8", 4096, 128256 // 8),
+           # rows split over thread-block clusters: a vocabulary-sized softmax, training- and decoding-sized
+           ("softmax", 4096, 128256), ("softmax", 16, 128256)]
 
 
 def run_sweep(ak, synth, dev, peak, shapes=None, iters=200, write=True, accuracy=True):
