@@ -56,6 +56,7 @@ xent_vp_partial_kernel(const typename XElem<DT>::type* __restrict__ logits, cons
 // One thread per row: all ranks' slices in (rank, slice) order, exactly the arithmetic of the
 // single-GPU split merge.  parts = [nranks][rows][nsplit + 1] pairs.
 constexpr int kVpMergeThreads = 128;
+constexpr int kVpBatch = 16;   // pairs (and ranks) per row held in registers by the merge
 __global__ void __launch_bounds__(kVpMergeThreads)
 xent_vp_merge_kernel(const float2* __restrict__ parts, int nranks, int nsplit, const int64_t* __restrict__ targets,
                      int64_t ignore_index, int64_t V_total, float* __restrict__ loss_rows, int64_t rows) {
@@ -70,18 +71,41 @@ xent_vp_merge_kernel(const float2* __restrict__ parts, int nranks, int nsplit, c
     } else {
         const int64_t stride = (int64_t)rows * (nsplit + 1);
         const float2* pr = parts + r * (nsplit + 1);
-        float M = -INFINITY;
-        for (int k = 0; k < nranks; ++k)
-            for (int i = 0; i < nsplit; ++i) M = fmaxf(M, __ldg(pr + k * stride + i).x);
-        const float MF = fmaxf(M * kLog2e, kFloor2);
-        float S = 0.0f, xt = 0.0f, owners = 0.0f;
-        for (int k = 0; k < nranks; ++k) {
-            for (int i = 0; i < nsplit; ++i) {
-                const float2 ps = __ldg(pr + k * stride + i);
-                S += ps.y * fast_exp2(fmaxf(ps.x * kLog2e, kFloor2) - MF);
+        float M = -INFINITY, S = 0.0f, xt = 0.0f, owners = 0.0f;
+        const int n = nranks * nsplit;
+        if (n <= kVpBatch && nranks <= kVpBatch) {
+            // the usual case (up to 16 pairs per row): every load of the row is issued before the
+            // first use, so the thread waits for memory once, not once per pair; same order of
+            // the arithmetic as the loops below
+            float2 p[kVpBatch], own[kVpBatch];
+#pragma unroll
+            for (int q = 0; q < kVpBatch; ++q) {
+                const int k = q / nsplit, i = q - k * nsplit;
+                if (q < n) p[q] = __ldg(pr + k * stride + i);
+                if (q < nranks) own[q] = __ldg(pr + q * stride + nsplit);
             }
-            const float2 own = __ldg(pr + k * stride + nsplit);
-            if (own.y != 0.0f) { xt = own.x; owners += 1.0f; }
+#pragma unroll
+            for (int q = 0; q < kVpBatch; ++q)
+                if (q < n) M = fmaxf(M, p[q].x);
+            const float MF = fmaxf(M * kLog2e, kFloor2);
+#pragma unroll
+            for (int q = 0; q < kVpBatch; ++q)
+                if (q < n) S += p[q].y * fast_exp2(fmaxf(p[q].x * kLog2e, kFloor2) - MF);
+#pragma unroll
+            for (int q = 0; q < kVpBatch; ++q)
+                if (q < nranks && own[q].y != 0.0f) { xt = own[q].x; owners += 1.0f; }
+        } else {
+            for (int k = 0; k < nranks; ++k)
+                for (int i = 0; i < nsplit; ++i) M = fmaxf(M, __ldg(pr + k * stride + i).x);
+            const float MF = fmaxf(M * kLog2e, kFloor2);
+            for (int k = 0; k < nranks; ++k) {
+                for (int i = 0; i < nsplit; ++i) {
+                    const float2 ps = __ldg(pr + k * stride + i);
+                    S += ps.y * fast_exp2(fmaxf(ps.x * kLog2e, kFloor2) - MF);
+                }
+                const float2 own = __ldg(pr + k * stride + nsplit);
+                if (own.y != 0.0f) { xt = own.x; owners += 1.0f; }
+            }
         }
         // exactly one shard owns a valid target when the shards tile [0, V_total)
         loss = (owners == 1.0f) ? finish_loss(M, S, xt) : __int_as_float(0x7fc00000);
