@@ -86,7 +86,7 @@ def test_validation_rejects_before_any_cuda_call():
     # vocabulary-parallel cross-entropy
     assert l.ak_xent_vp_partial_bytes(10, 3) == 10 * 4 * 8 and l.ak_xent_vp_partial_bytes(0, 3) == 0
     assert l.ak_xent_vp_nsplit(4096, 16032) == 1 and l.ak_xent_vp_nsplit(16, 16032) == 1
-    assert l.ak_xent_vp_nsplit(16, 64128) == 7
+    assert l.ak_xent_vp_nsplit(16, 64128) == 4                  # slices of at most 16384 elements
     assert l.ak_xent_vp_partial(None, P, -100, 0, 64, P, 1, 32, 1, 0, None) == 1
     assert l.ak_xent_vp_partial(P, P, -100, 40, 64, P, 1, 32, 1, 0, None) == 2   # shard sticks out of the vocabulary
     assert l.ak_xent_vp_partial(P, P, -100, 0, 64, P, 1, 0, 1, 0, None) == 2     # empty shard
@@ -150,7 +150,7 @@ def test_dispatch_is_a_pure_function_of_shape_and_alignment():
     path, ns = ak.ak_xent_choose_path(16, 128256)
     assert path == ak.AK_XENT_SPLIT and 2 <= ns <= 64
     assert ak.ak_xent_workspace_bytes(16, 128256) == 16 * ns * 8
-    assert ak.ak_xent_choose_path(1, 128256)[1] == 15            # capped by 8192-element slices
+    assert ak.ak_xent_choose_path(1, 128256)[1] == 8             # slices of at most 16384 elements
     assert ak.ak_xent_choose_path(16, 1000) == (ak.AK_XENT_ROW, 1)  # short rows never split
     # repeated queries agree (no hidden state)
     assert all(ak.ak_xent_choose_path(16, 128256) == (path, ns) for _ in range(3))
