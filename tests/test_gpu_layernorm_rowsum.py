@@ -158,7 +158,7 @@ def test_layernorm_unaligned_rows_with_the_shift_table(rows, D, xo, few):
 
 def test_layernorm_in_place_and_empty():
     for D, paths in ((512, _legal_paths(512)), (4096, _legal_paths(4096)), (4099, _legal_paths(4099)),
-                     (16384, _legal_paths(16384))):
+                     (16384, _legal_paths(16384)), (131072, _legal_paths(131072))):
         x, g, b = synth.layernorm_inputs(11, D, 194)
         xb, gb, bb = synth.to_bits(x), synth.to_bits(g), synth.to_bits(b)
         ref = oracle.layernorm(xb, gb, bb, EPS)

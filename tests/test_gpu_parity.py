@@ -262,7 +262,8 @@ def test_misaligned_base_pointers_take_generic_path():
 
 
 def test_in_place_is_allowed():
-    for D, paths in ((512, (WARP, CTA, GEN, SMEM)), (4096, (CTA, GEN, SMEM)), (4099, (GEN,)), (16384, (CTA, SMEM))):
+    for D, paths in ((512, (WARP, CTA, GEN, SMEM, CLUSTER)), (4096, (CTA, GEN, SMEM, CLUSTER)), (4099, (GEN,)),
+                     (16384, (CTA, SMEM, CLUSTER)), (131072, (CLUSTER,))):
         x, w = synth.rmsnorm_inputs(11, D, 94)
         ref = oracle.rmsnorm(synth.to_bits(x), synth.to_bits(w), 1e-6)
         xs = synth.softmax_inputs(11, D, 95)
