@@ -20,8 +20,13 @@ def _cases(seed, n):
     out = []
     for i in range(n):
         rows = int(rng.integers(1, 24))
-        kind = i % 4
-        if kind == 0:
+        kind = i % 5
+        if kind == 4:
+            # long rows: split over thread-block clusters when 16-byte aligned (up to 8 CTAs' shared
+            # memory), staged or multi-pass when not
+            rows = int(rng.integers(1, 5))
+            D = 8 * int(rng.integers(2048, 40000)) + int(rng.choice([0, 0, 0, 0, 1, -1, 4]))
+        elif kind == 0:
             D = int(rng.integers(1, 65))
         elif kind == 1:
             D = int(rng.integers(65, 2100))
