@@ -499,7 +499,7 @@ SWEEP = list(
     + [("rmsnorm", r, 4096) for r in (1, 17, 65536, 262144)] + [("rmsnorm", 8192, 4099), ("rmsnorm", 8192, 8190), ("rmsnorm", 4096, 65536), ("rmsnorm", 16, 128256)]
     + [("softmax", 16384, d) for d in (512, 1024, 2048, 4096, 8192, 32768)]
     + [("softmax", 262144, 4096), ("softmax", 16384, 4099), ("softmax", 4096, 65536), ("softmax", 4096, 128256),
-       ("softmax", 16, 128256), ("softmax", 1, 128256)]
+       ("softmax", 16, 128256), ("softmax", 1, 128256), ("softmax", 4096, 128257)]
     + [("xent", 4096, v) for v in (32000, 50304, 128256, 128257)] + [("xent", 16384, 128256), ("xent", 16, 128256)]
     + [("layernorm", 8192, 4096), ("layernorm", 4096, 5120), ("layernorm", 8192, 8192), ("layernorm", 65536, 4096),
        ("layernorm", 4096, 32768), ("layernorm", 8192, 4099), ("layernorm", 8192, 8190),

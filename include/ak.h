@@ -65,7 +65,7 @@ enum {
      * need 16-byte aligned pointers and rows that are a multiple of 16 bytes. */
     AK_PATH_WARP = 1,     /* one (or two) warps per row, row held in registers; rows <= 4 KiB (bf16 D <= 2048) */
     AK_PATH_CTA = 2,      /* one CTA per row, row held in registers; rows <= 64 KiB (bf16 D <= 32768) */
-    AK_PATH_GENERIC = 3,  /* any D, any element alignment; row staged in shared memory in its 16-byte phase or re-read from L1/L2, single DRAM pass */
+    AK_PATH_GENERIC = 3,  /* any D, any element alignment; the row is kept in registers or staged in shared memory (of one CTA, or of a cluster of up to eight for rows beyond 224 KiB and for a few long rows) in its 16-byte phase: a single DRAM pass; else re-read from L1/L2 */
     AK_PATH_SMEM = 4,     /* one CTA per row, row staged in shared memory by bulk (TMA) copies; rows <= 224 KiB (bf16 D <= 114688) */
     AK_PATH_CLUSTER = 5   /* a thread-block cluster of 2, 4 or 8 CTAs per row, each staging a slice in its shared memory, partial results exchanged through distributed shared memory; rows of 32 bytes .. 1792 KiB (bf16 D <= 917504).  The dispatcher takes it for aligned rows longer than 64 KiB, in slices of at most 32 KiB where eight CTAs can do that, and for at most 64 rows of 32 KiB or more (eight CTAs each); longer aligned rows than 1792 KiB take AK_PATH_GENERIC */
 };
@@ -177,7 +177,7 @@ int ak_choose_path_dt(int op, int64_t rows, int64_t D, int aligned16, int dtype)
  * Same path ids, size limits and alignment rules as RMSNorm (gamma and beta together play
  * the part of w).  Status codes as for RMSNorm.  One launch and no scratch, except for many
  * rows that are not 16-byte aligned (1024 or more of D <= about 32750, 256 or more longer ones
- * that fit in shared memory): then a small kernel first writes gamma and beta in all eight 2-byte shifts to
+ * up to 1792 KiB): then a small kernel first writes gamma and beta in all eight 2-byte shifts to
  * about 32 * D bytes of stream-ordered scratch obtained and released on `cuda_stream`, and
  * the row kernel runs as its programmatic dependent; if the scratch cannot be had the
  * single-launch kernel runs instead (same results).

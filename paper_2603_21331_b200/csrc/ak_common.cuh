@@ -425,6 +425,27 @@ inline cudaError_t launch_cluster(void (*kernel)(KArgs...), unsigned grid, unsig
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// Both: clusters of C CTAs, launched as a programmatic dependent of the work before it.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_cluster_dependent(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, int C,
+                                            cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)C;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // Launch `kernel` as a programmatic dependent of the work before it in the stream.
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,

@@ -130,6 +130,33 @@ int launch_stage(const uint16_t* x, const uint16_t* g, const uint16_t* b, uint16
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
+// unaligned rows split over a cluster of C CTAs (covering vectors of the worst phase: max_nv);
+// gamma and beta from the shift table from kShiftMinRowsStaged rows on
+template <int DT, int T>
+int launch_cluster_stage(const uint16_t* x, const uint16_t* g, const uint16_t* b, uint16_t* y, int64_t rows, int64_t D,
+                         int64_t max_nv, int C, float inv_D, float eps, cudaStream_t st) {
+    static const bool configured = [] {
+        return cudaFuncSetAttribute(layernorm_cluster_stage_kernel<T, DT, false>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxRowSmemBytes) == cudaSuccess &&
+               cudaFuncSetAttribute(layernorm_cluster_stage_kernel<T, DT, true>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxRowSmemBytes) == cudaSuccess;
+    }();
+    if (!configured) return AK_ERR_CUDA;
+    const size_t smem = (size_t)((max_nv + C - 1) / C) * 16;
+    int nvp = 0;
+    if (const uint4* tab = shift_table(g, b, rows, D, kShiftMinRowsStaged, st, &nvp)) {
+        const cudaError_t e = launch_cluster_dependent(layernorm_cluster_stage_kernel<T, DT, true>, (unsigned)(rows * C), T,
+                                                       smem, C, st, x, g, b, y, D, C, inv_D, eps, tab, nvp);
+        count_launch();
+        cudaFreeAsync(const_cast<uint4*>(tab), st);
+        return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+    }
+    const cudaError_t e = launch_cluster(layernorm_cluster_stage_kernel<T, DT, false>, (unsigned)(rows * C), T, smem, C, st,
+                                         x, g, b, y, D, C, inv_D, eps, static_cast<const uint4*>(nullptr), 0);
+    count_launch();
+    return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+}
+
 template <int DT, int THREADS, int VPT, int MINB>
 int launch_regp(const uint16_t* x, const uint16_t* g, const uint16_t* b, uint16_t* y, int64_t rows, int64_t D,
                 float inv_D, float eps, cudaStream_t st) {
@@ -240,6 +267,11 @@ int dispatch_t(const void* x, const void* gamma, const void* beta, void* y, int6
                 uint16_t* ys = static_cast<uint16_t*>(y);
                 // rows of up to 1024 covering vectors stay in the registers of a 128-thread CTA ...
                 const int64_t max_nv = (D + 14) >> 3;   // vectors covering the row at the worst phase
+                // rows beyond one CTA's shared memory (up to eight CTAs'), and a few long rows (at most
+                // 64 of 32 KiB or more): the covering vectors split over a thread-block cluster
+                const int Cu = cluster_ctas(rows, (int64_t)stage_bytes, kMaxRowSmemBytes + 16);
+                if (same_phase && params4 && Cu > 1 && rows * Cu <= 2147483647LL)
+                    return launch_cluster_stage<DT, 256>(xs, gs, bs, ys, rows, D, max_nv, Cu, inv_D, eps, st);
                 if (same_phase && params4 && max_nv <= 1024)
                     return launch_regp_vpt<DT, 128, 10, 6>((int)((max_nv + 127) / 128), xs, gs, bs, ys, rows, D, inv_D, eps, st);
                 // ... and of a 512-thread CTA from 3073 to 4096 (in between, the staged kernel below

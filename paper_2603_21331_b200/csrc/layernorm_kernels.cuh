@@ -366,6 +366,91 @@ layernorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restric
         yr[ej] = Elem<DT>::from_float(ln_out1<DT>(row16[ek * 8 + (threadIdx.x & 7)], __ldg(gamma + ej), __ldg(beta + ej), mu, rstd));
 }
 
+// ------------------------------------------------------------------ unaligned rows split over a cluster
+// The phase layout of layernorm_stage_kernel with the covering vectors of a row split over the C
+// CTAs of a thread-block cluster: CTA c stages covering vectors [nv * c / C, nv * (c + 1) / C),
+// the fully-inside ones by bulk copies; the edge elements (head: first CTA, tail: last CTA) are
+// single values in sixteen threads.  The partial sums meet through the mailboxes of
+// layernorm_cluster_kernel.  For unaligned rows longer than one CTA's shared memory (up to eight)
+// and for a few long unaligned rows.  Needs x and y rows in the same phase, gamma and beta 4-byte
+// aligned and nv >= C.  TAB as in layernorm_stage_kernel.  grid = rows * C, cluster = C.  Dynamic
+// shared memory = ceil(max nv / C) * 16 bytes.
+template <int T, int DT = AK_DTYPE_BF16, bool TAB = false>
+__global__ void __launch_bounds__(T)
+layernorm_cluster_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ gamma,
+                               const uint16_t* __restrict__ beta, uint16_t* __restrict__ y, int64_t D, int C,
+                               float inv_D, float eps, const uint4* tab, int nvp) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    uint4* row = reinterpret_cast<uint4*>(smem_raw);
+    __shared__ uint64_t bar;
+    __shared__ float slots[2 * kWarp];
+    __shared__ float box1[kMaxCluster], box2[kMaxCluster];
+    __shared__ uint64_t xbar1, xbar2;
+    const uint32_t c = cluster_rank();
+    const int64_t r = blockIdx.x / C;
+    const uint16_t* xr = x + r * D;
+    uint16_t* yr = y + r * D;
+    const int phase = (int)((reinterpret_cast<uintptr_t>(xr) >> 1) & 7);
+    const int nv = (int)((phase + D + 7) >> 3);
+    const int k_lo = phase ? 1 : 0;
+    const int k_hi = ((phase + D) & 7) ? nv - 1 : nv;
+    const uint4* xa = reinterpret_cast<const uint4*>(xr - phase);
+    uint4* ya = reinterpret_cast<uint4*>(yr - phase);
+    const int v0 = (int)((int64_t)nv * c / C), v1 = (int)((int64_t)nv * (c + 1) / C);
+    const int i0 = max(v0, k_lo), i1 = min(v1, k_hi);        // the fully-inside vectors of this CTA
+    // edge element of this thread: threads 0..7 the head vector (CTA 0), 8..15 the tail vector (last CTA)
+    const int ek = (threadIdx.x < 8) ? 0 : nv - 1;
+    const bool evec = (threadIdx.x < 8) ? (k_lo == 1 && v0 == 0) : (k_hi == nv - 1 && v1 == nv && !(nv == 1 && k_lo == 1));
+    const int64_t ej = (int64_t)ek * 8 - phase + (threadIdx.x & 7);
+    const bool edge = threadIdx.x < 16 && evec && ej >= 0 && ej < D;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        mailbox_arm(&xbar1, C);
+        mailbox_arm(&xbar2, C);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0)
+        bulk_load_span(smem_raw + (size_t)(i0 - v0) * 16, xa + i0, i1 > i0 ? (uint32_t)(i1 - i0) * 16u : 0u, &bar);
+    cluster_arrive_relaxed();
+    const float K = first_elem<DT>(xr);
+    const uint16_t xe = edge ? ld_stream_u16(xr + ej) : (uint16_t)0;
+    // a wait that gave up (never expected) contributes nothing and writes nothing, but still posts
+    bool ok = mbar_wait(&bar, 0);
+    const int j0 = i0 - v0, j1 = ok ? i1 - v0 : j0;          // local indices of the fully-inside vectors
+    float s1 = edge ? sub_h<DT>(xe, K) : 0.0f;
+    for (int k = j0 + threadIdx.x; k < j1; k += T) s1 += sumdev_v<DT>(row[k], K);
+    s1 = cta_sum<T>(s1, slots, 0);
+    cluster_wait();   // every CTA of the cluster runs, its mailboxes armed, before anything is posted to it
+    if (!mailbox_exchange(s1, box1, &xbar1, C, c)) ok = false;
+    float t1 = 0.0f;
+    for (int i = 0; i < C; ++i) t1 += box1[i];
+    const float mu = fmaf(t1, inv_D, K);
+    const float de = edge ? sub_h<DT>(xe, mu) : 0.0f;
+    float s2 = de * de;
+    for (int k = j0 + threadIdx.x; k < j1; k += T) s2 += sqdev_v<DT>(row[k], mu);
+    s2 = cta_sum<T>(s2, slots, 1);
+    if (!mailbox_exchange(s2, box2, &xbar2, C, c)) ok = false;
+    float t2 = 0.0f;
+    for (int i = 0; i < C; ++i) t2 += box2[i];
+    const float rstd = rsqrtf(fmaf(t2, inv_D, eps));
+    if (!ok) return;
+    if constexpr (TAB) {
+        pdl_wait();   // the table is complete and visible; plain loads (cached in L1), not the read-only path
+        const uint4* gt = tab + (size_t)phase * nvp;
+        const uint4* bt = tab + (size_t)(8 + phase) * nvp;
+#pragma unroll 2
+        for (int k = i0 + threadIdx.x; k < i1; k += T)
+            st_stream(ya + k, ln_out_v<DT>(row[k - v0], gt[k], bt[k], mu, rstd));
+    } else {
+        for (int k = i0 + threadIdx.x; k < i1; k += T) {
+            const int64_t e0 = (int64_t)k * 8 - phase;
+            st_stream(ya + k, ln_out_v<DT>(row[k - v0], ln_load_shifted(gamma, e0), ln_load_shifted(beta, e0), mu, rstd));
+        }
+    }
+    if (edge) yr[ej] = Elem<DT>::from_float(ln_out1<DT>(xe, __ldg(gamma + ej), __ldg(beta + ej), mu, rstd));
+}
+
 // ------------------------------------------------------------------ unaligned rows in registers
 // The phase layout of layernorm_stage_kernel without the trip through shared memory, for rows
 // short enough to sit in registers: interior vectors are loaded before the first use, the edge

@@ -16,6 +16,22 @@ namespace {
 // weights are then requested together with the row instead of after the reduction (no register
 // cap to keep: 1 x 1024 .. 1024 x 4096 run 5-47 % faster, e.g. 8 x 2048 3.2 -> 1.7 us; from 2048
 // rows or 8 MiB on the late fetch with its tighter register budget is as fast or faster).
+// unaligned rows split over a cluster of C CTAs (covering vectors of the worst phase: max_nv)
+template <int DT, int T>
+int launch_cluster_stage(const uint16_t* x, const uint16_t* w, uint16_t* y, int64_t rows, int64_t D, int64_t max_nv, int C,
+                         float inv_D, float eps, cudaStream_t st) {
+    static const bool configured = [] {
+        return cudaFuncSetAttribute(rmsnorm_cluster_stage_kernel<T, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    kMaxRowSmemBytes) == cudaSuccess;
+    }();
+    if (!configured) return AK_ERR_CUDA;
+    const size_t smem = (size_t)((max_nv + C - 1) / C) * 16;
+    const cudaError_t e = launch_cluster(rmsnorm_cluster_stage_kernel<T, DT>, (unsigned)(rows * C), T, smem, C, st, x, w, y,
+                                         D, C, inv_D, eps);
+    count_launch();
+    return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+}
+
 constexpr int64_t kEarlyWeightRows = 1024, kEarlyWeightBytes = 8 << 20;
 
 template <int DT, int THREADS, int GROUP, int VPT, int MINB, bool WE = false>
@@ -185,8 +201,13 @@ int dispatch_t(const void* x, const void* w, void* y, int64_t rows, int64_t D, f
                 const uint16_t* xs = static_cast<const uint16_t*>(x);
                 const uint16_t* ws = static_cast<const uint16_t*>(w);
                 uint16_t* ys = static_cast<uint16_t*>(y);
-                // rows of up to 1024 covering vectors stay in the registers of a 128-thread CTA ...
                 const int64_t max_nv = (D + 14) >> 3;   // vectors covering the row at the worst phase
+                // rows beyond one CTA's shared memory (up to eight CTAs'), and a few long rows (at most
+                // 64 of 32 KiB or more): the covering vectors split over a thread-block cluster
+                const int Cu = cluster_ctas(rows, (int64_t)stage_bytes, kMaxRowSmemBytes + 16);
+                if (same_phase && is_aligned(w, 4) && Cu > 1 && rows * Cu <= 2147483647LL)
+                    return launch_cluster_stage<DT, 256>(xs, ws, ys, rows, D, max_nv, Cu, inv_D, eps, st);
+                // rows of up to 1024 covering vectors stay in the registers of a 128-thread CTA ...
                 if (same_phase && is_aligned(w, 4) && max_nv <= 1024)
                     return launch_regp_vpt<DT, 128>((int)((max_nv + 127) / 128), xs, ws, ys, rows, D, inv_D, eps, st);
                 if (same_phase && is_aligned(w, 4) && max_nv <= 2048)   // ... or of a 256-thread CTA up to 2048

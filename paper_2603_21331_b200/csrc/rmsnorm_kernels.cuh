@@ -290,6 +290,75 @@ rmsnorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict_
     }
 }
 
+// ------------------------------------------------------------------ unaligned rows split over a cluster
+// The phase layout of rmsnorm_stage_kernel with the covering vectors of a row split over the C
+// CTAs of a thread-block cluster: CTA c stages covering vectors [nv * c / C, nv * (c + 1) / C),
+// the fully-inside ones by bulk copies; the first CTA fills the head edge vector and the last one
+// the tail edge vector element by element (zeros in the padding).  The partial sums of squares
+// meet through the mailbox of rmsnorm_cluster_kernel.  For unaligned rows longer than one CTA's
+// shared memory (up to eight) and for a few long unaligned rows.  Needs x and y rows in the same
+// phase, w 4-byte aligned and nv >= C.  grid = rows * C, cluster = C.  Dynamic shared memory =
+// ceil(max nv / C) * 16 bytes.
+template <int T, int DT = AK_DTYPE_BF16>
+__global__ void __launch_bounds__(T)
+rmsnorm_cluster_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, uint16_t* __restrict__ y,
+                             int64_t D, int C, float inv_D, float eps) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    uint4* row = reinterpret_cast<uint4*>(smem_raw);
+    uint16_t* row16 = reinterpret_cast<uint16_t*>(smem_raw);
+    __shared__ uint64_t bar;
+    __shared__ float slots[2 * kWarp];
+    __shared__ float box[kMaxCluster];
+    __shared__ uint64_t xbar;
+    const uint32_t c = cluster_rank();
+    const int64_t r = blockIdx.x / C;
+    const uint16_t* xr = x + r * D;
+    uint16_t* yr = y + r * D;
+    const int phase = (int)((reinterpret_cast<uintptr_t>(xr) >> 1) & 7);
+    const int nv = (int)((phase + D + 7) >> 3);
+    const int k_lo = phase ? 1 : 0;
+    const int k_hi = ((phase + D) & 7) ? nv - 1 : nv;
+    const uint4* xa = reinterpret_cast<const uint4*>(xr - phase);
+    uint4* ya = reinterpret_cast<uint4*>(yr - phase);
+    const int v0 = (int)((int64_t)nv * c / C), v1 = (int)((int64_t)nv * (c + 1) / C);
+    const int n = v1 - v0;                                   // covering vectors of this CTA
+    const int i0 = max(v0, k_lo), i1 = min(v1, k_hi);        // the fully-inside ones
+    // edge element of this thread: threads 0..7 the head vector (CTA 0), 8..15 the tail vector (last CTA)
+    const int ek = (threadIdx.x < 8) ? 0 : nv - 1;
+    const bool evec = (threadIdx.x < 8) ? (k_lo == 1 && v0 == 0) : (k_hi == nv - 1 && v1 == nv && !(nv == 1 && k_lo == 1));
+    const int64_t ej = (int64_t)ek * 8 - phase + (threadIdx.x & 7);
+    const bool my_edge = threadIdx.x < 16 && evec;
+    const bool my_elem = my_edge && ej >= 0 && ej < D;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        mailbox_arm(&xbar, C);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0)
+        bulk_load_span(smem_raw + (size_t)(i0 - v0) * 16, xa + i0, i1 > i0 ? (uint32_t)(i1 - i0) * 16u : 0u, &bar);
+    cluster_arrive_relaxed();
+    if (my_edge) row16[(ek - v0) * 8 + (threadIdx.x & 7)] = my_elem ? ld_stream_u16(xr + ej) : (uint16_t)0;
+    __syncthreads();
+    // a wait that gave up (never expected) contributes nothing and writes nothing, but still posts
+    bool ok = mbar_wait(&bar, 0);
+    const int nn = ok ? n : 0;
+    float ss = 0.0f;
+    for (int k = threadIdx.x; k < nn; k += T) ss += sumsq_v<DT>(row[k]);
+    ss = cta_sum<T>(ss, slots, 0);
+    cluster_wait();   // every CTA of the cluster runs, its mailbox armed, before anything is posted to it
+    if (!mailbox_exchange(ss, box, &xbar, C, c)) ok = false;
+    float tot = 0.0f;
+    for (int i = 0; i < C; ++i) tot += box[i];
+    const float rstd = rsqrtf(fmaf(tot, inv_D, eps));
+    if (!ok) return;
+    for (int k = i0 + threadIdx.x; k < i1; k += T)
+        st_stream(ya + k, scale_v<DT>(row[k - v0], load_w_shifted(w, (int64_t)k * 8 - phase), rstd));
+    if (my_elem)
+        yr[ej] = Elem<DT>::from_float(Elem<DT>::to_float(row16[(ek - v0) * 8 + (threadIdx.x & 7)]) *
+                                      Elem<DT>::to_float(__ldg(w + ej)) * rstd);
+}
+
 // ------------------------------------------------------------------ unaligned rows in registers
 // The phase layout of rmsnorm_stage_kernel without the trip through shared memory, for rows
 // short enough to sit in registers: every interior vector is loaded before the first use and

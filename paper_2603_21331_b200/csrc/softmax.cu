@@ -62,6 +62,20 @@ int launch_stage(const uint16_t* x, uint16_t* y, int64_t rows, int64_t D, size_t
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
+// unaligned rows split over a cluster of C CTAs (covering vectors of the worst phase: max_nv)
+template <int DT, int T>
+int launch_cluster_stage(const uint16_t* x, uint16_t* y, int64_t rows, int64_t D, int64_t max_nv, int C, cudaStream_t st) {
+    static const bool configured = [] {
+        return cudaFuncSetAttribute(softmax_cluster_stage_kernel<T, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    kMaxRowSmemBytes) == cudaSuccess;
+    }();
+    if (!configured) return AK_ERR_CUDA;
+    const size_t smem = (size_t)((max_nv + C - 1) / C) * 16;
+    const cudaError_t e = launch_cluster(softmax_cluster_stage_kernel<T, DT>, (unsigned)(rows * C), T, smem, C, st, x, y, D, C);
+    count_launch();
+    return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+}
+
 template <int DT, int THREADS, int VPT, int MINB>
 int launch_regp(const uint16_t* x, uint16_t* y, int64_t rows, int64_t D, cudaStream_t st) {
     softmax_regp_kernel<THREADS, VPT, MINB, DT><<<(unsigned)rows, THREADS, 0, st>>>(x, y, D);
@@ -166,6 +180,13 @@ int dispatch_t(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st,
                 const int64_t max_nv = (D + 14) >> 3;   // vectors covering the row at the worst phase
                 if (same_phase && max_nv <= 512)
                     return launch_regp_vpt<DT, 128, 5>((int)((max_nv + 127) / 128), xs, ys, rows, D, st);
+                // rows beyond one CTA's shared memory (up to eight CTAs'), and a few long rows: the
+                // covering vectors split over a thread-block cluster
+                const int Cu = cluster_ctas(rows, (int64_t)stage_bytes, kMaxRowSmemBytes + 16);
+                if (same_phase && Cu > 1 && rows * Cu <= 2147483647LL) {
+                    if (rows > 64 && (max_nv + Cu - 1) / Cu <= 2048) return launch_cluster_stage<DT, 128>(xs, ys, rows, D, max_nv, Cu, st);
+                    return launch_cluster_stage<DT, 256>(xs, ys, rows, D, max_nv, Cu, st);
+                }
                 if (same_phase && stage_bytes <= (size_t)kMaxRowSmemBytes) {
                     if (D <= 8192) return launch_stage<DT, 128>(xs, ys, rows, D, stage_bytes, st);
                     if (D <= 32768) return launch_stage<DT, 256>(xs, ys, rows, D, stage_bytes, st);

@@ -439,3 +439,56 @@ def test_small_launches_fetch_parameters_early_with_the_same_bits(D):
     assert torch.equal(l_big[:small].view(torch.int16), l_small.view(torch.int16))
     ref = oracle.rmsnorm(synth.to_bits(x[:small].cpu()), synth.to_bits(w.cpu()), 1e-6)
     assert_bf16_close(y_small, ref, f"rmsnorm {small}x{D} (early weights)")
+
+
+@pytest.mark.parametrize("rows,D,xo", [(3, 128257, 0), (2, 300001, 3), (20, 20001, 0), (64, 16385, 5), (1, 917490, 1),
+                                       (5, 114700, 7), (65, 114689, 0)])
+def test_unaligned_rows_split_over_a_cluster(rows, D, xo):
+    """Rows that are not 16-byte aligned and either too long for one CTA's shared memory or too few
+    to fill the GPU: the covering vectors of the row's own phase are split over a thread-block
+    cluster.  Guard bands around y; every row starts in a different phase."""
+    x = synth.softmax_inputs(rows, D, synth.case_seed(12, rows * 131 + D), mask_frac=0.3)
+    ref = oracle.softmax(synth.to_bits(x))
+    xbuf = torch.zeros(rows * D + 16, dtype=torch.bfloat16, device=DEV)
+    ybuf = torch.full((rows * D + 16,), 7.0, dtype=torch.bfloat16, device=DEV)
+    xv = xbuf[xo:xo + rows * D].view(rows, D)
+    yv = ybuf[xo:xo + rows * D].view(rows, D)
+    xv.copy_(x)
+    ak.ak_softmax_fwd(xv, yv)
+    torch.cuda.synchronize()
+    assert_bf16_close(yv, ref, f"softmax {rows}x{D} offset {xo}")
+    assert bool((ybuf[:xo] == 7.0).all()) and bool((ybuf[xo + rows * D:] == 7.0).all())
+    # RMSNorm and LayerNorm on the same layout (finite inputs)
+    xn, w = synth.rmsnorm_inputs(rows, D, synth.case_seed(13, rows * 131 + D))
+    _, g, b = synth.layernorm_inputs(1, D, 79)
+    xv.copy_(xn)
+    ybuf.fill_(7.0)
+    ak.ak_rmsnorm_fwd(xv, w.to(DEV), yv, eps=1e-6)
+    torch.cuda.synchronize()
+    assert_bf16_close(yv, oracle.rmsnorm(synth.to_bits(xn), synth.to_bits(w), 1e-6), f"rmsnorm {rows}x{D} offset {xo}")
+    assert bool((ybuf[:xo] == 7.0).all()) and bool((ybuf[xo + rows * D:] == 7.0).all())
+    ybuf.fill_(7.0)
+    ak.ak_layernorm_fwd(xv, g.to(DEV), b.to(DEV), yv, eps=1e-5)
+    torch.cuda.synchronize()
+    assert_bf16_close(yv, oracle.layernorm(synth.to_bits(xn), synth.to_bits(g), synth.to_bits(b), 1e-5),
+                      f"layernorm {rows}x{D} offset {xo}", tight=False)
+    assert bool((ybuf[:xo] == 7.0).all()) and bool((ybuf[xo + rows * D:] == 7.0).all())
+
+
+def test_layernorm_unaligned_cluster_with_the_shift_table():
+    """Enough long unaligned rows for both the cluster layout and the table of shifted parameters
+    (two launches: the table kernel, then the cluster kernel as its programmatic dependent)."""
+    rows, D = 300, 114700
+    x, g, b = synth.layernorm_inputs(rows, D, synth.case_seed(14, D), device=DEV)
+    n0 = ak.ak_launch_count()
+    y = ak.ak_layernorm_fwd(x, g, b, eps=1e-5)
+    torch.cuda.synchronize()
+    assert ak.ak_launch_count() - n0 == 2
+    idx = [0, 1, 7, 150, 299]
+    it = torch.tensor(idx, device=DEV)
+    ref = oracle.layernorm(synth.to_bits(x[it].cpu()), synth.to_bits(g.cpu()), synth.to_bits(b.cpu()), 1e-5)
+    assert_bf16_close(y[it], ref, "layernorm 300x114700 sampled rows (cluster + shift table)", tight=False)
+    # the same rows without the table (fewer rows): same bits
+    y2 = ak.ak_layernorm_fwd(x[:200].contiguous(), g, b, eps=1e-5)
+    torch.cuda.synchronize()
+    assert torch.equal(y2.view(torch.int16), y[:200].view(torch.int16))
