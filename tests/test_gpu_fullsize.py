@@ -56,7 +56,8 @@ def test_rmsnorm_full_size(rows, D):
 
 @pytest.mark.parametrize("rows,D", [(16384, 512), (16384, 1024), (16384, 2048), (16384, 4096),
                                     (16384, 8192), (16384, 32768), (262144, 4096), (4096, 4099),
-                                    (4096, 65536), (4096, 128256), (16, 128256), (1, 128256), (512, 262144)])
+                                    (4096, 65536), (4096, 128256), (16, 128256), (1, 128256), (512, 262144),
+                                    (4096, 128257), (16, 50257)])
 def test_softmax_full_size(rows, D):
     x = synth.softmax_inputs(rows, D, synth.case_seed(3, D + rows), device=DEV)
     y = ak.ak_softmax_fwd(x)
