@@ -106,8 +106,15 @@ def _check(status: int, where: str) -> None:
         raise AkError(status, where)
 
 
-def _stream_ptr(stream) -> int:
+# the raw handle of the current stream without building a torch.cuda.Stream object (about 2 us
+# less per call, which counts for decoding-sized launches); absent in some builds of torch
+_raw_current_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+
+
+def _stream_ptr(stream, like: Optional[torch.Tensor] = None) -> int:
     if stream is None:
+        if _raw_current_stream is not None and like is not None:
+            return _raw_current_stream(like.device.index)
         return torch.cuda.current_stream().cuda_stream
     if isinstance(stream, torch.cuda.Stream):
         return stream.cuda_stream
@@ -138,7 +145,7 @@ def ak_rmsnorm_fwd(x: torch.Tensor, w: torch.Tensor, y: Optional[torch.Tensor] =
     if y.shape != x.shape:
         raise ValueError("y must have the shape of x")
     _check(lib().ak_rmsnorm_fwd_path(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, D, eps,
-                                     _stream_ptr(stream), path), "ak_rmsnorm_fwd")
+                                     _stream_ptr(stream, x), path), "ak_rmsnorm_fwd")
     return y
 
 
@@ -164,7 +171,7 @@ def ak_rmsnorm_fwd_dt(x: torch.Tensor, w: torch.Tensor, y: Optional[torch.Tensor
     if y.shape != x.shape:
         raise ValueError("y must have the shape of x")
     _check(lib().ak_rmsnorm_fwd_dt(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, D, eps, dt,
-                                   _stream_ptr(stream), path), "ak_rmsnorm_fwd_dt")
+                                   _stream_ptr(stream, x), path), "ak_rmsnorm_fwd_dt")
     return y
 
 
@@ -178,7 +185,7 @@ def ak_softmax_fwd_dt(x: torch.Tensor, y: Optional[torch.Tensor] = None, stream=
     _dev_dt(y, "y", 2, x.dtype)
     if y.shape != x.shape:
         raise ValueError("y must have the shape of x")
-    _check(lib().ak_softmax_fwd_dt(x.data_ptr(), y.data_ptr(), rows, D, dt, _stream_ptr(stream), path),
+    _check(lib().ak_softmax_fwd_dt(x.data_ptr(), y.data_ptr(), rows, D, dt, _stream_ptr(stream, x), path),
            "ak_softmax_fwd_dt")
     return y
 
@@ -196,7 +203,7 @@ def ak_xent_fwd_dt(logits: torch.Tensor, targets: torch.Tensor, ignore_index: in
     loss_mean = torch.empty((1,), dtype=torch.float32, device=logits.device) if want_mean else None
     _check(lib().ak_xent_fwd_dt(logits.data_ptr(), targets.data_ptr(), ignore_index, loss_rows.data_ptr(),
                                 loss_mean.data_ptr() if want_mean else None, rows, V, dt,
-                                _stream_ptr(stream), path, nsplit), "ak_xent_fwd_dt")
+                                _stream_ptr(stream, logits), path, nsplit), "ak_xent_fwd_dt")
     return loss_rows, loss_mean
 
 
@@ -216,7 +223,7 @@ def ak_layernorm_fwd_dt(x: torch.Tensor, gamma: torch.Tensor, beta: torch.Tensor
     if y.shape != x.shape:
         raise ValueError("y must have the shape of x")
     _check(lib().ak_layernorm_fwd_dt(x.data_ptr(), gamma.data_ptr(), beta.data_ptr(), y.data_ptr(), rows, D,
-                                     eps, dt, _stream_ptr(stream), path), "ak_layernorm_fwd_dt")
+                                     eps, dt, _stream_ptr(stream, x), path), "ak_layernorm_fwd_dt")
     return y
 
 
@@ -228,7 +235,7 @@ def ak_rowsum_fwd_dt(x: torch.Tensor, out: Optional[torch.Tensor] = None, stream
         out = torch.empty((rows,), dtype=torch.float32, device=x.device)
     if not (out.is_cuda and out.dtype == torch.float32 and out.shape == (rows,) and out.is_contiguous()):
         raise TypeError("out must be a contiguous CUDA float32 tensor [rows]")
-    _check(lib().ak_rowsum_fwd_dt(x.data_ptr(), out.data_ptr(), rows, D, dt, _stream_ptr(stream)),
+    _check(lib().ak_rowsum_fwd_dt(x.data_ptr(), out.data_ptr(), rows, D, dt, _stream_ptr(stream, x)),
            "ak_rowsum_fwd_dt")
     return out
 
@@ -244,7 +251,7 @@ def ak_rope_fwd(x: torch.Tensor, y: Optional[torch.Tensor] = None, base: float =
     if y.shape != x.shape:
         raise ValueError("y must have the shape of x")
     _check(lib().ak_rope_fwd(x.data_ptr(), y.data_ptr(), n_seq, S, Dh, base, pos_offset, dt,
-                             _stream_ptr(stream)), "ak_rope_fwd")
+                             _stream_ptr(stream, x)), "ak_rope_fwd")
     return y
 
 
@@ -272,7 +279,7 @@ def ak_xent_vp_partial(logits_shard: torch.Tensor, targets: torch.Tensor, vocab_
         raise TypeError("partial must be a contiguous CUDA float32 tensor [rows, nsplit + 1, 2]")
     _check(lib().ak_xent_vp_partial(logits_shard.data_ptr(), targets.data_ptr(), ignore_index, vocab_start,
                                     V_total, partial.data_ptr(), rows, V_local, nsplit, dt,
-                                    _stream_ptr(stream)), "ak_xent_vp_partial")
+                                    _stream_ptr(stream, logits_shard)), "ak_xent_vp_partial")
     return partial
 
 
@@ -291,7 +298,7 @@ def ak_xent_vp_merge(partials: torch.Tensor, targets: torch.Tensor, V_total: int
     loss_mean = torch.empty((1,), dtype=torch.float32, device=partials.device) if want_mean else None
     _check(lib().ak_xent_vp_merge(partials.data_ptr(), nranks, ns1 - 1, targets.data_ptr(), ignore_index,
                                   V_total, loss_rows.data_ptr(), loss_mean.data_ptr() if want_mean else None,
-                                  rows, _stream_ptr(stream)), "ak_xent_vp_merge")
+                                  rows, _stream_ptr(stream, partials)), "ak_xent_vp_merge")
     return loss_rows, loss_mean
 
 
@@ -314,7 +321,7 @@ def ak_layernorm_fwd(x: torch.Tensor, gamma: torch.Tensor, beta: torch.Tensor,
     if y.shape != x.shape:
         raise ValueError("y must have the shape of x")
     _check(lib().ak_layernorm_fwd_path(x.data_ptr(), gamma.data_ptr(), beta.data_ptr(), y.data_ptr(),
-                                       rows, D, eps, _stream_ptr(stream), path), "ak_layernorm_fwd")
+                                       rows, D, eps, _stream_ptr(stream, x), path), "ak_layernorm_fwd")
     return y
 
 
@@ -325,7 +332,7 @@ def ak_rowsum_fwd(x: torch.Tensor, out: Optional[torch.Tensor] = None, stream=No
         out = torch.empty((rows,), dtype=torch.float32, device=x.device)
     if not (out.is_cuda and out.dtype == torch.float32 and out.shape == (rows,) and out.is_contiguous()):
         raise TypeError("out must be a contiguous CUDA float32 tensor [rows]")
-    _check(lib().ak_rowsum_fwd(x.data_ptr(), out.data_ptr(), rows, D, _stream_ptr(stream)), "ak_rowsum_fwd")
+    _check(lib().ak_rowsum_fwd(x.data_ptr(), out.data_ptr(), rows, D, _stream_ptr(stream, x)), "ak_rowsum_fwd")
     return out
 
 
@@ -338,7 +345,7 @@ def ak_softmax_fwd(x: torch.Tensor, y: Optional[torch.Tensor] = None, stream=Non
     _dev_bf16(y, "y", 2)
     if y.shape != x.shape:
         raise ValueError("y must have the shape of x")
-    _check(lib().ak_softmax_fwd_path(x.data_ptr(), y.data_ptr(), rows, D, _stream_ptr(stream), path),
+    _check(lib().ak_softmax_fwd_path(x.data_ptr(), y.data_ptr(), rows, D, _stream_ptr(stream, x), path),
            "ak_softmax_fwd")
     return y
 
@@ -362,7 +369,7 @@ def ak_xent_fwd(logits: torch.Tensor, targets: torch.Tensor, ignore_index: int =
             raise TypeError("loss buffers must be contiguous CUDA float32 tensors")
     mean_ptr = loss_mean.data_ptr() if loss_mean is not None else None
     _check(lib().ak_xent_fwd_path(logits.data_ptr(), targets.data_ptr(), ignore_index,
-                                  loss_rows.data_ptr(), mean_ptr, rows, V, _stream_ptr(stream),
+                                  loss_rows.data_ptr(), mean_ptr, rows, V, _stream_ptr(stream, logits),
                                   path, nsplit), "ak_xent_fwd")
     return loss_rows, loss_mean
 
@@ -387,7 +394,7 @@ def ak_xent_fwd_static(logits: torch.Tensor, targets: torch.Tensor, ignore_index
         loss_mean = torch.empty((1,), dtype=torch.float32, device=logits.device)
     _check(lib().ak_xent_fwd_static(logits.data_ptr(), targets.data_ptr(), ignore_index,
                                     loss_rows.data_ptr(), loss_mean.data_ptr(), rows, V,
-                                    _stream_ptr(stream)), "ak_xent_fwd_static")
+                                    _stream_ptr(stream, logits)), "ak_xent_fwd_static")
     return loss_rows, loss_mean
 
 
@@ -408,7 +415,7 @@ def ak_xent_fwd_ws(logits: torch.Tensor, targets: torch.Tensor, workspace: Optio
     ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
     _check(lib().ak_xent_fwd_ws(logits.data_ptr(), targets.data_ptr(), ignore_index,
                                 loss_rows.data_ptr(), loss_mean.data_ptr(), rows, V, ws_ptr, ws_bytes,
-                                _stream_ptr(stream)), "ak_xent_fwd_ws")
+                                _stream_ptr(stream, logits)), "ak_xent_fwd_ws")
     return loss_rows, loss_mean
 
 
