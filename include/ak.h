@@ -67,7 +67,7 @@ enum {
     AK_PATH_CTA = 2,      /* one CTA per row, row held in registers; rows <= 64 KiB (bf16 D <= 32768) */
     AK_PATH_GENERIC = 3,  /* any D, any element alignment; the row is kept in registers or staged in shared memory (of one CTA, or of a cluster of up to eight for rows beyond 224 KiB and for a few long rows) in its 16-byte phase: a single DRAM pass; else re-read from L1/L2 */
     AK_PATH_SMEM = 4,     /* one CTA per row, row staged in shared memory by bulk (TMA) copies; rows <= 224 KiB (bf16 D <= 114688) */
-    AK_PATH_CLUSTER = 5   /* a thread-block cluster of 2, 4 or 8 CTAs per row, each staging a slice in its shared memory, partial results exchanged through distributed shared memory; rows of 32 bytes .. 1792 KiB (bf16 D <= 917504).  The dispatcher takes it for aligned rows longer than 64 KiB, in slices of at most 32 KiB where eight CTAs can do that, and for at most 64 rows of 32 KiB or more (eight CTAs each); longer aligned rows than 1792 KiB take AK_PATH_GENERIC */
+    AK_PATH_CLUSTER = 5   /* a thread-block cluster of 2, 4 or 8 CTAs per row, each staging a slice in its shared memory, partial results exchanged through distributed shared memory; rows of 32 bytes and more.  The dispatcher takes it for aligned rows longer than 64 KiB, in slices of at most 32 KiB where eight CTAs can do that, and for at most 64 rows of 32 KiB or more (eight CTAs each); rows beyond 1792 KiB (bf16 D > 917504) do not fit eight CTAs' shared memory and are streamed from global memory by the eight CTAs instead (two or three reads, the later ones from the caches where they still hold the slice) */
 };
 /* Element types of the *_dt entry points.  The plain entry points are bf16. */
 enum {
@@ -101,7 +101,7 @@ int ak_rmsnorm_fwd_path(const void* x, const void* w, void* y,
  * outputs carry the fp32 arithmetic's own rounding).  Pointers must be aligned to the
  * element size; the fast paths need 16-byte aligned bases and rows that are a multiple of
  * 16 bytes (D % 8 == 0 for 16-bit types, D % 4 == 0 for fp32); the path limits of AK_PATH_*
- * scale with the row's BYTES (4 KiB / 64 KiB / 224 KiB; clusters 1792 KiB).  fp16 outputs beyond 65504
+ * scale with the row's BYTES (4 KiB / 64 KiB / 224 KiB; clusters stage up to 1792 KiB).  fp16 outputs beyond 65504
  * become inf, as the type dictates.  `path` (and `nsplit`) as in the *_path entry points;
  * 0 = automatic.  An unknown dtype gives AK_ERR_ARG.
  */

@@ -60,10 +60,12 @@ cudaError_t scratch_alloc(void** p, size_t bytes, cudaStream_t st) {
 //      SM and overlap their phases (4096 x 65536 softmax 235 -> 174 us, RMSNorm 186 -> 163 us;
 //      rows beyond one CTA's shared memory, 4096 x 128256: softmax 677 -> 362 us);
 //  (b) with at most 64 rows, rows of 32 KiB or more go to eight CTAs each (1.1x - 2.6x).
-// 1 = one CTA per row (also when the row does not fit eight CTAs' shared memory).
+// 1 = one CTA per row.  Rows beyond eight CTAs' shared memory get eight CTAs too (the callers
+// that cannot stage them stream them, or fall back, as they see fit).
 int cluster_ctas(int64_t rows, int64_t row_bytes, int64_t split_from) {
     constexpr int64_t kSliceBytes = 32768, kFewRows = 64, kFewRowsMinBytes = 32768;
-    if (rows < 1 || row_bytes > (int64_t)kMaxCluster * kMaxRowSmemBytes) return 1;
+    if (rows < 1) return 1;
+    if (row_bytes > (int64_t)kMaxCluster * kMaxRowSmemBytes) return kMaxCluster;
     int C = 1;
     if (row_bytes >= split_from)
         while (C < kMaxCluster && row_bytes > (int64_t)C * kSliceBytes) C *= 2;

@@ -243,7 +243,15 @@ int dispatch_t(const void* x, const void* gamma, const void* beta, void* y, int6
         case AK_PATH_CLUSTER: {
             int C = cluster_ctas(rows, row_bytes, kClusterFrom);
             if (C < 2) C = 2;   // forced by the caller
-            if (nvec < C || row_bytes > (int64_t)C * kMaxRowSmemBytes || rows * C > 2147483647LL) return AK_ERR_SHAPE;
+            if ((row_bytes >> 4) < C || rows * C > 2147483647LL) return AK_ERR_SHAPE;
+            if (row_bytes > (int64_t)C * kMaxRowSmemBytes) {   // too long to stage: streamed
+                const cudaError_t e = launch_cluster(layernorm_cluster_stream_kernel<512, DT>, (unsigned)(rows * C), 512, 0, C, st,
+                                                     static_cast<const uint4*>(x), static_cast<const uint4*>(gamma),
+                                                     static_cast<const uint4*>(beta), static_cast<uint4*>(y),
+                                                     (int64_t)(row_bytes >> 4), C, inv_D, eps);
+                count_launch();
+                return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+            }
             if ((nvec + C - 1) / C <= 4096)
                 return launch_cluster_rows<DT, 256>(x, gamma, beta, y, rows, nvec, C, inv_D, eps, st);
             return launch_cluster_rows<DT, 512>(x, gamma, beta, y, rows, nvec, C, inv_D, eps, st);
@@ -270,7 +278,7 @@ int dispatch_t(const void* x, const void* gamma, const void* beta, void* y, int6
                 // rows beyond one CTA's shared memory (up to eight CTAs'), and a few long rows (at most
                 // 64 of 32 KiB or more): the covering vectors split over a thread-block cluster
                 const int Cu = cluster_ctas(rows, (int64_t)stage_bytes, kMaxRowSmemBytes + 16);
-                if (same_phase && params4 && Cu > 1 && rows * Cu <= 2147483647LL)
+                if (same_phase && params4 && Cu > 1 && stage_bytes <= (size_t)kMaxCluster * kMaxRowSmemBytes && rows * Cu <= 2147483647LL)
                     return launch_cluster_stage<DT, 256>(xs, gs, bs, ys, rows, D, max_nv, Cu, inv_D, eps, st);
                 if (same_phase && params4 && max_nv <= 1024)
                     return launch_regp_vpt<DT, 128, 10, 6>((int)((max_nv + 127) / 128), xs, gs, bs, ys, rows, D, inv_D, eps, st);
@@ -301,7 +309,6 @@ int layernorm_choose(int64_t rows, int64_t D, bool aligned16, int dtype) {
     const int64_t bytes = D * dtype_bytes(dtype);
     if (!aligned16 || (bytes & 15) != 0) return AK_PATH_GENERIC;
     if (cluster_ctas(rows, bytes, kClusterFrom) > 1) return AK_PATH_CLUSTER;
-    if (bytes > kMaxRowSmemBytes) return AK_PATH_GENERIC;
     if (bytes <= 4096) return AK_PATH_WARP;
     if (bytes <= 65536) return AK_PATH_CTA;   // up to 64 KiB the register layout beats the staged one
     return AK_PATH_SMEM;

@@ -286,6 +286,55 @@ layernorm_cluster_kernel(const uint4* __restrict__ x, const uint4* __restrict__ 
         st_stream(yr + i, ln_out_v<DT>(row[i], __ldg(gr + i), __ldg(br + i), mu, rstd));
 }
 
+// ------------------------------------------------------------------ rows of any length streamed by a cluster
+// Rows too long for the shared memory of eight CTAs: the C CTAs of a cluster each stream their
+// slice of the row from global memory three times (sum of x - K, sum of (x - mu)^2, normalise and
+// store; partial sums through the mailboxes); the later reads find what the caches kept.  Needs
+// 16-byte aligned rows.  grid = rows * C, cluster = C.
+template <int T, int DT = AK_DTYPE_BF16>
+__global__ void __launch_bounds__(T)
+layernorm_cluster_stream_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamma,
+                                const uint4* __restrict__ beta, uint4* __restrict__ y, int64_t nvec, int C,
+                                float inv_D, float eps) {
+    __shared__ float slots[2 * kWarp];
+    __shared__ float box1[kMaxCluster], box2[kMaxCluster];
+    __shared__ uint64_t xbar1, xbar2;
+    const uint32_t c = cluster_rank();
+    const int64_t r = blockIdx.x / C;
+    const int64_t v0 = nvec / C * c + min((int64_t)c, nvec % C);
+    const int64_t v1 = v0 + nvec / C + ((int64_t)c < nvec % C ? 1 : 0);
+    if (threadIdx.x == 0) {
+        mailbox_arm(&xbar1, C);
+        mailbox_arm(&xbar2, C);
+    }
+    __syncthreads();
+    cluster_arrive_relaxed();
+    const uint4* xr = x + r * nvec;
+    const float K = first_elem<DT>(xr);
+    float s1 = 0.0f;
+#pragma unroll 8
+    for (int64_t i = v0 + threadIdx.x; i < v1; i += T) s1 += sumdev_v<DT>(xr[i], K);
+    s1 = cta_sum<T>(s1, slots, 0);
+    cluster_wait();   // every CTA of the cluster runs, its mailboxes armed, before anything is posted to it
+    bool ok = mailbox_exchange(s1, box1, &xbar1, C, c);
+    float t1 = 0.0f;
+    for (int i = 0; i < C; ++i) t1 += box1[i];
+    const float mu = fmaf(t1, inv_D, K);
+    float s2 = 0.0f;
+#pragma unroll 8
+    for (int64_t i = v0 + threadIdx.x; i < v1; i += T) s2 += sqdev_v<DT>(xr[i], mu);
+    s2 = cta_sum<T>(s2, slots, 1);
+    if (!mailbox_exchange(s2, box2, &xbar2, C, c)) ok = false;
+    float t2 = 0.0f;
+    for (int i = 0; i < C; ++i) t2 += box2[i];
+    const float rstd = rsqrtf(fmaf(t2, inv_D, eps));
+    if (!ok) return;   // a wait that gave up (never expected): nothing is written
+    uint4* yr = y + r * nvec;
+#pragma unroll 2
+    for (int64_t i = v0 + threadIdx.x; i < v1; i += T)
+        st_stream(yr + i, ln_out_v<DT>(ld_stream(xr + i), __ldg(gamma + i), __ldg(beta + i), mu, rstd));
+}
+
 // ------------------------------------------------------------------ unaligned rows staged in shared memory
 // D % 8 != 0 (or a misaligned base): one CTA per row copies the row into shared memory in the
 // 16-byte phase it has in global memory, so interior vectors are aligned 16-byte loads and

@@ -217,6 +217,41 @@ rmsnorm_cluster_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w,
     for (int i = threadIdx.x; i < nn; i += THREADS) st_stream(yr + i, scale_v<DT>(row[i], __ldg(wr + i), rstd));
 }
 
+// ------------------------------------------------------------------ rows of any length streamed by a cluster
+// Rows too long for the shared memory of eight CTAs: the C CTAs of a cluster each stream their
+// slice of the row from global memory twice, once for the sum of squares (partial sums through the
+// mailbox) and once more to scale and store; the second read finds what the caches kept (nothing
+// is staged).  Needs 16-byte aligned rows.  grid = rows * C, cluster = C.
+template <int T, int DT = AK_DTYPE_BF16>
+__global__ void __launch_bounds__(T)
+rmsnorm_cluster_stream_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w, uint4* __restrict__ y,
+                              int64_t nvec, int C, float inv_D, float eps) {
+    __shared__ float slots[2 * kWarp];
+    __shared__ float box[kMaxCluster];
+    __shared__ uint64_t xbar;
+    const uint32_t c = cluster_rank();
+    const int64_t r = blockIdx.x / C;
+    const int64_t v0 = nvec / C * c + min((int64_t)c, nvec % C);
+    const int64_t v1 = v0 + nvec / C + ((int64_t)c < nvec % C ? 1 : 0);
+    if (threadIdx.x == 0) mailbox_arm(&xbar, C);
+    __syncthreads();
+    cluster_arrive_relaxed();
+    const uint4* xr = x + r * nvec;
+    float ss = 0.0f;
+#pragma unroll 8
+    for (int64_t i = v0 + threadIdx.x; i < v1; i += T) ss += sumsq_v<DT>(xr[i]);
+    ss = cta_sum<T>(ss, slots, 0);
+    cluster_wait();   // every CTA of the cluster runs, its mailbox armed, before anything is posted to it
+    const bool ok = mailbox_exchange(ss, box, &xbar, C, c);
+    float tot = 0.0f;
+    for (int i = 0; i < C; ++i) tot += box[i];
+    const float rstd = rsqrtf(fmaf(tot, inv_D, eps));
+    if (!ok) return;   // a wait that gave up (never expected): nothing is written
+    uint4* yr = y + r * nvec;
+#pragma unroll 4
+    for (int64_t i = v0 + threadIdx.x; i < v1; i += T) st_stream(yr + i, scale_v<DT>(ld_stream(xr + i), __ldg(w + i), rstd));
+}
+
 // ------------------------------------------------------------------ unaligned rows staged in shared memory
 // D % 8 != 0 (or a misaligned base) makes the 16-byte phase of a row change from row to row.
 // One CTA per row copies the row into shared memory in the phase it has in global memory:

@@ -153,7 +153,14 @@ int dispatch_t(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st,
         case AK_PATH_CLUSTER: {
             int C = cluster_ctas(rows, row_bytes, kClusterFrom);
             if (C < 2) C = 2;   // forced by the caller
-            if (nvec < C || row_bytes > (int64_t)C * kMaxRowSmemBytes || rows * C > 2147483647LL) return AK_ERR_SHAPE;
+            if ((row_bytes >> 4) < C || rows * C > 2147483647LL) return AK_ERR_SHAPE;
+            if (row_bytes > (int64_t)C * kMaxRowSmemBytes) {   // too long to stage: streamed
+                const cudaError_t e = launch_cluster(softmax_cluster_stream_kernel<512, DT>, (unsigned)(rows * C), 512, 0, C, st,
+                                                     static_cast<const uint4*>(x), static_cast<uint4*>(y),
+                                                     (int64_t)(row_bytes >> 4), C);
+                count_launch();
+                return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+            }
             // many rows in slices of up to 32 KiB: 128-thread CTAs measured 2-12 % faster than 256
             // (and 64 slower); a few rows are better off with 256
             if ((nvec + C - 1) / C <= 2048 && rows > 64) return launch_cluster_rows<DT, 128, 4>(x, y, rows, nvec, C, st);
@@ -183,7 +190,7 @@ int dispatch_t(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st,
                 // rows beyond one CTA's shared memory (up to eight CTAs'), and a few long rows: the
                 // covering vectors split over a thread-block cluster
                 const int Cu = cluster_ctas(rows, (int64_t)stage_bytes, kMaxRowSmemBytes + 16);
-                if (same_phase && Cu > 1 && rows * Cu <= 2147483647LL) {
+                if (same_phase && Cu > 1 && stage_bytes <= (size_t)kMaxCluster * kMaxRowSmemBytes && rows * Cu <= 2147483647LL) {
                     if (rows > 64 && (max_nv + Cu - 1) / Cu <= 2048) return launch_cluster_stage<DT, 128>(xs, ys, rows, D, max_nv, Cu, st);
                     return launch_cluster_stage<DT, 256>(xs, ys, rows, D, max_nv, Cu, st);
                 }
@@ -210,7 +217,6 @@ int softmax_choose(int64_t rows, int64_t D, bool aligned16, int dtype) {
     const int64_t bytes = D * dtype_bytes(dtype);
     if (!aligned16 || (bytes & 15) != 0) return AK_PATH_GENERIC;
     if (cluster_ctas(rows, bytes, kClusterFrom) > 1) return AK_PATH_CLUSTER;
-    if (bytes > kMaxRowSmemBytes) return AK_PATH_GENERIC;
     if (bytes <= 4096) return AK_PATH_WARP;
     if (bytes <= 16384) return AK_PATH_CTA;
     return AK_PATH_SMEM;

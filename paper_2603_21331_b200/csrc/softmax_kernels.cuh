@@ -283,6 +283,55 @@ softmax_cluster_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int n
     }
 }
 
+// ------------------------------------------------------------------ rows of any length streamed by a cluster
+// Rows too long for the shared memory of eight CTAs: the C CTAs of a cluster each stream their
+// slice of the row from global memory three times (maximum, sum of exponentials, normalise and
+// store; maxima and sums through the mailboxes); the later reads find what the caches kept.
+// Needs 16-byte aligned rows.  grid = rows * C, cluster = C.
+template <int T, int DT = AK_DTYPE_BF16>
+__global__ void __launch_bounds__(T)
+softmax_cluster_stream_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t nvec, int C) {
+    __shared__ float slots[2 * kWarp];
+    __shared__ float box_m[kMaxCluster], box_s[kMaxCluster];
+    __shared__ uint64_t xbar_m, xbar_s;
+    const uint32_t c = cluster_rank();
+    const int64_t r = blockIdx.x / C;
+    const int64_t v0 = nvec / C * c + min((int64_t)c, nvec % C);
+    const int64_t v1 = v0 + nvec / C + ((int64_t)c < nvec % C ? 1 : 0);
+    if (threadIdx.x == 0) {
+        mailbox_arm(&xbar_m, C);
+        mailbox_arm(&xbar_s, C);
+    }
+    __syncthreads();
+    cluster_arrive_relaxed();
+    const uint4* xr = x + r * nvec;
+    uint32_t mx = neg_inf_word<DT>();
+#pragma unroll 8
+    for (int64_t i = v0 + threadIdx.x; i < v1; i += T) mx = max_w<DT>(mx, max_v<DT>(xr[i]));
+    const float m_cta = cta_max<T>(hmax_of<DT>(mx), slots, 0);
+    cluster_wait();   // every CTA of the cluster runs, its mailboxes armed, before anything is posted to it
+    bool ok = mailbox_exchange(m_cta, box_m, &xbar_m, C, c);
+    float m = box_m[0];
+    for (int i = 1; i < C; ++i) m = fmaxf(m, box_m[i]);
+    const float m2 = m * kLog2e;
+    float sum = 0.0f;
+    f32x2 e[kExpPairs<DT>];
+#pragma unroll 4
+    for (int64_t i = v0 + threadIdx.x; i < v1; i += T) sum += exp_v<DT>(xr[i], m2, e);
+    sum = cta_sum<T>(sum, slots, 1);
+    if (!mailbox_exchange(sum, box_s, &xbar_s, C, c)) ok = false;
+    float tot = 0.0f;
+    for (int i = 0; i < C; ++i) tot += box_s[i];
+    const float inv = 1.0f / tot;
+    if (!ok) return;   // a wait that gave up (never expected): nothing is written
+    uint4* yr = y + r * nvec;
+#pragma unroll 4
+    for (int64_t i = v0 + threadIdx.x; i < v1; i += T) {
+        exp_v<DT>(ld_stream(xr + i), m2, e);
+        st_stream(yr + i, norm_v<DT>(e, inv));
+    }
+}
+
 // ------------------------------------------------------------------ unaligned rows staged in shared memory
 // Same staging as the RMSNorm kernel of that name: the row sits in shared memory in the
 // 16-byte phase it has in global memory (x and y rows share it), fully-inside vectors move

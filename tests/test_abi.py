@@ -133,7 +133,7 @@ def test_dispatch_is_a_pure_function_of_shape_and_alignment():
     assert ak.ak_rmsnorm_choose_path(8192, 65536, True) == ak.AK_PATH_CLUSTER
     assert ak.ak_rmsnorm_choose_path(8192, 131072, True) == ak.AK_PATH_CLUSTER   # 256 KiB rows: four to eight CTAs' shared memory
     assert ak.ak_rmsnorm_choose_path(8192, 917504, True) == ak.AK_PATH_CLUSTER   # 8 x 224 KiB, the longest
-    assert ak.ak_rmsnorm_choose_path(8192, 917512, True) == ak.AK_PATH_GENERIC
+    assert ak.ak_rmsnorm_choose_path(8192, 917512, True) == ak.AK_PATH_CLUSTER   # beyond that: streamed by the cluster
     assert ak.ak_rmsnorm_choose_path(64, 16384, True) == ak.AK_PATH_CLUSTER      # few rows of 32 KiB or more
     assert ak.ak_rmsnorm_choose_path(65, 16384, True) == ak.AK_PATH_CTA
     assert ak.ak_rmsnorm_choose_path(64, 8192, True) == ak.AK_PATH_CTA

@@ -413,13 +413,39 @@ def test_cluster_path_rejects_rows_it_cannot_hold():
     w = torch.ones((8,), dtype=torch.bfloat16, device=DEV)
     with pytest.raises(ak.AkError):
         ak.ak_rmsnorm_fwd(x, w, path=CLUSTER)
-    big = torch.zeros((1, 917512), dtype=torch.bfloat16, device=DEV)    # one vector beyond 8 x 224 KiB
-    with pytest.raises(ak.AkError):
-        ak.ak_softmax_fwd(big, path=CLUSTER)
-    y = ak.ak_softmax_fwd(big)                                          # the dispatcher falls back to the multi-pass kernel
+    big = torch.zeros((1, 917512), dtype=torch.bfloat16, device=DEV)    # one vector beyond 8 x 224 KiB: streamed
+    y = ak.ak_softmax_fwd(big)
+    y2 = ak.ak_softmax_fwd(big, path=CLUSTER)
     torch.cuda.synchronize()
     v = y.float()
     assert bool((v == v[0, 0]).all()) and abs(float(v[0, 0]) * 917512 - 1.0) < 2.0 ** -8
+    assert torch.equal(y.view(torch.int16), y2.view(torch.int16))
+
+
+@pytest.mark.parametrize("rows,D", [(1, 917512), (3, 1048576), (2, 2000008), (70, 1000000)])
+def test_rows_of_any_length_streamed_by_a_cluster(rows, D):
+    """Aligned rows beyond the shared memory of eight CTAs: each CTA of the cluster streams its slice
+    from global memory, partial results through the mailboxes.  All three ops, in place as well."""
+    x, w = synth.rmsnorm_inputs(rows, D, synth.case_seed(15, rows * 131 + D))
+    _, g, b = synth.layernorm_inputs(1, D, 80)
+    xs = synth.softmax_inputs(rows, D, synth.case_seed(16, rows * 131 + D), mask_frac=0.3)
+    idx = sorted({0, rows - 1, rows // 2})
+    for name, run, ref in (
+            ("rmsnorm", lambda t, o: ak.ak_rmsnorm_fwd(t, w.to(DEV), o, eps=1e-6),
+             oracle.rmsnorm(synth.to_bits(x[idx]), synth.to_bits(w), 1e-6)),
+            ("layernorm", lambda t, o: ak.ak_layernorm_fwd(t, g.to(DEV), b.to(DEV), o, eps=1e-5),
+             oracle.layernorm(synth.to_bits(x[idx]), synth.to_bits(g), synth.to_bits(b), 1e-5)),
+            ("softmax", lambda t, o: ak.ak_softmax_fwd(t, o), oracle.softmax(synth.to_bits(xs[idx])))):
+        src = (xs if name == "softmax" else x).to(DEV)
+        y, check = guarded((rows, D), torch.bfloat16, DEV)
+        run(src, y)
+        torch.cuda.synchronize()
+        check()
+        assert_bf16_close(y[idx], ref, f"{name} {rows}x{D} (streamed)", tight=(name != "layernorm"))
+        first = y.clone()
+        run(src, src)                                                   # in place
+        torch.cuda.synchronize()
+        assert torch.equal(first.view(torch.int16), src.view(torch.int16))
 
 
 @pytest.mark.parametrize("D", [1024, 2048, 4096, 8192])
