@@ -328,6 +328,17 @@ xent_finish_kernel(const typename XElem<DT>::type* __restrict__ logits, const in
     constexpr int T = kFinishThreads;
     __shared__ double ssum[T / kWarp];
     __shared__ double scnt[T / kWarp];
+    // The targets are inputs, not results of the streaming kernel: which of this thread's first
+    // sixteen rows count is worked out before the wait, while that kernel is still running.
+    constexpr int B = 16;
+    uint32_t counted0 = 0;
+    if (out_mean != nullptr || out_pair != nullptr) {
+#pragma unroll
+        for (int k = 0; k < B; ++k) {
+            const int64_t r = threadIdx.x + (int64_t)k * T;
+            if (r < rows && targets[r] != ignore_index) counted0 |= 1u << k;
+        }
+    }
     pdl_wait();  // everything the streaming kernel wrote is visible from here on
     if (nsplit > 0) {
         for (int64_t r = threadIdx.x; r < rows; r += T) {
@@ -356,16 +367,30 @@ xent_finish_kernel(const typename XElem<DT>::type* __restrict__ logits, const in
     // Mean: batches of independent loads (a lone CTA is latency-bound, so sixteen rows are in
     // flight per thread), added in row order per thread.  A thread re-reads only rows it
     // wrote itself above, so program order makes them visible.
-    constexpr int B = 16;
     double acc = 0.0, cnt = 0.0;
-    for (int64_t base = threadIdx.x; base < rows; base += (int64_t)T * B) {
+    {   // the first batch: the counted rows are known already
+        float ll[B];
+#pragma unroll
+        for (int k = 0; k < B; ++k) {
+            const int64_t r = threadIdx.x + (int64_t)k * T;
+            ll[k] = (r < rows) ? __ldcg(loss_rows + r) : 0.0f;  // L2 read: written by the grid we depend on
+        }
+#pragma unroll
+        for (int k = 0; k < B; ++k) {
+            if (counted0 & (1u << k)) {
+                acc += (double)ll[k];
+                cnt += 1.0;
+            }
+        }
+    }
+    for (int64_t base = threadIdx.x + (int64_t)T * B; base < rows; base += (int64_t)T * B) {
         int64_t tt[B];
         float ll[B];
 #pragma unroll
         for (int k = 0; k < B; ++k) {
             const int64_t r = base + (int64_t)k * T;
             tt[k] = (r < rows) ? targets[r] : ignore_index;
-            ll[k] = (r < rows) ? __ldcg(loss_rows + r) : 0.0f;  // L2 read: written by the grid we depend on
+            ll[k] = (r < rows) ? __ldcg(loss_rows + r) : 0.0f;
         }
 #pragma unroll
         for (int k = 0; k < B; ++k) {
