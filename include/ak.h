@@ -28,6 +28,10 @@
  *     memory pool of the library's own (one per device, created at first use, keeps up to
  *     256 MiB cached between calls) through cudaMallocFromPoolAsync / cudaFreeAsync on the
  *     call's stream; such calls may be captured in CUDA graphs.
+ *   - Thread-block clusters: AK_PATH_CLUSTER kernels need the device to co-schedule up to eight
+ *     CTAs.  Where a cluster launch is refused (a partition of a device with too few SMs per
+ *     GPC), the dispatcher falls back to one CTA per row or the multi-pass kernels; setting
+ *     AK_DISABLE_CLUSTERS=1 in the environment (read once) makes that the choice from the start.
  *   - rows == 0 is legal: nothing is launched (cross-entropy still writes loss_mean = NaN).
  *   - Determinism: same inputs, shape, pointer alignment, library build and GPU model
  *     give bit-identical outputs.  Path selection is a pure function of

@@ -64,7 +64,13 @@ cudaError_t scratch_alloc(void** p, size_t bytes, cudaStream_t st) {
 // that cannot stage them stream them, or fall back, as they see fit).
 int cluster_ctas(int64_t rows, int64_t row_bytes, int64_t split_from) {
     constexpr int64_t kSliceBytes = 32768, kFewRows = 64, kFewRowsMinBytes = 32768;
-    if (rows < 1) return 1;
+    // AK_DISABLE_CLUSTERS=1 in the environment (read once) keeps every row on one CTA: for devices
+    // or partitions of one that cannot co-schedule clusters, and for comparing the layouts
+    static const bool disabled = [] {
+        const char* v = getenv("AK_DISABLE_CLUSTERS");
+        return v != nullptr && v[0] != '\0' && v[0] != '0';
+    }();
+    if (rows < 1 || disabled) return 1;
     if (row_bytes > (int64_t)kMaxCluster * kMaxRowSmemBytes) return kMaxCluster;
     int C = 1;
     if (row_bytes >= split_from)

@@ -204,7 +204,17 @@ int dispatch_t(const void* x, const void* gamma, const void* beta, void* y, int6
                cudaStream_t st, int path) {
     const int64_t row_bytes = D * Elem<DT>::kBytes;
     const bool aligned16 = is_aligned(x, 16) && is_aligned(y, 16) && is_aligned(gamma, 16) && is_aligned(beta, 16);
-    if (path == AK_PATH_AUTO) path = layernorm_choose(rows, D, aligned16, DT);
+    if (path == AK_PATH_AUTO) {
+        path = layernorm_choose(rows, D, aligned16, DT);
+        if (path == AK_PATH_CLUSTER) {
+            const int s = dispatch_t<DT>(x, gamma, beta, y, rows, D, eps, st, AK_PATH_CLUSTER);
+            if (s != AK_ERR_CUDA) return s;
+            // a device (or a partition of one) that cannot co-schedule the cluster: one CTA per row
+            // or, for rows beyond its shared memory, the multi-pass kernel
+            (void)cudaGetLastError();
+            path = row_bytes <= 65536 ? AK_PATH_CTA : (row_bytes <= kMaxRowSmemBytes ? AK_PATH_SMEM : AK_PATH_GENERIC);
+        }
+    }
     const float inv_D = 1.0f / (float)D;
     if (path != AK_PATH_GENERIC) {
         if ((row_bytes & 15) != 0) return AK_ERR_SHAPE;
@@ -278,8 +288,10 @@ int dispatch_t(const void* x, const void* gamma, const void* beta, void* y, int6
                 // rows beyond one CTA's shared memory (up to eight CTAs'), and a few long rows (at most
                 // 64 of 32 KiB or more): the covering vectors split over a thread-block cluster
                 const int Cu = cluster_ctas(rows, (int64_t)stage_bytes, kMaxRowSmemBytes + 16);
-                if (same_phase && params4 && Cu > 1 && stage_bytes <= (size_t)kMaxCluster * kMaxRowSmemBytes && rows * Cu <= 2147483647LL)
-                    return launch_cluster_stage<DT, 256>(xs, gs, bs, ys, rows, D, max_nv, Cu, inv_D, eps, st);
+                if (same_phase && params4 && Cu > 1 && stage_bytes <= (size_t)kMaxCluster * kMaxRowSmemBytes && rows * Cu <= 2147483647LL) {
+                    if (launch_cluster_stage<DT, 256>(xs, gs, bs, ys, rows, D, max_nv, Cu, inv_D, eps, st) == AK_OK) return AK_OK;
+                    (void)cudaGetLastError();   // the cluster cannot be co-scheduled here: the kernels below
+                }
                 if (same_phase && params4 && max_nv <= 1024)
                     return launch_regp_vpt<DT, 128, 10, 6>((int)((max_nv + 127) / 128), xs, gs, bs, ys, rows, D, inv_D, eps, st);
                 // ... and of a 512-thread CTA from 3073 to 4096 (in between, the staged kernel below
@@ -309,6 +321,7 @@ int layernorm_choose(int64_t rows, int64_t D, bool aligned16, int dtype) {
     const int64_t bytes = D * dtype_bytes(dtype);
     if (!aligned16 || (bytes & 15) != 0) return AK_PATH_GENERIC;
     if (cluster_ctas(rows, bytes, kClusterFrom) > 1) return AK_PATH_CLUSTER;
+    if (bytes > kMaxRowSmemBytes) return AK_PATH_GENERIC;   // only with clusters switched off
     if (bytes <= 4096) return AK_PATH_WARP;
     if (bytes <= 65536) return AK_PATH_CTA;   // up to 64 KiB the register layout beats the staged one
     return AK_PATH_SMEM;

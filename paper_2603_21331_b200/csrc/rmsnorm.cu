@@ -124,6 +124,7 @@ int rmsnorm_choose(int64_t rows, int64_t D, bool aligned16, int dtype) {
     const int64_t bytes = D * dtype_bytes(dtype);   // row bytes decide the layout
     if (!aligned16 || (bytes & 15) != 0) return AK_PATH_GENERIC;
     if (cluster_ctas(rows, bytes, kClusterFrom) > 1) return AK_PATH_CLUSTER;
+    if (bytes > kMaxRowSmemBytes) return AK_PATH_GENERIC;   // only with clusters switched off
     if (bytes <= 4096) return AK_PATH_WARP;
     if (bytes <= 65536) return AK_PATH_CTA;   // up to 64 KiB the register layout beats the staged one
     return AK_PATH_SMEM;
@@ -136,7 +137,17 @@ int dispatch_t(const void* x, const void* w, void* y, int64_t rows, int64_t D, f
     constexpr int kBytes = Elem<DT>::kBytes;
     const int64_t row_bytes = D * kBytes;
     const bool aligned16 = is_aligned(x, 16) && is_aligned(y, 16) && is_aligned(w, 16);
-    if (path == AK_PATH_AUTO) path = rmsnorm_choose(rows, D, aligned16, DT);
+    if (path == AK_PATH_AUTO) {
+        path = rmsnorm_choose(rows, D, aligned16, DT);
+        if (path == AK_PATH_CLUSTER) {
+            const int s = dispatch_t<DT>(x, w, y, rows, D, eps, st, AK_PATH_CLUSTER);
+            if (s != AK_ERR_CUDA) return s;
+            // a device (or a partition of one) that cannot co-schedule the cluster: one CTA per row
+            // or, for rows beyond its shared memory, the multi-pass kernel
+            (void)cudaGetLastError();
+            path = row_bytes <= 65536 ? AK_PATH_CTA : (row_bytes <= kMaxRowSmemBytes ? AK_PATH_SMEM : AK_PATH_GENERIC);
+        }
+    }
     const float inv_D = 1.0f / (float)D;
     if (path != AK_PATH_GENERIC) {
         if ((row_bytes & 15) != 0) return AK_ERR_SHAPE;
@@ -211,8 +222,10 @@ int dispatch_t(const void* x, const void* w, void* y, int64_t rows, int64_t D, f
                 // rows beyond one CTA's shared memory (up to eight CTAs'), and a few long rows (at most
                 // 64 of 32 KiB or more): the covering vectors split over a thread-block cluster
                 const int Cu = cluster_ctas(rows, (int64_t)stage_bytes, kMaxRowSmemBytes + 16);
-                if (same_phase && is_aligned(w, 4) && Cu > 1 && stage_bytes <= (size_t)kMaxCluster * kMaxRowSmemBytes && rows * Cu <= 2147483647LL)
-                    return launch_cluster_stage<DT, 256>(xs, ws, ys, rows, D, max_nv, Cu, inv_D, eps, st);
+                if (same_phase && is_aligned(w, 4) && Cu > 1 && stage_bytes <= (size_t)kMaxCluster * kMaxRowSmemBytes && rows * Cu <= 2147483647LL) {
+                    if (launch_cluster_stage<DT, 256>(xs, ws, ys, rows, D, max_nv, Cu, inv_D, eps, st) == AK_OK) return AK_OK;
+                    (void)cudaGetLastError();   // the cluster cannot be co-scheduled here: the kernels below
+                }
                 // rows of up to 1024 covering vectors stay in the registers of a 128-thread CTA ...
                 if (same_phase && is_aligned(w, 4) && max_nv <= 1024)
                     return launch_regp_vpt<DT, 128>((int)((max_nv + 127) / 128), xs, ws, ys, rows, D, inv_D, eps, st);

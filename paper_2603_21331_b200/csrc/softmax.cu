@@ -125,7 +125,17 @@ template <int DT>
 int dispatch_t(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st, int path) {
     const int64_t row_bytes = D * Elem<DT>::kBytes;
     const bool aligned16 = is_aligned(x, 16) && is_aligned(y, 16);
-    if (path == AK_PATH_AUTO) path = softmax_choose(rows, D, aligned16, DT);
+    if (path == AK_PATH_AUTO) {
+        path = softmax_choose(rows, D, aligned16, DT);
+        if (path == AK_PATH_CLUSTER) {
+            const int s = dispatch_t<DT>(x, y, rows, D, st, AK_PATH_CLUSTER);
+            if (s != AK_ERR_CUDA) return s;
+            // a device (or a partition of one) that cannot co-schedule the cluster: one CTA per row
+            // or, for rows beyond its shared memory, the multi-pass kernel
+            (void)cudaGetLastError();
+            path = row_bytes <= 16384 ? AK_PATH_CTA : (row_bytes <= kMaxRowSmemBytes ? AK_PATH_SMEM : AK_PATH_GENERIC);
+        }
+    }
     if (path != AK_PATH_GENERIC) {
         if ((row_bytes & 15) != 0) return AK_ERR_SHAPE;
         if (!aligned16) return AK_ERR_ALIGN;
@@ -191,8 +201,11 @@ int dispatch_t(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st,
                 // covering vectors split over a thread-block cluster
                 const int Cu = cluster_ctas(rows, (int64_t)stage_bytes, kMaxRowSmemBytes + 16);
                 if (same_phase && Cu > 1 && stage_bytes <= (size_t)kMaxCluster * kMaxRowSmemBytes && rows * Cu <= 2147483647LL) {
-                    if (rows > 64 && (max_nv + Cu - 1) / Cu <= 2048) return launch_cluster_stage<DT, 128>(xs, ys, rows, D, max_nv, Cu, st);
-                    return launch_cluster_stage<DT, 256>(xs, ys, rows, D, max_nv, Cu, st);
+                    const int s = (rows > 64 && (max_nv + Cu - 1) / Cu <= 2048)
+                                      ? launch_cluster_stage<DT, 128>(xs, ys, rows, D, max_nv, Cu, st)
+                                      : launch_cluster_stage<DT, 256>(xs, ys, rows, D, max_nv, Cu, st);
+                    if (s == AK_OK) return AK_OK;
+                    (void)cudaGetLastError();   // the cluster cannot be co-scheduled here: the kernels below
                 }
                 if (same_phase && stage_bytes <= (size_t)kMaxRowSmemBytes) {
                     if (D <= 8192) return launch_stage<DT, 128>(xs, ys, rows, D, stage_bytes, st);
@@ -217,6 +230,7 @@ int softmax_choose(int64_t rows, int64_t D, bool aligned16, int dtype) {
     const int64_t bytes = D * dtype_bytes(dtype);
     if (!aligned16 || (bytes & 15) != 0) return AK_PATH_GENERIC;
     if (cluster_ctas(rows, bytes, kClusterFrom) > 1) return AK_PATH_CLUSTER;
+    if (bytes > kMaxRowSmemBytes) return AK_PATH_GENERIC;   // only with clusters switched off
     if (bytes <= 4096) return AK_PATH_WARP;
     if (bytes <= 16384) return AK_PATH_CTA;
     return AK_PATH_SMEM;

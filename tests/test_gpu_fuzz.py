@@ -229,3 +229,40 @@ print("capture-first ok")
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     r = subprocess.run([sys.executable, "-c", code], cwd=root, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0 and "capture-first ok" in r.stdout, r.stdout[-2000:] + r.stderr[-4000:]
+
+
+def test_clusters_switched_off_by_the_environment():
+    """AK_DISABLE_CLUSTERS=1 keeps every row on one CTA (the layouts a device that cannot
+    co-schedule clusters falls back to): same results within tolerance, long rows included."""
+    import os
+    import subprocess
+    import sys
+    code = r"""
+import numpy as np, torch
+import oracle
+import paper_2603_21331_b200 as ak
+from paper_2603_21331_b200 import synth
+dev = "cuda"
+def widen(t):
+    bits = t.cpu().view(torch.int16).numpy().view(np.uint16)
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+for rows, D in ((5, 16384), (3, 65536), (2, 131072), (3, 128257), (4, 40001)):
+    assert ak.ak_softmax_choose_path(rows, D, True) != ak.AK_PATH_CLUSTER
+    x, w = synth.rmsnorm_inputs(rows, D, 700 + D)
+    y = ak.ak_rmsnorm_fwd(x.to(dev), w.to(dev))
+    ref = oracle.rmsnorm(synth.to_bits(x), synth.to_bits(w), 1e-6)
+    assert (np.abs(widen(y) - ref) / np.maximum(1.0, np.abs(ref))).max() <= 1.6e-2
+    xs = synth.softmax_inputs(rows, D, 800 + D)
+    ys = ak.ak_softmax_fwd(xs.to(dev))
+    refs = oracle.softmax(synth.to_bits(xs))
+    assert np.abs(widen(ys) - refs).max() <= 1.6e-2
+    xl, g, b = synth.layernorm_inputs(rows, D, 900 + D)
+    yl = ak.ak_layernorm_fwd(xl.to(dev), g.to(dev), b.to(dev))
+    refl = oracle.layernorm(synth.to_bits(xl), synth.to_bits(g), synth.to_bits(b), 1e-5)
+    assert (np.abs(widen(yl) - refl) / np.maximum(1.0, np.abs(refl))).max() <= 1.6e-2
+print("no clusters ok")
+"""
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, AK_DISABLE_CLUSTERS="1")
+    r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0 and "no clusters ok" in r.stdout, r.stdout[-2000:] + r.stderr[-4000:]
