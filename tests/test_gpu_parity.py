@@ -178,10 +178,37 @@ def test_softmax_ieee_conventions():
     x[2, 5] = float("nan")            # NaN -> NaN row
     x[3, :] = torch.arange(24) * 0.25  # ordinary row
     ref = oracle.softmax(synth.to_bits(x))
-    for path in (WARP, CTA, GEN, SMEM):
+    for path in (WARP, CTA, GEN, SMEM, CLUSTER):
         y = ak.ak_softmax_fwd(x.to(DEV), path=path)
         torch.cuda.synchronize()
         assert_bf16_close(y, ref, f"softmax conventions path {path}")
+
+
+@pytest.mark.parametrize("D", [65544, 131072, 128257, 1048576])
+def test_ieee_conventions_on_rows_split_over_clusters(D):
+    """The same conventions where a row is spread over several CTAs (staged slices, aligned and
+    not, and streamed slices): a NaN, a +inf or a fully masked row in ONE slice decides the whole
+    row; RMSNorm and LayerNorm rows with an inf or NaN element come out as the checker says."""
+    x = synth.softmax_inputs(5, D, synth.case_seed(17, D), mask_frac=0.0)
+    x[0, :] = float("-inf")                    # fully masked row -> NaN
+    x[1, D - 3] = float("inf")                 # +inf in the last slice -> NaN row
+    x[2, 5] = float("nan")                     # NaN in the first slice -> NaN row
+    x[3, D // 2:] = float("-inf")              # whole slices masked: exact zeros there
+    ref = oracle.softmax(synth.to_bits(x))
+    y = ak.ak_softmax_fwd(x.to(DEV))
+    torch.cuda.synchronize()
+    assert_bf16_close(y, ref, f"softmax conventions D={D}")
+    assert bool((y[3, D // 2:].view(torch.int16) == 0).all())
+    xn, w = synth.rmsnorm_inputs(4, D, synth.case_seed(18, D))
+    _, g, b = synth.layernorm_inputs(1, D, 81)
+    xn[1, D - 2] = float("inf")
+    xn[2, 7] = float("nan")
+    yr = ak.ak_rmsnorm_fwd(xn.to(DEV), w.to(DEV))
+    yl = ak.ak_layernorm_fwd(xn.to(DEV), g.to(DEV), b.to(DEV))
+    torch.cuda.synchronize()
+    assert_bf16_close(yr, oracle.rmsnorm(synth.to_bits(xn), synth.to_bits(w), 1e-6), f"rmsnorm conventions D={D}")
+    assert_bf16_close(yl, oracle.layernorm(synth.to_bits(xn), synth.to_bits(g), synth.to_bits(b), 1e-5),
+                      f"layernorm conventions D={D}", tight=False)
 
 
 @pytest.mark.parametrize("kind", synth.ADVERSARIAL_KINDS)
