@@ -203,7 +203,7 @@ __device__ __forceinline__ float cta_max(float v, float* slots, int phase) {
 // ---------------------------------------------------------------- bulk (TMA) copies into shared memory
 // One elected thread asks the copy engine for a whole contiguous span (a row); the bytes
 // land in shared memory without passing through registers and an mbarrier counts them in.
-// Source, destination and size must be multiples of 16 bytes.  No multicast is used.
+// Source, destination and size must be multiples of 16 bytes.  Every copy has one destination CTA.
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, int arrivals) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals));
