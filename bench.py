@@ -538,7 +538,7 @@ def time_op(fn_for_set, nsets, iters=200, warmup=20):
     b.record()
     torch.cuda.synchronize()
     est_us = max(a.elapsed_time(b) * 1e3 / nsets, 1.0)
-    per_graph = nsets * max(1, int(np.ceil(300.0 / est_us / nsets)))
+    per_graph = nsets * max(1, int(np.ceil(float(os.environ.get('AK_SAMPLE_US', 300.0)) / est_us / nsets)))
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
     graph = torch.cuda.CUDAGraph()

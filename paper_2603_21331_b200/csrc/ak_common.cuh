@@ -149,6 +149,18 @@ __device__ __forceinline__ void st_stream(uint4* p, uint4 v) { __stcs(p, v); }
 __device__ __forceinline__ uint16_t ld_stream_u16(const uint16_t* p) { return __ldcs(p); }
 __device__ __forceinline__ void st_stream_u16(uint16_t* p, uint16_t v) { __stcs(p, v); }
 
+// Ask for the 128-byte line at p to be brought into L2.  No data is returned and nothing is
+// observed, so it may be issued where a load may not (before griddepcontrol.wait).
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+// blockIdx.x through an opaque read: the compiler cannot merge it with an earlier use of
+// blockIdx.x, so values derived from the earlier one need not live across the code in between.
+__device__ __forceinline__ unsigned cta_id_x() {
+    unsigned r;
+    asm volatile("mov.u32 %0, %%ctaid.x;" : "=r"(r));
+    return r;
+}
+
 // exp2 on the SFU (max relative error 2^-22; ex2(-inf) = 0, ex2(NaN) = NaN).
 __device__ __forceinline__ float fast_exp2(float t) {
     float r;

@@ -29,9 +29,10 @@ template <int DT>
 int launch_finish(const typename XElem<DT>::type* logits, const int64_t* targets, int64_t ignore_index, const float2* partial,
                   int nsplit, float* loss_rows, int64_t rows, int64_t V, float* out_mean, double* out_pair,
                   cudaStream_t st, bool dependent) {
+    const bool many = rows > kFinishSmallRows;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(1);
-    cfg.blockDim = dim3(kFinishThreads);
+    cfg.blockDim = dim3(many ? kFinishThreadsMany : kFinishThreads);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -39,8 +40,10 @@ int launch_finish(const typename XElem<DT>::type* logits, const int64_t* targets
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = dependent ? 1 : 0;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, xent_finish_kernel<DT>, logits, targets, ignore_index, partial, nsplit,
-                                       loss_rows, rows, V, out_mean, out_pair);
+    cudaError_t e = many ? cudaLaunchKernelEx(&cfg, xent_finish_kernel<DT, kFinishThreadsMany>, logits, targets,
+                                              ignore_index, partial, nsplit, loss_rows, rows, V, out_mean, out_pair)
+                         : cudaLaunchKernelEx(&cfg, xent_finish_kernel<DT, kFinishThreads>, logits, targets,
+                                              ignore_index, partial, nsplit, loss_rows, rows, V, out_mean, out_pair);
     count_launch();
     return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
@@ -98,10 +101,13 @@ int dispatch_t(const void* logits, const int64_t* targets, int64_t ignore_index,
         return launch_finish<DT>(lg, targets, ignore_index, nullptr, 0, loss_rows, 0, V, loss_mean, nullptr, st, false);
     }
     if (path == AK_XENT_ROW) {
-        xent_row_kernel<kRowUnroll, kPoly, kRowMinCtas, kRowThreads, DT><<<(unsigned)rows, kRowThreads, 0, st>>>(
-            lg, targets, ignore_index, loss_rows, V);
+        // fp32 logits: seven CTAs per SM (72 registers); at eight the compiler spills
+        constexpr int kMinCtas = (DT == AK_DTYPE_F32) ? kRowMinCtas - 1 : kRowMinCtas;
+        const cudaError_t e = launch_dependent(xent_row_kernel<kRowUnroll, kPoly, kMinCtas, kRowThreads, DT>,
+                                               dim3((unsigned)rows), dim3(kRowThreads), 0, st, lg, targets, ignore_index,
+                                               loss_rows, V, kMinCtas * sm_count());
         count_launch();
-        if (cudaGetLastError() != cudaSuccess) return AK_ERR_CUDA;
+        if (e != cudaSuccess) return AK_ERR_CUDA;
         if (loss_mean == nullptr) return AK_OK;
         return launch_finish<DT>(lg, targets, ignore_index, nullptr, 0, loss_rows, rows, V, loss_mean, nullptr, st, true);
     }

@@ -159,10 +159,12 @@ __device__ __forceinline__ void absorb_scalar(Online& o, float v) {
 // moving pointer); a single masked batch finishes the slice.
 template <int DT>
 struct Slice {
-    const typename XElem<DT>::type* p;
-    int64_t n, head, nbody, tail0, nfull;
-    const uint4* body;
-    int rest;  // vectors in the masked last batch, < T * UNROLL
+    const typename XElem<DT>::type* p;   // first element
+    int64_t n;                           // elements
+    int head, ntail;                     // single elements before / after the aligned body (< kPerVec each)
+    int rest;                            // vectors in the masked last batch, < T * UNROLL
+    const uint4* body;                   // first aligned vector
+    const uint4* full_end;               // end of the full batches (== body when there is none)
 };
 template <int UNROLL, int T, int DT>
 __device__ __forceinline__ Slice<DT> make_slice(const typename XElem<DT>::type* __restrict__ xr, int64_t begin, int64_t end) {
@@ -171,28 +173,44 @@ __device__ __forceinline__ Slice<DT> make_slice(const typename XElem<DT>::type* 
     Slice<DT> s;
     s.p = xr + begin;
     s.n = end - begin;
-    s.head = (PV - (int)((reinterpret_cast<uintptr_t>(s.p) >> LOG_BYTES) & (PV - 1))) & (PV - 1);
-    if (s.head > s.n) s.head = s.n;
-    s.nbody = (s.n - s.head) >> LOG_PV;
-    s.tail0 = s.head + (s.nbody << LOG_PV);
-    s.body = reinterpret_cast<const uint4*>(s.p + s.head);
-    s.nfull = s.nbody / ((int64_t)T * UNROLL);
-    s.rest = (int)(s.nbody - s.nfull * T * UNROLL);
+    int64_t head = (PV - (int)((reinterpret_cast<uintptr_t>(s.p) >> LOG_BYTES) & (PV - 1))) & (PV - 1);
+    if (head > s.n) head = s.n;
+    const int64_t nbody = (s.n - head) >> LOG_PV;
+    s.head = (int)head;
+    s.ntail = (int)(s.n - head - (nbody << LOG_PV));
+    s.body = reinterpret_cast<const uint4*>(s.p + head);
+    const int64_t nfull = nbody / ((int64_t)T * UNROLL);
+    s.rest = (int)(nbody - nfull * T * UNROLL);
+    s.full_end = s.body + nfull * T * UNROLL;
     return s;
 }
-// The slice's first batch (full if there is a full batch, otherwise the masked one).
+// The masked batch holds `rest` vectors: thread i owns vectors i, i + T, ... below `rest`, so only
+// the first ceil(rest / T) of a thread's UNROLL slots can hold data, the same number for every
+// thread of the CTA.  Loading and absorbing stop there (a row of 50304 bf16 is 6.14 batches of
+// 16 KiB: its seventh batch fills 2 of 8 slots); the skipped slots would have added exact zeros.
+template <int T>
+__device__ __forceinline__ int masked_slots(int rest) { return (rest + T - 1) / T; }
+template <int UNROLL, int T, int DT>
+__device__ __forceinline__ void load_masked_batch(const uint4* src, int rest, int nk, uint4 (&q)[UNROLL]) {
+#pragma unroll
+    for (int k = 0; k < UNROLL; ++k) {
+        if (k < nk) {
+            const int i = (int)threadIdx.x + k * T;
+            q[k] = (i < rest) ? ld_stream(src + k * T) : xneg_inf_vec<DT>();
+        }
+    }
+}
+// The slice's first batch (full if there is a full batch, otherwise the masked one; slot 0 is
+// always defined, all padding when the slice has no body).
 template <int UNROLL, int T, int DT>
 __device__ __forceinline__ void load_first_batch(const Slice<DT>& s, uint4 (&q)[UNROLL]) {
     const uint4* src = s.body + threadIdx.x;
-    if (s.nfull > 0) {
+    if (s.full_end != s.body) {
 #pragma unroll
         for (int k = 0; k < UNROLL; ++k) q[k] = ld_stream(src + k * T);
     } else {
-#pragma unroll
-        for (int k = 0; k < UNROLL; ++k) {
-            const int i = (int)threadIdx.x + k * T;
-            q[k] = (i < s.rest) ? ld_stream(src + k * T) : xneg_inf_vec<DT>();
-        }
+        q[0] = xneg_inf_vec<DT>();
+        load_masked_batch<UNROLL, T, DT>(src, s.rest, masked_slots<T>(s.rest), q);
     }
 }
 
@@ -214,23 +232,39 @@ __device__ __forceinline__ void slice_lse(const Slice<DT>& sl, uint4 (&q)[UNROLL
         for (int k = 1; k < UNROLL; ++k) acc = add2(acc, sumexp_v<POLY, DT>(v[k], l2, nmf2));
         o.s2 = add2(o.s2, acc);
     };
-    absorb_batch(q);  // batch 0 (all padding when the slice has no body)
-    const uint4* src = sl.body + threadIdx.x + T * UNROLL;
-    for (int64_t b = 1; b < sl.nfull; ++b, src += T * UNROLL) {
+    // slots 0 .. nk - 1 only (nk >= 1, uniform over the CTA)
+    auto absorb_masked = [&](const uint4 (&v)[UNROLL], int nk) {
+        uint32_t mx = xmax_v<DT>(v[0]);
 #pragma unroll
-        for (int k = 0; k < UNROLL; ++k) q[k] = ld_stream(src + k * T);
+        for (int k = 1; k < UNROLL; ++k)
+            if (k < nk) mx = xmax_w<DT>(mx, xmax_v<DT>(v[k]));
+        raise_max(o, xhmax_of<DT>(mx));
+        const f32x2 nmf2 = pack2(-o.mf, -o.mf);
+        f32x2 acc = sumexp_v<POLY, DT>(v[0], l2, nmf2);
+#pragma unroll
+        for (int k = 1; k < UNROLL; ++k)
+            if (k < nk) acc = add2(acc, sumexp_v<POLY, DT>(v[k], l2, nmf2));
+        o.s2 = add2(o.s2, acc);
+    };
+    const int nk = masked_slots<T>(sl.rest);
+    if (sl.full_end != sl.body) {
         absorb_batch(q);
-    }
-    if (sl.nfull > 0 && sl.rest > 0) {
+        // this thread's vector k of batch b sits at body + b * T * UNROLL + k * T + threadIdx.x
+        const uint4* src = sl.body + threadIdx.x + T * UNROLL;
+        for (; src < sl.full_end; src += T * UNROLL) {
 #pragma unroll
-        for (int k = 0; k < UNROLL; ++k) {
-            const int i = (int)threadIdx.x + k * T;
-            q[k] = (i < sl.rest) ? ld_stream(src + k * T) : xneg_inf_vec<DT>();
+            for (int k = 0; k < UNROLL; ++k) q[k] = ld_stream(src + k * T);
+            absorb_batch(q);
         }
-        absorb_batch(q);
+        if (nk > 0) {
+            load_masked_batch<UNROLL, T, DT>(sl.full_end + threadIdx.x, sl.rest, nk, q);
+            absorb_masked(q, nk);
+        }
+    } else {
+        absorb_masked(q, nk > 0 ? nk : 1);   // the first batch was the masked one
     }
-    if ((int64_t)threadIdx.x < sl.head) absorb_scalar(o, xload<DT>(sl.p + threadIdx.x));
-    if (sl.tail0 + threadIdx.x < sl.n) absorb_scalar(o, xload<DT>(sl.p + sl.tail0 + threadIdx.x));
+    if ((int)threadIdx.x < sl.head) absorb_scalar(o, xload<DT>(sl.p + threadIdx.x));
+    if ((int)threadIdx.x < sl.ntail) absorb_scalar(o, xload<DT>(sl.p + (sl.n - sl.ntail) + threadIdx.x));
 
     // NaN must win the max: fmaxf in cta_max would drop it, so it travels as +inf plus a flag
     const bool has_nan = (o.m != o.m) || (o.m == INFINITY);  // +inf makes inf - inf: NaN row as well
@@ -255,29 +289,49 @@ __device__ __forceinline__ float finish_loss(float M, float S, float xt) {
 }
 
 // ------------------------------------------------------------------ one CTA per row
+// Launched as a programmatic dependent of whatever precedes it in the stream: nothing is read
+// or written before griddepcontrol.wait, and its own dependents (the finish kernel) are let in
+// only after the wait, so that they may read this kernel's inputs before their own wait.
 template <int UNROLL, int POLY, int MINB = 1, int T = kXentThreads, int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(T, MINB)
 xent_row_kernel(const typename XElem<DT>::type* __restrict__ logits, const int64_t* __restrict__ targets,
-                int64_t ignore_index, float* __restrict__ loss_rows, int64_t V) {
+                int64_t ignore_index, float* __restrict__ loss_rows, int64_t V, int first_wave) {
     __shared__ float slots[2 * kWarp];
+    if (blockIdx.x < first_wave) {
+        // The CTAs of the first wave (as many as the device holds at once) become resident while
+        // the grids before this one drain, and would idle at the wait.  Meanwhile they ask for the
+        // first 128 bytes per thread of their row (one batch is eight times that) and for the
+        // target to be brought into L2: a prefetch reads nothing architecturally, so it may precede
+        // the wait.  Later CTAs start on a busy machine and skip it; prefetching more than this,
+        // or in every CTA, measured slower.
+        const int64_t row0 = blockIdx.x;
+        const char* head = reinterpret_cast<const char*>(logits + row0 * V);
+        const int64_t left = ((int64_t)gridDim.x - row0) * V * (int64_t)sizeof(typename XElem<DT>::type);
+        const int64_t off = (int64_t)threadIdx.x * 128;
+        if (off < left) prefetch_l2(head + off);
+        if (threadIdx.x == 0) prefetch_l2(targets + row0);
+    }
+    pdl_wait();
     pdl_launch_dependents();
-    const int64_t row = blockIdx.x;
+    const int64_t row = cta_id_x();   // read again, so that nothing computed above stays in registers
     const typename XElem<DT>::type* xr = logits + row * V;
     const int64_t t = targets[row];
-    if (t == ignore_index || t < 0 || t >= V) {  // uniform across the CTA: nothing is read
-        if (threadIdx.x == 0) loss_rows[row] = (t == ignore_index) ? 0.0f : __int_as_float(0x7fc00000);
-        return;
+    // (The compiler keeps this kernel inside its 64 registers without spilling only in this
+    // if / else form; an early return for the rows that are not read costs a spill slot.)
+    if (t != ignore_index && t >= 0 && t < V) {  // uniform across the CTA
+        // (Requesting the first batch before the target is known was measured: no gain, and
+        // ignored rows would be touched.)
+        const Slice<DT> sl = make_slice<UNROLL, T, DT>(xr, 0, V);
+        uint4 q[UNROLL];
+        load_first_batch<UNROLL, T, DT>(sl, q);
+        // the target logit is fetched now, under the row's own traffic, not after the reduction
+        const float xt = (threadIdx.x == 0) ? xread<DT>(xr + t) : 0.0f;
+        float M, S;
+        slice_lse<UNROLL, POLY, T, DT>(sl, q, slots, M, S);
+        if (threadIdx.x == 0) loss_rows[row] = finish_loss(M, S, xt);
+    } else if (threadIdx.x == 0) {   // nothing of the row is read
+        loss_rows[row] = (t == ignore_index) ? 0.0f : __int_as_float(0x7fc00000);
     }
-    // (Requesting the first batch before the target is known was measured: no gain, and
-    // ignored rows would be touched.)
-    const Slice<DT> sl = make_slice<UNROLL, T, DT>(xr, 0, V);
-    uint4 q[UNROLL];
-    load_first_batch<UNROLL, T, DT>(sl, q);
-    // the target logit is fetched now, under the row's own traffic, not after the reduction
-    const float xt = (threadIdx.x == 0) ? xread<DT>(xr + t) : 0.0f;
-    float M, S;
-    slice_lse<UNROLL, POLY, T, DT>(sl, q, slots, M, S);
-    if (threadIdx.x == 0) loss_rows[row] = finish_loss(M, S, xt);
 }
 
 // ------------------------------------------------------------------ split row, phase 1
@@ -288,6 +342,7 @@ __global__ void __launch_bounds__(kXentThreads)
 xent_split_kernel(const typename XElem<DT>::type* __restrict__ logits, const int64_t* __restrict__ targets,
                   int64_t ignore_index, float2* __restrict__ partial, int64_t V, int nsplit) {
     __shared__ float slots[2 * kWarp];
+    pdl_wait();
     pdl_launch_dependents();
     const int64_t row = blockIdx.y;
     const int sp = blockIdx.x;
@@ -306,12 +361,20 @@ xent_split_kernel(const typename XElem<DT>::type* __restrict__ logits, const int
 }
 
 // ------------------------------------------------------------------ finish: merge + mean
-// One CTA, launched as a programmatic dependent of the streaming kernel.  Thread i owns
-// rows i, i + T, i + 2T, ...: for the split layout it first merges the row's partials in
-// split order and writes the loss; then (if out_mean / out_pair is given) it adds its
-// rows' counted losses in fp64 in that order, and a fixed shuffle + shared-memory tree
-// adds the threads.  out_mean = sum / count (0/0 = NaN); out_pair = {sum, count}.
-constexpr int kFinishThreads = 1024;
+// One CTA, launched as a programmatic dependent of the streaming kernel.  For the split layout
+// thread i first merges the partials of rows i, i + T, ... in split order and writes the losses.
+// Then (if out_mean / out_pair is given) the counted losses are added in fp64 in ONE fixed order,
+// whatever the CTA's size T: "virtual" thread v of kFinishVirtual = 1024 adds rows v, v + 1024, ...
+// in that order; a butterfly adds the 32 lanes of each virtual warp; a second butterfly adds the
+// 32 warp sums.  Physical thread i plays virtual threads i, i + T, ...: its lane is their lane,
+// so the butterflies are the same and every T gives the same bits.  A small CTA (T = 256) finds a
+// free slot on an SM, and lets the next kernel of the stream in, while the streaming kernel's
+// last CTAs are still running; a 1024-thread CTA with its registers needs a whole empty SM.
+// out_mean = sum / count (0/0 = NaN); out_pair = {sum, count}.
+constexpr int kFinishVirtual = 1024;
+constexpr int kFinishThreads = 256;        // up to kFinishSmallRows rows
+constexpr int kFinishThreadsMany = 1024;
+constexpr int64_t kFinishSmallRows = 8192;
 
 __device__ __forceinline__ double warp_sum_f64(double v) {
 #pragma unroll
@@ -319,25 +382,39 @@ __device__ __forceinline__ double warp_sum_f64(double v) {
     return v;
 }
 
-template <int DT = AK_DTYPE_BF16>
-__global__ void __launch_bounds__(kFinishThreads)
+template <int DT, int T>
+__global__ void __launch_bounds__(T)
 xent_finish_kernel(const typename XElem<DT>::type* __restrict__ logits, const int64_t* __restrict__ targets,
                    int64_t ignore_index, const float2* __restrict__ partial, int nsplit,
                    float* __restrict__ loss_rows, int64_t rows, int64_t V,
                    float* __restrict__ out_mean, double* __restrict__ out_pair) {
-    constexpr int T = kFinishThreads;
-    __shared__ double ssum[T / kWarp];
-    __shared__ double scnt[T / kWarp];
-    // The targets are inputs, not results of the streaming kernel: which of this thread's first
-    // sixteen rows count is worked out before the wait, while that kernel is still running.
-    constexpr int B = 16;
+    constexpr int J = kFinishVirtual / T;   // virtual threads per thread
+    constexpr int KB = 16 / J;              // 16 rows per thread and batch: independent loads in flight
+    __shared__ double ssum[kFinishVirtual / kWarp];
+    __shared__ int scnt[T / kWarp];
+    pdl_launch_dependents();   // the next kernel may take free slots now (it reads nothing before its own wait)
+    const bool want_sum = out_mean != nullptr || out_pair != nullptr;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // The targets are inputs of the streaming kernel, final before it let this kernel in: which
+    // rows count is worked out before the wait, while that kernel is still running.  The first
+    // batch's flags are kept; later batches (more than 1024 * KB rows) read their targets again.
     uint32_t counted0 = 0;
-    if (out_mean != nullptr || out_pair != nullptr) {
+    int n_counted = 0;
+    if (want_sum) {
+        for (int64_t base = 0; base < rows; base += (int64_t)kFinishVirtual * KB) {
 #pragma unroll
-        for (int k = 0; k < B; ++k) {
-            const int64_t r = threadIdx.x + (int64_t)k * T;
-            if (r < rows && targets[r] != ignore_index) counted0 |= 1u << k;
+            for (int k = 0; k < KB; ++k)
+#pragma unroll
+                for (int j = 0; j < J; ++j) {
+                    const int64_t r = base + (int64_t)k * kFinishVirtual + j * T + threadIdx.x;
+                    if (r < rows && targets[r] != ignore_index) {
+                        ++n_counted;
+                        if (base == 0) counted0 |= 1u << (k * J + j);
+                    }
+                }
         }
+        n_counted = __reduce_add_sync(0xffffffffu, n_counted);
+        if (lane == 0) scnt[warp] = n_counted;
     }
     pdl_wait();  // everything the streaming kernel wrote is visible from here on
     if (nsplit > 0) {
@@ -362,55 +439,58 @@ xent_finish_kernel(const typename XElem<DT>::type* __restrict__ logits, const in
             }
             loss_rows[r] = loss;
         }
+        // virtual thread v = i + j * T reads rows written by thread (v mod T) = i: its own
     }
-    if (out_mean == nullptr && out_pair == nullptr) return;
-    // Mean: batches of independent loads (a lone CTA is latency-bound, so sixteen rows are in
-    // flight per thread), added in row order per thread.  A thread re-reads only rows it
-    // wrote itself above, so program order makes them visible.
-    double acc = 0.0, cnt = 0.0;
+    if (!want_sum) return;
+    double acc[J];
+#pragma unroll
+    for (int j = 0; j < J; ++j) acc[j] = 0.0;
     {   // the first batch: the counted rows are known already
-        float ll[B];
+        float ll[KB][J];
 #pragma unroll
-        for (int k = 0; k < B; ++k) {
-            const int64_t r = threadIdx.x + (int64_t)k * T;
-            ll[k] = (r < rows) ? __ldcg(loss_rows + r) : 0.0f;  // L2 read: written by the grid we depend on
-        }
+        for (int k = 0; k < KB; ++k)
 #pragma unroll
-        for (int k = 0; k < B; ++k) {
-            if (counted0 & (1u << k)) {
-                acc += (double)ll[k];
-                cnt += 1.0;
+            for (int j = 0; j < J; ++j) {
+                const int64_t r = (int64_t)k * kFinishVirtual + j * T + threadIdx.x;
+                ll[k][j] = (r < rows) ? __ldcg(loss_rows + r) : 0.0f;  // L2: written by the grid we depend on
             }
-        }
+#pragma unroll
+        for (int k = 0; k < KB; ++k)
+#pragma unroll
+            for (int j = 0; j < J; ++j)
+                if (counted0 & (1u << (k * J + j))) acc[j] += (double)ll[k][j];
     }
-    for (int64_t base = threadIdx.x + (int64_t)T * B; base < rows; base += (int64_t)T * B) {
-        int64_t tt[B];
-        float ll[B];
+    for (int64_t base = (int64_t)kFinishVirtual * KB; base < rows; base += (int64_t)kFinishVirtual * KB) {
+        int64_t tt[KB][J];
+        float ll[KB][J];
 #pragma unroll
-        for (int k = 0; k < B; ++k) {
-            const int64_t r = base + (int64_t)k * T;
-            tt[k] = (r < rows) ? targets[r] : ignore_index;
-            ll[k] = (r < rows) ? __ldcg(loss_rows + r) : 0.0f;
-        }
+        for (int k = 0; k < KB; ++k)
 #pragma unroll
-        for (int k = 0; k < B; ++k) {
-            if (tt[k] != ignore_index) {
-                acc += (double)ll[k];
-                cnt += 1.0;
+            for (int j = 0; j < J; ++j) {
+                const int64_t r = base + (int64_t)k * kFinishVirtual + j * T + threadIdx.x;
+                tt[k][j] = (r < rows) ? targets[r] : ignore_index;
+                ll[k][j] = (r < rows) ? __ldcg(loss_rows + r) : 0.0f;
             }
-        }
+#pragma unroll
+        for (int k = 0; k < KB; ++k)
+#pragma unroll
+            for (int j = 0; j < J; ++j)
+                if (tt[k][j] != ignore_index) acc[j] += (double)ll[k][j];
     }
-    acc = warp_sum_f64(acc);
-    cnt = warp_sum_f64(cnt);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (lane == 0) { ssum[warp] = acc; scnt[warp] = cnt; }
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+        const double v = warp_sum_f64(acc[j]);
+        if (lane == 0) ssum[warp + j * (T / kWarp)] = v;
+    }
     __syncthreads();
     if (warp == 0) {
-        acc = warp_sum_f64(ssum[lane]);
-        cnt = warp_sum_f64(scnt[lane]);
+        const double total = warp_sum_f64(ssum[lane]);
+        int c = (lane < T / kWarp) ? scnt[lane] : 0;
+        c = __reduce_add_sync(0xffffffffu, c);
         if (lane == 0) {
-            if (out_mean) out_mean[0] = (cnt > 0.0) ? (float)(acc / cnt) : __int_as_float(0x7fc00000);
-            if (out_pair) { out_pair[0] = acc; out_pair[1] = cnt; }
+            const double cnt = (double)c;
+            if (out_mean) out_mean[0] = (cnt > 0.0) ? (float)(total / cnt) : __int_as_float(0x7fc00000);
+            if (out_pair) { out_pair[0] = total; out_pair[1] = cnt; }
         }
     }
 }

@@ -82,8 +82,12 @@ extern "C" int ak_xent_fwd_static(const void* logits, const int64_t* targets, in
         return AK_OK;
     }
     // merge the slices in split order, write the losses, then the fixed-order mean
-    xent_finish_kernel<AK_DTYPE_BF16><<<1, kFinishThreads, 0, st>>>(lg, targets, ignore_index, scratch, rows > 0 ? nsplit : 0,
-                                                    loss_rows, rows, V, loss_mean, nullptr);
+    if (rows > kFinishSmallRows)
+        xent_finish_kernel<AK_DTYPE_BF16, kFinishThreadsMany><<<1, kFinishThreadsMany, 0, st>>>(
+            lg, targets, ignore_index, scratch, nsplit, loss_rows, rows, V, loss_mean, nullptr);
+    else
+        xent_finish_kernel<AK_DTYPE_BF16, kFinishThreads><<<1, kFinishThreads, 0, st>>>(
+            lg, targets, ignore_index, scratch, rows > 0 ? nsplit : 0, loss_rows, rows, V, loss_mean, nullptr);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }

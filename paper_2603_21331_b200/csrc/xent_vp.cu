@@ -30,26 +30,27 @@ xent_vp_partial_kernel(const typename XElem<DT>::type* __restrict__ logits, cons
     const int64_t row = blockIdx.x;
     const int sp = blockIdx.y;
     const int64_t t = targets[row];
-    if (t == ignore_index || t < 0 || t >= V_total) return;
-    const typename XElem<DT>::type* xr = logits + row * V_local;
-    const int64_t groups = (V_local + 7) >> 3;
-    int64_t begin = ((groups * sp) / nsplit) << 3;
-    int64_t end = ((groups * (sp + 1)) / nsplit) << 3;
-    if (end > V_local) end = V_local;
-    const Slice<DT> sl = make_slice<UNROLL, T, DT>(xr, begin, end);
-    uint4 q[UNROLL];
-    load_first_batch<UNROLL, T, DT>(sl, q);
-    float2 mine = make_float2(0.0f, 0.0f);
-    if (sp == 0 && threadIdx.x == 0) {
-        const int64_t tl = t - vocab_start;
-        if (tl >= 0 && tl < V_local) mine = make_float2(xread<DT>(xr + tl), 1.0f);
-    }
-    float M, S;
-    slice_lse<UNROLL, POLY, T, DT>(sl, q, slots, M, S);
-    if (threadIdx.x == 0) {
-        float2* pr = part + row * (nsplit + 1);
-        pr[sp] = make_float2(M, S);
-        if (sp == 0) pr[nsplit] = mine;
+    if (t != ignore_index && t >= 0 && t < V_total) {   // (this form, not an early return, keeps the compiler from spilling)
+        const typename XElem<DT>::type* xr = logits + row * V_local;
+        const int64_t groups = (V_local + 7) >> 3;
+        int64_t begin = ((groups * sp) / nsplit) << 3;
+        int64_t end = ((groups * (sp + 1)) / nsplit) << 3;
+        if (end > V_local) end = V_local;
+        const Slice<DT> sl = make_slice<UNROLL, T, DT>(xr, begin, end);
+        uint4 q[UNROLL];
+        load_first_batch<UNROLL, T, DT>(sl, q);
+        float2 mine = make_float2(0.0f, 0.0f);
+        if (sp == 0 && threadIdx.x == 0) {
+            const int64_t tl = t - vocab_start;
+            if (tl >= 0 && tl < V_local) mine = make_float2(xread<DT>(xr + tl), 1.0f);
+        }
+        float M, S;
+        slice_lse<UNROLL, POLY, T, DT>(sl, q, slots, M, S);
+        if (threadIdx.x == 0) {
+            float2* pr = part + row * (nsplit + 1);
+            pr[sp] = make_float2(M, S);
+            if (sp == 0) pr[nsplit] = mine;
+        }
     }
 }
 
@@ -119,9 +120,11 @@ int partial_t(const void* logits, const int64_t* targets, int64_t ignore_index, 
     using elem_t = typename XElem<DT>::type;
     const elem_t* lg = static_cast<const elem_t*>(logits);
     const dim3 grid((unsigned)rows, (unsigned)nsplit);
-    if (nsplit == 1)   // the single-GPU row layout: 128 threads x 8 vectors, 64 registers
-        xent_vp_partial_kernel<8, 2, 8, 128, DT><<<grid, 128, 0, st>>>(lg, targets, ignore_index, vocab_start, V_total,
-                                                                      part, V_local, nsplit);
+    // the single-GPU row layout: 128 threads x 8 vectors, 64 registers (fp32: 72, seven CTAs per SM)
+    constexpr int kMinCtas = (DT == AK_DTYPE_F32) ? 7 : 8;
+    if (nsplit == 1)
+        xent_vp_partial_kernel<8, 2, kMinCtas, 128, DT><<<grid, 128, 0, st>>>(lg, targets, ignore_index, vocab_start,
+                                                                             V_total, part, V_local, nsplit);
     else
         xent_vp_partial_kernel<4, 2, 1, kXentThreads, DT><<<grid, kXentThreads, 0, st>>>(
             lg, targets, ignore_index, vocab_start, V_total, part, V_local, nsplit);
