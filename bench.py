@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the row-reduction hot path (RMSNorm, softmax, cross-entropy forward).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--sweep]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--sweep [--out FILE]]
 
 One "step" is one pass of the whole hot path over one batch of synthetic bf16 input:
 RMSNorm [8192, 8192], last-dim softmax [16384, 8192] and fused cross-entropy
@@ -15,8 +15,9 @@ weak scaling, no data-path collective) and the cross-entropy mean is made global
 16-byte all-gather per step.
 
 ``--impl reference`` times the fp64 CPU checker on the host cores on a bounded sample of
-the same workload.  ``--sweep`` additionally times every benchmark shape one by one and
-writes a table (sweep.json, in the scratch output folder; not part of the JSON line contract).
+the same workload.  ``--sweep`` additionally times every benchmark shape one by one, beside a
+plain copy (or read) of the same size, prints the table to stderr and writes it to the file
+``--out`` names (not part of the JSON line contract).
 """
 from __future__ import annotations
 
@@ -74,10 +75,14 @@ def algorithmic_bytes(op, rows, D, n_valid=None):
 
 # --------------------------------------------------------------------------- clocks
 class ClockSampler:
-    """Polls NVML for SM clock and throttle reasons while the timed region runs."""
+    """Polls NVML for SM clock and throttle reasons while a timed region runs.  Every sample
+    carries its host time, so a region can be summarised as a whole or per time window."""
 
-    def __init__(self, index, period=0.01):
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+    REASONS = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap", "hw_power_brake")
+
+    def __init__(self, index, period=0.005):
+        self.samples = []          # (host time, SM MHz, set of active reasons)
+        self.max_mhz = None
         self._stop = threading.Event()
         self._thr = None
         self.period = period
@@ -92,7 +97,7 @@ class ClockSampler:
 
     def _run(self):
         nv = self.nv
-        names = {
+        bits = {
             "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
             "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
             "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
@@ -101,14 +106,12 @@ class ClockSampler:
         }
         while not self._stop.is_set():
             try:
-                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
                 try:
                     mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
                 except Exception:
                     mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
-                for k, bit in names.items():
-                    if mask & bit:
-                        self.reasons.add(k)
+                self.samples.append((time.perf_counter(), mhz, frozenset(k for k, bit in bits.items() if mask & bit)))
             except Exception:
                 pass
             self._stop.wait(self.period)
@@ -124,10 +127,55 @@ class ClockSampler:
         if self._thr is not None:
             self._thr.join()
 
-    def summary(self):
-        med = float(np.median(self.samples)) if self.samples else None
-        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples)}
+    def summary(self, t_lo=None, t_hi=None):
+        sel = [(m, r) for t, m, r in self.samples
+               if (t_lo is None or t >= t_lo) and (t_hi is None or t < t_hi)]
+        med = float(np.median([m for m, _ in sel])) if sel else None
+        reasons = sorted(set().union(*[r for _, r in sel])) if sel else []
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(sel)}
+
+
+# --------------------------------------------------------------------------- timed blocks
+MIN_TIMED_S = 1.0          # the device-timed region lasts at least this long, whatever --steps says
+SUSTAINED_AFTER_S = 0.3    # blocks that start later than this are the sustained regime
+IDLE_BEFORE_S = 1.0        # the GPU idles this long before a timed region, so its first block is a burst
+
+
+def timed_blocks(run_block, est_block_ms, device_index, min_s=MIN_TIMED_S, sync=None):
+    """Runs `run_block` (K steps, enqueued without a synchronise) back to back until at least
+    `min_s` seconds of device time have been timed, a CUDA event between blocks.  Returns the
+    per-block milliseconds, each block's start offset in seconds, and the clock samples."""
+    nblocks = max(3, int(np.ceil(min_s * 1e3 / max(est_block_ms, 1e-3))))
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(nblocks + 1)]
+    time.sleep(IDLE_BEFORE_S)
+    if sync is not None:
+        sync()
+    with ClockSampler(device_index) as clk:
+        t0 = time.perf_counter()
+        ev[0].record()
+        for b in range(nblocks):
+            run_block()
+            ev[b + 1].record()
+        torch.cuda.synchronize()
+        t1 = time.perf_counter()
+    ms = np.array([ev[b].elapsed_time(ev[b + 1]) for b in range(nblocks)])
+    starts = np.concatenate([[0.0], np.cumsum(ms)[:-1]]) * 1e-3
+    return ms, starts, clk, t0, t1
+
+
+def regimes(ms, starts, clk, t0, t1):
+    """Block time (ms) and clocks of the burst regime (the first block), the sustained regime
+    (median of the blocks that start after SUSTAINED_AFTER_S of load) and of all blocks (median)."""
+    late = starts >= SUSTAINED_AFTER_S
+    if not late.any():
+        late[-1] = True
+    t_first_end = t0 + ms[0] * 1e-3
+    return {
+        "burst": {"block_ms": float(ms[0]), "blocks": 1, "clocks": clk.summary(t0, max(t_first_end, t0 + 0.02))},
+        "sustained": {"block_ms": float(np.median(ms[late])), "blocks": int(late.sum()),
+                      "clocks": clk.summary(t0 + SUSTAINED_AFTER_S, t1)},
+        "all": {"block_ms": float(np.median(ms)), "blocks": int(len(ms)), "clocks": clk.summary(t0, t1)},
+    }
 
 
 # --------------------------------------------------------------------------- reference arm
@@ -311,9 +359,12 @@ def run_ours(args, rank, world, local_rank):
         torch.cuda.synchronize()
 
     K = args.steps
-    # ---- timed region.  One GPU: the step is captured once into a CUDA graph and replayed K
-    # times (no host launch gaps between the four kernels).  Several GPUs: K eager steps, each
-    # followed by the 16-byte mean exchange over NCCL.
+    # ---- timed region.  One GPU: the step is captured once into a CUDA graph and a block is K
+    # replays of it (no host launch gaps between the kernels).  Several GPUs: a block is K eager
+    # steps, each followed by the 16-byte mean exchange over NCCL.  Blocks of K steps repeat, a CUDA
+    # event between them, until at least MIN_TIMED_S of device time: `value` and `ms_per_step` come
+    # from the median block; the first block (after a second of idling) is the burst regime, the
+    # blocks that start after SUSTAINED_AFTER_S of load are the sustained one (power cap reached).
     use_graph = world == 1 and not os.environ.get("AK_BENCH_EAGER")
     launches0 = ak.ak_launch_count()
     step()
@@ -321,48 +372,8 @@ def run_ours(args, rank, world, local_rank):
         global_mean()
     torch.cuda.synchronize()
     kernels_per_step = ak.ak_launch_count() - launches0
-    graph = None
-    if use_graph:
-        side = torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(side):
-            with torch.cuda.graph(graph, stream=side):
-                step()
-        torch.cuda.current_stream().wait_stream(side)
-        for _ in range(3):
-            graph.replay()
-        torch.cuda.synchronize()
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if world > 1:
-        dist.barrier()
-        torch.cuda.synchronize()
-    with ClockSampler(local_rank) as clk:
-        start.record()
-        for i in range(K):
-            if graph is not None:
-                graph.replay()
-            else:
-                step()
-                if world > 1:
-                    global_mean()
-        end.record()
-        torch.cuda.synchronize()
-    launches = kernels_per_step * K
-    total_ms = start.elapsed_time(end)
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-        dist.barrier()
 
-    # ---- instrumented pass: per-op durations behind `per_op` and `roofline`.  Events cannot sit
-    # inside a replayed graph, so each op gets its own single-op CUDA graph, replayed K times
-    # back to back between two CUDA events on the same stream and buffers: duration = interval / K
-    # (kernel time plus the graph's kernel-to-kernel gap; for cross-entropy the streaming kernel
-    # and its 1-CTA finish kernel).  The eager per-call interval (host launch gaps included) is
-    # reported beside it.
-    def one_op_graph(fn):
+    def graph_of(fn):
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
         g = torch.cuda.CUDAGraph()
@@ -372,21 +383,64 @@ def run_ours(args, rank, world, local_rank):
         torch.cuda.current_stream().wait_stream(side)
         return g
 
+    def block_runner(fn_or_graph):
+        def run():
+            for _ in range(K):
+                fn_or_graph()
+        return run
+
+    def probe_ms(run_block):
+        a_ev, b_ev = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a_ev.record()
+        run_block()
+        b_ev.record()
+        torch.cuda.synchronize()
+        return a_ev.elapsed_time(b_ev)
+
+    def sync_ranks():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    if use_graph:
+        graph = graph_of(step)
+        run_step_block = block_runner(graph.replay)
+    else:
+        graph = None
+
+        def eager_step():
+            step()
+            if world > 1:
+                global_mean()
+        run_step_block = block_runner(eager_step)
+    est = probe_ms(run_step_block)
+    ms, starts, clk, t0, t1 = timed_blocks(run_step_block, est, local_rank, sync=sync_ranks)
+    if world > 1:
+        t = torch.tensor(ms, dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = t.cpu().numpy()
+        starts = np.concatenate([[0.0], np.cumsum(ms)[:-1]]) * 1e-3
+        dist.barrier()
+    step_reg = regimes(ms, starts, clk, t0, t1)
+    launches = kernels_per_step * K * len(ms)
+    total_ms = float(ms.sum())
+
+    # ---- instrumented pass: per-op durations behind `per_op` and `roofline`.  Events cannot sit
+    # inside a replayed graph, so each op gets its own single-op CUDA graph; a block is K replays of
+    # it back to back on the same stream and buffers, duration = block / K (kernel time plus the
+    # graph's kernel-to-kernel gap; for cross-entropy the streaming kernel and its 1-CTA finish
+    # kernel).  Blocks and regimes as for the step.  The eager per-call interval (host launch gaps
+    # included) is reported beside it.
     op_fns = {"rmsnorm": lambda: ak.ak_rmsnorm_fwd(x, w, y, eps=1e-6),
               "softmax": lambda: ak.ak_softmax_fwd(xs, ys),
               "xent": lambda: ak.ak_xent_fwd(lg, tg, -100, loss, mean)}
-    op_ms, op_ms_eager = {}, {}
+    op_reg, op_ms_eager = {}, {}
     for op, fn in op_fns.items():
-        g = one_op_graph(fn)
-        for _ in range(3):
-            g.replay()
-        a_ev, b_ev = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a_ev.record()
-        for _ in range(K):
-            g.replay()
-        b_ev.record()
-        torch.cuda.synchronize()
-        op_ms[op] = a_ev.elapsed_time(b_ev) / K
+        run_op_block = block_runner(graph_of(fn).replay)
+        est = probe_ms(run_op_block)
+        o_ms, o_starts, o_clk, o_t0, o_t1 = timed_blocks(run_op_block, est, local_rank,
+                                                         min_s=SUSTAINED_AFTER_S + 0.4)
+        op_reg[op] = regimes(o_ms, o_starts, o_clk, o_t0, o_t1)
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(min(K, 200))]
     for e in ev:
         e[0].record()
@@ -401,41 +455,67 @@ def run_ours(args, rank, world, local_rank):
         op_ms_eager[op] = float(np.mean([e[j].elapsed_time(e[j + 1]) for e in ev]))
 
     peak, peak_kind = measured_peak()
-    per_op = {}
     rows_of = {"rmsnorm": rr, "softmax": sr, "xent": xr}
-    for op in op_ms:
-        gbs = nbytes[op] / (op_ms[op] * 1e-3) / 1e9
-        per_op[op] = {"us": op_ms[op] * 1e3, "GB/s": gbs, "rows_per_s": rows_of[op] / (op_ms[op] * 1e-3),
-                      "frac_of_measured_peak": gbs / peak, "frac_of_8TBs": gbs / NOMINAL_HBM_GBS,
-                      "us_eager_call_interval": op_ms_eager[op] * 1e3}
-    dominant = max(op_ms, key=op_ms.get)
-    value = step_bytes * K * world / (total_ms * 1e-3) / 1e9
+
+    def op_entry(op, reg):
+        us = reg["block_ms"] / K * 1e3
+        gbs = nbytes[op] / (us * 1e-6) / 1e9
+        mhz = reg["clocks"]["sm_mhz"]
+        return {"us": us, "GB/s": gbs, "rows_per_s": rows_of[op] / (us * 1e-6), "frac_of_measured_peak": gbs / peak,
+                "frac_of_8TBs": gbs / NOMINAL_HBM_GBS, "sm_mhz": mhz, "us_x_mhz": (us * mhz if mhz else None),
+                "blocks": reg["blocks"]}
+
+    per_op = {op: op_entry(op, op_reg[op]["all"]) for op in op_reg}
+    for op in per_op:
+        per_op[op]["us_eager_call_interval"] = op_ms_eager[op] * 1e3
+    dominant = max(per_op, key=lambda o: per_op[o]["us"])
+
+    def step_entry(reg):
+        ms_step = reg["block_ms"] / K
+        return {"value": step_bytes * world / (ms_step * 1e-3) / 1e9, "ms_per_step": ms_step,
+                "blocks": reg["blocks"], "clocks": reg["clocks"]}
+
+    value = step_entry(step_reg["all"])["value"]
     sol = speed_of_light(ak, dev)
     for op in per_op:
         ceiling = sol["read_GB/s"] if op == "xent" else sol["copy_GB/s"]
         per_op[op]["frac_of_in_process_ceiling"] = per_op[op]["GB/s"] / ceiling
+    regime_out = {}
+    for name in ("burst", "sustained"):
+        e = step_entry(step_reg[name])
+        e["per_op"] = {op: op_entry(op, op_reg[op][name]) for op in op_reg}
+        e["roofline_frac"] = e["per_op"][dominant]["frac_of_measured_peak"]
+        regime_out[name] = e
 
     out = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K,
-        "warmup": max(args.warmup, 3), "ms_per_step": total_ms / K, "higher_is_better": True,
+        "warmup": max(args.warmup, 3), "ms_per_step": step_reg["all"]["block_ms"] / K, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": WORKLOAD_NAME, "l2": "every op's working set (268 MB / 537 MB / 1.05 GB) "
                    "exceeds the 126 MB L2; no flush needed", "parallelism": f"rows sharded x{world}",
                    "io_dtype": "bf16",
-                   "timed_region": ("K replays of a CUDA graph holding one step" if graph is not None
-                                    else "K eager steps + NCCL mean exchange")},
-        "rows_per_s": sum(rows_of.values()) * K * world / (total_ms * 1e-3),
+                   "timed_region": (("blocks of K replays of a CUDA graph holding one step" if graph is not None
+                                     else "blocks of K eager steps + NCCL mean exchange")
+                                    + f", repeated for >= {MIN_TIMED_S} s of device time after {IDLE_BEFORE_S} s of "
+                                      "idling; value / ms_per_step = median block; burst = first block; sustained "
+                                      f"= median of the blocks starting after {SUSTAINED_AFTER_S} s"),
+                   "blocks": int(len(ms)), "timed_seconds": total_ms * 1e-3},
+        "rows_per_s": sum(rows_of.values()) * world / (step_reg["all"]["block_ms"] / K * 1e-3),
+        "burst": regime_out["burst"], "sustained": regime_out["sustained"],
         "per_op": per_op,
         "roofline": {"bound": "hbm", "kernel": f"{dominant} {WORKLOAD[dominant][0]}x{WORKLOAD[dominant][1]}",
                      "achieved": per_op[dominant]["GB/s"], "peak": peak, "peak_kind": f"of {peak_kind}",
                      "unit": "GB/s", "frac": per_op[dominant]["GB/s"] / peak,
+                     "frac_burst": regime_out["burst"]["roofline_frac"],
+                     "frac_sustained": regime_out["sustained"]["roofline_frac"],
                      "frac_of_nominal_8TBs": per_op[dominant]["GB/s"] / NOMINAL_HBM_GBS,
                      "traffic": NCU_TRAFFIC_BYTES_DOMINANT.get(dominant), "algorithmic_bytes": nbytes[dominant],
-                     "note": "duration = CUDA-event interval over K back-to-back replays of a single-op CUDA "
-                             "graph / K, same stream and buffers (for cross-entropy: streaming kernel + "
-                             "1-CTA finish kernel)"},
+                     "note": "duration = median block of K back-to-back replays of a single-op CUDA graph / K, "
+                             "same stream and buffers (for cross-entropy: streaming kernel + 1-CTA finish kernel); "
+                             "frac_burst / frac_sustained: first block after idling / blocks after "
+                             f"{SUSTAINED_AFTER_S} s of load"},
         "gpu_launches": launches,
-        "clocks": clk.summary(),
+        "clocks": step_reg["all"]["clocks"],
         "speed_of_light": sol,
     }
 
@@ -484,7 +564,7 @@ def run_ours(args, rank, world, local_rank):
         out["cpu_baseline"] = None
 
     if args.sweep and rank == 0:
-        run_sweep(ak, synth, dev, peak)
+        run_sweep(ak, synth, dev, peak, out_path=args.out)
 
     if world > 1:
         dist.barrier()
@@ -538,7 +618,7 @@ def time_op(fn_for_set, nsets, iters=200, warmup=20):
     b.record()
     torch.cuda.synchronize()
     est_us = max(a.elapsed_time(b) * 1e3 / nsets, 1.0)
-    per_graph = nsets * max(1, int(np.ceil(float(os.environ.get('AK_SAMPLE_US', 300.0)) / est_us / nsets)))
+    per_graph = nsets * max(1, int(np.ceil(300.0 / est_us / nsets)))
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
     graph = torch.cuda.CUDAGraph()
@@ -717,7 +797,29 @@ WIDENED = [("layernorm", 8192, 4096), ("rowsum", 16384, 4096), ("rope.f16", 64 *
            ("softmax", 4096, 128256), ("softmax", 16, 128256)]
 
 
-def run_sweep(ak, synth, dev, peak, shapes=None, iters=200, write=True, accuracy=True):
+def size_matched_sol(ak, op_base, sets, nsets, esize, rows, D, iters):
+    """The library's plain copy (read-only ops: plain read) over buffers of the op's own size,
+    same timing protocol and buffer rotation: what this GPU gives a kernel of that size that
+    does no arithmetic.  Returns microseconds, or None where the buffers do not fit the aid."""
+    nbytes = esize * rows * D
+    if nbytes % 16 or any(t[0].data_ptr() % 16 for t in sets):
+        return None
+    l = ak.lib()
+    if op_base in ("xent", "rowsum", "xent_vp8"):
+        sink = torch.zeros((1,), dtype=torch.int32, device=sets[0][0].device)
+        fn = lambda i: l.ak_sol_read(sets[i][0].data_ptr(), nbytes, sink.data_ptr(),
+                                     torch.cuda.current_stream().cuda_stream)
+    else:
+        dst = [t[-1] for t in sets]
+        if any(d.data_ptr() % 16 or d.numel() * d.element_size() != nbytes for d in dst):
+            return None
+        fn = lambda i: l.ak_sol_copy(sets[i][0].data_ptr(), dst[i].data_ptr(), nbytes,
+                                     torch.cuda.current_stream().cuda_stream)
+    us, _, _ = time_op(fn, nsets, iters=iters)
+    return us
+
+
+def run_sweep(ak, synth, dev, peak, shapes=None, iters=200, write=True, accuracy=True, out_path=None):
     rows_out = []
     only = os.environ.get("AK_SWEEP_OPS") if shapes is None else None
     for op, rows, D in (SWEEP if shapes is None else shapes):
@@ -802,23 +904,29 @@ def run_sweep(ak, synth, dev, peak, shapes=None, iters=200, write=True, accuracy
             nb = algorithmic_bytes(op, rows, D, int((sets[0][1] != -100).sum()))
         us, us_min, us_med = time_op(fn, nsets, iters=iters)
         gbs = nb / (us * 1e-6) / 1e9
+        sol_us = size_matched_sol(ak, base, sets, nsets, esize, rows, D, max(iters // 2, 30)) if write else None
         # errors against the CPU checker and its timing belong to the per-shape CPU-baseline report
         acc = sweep_accuracy(ak, synth, op, rows, D, sets[0]) if accuracy else {}
         rows_out.append({"op": op, "rows": rows, "D": D, "us_trimmed_mean": us, "us_min": us_min,
                          "us_median": us_med, "GB/s": gbs, "frac_of_8TBs": gbs / NOMINAL_HBM_GBS,
                          "frac_of_measured_copy": gbs / peak, "rows_per_s": rows / (us * 1e-6),
-                         "buffer_sets": nsets, "large_shape": one_set >= (250 << 20), **acc})
+                         "buffer_sets": nsets, "large_shape": one_set >= (250 << 20),
+                         "us_size_matched_copy": sol_us,
+                         "frac_of_size_matched_copy": (sol_us / us if sol_us else None), **acc})
         del sets
         torch.cuda.empty_cache()
     if not write:
         return rows_out
-    os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
-    with open(os.path.join(ROOT, "gpurun_out", "sweep.json"), "w") as f:
-        json.dump(rows_out, f, indent=1)
+    if out_path:
+        os.makedirs(os.path.dirname(os.path.abspath(out_path)), exist_ok=True)
+        with open(out_path, "w") as f:
+            json.dump(rows_out, f, indent=1)
     for r in rows_out:
+        sm = r["frac_of_size_matched_copy"]
         print(f"# {r['op']:11s} {r['rows']:7d} x {r['D']:6d}  {r['us_trimmed_mean']:9.1f} us  "
               f"{r['GB/s']:7.0f} GB/s  {100 * r['frac_of_8TBs']:5.1f}% of 8TB/s  "
-              f"{100 * r['frac_of_measured_copy']:5.1f}% of copy", file=sys.stderr)
+              f"{100 * r['frac_of_measured_copy']:5.1f}% of copy  "
+              + (f"{100 * sm:5.1f}% of a copy / read of its size" if sm else ""), file=sys.stderr)
 
 
 def run_case(args):
@@ -886,6 +994,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--out", default=None, help="file the --sweep table is written to (JSON)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -900,7 +1009,7 @@ def main():
         args.warmup = 1 if args.warmup is None else args.warmup
         run_reference(args, rank, world)
         return
-    args.steps = 1000 if args.steps is None else args.steps
+    args.steps = 100 if args.steps is None else args.steps
     args.warmup = 10 if args.warmup is None else args.warmup
     run_ours(args, rank, world, local_rank)
 

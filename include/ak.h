@@ -283,6 +283,9 @@ int ak_xent_fwd_static(const void* logits, const int64_t* targets, int64_t ignor
  * is bit-identical on every rank.  The paper's system is single-GPU (Section "Limitations");
  * this is the row-shard extension of the mean in ak_xent_fwd.
  * sum_count: device double[2]; sum_count_pairs: device double[2 * n]; loss_mean: device fp32[1].
+ * An empty block (rows == 0: loss_rows and targets may be NULL) contributes {0, 0}; n == 0
+ * (sum_count_pairs may be NULL) gives NaN.  Both calls only enqueue work on cuda_stream: the
+ * all-gather between them has to be ordered on that same stream by the caller.
  */
 int ak_xent_sum_count(const float* loss_rows, const int64_t* targets, int64_t ignore_index,
                       int64_t rows, double* sum_count, void* cuda_stream);

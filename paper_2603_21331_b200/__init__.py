@@ -10,5 +10,6 @@ from .binding import (  # noqa: F401
     ak_rmsnorm_fwd, ak_rmsnorm_fwd_host, ak_rope_fwd, ak_rowsum_fwd,
     ak_softmax_choose_path, ak_softmax_fwd, ak_softmax_fwd_host, ak_status_string, ak_version,
     ak_xent_choose_path, ak_xent_fwd, ak_xent_fwd_host, ak_xent_fwd_static, ak_xent_fwd_ws,
+    ak_xent_mean_merge, ak_xent_sum_count,
     ak_xent_vp_merge, ak_xent_vp_nsplit, ak_xent_vp_partial, ak_xent_workspace_bytes, lib,
 )

@@ -121,6 +121,38 @@ def _stream_ptr(stream, like: Optional[torch.Tensor] = None) -> int:
     return int(stream)
 
 
+class _on_device_of:
+    """Makes the tensors' device the current CUDA device around a library call (the library
+    launches on the current device; function attributes, scratch pools and streams belong to
+    it) and puts the previous one back.  Tensors on different devices are refused."""
+    __slots__ = ("index", "previous")
+
+    def __init__(self, *tensors):
+        index = None
+        for t in tensors:
+            if t is None:
+                continue
+            if index is None:
+                index = t.device.index
+            elif t.device.index != index:
+                raise ValueError("all tensors of a call must be on the same CUDA device")
+        self.index = index
+        self.previous = None
+
+    def __enter__(self):
+        if self.index is not None:
+            current = torch.cuda.current_device()
+            if current != self.index:
+                self.previous = current
+                torch.cuda.set_device(self.index)
+        return self
+
+    def __exit__(self, *exc):
+        if self.previous is not None:
+            torch.cuda.set_device(self.previous)
+        return False
+
+
 def _dev_bf16(t: torch.Tensor, name: str, ndim: int) -> None:
     if not (t.is_cuda and t.dtype == torch.bfloat16 and t.dim() == ndim and t.is_contiguous()):
         raise TypeError(f"{name} must be a contiguous CUDA bfloat16 tensor with {ndim} dims")
@@ -144,8 +176,9 @@ def ak_rmsnorm_fwd(x: torch.Tensor, w: torch.Tensor, y: Optional[torch.Tensor] =
     _dev_bf16(y, "y", 2)
     if y.shape != x.shape:
         raise ValueError("y must have the shape of x")
-    _check(lib().ak_rmsnorm_fwd_path(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, D, eps,
-                                     _stream_ptr(stream, x), path), "ak_rmsnorm_fwd")
+    with _on_device_of(x, w, y):
+        _check(lib().ak_rmsnorm_fwd_path(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, D, eps,
+                                         _stream_ptr(stream, x), path), "ak_rmsnorm_fwd")
     return y
 
 
@@ -170,8 +203,9 @@ def ak_rmsnorm_fwd_dt(x: torch.Tensor, w: torch.Tensor, y: Optional[torch.Tensor
     _dev_dt(y, "y", 2, x.dtype)
     if y.shape != x.shape:
         raise ValueError("y must have the shape of x")
-    _check(lib().ak_rmsnorm_fwd_dt(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, D, eps, dt,
-                                   _stream_ptr(stream, x), path), "ak_rmsnorm_fwd_dt")
+    with _on_device_of(x, w, y):
+        _check(lib().ak_rmsnorm_fwd_dt(x.data_ptr(), w.data_ptr(), y.data_ptr(), rows, D, eps, dt,
+                                       _stream_ptr(stream, x), path), "ak_rmsnorm_fwd_dt")
     return y
 
 
@@ -185,8 +219,9 @@ def ak_softmax_fwd_dt(x: torch.Tensor, y: Optional[torch.Tensor] = None, stream=
     _dev_dt(y, "y", 2, x.dtype)
     if y.shape != x.shape:
         raise ValueError("y must have the shape of x")
-    _check(lib().ak_softmax_fwd_dt(x.data_ptr(), y.data_ptr(), rows, D, dt, _stream_ptr(stream, x), path),
-           "ak_softmax_fwd_dt")
+    with _on_device_of(x, y):
+        _check(lib().ak_softmax_fwd_dt(x.data_ptr(), y.data_ptr(), rows, D, dt, _stream_ptr(stream, x), path),
+               "ak_softmax_fwd_dt")
     return y
 
 
@@ -201,9 +236,10 @@ def ak_xent_fwd_dt(logits: torch.Tensor, targets: torch.Tensor, ignore_index: in
         raise TypeError("targets must be a contiguous CUDA int64 tensor [rows]")
     loss_rows = torch.empty((rows,), dtype=torch.float32, device=logits.device)
     loss_mean = torch.empty((1,), dtype=torch.float32, device=logits.device) if want_mean else None
-    _check(lib().ak_xent_fwd_dt(logits.data_ptr(), targets.data_ptr(), ignore_index, loss_rows.data_ptr(),
-                                loss_mean.data_ptr() if want_mean else None, rows, V, dt,
-                                _stream_ptr(stream, logits), path, nsplit), "ak_xent_fwd_dt")
+    with _on_device_of(logits, targets, loss_rows, loss_mean):
+        _check(lib().ak_xent_fwd_dt(logits.data_ptr(), targets.data_ptr(), ignore_index, loss_rows.data_ptr(),
+                                    loss_mean.data_ptr() if want_mean else None, rows, V, dt,
+                                    _stream_ptr(stream, logits), path, nsplit), "ak_xent_fwd_dt")
     return loss_rows, loss_mean
 
 
@@ -222,8 +258,9 @@ def ak_layernorm_fwd_dt(x: torch.Tensor, gamma: torch.Tensor, beta: torch.Tensor
     _dev_dt(y, "y", 2, x.dtype)
     if y.shape != x.shape:
         raise ValueError("y must have the shape of x")
-    _check(lib().ak_layernorm_fwd_dt(x.data_ptr(), gamma.data_ptr(), beta.data_ptr(), y.data_ptr(), rows, D,
-                                     eps, dt, _stream_ptr(stream, x), path), "ak_layernorm_fwd_dt")
+    with _on_device_of(x, gamma, beta, y):
+        _check(lib().ak_layernorm_fwd_dt(x.data_ptr(), gamma.data_ptr(), beta.data_ptr(), y.data_ptr(), rows, D,
+                                         eps, dt, _stream_ptr(stream, x), path), "ak_layernorm_fwd_dt")
     return y
 
 
@@ -235,8 +272,9 @@ def ak_rowsum_fwd_dt(x: torch.Tensor, out: Optional[torch.Tensor] = None, stream
         out = torch.empty((rows,), dtype=torch.float32, device=x.device)
     if not (out.is_cuda and out.dtype == torch.float32 and out.shape == (rows,) and out.is_contiguous()):
         raise TypeError("out must be a contiguous CUDA float32 tensor [rows]")
-    _check(lib().ak_rowsum_fwd_dt(x.data_ptr(), out.data_ptr(), rows, D, dt, _stream_ptr(stream, x)),
-           "ak_rowsum_fwd_dt")
+    with _on_device_of(x, out):
+        _check(lib().ak_rowsum_fwd_dt(x.data_ptr(), out.data_ptr(), rows, D, dt, _stream_ptr(stream, x)),
+               "ak_rowsum_fwd_dt")
     return out
 
 
@@ -250,8 +288,9 @@ def ak_rope_fwd(x: torch.Tensor, y: Optional[torch.Tensor] = None, base: float =
     _dev_dt(y, "y", 3, x.dtype)
     if y.shape != x.shape:
         raise ValueError("y must have the shape of x")
-    _check(lib().ak_rope_fwd(x.data_ptr(), y.data_ptr(), n_seq, S, Dh, base, pos_offset, dt,
-                             _stream_ptr(stream, x)), "ak_rope_fwd")
+    with _on_device_of(x, y):
+        _check(lib().ak_rope_fwd(x.data_ptr(), y.data_ptr(), n_seq, S, Dh, base, pos_offset, dt,
+                                 _stream_ptr(stream, x)), "ak_rope_fwd")
     return y
 
 
@@ -277,9 +316,10 @@ def ak_xent_vp_partial(logits_shard: torch.Tensor, targets: torch.Tensor, vocab_
     if not (partial.is_cuda and partial.dtype == torch.float32 and partial.shape == (rows, nsplit + 1, 2)
             and partial.is_contiguous()):
         raise TypeError("partial must be a contiguous CUDA float32 tensor [rows, nsplit + 1, 2]")
-    _check(lib().ak_xent_vp_partial(logits_shard.data_ptr(), targets.data_ptr(), ignore_index, vocab_start,
-                                    V_total, partial.data_ptr(), rows, V_local, nsplit, dt,
-                                    _stream_ptr(stream, logits_shard)), "ak_xent_vp_partial")
+    with _on_device_of(logits_shard, targets, partial):
+        _check(lib().ak_xent_vp_partial(logits_shard.data_ptr(), targets.data_ptr(), ignore_index, vocab_start,
+                                        V_total, partial.data_ptr(), rows, V_local, nsplit, dt,
+                                        _stream_ptr(stream, logits_shard)), "ak_xent_vp_partial")
     return partial
 
 
@@ -296,9 +336,10 @@ def ak_xent_vp_merge(partials: torch.Tensor, targets: torch.Tensor, V_total: int
         raise TypeError("targets must be a contiguous CUDA int64 tensor [rows]")
     loss_rows = torch.empty((rows,), dtype=torch.float32, device=partials.device)
     loss_mean = torch.empty((1,), dtype=torch.float32, device=partials.device) if want_mean else None
-    _check(lib().ak_xent_vp_merge(partials.data_ptr(), nranks, ns1 - 1, targets.data_ptr(), ignore_index,
-                                  V_total, loss_rows.data_ptr(), loss_mean.data_ptr() if want_mean else None,
-                                  rows, _stream_ptr(stream, partials)), "ak_xent_vp_merge")
+    with _on_device_of(partials, targets, loss_rows, loss_mean):
+        _check(lib().ak_xent_vp_merge(partials.data_ptr(), nranks, ns1 - 1, targets.data_ptr(), ignore_index,
+                                      V_total, loss_rows.data_ptr(), loss_mean.data_ptr() if want_mean else None,
+                                      rows, _stream_ptr(stream, partials)), "ak_xent_vp_merge")
     return loss_rows, loss_mean
 
 
@@ -320,8 +361,9 @@ def ak_layernorm_fwd(x: torch.Tensor, gamma: torch.Tensor, beta: torch.Tensor,
     _dev_bf16(y, "y", 2)
     if y.shape != x.shape:
         raise ValueError("y must have the shape of x")
-    _check(lib().ak_layernorm_fwd_path(x.data_ptr(), gamma.data_ptr(), beta.data_ptr(), y.data_ptr(),
-                                       rows, D, eps, _stream_ptr(stream, x), path), "ak_layernorm_fwd")
+    with _on_device_of(x, gamma, beta, y):
+        _check(lib().ak_layernorm_fwd_path(x.data_ptr(), gamma.data_ptr(), beta.data_ptr(), y.data_ptr(),
+                                           rows, D, eps, _stream_ptr(stream, x), path), "ak_layernorm_fwd")
     return y
 
 
@@ -332,7 +374,8 @@ def ak_rowsum_fwd(x: torch.Tensor, out: Optional[torch.Tensor] = None, stream=No
         out = torch.empty((rows,), dtype=torch.float32, device=x.device)
     if not (out.is_cuda and out.dtype == torch.float32 and out.shape == (rows,) and out.is_contiguous()):
         raise TypeError("out must be a contiguous CUDA float32 tensor [rows]")
-    _check(lib().ak_rowsum_fwd(x.data_ptr(), out.data_ptr(), rows, D, _stream_ptr(stream, x)), "ak_rowsum_fwd")
+    with _on_device_of(x, out):
+        _check(lib().ak_rowsum_fwd(x.data_ptr(), out.data_ptr(), rows, D, _stream_ptr(stream, x)), "ak_rowsum_fwd")
     return out
 
 
@@ -345,8 +388,9 @@ def ak_softmax_fwd(x: torch.Tensor, y: Optional[torch.Tensor] = None, stream=Non
     _dev_bf16(y, "y", 2)
     if y.shape != x.shape:
         raise ValueError("y must have the shape of x")
-    _check(lib().ak_softmax_fwd_path(x.data_ptr(), y.data_ptr(), rows, D, _stream_ptr(stream, x), path),
-           "ak_softmax_fwd")
+    with _on_device_of(x, y):
+        _check(lib().ak_softmax_fwd_path(x.data_ptr(), y.data_ptr(), rows, D, _stream_ptr(stream, x), path),
+               "ak_softmax_fwd")
     return y
 
 
@@ -368,9 +412,10 @@ def ak_xent_fwd(logits: torch.Tensor, targets: torch.Tensor, ignore_index: int =
                                   and t.is_contiguous()):
             raise TypeError("loss buffers must be contiguous CUDA float32 tensors")
     mean_ptr = loss_mean.data_ptr() if loss_mean is not None else None
-    _check(lib().ak_xent_fwd_path(logits.data_ptr(), targets.data_ptr(), ignore_index,
-                                  loss_rows.data_ptr(), mean_ptr, rows, V, _stream_ptr(stream, logits),
-                                  path, nsplit), "ak_xent_fwd")
+    with _on_device_of(logits, targets, loss_rows, loss_mean):
+        _check(lib().ak_xent_fwd_path(logits.data_ptr(), targets.data_ptr(), ignore_index,
+                                      loss_rows.data_ptr(), mean_ptr, rows, V, _stream_ptr(stream, logits),
+                                      path, nsplit), "ak_xent_fwd")
     return loss_rows, loss_mean
 
 
@@ -392,10 +437,48 @@ def ak_xent_fwd_static(logits: torch.Tensor, targets: torch.Tensor, ignore_index
         loss_rows = torch.empty((rows,), dtype=torch.float32, device=logits.device)
     if loss_mean is None:
         loss_mean = torch.empty((1,), dtype=torch.float32, device=logits.device)
-    _check(lib().ak_xent_fwd_static(logits.data_ptr(), targets.data_ptr(), ignore_index,
-                                    loss_rows.data_ptr(), loss_mean.data_ptr(), rows, V,
-                                    _stream_ptr(stream, logits)), "ak_xent_fwd_static")
+    with _on_device_of(logits, targets, loss_rows, loss_mean):
+        _check(lib().ak_xent_fwd_static(logits.data_ptr(), targets.data_ptr(), ignore_index,
+                                        loss_rows.data_ptr(), loss_mean.data_ptr(), rows, V,
+                                        _stream_ptr(stream, logits)), "ak_xent_fwd_static")
     return loss_rows, loss_mean
+
+
+def ak_xent_sum_count(loss_rows: torch.Tensor, targets: torch.Tensor, ignore_index: int = -100,
+                      out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """{fp64 sum of the counted rows' losses, their count} of this rank's block of rows -> float64 [2]
+    (the 16 bytes a rank contributes to the mean over row shards)."""
+    rows = loss_rows.numel()
+    if not (loss_rows.is_cuda and loss_rows.dtype == torch.float32 and loss_rows.is_contiguous()):
+        raise TypeError("loss_rows must be a contiguous CUDA float32 tensor")
+    if not (targets.is_cuda and targets.dtype == torch.int64 and targets.numel() == rows and targets.is_contiguous()):
+        raise TypeError("targets must be a contiguous CUDA int64 tensor [rows]")
+    if out is None:
+        out = torch.empty((2,), dtype=torch.float64, device=loss_rows.device)
+    if not (out.is_cuda and out.dtype == torch.float64 and out.numel() == 2 and out.is_contiguous()):
+        raise TypeError("out must be a contiguous CUDA float64 tensor with 2 elements")
+    with _on_device_of(loss_rows, targets, out):
+        _check(lib().ak_xent_sum_count(loss_rows.data_ptr() if rows else None, targets.data_ptr() if rows else None,
+                                       ignore_index, rows, out.data_ptr(), _stream_ptr(stream, loss_rows)),
+               "ak_xent_sum_count")
+    return out
+
+
+def ak_xent_mean_merge(pairs: torch.Tensor, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Mean over row shards: ``pairs`` = float64 [n, 2] of (sum, count) in rank order, added in
+    that order -> float32 [1] (NaN when nothing counts)."""
+    if not (pairs.is_cuda and pairs.dtype == torch.float64 and pairs.dim() == 2 and pairs.shape[1] == 2
+            and pairs.is_contiguous()):
+        raise TypeError("pairs must be a contiguous CUDA float64 tensor [n, 2]")
+    if out is None:
+        out = torch.empty((1,), dtype=torch.float32, device=pairs.device)
+    if not (out.is_cuda and out.dtype == torch.float32 and out.numel() == 1):
+        raise TypeError("out must be a CUDA float32 tensor with 1 element")
+    with _on_device_of(pairs, out):
+        _check(lib().ak_xent_mean_merge(pairs.data_ptr() if pairs.shape[0] else None, pairs.shape[0], out.data_ptr(),
+                                        _stream_ptr(stream, pairs)),
+               "ak_xent_mean_merge")
+    return out
 
 
 def ak_xent_workspace_bytes(rows: int, V: int) -> int:
@@ -413,9 +496,10 @@ def ak_xent_fwd_ws(logits: torch.Tensor, targets: torch.Tensor, workspace: Optio
         loss_mean = torch.empty((1,), dtype=torch.float32, device=logits.device)
     ws_ptr = workspace.data_ptr() if workspace is not None else None
     ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
-    _check(lib().ak_xent_fwd_ws(logits.data_ptr(), targets.data_ptr(), ignore_index,
-                                loss_rows.data_ptr(), loss_mean.data_ptr(), rows, V, ws_ptr, ws_bytes,
-                                _stream_ptr(stream, logits)), "ak_xent_fwd_ws")
+    with _on_device_of(logits, targets, loss_rows, loss_mean, workspace):
+        _check(lib().ak_xent_fwd_ws(logits.data_ptr(), targets.data_ptr(), ignore_index,
+                                    loss_rows.data_ptr(), loss_mean.data_ptr(), rows, V, ws_ptr, ws_bytes,
+                                    _stream_ptr(stream, logits)), "ak_xent_fwd_ws")
     return loss_rows, loss_mean
 
 

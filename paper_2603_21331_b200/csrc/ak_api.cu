@@ -3,7 +3,10 @@
 #include <atomic>
 #include <cmath>
 #include <cstdlib>
+#include <map>
 #include <mutex>
+#include <set>
+#include <tuple>
 
 #include "ak_common.cuh"
 
@@ -91,6 +94,49 @@ int sm_count() {
         cached[dev] = n;
     }
     return cached[dev];
+}
+
+namespace {
+constexpr int kMaxDev = 64;
+int current_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) return -1;
+    return dev;
+}
+}  // namespace
+
+bool dyn_smem_configured(const void* kernel) {
+    static std::mutex mu;
+    static std::set<const void*> done[kMaxDev];
+    const int dev = current_device();
+    if (dev < 0) return false;
+    std::lock_guard<std::mutex> lock(mu);
+    if (done[dev].count(kernel)) return true;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxRowSmemBytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return false;
+    }
+    done[dev].insert(kernel);
+    return true;
+}
+
+int resident_ctas_of(const void* kernel, int threads, size_t dyn_smem) {
+    static std::mutex mu;
+    static std::map<std::tuple<const void*, int, size_t>, int> memo[kMaxDev];
+    const int dev = current_device();
+    const int sms = sm_count();
+    if (dev < 0) return sms;
+    std::lock_guard<std::mutex> lock(mu);
+    const auto key = std::make_tuple(kernel, threads, dyn_smem);
+    auto it = memo[dev].find(key);
+    if (it != memo[dev].end()) return it->second;
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, dyn_smem) != cudaSuccess || per_sm < 1) {
+        (void)cudaGetLastError();
+        per_sm = 1;
+    }
+    memo[dev][key] = per_sm * sms;
+    return per_sm * sms;
 }
 
 namespace {
@@ -316,16 +362,16 @@ int ak_xent_fwd_ws(const void* logits, const int64_t* targets, int64_t ignore_in
 
 int ak_xent_sum_count(const float* loss_rows, const int64_t* targets, int64_t ignore_index, int64_t rows,
                       double* sum_count, void* cuda_stream) {
-    if (!loss_rows || !targets || !sum_count) return AK_ERR_NULL;
     if (rows < 0) return AK_ERR_SHAPE;
+    if (!sum_count || (rows != 0 && (!loss_rows || !targets))) return AK_ERR_NULL;  // an empty block may carry NULL data
     if (!is_aligned(loss_rows, 4) || !is_aligned(targets, 8) || !is_aligned(sum_count, 8)) return AK_ERR_ALIGN;
     return xent_sum_count_launch(loss_rows, targets, ignore_index, rows, sum_count,
                                  static_cast<cudaStream_t>(cuda_stream));
 }
 
 int ak_xent_mean_merge(const double* sum_count_pairs, int64_t n, float* loss_mean, void* cuda_stream) {
-    if (!sum_count_pairs || !loss_mean) return AK_ERR_NULL;
     if (n < 0) return AK_ERR_SHAPE;
+    if (!loss_mean || (n != 0 && !sum_count_pairs)) return AK_ERR_NULL;  // no pairs: the mean is NaN
     if (!is_aligned(sum_count_pairs, 8) || !is_aligned(loss_mean, 4)) return AK_ERR_ALIGN;
     return xent_mean_merge_launch(sum_count_pairs, n, loss_mean, static_cast<cudaStream_t>(cuda_stream));
 }

@@ -344,6 +344,18 @@ int cluster_ctas(int64_t rows, int64_t row_bytes, int64_t split_from);
 // faster: softmax 16384 x 32768 317 us against 338 us in clusters of two)
 constexpr int64_t kClusterFrom = 65536 + 16;
 int sm_count();  // SMs of the current device (cached per device)
+// Per-device memos, keyed by kernel (a process may drive several GPUs, and function attributes
+// and occupancy belong to the device that is current at the call):
+//   dyn_smem_configured  cudaFuncAttributeMaxDynamicSharedMemorySize = kMaxRowSmemBytes set once
+//   resident_ctas_of     CTAs of this kernel the whole device holds at once (>= 1 per SM)
+bool dyn_smem_configured(const void* kernel);
+int resident_ctas_of(const void* kernel, int threads, size_t dyn_smem);
+template <typename... A>
+inline bool allow_big_smem(void (*kernel)(A...)) { return dyn_smem_configured(reinterpret_cast<const void*>(kernel)); }
+template <typename... A>
+inline int resident_ctas(void (*kernel)(A...), int threads, size_t dyn_smem) {
+    return resident_ctas_of(reinterpret_cast<const void*>(kernel), threads, dyn_smem);
+}
 
 // Per-op host dispatchers (each defined next to its kernels).  All arguments have been
 // validated; `path` is a concrete path id or AUTO.  They return an ak_status.
@@ -384,6 +396,22 @@ inline bool is_aligned(const void* p, size_t a) { return (reinterpret_cast<uintp
 // grid is still running (it waits for our completion with pdl_wait before it reads).
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Prologue of a kernel launched as a programmatic dependent of whatever precedes it in the stream.
+// Its CTAs may become resident while the grids before it still drain; nothing may be read or
+// written until griddepcontrol.wait returns.  The CTAs of the first wave (blockIdx.x < first_wave
+// = as many CTAs as the device holds at once) use that time to ask for the first 128 bytes per
+// thread of their input span to be brought into L2: a prefetch reads nothing architecturally.
+// Later CTAs start on a busy machine and skip it.  After the wait the kernel lets its own
+// dependents in at once (they wait for this grid's completion in turn).
+__device__ __forceinline__ void pdl_prologue(const void* span, int64_t span_bytes, int first_wave) {
+    if ((int)blockIdx.x < first_wave) {
+        const int64_t off = (int64_t)threadIdx.x * 128;
+        if (off < span_bytes) prefetch_l2(static_cast<const char*>(span) + off);
+    }
+    pdl_wait();
+    pdl_launch_dependents();
+}
 
 // ------------------------------------------------------------------ pre-shifted parameter vectors
 // Rows of 2-byte elements that do not start on a 16-byte boundary are processed in their own

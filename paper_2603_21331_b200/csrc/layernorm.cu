@@ -22,11 +22,13 @@ int launch_reg(const void* x, const void* g, const void* b, void* y, int64_t row
                float eps, cudaStream_t st) {
     constexpr int GROUPS = THREADS / GROUP;
     const int64_t grid = (rows + GROUPS - 1) / GROUPS;
-    layernorm_reg_kernel<THREADS, GROUP, VPT, MINB, DT, PE><<<(unsigned)grid, THREADS, 0, st>>>(
-        static_cast<const uint4*>(x), static_cast<const uint4*>(g), static_cast<const uint4*>(b),
-        static_cast<uint4*>(y), rows, nvec, inv_D, eps);
+    auto kernel = layernorm_reg_kernel<THREADS, GROUP, VPT, MINB, DT, PE>;
+    const cudaError_t e = launch_dependent(kernel, dim3((unsigned)grid), dim3(THREADS), 0, st,
+                                           static_cast<const uint4*>(x), static_cast<const uint4*>(g),
+                                           static_cast<const uint4*>(b), static_cast<uint4*>(y), rows, nvec, inv_D, eps,
+                                           resident_ctas(kernel, THREADS, 0));
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+    return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
 // vectors per thread 1..8 for a fixed (THREADS, GROUP); the minimum-CTAs-per-SM hint (a register
@@ -51,11 +53,7 @@ template <int DT, int THREADS>
 int launch_smem(const void* x, const void* g, const void* b, void* y, int64_t rows, int nvec, float inv_D,
                 float eps, cudaStream_t st) {
     const size_t smem = (size_t)nvec * 16;
-    static const bool configured = [] {
-        return cudaFuncSetAttribute(layernorm_smem_kernel<THREADS, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    kMaxRowSmemBytes) == cudaSuccess;
-    }();
-    if (!configured) return AK_ERR_CUDA;
+    if (!allow_big_smem(layernorm_smem_kernel<THREADS, DT>)) return AK_ERR_CUDA;
     layernorm_smem_kernel<THREADS, DT><<<(unsigned)rows, THREADS, smem, st>>>(
         static_cast<const uint4*>(x), static_cast<const uint4*>(g), static_cast<const uint4*>(b),
         static_cast<uint4*>(y), nvec, inv_D, eps);
@@ -67,11 +65,7 @@ int launch_smem(const void* x, const void* g, const void* b, void* y, int64_t ro
 template <int DT, int THREADS>
 int launch_cluster_rows(const void* x, const void* g, const void* b, void* y, int64_t rows, int nvec, int C, float inv_D,
                         float eps, cudaStream_t st) {
-    static const bool configured = [] {
-        return cudaFuncSetAttribute(layernorm_cluster_kernel<THREADS, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    kMaxRowSmemBytes) == cudaSuccess;
-    }();
-    if (!configured) return AK_ERR_CUDA;
+    if (!allow_big_smem(layernorm_cluster_kernel<THREADS, DT>)) return AK_ERR_CUDA;
     const size_t smem = (size_t)((nvec + C - 1) / C) * 16;
     const cudaError_t e = launch_cluster(layernorm_cluster_kernel<THREADS, DT>, (unsigned)(rows * C), THREADS, smem, C, st,
                                          static_cast<const uint4*>(x), static_cast<const uint4*>(g),
@@ -110,13 +104,7 @@ constexpr int64_t kShiftMinRowsStaged = 256;   // longer rows staged in shared m
 template <int DT, int T>
 int launch_stage(const uint16_t* x, const uint16_t* g, const uint16_t* b, uint16_t* y, int64_t rows, int64_t D,
                  size_t stage_bytes, float inv_D, float eps, cudaStream_t st) {
-    static const bool configured = [] {
-        return cudaFuncSetAttribute(layernorm_stage_kernel<T, DT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    kMaxRowSmemBytes) == cudaSuccess &&
-               cudaFuncSetAttribute(layernorm_stage_kernel<T, DT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    kMaxRowSmemBytes) == cudaSuccess;
-    }();
-    if (!configured) return AK_ERR_CUDA;
+    if (!allow_big_smem(layernorm_stage_kernel<T, DT, false>) || !allow_big_smem(layernorm_stage_kernel<T, DT, true>)) return AK_ERR_CUDA;
     int nvp = 0;
     if (const uint4* tab = shift_table(g, b, rows, D, kShiftMinRowsStaged, st, &nvp)) {
         const cudaError_t e = launch_dependent(layernorm_stage_kernel<T, DT, true>, dim3((unsigned)rows), dim3(T),
@@ -135,13 +123,7 @@ int launch_stage(const uint16_t* x, const uint16_t* g, const uint16_t* b, uint16
 template <int DT, int T>
 int launch_cluster_stage(const uint16_t* x, const uint16_t* g, const uint16_t* b, uint16_t* y, int64_t rows, int64_t D,
                          int64_t max_nv, int C, float inv_D, float eps, cudaStream_t st) {
-    static const bool configured = [] {
-        return cudaFuncSetAttribute(layernorm_cluster_stage_kernel<T, DT, false>,
-                                    cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxRowSmemBytes) == cudaSuccess &&
-               cudaFuncSetAttribute(layernorm_cluster_stage_kernel<T, DT, true>,
-                                    cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxRowSmemBytes) == cudaSuccess;
-    }();
-    if (!configured) return AK_ERR_CUDA;
+    if (!allow_big_smem(layernorm_cluster_stage_kernel<T, DT, false>) || !allow_big_smem(layernorm_cluster_stage_kernel<T, DT, true>)) return AK_ERR_CUDA;
     const size_t smem = (size_t)((max_nv + C - 1) / C) * 16;
     int nvp = 0;
     if (const uint4* tab = shift_table(g, b, rows, D, kShiftMinRowsStaged, st, &nvp)) {
@@ -189,14 +171,6 @@ int launch_regp_vpt(int vpt, const uint16_t* x, const uint16_t* g, const uint16_
         case 8: return launch_regp<DT, THREADS, 8, M68>(x, g, b, y, rows, D, inv_D, eps, st);
         default: return AK_ERR_SHAPE;
     }
-}
-
-template <typename K>
-int resident_ctas(K kernel, int threads) {
-    int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, 0) != cudaSuccess || per_sm < 1)
-        per_sm = 1;
-    return per_sm * sm_count();
 }
 
 template <int DT>
@@ -268,7 +242,7 @@ int dispatch_t(const void* x, const void* gamma, const void* beta, void* y, int6
         }
         case AK_PATH_GENERIC: {
             if constexpr (DT == AK_DTYPE_F32) {
-                static const int resident = resident_ctas(layernorm_generic32_kernel, kLnGenericThreads);
+                const int resident = resident_ctas(layernorm_generic32_kernel, kLnGenericThreads, 0);
                 const int grid = (int)(rows < resident ? rows : resident);
                 layernorm_generic32_kernel<<<grid, kLnGenericThreads, 0, st>>>(
                     static_cast<const float*>(x), static_cast<const float*>(gamma), static_cast<const float*>(beta),
@@ -303,7 +277,7 @@ int dispatch_t(const void* x, const void* gamma, const void* beta, void* y, int6
                     if (D <= 32768) return launch_stage<DT, 256>(xs, gs, bs, ys, rows, D, stage_bytes, inv_D, eps, st);
                     return launch_stage<DT, 512>(xs, gs, bs, ys, rows, D, stage_bytes, inv_D, eps, st);
                 }
-                static const int resident = resident_ctas(layernorm_generic_kernel<DT>, kLnGenericThreads);
+                const int resident = resident_ctas(layernorm_generic_kernel<DT>, kLnGenericThreads, 0);
                 const int grid = (int)(rows < resident ? rows : resident);
                 layernorm_generic_kernel<DT><<<grid, kLnGenericThreads, 0, st>>>(xs, gs, bs, ys, rows, D, inv_D, eps);
                 count_launch();

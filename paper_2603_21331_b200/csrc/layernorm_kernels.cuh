@@ -114,11 +114,16 @@ __device__ __forceinline__ float first_elem(const void* row) {
 template <int THREADS, int GROUP, int VPT, int MINB, int DT = AK_DTYPE_BF16, bool P_EARLY = false>
 __global__ void __launch_bounds__(THREADS, MINB)
 layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamma, const uint4* __restrict__ beta,
-                     uint4* __restrict__ y, int64_t rows, int nvec, float inv_D, float eps) {
+                     uint4* __restrict__ y, int64_t rows, int nvec, float inv_D, float eps, int first_wave) {
     constexpr int GROUPS = THREADS / GROUP;
     constexpr int WARPS_PER_GROUP = GROUP / kWarp;
     static_assert(GROUP % kWarp == 0 && THREADS % GROUP == 0, "groups are whole warps");
     __shared__ float slots[2][THREADS / kWarp];
+    {
+        const int64_t r0 = (int64_t)blockIdx.x * GROUPS;
+        const int64_t nr = rows - r0 < GROUPS ? rows - r0 : GROUPS;
+        pdl_prologue(x + r0 * nvec, nr * nvec * 16, first_wave);
+    }
     const int g = threadIdx.x / GROUP;
     const int t = threadIdx.x % GROUP;
     const int lane = threadIdx.x & 31;

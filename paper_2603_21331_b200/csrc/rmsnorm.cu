@@ -20,11 +20,7 @@ namespace {
 template <int DT, int T>
 int launch_cluster_stage(const uint16_t* x, const uint16_t* w, uint16_t* y, int64_t rows, int64_t D, int64_t max_nv, int C,
                          float inv_D, float eps, cudaStream_t st) {
-    static const bool configured = [] {
-        return cudaFuncSetAttribute(rmsnorm_cluster_stage_kernel<T, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    kMaxRowSmemBytes) == cudaSuccess;
-    }();
-    if (!configured) return AK_ERR_CUDA;
+    if (!allow_big_smem(rmsnorm_cluster_stage_kernel<T, DT>)) return AK_ERR_CUDA;
     const size_t smem = (size_t)((max_nv + C - 1) / C) * 16;
     const cudaError_t e = launch_cluster(rmsnorm_cluster_stage_kernel<T, DT>, (unsigned)(rows * C), T, smem, C, st, x, w, y,
                                          D, C, inv_D, eps);
@@ -39,10 +35,13 @@ int launch_reg(const void* x, const void* w, void* y, int64_t rows, int nvec, fl
                cudaStream_t st) {
     constexpr int GROUPS = THREADS / GROUP;
     const int64_t grid = (rows + GROUPS - 1) / GROUPS;
-    rmsnorm_reg_kernel<THREADS, GROUP, VPT, MINB, WE, DT><<<(unsigned)grid, THREADS, 0, st>>>(
-        static_cast<const uint4*>(x), static_cast<const uint4*>(w), static_cast<uint4*>(y), rows, nvec, inv_D, eps);
+    auto kernel = rmsnorm_reg_kernel<THREADS, GROUP, VPT, MINB, WE, DT>;
+    const cudaError_t e = launch_dependent(kernel, dim3((unsigned)grid), dim3(THREADS), 0, st,
+                                           static_cast<const uint4*>(x), static_cast<const uint4*>(w),
+                                           static_cast<uint4*>(y), rows, nvec, inv_D, eps,
+                                           resident_ctas(kernel, THREADS, 0));
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+    return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
 // vectors per thread 1..MAXV for a fixed (THREADS, GROUP)
@@ -66,11 +65,7 @@ template <int DT, int THREADS>
 int launch_smem(const void* x, const void* w, void* y, int64_t rows, int nvec, float inv_D, float eps,
                 cudaStream_t st) {
     const size_t smem = (size_t)nvec * 16;
-    static const bool configured = [] {
-        return cudaFuncSetAttribute(rmsnorm_smem_kernel<THREADS, 1, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    kMaxRowSmemBytes) == cudaSuccess;
-    }();
-    if (!configured) return AK_ERR_CUDA;
+    if (!allow_big_smem(rmsnorm_smem_kernel<THREADS, 1, DT>)) return AK_ERR_CUDA;
     rmsnorm_smem_kernel<THREADS, 1, DT><<<(unsigned)rows, THREADS, smem, st>>>(
         static_cast<const uint4*>(x), static_cast<const uint4*>(w), static_cast<uint4*>(y), nvec, inv_D, eps);
     count_launch();
@@ -81,11 +76,7 @@ int launch_smem(const void* x, const void* w, void* y, int64_t rows, int nvec, f
 template <int DT, int THREADS>
 int launch_cluster_rows(const void* x, const void* w, void* y, int64_t rows, int nvec, int C, float inv_D, float eps,
                         cudaStream_t st) {
-    static const bool configured = [] {
-        return cudaFuncSetAttribute(rmsnorm_cluster_kernel<THREADS, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    kMaxRowSmemBytes) == cudaSuccess;
-    }();
-    if (!configured) return AK_ERR_CUDA;
+    if (!allow_big_smem(rmsnorm_cluster_kernel<THREADS, DT>)) return AK_ERR_CUDA;
     const size_t smem = (size_t)((nvec + C - 1) / C) * 16;
     const cudaError_t e = launch_cluster(rmsnorm_cluster_kernel<THREADS, DT>, (unsigned)(rows * C), THREADS, smem, C, st,
                                          static_cast<const uint4*>(x), static_cast<const uint4*>(w),
@@ -198,13 +189,7 @@ int dispatch_t(const void* x, const void* w, void* y, int64_t rows, int64_t D, f
         }
         case AK_PATH_GENERIC: {
             if constexpr (DT == AK_DTYPE_F32) {
-                static const int resident32 = [] {
-                    int per_sm = 0;
-                    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rmsnorm_generic32_kernel,
-                                                                      kRmsGenericThreads, 0) != cudaSuccess || per_sm < 1)
-                        per_sm = 1;
-                    return per_sm * sm_count();
-                }();
+                const int resident32 = resident_ctas(rmsnorm_generic32_kernel, kRmsGenericThreads, 0);
                 const int grid = (int)(rows < resident32 ? rows : resident32);
                 rmsnorm_generic32_kernel<<<grid, kRmsGenericThreads, 0, st>>>(
                     static_cast<const float*>(x), static_cast<const float*>(w), static_cast<float*>(y), rows, D, inv_D, eps);
@@ -234,15 +219,7 @@ int dispatch_t(const void* x, const void* w, void* y, int64_t rows, int64_t D, f
                 if (same_phase && is_aligned(w, 4) && max_nv <= 4096)   // ... 512 threads up to 4096
                     return launch_regp_vpt<DT, 512>((int)((max_nv + 511) / 512), xs, ws, ys, rows, D, inv_D, eps, st);
                 if (same_phase && is_aligned(w, 4) && stage_bytes <= (size_t)kMaxRowSmemBytes) {
-                    static const bool configured = [] {
-                        return cudaFuncSetAttribute(rmsnorm_stage_kernel<128, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                    kMaxRowSmemBytes) == cudaSuccess &&
-                               cudaFuncSetAttribute(rmsnorm_stage_kernel<256, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                    kMaxRowSmemBytes) == cudaSuccess &&
-                               cudaFuncSetAttribute(rmsnorm_stage_kernel<512, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                    kMaxRowSmemBytes) == cudaSuccess;
-                    }();
-                    if (!configured) return AK_ERR_CUDA;
+                    if (!allow_big_smem(rmsnorm_stage_kernel<128, DT>) || !allow_big_smem(rmsnorm_stage_kernel<256, DT>) || !allow_big_smem(rmsnorm_stage_kernel<512, DT>)) return AK_ERR_CUDA;
                     if (D <= 8192)
                         rmsnorm_stage_kernel<128, DT><<<(unsigned)rows, 128, stage_bytes, st>>>(xs, ws, ys, D, inv_D, eps);
                     else if (D <= 32768)
@@ -252,13 +229,7 @@ int dispatch_t(const void* x, const void* w, void* y, int64_t rows, int64_t D, f
                     count_launch();
                     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
                 }
-                static const int resident = [] {
-                    int per_sm = 0;
-                    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, rmsnorm_generic_kernel<DT>,
-                                                                      kRmsGenericThreads, 0) != cudaSuccess || per_sm < 1)
-                        per_sm = 1;
-                    return per_sm * sm_count();
-                }();
+                const int resident = resident_ctas(rmsnorm_generic_kernel<DT>, kRmsGenericThreads, 0);
                 const int grid = (int)(rows < resident ? rows : resident);
                 rmsnorm_generic_kernel<DT><<<grid, kRmsGenericThreads, 0, st>>>(xs, ws, ys, rows, D, inv_D, eps);
                 count_launch();

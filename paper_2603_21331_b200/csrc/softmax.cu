@@ -15,10 +15,12 @@ template <int DT, int THREADS, int GROUP, int VPT, int MINB>
 int launch_reg(const void* x, void* y, int64_t rows, int nvec, cudaStream_t st) {
     constexpr int GROUPS = THREADS / GROUP;
     const int64_t grid = (rows + GROUPS - 1) / GROUPS;
-    softmax_reg_kernel<THREADS, GROUP, VPT, MINB, false, DT><<<(unsigned)grid, THREADS, 0, st>>>(
-        static_cast<const uint4*>(x), static_cast<uint4*>(y), rows, nvec);
+    auto kernel = softmax_reg_kernel<THREADS, GROUP, VPT, MINB, false, DT>;
+    const cudaError_t e = launch_dependent(kernel, dim3((unsigned)grid), dim3(THREADS), 0, st,
+                                           static_cast<const uint4*>(x), static_cast<uint4*>(y), rows, nvec,
+                                           resident_ctas(kernel, THREADS, 0));
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+    return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
 template <int DT, int THREADS, int GROUP, int MINB_LO, int MINB_HI>
@@ -39,24 +41,18 @@ int launch_reg_vpt(int vpt, const void* x, void* y, int64_t rows, int nvec, cuda
 template <int DT, int THREADS, int KEEP>
 int launch_smem(const void* x, void* y, int64_t rows, int nvec, cudaStream_t st) {
     const size_t smem = (size_t)nvec * 16;
-    static const bool configured = [] {
-        return cudaFuncSetAttribute(softmax_smem_kernel<THREADS, 1, KEEP, DT>,
-                                    cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxRowSmemBytes) == cudaSuccess;
-    }();
-    if (!configured) return AK_ERR_CUDA;
-    softmax_smem_kernel<THREADS, 1, KEEP, DT><<<(unsigned)rows, THREADS, smem, st>>>(
-        static_cast<const uint4*>(x), static_cast<uint4*>(y), nvec);
+    if (!allow_big_smem(softmax_smem_kernel<THREADS, 1, KEEP, DT>)) return AK_ERR_CUDA;
+    auto kernel = softmax_smem_kernel<THREADS, 1, KEEP, DT>;
+    const cudaError_t e = launch_dependent(kernel, dim3((unsigned)rows), dim3(THREADS), smem, st,
+                                           static_cast<const uint4*>(x), static_cast<uint4*>(y), nvec,
+                                           resident_ctas(kernel, THREADS, smem));
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+    return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
 template <int DT, int T>
 int launch_stage(const uint16_t* x, uint16_t* y, int64_t rows, int64_t D, size_t stage_bytes, cudaStream_t st) {
-    static const bool configured = [] {
-        return cudaFuncSetAttribute(softmax_stage_kernel<T, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    kMaxRowSmemBytes) == cudaSuccess;
-    }();
-    if (!configured) return AK_ERR_CUDA;
+    if (!allow_big_smem(softmax_stage_kernel<T, DT>)) return AK_ERR_CUDA;
     softmax_stage_kernel<T, DT><<<(unsigned)rows, T, stage_bytes, st>>>(x, y, D);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
@@ -65,11 +61,7 @@ int launch_stage(const uint16_t* x, uint16_t* y, int64_t rows, int64_t D, size_t
 // unaligned rows split over a cluster of C CTAs (covering vectors of the worst phase: max_nv)
 template <int DT, int T>
 int launch_cluster_stage(const uint16_t* x, uint16_t* y, int64_t rows, int64_t D, int64_t max_nv, int C, cudaStream_t st) {
-    static const bool configured = [] {
-        return cudaFuncSetAttribute(softmax_cluster_stage_kernel<T, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    kMaxRowSmemBytes) == cudaSuccess;
-    }();
-    if (!configured) return AK_ERR_CUDA;
+    if (!allow_big_smem(softmax_cluster_stage_kernel<T, DT>)) return AK_ERR_CUDA;
     const size_t smem = (size_t)((max_nv + C - 1) / C) * 16;
     const cudaError_t e = launch_cluster(softmax_cluster_stage_kernel<T, DT>, (unsigned)(rows * C), T, smem, C, st, x, y, D, C);
     count_launch();
@@ -85,11 +77,7 @@ int launch_regp(const uint16_t* x, uint16_t* y, int64_t rows, int64_t D, cudaStr
 // a cluster of C CTAs per row (C from cluster_ctas, at least 2)
 template <int DT, int THREADS, int KEEP>
 int launch_cluster_rows(const void* x, void* y, int64_t rows, int nvec, int C, cudaStream_t st) {
-    static const bool configured = [] {
-        return cudaFuncSetAttribute(softmax_cluster_kernel<THREADS, KEEP, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    kMaxRowSmemBytes) == cudaSuccess;
-    }();
-    if (!configured) return AK_ERR_CUDA;
+    if (!allow_big_smem(softmax_cluster_kernel<THREADS, KEEP, DT>)) return AK_ERR_CUDA;
     const size_t smem = (size_t)((nvec + C - 1) / C) * 16;
     const cudaError_t e = launch_cluster(softmax_cluster_kernel<THREADS, KEEP, DT>, (unsigned)(rows * C), THREADS, smem, C, st,
                                          static_cast<const uint4*>(x), static_cast<uint4*>(y), nvec, C);
@@ -111,14 +99,6 @@ int launch_regp_vpt(int vpt, const uint16_t* x, uint16_t* y, int64_t rows, int64
         case 8: return launch_regp<DT, THREADS, 8, MINB>(x, y, rows, D, st);
         default: return AK_ERR_SHAPE;
     }
-}
-
-template <typename K>
-int resident_ctas(K kernel, int threads) {
-    int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, 0) != cudaSuccess || per_sm < 1)
-        per_sm = 1;
-    return per_sm * sm_count();
 }
 
 template <int DT>
@@ -179,7 +159,7 @@ int dispatch_t(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st,
         }
         case AK_PATH_GENERIC: {
             if constexpr (DT == AK_DTYPE_F32) {
-                static const int resident = resident_ctas(softmax_generic32_kernel, kSmGenericThreads);
+                const int resident = resident_ctas(softmax_generic32_kernel, kSmGenericThreads, 0);
                 const int grid = (int)(rows < resident ? rows : resident);
                 softmax_generic32_kernel<<<grid, kSmGenericThreads, 0, st>>>(
                     static_cast<const float*>(x), static_cast<float*>(y), rows, D);
@@ -212,7 +192,7 @@ int dispatch_t(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st,
                     if (D <= 32768) return launch_stage<DT, 256>(xs, ys, rows, D, stage_bytes, st);
                     return launch_stage<DT, 512>(xs, ys, rows, D, stage_bytes, st);
                 }
-                static const int resident = resident_ctas(softmax_generic_kernel<DT>, kSmGenericThreads);
+                const int resident = resident_ctas(softmax_generic_kernel<DT>, kSmGenericThreads, 0);
                 const int grid = (int)(rows < resident ? rows : resident);
                 softmax_generic_kernel<DT><<<grid, kSmGenericThreads, 0, st>>>(xs, ys, rows, D);
                 count_launch();

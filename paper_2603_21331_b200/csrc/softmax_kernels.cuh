@@ -100,11 +100,16 @@ template <int DT> constexpr int kExpPairs = (DT == AK_DTYPE_F32) ? 2 : 4;
 // rows too long to hold in fp32.
 template <int THREADS, int GROUP, int VPT, int MINB, bool RECOMPUTE, int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(THREADS, MINB)
-softmax_reg_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t rows, int nvec) {
+softmax_reg_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t rows, int nvec, int first_wave) {
     constexpr int GROUPS = THREADS / GROUP;
     constexpr int WARPS_PER_GROUP = GROUP / kWarp;
     static_assert(GROUP % kWarp == 0 && THREADS % GROUP == 0, "groups are whole warps");
     __shared__ float slots[2][THREADS / kWarp];
+    {
+        const int64_t r0 = (int64_t)blockIdx.x * GROUPS;
+        const int64_t nr = rows - r0 < GROUPS ? rows - r0 : GROUPS;
+        pdl_prologue(x + r0 * nvec, nr * nvec * 16, first_wave);
+    }
     const int g = threadIdx.x / GROUP;
     const int t = threadIdx.x % GROUP;
     const int lane = threadIdx.x & 31;
@@ -164,12 +169,13 @@ constexpr uint32_t kSmBulkChunk = 32768;
 
 template <int THREADS, int MINB, int KEEP, int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(THREADS, MINB)
-softmax_smem_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int nvec) {
+softmax_smem_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int nvec, int first_wave) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint4* row = reinterpret_cast<const uint4*>(smem_raw);
     __shared__ uint64_t bar;
     __shared__ float slots[2 * kWarp];
     const int64_t r = blockIdx.x;
+    pdl_prologue(x + r * nvec, (int64_t)nvec * 16, first_wave);
     if (threadIdx.x == 0) mbar_init(&bar, 1);
     __syncthreads();
     if (threadIdx.x == 0) {

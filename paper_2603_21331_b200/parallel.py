@@ -57,6 +57,16 @@ def gather_partials(partial: torch.Tensor, group=None) -> torch.Tensor:
     return out
 
 
+def _stream_of(stream, device: torch.device) -> "torch.cuda.Stream":
+    """``stream`` (None = the current one, a torch stream, or a raw cudaStream_t handle) as a torch
+    stream object of ``device``."""
+    if stream is None:
+        return torch.cuda.current_stream(device)
+    if isinstance(stream, torch.cuda.Stream):
+        return stream
+    return torch.cuda.ExternalStream(int(stream), device=device)
+
+
 def vocab_parallel_xent(logits_shard: torch.Tensor, targets: torch.Tensor, vocab_start: int, V_total: int,
                         ignore_index: int = -100, group=None, stream=None, nsplit: int = 0):
     """Cross-entropy of [rows, V_total] logits whose columns are sharded over the ranks of
@@ -68,23 +78,25 @@ def vocab_parallel_xent(logits_shard: torch.Tensor, targets: torch.Tensor, vocab
     if nsplit == 0:
         world = dist.get_world_size(group)
         nsplit = binding.ak_xent_vp_nsplit(rows, shard_vocab(V_total, 0, world)[1])
-    part = binding.ak_xent_vp_partial(logits_shard, targets, vocab_start, V_total, nsplit, ignore_index,
-                                      stream=stream)
-    parts = gather_partials(part, group)
-    return binding.ak_xent_vp_merge(parts, targets, V_total, ignore_index, stream=stream)
+    # The collective orders itself against the CURRENT stream, so `stream` is made current for
+    # the whole sequence: partial kernel -> all-gather -> merge kernel run in that order on it.
+    st = _stream_of(stream, logits_shard.device)
+    with torch.cuda.stream(st):
+        part = binding.ak_xent_vp_partial(logits_shard, targets, vocab_start, V_total, nsplit, ignore_index,
+                                          stream=st)
+        parts = gather_partials(part, group)
+        return binding.ak_xent_vp_merge(parts, targets, V_total, ignore_index, stream=st)
 
 
 def global_xent_mean(loss_rows: torch.Tensor, targets: torch.Tensor, ignore_index: int = -100,
                      group=None, stream=None) -> torch.Tensor:
-    """Mean cross-entropy over all ranks' rows (device tensors; kernels from libak)."""
+    """Mean cross-entropy over all ranks' rows (device tensors; kernels from libak).  The two
+    kernels and the 16-byte all-gather between them run on ``stream`` (default: the current one),
+    which is made current for the sequence because the collective orders itself against the
+    current stream."""
     from . import binding
-    lib = binding.lib()
-    st = binding._stream_ptr(stream)
-    pair = torch.empty((2,), dtype=torch.float64, device=loss_rows.device)
-    binding._check(lib.ak_xent_sum_count(loss_rows.data_ptr(), targets.data_ptr(), ignore_index,
-                                         loss_rows.numel(), pair.data_ptr(), st), "ak_xent_sum_count")
-    pairs = gather_pairs(pair, group)
-    mean = torch.empty((1,), dtype=torch.float32, device=loss_rows.device)
-    binding._check(lib.ak_xent_mean_merge(pairs.data_ptr(), pairs.shape[0], mean.data_ptr(), st),
-                   "ak_xent_mean_merge")
-    return mean
+    st = _stream_of(stream, loss_rows.device)
+    with torch.cuda.stream(st):
+        pair = binding.ak_xent_sum_count(loss_rows, targets, ignore_index, stream=st)
+        pairs = gather_pairs(pair, group)
+        return binding.ak_xent_mean_merge(pairs, stream=st)
