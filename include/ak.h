@@ -23,7 +23,18 @@
  *     Device entry points only enqueue work; they never synchronise.
  *   - The return value is an ak_status.  Arguments are validated on the host before any
  *     launch.  Data-dependent problems (an out-of-range target) cannot be reported
- *     synchronously and are encoded in the output (NaN); no kernel ever traps.
+ *     synchronously and are encoded in the output (NaN); no kernel ever traps.  The one
+ *     device-side failure that is not encoded in the output, a bounded wait that gave up, is
+ *     reported by ak_wait_timeouts().
+ *   - Calls act on the CURRENT CUDA device: pointers must belong to it, and a process that
+ *     drives several GPUs makes the tensors' device current before each call (the Python
+ *     binding does).  Function attributes, occupancy figures, scratch pools, the host-buffer
+ *     arena and the static scratch are kept per device.
+ *   - Kernels are launched as programmatic dependents (programmatic stream serialisation): their
+ *     CTAs may become resident while the previous kernel of the stream drains, but every read and
+ *     write comes after griddepcontrol.wait, i.e. after that kernel has completed and flushed;
+ *     before the wait they only prefetch their first inputs into L2.  Stream order is therefore
+ *     observed exactly as for ordinary launches, with any kernel before or after.
  *   - Stream-ordered scratch, where an entry point says it uses some, comes from a CUDA
  *     memory pool of the library's own (one per device, created at first use, keeps up to
  *     256 MiB cached between calls) through cudaMallocFromPoolAsync / cudaFreeAsync on the
@@ -91,6 +102,10 @@ enum {
  *   y[r, j] = bf16_rne( x[r, j] * w[j] * rsqrt( (1/D) sum_k x[r, k]^2 + eps ) )
  * x, y: device bf16 [rows, D]; w: device bf16 [D]; accumulation in fp32.
  * eps must be finite and >= 0.
+ * Range: the squares are added in fp32, so a row whose sum of squares exceeds 3.4e38 (|x| of
+ * about 1e19 / sqrt(D) and more; bf16 itself reaches 3.4e38) gives inf, rstd = 0 and an output
+ * row of exact zeros where the definition gives about +-w.  (LayerNorm likewise returns beta for
+ * a row whose squared deviations overflow.)  Softmax and cross-entropy have no such limit.
  */
 int ak_rmsnorm_fwd(const void* x, const void* w, void* y,
                    int64_t rows, int64_t D, float eps, void* cuda_stream);
@@ -131,9 +146,11 @@ int ak_rowsum_fwd_dt(const void* x, float* out, int64_t rows, int64_t D, int dty
  *     y[2i]     = rne( x[2i] cos(theta) - x[2i + 1] sin(theta) )
  *     y[2i + 1] = rne( x[2i] sin(theta) + x[2i + 1] cos(theta) )
  * Dh even, 2 <= Dh <= 512 (else AK_ERR_SHAPE); base finite and > 0 (typically 10000);
- * 0 <= pos_offset < 2^52.  Frequencies are formed in double on the host, angles reduced in
- * double on the device, so cos / sin are right to fp32 rounding at any position; products
- * and sums in fp32.  Fast path: 16-byte aligned x and y and Dh a multiple of the elements in
+ * 0 <= pos_offset < 2^52.  Frequencies f_i = base^(-2i / Dh) are formed in double on the host;
+ * the angle is the double product fl(p * f_i), reduced to [-pi, pi] in double on the device, so
+ * cos / sin of that angle are right to fp32 rounding at any accepted position.  The double
+ * product itself is within p * f_i * 2^-53 rad of the real one: below fp32's rounding while
+ * p * f_i < 2^28, 6e-5 rad at 2^40.  Products and sums in fp32.  Fast path: 16-byte aligned x and y and Dh a multiple of the elements in
  * 16 bytes; anything else takes an element-wise kernel.  One launch, no scratch.
  */
 int ak_rope_fwd(const void* x, void* y, int64_t n_seq, int64_t S, int64_t Dh, float base,
@@ -195,7 +212,7 @@ int ak_layernorm_fwd_path(const void* x, const void* gamma, const void* beta, vo
  * Row-sum reduce (Table 3 "reduce").
  *   out[r] = fp32( sum_k x[r, k] ),  fp32 accumulation in a fixed order
  * x: device bf16 [rows, D], 2-byte aligned, any D >= 1; out: device fp32 [rows], caller
- * owned.  One launch and no scratch, except for a few long rows (rows < 592 and D >= 16384; a
+ * owned.  One launch and no scratch, except for a few long rows (rows < 4 * SMs = 592 and D >= 16384; a
  * vector sum is rows == 1): then nsplit CTAs per row write partial sums and a second launch
  * adds them in a fixed order, with rows * nsplit * 4 bytes of stream-ordered scratch obtained
  * and released on `cuda_stream` (AK_ERR_NOMEM if that fails).  inf/NaN propagate per IEEE-754.
@@ -323,7 +340,8 @@ int ak_sol_read(const void* src, size_t bytes, void* sink4, void* cuda_stream);
  * Introspection.
  */
 /* Path id the dispatcher picks for (rows, D) with fully aligned pointers (`aligned16` != 0)
- * or not.  Pure functions; no CUDA calls. */
+ * or not.  Pure functions of their arguments and of the current device's SM count (which decides
+ * when few rows are split over more CTAs); they launch nothing. */
 int ak_rmsnorm_choose_path(int64_t rows, int64_t D, int aligned16);
 int ak_layernorm_choose_path(int64_t rows, int64_t D, int aligned16);
 int ak_softmax_choose_path(int64_t rows, int64_t D, int aligned16);
@@ -332,6 +350,22 @@ int ak_xent_choose_path(int64_t rows, int64_t V, int* nsplit_out);
 
 /* Number of kernel launches this library has enqueued in this process so far. */
 int64_t ak_launch_count(void);
+
+/* SMs of the current device as the dispatch rules see them (148 on a full B200; also 148 when
+ * no device can be queried).  The split rules are stated in multiples of it: cross-entropy
+ * splits rows when rows < 4 * SMs, the row sum when rows < 4 * SMs as well. */
+int ak_sm_count(void);
+
+/* Bounded waits.  The kernels that stage rows through shared memory wait for their own bulk
+ * copies (and, in the cluster layouts, for their cluster partners' mailbox posts) on mbarriers,
+ * polling at most 2^20 times; they never spin without a limit and never trap.  A wait that gives
+ * up is not expected on a healthy device; the threads that hit it stop and leave their part of
+ * the output unwritten, and a flag is set on the device.  The status of the call that launched
+ * the kernel cannot show this (calls only enqueue): this function reads the flags of the
+ * current device, synchronising with it, and returns 0 if no wait ever gave up, the number of
+ * kernel families (RMSNorm, softmax, LayerNorm) that saw one otherwise, -1 if the flags cannot be
+ * read (no device).  The flags stay set until the process ends. */
+int ak_wait_timeouts(void);
 
 /* Static, never-freed description of a status code. */
 const char* ak_status_string(int status);

@@ -70,6 +70,8 @@ SIGNATURES = {
     "ak_softmax_choose_path": (_int, [_i64, _i64, _int]),
     "ak_xent_choose_path": (_int, [_i64, _i64, ctypes.POINTER(_int)]),
     "ak_launch_count": (_i64, []),
+    "ak_sm_count": (_int, []),
+    "ak_wait_timeouts": (_int, []),
     "ak_status_string": (ctypes.c_char_p, [_int]),
     "ak_version": (_int, []),
 }
@@ -551,6 +553,15 @@ def ak_xent_choose_path(rows: int, V: int) -> Tuple[int, int]:
     ns = ctypes.c_int(0)
     path = int(lib().ak_xent_choose_path(rows, V, ctypes.byref(ns)))
     return path, int(ns.value)
+
+
+def ak_sm_count() -> int:
+    return int(lib().ak_sm_count())
+
+
+def ak_wait_timeouts() -> int:
+    """0 if no bounded wait of a kernel ever gave up on the current device (see ak.h); synchronises."""
+    return int(lib().ak_wait_timeouts())
 
 
 def ak_launch_count() -> int:

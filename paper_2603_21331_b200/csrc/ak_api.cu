@@ -163,8 +163,10 @@ int validate_softmax(const void* x, void* y, int64_t rows, int64_t D, size_t esi
     if (!is_aligned(x, esize) || !is_aligned(y, esize)) return AK_ERR_ALIGN;
     return AK_OK;
 }
+}  // namespace
+
 int validate_xent(const void* logits, const int64_t* targets, float* loss_rows, float* loss_mean,
-                  int64_t rows, int64_t V, size_t esize = 2) {
+                  int64_t rows, int64_t V, size_t esize) {
     if (rows != 0 && (!logits || !targets || !loss_rows)) return AK_ERR_NULL;
     if (int s = check_rows_cols(rows, V)) return s;
     if (!is_aligned(logits, esize) || !is_aligned(targets, 8) || !is_aligned(loss_rows, 4) ||
@@ -173,7 +175,6 @@ int validate_xent(const void* logits, const int64_t* targets, float* loss_rows, 
     return AK_OK;
 }
 
-}  // namespace
 }  // namespace ak
 
 using namespace ak;
@@ -389,6 +390,14 @@ int ak_xent_choose_path(int64_t rows, int64_t V, int* nsplit_out) { return xent_
 
 int64_t ak_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
+int ak_sm_count(void) { return sm_count(); }
+
+int ak_wait_timeouts(void) {
+    const int a = rmsnorm_wait_timeouts(), b = softmax_wait_timeouts(), c = layernorm_wait_timeouts();
+    if (a < 0 || b < 0 || c < 0) return -1;
+    return (a != 0) + (b != 0) + (c != 0);
+}
+
 const char* ak_status_string(int status) {
     switch (status) {
         case AK_OK: return "ok";
@@ -578,10 +587,11 @@ int ak_xent_fwd_host(const void* logits_host, const int64_t* targets_host, int64
     std::lock_guard<std::mutex> lock(g_arena_mu);
     const int64_t rc = rows_per_chunk(rows, V);
     const size_t chunk = (size_t)rc * (size_t)V * 2;
-    // per-lane scratch for the split-row path lives in the lane's `out` buffer
-    int ns = 1;
-    xent_choose(rc, V, &ns);
-    const size_t ws_bytes = (size_t)rc * 64 * sizeof(float2);  // enough for any split count
+    // per-lane scratch for the split-row path lives in the lane's `out` buffer: what a full chunk
+    // and the last, shorter chunk need (nothing when both take one CTA per row)
+    const int64_t tail_rows = rows % rc;
+    size_t ws_bytes = ak_xent_workspace_bytes(rc, V);
+    if (tail_rows > 0 && ak_xent_workspace_bytes(tail_rows, V) > ws_bytes) ws_bytes = ak_xent_workspace_bytes(tail_rows, V);
     // aux: targets [rows] int64 | loss rows [rows] fp32 | mean fp32 (8-byte slots)
     const size_t t_bytes = (size_t)rows * 8, l_bytes = ((size_t)rows * 4 + 7) & ~(size_t)7;
     Arena* a = nullptr;
@@ -599,7 +609,8 @@ int ak_xent_fwd_host(const void* logits_host, const int64_t* targets_host, int64
         const size_t bytes = (size_t)nr * (size_t)V * 2, off = (size_t)r0 * (size_t)V * 2;
         AK_TRY_CUDA(cudaMemcpyAsync(a->in[lane], xs + off, bytes, cudaMemcpyHostToDevice, a->st[lane]));
         if (int s = xent_dispatch(a->in[lane], d_targets + r0, ignore_index, d_loss + r0, nullptr, nr, V,
-                                  a->out[lane], a->out_cap, false, a->st[lane], AK_XENT_AUTO, 0)) {
+                                  ws_bytes ? a->out[lane] : nullptr, ws_bytes ? a->out_cap : 0, false, a->st[lane],
+                                  AK_XENT_AUTO, 0)) {
             sync_all(*a);
             return s;
         }

@@ -233,9 +233,23 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, 
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
 }
-// Set when a bounded wait gave up (never expected; a kernel that sees it returns early and
-// leaves its outputs unwritten rather than spinning).
+// Set when a bounded wait gave up (never expected; a thread that sees it returns early and
+// leaves its outputs unwritten rather than spinning).  The library is built without relocatable
+// device code, so every translation unit that includes this header has its own copy of the flag;
+// each of them that waits on mbarriers exports a reader (AK_DEFINE_WAIT_TIMEOUT_READER) and
+// ak_wait_timeouts() adds them up.
 static __device__ int g_wait_timeout;
+// Host side: this translation unit's flag on the current device (-1 if it cannot be read).
+static inline int read_wait_timeout_flag() {
+    int v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_wait_timeout, sizeof(int)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return -1;
+    }
+    return v;
+}
+#define AK_DEFINE_WAIT_TIMEOUT_READER(name) \
+    int name() { return read_wait_timeout_flag(); }
 // Bounded wait for the phase with the given parity.  Returns false after ~2^20 polls.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     for (int it = 0; it < (1 << 20); ++it) {
@@ -344,6 +358,10 @@ int cluster_ctas(int64_t rows, int64_t row_bytes, int64_t split_from);
 // faster: softmax 16384 x 32768 317 us against 338 us in clusters of two)
 constexpr int64_t kClusterFrom = 65536 + 16;
 int sm_count();  // SMs of the current device (cached per device)
+// per translation unit: has a bounded mbarrier wait of its kernels ever given up on this device?
+int rmsnorm_wait_timeouts();
+int softmax_wait_timeouts();
+int layernorm_wait_timeouts();
 // Per-device memos, keyed by kernel (a process may drive several GPUs, and function attributes
 // and occupancy belong to the device that is current at the call):
 //   dyn_smem_configured  cudaFuncAttributeMaxDynamicSharedMemorySize = kMaxRowSmemBytes set once
@@ -388,6 +406,10 @@ int rowsum_dispatch(const void* x, float* out, int64_t rows, int64_t D, cudaStre
 int rmsnorm_choose(int64_t rows, int64_t D, bool aligned16, int dtype = AK_DTYPE_BF16);
 int softmax_choose(int64_t rows, int64_t D, bool aligned16, int dtype = AK_DTYPE_BF16);
 int xent_choose(int64_t rows, int64_t V, int* nsplit);
+
+// Argument checks shared by every cross-entropy entry point (pointers, shape limits, alignment).
+int validate_xent(const void* logits, const int64_t* targets, float* loss_rows, float* loss_mean,
+                  int64_t rows, int64_t V, size_t esize = 2);
 
 inline int dtype_bytes(int dtype) { return dtype == AK_DTYPE_F32 ? 4 : 2; }
 inline bool is_aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }

@@ -311,4 +311,6 @@ int layernorm_dispatch(const void* x, const void* gamma, const void* beta, void*
     }
 }
 
+AK_DEFINE_WAIT_TIMEOUT_READER(layernorm_wait_timeouts)
+
 }  // namespace ak

@@ -211,7 +211,7 @@ layernorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gam
         for (uint32_t off = 0; off < bytes; off += kLnBulkChunk)
             bulk_load(smem_raw + off, src + off, min(kLnBulkChunk, bytes - off), &bar);
     }
-    if (!mbar_wait(&bar, 0)) return;  // uniform: every thread waits on the same barrier
+    if (!mbar_wait(&bar, 0)) return;  // gave up (flag set, see ak_wait_timeouts): a thread that exits no longer counts at later barriers
     float K;
     if constexpr (DT == AK_DTYPE_F32) K = reinterpret_cast<const float*>(smem_raw)[0];
     else K = Elem<DT>::to_float(reinterpret_cast<const uint16_t*>(smem_raw)[0]);
@@ -388,7 +388,7 @@ layernorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restric
     stage_interior_bulk(smem_raw, xa, k_lo, k_hi, &bar);   // the copy engine brings the inside vectors
     if (edge) row16[ek * 8 + (threadIdx.x & 7)] = ld_stream_u16(xr + ej);
     __syncthreads();
-    if (!mbar_wait(&bar, 0)) return;  // uniform: every thread waits on the same barrier
+    if (!mbar_wait(&bar, 0)) return;  // gave up (flag set, see ak_wait_timeouts): a thread that exits no longer counts at later barriers
     const float K = Elem<DT>::to_float(row16[phase]);
     float s1 = 0.0f;
     for (int k = k_lo + threadIdx.x; k < k_hi; k += T) s1 += sumdev_v<DT>(row[k], K);

@@ -253,4 +253,6 @@ int rmsnorm_dispatch(const void* x, const void* w, void* y, int64_t rows, int64_
     }
 }
 
+AK_DEFINE_WAIT_TIMEOUT_READER(rmsnorm_wait_timeouts)
+
 }  // namespace ak

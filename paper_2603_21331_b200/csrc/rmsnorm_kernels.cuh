@@ -166,7 +166,7 @@ rmsnorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w, ui
         for (uint32_t off = 0; off < bytes; off += kBulkChunk)
             bulk_load(smem_raw + off, src + off, min(kBulkChunk, bytes - off), &bar);
     }
-    if (!mbar_wait(&bar, 0)) return;  // uniform: every thread waits on the same barrier
+    if (!mbar_wait(&bar, 0)) return;  // gave up (flag set, see ak_wait_timeouts): a thread that exits no longer counts at later barriers
     float ss = 0.0f;
 #pragma unroll 4
     for (int i = threadIdx.x; i < nvec; i += THREADS) ss += sumsq_v<DT>(row[i]);
@@ -313,7 +313,7 @@ rmsnorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict_
         }
     }
     __syncthreads();
-    if (!mbar_wait(&bar, 0)) return;  // uniform: every thread waits on the same barrier
+    if (!mbar_wait(&bar, 0)) return;  // gave up (flag set, see ak_wait_timeouts): a thread that exits no longer counts at later barriers
     float ss = 0.0f;
     for (int k = threadIdx.x; k < nv; k += T) ss += sumsq_v<DT>(row[k]);
     ss = cta_sum<T>(ss, slots, 0);

@@ -10,9 +10,14 @@
 // them: the transcendental work is amortised over n_seq / chunks rows and the inner loop is
 // a handful of packed multiply-adds per 16 bytes.  Since the trigonometry is off the hot loop
 // it can afford to be exact: the frequencies base^(-2i/Dh) are computed on the host in double
-// and travel as kernel parameters; the angle is formed and reduced to [-pi, pi] in double, and
-// only the reduced argument goes to single-precision sincosf (its accurate small-argument
-// branch).  The cosine and sine are therefore right to fp32 rounding at any position.
+// and travel as kernel parameters; the angle is the double product fl(p * f) - the angle an
+// fp64 evaluation of the definition uses - reduced to [-pi, pi] in double with a two-term 2 pi,
+// and only the reduced argument goes to single-precision sincosf (its accurate small-argument
+// branch).  The cosine and sine OF THAT ANGLE are right to fp32 rounding at any position up to
+// 2^52.  Against the real-number product the angle itself carries the rounding of the double
+// multiplication, at most p * f * 2^-53 rad: below fp32's own rounding while p * f < 2^28, 6e-5
+// rad at p * f = 2^40.  (Carrying the product's low part would remove that, and would then
+// disagree with every fp64 evaluation of p * f by the same amount: not done.)
 #include <cmath>
 
 #include "ak_common.cuh"
@@ -146,7 +151,8 @@ rope_pair_kernel(const void* __restrict__ xv, void* __restrict__ yv, int64_t n_s
 // (Timed on B200 for 296 .. 4736 CTAs and 4 / 8 / 16 sequences: within 10 % of each other; this
 // choice was best or tied on every shape.)
 void chunking(int64_t gx, int64_t n_seq, int* seq_per_cta, unsigned* gy) {
-    constexpr int64_t target = 148 * 32, minseq = 8;
+    const int64_t target = (int64_t)sm_count() * 32;
+    constexpr int64_t minseq = 8;
     int64_t want = (target + gx - 1) / gx;
     int64_t most = n_seq / minseq > 1 ? n_seq / minseq : 1;
     if (want > most) want = most;

@@ -136,10 +136,11 @@ rowsum_finish_kernel(const float* __restrict__ partial, float* __restrict__ out,
     if (threadIdx.x == 0) out[row] = s;
 }
 
-// Split count: a pure function of (rows, D).  Enough CTAs for about one wave, more for very
+// Split count: a pure function of (rows, D) and the device's SM count.  Enough CTAs for about one wave, more for very
 // long rows (slices of about 64K elements), slices of at least 8192 elements, at most 8192 of them.
 int rowsum_nsplit(int64_t rows, int64_t D) {
-    constexpr int64_t kTargetCtas = 148 * 8, kMinSlice = 8192;
+    const int64_t kTargetCtas = (int64_t)sm_count() * 8;   // 1184 on a full B200
+    constexpr int64_t kMinSlice = 8192;
     if (rows <= 0 || rows >= kTargetCtas / 2) return 1;
     int64_t want = (kTargetCtas + rows - 1) / rows;
     if (want < D / 65536) want = D / 65536;

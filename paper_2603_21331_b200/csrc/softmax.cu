@@ -225,4 +225,6 @@ int softmax_dispatch(const void* x, void* y, int64_t rows, int64_t D, cudaStream
     }
 }
 
+AK_DEFINE_WAIT_TIMEOUT_READER(softmax_wait_timeouts)
+
 }  // namespace ak

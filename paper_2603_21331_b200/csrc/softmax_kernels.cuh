@@ -185,7 +185,7 @@ softmax_smem_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int nvec
         for (uint32_t off = 0; off < bytes; off += kSmBulkChunk)
             bulk_load(smem_raw + off, src + off, min(kSmBulkChunk, bytes - off), &bar);
     }
-    if (!mbar_wait(&bar, 0)) return;  // uniform: every thread waits on the same barrier
+    if (!mbar_wait(&bar, 0)) return;  // gave up (flag set, see ak_wait_timeouts): a thread that exits no longer counts at later barriers
 
     uint32_t mx = neg_inf_word<DT>();
 #pragma unroll 4
@@ -368,7 +368,7 @@ softmax_stage_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, i
     stage_interior_bulk(smem_raw, xa, k_lo, k_hi, &bar);   // the copy engine brings the inside vectors
     if (my_edge) row16[my_edge_k * 8 + (threadIdx.x & 7)] = (my_j >= 0 && my_j < D) ? ld_stream_u16(xr + my_j) : Elem<DT>::kNegInf;
     __syncthreads();
-    if (!mbar_wait(&bar, 0)) return;  // uniform: every thread waits on the same barrier
+    if (!mbar_wait(&bar, 0)) return;  // gave up (flag set, see ak_wait_timeouts): a thread that exits no longer counts at later barriers
 
     uint32_t mx = neg_inf_word<DT>();
     for (int k = threadIdx.x; k < nv; k += T) mx = max_w<DT>(mx, max_v<DT>(row[k]));

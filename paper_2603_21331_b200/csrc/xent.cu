@@ -51,11 +51,11 @@ int launch_finish(const typename XElem<DT>::type* logits, const int64_t* targets
 }  // namespace
 
 // Split when one CTA per row cannot fill the machine (few rows) and the row is long
-// enough for slices of about 16384 elements.  Pure function of (rows, V).  (Timed for 1 .. 512
+// enough for slices of about 16384 elements.  Pure function of (rows, V) and the device's SM count.  (Timed for 1 .. 512
 // rows with 2 .. 64 slices: about four CTAs per SM in total and slices no shorter than that were
 // best or tied: 64 x 128256 13.4 -> 9.6 us, 16 x 128256 8.7 -> 7.3 us against eight per SM / 8192.)
 int xent_choose(int64_t rows, int64_t V, int* nsplit) {
-    constexpr int64_t kTargetCtas = 148 * 4;
+    const int64_t kTargetCtas = (int64_t)sm_count() * 4;   // 592 on a full B200: a fixed number for a given device
     constexpr int64_t kMinSlice = 16384;      // elements
     int ns = 1;
     if (rows > 0 && rows < kTargetCtas) {

@@ -59,11 +59,7 @@ using namespace ak;
 extern "C" int ak_xent_fwd_static(const void* logits, const int64_t* targets, int64_t ignore_index,
                                   float* loss_rows, float* loss_mean, int64_t rows, int64_t V,
                                   void* cuda_stream) {
-    if (rows < 0 || V <= 0) return AK_ERR_SHAPE;
-    if (rows != 0 && (!logits || !targets || !loss_rows)) return AK_ERR_NULL;
-    if (!is_aligned(logits, 2) || !is_aligned(targets, 8) || !is_aligned(loss_rows, 4) ||
-        (loss_mean && !is_aligned(loss_mean, 4)))
-        return AK_ERR_ALIGN;
+    if (int s = validate_xent(logits, targets, loss_rows, loss_mean, rows, V)) return s;
     int nsplit = 1;
     xent_choose(rows, V, &nsplit);  // same split count as the allocating entry point would use
     // capacity check before anything is launched: rows * nsplit pairs of 8 bytes

@@ -4,7 +4,8 @@ Every value is a mathematical closed form evaluated with 40-digit arithmetic (mp
 only: nothing from the CPU checker or the CUDA library is called), so the checker can
 be pinned to numbers it did not produce.  The paper prints no worked numeric example
 for these ops; the closed forms are the ones its correctness stages imply (Section 4:
-identical-value rows, near-zero variance) and the benchmark brief lists.
+identical-value rows, near-zero variance) together with textbook identities of the ops
+(softplus, log V for equal logits, the 3-4-5 row, cos / sin of small integers).
 
 Run:  python tests/golden/make_closed_forms.py
 """

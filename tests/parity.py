@@ -76,6 +76,35 @@ def assert_close_dt(gpu: torch.Tensor, ref: np.ndarray, what: str = "", tight: b
     return worst
 
 
+def assert_close_on_device(gpu: torch.Tensor, ref: np.ndarray, what: str = "", tight: bool = True):
+    """The rules of assert_close_dt for whole benchmark-sized tensors: the fp64 reference is
+    copied to the GPU tensor's device and the element-by-element comparison runs there in fp64
+    (widening the output to fp64 is exact), so that every element of a 500 MB output can be
+    checked in seconds.  Only the comparison runs on the device; the reference is the CPU checker's."""
+    dev = gpu.device
+    r = torch.from_numpy(np.ascontiguousarray(ref)).to(dev)
+    g = gpu.detach().double().reshape(r.shape)
+    nan_ref, inf_ref = torch.isnan(r), torch.isinf(r)
+    assert torch.equal(torch.isnan(g), nan_ref), f"{what}: NaN pattern differs"
+    assert torch.equal(torch.isinf(g), inf_ref), f"{what}: inf pattern differs"
+    assert torch.equal(g[inf_ref], r[inf_ref]), f"{what}: inf sign differs"
+    fin = ~(nan_ref | inf_ref)
+    zero = torch.zeros((), dtype=torch.float64, device=dev)
+    err = torch.where(fin, (g - r).abs(), zero)
+    mag = torch.where(fin, r.abs(), zero)
+    if gpu.dtype == torch.bfloat16:
+        tol, rel, quantum = BF16_TOL, BF16_TIGHT, 1.2e-38
+    else:
+        tol = DT_TOL[gpu.dtype]
+        rel, quantum = DT_TIGHT[gpu.dtype]
+    worst = float((err / (tol * mag.clamp(min=1.0))).max()) if err.numel() else 0.0
+    assert worst <= 1.0, f"{what}: max err/bound = {worst:.3f}"
+    if tight and err.numel():
+        worst_t = float((err / (rel * mag + quantum)).max())
+        assert worst_t <= 1.0, f"{what}: exceeds one-rounding bound by {worst_t:.3f}x"
+    return worst
+
+
 def assert_loss_close(gpu: torch.Tensor, ref: np.ndarray, what: str = ""):
     got = gpu.detach().cpu().double().numpy().reshape(ref.shape)
     nan_ref = np.isnan(ref)

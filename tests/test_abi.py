@@ -151,6 +151,11 @@ def test_dispatch_is_a_pure_function_of_shape_and_alignment():
     assert path == ak.AK_XENT_SPLIT and 2 <= ns <= 64
     assert ak.ak_xent_workspace_bytes(16, 128256) == 16 * ns * 8
     assert ak.ak_xent_choose_path(1, 128256)[1] == 8             # slices of at most 16384 elements
+    # the split rules are stated in SMs of the current device (148 when none can be queried)
+    sms = ak.ak_sm_count()
+    assert sms >= 1
+    assert ak.ak_xent_choose_path(4 * sms - 1, 128256)[0] == ak.AK_XENT_SPLIT
+    assert ak.ak_xent_choose_path(4 * sms, 128256) == (ak.AK_XENT_ROW, 1)
     assert ak.ak_xent_choose_path(16, 1000) == (ak.AK_XENT_ROW, 1)  # short rows never split
     # repeated queries agree (no hidden state)
     assert all(ak.ak_xent_choose_path(16, 128256) == (path, ns) for _ in range(3))
@@ -178,3 +183,31 @@ def test_product_does_not_import_the_checker():
         if f.endswith((".py", ".c")):
             text = open(os.path.join(ROOT, "oracle", f)).read()
             assert "paper_2603_21331_b200" not in text and "libak" not in text
+
+
+def test_calls_act_on_the_tensors_device():
+    """The library launches on the current CUDA device, so the binding makes the tensors' device
+    current around a call and refuses a call whose tensors sit on different devices.  Checked
+    here with stand-ins for tensors (no GPU needed): only `.device.index` is looked at."""
+    import types
+    from unittest import mock
+
+    def on(index):
+        return types.SimpleNamespace(device=types.SimpleNamespace(index=index))
+
+    with pytest.raises(ValueError):
+        binding._on_device_of(on(0), on(1))
+    seen = []
+    with mock.patch.object(binding.torch.cuda, "current_device", return_value=0), \
+            mock.patch.object(binding.torch.cuda, "set_device", side_effect=seen.append):
+        with binding._on_device_of(on(0), None, on(0)):
+            pass
+        assert seen == []                      # already current: nothing is switched
+        with binding._on_device_of(on(1), on(1)):
+            assert seen == [1]
+        assert seen == [1, 0]                  # and put back afterwards
+
+
+def test_wait_timeout_flags_have_a_host_reader():
+    # without a device the flags cannot be read (-1); with one, no wait has ever given up (0)
+    assert ak.ak_wait_timeouts() in (-1, 0)

@@ -1,8 +1,10 @@
-"""Full-size benchmark shapes in the launch configuration the benchmark times: sampled rows
-are checked one by one against the fp64 CPU checker, the rest through properties that hold
-at any size (finite, row sums, mean = fp64 mean of the per-row losses), plus bitwise
-run-to-run determinism.  Inputs are generated on the device from a seed; the sampled rows'
-bit patterns are copied back so both sides see identical bits."""
+"""Full-size benchmark shapes in the launch configuration the benchmark times.  Tensors of up to
+1 GiB (every shape of the benchmark configurations but two) are compared with the fp64 CPU
+checker element by element over ALL rows, in row chunks; the two larger ones (262144 x 4096,
+16384 x 128256) over 1024 sampled rows plus first / middle / last.  Every shape is also checked
+through properties that hold at any size (finite, row sums, mean = fp64 mean of the per-row
+losses) and for bitwise run-to-run determinism.  Inputs are generated on the device from a
+seed; their bit patterns are copied back chunk by chunk so both sides see identical bits."""
 import math
 
 import numpy as np
@@ -12,10 +14,23 @@ import torch
 import oracle
 import paper_2603_21331_b200 as ak
 from paper_2603_21331_b200 import synth
-from parity import assert_bf16_close, assert_loss_close
+from parity import assert_bf16_close, assert_close_on_device, assert_loss_close
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
+ALL_ROWS_UP_TO = 1 << 29      # elements: tensors of up to 1 GiB (bf16) are compared whole
+CHUNK_ELEMS = 1 << 25         # elements per chunk handed to the checker (256 MB of fp64)
+
+
+def _row_chunks(rows, D, sample=1024, seed=0):
+    """Index tensors (on the device) of the rows to compare, chunk by chunk: every row when the
+    tensor has at most ALL_ROWS_UP_TO elements, else `sample` random rows plus first, middle, last."""
+    if rows * D <= ALL_ROWS_UP_TO:
+        idx = np.arange(rows, dtype=np.int64)
+    else:
+        idx = _sample_rows(rows, n=sample, seed=seed)
+    per = max(1, CHUNK_ELEMS // D)
+    return [torch.from_numpy(idx[i:i + per]).to(DEV) for i in range(0, len(idx), per)]
 
 
 def _sample_rows(rows, n=40, seed=0):
@@ -40,10 +55,9 @@ def test_rmsnorm_full_size(rows, D):
     torch.cuda.synchronize()
     assert torch.equal(y.view(torch.int16), y2.view(torch.int16))
     del y2
-    idx = _sample_rows(rows, seed=D)
-    it = torch.from_numpy(idx).to(DEV)
-    ref = oracle.rmsnorm(synth.to_bits(x[it]), synth.to_bits(w), 1e-6)
-    assert_bf16_close(y[it], ref, f"rmsnorm {rows}x{D} sampled rows")
+    for it in _row_chunks(rows, D, seed=D):
+        ref = oracle.rmsnorm(synth.to_bits(x[it]), synth.to_bits(w), 1e-6)
+        assert_close_on_device(y[it], ref, f"rmsnorm {rows}x{D} rows {int(it[0])}..{int(it[-1])}")
     # property: mean square of y / w is 1 (eps is negligible for N(0,1) rows)
     for r0 in range(0, rows, 32768):
         blk = y[r0:r0 + 32768].float() / w.float()[None, :]
@@ -65,13 +79,13 @@ def test_softmax_full_size(rows, D):
     torch.cuda.synchronize()
     assert torch.equal(y.view(torch.int16), y2.view(torch.int16))
     del y2
-    idx = _sample_rows(rows, seed=D)
-    # make sure masked rows are among the samples
-    masked = torch.nonzero(x[:, -1].float() == float("-inf")).flatten()[:8].cpu().numpy()
-    idx = np.unique(np.concatenate([idx, masked]))
-    it = torch.from_numpy(idx).to(DEV)
-    ref = oracle.softmax(synth.to_bits(x[it]))
-    assert_bf16_close(y[it], ref, f"softmax {rows}x{D} sampled rows")
+    chunks = _row_chunks(rows, D, seed=D)
+    if rows * D > ALL_ROWS_UP_TO:   # make sure masked rows are among the samples
+        chunks.append(torch.nonzero(x[:, -1].float() == float("-inf")).flatten()[:8])
+    for it in chunks:
+        if it.numel():
+            ref = oracle.softmax(synth.to_bits(x[it]))
+            assert_close_on_device(y[it], ref, f"softmax {rows}x{D} rows {int(it[0])}..{int(it[-1])}")
     for r0 in range(0, rows, 16384):
         blk = y[r0:r0 + 16384].float()
         assert torch.isfinite(blk).all() and bool((blk >= 0).all())
@@ -90,11 +104,17 @@ def test_xent_full_size(rows, V):
     torch.cuda.synchronize()
     assert torch.equal(loss.view(torch.int32), loss2.view(torch.int32))
     assert torch.equal(mean.view(torch.int32), mean2.view(torch.int32))
-    idx = _sample_rows(rows, seed=V)
-    it = torch.from_numpy(idx).to(DEV)
-    ref_rows, _, _ = oracle.xent(synth.to_bits(logits[it]), targets[it].cpu().numpy())
-    assert_loss_close(loss[it], ref_rows, f"xent {rows}x{V} sampled rows")
+    ref_all, idx_all = [], []
+    for it in _row_chunks(rows, V, seed=V):
+        ref_rows, _, _ = oracle.xent(synth.to_bits(logits[it]), targets[it].cpu().numpy())
+        assert_loss_close(loss[it], ref_rows, f"xent {rows}x{V} rows {int(it[0])}..{int(it[-1])}")
+        ref_all.append(ref_rows)
+        idx_all.append(it)
     valid = targets != -100
+    if rows * V <= ALL_ROWS_UP_TO:   # every row was checked: the checker's own mean is at hand
+        ref_rows = np.concatenate(ref_all)
+        ref_mean = ref_rows[valid.cpu().numpy()].sum() / int(valid.sum())
+        assert_loss_close(mean, np.array([ref_mean]), f"xent {rows}x{V} mean against the checker")
     assert bool((loss[~valid] == 0).all()) and bool((loss[valid] > 0).all())
     want_mean = loss[valid].double().sum().item() / int(valid.sum())
     assert abs(mean.item() - want_mean) <= 1e-6 * want_mean
@@ -113,10 +133,9 @@ def test_layernorm_full_size(rows, D):
     torch.cuda.synchronize()
     assert torch.equal(y.view(torch.int16), y2.view(torch.int16))
     del y2
-    idx = _sample_rows(rows, seed=D)
-    it = torch.from_numpy(idx).to(DEV)
-    ref = oracle.layernorm(synth.to_bits(x[it]), synth.to_bits(g), synth.to_bits(b), 1e-5)
-    assert_bf16_close(y[it], ref, f"layernorm {rows}x{D} sampled rows", tight=False)
+    for it in _row_chunks(rows, D, seed=D):
+        ref = oracle.layernorm(synth.to_bits(x[it]), synth.to_bits(g), synth.to_bits(b), 1e-5)
+        assert_close_on_device(y[it], ref, f"layernorm {rows}x{D} rows {int(it[0])}..{int(it[-1])}", tight=False)
     # property: (y - beta) / gamma has zero mean and unit variance in every row
     for r0 in range(0, rows, 16384):
         z = (y[r0:r0 + 16384].float() - b.float()[None, :]) / g.float()[None, :]
@@ -135,13 +154,12 @@ def test_rowsum_full_size(rows, D):
     s2 = ak.ak_rowsum_fwd(x)
     torch.cuda.synchronize()
     assert torch.equal(s.view(torch.int32), s2.view(torch.int32))
-    idx = _sample_rows(rows, seed=D)
-    it = torch.from_numpy(idx).to(DEV)
-    xb = synth.to_bits(x[it])
-    ref = oracle.rowsum(xb)
-    mag = np.abs(oracle.bf16_to_f64(xb)).sum(axis=1)
-    err = np.abs(s[it].cpu().double().numpy() - ref)
-    assert float(np.max(err / (1e-6 * mag + 2.0 ** -24 * np.abs(ref)))) <= 1.0
+    for it in _row_chunks(rows, D, seed=D):
+        xb = synth.to_bits(x[it])
+        ref = oracle.rowsum(xb)
+        mag = x[it].double().abs().sum(dim=-1).cpu().numpy()
+        err = np.abs(s[it].cpu().double().numpy() - ref)
+        assert float(np.max(err / (1e-6 * mag + 2.0 ** -24 * np.abs(ref)))) <= 1.0
     # property at any size: agrees with a float64 sum done by another library on the device
     for r0 in range(0, rows, 8192):
         want = x[r0:r0 + 8192].double().sum(dim=-1)

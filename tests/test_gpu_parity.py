@@ -545,3 +545,42 @@ def test_layernorm_unaligned_cluster_with_the_shift_table():
     y2 = ak.ak_layernorm_fwd(x[:200].contiguous(), g, b, eps=1e-5)
     torch.cuda.synchronize()
     assert torch.equal(y2.view(torch.int16), y[:200].view(torch.int16))
+
+
+def test_magnitudes_beyond_the_square_range_of_fp32_are_pinned():
+    """bf16 holds magnitudes up to 3.4e38, but the norms add squares in fp32: once a row's sum
+    of squares (RMSNorm) or of squared deviations (LayerNorm) passes 3.4e38 it becomes inf,
+    1/sqrt(inf) is 0 and the row comes out as 0 (RMSNorm) or as beta (LayerNorm), where the fp64
+    definition gives +-w and +-gamma + beta.  This is the documented behaviour (ak.h), stated
+    here so that it cannot change unnoticed: exact zeros / beta, never NaN or garbage; rows just
+    inside the range follow the definition; softmax and cross-entropy, which only subtract the
+    maximum, follow the definition at any magnitude."""
+    D = 1024
+    sign = torch.tensor([1.0, -1.0]).repeat(D // 2)
+    w = (1.0 + 0.25 * torch.arange(D) / D).to(torch.bfloat16)
+    beta = (0.5 - torch.arange(D) / D).to(torch.bfloat16)
+    for exp2, inside in ((70, False), (62, False), (50, True)):
+        # D * (2^e)^2 = 2^(2e + 10): beyond fp32's 2^128 for e = 62 and 70, inside for e = 50
+        x = (sign * 2.0 ** exp2).to(torch.bfloat16).repeat(3, 1)
+        xb = synth.to_bits(x)
+        ref_r = oracle.rmsnorm(xb, synth.to_bits(w), 1e-6)
+        ref_l = oracle.layernorm(xb, synth.to_bits(w), synth.to_bits(beta), 1e-5)
+        assert np.isfinite(ref_r).all() and np.isfinite(ref_l).all()       # the definition is finite
+        for path in (ak.AK_PATH_AUTO, GEN, SMEM, CLUSTER):
+            yr = ak.ak_rmsnorm_fwd(x.to(DEV), w.to(DEV), eps=1e-6, path=path)
+            yl = ak.ak_layernorm_fwd(x.to(DEV), w.to(DEV), beta.to(DEV), eps=1e-5, path=path)
+            torch.cuda.synchronize()
+            if inside:
+                assert_bf16_close(yr, ref_r, f"rmsnorm |x| = 2^{exp2} path {path}")
+                assert_bf16_close(yl, ref_l, f"layernorm |x| = 2^{exp2} path {path}", tight=False)
+            else:
+                assert bool((yr.float() == 0).all()), f"rmsnorm |x| = 2^{exp2}: not exact (signed) zeros"
+                assert torch.equal(yl.cpu().view(torch.int16), beta.repeat(3, 1).view(torch.int16)), \
+                    f"layernorm |x| = 2^{exp2}: not beta"
+        ys = ak.ak_softmax_fwd(x.to(DEV))
+        assert_bf16_close(ys, oracle.softmax(xb), f"softmax |x| = 2^{exp2}")
+        t = torch.tensor([0, 1, 2])
+        loss, mean = ak.ak_xent_fwd(x.to(DEV), t.to(DEV))
+        ref_rows, ref_mean, _ = oracle.xent(xb, t.numpy())
+        assert_loss_close(loss, ref_rows, f"xent |x| = 2^{exp2}")
+        assert_loss_close(mean, np.array([ref_mean]), f"xent mean |x| = 2^{exp2}")
