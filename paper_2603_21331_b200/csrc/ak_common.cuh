@@ -386,8 +386,11 @@ int xent_dispatch(const void* logits, const int64_t* targets, int64_t ignore_ind
                   void* workspace, size_t workspace_bytes, bool may_allocate,
                   cudaStream_t st, int path, int nsplit, int dtype = AK_DTYPE_BF16);
 // Fixed-order fp64 mean of loss_rows over rows whose target != ignore_index (one small launch).
+// dependent: launch it as a programmatic dependent of the kernel enqueued just before, which must
+// be one that lets its dependents in only after its own wait (the mean kernel reads the targets
+// before it waits).
 int xent_mean_launch(const float* loss_rows, const int64_t* targets, int64_t ignore_index, int64_t rows,
-                     float* loss_mean, cudaStream_t st);
+                     float* loss_mean, cudaStream_t st, bool dependent = false);
 int xent_sum_count_launch(const float* loss_rows, const int64_t* targets, int64_t ignore_index, int64_t rows,
                           double* sum_count, cudaStream_t st);
 // Vocabulary-parallel cross-entropy (defined in xent_vp.cu).

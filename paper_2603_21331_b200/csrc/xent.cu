@@ -157,9 +157,9 @@ int xent_dispatch(const void* logits, const int64_t* targets, int64_t ignore_ind
 }
 
 int xent_mean_launch(const float* loss_rows, const int64_t* targets, int64_t ignore_index, int64_t rows,
-                     float* loss_mean, cudaStream_t st) {
+                     float* loss_mean, cudaStream_t st, bool dependent) {
     return launch_finish<AK_DTYPE_BF16>(nullptr, targets, ignore_index, nullptr, 0, const_cast<float*>(loss_rows), rows,
-                                        0, loss_mean, nullptr, st, false);
+                                        0, loss_mean, nullptr, st, dependent);
 }
 
 int xent_sum_count_launch(const float* loss_rows, const int64_t* targets, int64_t ignore_index, int64_t rows,

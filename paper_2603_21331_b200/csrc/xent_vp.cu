@@ -25,9 +25,12 @@ template <int UNROLL, int POLY, int MINB, int T, int DT>
 __global__ void __launch_bounds__(T, MINB)
 xent_vp_partial_kernel(const typename XElem<DT>::type* __restrict__ logits, const int64_t* __restrict__ targets,
                        int64_t ignore_index, int64_t vocab_start, int64_t V_total, float2* __restrict__ part,
-                       int64_t V_local, int nsplit) {
+                       int64_t V_local, int nsplit, int first_wave) {
     __shared__ float slots[2 * kWarp];
-    const int64_t row = blockIdx.x;
+    // launched as a programmatic dependent; with one slice per row the first wave prefetches the
+    // head of its rows while the grids before drain (first_wave is 0 for split rows)
+    pdl_prologue(logits + (int64_t)blockIdx.x * V_local, V_local * (int64_t)sizeof(typename XElem<DT>::type), first_wave);
+    const int64_t row = cta_id_x();
     const int sp = blockIdx.y;
     const int64_t t = targets[row];
     if (t != ignore_index && t >= 0 && t < V_total) {   // (this form, not an early return, keeps the compiler from spilling)
@@ -61,6 +64,8 @@ constexpr int kVpBatch = 16;   // pairs (and ranks) per row held in registers by
 __global__ void __launch_bounds__(kVpMergeThreads)
 xent_vp_merge_kernel(const float2* __restrict__ parts, int nranks, int nsplit, const int64_t* __restrict__ targets,
                      int64_t ignore_index, int64_t V_total, float* __restrict__ loss_rows, int64_t rows) {
+    pdl_wait();                 // launched as a programmatic dependent of whatever precedes it
+    pdl_launch_dependents();    // the mean kernel may take a slot now (it reads the targets, which are final)
     const int64_t r = (int64_t)blockIdx.x * kVpMergeThreads + threadIdx.x;
     if (r >= rows) return;
     const int64_t t = targets[r];
@@ -120,16 +125,19 @@ int partial_t(const void* logits, const int64_t* targets, int64_t ignore_index, 
     using elem_t = typename XElem<DT>::type;
     const elem_t* lg = static_cast<const elem_t*>(logits);
     const dim3 grid((unsigned)rows, (unsigned)nsplit);
-    // the single-GPU row layout: 128 threads x 8 vectors, 64 registers (fp32: 72, seven CTAs per SM)
-    constexpr int kMinCtas = (DT == AK_DTYPE_F32) ? 7 : 8;
-    if (nsplit == 1)
-        xent_vp_partial_kernel<8, 2, kMinCtas, 128, DT><<<grid, 128, 0, st>>>(lg, targets, ignore_index, vocab_start,
-                                                                             V_total, part, V_local, nsplit);
-    else
-        xent_vp_partial_kernel<4, 2, 1, kXentThreads, DT><<<grid, kXentThreads, 0, st>>>(
-            lg, targets, ignore_index, vocab_start, V_total, part, V_local, nsplit);
+    // the single-GPU row layout: 128 threads x 8 vectors, 64 registers (fp32: no cap, 112 registers; every cap tried made the compiler spill)
+    constexpr int kMinCtas = (DT == AK_DTYPE_F32) ? 1 : 8;
+    cudaError_t e;
+    if (nsplit == 1) {
+        auto kernel = xent_vp_partial_kernel<8, 2, kMinCtas, 128, DT>;
+        e = launch_dependent(kernel, grid, dim3(128), 0, st, lg, targets, ignore_index, vocab_start, V_total, part,
+                             V_local, nsplit, resident_ctas(kernel, 128, 0));
+    } else {
+        e = launch_dependent(xent_vp_partial_kernel<4, 2, 1, kXentThreads, DT>, grid, dim3(kXentThreads), 0, st, lg,
+                             targets, ignore_index, vocab_start, V_total, part, V_local, nsplit, 0);
+    }
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+    return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
 }  // namespace
@@ -154,13 +162,14 @@ int xent_vp_merge_launch(const void* parts, int nranks, int nsplit, const int64_
                          int64_t V_total, float* loss_rows, float* loss_mean, int64_t rows, cudaStream_t st) {
     if (rows > 0) {
         const unsigned grid = (unsigned)((rows + kVpMergeThreads - 1) / kVpMergeThreads);
-        xent_vp_merge_kernel<<<grid, kVpMergeThreads, 0, st>>>(static_cast<const float2*>(parts), nranks, nsplit, targets,
-                                                              ignore_index, V_total, loss_rows, rows);
+        const cudaError_t e = launch_dependent(xent_vp_merge_kernel, dim3(grid), dim3(kVpMergeThreads), 0, st,
+                                               static_cast<const float2*>(parts), nranks, nsplit, targets, ignore_index,
+                                               V_total, loss_rows, rows);
         count_launch();
-        if (cudaGetLastError() != cudaSuccess) return AK_ERR_CUDA;
+        if (e != cudaSuccess) return AK_ERR_CUDA;
     }
     if (loss_mean == nullptr) return AK_OK;
-    return xent_mean_launch(loss_rows, targets, ignore_index, rows, loss_mean, st);
+    return xent_mean_launch(loss_rows, targets, ignore_index, rows, loss_mean, st, rows > 0);
 }
 
 }  // namespace ak
