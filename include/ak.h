@@ -33,7 +33,8 @@
  *   - Kernels are launched as programmatic dependents (programmatic stream serialisation): their
  *     CTAs may become resident while the previous kernel of the stream drains, but every read and
  *     write comes after griddepcontrol.wait, i.e. after that kernel has completed and flushed;
- *     before the wait they only prefetch their first inputs into L2.  Stream order is therefore
+ *     before the wait they only prefetch their first inputs into L2 (AK_DISABLE_PREFETCH=1 in
+ *     the environment, read once, switches that prefetch off).  Stream order is therefore
  *     observed exactly as for ordinary launches, with any kernel before or after.
  *   - Stream-ordered scratch, where an entry point says it uses some, comes from a CUDA
  *     memory pool of the library's own (one per device, created at first use, keeps up to

@@ -120,6 +120,17 @@ bool dyn_smem_configured(const void* kernel) {
     return true;
 }
 
+// AK_DISABLE_PREFETCH=1 in the environment (read once) switches off the L2 prefetch the first
+// wave of a kernel issues before its griddepcontrol.wait (for comparing, or where the kernel
+// before in the stream should keep all of the memory system to itself until it ends).
+bool first_wave_prefetch_enabled() {
+    static const bool off = [] {
+        const char* v = getenv("AK_DISABLE_PREFETCH");
+        return v != nullptr && v[0] != '\0' && v[0] != '0';
+    }();
+    return !off;
+}
+
 int resident_ctas_of(const void* kernel, int threads, size_t dyn_smem) {
     static std::mutex mu;
     static std::map<std::tuple<const void*, int, size_t>, int> memo[kMaxDev];

@@ -374,6 +374,12 @@ template <typename... A>
 inline int resident_ctas(void (*kernel)(A...), int threads, size_t dyn_smem) {
     return resident_ctas_of(reinterpret_cast<const void*>(kernel), threads, dyn_smem);
 }
+// CTAs of the first wave that prefetch before the wait (see pdl_prologue); 0 switches it off
+bool first_wave_prefetch_enabled();
+template <typename... A>
+inline int first_wave_ctas(void (*kernel)(A...), int threads, size_t dyn_smem) {
+    return first_wave_prefetch_enabled() ? resident_ctas(kernel, threads, dyn_smem) : 0;
+}
 
 // Per-op host dispatchers (each defined next to its kernels).  All arguments have been
 // validated; `path` is a concrete path id or AUTO.  They return an ak_status.

@@ -26,7 +26,7 @@ int launch_reg(const void* x, const void* g, const void* b, void* y, int64_t row
     const cudaError_t e = launch_dependent(kernel, dim3((unsigned)grid), dim3(THREADS), 0, st,
                                            static_cast<const uint4*>(x), static_cast<const uint4*>(g),
                                            static_cast<const uint4*>(b), static_cast<uint4*>(y), rows, nvec, inv_D, eps,
-                                           resident_ctas(kernel, THREADS, 0));
+                                           first_wave_ctas(kernel, THREADS, 0));
     count_launch();
     return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }

@@ -39,7 +39,7 @@ int launch_reg(const void* x, const void* w, void* y, int64_t rows, int nvec, fl
     const cudaError_t e = launch_dependent(kernel, dim3((unsigned)grid), dim3(THREADS), 0, st,
                                            static_cast<const uint4*>(x), static_cast<const uint4*>(w),
                                            static_cast<uint4*>(y), rows, nvec, inv_D, eps,
-                                           resident_ctas(kernel, THREADS, 0));
+                                           first_wave_ctas(kernel, THREADS, 0));
     count_launch();
     return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
@@ -89,9 +89,11 @@ int launch_cluster_rows(const void* x, const void* w, void* y, int64_t rows, int
 template <int DT, int THREADS, int VPT>
 int launch_regp(const uint16_t* x, const uint16_t* w, uint16_t* y, int64_t rows, int64_t D, float inv_D, float eps,
                 cudaStream_t st) {
-    rmsnorm_regp_kernel<THREADS, VPT, DT><<<(unsigned)rows, THREADS, 0, st>>>(x, w, y, D, inv_D, eps);
+    auto kernel = rmsnorm_regp_kernel<THREADS, VPT, DT>;
+    const cudaError_t e = launch_dependent(kernel, dim3((unsigned)rows), dim3(THREADS), 0, st, x, w, y, D, inv_D, eps,
+                                           first_wave_ctas(kernel, THREADS, 0));
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+    return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 template <int DT, int THREADS>
 int launch_regp_vpt(int vpt, const uint16_t* x, const uint16_t* w, uint16_t* y, int64_t rows, int64_t D, float inv_D,
@@ -220,14 +222,18 @@ int dispatch_t(const void* x, const void* w, void* y, int64_t rows, int64_t D, f
                     return launch_regp_vpt<DT, 512>((int)((max_nv + 511) / 512), xs, ws, ys, rows, D, inv_D, eps, st);
                 if (same_phase && is_aligned(w, 4) && stage_bytes <= (size_t)kMaxRowSmemBytes) {
                     if (!allow_big_smem(rmsnorm_stage_kernel<128, DT>) || !allow_big_smem(rmsnorm_stage_kernel<256, DT>) || !allow_big_smem(rmsnorm_stage_kernel<512, DT>)) return AK_ERR_CUDA;
+                    cudaError_t e;
                     if (D <= 8192)
-                        rmsnorm_stage_kernel<128, DT><<<(unsigned)rows, 128, stage_bytes, st>>>(xs, ws, ys, D, inv_D, eps);
+                        e = launch_dependent(rmsnorm_stage_kernel<128, DT>, dim3((unsigned)rows), dim3(128), stage_bytes, st, xs, ws,
+                                             ys, D, inv_D, eps, first_wave_ctas(rmsnorm_stage_kernel<128, DT>, 128, stage_bytes));
                     else if (D <= 32768)
-                        rmsnorm_stage_kernel<256, DT><<<(unsigned)rows, 256, stage_bytes, st>>>(xs, ws, ys, D, inv_D, eps);
+                        e = launch_dependent(rmsnorm_stage_kernel<256, DT>, dim3((unsigned)rows), dim3(256), stage_bytes, st, xs, ws,
+                                             ys, D, inv_D, eps, first_wave_ctas(rmsnorm_stage_kernel<256, DT>, 256, stage_bytes));
                     else
-                        rmsnorm_stage_kernel<512, DT><<<(unsigned)rows, 512, stage_bytes, st>>>(xs, ws, ys, D, inv_D, eps);
+                        e = launch_dependent(rmsnorm_stage_kernel<512, DT>, dim3((unsigned)rows), dim3(512), stage_bytes, st, xs, ws,
+                                             ys, D, inv_D, eps, first_wave_ctas(rmsnorm_stage_kernel<512, DT>, 512, stage_bytes));
                     count_launch();
-                    return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+                    return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
                 }
                 const int resident = resident_ctas(rmsnorm_generic_kernel<DT>, kRmsGenericThreads, 0);
                 const int grid = (int)(rows < resident ? rows : resident);

@@ -284,13 +284,14 @@ __device__ __forceinline__ uint4 load_w_shifted(const uint16_t* __restrict__ w, 
 template <int T, int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(T)
 rmsnorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, uint16_t* __restrict__ y,
-                     int64_t D, float inv_D, float eps) {
+                     int64_t D, float inv_D, float eps, int first_wave) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     uint4* row = reinterpret_cast<uint4*>(smem_raw);
     uint16_t* row16 = reinterpret_cast<uint16_t*>(smem_raw);
     __shared__ uint64_t bar;
     __shared__ float slots[2 * kWarp];
     const int64_t r = blockIdx.x;
+    pdl_prologue(x + r * D, D * 2, first_wave);
     const uint16_t* xr = x + r * D;
     uint16_t* yr = y + r * D;
     const int phase = (int)((reinterpret_cast<uintptr_t>(xr) >> 1) & 7);
@@ -407,9 +408,10 @@ rmsnorm_cluster_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __r
 template <int THREADS, int VPT, int DT>
 __global__ void __launch_bounds__(THREADS)
 rmsnorm_regp_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ w, uint16_t* __restrict__ y,
-                    int64_t D, float inv_D, float eps) {
+                    int64_t D, float inv_D, float eps, int first_wave) {
     __shared__ float slots[2 * kWarp];
     const int64_t r = blockIdx.x;
+    pdl_prologue(x + r * D, D * 2, first_wave);
     const uint16_t* xr = x + r * D;
     uint16_t* yr = y + r * D;
     // interior vectors k_lo .. k_hi - 1 live in registers (slot i of thread t holds vector

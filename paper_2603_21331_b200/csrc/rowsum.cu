@@ -76,11 +76,17 @@ __device__ __forceinline__ void span_sum(const typename RsElem<DT>::type* p, int
 
 template <int THREADS, int GROUP, int UNROLL, int MINB, int DT>
 __global__ void __launch_bounds__(THREADS, MINB)
-rowsum_kernel(const typename RsElem<DT>::type* __restrict__ x, float* __restrict__ out, int64_t rows, int64_t D) {
+rowsum_kernel(const typename RsElem<DT>::type* __restrict__ x, float* __restrict__ out, int64_t rows, int64_t D,
+              int first_wave) {
     constexpr int GROUPS = THREADS / GROUP;
     constexpr int WARPS_PER_GROUP = GROUP / kWarp;
     static_assert(GROUP % kWarp == 0 && THREADS % GROUP == 0, "groups are whole warps");
     __shared__ float slots[THREADS / kWarp];
+    {
+        const int64_t r0 = (int64_t)blockIdx.x * GROUPS;
+        const int64_t nr = rows - r0 < GROUPS ? rows - r0 : GROUPS;
+        pdl_prologue(x + r0 * D, nr * D * (int64_t)sizeof(typename RsElem<DT>::type), first_wave);
+    }
     const int g = threadIdx.x / GROUP;
     const int t = threadIdx.x % GROUP;
     const int lane = threadIdx.x & 31;
@@ -129,6 +135,7 @@ __global__ void __launch_bounds__(kRsSplitThreads)
 rowsum_finish_kernel(const float* __restrict__ partial, float* __restrict__ out, int nsplit) {
     __shared__ float slots[2 * kWarp];
     asm volatile("griddepcontrol.wait;" ::: "memory");   // the partials of the whole grid before are visible
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int64_t row = blockIdx.x;
     float s = 0.0f;
     for (int i = threadIdx.x; i < nsplit; i += kRsSplitThreads) s += __ldcg(partial + row * nsplit + i);
@@ -185,10 +192,12 @@ int launch(const void* x, float* out, int64_t rows, int64_t D, cudaStream_t st) 
     constexpr int GROUPS = THREADS / GROUP;
     const int64_t grid = (rows + GROUPS - 1) / GROUPS;
     if (grid > 2147483647LL) return AK_ERR_SHAPE;
-    rowsum_kernel<THREADS, GROUP, UNROLL, MINB, DT><<<(unsigned)grid, THREADS, 0, st>>>(
-        static_cast<const typename RsElem<DT>::type*>(x), out, rows, D);
+    auto kernel = rowsum_kernel<THREADS, GROUP, UNROLL, MINB, DT>;
+    const cudaError_t e = launch_dependent(kernel, dim3((unsigned)grid), dim3(THREADS), 0, st,
+                                           static_cast<const typename RsElem<DT>::type*>(x), out, rows, D,
+                                           first_wave_ctas(kernel, THREADS, 0));
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+    return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
 template <int DT>

@@ -18,7 +18,7 @@ int launch_reg(const void* x, void* y, int64_t rows, int nvec, cudaStream_t st) 
     auto kernel = softmax_reg_kernel<THREADS, GROUP, VPT, MINB, false, DT>;
     const cudaError_t e = launch_dependent(kernel, dim3((unsigned)grid), dim3(THREADS), 0, st,
                                            static_cast<const uint4*>(x), static_cast<uint4*>(y), rows, nvec,
-                                           resident_ctas(kernel, THREADS, 0));
+                                           first_wave_ctas(kernel, THREADS, 0));
     count_launch();
     return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
@@ -45,7 +45,7 @@ int launch_smem(const void* x, void* y, int64_t rows, int nvec, cudaStream_t st)
     auto kernel = softmax_smem_kernel<THREADS, 1, KEEP, DT>;
     const cudaError_t e = launch_dependent(kernel, dim3((unsigned)rows), dim3(THREADS), smem, st,
                                            static_cast<const uint4*>(x), static_cast<uint4*>(y), nvec,
-                                           resident_ctas(kernel, THREADS, smem));
+                                           first_wave_ctas(kernel, THREADS, smem));
     count_launch();
     return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
@@ -53,9 +53,11 @@ int launch_smem(const void* x, void* y, int64_t rows, int nvec, cudaStream_t st)
 template <int DT, int T>
 int launch_stage(const uint16_t* x, uint16_t* y, int64_t rows, int64_t D, size_t stage_bytes, cudaStream_t st) {
     if (!allow_big_smem(softmax_stage_kernel<T, DT>)) return AK_ERR_CUDA;
-    softmax_stage_kernel<T, DT><<<(unsigned)rows, T, stage_bytes, st>>>(x, y, D);
+    auto kernel = softmax_stage_kernel<T, DT>;
+    const cudaError_t e = launch_dependent(kernel, dim3((unsigned)rows), dim3(T), stage_bytes, st, x, y, D,
+                                           first_wave_ctas(kernel, T, stage_bytes));
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+    return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 
 // unaligned rows split over a cluster of C CTAs (covering vectors of the worst phase: max_nv)
@@ -70,9 +72,11 @@ int launch_cluster_stage(const uint16_t* x, uint16_t* y, int64_t rows, int64_t D
 
 template <int DT, int THREADS, int VPT, int MINB>
 int launch_regp(const uint16_t* x, uint16_t* y, int64_t rows, int64_t D, cudaStream_t st) {
-    softmax_regp_kernel<THREADS, VPT, MINB, DT><<<(unsigned)rows, THREADS, 0, st>>>(x, y, D);
+    auto kernel = softmax_regp_kernel<THREADS, VPT, MINB, DT>;
+    const cudaError_t e = launch_dependent(kernel, dim3((unsigned)rows), dim3(THREADS), 0, st, x, y, D,
+                                           first_wave_ctas(kernel, THREADS, 0));
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
+    return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
 // a cluster of C CTAs per row (C from cluster_ctas, at least 2)
 template <int DT, int THREADS, int KEEP>

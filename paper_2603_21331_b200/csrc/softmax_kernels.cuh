@@ -345,13 +345,14 @@ softmax_cluster_stream_kernel(const uint4* __restrict__ x, uint4* __restrict__ y
 // standing in for the neighbours' bytes.  Three passes over shared memory.
 template <int T, int DT = AK_DTYPE_BF16>
 __global__ void __launch_bounds__(T)
-softmax_stage_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, int64_t D) {
+softmax_stage_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, int64_t D, int first_wave) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     uint4* row = reinterpret_cast<uint4*>(smem_raw);
     uint16_t* row16 = reinterpret_cast<uint16_t*>(smem_raw);
     __shared__ uint64_t bar;
     __shared__ float slots[2 * kWarp];
     const int64_t r = blockIdx.x;
+    pdl_prologue(x + r * D, D * 2, first_wave);
     const uint16_t* xr = x + r * D;
     uint16_t* yr = y + r * D;
     const int phase = (int)((reinterpret_cast<uintptr_t>(xr) >> 1) & 7);
@@ -473,9 +474,10 @@ softmax_cluster_stage_kernel(const uint16_t* __restrict__ x, uint16_t* __restric
 // rows in the same phase and at most THREADS * VPT covering vectors.
 template <int THREADS, int VPT, int MINB, int DT>
 __global__ void __launch_bounds__(THREADS, MINB)
-softmax_regp_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, int64_t D) {
+softmax_regp_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, int64_t D, int first_wave) {
     __shared__ float slots[2 * kWarp];
     const int64_t r = blockIdx.x;
+    pdl_prologue(x + r * D, D * 2, first_wave);
     const uint16_t* xr = x + r * D;
     uint16_t* yr = y + r * D;
     // interior vectors k_lo .. k_hi - 1 live in registers (slot i of thread t holds vector

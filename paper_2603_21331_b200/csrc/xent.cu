@@ -105,7 +105,7 @@ int dispatch_t(const void* logits, const int64_t* targets, int64_t ignore_index,
         constexpr int kMinCtas = (DT == AK_DTYPE_F32) ? kRowMinCtas - 1 : kRowMinCtas;
         const cudaError_t e = launch_dependent(xent_row_kernel<kRowUnroll, kPoly, kMinCtas, kRowThreads, DT>,
                                                dim3((unsigned)rows), dim3(kRowThreads), 0, st, lg, targets, ignore_index,
-                                               loss_rows, V, kMinCtas * sm_count());
+                                               loss_rows, V, first_wave_prefetch_enabled() ? kMinCtas * sm_count() : 0);
         count_launch();
         if (e != cudaSuccess) return AK_ERR_CUDA;
         if (loss_mean == nullptr) return AK_OK;

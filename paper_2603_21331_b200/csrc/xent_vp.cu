@@ -131,7 +131,7 @@ int partial_t(const void* logits, const int64_t* targets, int64_t ignore_index, 
     if (nsplit == 1) {
         auto kernel = xent_vp_partial_kernel<8, 2, kMinCtas, 128, DT>;
         e = launch_dependent(kernel, grid, dim3(128), 0, st, lg, targets, ignore_index, vocab_start, V_total, part,
-                             V_local, nsplit, resident_ctas(kernel, 128, 0));
+                             V_local, nsplit, first_wave_ctas(kernel, 128, 0));
     } else {
         e = launch_dependent(xent_vp_partial_kernel<4, 2, 1, kXentThreads, DT>, grid, dim3(kXentThreads), 0, st, lg,
                              targets, ignore_index, vocab_start, V_total, part, V_local, nsplit, 0);
