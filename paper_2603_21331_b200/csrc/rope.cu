@@ -71,7 +71,7 @@ __device__ __forceinline__ uint4 rotate_vec(const uint4& v, const f32x2* cc, con
 template <int DT, int UNROLL>
 __global__ void __launch_bounds__(kRopeThreads)
 rope_vec_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t n_seq, int64_t nvs, int vpr,
-                int64_t pos_offset, int seq_per_cta, int first_wave, const __grid_constant__ RopeFreq freq) {
+                int64_t pos_offset, int seq_per_cta, const __grid_constant__ RopeFreq freq) {
     constexpr int PPV = Elem<DT>::kPerVec / 2;   // pairs per vector
     const int64_t v = (int64_t)blockIdx.x * kRopeThreads + threadIdx.x;
     int64_t n = (int64_t)blockIdx.y * seq_per_cta;
@@ -80,13 +80,8 @@ rope_vec_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t n_se
     const uint4* xp = x + n * nvs + v;
     uint4* yp = y + n * nvs + v;
     // Launched as a programmatic dependent; nothing is read or written before the wait.  (The
-    // prefetch of the first wave that the row kernels do before their wait is switched off here,
-    // first_wave = 0: for these strided 2 KiB segments it measured 0.8-1.4 us slower per launch.)
-    if ((int64_t)blockIdx.y * gridDim.x + blockIdx.x < first_wave && (threadIdx.x & 7) == 0 && v < nvs) {
-#pragma unroll
-        for (int u = 0; u < UNROLL; ++u)
-            if (n + u < n_end) prefetch_l2(xp + u * nvs);
-    }
+    // prefetch of the first wave that the row kernels do before their wait is left out here: for
+    // these strided 2 KiB segments it measured 0.8-1.4 us slower per launch.)
     pdl_wait();
     pdl_launch_dependents();
     if (v >= nvs) return;
@@ -190,7 +185,7 @@ int rope_t(const void* x, void* y, int64_t n_seq, int64_t S, int64_t Dh, int64_t
         auto kernel = rope_vec_kernel<DT, 8>;
         const cudaError_t e = launch_dependent(kernel, dim3((unsigned)gx, gy), dim3(kRopeThreads), 0, st,
                                                static_cast<const uint4*>(x), static_cast<uint4*>(y), n_seq, nvs, vpr,
-                                               pos_offset, seq_per_cta, 0, freq);
+                                               pos_offset, seq_per_cta, freq);
         count_launch();
         return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
     } else {

@@ -29,7 +29,7 @@ template <int DT>
 int launch_finish(const typename XElem<DT>::type* logits, const int64_t* targets, int64_t ignore_index, const float2* partial,
                   int nsplit, float* loss_rows, int64_t rows, int64_t V, float* out_mean, double* out_pair,
                   cudaStream_t st, bool dependent) {
-    const bool many = rows > kFinishSmallRows;
+    const bool many = rows >= kFinishSmallRows;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(1);
     cfg.blockDim = dim3(many ? kFinishThreadsMany : kFinishThreads);
@@ -103,9 +103,19 @@ int dispatch_t(const void* logits, const int64_t* targets, int64_t ignore_index,
     if (path == AK_XENT_ROW) {
         // fp32 logits: seven CTAs per SM (72 registers); at eight the compiler spills
         constexpr int kMinCtas = (DT == AK_DTYPE_F32) ? kRowMinCtas - 1 : kRowMinCtas;
-        const cudaError_t e = launch_dependent(xent_row_kernel<kRowUnroll, kPoly, kMinCtas, kRowThreads, DT>,
-                                               dim3((unsigned)rows), dim3(kRowThreads), 0, st, lg, targets, ignore_index,
-                                               loss_rows, V, first_wave_prefetch_enabled() ? kMinCtas * sm_count() : 0);
+        // The last batch of a row is masked; when at most five of its eight slots per thread can
+        // hold data (a 50304-column bf16 row: two) the kernel form that stops at the filled slots
+        // is taken (1-2 us per launch there); otherwise the plain form, whose straight-line code is
+        // 1-3 % faster when the last batch is full or nearly so.  Same bits either way.
+        const int64_t nvec_row = V * (int64_t)sizeof(elem_t) / 16;
+        const int64_t rest = nvec_row % ((int64_t)kRowThreads * kRowUnroll);
+        const bool trim = nvec_row >= (int64_t)kRowThreads * kRowUnroll && rest > 0 && (rest + kRowThreads - 1) / kRowThreads <= 5;
+        const int first_wave = first_wave_prefetch_enabled() ? kMinCtas * sm_count() : 0;
+        const cudaError_t e =
+            trim ? launch_dependent(xent_row_kernel<kRowUnroll, kPoly, kMinCtas, kRowThreads, DT, true>, dim3((unsigned)rows),
+                                    dim3(kRowThreads), 0, st, lg, targets, ignore_index, loss_rows, V, first_wave)
+                 : launch_dependent(xent_row_kernel<kRowUnroll, kPoly, kMinCtas, kRowThreads, DT, false>, dim3((unsigned)rows),
+                                    dim3(kRowThreads), 0, st, lg, targets, ignore_index, loss_rows, V, first_wave);
         count_launch();
         if (e != cudaSuccess) return AK_ERR_CUDA;
         if (loss_mean == nullptr) return AK_OK;

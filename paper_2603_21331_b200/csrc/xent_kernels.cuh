@@ -152,6 +152,94 @@ __device__ __forceinline__ void absorb_scalar(Online& o, float v) {
     o.s2 = add2(o.s2, pack2(fast_exp2(fmaf(v, kLog2e, -o.mf)), 0.0f));
 }
 
+// ---- plain form: the masked last batch is a whole batch (used unless the row's last batch is
+// mostly padding; see the trimmed form below, which gives the same bits).
+// A slice = elements [begin, end) of one row, cut into up to kPerVec - 1 head elements (single
+// loads until the address is 16-byte aligned), nbody aligned 16-byte vectors, and up to
+// kPerVec - 1 tail elements.  One batch = UNROLL vectors per thread, all loaded before the
+// first use.  Full batches run without any per-vector bounds test (constant offsets from one
+// moving pointer); a single masked batch finishes the slice.
+template <int DT>
+struct SliceF {
+    const typename XElem<DT>::type* p;
+    int64_t n, head, nbody, tail0, nfull;
+    const uint4* body;
+    int rest;  // vectors in the masked last batch, < T * UNROLL
+};
+template <int UNROLL, int T, int DT>
+__device__ __forceinline__ SliceF<DT> make_slice_full(const typename XElem<DT>::type* __restrict__ xr, int64_t begin, int64_t end) {
+    constexpr int PV = Elem<DT>::kPerVec;
+    constexpr int LOG_PV = (PV == 8) ? 3 : 2, LOG_BYTES = (Elem<DT>::kBytes == 2) ? 1 : 2;
+    SliceF<DT> s;
+    s.p = xr + begin;
+    s.n = end - begin;
+    s.head = (PV - (int)((reinterpret_cast<uintptr_t>(s.p) >> LOG_BYTES) & (PV - 1))) & (PV - 1);
+    if (s.head > s.n) s.head = s.n;
+    s.nbody = (s.n - s.head) >> LOG_PV;
+    s.tail0 = s.head + (s.nbody << LOG_PV);
+    s.body = reinterpret_cast<const uint4*>(s.p + s.head);
+    s.nfull = s.nbody / ((int64_t)T * UNROLL);
+    s.rest = (int)(s.nbody - s.nfull * T * UNROLL);
+    return s;
+}
+// The slice's first batch (full if there is a full batch, otherwise the masked one).
+template <int UNROLL, int T, int DT>
+__device__ __forceinline__ void load_first_batch_full(const SliceF<DT>& s, uint4 (&q)[UNROLL]) {
+    const uint4* src = s.body + threadIdx.x;
+    if (s.nfull > 0) {
+#pragma unroll
+        for (int k = 0; k < UNROLL; ++k) q[k] = ld_stream(src + k * T);
+    } else {
+#pragma unroll
+        for (int k = 0; k < UNROLL; ++k) {
+            const int i = (int)threadIdx.x + k * T;
+            q[k] = (i < s.rest) ? ld_stream(src + k * T) : xneg_inf_vec<DT>();
+        }
+    }
+}
+
+// One thread's online (m, s) over its share of a slice whose first batch `q` is already in flight:
+// every batch, the masked last one included, absorbs all UNROLL slots (padding adds exact zeros).
+template <int UNROLL, int POLY, int T, int DT>
+__device__ __forceinline__ Online slice_stream_full(const SliceF<DT>& sl, uint4 (&q)[UNROLL]) {
+    Online o{-INFINITY, kFloor2, pack2(0.0f, 0.0f)};
+    const f32x2 l2 = pack2(kLog2e, kLog2e);
+    auto absorb_batch = [&](const uint4 (&v)[UNROLL]) {
+        uint32_t mx = xmax_v<DT>(v[0]);
+#pragma unroll
+        for (int k = 1; k < UNROLL; ++k) mx = xmax_w<DT>(mx, xmax_v<DT>(v[k]));
+        raise_max(o, xhmax_of<DT>(mx));
+        const f32x2 nmf2 = pack2(-o.mf, -o.mf);
+        f32x2 acc = sumexp_v<POLY, DT>(v[0], l2, nmf2);
+#pragma unroll
+        for (int k = 1; k < UNROLL; ++k) acc = add2(acc, sumexp_v<POLY, DT>(v[k], l2, nmf2));
+        o.s2 = add2(o.s2, acc);
+    };
+    // (taken before the loop as two small ints and a pointer: with the 64-bit fields kept alive
+    // across the loop the compiler needs a spill slot)
+    const int ihead = (int)sl.head, ntail = (int)(sl.n - sl.tail0);
+    const typename XElem<DT>::type* ptail = sl.p + sl.tail0;
+    absorb_batch(q);  // batch 0 (all padding when the slice has no body)
+    const uint4* src = sl.body + threadIdx.x + T * UNROLL;
+    for (int64_t b = 1; b < sl.nfull; ++b, src += T * UNROLL) {
+#pragma unroll
+        for (int k = 0; k < UNROLL; ++k) q[k] = ld_stream(src + k * T);
+        absorb_batch(q);
+    }
+    if (sl.nfull > 0 && sl.rest > 0) {
+#pragma unroll
+        for (int k = 0; k < UNROLL; ++k) {
+            const int i = (int)threadIdx.x + k * T;
+            q[k] = (i < sl.rest) ? ld_stream(src + k * T) : xneg_inf_vec<DT>();
+        }
+        absorb_batch(q);
+    }
+    if ((int)threadIdx.x < ihead) absorb_scalar(o, xload<DT>(sl.p + threadIdx.x));
+    if ((int)threadIdx.x < ntail) absorb_scalar(o, xload<DT>(ptail + threadIdx.x));
+    return o;
+}
+
+// ---- trimmed form
 // A slice = elements [begin, end) of one row, cut into up to kPerVec - 1 head elements (single
 // loads until the address is 16-byte aligned), nbody aligned 16-byte vectors, and up to
 // kPerVec - 1 tail elements.  One batch = UNROLL vectors per thread, all loaded before the
@@ -305,10 +393,26 @@ __device__ __forceinline__ void slice_combine(const Online& o, float* slots, flo
     }
 }
 
-// CTA-wide online (m, s) over a slice whose first batch `q` is already in flight.
-template <int UNROLL, int POLY, int T, int DT>
-__device__ __forceinline__ void slice_lse(const Slice<DT>& sl, uint4 (&q)[UNROLL], float* slots, float& M, float& S) {
-    const Online o = slice_stream<UNROLL, POLY, T, DT>(sl, q);
+// CTA-wide online (m, s) over elements [begin, end) of the row at xr: the first batch is requested,
+// `early` runs (loads that should sit under the row's own traffic, not after the reduction), the
+// slice is streamed and the threads' pairs are combined.  TRIM picks the form of the masked last
+// batch (same bits either way).
+template <int UNROLL, int POLY, int T, int DT, bool TRIM, typename Early>
+__device__ __forceinline__ void row_lse(const typename XElem<DT>::type* xr, int64_t begin, int64_t end, float* slots,
+                                        float& M, float& S, Early early) {
+    uint4 q[UNROLL];
+    Online o;
+    if constexpr (TRIM) {
+        const Slice<DT> sl = make_slice<UNROLL, T, DT>(xr, begin, end);
+        load_first_batch<UNROLL, T, DT>(sl, q);
+        early();
+        o = slice_stream<UNROLL, POLY, T, DT>(sl, q);
+    } else {
+        const SliceF<DT> sl = make_slice_full<UNROLL, T, DT>(xr, begin, end);
+        load_first_batch_full<UNROLL, T, DT>(sl, q);
+        early();
+        o = slice_stream_full<UNROLL, POLY, T, DT>(sl, q);
+    }
     slice_combine<T>(o, slots, M, S);
 }
 
@@ -327,7 +431,7 @@ __device__ __forceinline__ float finish_loss(float M, float S, float xt) {
 // Launched as a programmatic dependent of whatever precedes it in the stream: nothing is read
 // or written before griddepcontrol.wait, and its own dependents (the finish kernel) are let in
 // only after the wait, so that they may read this kernel's inputs before their own wait.
-template <int UNROLL, int POLY, int MINB = 1, int T = kXentThreads, int DT = AK_DTYPE_BF16>
+template <int UNROLL, int POLY, int MINB = 1, int T = kXentThreads, int DT = AK_DTYPE_BF16, bool TRIM = false>
 __global__ void __launch_bounds__(T, MINB)
 xent_row_kernel(const typename XElem<DT>::type* __restrict__ logits, const int64_t* __restrict__ targets,
                 int64_t ignore_index, float* __restrict__ loss_rows, int64_t V, int first_wave) {
@@ -356,13 +460,9 @@ xent_row_kernel(const typename XElem<DT>::type* __restrict__ logits, const int64
     if (t != ignore_index && t >= 0 && t < V) {  // uniform across the CTA
         // (Requesting the first batch before the target is known was measured: no gain, and
         // ignored rows would be touched.)
-        const Slice<DT> sl = make_slice<UNROLL, T, DT>(xr, 0, V);
-        uint4 q[UNROLL];
-        load_first_batch<UNROLL, T, DT>(sl, q);
-        // the target logit is fetched now, under the row's own traffic, not after the reduction
-        const float xt = (threadIdx.x == 0) ? xread<DT>(xr + t) : 0.0f;
-        float M, S;
-        slice_lse<UNROLL, POLY, T, DT>(sl, q, slots, M, S);
+        float xt = 0.0f, M, S;
+        // the target logit is fetched under the row's own traffic, not after the reduction
+        row_lse<UNROLL, POLY, T, DT, TRIM>(xr, 0, V, slots, M, S, [&] { if (threadIdx.x == 0) xt = xread<DT>(xr + t); });
         if (threadIdx.x == 0) loss_rows[row] = finish_loss(M, S, xt);
     } else if (threadIdx.x == 0) {   // nothing of the row is read
         loss_rows[row] = (t == ignore_index) ? 0.0f : __int_as_float(0x7fc00000);
@@ -387,11 +487,8 @@ xent_split_kernel(const typename XElem<DT>::type* __restrict__ logits, const int
     int64_t begin = ((groups * sp) / nsplit) << 3;
     int64_t end = ((groups * (sp + 1)) / nsplit) << 3;
     if (end > V) end = V;
-    const Slice<DT> sl = make_slice<UNROLL, kXentThreads, DT>(logits + row * V, begin, end);
-    uint4 q[UNROLL];
-    load_first_batch<UNROLL, kXentThreads, DT>(sl, q);
     float M, S;
-    slice_lse<UNROLL, POLY, kXentThreads, DT>(sl, q, slots, M, S);
+    row_lse<UNROLL, POLY, kXentThreads, DT, false>(logits + row * V, begin, end, slots, M, S, [] {});
     if (threadIdx.x == 0) partial[row * nsplit + sp] = make_float2(M, S);
 }
 
@@ -407,9 +504,9 @@ xent_split_kernel(const typename XElem<DT>::type* __restrict__ logits, const int
 // last CTAs are still running; a 1024-thread CTA with its registers needs a whole empty SM.
 // out_mean = sum / count (0/0 = NaN); out_pair = {sum, count}.
 constexpr int kFinishVirtual = 1024;
-constexpr int kFinishThreads = 256;        // up to kFinishSmallRows rows
+constexpr int kFinishThreads = 256;        // fewer than kFinishSmallRows rows
 constexpr int kFinishThreadsMany = 1024;
-constexpr int64_t kFinishSmallRows = 8192;
+constexpr int64_t kFinishSmallRows = 1024;
 
 __device__ __forceinline__ double warp_sum_f64(double v) {
 #pragma unroll
@@ -437,16 +534,22 @@ xent_finish_kernel(const typename XElem<DT>::type* __restrict__ logits, const in
     int n_counted = 0;
     if (want_sum) {
         for (int64_t base = 0; base < rows; base += (int64_t)kFinishVirtual * KB) {
+            int64_t tt[KB][J];   // all of a batch's targets are requested before the first is looked at
 #pragma unroll
             for (int k = 0; k < KB; ++k)
 #pragma unroll
                 for (int j = 0; j < J; ++j) {
                     const int64_t r = base + (int64_t)k * kFinishVirtual + j * T + threadIdx.x;
-                    if (r < rows && targets[r] != ignore_index) {
+                    tt[k][j] = (r < rows) ? targets[r] : ignore_index;
+                }
+#pragma unroll
+            for (int k = 0; k < KB; ++k)
+#pragma unroll
+                for (int j = 0; j < J; ++j)
+                    if (tt[k][j] != ignore_index) {
                         ++n_counted;
                         if (base == 0) counted0 |= 1u << (k * J + j);
                     }
-                }
         }
         n_counted = __reduce_add_sync(0xffffffffu, n_counted);
         if (lane == 0) scnt[warp] = n_counted;

@@ -78,7 +78,7 @@ extern "C" int ak_xent_fwd_static(const void* logits, const int64_t* targets, in
         return AK_OK;
     }
     // merge the slices in split order, write the losses, then the fixed-order mean
-    if (rows > kFinishSmallRows)
+    if (rows >= kFinishSmallRows)
         xent_finish_kernel<AK_DTYPE_BF16, kFinishThreadsMany><<<1, kFinishThreadsMany, 0, st>>>(
             lg, targets, ignore_index, scratch, nsplit, loss_rows, rows, V, loss_mean, nullptr);
     else

@@ -21,7 +21,7 @@ namespace {
 // part[row * (nsplit + 1) + nsplit] = (x_t, 1) if the shard owns column t, else (0, 0).
 // Rows whose target is ignore_index or outside [0, V_total) are not read and their entries
 // are not written (the merge never looks at them).
-template <int UNROLL, int POLY, int MINB, int T, int DT>
+template <int UNROLL, int POLY, int MINB, int T, int DT, bool ONE_SLICE>
 __global__ void __launch_bounds__(T, MINB)
 xent_vp_partial_kernel(const typename XElem<DT>::type* __restrict__ logits, const int64_t* __restrict__ targets,
                        int64_t ignore_index, int64_t vocab_start, int64_t V_total, float2* __restrict__ part,
@@ -35,24 +35,27 @@ xent_vp_partial_kernel(const typename XElem<DT>::type* __restrict__ logits, cons
     const int64_t t = targets[row];
     if (t != ignore_index && t >= 0 && t < V_total) {   // (this form, not an early return, keeps the compiler from spilling)
         const typename XElem<DT>::type* xr = logits + row * V_local;
-        const int64_t groups = (V_local + 7) >> 3;
-        int64_t begin = ((groups * sp) / nsplit) << 3;
-        int64_t end = ((groups * (sp + 1)) / nsplit) << 3;
-        if (end > V_local) end = V_local;
-        const Slice<DT> sl = make_slice<UNROLL, T, DT>(xr, begin, end);
-        uint4 q[UNROLL];
-        load_first_batch<UNROLL, T, DT>(sl, q);
-        float2 mine = make_float2(0.0f, 0.0f);
-        if (sp == 0 && threadIdx.x == 0) {
-            const int64_t tl = t - vocab_start;
-            if (tl >= 0 && tl < V_local) mine = make_float2(xread<DT>(xr + tl), 1.0f);
+        int64_t begin = 0, end = V_local;
+        if constexpr (!ONE_SLICE) {
+            const int64_t groups = (V_local + 7) >> 3;
+            begin = ((groups * sp) / nsplit) << 3;
+            end = ((groups * (sp + 1)) / nsplit) << 3;
+            if (end > V_local) end = V_local;
         }
-        float M, S;
-        slice_lse<UNROLL, POLY, T, DT>(sl, q, slots, M, S);
+        // slice 0 of the shard that owns the target's column fetches the target logit
+        const int64_t tl = t - vocab_start;
+        float M, S, xt = 0.0f;
+        row_lse<UNROLL, POLY, T, DT, ONE_SLICE>(xr, begin, end, slots, M, S, [&] {   // (one slice: the pointer-loop form, which fits 64 registers here without a spill slot)
+            if (sp == 0 && tl >= 0 && tl < V_local && threadIdx.x == 0) xt = xread<DT>(xr + tl);
+        });
         if (threadIdx.x == 0) {
-            float2* pr = part + row * (nsplit + 1);
+            // (row, slice and ownership are worked out again here rather than kept in registers
+            // across the loop: at 64 registers the compiler would spill them)
+            const int64_t row2 = cta_id_x();
+            const int64_t tl2 = targets[row2] - vocab_start;
+            float2* pr = part + row2 * (nsplit + 1);
             pr[sp] = make_float2(M, S);
-            if (sp == 0) pr[nsplit] = mine;
+            if (sp == 0) pr[nsplit] = (tl2 >= 0 && tl2 < V_local) ? make_float2(xt, 1.0f) : make_float2(0.0f, 0.0f);
         }
     }
 }
@@ -125,15 +128,15 @@ int partial_t(const void* logits, const int64_t* targets, int64_t ignore_index, 
     using elem_t = typename XElem<DT>::type;
     const elem_t* lg = static_cast<const elem_t*>(logits);
     const dim3 grid((unsigned)rows, (unsigned)nsplit);
-    // the single-GPU row layout: 128 threads x 8 vectors, 64 registers (fp32: no cap, 112 registers; every cap tried made the compiler spill)
+    // the single-GPU row layout: 128 threads x 8 vectors, 64 registers (fp32: no cap)
     constexpr int kMinCtas = (DT == AK_DTYPE_F32) ? 1 : 8;
     cudaError_t e;
     if (nsplit == 1) {
-        auto kernel = xent_vp_partial_kernel<8, 2, kMinCtas, 128, DT>;
+        auto kernel = xent_vp_partial_kernel<8, 2, kMinCtas, 128, DT, true>;
         e = launch_dependent(kernel, grid, dim3(128), 0, st, lg, targets, ignore_index, vocab_start, V_total, part,
                              V_local, nsplit, first_wave_ctas(kernel, 128, 0));
     } else {
-        e = launch_dependent(xent_vp_partial_kernel<4, 2, 1, kXentThreads, DT>, grid, dim3(kXentThreads), 0, st, lg,
+        e = launch_dependent(xent_vp_partial_kernel<4, 2, 1, kXentThreads, DT, false>, grid, dim3(kXentThreads), 0, st, lg,
                              targets, ignore_index, vocab_start, V_total, part, V_local, nsplit, 0);
     }
     count_launch();
