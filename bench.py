@@ -322,10 +322,15 @@ def run_ours(args, rank, world, local_rank):
         raise RuntimeError("bench.py needs a CUDA device; the ops have no CPU fallback")
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
+    # AK_BENCH_DIST=1 takes the multi-GPU code path (eager steps + the NCCL mean exchange, a process
+    # group, barriers, max over ranks) with ONE rank, so that path can be exercised on one GPU
+    multi = world > 1 or bool(os.environ.get("AK_BENCH_DIST"))
     dist = None
-    if world > 1:
+    if multi:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device(dev))
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29533")
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=torch.device(dev))
 
     seed0 = 100 * rank
     (rr, rd), (sr, sd), (xr, xv) = WORKLOAD["rmsnorm"], WORKLOAD["softmax"], WORKLOAD["xent"]
@@ -353,10 +358,10 @@ def run_ours(args, rank, world, local_rank):
 
     for _ in range(max(args.warmup, 3)):
         step()
-        if world > 1:
+        if multi:
             global_mean()
     torch.cuda.synchronize()
-    if world > 1:
+    if multi:
         dist.barrier()
         torch.cuda.synchronize()
 
@@ -367,10 +372,10 @@ def run_ours(args, rank, world, local_rank):
     # event between them, until at least MIN_TIMED_S of device time: `value` and `ms_per_step` come
     # from the median block; the first block (after a second of idling) is the burst regime, the
     # blocks that start after SUSTAINED_AFTER_S of load are the sustained one (power cap reached).
-    use_graph = world == 1 and not os.environ.get("AK_BENCH_EAGER")
+    use_graph = not multi and not os.environ.get("AK_BENCH_EAGER")
     launches0 = ak.ak_launch_count()
     step()
-    if world > 1:
+    if multi:
         global_mean()
     torch.cuda.synchronize()
     kernels_per_step = ak.ak_launch_count() - launches0
@@ -400,7 +405,7 @@ def run_ours(args, rank, world, local_rank):
         return a_ev.elapsed_time(b_ev)
 
     def sync_ranks():
-        if world > 1:
+        if multi:
             dist.barrier()
         torch.cuda.synchronize()
 
@@ -412,12 +417,12 @@ def run_ours(args, rank, world, local_rank):
 
         def eager_step():
             step()
-            if world > 1:
+            if multi:
                 global_mean()
         run_step_block = block_runner(eager_step)
     est = probe_ms(run_step_block)
     ms, starts, clk, t0, t1 = timed_blocks(run_step_block, est, local_rank, sync=sync_ranks)
-    if world > 1:
+    if multi:
         t = torch.tensor(ms, dtype=torch.float64, device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms = t.cpu().numpy()
@@ -522,7 +527,7 @@ def run_ours(args, rank, world, local_rank):
     }
 
     # ---- end to end: host buffers in pinned memory, copies inside the timed region
-    if rank == 0 or world > 1:
+    if rank == 0 or multi:
         xh, wh, yh = x.cpu().pin_memory(), w.cpu(), torch.empty(x.shape, dtype=x.dtype).pin_memory()
         xsh, ysh = xs.cpu().pin_memory(), torch.empty(xs.shape, dtype=xs.dtype).pin_memory()
         lgh, tgh = lg.cpu().pin_memory(), tg.cpu()
@@ -537,14 +542,14 @@ def run_ours(args, rank, world, local_rank):
         e2e_steps = max(2, min(K, 5))
         e2e_step()
         torch.cuda.synchronize()
-        if world > 1:
+        if multi:
             dist.barrier()
         t0 = time.perf_counter()
         for _ in range(e2e_steps):
             e2e_step()
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        if world > 1:
+        if multi:
             t = torch.tensor([dt], dtype=torch.float64, device=dev)
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             dt = float(t.item())
@@ -568,7 +573,7 @@ def run_ours(args, rank, world, local_rank):
     if args.sweep and rank == 0:
         run_sweep(ak, synth, dev, peak, out_path=args.out)
 
-    if world > 1:
+    if multi:
         dist.barrier()
         dist.destroy_process_group()
     if rank == 0:
