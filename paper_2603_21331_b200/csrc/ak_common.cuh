@@ -328,6 +328,24 @@ __device__ __forceinline__ bool mailbox_exchange(float v, float* box, uint64_t* 
     }
     return mbar_wait(xbar, 0);
 }
+// the same for a pair of values per CTA (`box`: C float2, 8-byte aligned; armed for C x 8 bytes)
+__device__ __forceinline__ void mailbox_arm2(uint64_t* xbar, int C) {
+    mbar_init(xbar, 1);
+    mbar_expect_tx(xbar, (uint32_t)C * 8u);
+}
+__device__ __forceinline__ bool mailbox_exchange2(float a, float b, float2* box, uint64_t* xbar, int C, uint32_t rank) {
+    if ((int)threadIdx.x < C) {
+        uint32_t rbox, rbar;
+        uint64_t v;
+        asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(a), "f"(b));
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbox) : "r"(smem_addr(box + rank)), "r"(threadIdx.x));
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(smem_addr(xbar)), "r"(threadIdx.x));
+        asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.b64 [%0], %1, [%2];" ::"r"(rbox), "l"(v),
+                     "r"(rbar)
+                     : "memory");
+    }
+    return mbar_wait(xbar, 0);
+}
 // One thread starts the bulk copies of a contiguous, 16-byte aligned span into shared memory
 // (nothing to copy: a plain arrival, so the wait still completes).  The mbarrier must be
 // initialised and that made visible (a CTA barrier) before.

@@ -38,6 +38,76 @@ __device__ __forceinline__ f32x2 dev2(uint32_t u, float c) {
     ln_halves(u, lo, hi);
     return pack2(sub_h<DT>(lo, c), sub_h<DT>(hi, c));
 }
+// s += (x - c), q += (x - c)^2 over the elements of a vector, lane-wise in packed pairs
+template <int DT>
+__device__ __forceinline__ void moments_v(const uint4& v, float c, f32x2& s, f32x2& q) {
+    if constexpr (DT == AK_DTYPE_F32) {
+        const f32x2 c2 = pack2(c, c);
+        const f32x2 a = sub2(pack2(__uint_as_float(v.x), __uint_as_float(v.y)), c2);
+        const f32x2 b = sub2(pack2(__uint_as_float(v.z), __uint_as_float(v.w)), c2);
+        s = add2(s, add2(a, b));
+        q = fma2(b, b, fma2(a, a, q));
+    } else {
+        // word by word: two live temporaries instead of eight
+        f32x2 d = dev2<DT>(v.x, c);
+        s = add2(s, d);
+        q = fma2(d, d, q);
+        d = dev2<DT>(v.y, c);
+        s = add2(s, d);
+        q = fma2(d, d, q);
+        d = dev2<DT>(v.z, c);
+        s = add2(s, d);
+        q = fma2(d, d, q);
+        d = dev2<DT>(v.w, c);
+        s = add2(s, d);
+        q = fma2(d, d, q);
+    }
+}
+// The shift of the one-sweep moments: the mean of the row's first 16 bytes.  Exactly c for a
+// constant row (every term is c scaled by a power of two and the partial sums are multiples of
+// it); scaled before summing so that eight large values cannot overflow.
+template <int DT>
+__device__ __forceinline__ float head_mean(const uint4 v) {
+    if constexpr (DT == AK_DTYPE_F32) {
+        return (__uint_as_float(v.x) * 0.25f + __uint_as_float(v.y) * 0.25f) +
+               (__uint_as_float(v.z) * 0.25f + __uint_as_float(v.w) * 0.25f);
+    } else {
+        const float a = Elem<DT>::lo(v.x) * 0.125f + Elem<DT>::hi(v.x) * 0.125f;
+        const float b = Elem<DT>::lo(v.y) * 0.125f + Elem<DT>::hi(v.y) * 0.125f;
+        const float c = Elem<DT>::lo(v.z) * 0.125f + Elem<DT>::hi(v.z) * 0.125f;
+        const float d = Elem<DT>::lo(v.w) * 0.125f + Elem<DT>::hi(v.w) * 0.125f;
+        return (a + b) + (c + d);
+    }
+}
+// Mean and variance from the one-sweep sums s = sum(x - K), q = sum((x - K)^2).  False when the
+// shift is so far from the mean (or something is not a number) that the subtraction
+// q/D - (s/D)^2 would lose accuracy: the caller then makes the centred pass sum((x - mu)^2).
+__device__ __forceinline__ bool sweep_stats(float s, float q, float inv_D, float K, float& mu, float& var) {
+    const float m = s * inv_D;   // mean - K
+    mu = K + m;
+    var = fmaf(q, inv_D, -(m * m));
+    return m * m <= var;
+}
+// the lane sums of packed accumulators, added over the CTA with one barrier (slot sets 0 and 1)
+template <int THREADS>
+__device__ __forceinline__ void cta_sum2(f32x2 sp, f32x2 qp, float* slots, float& s, float& q) {
+    constexpr int NW = THREADS / kWarp;
+    float lo, hi;
+    unpack2(sp, lo, hi);
+    s = warp_sum(lo + hi);
+    unpack2(qp, lo, hi);
+    q = warp_sum(lo + hi);
+    if constexpr (NW > 1) {
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        if (lane == 0) {
+            slots[warp] = s;
+            slots[kWarp + warp] = q;
+        }
+        __syncthreads();
+        s = warp_sum((lane < NW) ? slots[lane] : 0.0f);
+        q = warp_sum((lane < NW) ? slots[kWarp + lane] : 0.0f);
+    }
+}
 // sum over the elements of (x - c)
 template <int DT>
 __device__ __forceinline__ float sumdev_v(const uint4& v, float c) {
@@ -107,18 +177,38 @@ __device__ __forceinline__ float first_elem(const void* row) {
 
 // ------------------------------------------------------------------ row in registers
 // Same thread layout as the RMSNorm register kernel (a group of GROUP threads owns a row,
-// thread t holds vectors t, t + GROUP, ...), two reductions per row.  Padding slots hold
-// copies of K so they add exactly zero to the first sum and are excluded from the second.
+// thread t holds vectors t, t + GROUP, ...).
+//
+// Groups of one or two warps (short rows) make two centred reductions: the mean from
+// sum(x - K) with K the row's first element, then sum((x - mean)^2).
+//
+// Groups of 128 threads and more (a CTA per row) make ONE sweep over the registers and one
+// barrier: s = sum(x - K) and q = sum((x - K)^2) with K the mean of the row's first 16 bytes,
+// mean = K + s/D, variance = q/D - (s/D)^2.  The subtraction loses accuracy only when the shift
+// is far from the mean, so the result is kept when (s/D)^2 <= variance (the relative error of
+// the variance is then at most three times that of q) and the centred second pass runs
+// otherwise (a whole row at a time, so the branch does not diverge).  A constant row gives
+// s = q = 0 exactly, hence the output beta bit for bit.
+//
 // P_EARLY: gamma and beta are requested together with the row instead of after the reductions
 // (8 * VPT more live registers; for launches too small to fill the GPU, where latency counts).
-template <int THREADS, int GROUP, int VPT, int MINB, int DT = AK_DTYPE_BF16, bool P_EARLY = false>
+// FULL: every thread holds exactly VPT vectors of a live row (nvec == VPT * GROUP and one row
+// per CTA), so the loads and the sweep test no bounds; with AHEAD neither does the output phase,
+// which lets the compiler fetch gamma and beta several vectors ahead (at the cost of registers).
+template <int THREADS, int GROUP, int VPT, int MINB, int DT = AK_DTYPE_BF16, bool P_EARLY = false, bool FULL = false,
+          bool AHEAD = false>
 __global__ void __launch_bounds__(THREADS, MINB)
 layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamma, const uint4* __restrict__ beta,
                      uint4* __restrict__ y, int64_t rows, int nvec, float inv_D, float eps, int first_wave) {
     constexpr int GROUPS = THREADS / GROUP;
     constexpr int WARPS_PER_GROUP = GROUP / kWarp;
+    constexpr bool SWEEP1 = GROUP >= 128;
     static_assert(GROUP % kWarp == 0 && THREADS % GROUP == 0, "groups are whole warps");
-    __shared__ float slots[2][THREADS / kWarp];
+    static_assert(!FULL || GROUPS == 1, "FULL is for one row per CTA");
+    // SWEEP1 alternates between two sets of slots by row, so that one barrier per row is enough:
+    // a warp can be at most one barrier ahead of the slowest reader
+    __shared__ float slots2[2][3][THREADS / kWarp];
+    int par = 0;
     {
         const int64_t r0 = (int64_t)blockIdx.x * GROUPS;
         const int64_t nr = rows - r0 < GROUPS ? rows - r0 : GROUPS;
@@ -134,56 +224,90 @@ layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamm
 #pragma unroll
         for (int k = 0; k < VPT; ++k) {
             const int i = t + k * GROUP;
-            if (i < nvec) {
+            if (FULL || i < nvec) {
                 gv[k] = __ldg(gamma + i);
                 bv[k] = __ldg(beta + i);
             }
         }
     }
-    for (int64_t row0 = (int64_t)blockIdx.x * GROUPS; row0 < rows; row0 += (int64_t)gridDim.x * GROUPS) {
+    // FULL: the grid has one CTA per row, so the loop body runs once
+    for (int64_t row0 = (int64_t)blockIdx.x * GROUPS; FULL || row0 < rows; row0 += (int64_t)gridDim.x * GROUPS) {
         const int64_t row = row0 + g;
-        const bool live = row < rows;
+        const bool live = FULL || row < rows;
         const uint4* xr = x + row * nvec;
-        const float K = live ? first_elem<DT>(xr) : 0.0f;
+        float (*slots)[THREADS / kWarp] = slots2[par];
+        // sum over the group of a per-thread partial (slot set `which`, one barrier)
+        auto group_sum = [&](float v, int which) {
+            v = warp_sum(v);
+            if constexpr (WARPS_PER_GROUP > 1) {
+                float* s = slots[which] + g * WARPS_PER_GROUP;
+                if (lane == 0) s[warp_in_group] = v;
+                __syncthreads();
+                v = warp_sum((lane < WARPS_PER_GROUP) ? s[lane] : 0.0f);
+            }
+            return v;
+        };
+        const float K = !live ? 0.0f : (SWEEP1 ? head_mean<DT>(__ldg(xr)) : first_elem<DT>(xr));
         uint4 xv[VPT];
 #pragma unroll
         for (int k = 0; k < VPT; ++k) {
             const int i = t + k * GROUP;
-            if (live && i < nvec) xv[k] = ld_stream(xr + i);
+            if (FULL || (live && i < nvec)) xv[k] = ld_stream(xr + i);
         }
-        float s1 = 0.0f;
+        float mu, var;
+        if constexpr (SWEEP1) {
+            f32x2 sp = pack2(0.0f, 0.0f), qp = sp;
 #pragma unroll
-        for (int k = 0; k < VPT; ++k)
-            if (live && t + k * GROUP < nvec) s1 += sumdev_v<DT>(xv[k], K);
-        s1 = warp_sum(s1);
-        if constexpr (WARPS_PER_GROUP > 1) {
-            float* s = slots[0] + g * WARPS_PER_GROUP;
-            if (lane == 0) s[warp_in_group] = s1;
-            __syncthreads();
-            s1 = warp_sum((lane < WARPS_PER_GROUP) ? s[lane] : 0.0f);
-        }
-        const float mu = fmaf(s1, inv_D, K);
-        float s2 = 0.0f;
+            for (int k = 0; k < VPT; ++k)
+                if (FULL || (live && t + k * GROUP < nvec)) moments_v<DT>(xv[k], K, sp, qp);
+            float s1, q1, lo, hi;
+            unpack2(sp, lo, hi);
+            s1 = warp_sum(lo + hi);
+            unpack2(qp, lo, hi);
+            q1 = warp_sum(lo + hi);
+            {
+                float* s = slots[0] + g * WARPS_PER_GROUP;
+                float* q = slots[1] + g * WARPS_PER_GROUP;
+                if (lane == 0) {
+                    s[warp_in_group] = s1;
+                    q[warp_in_group] = q1;
+                }
+                __syncthreads();
+                s1 = warp_sum((lane < WARPS_PER_GROUP) ? s[lane] : 0.0f);
+                q1 = warp_sum((lane < WARPS_PER_GROUP) ? q[lane] : 0.0f);
+            }
+            if (!sweep_stats(s1, q1, inv_D, K, mu, var)) {
+                float s2 = 0.0f;
 #pragma unroll
-        for (int k = 0; k < VPT; ++k)
-            if (live && t + k * GROUP < nvec) s2 += sqdev_v<DT>(xv[k], mu);
-        s2 = warp_sum(s2);
-        if constexpr (WARPS_PER_GROUP > 1) {
-            float* s = slots[1] + g * WARPS_PER_GROUP;
-            if (lane == 0) s[warp_in_group] = s2;
-            __syncthreads();
-            s2 = warp_sum((lane < WARPS_PER_GROUP) ? s[lane] : 0.0f);
+                for (int k = 0; k < VPT; ++k)
+                    if (FULL || (live && t + k * GROUP < nvec)) s2 += sqdev_v<DT>(xv[k], mu);
+                var = group_sum(s2, 2) * inv_D;
+            }
+            par ^= 1;
+        } else {
+            float s1 = 0.0f;
+#pragma unroll
+            for (int k = 0; k < VPT; ++k)
+                if (live && t + k * GROUP < nvec) s1 += sumdev_v<DT>(xv[k], K);
+            mu = fmaf(group_sum(s1, 0), inv_D, K);
+            float s2 = 0.0f;
+#pragma unroll
+            for (int k = 0; k < VPT; ++k)
+                if (live && t + k * GROUP < nvec) s2 += sqdev_v<DT>(xv[k], mu);
+            var = group_sum(s2, 1) * inv_D;
         }
-        const float rstd = rsqrtf(fmaf(s2, inv_D, eps));
-        uint4* yr = y + row * nvec;
+        const float rstd = rsqrtf(var + eps);
+        // FULL: the row index is read again rather than kept in registers across the reductions
+        uint4* yr = y + (FULL ? (int64_t)cta_id_x() : row) * nvec;
 #pragma unroll
         for (int k = 0; k < VPT; ++k) {
             const int i = t + k * GROUP;
-            if (live && i < nvec) {
+            if ((FULL && (P_EARLY || AHEAD)) || (live && i < nvec)) {
                 if constexpr (P_EARLY) st_stream(yr + i, ln_out_v<DT>(xv[k], gv[k], bv[k], mu, rstd));
                 else st_stream(yr + i, ln_out_v<DT>(xv[k], __ldg(gamma + i), __ldg(beta + i), mu, rstd));
             }
         }
+        if constexpr (FULL) break;
     }
 }
 
@@ -200,7 +324,7 @@ layernorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gam
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint4* row = reinterpret_cast<const uint4*>(smem_raw);
     __shared__ uint64_t bar;
-    __shared__ float slots[2 * kWarp];
+    __shared__ float slots[3 * kWarp];
     const int64_t r = blockIdx.x;
     if (threadIdx.x == 0) mbar_init(&bar, 1);
     __syncthreads();
@@ -212,19 +336,19 @@ layernorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gam
             bulk_load(smem_raw + off, src + off, min(kLnBulkChunk, bytes - off), &bar);
     }
     if (!mbar_wait(&bar, 0)) return;  // gave up (flag set, see ak_wait_timeouts): a thread that exits no longer counts at later barriers
-    float K;
-    if constexpr (DT == AK_DTYPE_F32) K = reinterpret_cast<const float*>(smem_raw)[0];
-    else K = Elem<DT>::to_float(reinterpret_cast<const uint16_t*>(smem_raw)[0]);
-    float s1 = 0.0f;
+    const float K = head_mean<DT>(row[0]);
+    f32x2 sp = pack2(0.0f, 0.0f), qp = sp;
 #pragma unroll 4
-    for (int i = threadIdx.x; i < nvec; i += THREADS) s1 += sumdev_v<DT>(row[i], K);
-    s1 = cta_sum<THREADS>(s1, slots, 0);
-    const float mu = fmaf(s1, inv_D, K);
-    float s2 = 0.0f;
+    for (int i = threadIdx.x; i < nvec; i += THREADS) moments_v<DT>(row[i], K, sp, qp);
+    float s1, q1, mu, var;
+    cta_sum2<THREADS>(sp, qp, slots, s1, q1);
+    if (!sweep_stats(s1, q1, inv_D, K, mu, var)) {
+        float s2 = 0.0f;
 #pragma unroll 4
-    for (int i = threadIdx.x; i < nvec; i += THREADS) s2 += sqdev_v<DT>(row[i], mu);
-    s2 = cta_sum<THREADS>(s2, slots, 1);
-    const float rstd = rsqrtf(fmaf(s2, inv_D, eps));
+        for (int i = threadIdx.x; i < nvec; i += THREADS) s2 += sqdev_v<DT>(row[i], mu);
+        var = cta_sum<THREADS>(s2, slots, 2) * inv_D;
+    }
+    const float rstd = rsqrtf(var + eps);
     uint4* yr = y + r * nvec;
 #pragma unroll 2
     for (int i = threadIdx.x; i < nvec; i += THREADS)
@@ -239,14 +363,15 @@ layernorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gam
 // distributed shared memory and are added in rank order in every CTA.  grid = rows * C,
 // cluster = C.  Dynamic shared memory = ceil(nvec / C) * 16 bytes.
 template <int THREADS, int DT = AK_DTYPE_BF16>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, 2)
 layernorm_cluster_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamma, const uint4* __restrict__ beta,
                          uint4* __restrict__ y, int nvec, int C, float inv_D, float eps) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint4* row = reinterpret_cast<const uint4*>(smem_raw);
     __shared__ uint64_t bar;
-    __shared__ float slots[2 * kWarp];
-    __shared__ float box1[kMaxCluster], box2[kMaxCluster];
+    __shared__ float slots[3 * kWarp];
+    __shared__ __align__(8) float2 box1[kMaxCluster];
+    __shared__ float box2[kMaxCluster];
     __shared__ uint64_t xbar1, xbar2;
     const uint32_t c = cluster_rank();
     const int64_t r = blockIdx.x / C;
@@ -254,35 +379,40 @@ layernorm_cluster_kernel(const uint4* __restrict__ x, const uint4* __restrict__ 
     const int n = (int)((int64_t)nvec * (c + 1) / C) - v0;
     if (threadIdx.x == 0) {
         mbar_init(&bar, 1);
-        mailbox_arm(&xbar1, C);
+        mailbox_arm2(&xbar1, C);
         mailbox_arm(&xbar2, C);
     }
     __syncthreads();
     if (threadIdx.x == 0) bulk_load_span(smem_raw, x + r * nvec + v0, (uint32_t)n * 16u, &bar);
-    const uint32_t first = __ldg(reinterpret_cast<const uint32_t*>(x + r * nvec));
-    float K;
-    if constexpr (DT == AK_DTYPE_F32) K = __uint_as_float(first);
-    else K = Elem<DT>::to_float((uint16_t)(first & 0xffffu));
+    const float K = head_mean<DT>(__ldg(x + r * nvec));
     cluster_arrive_relaxed();
     // a wait that gave up (never expected) contributes nothing and writes nothing, but still posts
     int nn = mbar_wait(&bar, 0) ? n : 0;
-    float s1 = 0.0f;
+    f32x2 sp = pack2(0.0f, 0.0f), qp = sp;
 #pragma unroll 4
-    for (int i = threadIdx.x; i < nn; i += THREADS) s1 += sumdev_v<DT>(row[i], K);
-    s1 = cta_sum<THREADS>(s1, slots, 0);
+    for (int i = threadIdx.x; i < nn; i += THREADS) moments_v<DT>(row[i], K, sp, qp);
+    float s1, q1;
+    cta_sum2<THREADS>(sp, qp, slots, s1, q1);
     cluster_wait();   // every CTA of the cluster runs, its mailboxes armed, before anything is posted to it
-    if (!mailbox_exchange(s1, box1, &xbar1, C, c)) nn = 0;
-    float t1 = 0.0f;
-    for (int i = 0; i < C; ++i) t1 += box1[i];
-    const float mu = fmaf(t1, inv_D, K);
-    float s2 = 0.0f;
+    if (!mailbox_exchange2(s1, q1, box1, &xbar1, C, c)) nn = 0;
+    float t1 = 0.0f, tq = 0.0f;
+    for (int i = 0; i < C; ++i) {
+        t1 += box1[i].x;
+        tq += box1[i].y;
+    }
+    float mu, var;
+    // every CTA adds the same values in the same order, so the whole cluster takes the same branch
+    if (!sweep_stats(t1, tq, inv_D, K, mu, var)) {
+        float s2 = 0.0f;
 #pragma unroll 4
-    for (int i = threadIdx.x; i < nn; i += THREADS) s2 += sqdev_v<DT>(row[i], mu);
-    s2 = cta_sum<THREADS>(s2, slots, 1);
-    if (!mailbox_exchange(s2, box2, &xbar2, C, c)) nn = 0;
-    float t2 = 0.0f;
-    for (int i = 0; i < C; ++i) t2 += box2[i];
-    const float rstd = rsqrtf(fmaf(t2, inv_D, eps));
+        for (int i = threadIdx.x; i < nn; i += THREADS) s2 += sqdev_v<DT>(row[i], mu);
+        s2 = cta_sum<THREADS>(s2, slots, 2);
+        if (!mailbox_exchange(s2, box2, &xbar2, C, c)) nn = 0;
+        float t2 = 0.0f;
+        for (int i = 0; i < C; ++i) t2 += box2[i];
+        var = t2 * inv_D;
+    }
+    const float rstd = rsqrtf(var + eps);
     uint4* yr = y + r * nvec + v0;
     const uint4* gr = gamma + v0;
     const uint4* br = beta + v0;
@@ -301,38 +431,47 @@ __global__ void __launch_bounds__(T)
 layernorm_cluster_stream_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamma,
                                 const uint4* __restrict__ beta, uint4* __restrict__ y, int64_t nvec, int C,
                                 float inv_D, float eps) {
-    __shared__ float slots[2 * kWarp];
-    __shared__ float box1[kMaxCluster], box2[kMaxCluster];
+    __shared__ float slots[3 * kWarp];
+    __shared__ __align__(8) float2 box1[kMaxCluster];
+    __shared__ float box2[kMaxCluster];
     __shared__ uint64_t xbar1, xbar2;
     const uint32_t c = cluster_rank();
     const int64_t r = blockIdx.x / C;
     const int64_t v0 = nvec / C * c + min((int64_t)c, nvec % C);
     const int64_t v1 = v0 + nvec / C + ((int64_t)c < nvec % C ? 1 : 0);
     if (threadIdx.x == 0) {
-        mailbox_arm(&xbar1, C);
+        mailbox_arm2(&xbar1, C);
         mailbox_arm(&xbar2, C);
     }
     __syncthreads();
     cluster_arrive_relaxed();
     const uint4* xr = x + r * nvec;
-    const float K = first_elem<DT>(xr);
-    float s1 = 0.0f;
+    const float K = head_mean<DT>(__ldg(xr));
+    f32x2 sp = pack2(0.0f, 0.0f), qp = sp;
 #pragma unroll 8
-    for (int64_t i = v0 + threadIdx.x; i < v1; i += T) s1 += sumdev_v<DT>(xr[i], K);
-    s1 = cta_sum<T>(s1, slots, 0);
+    for (int64_t i = v0 + threadIdx.x; i < v1; i += T) moments_v<DT>(xr[i], K, sp, qp);
+    float s1, q1;
+    cta_sum2<T>(sp, qp, slots, s1, q1);
     cluster_wait();   // every CTA of the cluster runs, its mailboxes armed, before anything is posted to it
-    bool ok = mailbox_exchange(s1, box1, &xbar1, C, c);
-    float t1 = 0.0f;
-    for (int i = 0; i < C; ++i) t1 += box1[i];
-    const float mu = fmaf(t1, inv_D, K);
-    float s2 = 0.0f;
+    bool ok = mailbox_exchange2(s1, q1, box1, &xbar1, C, c);
+    float t1 = 0.0f, tq = 0.0f;
+    for (int i = 0; i < C; ++i) {
+        t1 += box1[i].x;
+        tq += box1[i].y;
+    }
+    float mu, var;
+    // every CTA adds the same values in the same order, so the whole cluster takes the same branch
+    if (!sweep_stats(t1, tq, inv_D, K, mu, var)) {
+        float s2 = 0.0f;
 #pragma unroll 8
-    for (int64_t i = v0 + threadIdx.x; i < v1; i += T) s2 += sqdev_v<DT>(xr[i], mu);
-    s2 = cta_sum<T>(s2, slots, 1);
-    if (!mailbox_exchange(s2, box2, &xbar2, C, c)) ok = false;
-    float t2 = 0.0f;
-    for (int i = 0; i < C; ++i) t2 += box2[i];
-    const float rstd = rsqrtf(fmaf(t2, inv_D, eps));
+        for (int64_t i = v0 + threadIdx.x; i < v1; i += T) s2 += sqdev_v<DT>(xr[i], mu);
+        s2 = cta_sum<T>(s2, slots, 2);
+        if (!mailbox_exchange(s2, box2, &xbar2, C, c)) ok = false;
+        float t2 = 0.0f;
+        for (int i = 0; i < C; ++i) t2 += box2[i];
+        var = t2 * inv_D;
+    }
+    const float rstd = rsqrtf(var + eps);
     if (!ok) return;   // a wait that gave up (never expected): nothing is written
     uint4* yr = y + r * nvec;
 #pragma unroll 2
@@ -368,7 +507,7 @@ layernorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restric
     uint4* row = reinterpret_cast<uint4*>(smem_raw);
     uint16_t* row16 = reinterpret_cast<uint16_t*>(smem_raw);
     __shared__ uint64_t bar;
-    __shared__ float slots[2 * kWarp];
+    __shared__ float slots[3 * kWarp];
     const int64_t r = blockIdx.x;
     const uint16_t* xr = x + r * D;
     uint16_t* yr = y + r * D;
@@ -389,20 +528,25 @@ layernorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restric
     if (edge) row16[ek * 8 + (threadIdx.x & 7)] = ld_stream_u16(xr + ej);
     __syncthreads();
     if (!mbar_wait(&bar, 0)) return;  // gave up (flag set, see ak_wait_timeouts): a thread that exits no longer counts at later barriers
-    const float K = Elem<DT>::to_float(row16[phase]);
-    float s1 = 0.0f;
-    for (int k = k_lo + threadIdx.x; k < k_hi; k += T) s1 += sumdev_v<DT>(row[k], K);
-    if (edge) s1 += sub_h<DT>(row16[ek * 8 + (threadIdx.x & 7)], K);
-    s1 = cta_sum<T>(s1, slots, 0);
-    const float mu = fmaf(s1, inv_D, K);
-    float s2 = 0.0f;
-    for (int k = k_lo + threadIdx.x; k < k_hi; k += T) s2 += sqdev_v<DT>(row[k], mu);
-    if (edge) {
-        const float d = sub_h<DT>(row16[ek * 8 + (threadIdx.x & 7)], mu);
-        s2 = fmaf(d, d, s2);
+    // the shift of the one-sweep moments: the mean of the first inside vector, or the row's first
+    // element when there is none
+    const float K = (k_lo < k_hi) ? head_mean<DT>(row[k_lo]) : Elem<DT>::to_float(row16[phase]);
+    const float d0 = edge ? sub_h<DT>(row16[ek * 8 + (threadIdx.x & 7)], K) : 0.0f;
+    f32x2 sp = pack2(d0, 0.0f), qp = pack2(d0 * d0, 0.0f);
+#pragma unroll 4
+    for (int k = k_lo + threadIdx.x; k < k_hi; k += T) moments_v<DT>(row[k], K, sp, qp);
+    float s1, q1, mu, var;
+    cta_sum2<T>(sp, qp, slots, s1, q1);
+    if (!sweep_stats(s1, q1, inv_D, K, mu, var)) {
+        float s2 = 0.0f;
+        for (int k = k_lo + threadIdx.x; k < k_hi; k += T) s2 += sqdev_v<DT>(row[k], mu);
+        if (edge) {
+            const float d = sub_h<DT>(row16[ek * 8 + (threadIdx.x & 7)], mu);
+            s2 = fmaf(d, d, s2);
+        }
+        var = cta_sum<T>(s2, slots, 2) * inv_D;
     }
-    s2 = cta_sum<T>(s2, slots, 1);
-    const float rstd = rsqrtf(fmaf(s2, inv_D, eps));
+    const float rstd = rsqrtf(var + eps);
     if constexpr (TAB) {
         pdl_wait();   // the table is complete and visible; plain loads (cached in L1), not the read-only path
         const uint4* gt = tab + (size_t)phase * nvp;
@@ -430,15 +574,16 @@ layernorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restric
 // aligned and nv >= C.  TAB as in layernorm_stage_kernel.  grid = rows * C, cluster = C.  Dynamic
 // shared memory = ceil(max nv / C) * 16 bytes.
 template <int T, int DT = AK_DTYPE_BF16, bool TAB = false>
-__global__ void __launch_bounds__(T)
+__global__ void __launch_bounds__(T, 2)
 layernorm_cluster_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ gamma,
                                const uint16_t* __restrict__ beta, uint16_t* __restrict__ y, int64_t D, int C,
                                float inv_D, float eps, const uint4* tab, int nvp) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     uint4* row = reinterpret_cast<uint4*>(smem_raw);
     __shared__ uint64_t bar;
-    __shared__ float slots[2 * kWarp];
-    __shared__ float box1[kMaxCluster], box2[kMaxCluster];
+    __shared__ float slots[3 * kWarp];
+    __shared__ __align__(8) float2 box1[kMaxCluster];
+    __shared__ float box2[kMaxCluster];
     __shared__ uint64_t xbar1, xbar2;
     const uint32_t c = cluster_rank();
     const int64_t r = blockIdx.x / C;
@@ -460,34 +605,46 @@ layernorm_cluster_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* _
 
     if (threadIdx.x == 0) {
         mbar_init(&bar, 1);
-        mailbox_arm(&xbar1, C);
+        mailbox_arm2(&xbar1, C);
         mailbox_arm(&xbar2, C);
     }
     __syncthreads();
     if (threadIdx.x == 0)
         bulk_load_span(smem_raw + (size_t)(i0 - v0) * 16, xa + i0, i1 > i0 ? (uint32_t)(i1 - i0) * 16u : 0u, &bar);
     cluster_arrive_relaxed();
-    const float K = first_elem<DT>(xr);
+    // the shift of the one-sweep moments, the same in every CTA of the cluster: the mean of the
+    // row's first inside vector, or its first element when there is none
+    const float K = (k_lo < k_hi) ? head_mean<DT>(__ldg(xa + k_lo)) : first_elem<DT>(xr);
     const uint16_t xe = edge ? ld_stream_u16(xr + ej) : (uint16_t)0;
     // a wait that gave up (never expected) contributes nothing and writes nothing, but still posts
     bool ok = mbar_wait(&bar, 0);
     const int j0 = i0 - v0, j1 = ok ? i1 - v0 : j0;          // local indices of the fully-inside vectors
-    float s1 = edge ? sub_h<DT>(xe, K) : 0.0f;
-    for (int k = j0 + threadIdx.x; k < j1; k += T) s1 += sumdev_v<DT>(row[k], K);
-    s1 = cta_sum<T>(s1, slots, 0);
+    const float d0 = edge ? sub_h<DT>(xe, K) : 0.0f;
+    f32x2 sp = pack2(d0, 0.0f), qp = pack2(d0 * d0, 0.0f);
+#pragma unroll 4
+    for (int k = j0 + threadIdx.x; k < j1; k += T) moments_v<DT>(row[k], K, sp, qp);
+    float s1, q1;
+    cta_sum2<T>(sp, qp, slots, s1, q1);
     cluster_wait();   // every CTA of the cluster runs, its mailboxes armed, before anything is posted to it
-    if (!mailbox_exchange(s1, box1, &xbar1, C, c)) ok = false;
-    float t1 = 0.0f;
-    for (int i = 0; i < C; ++i) t1 += box1[i];
-    const float mu = fmaf(t1, inv_D, K);
-    const float de = edge ? sub_h<DT>(xe, mu) : 0.0f;
-    float s2 = de * de;
-    for (int k = j0 + threadIdx.x; k < j1; k += T) s2 += sqdev_v<DT>(row[k], mu);
-    s2 = cta_sum<T>(s2, slots, 1);
-    if (!mailbox_exchange(s2, box2, &xbar2, C, c)) ok = false;
-    float t2 = 0.0f;
-    for (int i = 0; i < C; ++i) t2 += box2[i];
-    const float rstd = rsqrtf(fmaf(t2, inv_D, eps));
+    if (!mailbox_exchange2(s1, q1, box1, &xbar1, C, c)) ok = false;
+    float t1 = 0.0f, tq = 0.0f;
+    for (int i = 0; i < C; ++i) {
+        t1 += box1[i].x;
+        tq += box1[i].y;
+    }
+    float mu, var;
+    // every CTA adds the same values in the same order, so the whole cluster takes the same branch
+    if (!sweep_stats(t1, tq, inv_D, K, mu, var)) {
+        const float de = edge ? sub_h<DT>(xe, mu) : 0.0f;
+        float s2 = de * de;
+        for (int k = j0 + threadIdx.x; k < j1; k += T) s2 += sqdev_v<DT>(row[k], mu);
+        s2 = cta_sum<T>(s2, slots, 2);
+        if (!mailbox_exchange(s2, box2, &xbar2, C, c)) ok = false;
+        float t2 = 0.0f;
+        for (int i = 0; i < C; ++i) t2 += box2[i];
+        var = t2 * inv_D;
+    }
+    const float rstd = rsqrtf(var + eps);
     if (!ok) return;
     if constexpr (TAB) {
         pdl_wait();   // the table is complete and visible; plain loads (cached in L1), not the read-only path
