@@ -269,9 +269,11 @@ int dispatch_t(const void* x, const void* gamma, const void* beta, void* y, int6
                 uint16_t* ys = static_cast<uint16_t*>(y);
                 // rows of up to 1024 covering vectors stay in the registers of a 128-thread CTA ...
                 const int64_t max_nv = (D + 14) >> 3;   // vectors covering the row at the worst phase
-                // rows beyond one CTA's shared memory (up to eight CTAs'), and a few long rows (at most
-                // 64 of 32 KiB or more): the covering vectors split over a thread-block cluster
-                const int Cu = cluster_ctas(rows, (int64_t)stage_bytes, kMaxRowSmemBytes + 16);
+                // long rows (up to eight CTAs' shared memory), and a few rows (at most 64) of 32 KiB or
+                // more: the covering vectors split over a thread-block cluster;
+                // unaligned rows are split over a cluster from 160 KiB on (4096 x 100001: 376 -> 348 us; at 128 KiB
+                // and below one CTA per row is as fast or faster)
+                const int Cu = cluster_ctas(rows, (int64_t)stage_bytes, 163840 + 16);
                 if (same_phase && params4 && Cu > 1 && stage_bytes <= (size_t)kMaxCluster * kMaxRowSmemBytes && rows * Cu <= 2147483647LL) {
                     if (launch_cluster_stage<DT, 256>(xs, gs, bs, ys, rows, D, max_nv, Cu, inv_D, eps, st) == AK_OK) return AK_OK;
                     (void)cudaGetLastError();   // the cluster cannot be co-scheduled here: the kernels below

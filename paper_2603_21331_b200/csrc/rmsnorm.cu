@@ -206,9 +206,11 @@ int dispatch_t(const void* x, const void* w, void* y, int64_t rows, int64_t D, f
                 const uint16_t* ws = static_cast<const uint16_t*>(w);
                 uint16_t* ys = static_cast<uint16_t*>(y);
                 const int64_t max_nv = (D + 14) >> 3;   // vectors covering the row at the worst phase
-                // rows beyond one CTA's shared memory (up to eight CTAs'), and a few long rows (at most
-                // 64 of 32 KiB or more): the covering vectors split over a thread-block cluster
-                const int Cu = cluster_ctas(rows, (int64_t)stage_bytes, kMaxRowSmemBytes + 16);
+                // long rows (up to eight CTAs' shared memory), and a few rows (at most 64) of 32 KiB or
+                // more: the covering vectors split over a thread-block cluster;
+                // unaligned rows are split over a cluster from 128 KiB on (4096 x 65539: 235 -> 229 us, 4096 x 100001:
+                // 337 -> 322 us; at 100 KiB one CTA per row is 4 % faster)
+                const int Cu = cluster_ctas(rows, (int64_t)stage_bytes, 131072 + 16);
                 if (same_phase && is_aligned(w, 4) && Cu > 1 && stage_bytes <= (size_t)kMaxCluster * kMaxRowSmemBytes && rows * Cu <= 2147483647LL) {
                     if (launch_cluster_stage<DT, 256>(xs, ws, ys, rows, D, max_nv, Cu, inv_D, eps, st) == AK_OK) return AK_OK;
                     (void)cudaGetLastError();   // the cluster cannot be co-scheduled here: the kernels below

@@ -228,7 +228,7 @@ rmsnorm_cluster_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w,
 // mailbox) and once more to scale and store; the second read finds what the caches kept (nothing
 // is staged).  Needs 16-byte aligned rows.  grid = rows * C, cluster = C.
 template <int T, int DT = AK_DTYPE_BF16>
-__global__ void __launch_bounds__(T)
+__global__ void __launch_bounds__(T, 1)
 rmsnorm_cluster_stream_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w, uint4* __restrict__ y,
                               int64_t nvec, int C, float inv_D, float eps) {
     __shared__ float slots[2 * kWarp];

@@ -61,11 +61,11 @@ int launch_stage(const uint16_t* x, uint16_t* y, int64_t rows, int64_t D, size_t
 }
 
 // unaligned rows split over a cluster of C CTAs (covering vectors of the worst phase: max_nv)
-template <int DT, int T>
+template <int DT, int T, int KEEP>
 int launch_cluster_stage(const uint16_t* x, uint16_t* y, int64_t rows, int64_t D, int64_t max_nv, int C, cudaStream_t st) {
-    if (!allow_big_smem(softmax_cluster_stage_kernel<T, DT>)) return AK_ERR_CUDA;
+    if (!allow_big_smem(softmax_cluster_stage_kernel<T, DT, KEEP>)) return AK_ERR_CUDA;
     const size_t smem = (size_t)((max_nv + C - 1) / C) * 16;
-    const cudaError_t e = launch_cluster(softmax_cluster_stage_kernel<T, DT>, (unsigned)(rows * C), T, smem, C, st, x, y, D, C);
+    const cudaError_t e = launch_cluster(softmax_cluster_stage_kernel<T, DT, KEEP>, (unsigned)(rows * C), T, smem, C, st, x, y, D, C);
     count_launch();
     return e == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
@@ -157,8 +157,10 @@ int dispatch_t(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st,
             }
             // many rows in slices of up to 32 KiB: 128-thread CTAs measured 2-12 % faster than 256
             // (and 64 slower); a few rows are better off with 256
-            if ((nvec + C - 1) / C <= 2048 && rows > 64) return launch_cluster_rows<DT, 128, 4>(x, y, rows, nvec, C, st);
-            if ((nvec + C - 1) / C <= 4096) return launch_cluster_rows<DT, 256, 4>(x, y, rows, nvec, C, st);
+            // kept exponentials per thread picked by timing (4096 x 65536: 4 kept 177 us, 6 kept 166 us,
+            // 8 kept 179 us: 72 registers still leave the seven CTAs per SM that shared memory allows)
+            if ((nvec + C - 1) / C <= 2048 && rows > 64) return launch_cluster_rows<DT, 128, 6>(x, y, rows, nvec, C, st);
+            if ((nvec + C - 1) / C <= 4096) return launch_cluster_rows<DT, 256, 7>(x, y, rows, nvec, C, st);
             return launch_cluster_rows<DT, 512, 0>(x, y, rows, nvec, C, st);
         }
         case AK_PATH_GENERIC: {
@@ -181,13 +183,17 @@ int dispatch_t(const void* x, void* y, int64_t rows, int64_t D, cudaStream_t st,
                 const int64_t max_nv = (D + 14) >> 3;   // vectors covering the row at the worst phase
                 if (same_phase && max_nv <= 512)
                     return launch_regp_vpt<DT, 128, 5>((int)((max_nv + 127) / 128), xs, ys, rows, D, st);
-                // rows beyond one CTA's shared memory (up to eight CTAs'), and a few long rows: the
-                // covering vectors split over a thread-block cluster
-                const int Cu = cluster_ctas(rows, (int64_t)stage_bytes, kMaxRowSmemBytes + 16);
+                // rows of more than 96 KiB (up to eight CTAs' shared memory), and a few long rows: the
+                // covering vectors split over a thread-block cluster (4096 x 65539: 257 us staged by one
+                // CTA, 207 us in clusters; 4096 x 40001: 115 us against 126 us)
+                const int Cu = cluster_ctas(rows, (int64_t)stage_bytes, 98304 + 16);
                 if (same_phase && Cu > 1 && stage_bytes <= (size_t)kMaxCluster * kMaxRowSmemBytes && rows * Cu <= 2147483647LL) {
-                    const int s = (rows > 64 && (max_nv + Cu - 1) / Cu <= 2048)
-                                      ? launch_cluster_stage<DT, 128>(xs, ys, rows, D, max_nv, Cu, st)
-                                      : launch_cluster_stage<DT, 256>(xs, ys, rows, D, max_nv, Cu, st);
+                    // exponentials kept per thread as in the aligned cluster kernel; a few rows (latency-
+                    // bound) are better off with fewer registers (64 x 128257: 4 kept 11.7 us, 7 kept 14.3 us)
+                    const int s = rows <= 64 ? launch_cluster_stage<DT, 256, 4>(xs, ys, rows, D, max_nv, Cu, st)
+                                  : (max_nv + Cu - 1) / Cu <= 2048
+                                      ? launch_cluster_stage<DT, 128, 6>(xs, ys, rows, D, max_nv, Cu, st)
+                                      : launch_cluster_stage<DT, 256, 7>(xs, ys, rows, D, max_nv, Cu, st);
                     if (s == AK_OK) return AK_OK;
                     (void)cudaGetLastError();   // the cluster cannot be co-scheduled here: the kernels below
                 }

@@ -227,7 +227,7 @@ softmax_smem_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int nvec
 // rank order in every CTA.  The first KEEP vectors of a thread keep their exponentials in
 // registers.  grid = rows * C, cluster = C.  Dynamic shared memory = ceil(nvec / C) * 16 bytes.
 template <int THREADS, int KEEP, int DT = AK_DTYPE_BF16>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, THREADS <= 128 ? 7 : (THREADS <= 256 ? 3 : 1))
 softmax_cluster_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int nvec, int C) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint4* row = reinterpret_cast<const uint4*>(smem_raw);
@@ -397,7 +397,7 @@ softmax_stage_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, i
 // softmax_cluster_kernel.  For unaligned rows longer than one CTA's shared memory (up to eight) and
 // for a few long unaligned rows.  Needs x and y rows in the same phase and nv >= C.
 // grid = rows * C, cluster = C.  Dynamic shared memory = ceil(max nv / C) * 16 bytes.
-template <int T, int DT = AK_DTYPE_BF16>
+template <int T, int DT = AK_DTYPE_BF16, int KEEP = 0>
 __global__ void __launch_bounds__(T)
 softmax_cluster_stage_kernel(const uint16_t* __restrict__ x, uint16_t* __restrict__ y, int64_t D, int C) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -451,15 +451,28 @@ softmax_cluster_stage_kernel(const uint16_t* __restrict__ x, uint16_t* __restric
     for (int i = 1; i < C; ++i) m = fmaxf(m, box_m[i]);
     const float m2 = m * kLog2e;
     float sum = 0.0f;
+    f32x2 kept[KEEP > 0 ? KEEP : 1][kExpPairs<DT>];
     f32x2 e[kExpPairs<DT>];
-    for (int k = threadIdx.x; k < nn; k += T) sum += exp_v<DT>(row[k], m2, e);
+#pragma unroll
+    for (int j = 0; j < KEEP; ++j) {
+        const int k = threadIdx.x + j * T;
+        if (k < nn) sum += exp_v<DT>(row[k], m2, kept[j]);
+    }
+    for (int k = threadIdx.x + KEEP * T; k < nn; k += T) sum += exp_v<DT>(row[k], m2, e);
     sum = cta_sum<T>(sum, slots, 1);
     if (!mailbox_exchange(sum, box_s, &xbar_s, C, c)) ok = false;
     float tot = 0.0f;
     for (int i = 0; i < C; ++i) tot += box_s[i];
     const float inv = 1.0f / tot;
     if (!ok) return;
-    for (int k = i0 + threadIdx.x; k < i1; k += T) {
+    // local vector k is covering vector v0 + k of the row; only the fully-inside ones are stored whole
+#pragma unroll
+    for (int j = 0; j < KEEP; ++j) {
+        const int k = v0 + threadIdx.x + j * T;
+        if (k >= i0 && k < i1) st_stream(ya + k, norm_v<DT>(kept[j], inv));
+    }
+    for (int k = v0 + threadIdx.x + KEEP * T; k < i1; k += T) {
+        if (k < i0) continue;
         exp_v<DT>(row[k - v0], m2, e);
         st_stream(ya + k, norm_v<DT>(e, inv));
     }
