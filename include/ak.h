@@ -196,11 +196,13 @@ int ak_choose_path_dt(int op, int64_t rows, int64_t D, int aligned16, int dtype)
  * x, y: device bf16 [rows, D] (y may alias x); gamma, beta: device bf16 [D]; moments in
  * fp32 and fixed order over the on-chip copy of the row, shifted by a value K taken from the
  * row itself (its first element, or the mean of its first 16 bytes): mu = K + mean(x - K),
- * so a constant row gives exactly beta.  Short rows and rows that are not 16-byte aligned
- * make a second centred pass for the variance; the other layouts take sum((x - K)^2) in the
- * same sweep and use var = mean((x - K)^2) - (mu - K)^2 when (mu - K)^2 <= var (the
- * subtraction then costs at most a factor three in the relative error of var), and make
- * the centred pass otherwise.  eps finite, >= 0.
+ * so a constant row gives exactly beta.  Short rows and unaligned rows held in registers then
+ * sum x - mu and (x - mu)^2 in a second pass: var = mean((x - mu)^2) - mean(x - mu)^2, and
+ * mean(x - mu) is added to mu, which removes what a shift far from the mean (an outlier as
+ * first element) had cost it.  The other layouts take sum((x - K)^2) in the first sweep and use
+ * var = mean((x - K)^2) - (mu - K)^2 when (mu - K)^2 <= var (the subtraction then costs at
+ * most a factor three in the relative error of var); otherwise they make that second pass
+ * too.  eps finite, >= 0.
  * Same path ids, size limits and alignment rules as RMSNorm (gamma and beta together play
  * the part of w).  Status codes as for RMSNorm.  One launch and no scratch, except for many
  * rows that are not 16-byte aligned (1024 or more of D <= about 32750, 256 or more longer ones

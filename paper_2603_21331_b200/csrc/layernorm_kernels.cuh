@@ -81,14 +81,22 @@ __device__ __forceinline__ float head_mean(const uint4 v) {
 }
 // Mean and variance from the one-sweep sums s = sum(x - K), q = sum((x - K)^2).  False when the
 // shift is so far from the mean (or something is not a number) that the subtraction
-// q/D - (s/D)^2 would lose accuracy: the caller then makes the centred pass sum((x - mu)^2).
+// q/D - (s/D)^2 would lose accuracy: the caller then sweeps again with the shift mu (refine_stats).
 __device__ __forceinline__ bool sweep_stats(float s, float q, float inv_D, float K, float& mu, float& var) {
     const float m = s * inv_D;   // mean - K
     mu = K + m;
     var = fmaf(q, inv_D, -(m * m));
     return m * m <= var;
 }
-// the lane sums of packed accumulators, added over the CTA with one barrier (slot sets 0 and 1)
+// The second sweep of such a row is shifted by the first estimate of the mean: s and q are now
+// sums of x - mu and (x - mu)^2, what is left of the mean is tiny against the spread, and the
+// subtraction is harmless.  The mean gains the accuracy the far shift had cost it.
+__device__ __forceinline__ void refine_stats(float s, float q, float inv_D, float& mu, float& var) {
+    const float m = s * inv_D;
+    mu += m;
+    var = fmaxf(fmaf(q, inv_D, -(m * m)), 0.0f);
+}
+// the lane sums of packed accumulators, added over the CTA with one barrier (two sets of slots)
 template <int THREADS>
 __device__ __forceinline__ void cta_sum2(f32x2 sp, f32x2 qp, float* slots, float& s, float& q) {
     constexpr int NW = THREADS / kWarp;
@@ -186,9 +194,10 @@ __device__ __forceinline__ float first_elem(const void* row) {
 // barrier: s = sum(x - K) and q = sum((x - K)^2) with K the mean of the row's first 16 bytes,
 // mean = K + s/D, variance = q/D - (s/D)^2.  The subtraction loses accuracy only when the shift
 // is far from the mean, so the result is kept when (s/D)^2 <= variance (the relative error of
-// the variance is then at most three times that of q) and the centred second pass runs
-// otherwise (a whole row at a time, so the branch does not diverge).  A constant row gives
-// s = q = 0 exactly, hence the output beta bit for bit.
+// the variance is then at most three times that of q); otherwise the registers are swept once
+// more with the shift K := mean estimate, which corrects the mean as well (a whole row at a
+// time, so the branch does not diverge).  A constant row gives s = q = 0 exactly, hence the
+// output beta bit for bit.
 //
 // P_EARLY: gamma and beta are requested together with the row instead of after the reductions
 // (8 * VPT more live registers; for launches too small to fill the GPU, where latency counts).
@@ -207,7 +216,7 @@ layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamm
     static_assert(!FULL || GROUPS == 1, "FULL is for one row per CTA");
     // SWEEP1 alternates between two sets of slots by row, so that one barrier per row is enough:
     // a warp can be at most one barrier ahead of the slowest reader
-    __shared__ float slots2[2][3][THREADS / kWarp];
+    __shared__ float slots2[2][4][THREADS / kWarp];
     int par = 0;
     {
         const int64_t r0 = (int64_t)blockIdx.x * GROUPS;
@@ -277,11 +286,25 @@ layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamm
                 q1 = warp_sum((lane < WARPS_PER_GROUP) ? q[lane] : 0.0f);
             }
             if (!sweep_stats(s1, q1, inv_D, K, mu, var)) {
-                float s2 = 0.0f;
+                sp = pack2(0.0f, 0.0f);
+                qp = sp;
 #pragma unroll
                 for (int k = 0; k < VPT; ++k)
-                    if (FULL || (live && t + k * GROUP < nvec)) s2 += sqdev_v<DT>(xv[k], mu);
-                var = group_sum(s2, 2) * inv_D;
+                    if (FULL || (live && t + k * GROUP < nvec)) moments_v<DT>(xv[k], mu, sp, qp);
+                unpack2(sp, lo, hi);
+                s1 = warp_sum(lo + hi);
+                unpack2(qp, lo, hi);
+                q1 = warp_sum(lo + hi);
+                float* s = slots[2] + g * WARPS_PER_GROUP;
+                float* q = slots[3] + g * WARPS_PER_GROUP;
+                if (lane == 0) {
+                    s[warp_in_group] = s1;
+                    q[warp_in_group] = q1;
+                }
+                __syncthreads();
+                s1 = warp_sum((lane < WARPS_PER_GROUP) ? s[lane] : 0.0f);
+                q1 = warp_sum((lane < WARPS_PER_GROUP) ? q[lane] : 0.0f);
+                refine_stats(s1, q1, inv_D, mu, var);
             }
             par ^= 1;
         } else {
@@ -290,11 +313,29 @@ layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamm
             for (int k = 0; k < VPT; ++k)
                 if (live && t + k * GROUP < nvec) s1 += sumdev_v<DT>(xv[k], K);
             mu = fmaf(group_sum(s1, 0), inv_D, K);
-            float s2 = 0.0f;
+            // the second pass also sums x - mu: what the first element as shift cost the mean
+            // (it may be an outlier) is corrected, see refine_stats
+            f32x2 sp = pack2(0.0f, 0.0f), qp = sp;
 #pragma unroll
             for (int k = 0; k < VPT; ++k)
-                if (live && t + k * GROUP < nvec) s2 += sqdev_v<DT>(xv[k], mu);
-            var = group_sum(s2, 1) * inv_D;
+                if (live && t + k * GROUP < nvec) moments_v<DT>(xv[k], mu, sp, qp);
+            float lo, hi;
+            unpack2(sp, lo, hi);
+            float s2 = warp_sum(lo + hi);
+            unpack2(qp, lo, hi);
+            float q2 = warp_sum(lo + hi);
+            if constexpr (WARPS_PER_GROUP > 1) {
+                float* s = slots[1] + g * WARPS_PER_GROUP;
+                float* q = slots[2] + g * WARPS_PER_GROUP;
+                if (lane == 0) {
+                    s[warp_in_group] = s2;
+                    q[warp_in_group] = q2;
+                }
+                __syncthreads();
+                s2 = warp_sum((lane < WARPS_PER_GROUP) ? s[lane] : 0.0f);
+                q2 = warp_sum((lane < WARPS_PER_GROUP) ? q[lane] : 0.0f);
+            }
+            refine_stats(s2, q2, inv_D, mu, var);
         }
         const float rstd = rsqrtf(var + eps);
         // FULL: the row index is read again rather than kept in registers across the reductions
@@ -324,7 +365,7 @@ layernorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gam
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint4* row = reinterpret_cast<const uint4*>(smem_raw);
     __shared__ uint64_t bar;
-    __shared__ float slots[3 * kWarp];
+    __shared__ float slots[4 * kWarp];
     const int64_t r = blockIdx.x;
     if (threadIdx.x == 0) mbar_init(&bar, 1);
     __syncthreads();
@@ -343,10 +384,12 @@ layernorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gam
     float s1, q1, mu, var;
     cta_sum2<THREADS>(sp, qp, slots, s1, q1);
     if (!sweep_stats(s1, q1, inv_D, K, mu, var)) {
-        float s2 = 0.0f;
+        sp = pack2(0.0f, 0.0f);
+        qp = sp;
 #pragma unroll 4
-        for (int i = threadIdx.x; i < nvec; i += THREADS) s2 += sqdev_v<DT>(row[i], mu);
-        var = cta_sum<THREADS>(s2, slots, 2) * inv_D;
+        for (int i = threadIdx.x; i < nvec; i += THREADS) moments_v<DT>(row[i], mu, sp, qp);
+        cta_sum2<THREADS>(sp, qp, slots + 2 * kWarp, s1, q1);
+        refine_stats(s1, q1, inv_D, mu, var);
     }
     const float rstd = rsqrtf(var + eps);
     uint4* yr = y + r * nvec;
@@ -369,9 +412,8 @@ layernorm_cluster_kernel(const uint4* __restrict__ x, const uint4* __restrict__ 
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint4* row = reinterpret_cast<const uint4*>(smem_raw);
     __shared__ uint64_t bar;
-    __shared__ float slots[3 * kWarp];
-    __shared__ __align__(8) float2 box1[kMaxCluster];
-    __shared__ float box2[kMaxCluster];
+    __shared__ float slots[4 * kWarp];
+    __shared__ __align__(8) float2 box1[kMaxCluster], box2[kMaxCluster];
     __shared__ uint64_t xbar1, xbar2;
     const uint32_t c = cluster_rank();
     const int64_t r = blockIdx.x / C;
@@ -380,7 +422,7 @@ layernorm_cluster_kernel(const uint4* __restrict__ x, const uint4* __restrict__ 
     if (threadIdx.x == 0) {
         mbar_init(&bar, 1);
         mailbox_arm2(&xbar1, C);
-        mailbox_arm(&xbar2, C);
+        mailbox_arm2(&xbar2, C);
     }
     __syncthreads();
     if (threadIdx.x == 0) bulk_load_span(smem_raw, x + r * nvec + v0, (uint32_t)n * 16u, &bar);
@@ -403,14 +445,19 @@ layernorm_cluster_kernel(const uint4* __restrict__ x, const uint4* __restrict__ 
     float mu, var;
     // every CTA adds the same values in the same order, so the whole cluster takes the same branch
     if (!sweep_stats(t1, tq, inv_D, K, mu, var)) {
-        float s2 = 0.0f;
+        sp = pack2(0.0f, 0.0f);
+        qp = sp;
 #pragma unroll 4
-        for (int i = threadIdx.x; i < nn; i += THREADS) s2 += sqdev_v<DT>(row[i], mu);
-        s2 = cta_sum<THREADS>(s2, slots, 2);
-        if (!mailbox_exchange(s2, box2, &xbar2, C, c)) nn = 0;
-        float t2 = 0.0f;
-        for (int i = 0; i < C; ++i) t2 += box2[i];
-        var = t2 * inv_D;
+        for (int i = threadIdx.x; i < nn; i += THREADS) moments_v<DT>(row[i], mu, sp, qp);
+        cta_sum2<THREADS>(sp, qp, slots + 2 * kWarp, s1, q1);
+        if (!mailbox_exchange2(s1, q1, box2, &xbar2, C, c)) nn = 0;
+        t1 = 0.0f;
+        tq = 0.0f;
+        for (int i = 0; i < C; ++i) {
+            t1 += box2[i].x;
+            tq += box2[i].y;
+        }
+        refine_stats(t1, tq, inv_D, mu, var);
     }
     const float rstd = rsqrtf(var + eps);
     uint4* yr = y + r * nvec + v0;
@@ -431,9 +478,8 @@ __global__ void __launch_bounds__(T)
 layernorm_cluster_stream_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamma,
                                 const uint4* __restrict__ beta, uint4* __restrict__ y, int64_t nvec, int C,
                                 float inv_D, float eps) {
-    __shared__ float slots[3 * kWarp];
-    __shared__ __align__(8) float2 box1[kMaxCluster];
-    __shared__ float box2[kMaxCluster];
+    __shared__ float slots[4 * kWarp];
+    __shared__ __align__(8) float2 box1[kMaxCluster], box2[kMaxCluster];
     __shared__ uint64_t xbar1, xbar2;
     const uint32_t c = cluster_rank();
     const int64_t r = blockIdx.x / C;
@@ -441,7 +487,7 @@ layernorm_cluster_stream_kernel(const uint4* __restrict__ x, const uint4* __rest
     const int64_t v1 = v0 + nvec / C + ((int64_t)c < nvec % C ? 1 : 0);
     if (threadIdx.x == 0) {
         mailbox_arm2(&xbar1, C);
-        mailbox_arm(&xbar2, C);
+        mailbox_arm2(&xbar2, C);
     }
     __syncthreads();
     cluster_arrive_relaxed();
@@ -462,14 +508,19 @@ layernorm_cluster_stream_kernel(const uint4* __restrict__ x, const uint4* __rest
     float mu, var;
     // every CTA adds the same values in the same order, so the whole cluster takes the same branch
     if (!sweep_stats(t1, tq, inv_D, K, mu, var)) {
-        float s2 = 0.0f;
+        sp = pack2(0.0f, 0.0f);
+        qp = sp;
 #pragma unroll 8
-        for (int64_t i = v0 + threadIdx.x; i < v1; i += T) s2 += sqdev_v<DT>(xr[i], mu);
-        s2 = cta_sum<T>(s2, slots, 2);
-        if (!mailbox_exchange(s2, box2, &xbar2, C, c)) ok = false;
-        float t2 = 0.0f;
-        for (int i = 0; i < C; ++i) t2 += box2[i];
-        var = t2 * inv_D;
+        for (int64_t i = v0 + threadIdx.x; i < v1; i += T) moments_v<DT>(xr[i], mu, sp, qp);
+        cta_sum2<T>(sp, qp, slots + 2 * kWarp, s1, q1);
+        if (!mailbox_exchange2(s1, q1, box2, &xbar2, C, c)) ok = false;
+        t1 = 0.0f;
+        tq = 0.0f;
+        for (int i = 0; i < C; ++i) {
+            t1 += box2[i].x;
+            tq += box2[i].y;
+        }
+        refine_stats(t1, tq, inv_D, mu, var);
     }
     const float rstd = rsqrtf(var + eps);
     if (!ok) return;   // a wait that gave up (never expected): nothing is written
@@ -507,7 +558,7 @@ layernorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restric
     uint4* row = reinterpret_cast<uint4*>(smem_raw);
     uint16_t* row16 = reinterpret_cast<uint16_t*>(smem_raw);
     __shared__ uint64_t bar;
-    __shared__ float slots[3 * kWarp];
+    __shared__ float slots[4 * kWarp];
     const int64_t r = blockIdx.x;
     const uint16_t* xr = x + r * D;
     uint16_t* yr = y + r * D;
@@ -538,13 +589,13 @@ layernorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restric
     float s1, q1, mu, var;
     cta_sum2<T>(sp, qp, slots, s1, q1);
     if (!sweep_stats(s1, q1, inv_D, K, mu, var)) {
-        float s2 = 0.0f;
-        for (int k = k_lo + threadIdx.x; k < k_hi; k += T) s2 += sqdev_v<DT>(row[k], mu);
-        if (edge) {
-            const float d = sub_h<DT>(row16[ek * 8 + (threadIdx.x & 7)], mu);
-            s2 = fmaf(d, d, s2);
-        }
-        var = cta_sum<T>(s2, slots, 2) * inv_D;
+        const float d1 = edge ? sub_h<DT>(row16[ek * 8 + (threadIdx.x & 7)], mu) : 0.0f;
+        sp = pack2(d1, 0.0f);
+        qp = pack2(d1 * d1, 0.0f);
+#pragma unroll 4
+        for (int k = k_lo + threadIdx.x; k < k_hi; k += T) moments_v<DT>(row[k], mu, sp, qp);
+        cta_sum2<T>(sp, qp, slots + 2 * kWarp, s1, q1);
+        refine_stats(s1, q1, inv_D, mu, var);
     }
     const float rstd = rsqrtf(var + eps);
     if constexpr (TAB) {
@@ -581,9 +632,8 @@ layernorm_cluster_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* _
     extern __shared__ __align__(128) unsigned char smem_raw[];
     uint4* row = reinterpret_cast<uint4*>(smem_raw);
     __shared__ uint64_t bar;
-    __shared__ float slots[3 * kWarp];
-    __shared__ __align__(8) float2 box1[kMaxCluster];
-    __shared__ float box2[kMaxCluster];
+    __shared__ float slots[4 * kWarp];
+    __shared__ __align__(8) float2 box1[kMaxCluster], box2[kMaxCluster];
     __shared__ uint64_t xbar1, xbar2;
     const uint32_t c = cluster_rank();
     const int64_t r = blockIdx.x / C;
@@ -606,7 +656,7 @@ layernorm_cluster_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* _
     if (threadIdx.x == 0) {
         mbar_init(&bar, 1);
         mailbox_arm2(&xbar1, C);
-        mailbox_arm(&xbar2, C);
+        mailbox_arm2(&xbar2, C);
     }
     __syncthreads();
     if (threadIdx.x == 0)
@@ -635,14 +685,20 @@ layernorm_cluster_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* _
     float mu, var;
     // every CTA adds the same values in the same order, so the whole cluster takes the same branch
     if (!sweep_stats(t1, tq, inv_D, K, mu, var)) {
-        const float de = edge ? sub_h<DT>(xe, mu) : 0.0f;
-        float s2 = de * de;
-        for (int k = j0 + threadIdx.x; k < j1; k += T) s2 += sqdev_v<DT>(row[k], mu);
-        s2 = cta_sum<T>(s2, slots, 2);
-        if (!mailbox_exchange(s2, box2, &xbar2, C, c)) ok = false;
-        float t2 = 0.0f;
-        for (int i = 0; i < C; ++i) t2 += box2[i];
-        var = t2 * inv_D;
+        const float d1 = edge ? sub_h<DT>(xe, mu) : 0.0f;
+        sp = pack2(d1, 0.0f);
+        qp = pack2(d1 * d1, 0.0f);
+#pragma unroll 4
+        for (int k = j0 + threadIdx.x; k < j1; k += T) moments_v<DT>(row[k], mu, sp, qp);
+        cta_sum2<T>(sp, qp, slots + 2 * kWarp, s1, q1);
+        if (!mailbox_exchange2(s1, q1, box2, &xbar2, C, c)) ok = false;
+        t1 = 0.0f;
+        tq = 0.0f;
+        for (int i = 0; i < C; ++i) {
+            t1 += box2[i].x;
+            tq += box2[i].y;
+        }
+        refine_stats(t1, tq, inv_D, mu, var);
     }
     const float rstd = rsqrtf(var + eps);
     if (!ok) return;
@@ -675,7 +731,7 @@ __global__ void __launch_bounds__(THREADS, MINB)
 layernorm_regp_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict__ gamma,
                       const uint16_t* __restrict__ beta, uint16_t* __restrict__ y, int64_t D, float inv_D, float eps,
                       const uint4* tab, int nvp) {
-    __shared__ float slots[2 * kWarp];
+    __shared__ float slots[3 * kWarp];
     const int64_t r = blockIdx.x;
     const uint16_t* xr = x + r * D;
     uint16_t* yr = y + r * D;
@@ -704,14 +760,18 @@ layernorm_regp_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict
     for (int i = 0; i < VPT; ++i)
         if (k_lo + (int)threadIdx.x + i * THREADS < k_hi) s1 += sumdev_v<DT>(xv[i], K);
     s1 = cta_sum<THREADS>(s1, slots, 0);
-    const float mu = fmaf(s1, inv_D, K);
+    float mu = fmaf(s1, inv_D, K), var;
+    // the second pass also sums x - mu: what the first element as shift cost the mean (it may
+    // be an outlier) is corrected, see refine_stats
     const float de = edge ? sub_h<DT>(xe, mu) : 0.0f;
-    float s2 = de * de;
+    f32x2 sp = pack2(de, 0.0f), qp = pack2(de * de, 0.0f);
 #pragma unroll
     for (int i = 0; i < VPT; ++i)
-        if (k_lo + (int)threadIdx.x + i * THREADS < k_hi) s2 += sqdev_v<DT>(xv[i], mu);
-    s2 = cta_sum<THREADS>(s2, slots, 1);
-    const float rstd = rsqrtf(fmaf(s2, inv_D, eps));
+        if (k_lo + (int)threadIdx.x + i * THREADS < k_hi) moments_v<DT>(xv[i], mu, sp, qp);
+    float s2, q2;
+    cta_sum2<THREADS>(sp, qp, slots + kWarp, s2, q2);
+    refine_stats(s2, q2, inv_D, mu, var);
+    const float rstd = rsqrtf(var + eps);
     if constexpr (TAB) {
         pdl_wait();   // the table is complete and visible; plain loads (cached in L1), not the read-only path
         const uint4* gt = tab + (size_t)phase * nvp;
@@ -746,7 +806,7 @@ layernorm_generic_kernel(const uint16_t* __restrict__ x, const uint16_t* __restr
                          const uint16_t* __restrict__ beta, uint16_t* __restrict__ y, int64_t rows, int64_t D,
                          float inv_D, float eps) {
     constexpr int T = kLnGenericThreads;
-    __shared__ float slots[2 * kWarp];
+    __shared__ float slots[3 * kWarp];
     for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
         const uint16_t* xr = x + row * D;
         uint16_t* yr = y + row * D;
@@ -754,14 +814,17 @@ layernorm_generic_kernel(const uint16_t* __restrict__ x, const uint16_t* __restr
         float s1 = 0.0f;
         for (int64_t j = threadIdx.x; j < D; j += T) s1 += sub_h<DT>(xr[j], K);
         s1 = cta_sum<T>(s1, slots, 0);
-        const float mu = fmaf(s1, inv_D, K);
-        float s2 = 0.0f;
+        float mu = fmaf(s1, inv_D, K), var;
+        float r2 = 0.0f, s2 = 0.0f;   // the second pass also sums x - mu, see refine_stats
         for (int64_t j = threadIdx.x; j < D; j += T) {
             const float d = sub_h<DT>(xr[j], mu);
+            r2 += d;
             s2 = fmaf(d, d, s2);
         }
-        s2 = cta_sum<T>(s2, slots, 1);
-        const float rstd = rsqrtf(fmaf(s2, inv_D, eps));
+        r2 = cta_sum<T>(r2, slots, 1);
+        s2 = cta_sum<T>(s2, slots, 2);
+        refine_stats(r2, s2, inv_D, mu, var);
+        const float rstd = rsqrtf(var + eps);
         for (int64_t j = threadIdx.x; j < D; j += T)
             yr[j] = Elem<DT>::from_float(ln_out1<DT>(xr[j], __ldg(gamma + j), __ldg(beta + j), mu, rstd));
     }
@@ -772,7 +835,7 @@ __global__ void __launch_bounds__(kLnGenericThreads)
 layernorm_generic32_kernel(const float* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
                            float* __restrict__ y, int64_t rows, int64_t D, float inv_D, float eps) {
     constexpr int T = kLnGenericThreads;
-    __shared__ float slots[2 * kWarp];
+    __shared__ float slots[3 * kWarp];
     for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
         const float* xr = x + row * D;
         float* yr = y + row * D;
@@ -780,14 +843,17 @@ layernorm_generic32_kernel(const float* __restrict__ x, const float* __restrict_
         float s1 = 0.0f;
         for (int64_t j = threadIdx.x; j < D; j += T) s1 += xr[j] - K;
         s1 = cta_sum<T>(s1, slots, 0);
-        const float mu = fmaf(s1, inv_D, K);
-        float s2 = 0.0f;
+        float mu = fmaf(s1, inv_D, K), var;
+        float r2 = 0.0f, s2 = 0.0f;   // the second pass also sums x - mu, see refine_stats
         for (int64_t j = threadIdx.x; j < D; j += T) {
             const float d = xr[j] - mu;
+            r2 += d;
             s2 = fmaf(d, d, s2);
         }
-        s2 = cta_sum<T>(s2, slots, 1);
-        const float rstd = rsqrtf(fmaf(s2, inv_D, eps));
+        r2 = cta_sum<T>(r2, slots, 1);
+        s2 = cta_sum<T>(s2, slots, 2);
+        refine_stats(r2, s2, inv_D, mu, var);
+        const float rstd = rsqrtf(var + eps);
         for (int64_t j = threadIdx.x; j < D; j += T) yr[j] = fmaf((xr[j] - mu) * rstd, __ldg(gamma + j), __ldg(beta + j));
     }
 }

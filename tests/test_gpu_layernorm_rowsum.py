@@ -156,6 +156,32 @@ def test_layernorm_unaligned_rows_with_the_shift_table(rows, D, xo, few):
                      f"layernorm {rows}x{D} offset {xo} (shift table, new parameters)")
 
 
+@pytest.mark.parametrize("rows,D", [(72, 4096), (72, 8192), (70, 32768), (72, 65536), (80, 40000), (66, 131080),
+                                    (65, 128256), (70, 262144), (68, 36872), (66, 8190), (66, 65539), (65, 100001)])
+def test_layernorm_far_shift_constant_and_offset_rows(rows, D):
+    """The one-sweep moments are shifted by the mean of the row's first 16 bytes.  Every fourth
+    row here has a huge first entry, so that shift lands far from the mean and the second sweep
+    (shifted by the first mean estimate) runs; others are constant (output exactly beta) or sit at
+    an offset of 1024 with a spread of 8.  More than 64 rows, so long rows take the many-row
+    cluster layouts; every path that accepts the shape is run."""
+    x, g, b = synth.layernorm_inputs(rows, D, synth.case_seed(23, rows * 131 + D))
+    x[1::4, 0] = 65024.0
+    x[2::8] = 3.5
+    x[3::8] = (1024.0 + 8.0 * torch.randint(0, 4, x[3::8].shape, generator=torch.Generator().manual_seed(5))).to(x.dtype)
+    xb, gb, bb = synth.to_bits(x), synth.to_bits(g), synth.to_bits(b)
+    ref = oracle.layernorm(xb, gb, bb, EPS)
+    xd, gd, bd = x.to(DEV), g.to(DEV), b.to(DEV)
+    for path in [ak.AK_PATH_AUTO] + _legal_paths(D):
+        y, check = guarded((rows, D), torch.bfloat16, DEV)
+        ak.ak_layernorm_fwd(xd, gd, bd, y, eps=EPS, path=path)
+        torch.cuda.synchronize()
+        check()
+        _assert_ln_close(y, ref, xb, gb, bb, f"layernorm {rows}x{D} path {path}")
+        # a constant row has zero deviation: the output is beta, bit for bit
+        assert torch.equal(y[2::8].view(torch.int16).cpu(), b.view(torch.int16)[None, :].expand(len(range(2, rows, 8)), D))
+    assert ak.ak_wait_timeouts() == 0
+
+
 def test_layernorm_in_place_and_empty():
     for D, paths in ((512, _legal_paths(512)), (4096, _legal_paths(4096)), (4099, _legal_paths(4099)),
                      (16384, _legal_paths(16384)), (131072, _legal_paths(131072))):
