@@ -202,7 +202,9 @@ int ak_choose_path_dt(int op, int64_t rows, int64_t D, int aligned16, int dtype)
  * first element) had cost it.  The other layouts take sum((x - K)^2) in the first sweep and use
  * var = mean((x - K)^2) - (mu - K)^2 when (mu - K)^2 <= var (the subtraction then costs at
  * most a factor three in the relative error of var); otherwise they make that second pass
- * too.  eps finite, >= 0.
+ * too.  With fp32 elements (ak_layernorm_fwd_dt) the mean is kept as a sum of two floats and
+ * the output subtracts them one after the other, so a mean far above the spread (1024 +- 8)
+ * costs no accuracy either.  eps finite, >= 0.
  * Same path ids, size limits and alignment rules as RMSNorm (gamma and beta together play
  * the part of w).  Status codes as for RMSNorm.  One launch and no scratch, except for many
  * rows that are not 16-byte aligned (1024 or more of D <= about 32750, 256 or more longer ones

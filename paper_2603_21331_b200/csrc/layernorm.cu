@@ -24,11 +24,11 @@ int launch_reg(const void* x, const void* g, const void* b, void* y, int64_t row
     const int64_t grid = (rows + GROUPS - 1) / GROUPS;
     auto kernel = layernorm_reg_kernel<THREADS, GROUP, VPT, MINB, DT, PE>;
     // Every thread holds exactly VPT vectors: the form without bounds tests.  Its output phase may
-    // fetch gamma and beta several vectors ahead, which at 4 and 8 vectors per thread needs a few
-    // registers more than MINB CTAs per SM leave: one CTA fewer there (measured faster: 8192 x 8192
+    // fetch gamma and beta several vectors ahead, which at 4 and 8 vectors per thread (fp32: 6 and 7 too)
+    // needs a few registers more than MINB CTAs per SM leave: one CTA fewer there (measured faster: 8192 x 8192
     // 45.5 -> 41.9 us), and bounds-tested output for the 512-thread shape, which has no CTA to give.
     if constexpr (GROUPS == 1) {
-        constexpr bool tight = (VPT == 8 || VPT == 4) && !PE;
+        constexpr bool tight = (VPT == 8 || VPT == 4 || ((VPT == 6 || VPT == 7) && DT == AK_DTYPE_F32)) && !PE;
         constexpr bool ahead = !(tight && THREADS == 512);
         constexpr int minb = (tight && THREADS < 512) ? MINB - 1 : MINB;
         if (nvec == VPT * GROUP) kernel = layernorm_reg_kernel<THREADS, GROUP, VPT, minb, DT, PE, true, ahead>;

@@ -82,18 +82,37 @@ __device__ __forceinline__ float head_mean(const uint4 v) {
 // Mean and variance from the one-sweep sums s = sum(x - K), q = sum((x - K)^2).  False when the
 // shift is so far from the mean (or something is not a number) that the subtraction
 // q/D - (s/D)^2 would lose accuracy: the caller then sweeps again with the shift mu (refine_stats).
-__device__ __forceinline__ bool sweep_stats(float s, float q, float inv_D, float K, float& mu, float& var) {
+template <int DT>
+__device__ __forceinline__ bool sweep_stats(float s, float q, float inv_D, float K, float& mu, float& mc,
+                                            float& var) {
     const float m = s * inv_D;   // mean - K
-    mu = K + m;
+    if constexpr (DT == AK_DTYPE_F32) {
+        mu = K;
+        mc = m;
+    } else {
+        mu = K + m;
+        mc = 0.0f;
+    }
     var = fmaf(q, inv_D, -(m * m));
     return m * m <= var;
 }
-// The second sweep of such a row is shifted by the first estimate of the mean: s and q are now
-// sums of x - mu and (x - mu)^2, what is left of the mean is tiny against the spread, and the
-// subtraction is harmless.  The mean gains the accuracy the far shift had cost it.
-__device__ __forceinline__ void refine_stats(float s, float q, float inv_D, float& mu, float& var) {
+// The second sweep of such a row is shifted by the first estimate of the mean (one float): s and
+// q are now sums of x - mu and (x - mu)^2, what is left of the mean is tiny against the spread,
+// and the subtraction is harmless.  16-bit element types add the residual to mu.  fp32 keeps the
+// mean in two parts, mu + mc with mc of the order of the spread at most, and its output subtracts
+// them one after the other: a mean far above the spread does not fit one float to the accuracy
+// of an fp32 result (1024 +- 8 would lose 1e-5 of it), while the rounding of a 16-bit output is
+// coarser than that.
+template <int DT>
+__device__ __forceinline__ float second_shift(float& mu, float mc) {   // the shift of the second sweep
+    if constexpr (DT == AK_DTYPE_F32) mu += mc;
+    return mu;
+}
+template <int DT>
+__device__ __forceinline__ void refine_stats(float s, float q, float inv_D, float& mu, float& mc, float& var) {
     const float m = s * inv_D;
-    mu += m;
+    if constexpr (DT == AK_DTYPE_F32) mc = m;
+    else mu += m;
     var = fmaxf(fmaf(q, inv_D, -(m * m)), 0.0f);
 }
 // the lane sums of packed accumulators, added over the CTA with one barrier (two sets of slots)
@@ -148,7 +167,7 @@ __device__ __forceinline__ float sqdev_v(const uint4& v, float c) {
     }
     return lo + hi;
 }
-// ((x - mu) * rstd) * gamma + beta per element, rounded once to the output type
+// ((x - mean) * rstd) * gamma + beta per element, rounded once to the output type; mean = mu + mc
 template <int DT>
 __device__ __forceinline__ uint32_t ln_out2(uint32_t x, uint32_t g, uint32_t b, float mu, f32x2 rstd2) {
     const f32x2 t = fma2(mul2(dev2<DT>(x, mu), rstd2), widen2_t<DT>(g), widen2_t<DT>(b));
@@ -157,23 +176,25 @@ __device__ __forceinline__ uint32_t ln_out2(uint32_t x, uint32_t g, uint32_t b, 
     return Elem<DT>::pack(lo, hi);
 }
 template <int DT>
-__device__ __forceinline__ uint4 ln_out_v(const uint4& x, const uint4& g, const uint4& b, float mu, float rstd) {
+__device__ __forceinline__ uint4 ln_out_v(const uint4& x, const uint4& g, const uint4& b, float mu, float mc, float rstd) {
     const f32x2 r2 = pack2(rstd, rstd);
     if constexpr (DT == AK_DTYPE_F32) {
-        const f32x2 m2 = pack2(mu, mu);
+        const f32x2 m2 = pack2(mu, mu), c2 = pack2(mc, mc);
         float o0, o1, o2, o3;
-        unpack2(fma2(mul2(sub2(pack2(__uint_as_float(x.x), __uint_as_float(x.y)), m2), r2),
+        unpack2(fma2(mul2(sub2(sub2(pack2(__uint_as_float(x.x), __uint_as_float(x.y)), m2), c2), r2),
                      pack2(__uint_as_float(g.x), __uint_as_float(g.y)), pack2(__uint_as_float(b.x), __uint_as_float(b.y))), o0, o1);
-        unpack2(fma2(mul2(sub2(pack2(__uint_as_float(x.z), __uint_as_float(x.w)), m2), r2),
+        unpack2(fma2(mul2(sub2(sub2(pack2(__uint_as_float(x.z), __uint_as_float(x.w)), m2), c2), r2),
                      pack2(__uint_as_float(g.z), __uint_as_float(g.w)), pack2(__uint_as_float(b.z), __uint_as_float(b.w))), o2, o3);
         return make_uint4(__float_as_uint(o0), __float_as_uint(o1), __float_as_uint(o2), __float_as_uint(o3));
     } else {
+        // 16-bit types: mu is the whole mean (see refine_stats)
         return make_uint4(ln_out2<DT>(x.x, g.x, b.x, mu, r2), ln_out2<DT>(x.y, g.y, b.y, mu, r2),
                           ln_out2<DT>(x.z, g.z, b.z, mu, r2), ln_out2<DT>(x.w, g.w, b.w, mu, r2));
     }
 }
 template <int DT>
-__device__ __forceinline__ float ln_out1(uint16_t x, uint16_t g, uint16_t b, float mu, float rstd) {
+__device__ __forceinline__ float ln_out1(uint16_t x, uint16_t g, uint16_t b, float mu, float mc, float rstd) {
+    (void)mc;   // 16-bit types only: mu is the whole mean
     return fmaf(sub_h<DT>(x, mu) * rstd, Elem<DT>::to_float(g), Elem<DT>::to_float(b));
 }
 // first element of a row (any element type), the shift K of the mean
@@ -263,7 +284,7 @@ layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamm
             const int i = t + k * GROUP;
             if (FULL || (live && i < nvec)) xv[k] = ld_stream(xr + i);
         }
-        float mu, var;
+        float mu, mc = 0.0f, var;
         if constexpr (SWEEP1) {
             f32x2 sp = pack2(0.0f, 0.0f), qp = sp;
 #pragma unroll
@@ -285,7 +306,8 @@ layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamm
                 s1 = warp_sum((lane < WARPS_PER_GROUP) ? s[lane] : 0.0f);
                 q1 = warp_sum((lane < WARPS_PER_GROUP) ? q[lane] : 0.0f);
             }
-            if (!sweep_stats(s1, q1, inv_D, K, mu, var)) {
+            if (!sweep_stats<DT>(s1, q1, inv_D, K, mu, mc, var)) {
+                second_shift<DT>(mu, mc);   // the second sweep is shifted by the first estimate of the mean
                 sp = pack2(0.0f, 0.0f);
                 qp = sp;
 #pragma unroll
@@ -304,7 +326,7 @@ layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamm
                 __syncthreads();
                 s1 = warp_sum((lane < WARPS_PER_GROUP) ? s[lane] : 0.0f);
                 q1 = warp_sum((lane < WARPS_PER_GROUP) ? q[lane] : 0.0f);
-                refine_stats(s1, q1, inv_D, mu, var);
+                refine_stats<DT>(s1, q1, inv_D, mu, mc, var);
             }
             par ^= 1;
         } else {
@@ -335,7 +357,7 @@ layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamm
                 s2 = warp_sum((lane < WARPS_PER_GROUP) ? s[lane] : 0.0f);
                 q2 = warp_sum((lane < WARPS_PER_GROUP) ? q[lane] : 0.0f);
             }
-            refine_stats(s2, q2, inv_D, mu, var);
+            refine_stats<DT>(s2, q2, inv_D, mu, mc, var);
         }
         const float rstd = rsqrtf(var + eps);
         // FULL: the row index is read again rather than kept in registers across the reductions
@@ -344,8 +366,8 @@ layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamm
         for (int k = 0; k < VPT; ++k) {
             const int i = t + k * GROUP;
             if ((FULL && (P_EARLY || AHEAD)) || (live && i < nvec)) {
-                if constexpr (P_EARLY) st_stream(yr + i, ln_out_v<DT>(xv[k], gv[k], bv[k], mu, rstd));
-                else st_stream(yr + i, ln_out_v<DT>(xv[k], __ldg(gamma + i), __ldg(beta + i), mu, rstd));
+                if constexpr (P_EARLY) st_stream(yr + i, ln_out_v<DT>(xv[k], gv[k], bv[k], mu, mc, rstd));
+                else st_stream(yr + i, ln_out_v<DT>(xv[k], __ldg(gamma + i), __ldg(beta + i), mu, mc, rstd));
             }
         }
         if constexpr (FULL) break;
@@ -381,21 +403,22 @@ layernorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gam
     f32x2 sp = pack2(0.0f, 0.0f), qp = sp;
 #pragma unroll 4
     for (int i = threadIdx.x; i < nvec; i += THREADS) moments_v<DT>(row[i], K, sp, qp);
-    float s1, q1, mu, var;
+    float s1, q1, mu, mc = 0.0f, var;
     cta_sum2<THREADS>(sp, qp, slots, s1, q1);
-    if (!sweep_stats(s1, q1, inv_D, K, mu, var)) {
+    if (!sweep_stats<DT>(s1, q1, inv_D, K, mu, mc, var)) {
+        second_shift<DT>(mu, mc);   // the second sweep is shifted by the first estimate of the mean
         sp = pack2(0.0f, 0.0f);
         qp = sp;
 #pragma unroll 4
         for (int i = threadIdx.x; i < nvec; i += THREADS) moments_v<DT>(row[i], mu, sp, qp);
         cta_sum2<THREADS>(sp, qp, slots + 2 * kWarp, s1, q1);
-        refine_stats(s1, q1, inv_D, mu, var);
+        refine_stats<DT>(s1, q1, inv_D, mu, mc, var);
     }
     const float rstd = rsqrtf(var + eps);
     uint4* yr = y + r * nvec;
 #pragma unroll 2
     for (int i = threadIdx.x; i < nvec; i += THREADS)
-        st_stream(yr + i, ln_out_v<DT>(row[i], __ldg(gamma + i), __ldg(beta + i), mu, rstd));
+        st_stream(yr + i, ln_out_v<DT>(row[i], __ldg(gamma + i), __ldg(beta + i), mu, mc, rstd));
 }
 
 // ------------------------------------------------------------------ rows split over a cluster
@@ -442,9 +465,10 @@ layernorm_cluster_kernel(const uint4* __restrict__ x, const uint4* __restrict__ 
         t1 += box1[i].x;
         tq += box1[i].y;
     }
-    float mu, var;
+    float mu, mc = 0.0f, var;
     // every CTA adds the same values in the same order, so the whole cluster takes the same branch
-    if (!sweep_stats(t1, tq, inv_D, K, mu, var)) {
+    if (!sweep_stats<DT>(t1, tq, inv_D, K, mu, mc, var)) {
+        second_shift<DT>(mu, mc);   // the second sweep is shifted by the first estimate of the mean
         sp = pack2(0.0f, 0.0f);
         qp = sp;
 #pragma unroll 4
@@ -457,7 +481,7 @@ layernorm_cluster_kernel(const uint4* __restrict__ x, const uint4* __restrict__ 
             t1 += box2[i].x;
             tq += box2[i].y;
         }
-        refine_stats(t1, tq, inv_D, mu, var);
+        refine_stats<DT>(t1, tq, inv_D, mu, mc, var);
     }
     const float rstd = rsqrtf(var + eps);
     uint4* yr = y + r * nvec + v0;
@@ -465,7 +489,7 @@ layernorm_cluster_kernel(const uint4* __restrict__ x, const uint4* __restrict__ 
     const uint4* br = beta + v0;
 #pragma unroll 2
     for (int i = threadIdx.x; i < nn; i += THREADS)
-        st_stream(yr + i, ln_out_v<DT>(row[i], __ldg(gr + i), __ldg(br + i), mu, rstd));
+        st_stream(yr + i, ln_out_v<DT>(row[i], __ldg(gr + i), __ldg(br + i), mu, mc, rstd));
 }
 
 // ------------------------------------------------------------------ rows of any length streamed by a cluster
@@ -505,9 +529,10 @@ layernorm_cluster_stream_kernel(const uint4* __restrict__ x, const uint4* __rest
         t1 += box1[i].x;
         tq += box1[i].y;
     }
-    float mu, var;
+    float mu, mc = 0.0f, var;
     // every CTA adds the same values in the same order, so the whole cluster takes the same branch
-    if (!sweep_stats(t1, tq, inv_D, K, mu, var)) {
+    if (!sweep_stats<DT>(t1, tq, inv_D, K, mu, mc, var)) {
+        second_shift<DT>(mu, mc);   // the second sweep is shifted by the first estimate of the mean
         sp = pack2(0.0f, 0.0f);
         qp = sp;
 #pragma unroll 8
@@ -520,14 +545,14 @@ layernorm_cluster_stream_kernel(const uint4* __restrict__ x, const uint4* __rest
             t1 += box2[i].x;
             tq += box2[i].y;
         }
-        refine_stats(t1, tq, inv_D, mu, var);
+        refine_stats<DT>(t1, tq, inv_D, mu, mc, var);
     }
     const float rstd = rsqrtf(var + eps);
     if (!ok) return;   // a wait that gave up (never expected): nothing is written
     uint4* yr = y + r * nvec;
 #pragma unroll 2
     for (int64_t i = v0 + threadIdx.x; i < v1; i += T)
-        st_stream(yr + i, ln_out_v<DT>(ld_stream(xr + i), __ldg(gamma + i), __ldg(beta + i), mu, rstd));
+        st_stream(yr + i, ln_out_v<DT>(ld_stream(xr + i), __ldg(gamma + i), __ldg(beta + i), mu, mc, rstd));
 }
 
 // ------------------------------------------------------------------ unaligned rows staged in shared memory
@@ -586,16 +611,17 @@ layernorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restric
     f32x2 sp = pack2(d0, 0.0f), qp = pack2(d0 * d0, 0.0f);
 #pragma unroll 4
     for (int k = k_lo + threadIdx.x; k < k_hi; k += T) moments_v<DT>(row[k], K, sp, qp);
-    float s1, q1, mu, var;
+    float s1, q1, mu, mc = 0.0f, var;
     cta_sum2<T>(sp, qp, slots, s1, q1);
-    if (!sweep_stats(s1, q1, inv_D, K, mu, var)) {
+    if (!sweep_stats<DT>(s1, q1, inv_D, K, mu, mc, var)) {
+        second_shift<DT>(mu, mc);   // the second sweep is shifted by the first estimate of the mean
         const float d1 = edge ? sub_h<DT>(row16[ek * 8 + (threadIdx.x & 7)], mu) : 0.0f;
         sp = pack2(d1, 0.0f);
         qp = pack2(d1 * d1, 0.0f);
 #pragma unroll 4
         for (int k = k_lo + threadIdx.x; k < k_hi; k += T) moments_v<DT>(row[k], mu, sp, qp);
         cta_sum2<T>(sp, qp, slots + 2 * kWarp, s1, q1);
-        refine_stats(s1, q1, inv_D, mu, var);
+        refine_stats<DT>(s1, q1, inv_D, mu, mc, var);
     }
     const float rstd = rsqrtf(var + eps);
     if constexpr (TAB) {
@@ -604,15 +630,15 @@ layernorm_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* __restric
         const uint4* bt = tab + (size_t)(8 + phase) * nvp;
 #pragma unroll 2
         for (int k = k_lo + threadIdx.x; k < k_hi; k += T)
-            st_stream(ya + k, ln_out_v<DT>(row[k], gt[k], bt[k], mu, rstd));
+            st_stream(ya + k, ln_out_v<DT>(row[k], gt[k], bt[k], mu, mc, rstd));
     } else {
         for (int k = k_lo + threadIdx.x; k < k_hi; k += T) {
             const int64_t j0 = (int64_t)k * 8 - phase;
-            st_stream(ya + k, ln_out_v<DT>(row[k], ln_load_shifted(gamma, j0), ln_load_shifted(beta, j0), mu, rstd));
+            st_stream(ya + k, ln_out_v<DT>(row[k], ln_load_shifted(gamma, j0), ln_load_shifted(beta, j0), mu, mc, rstd));
         }
     }
     if (edge)
-        yr[ej] = Elem<DT>::from_float(ln_out1<DT>(row16[ek * 8 + (threadIdx.x & 7)], __ldg(gamma + ej), __ldg(beta + ej), mu, rstd));
+        yr[ej] = Elem<DT>::from_float(ln_out1<DT>(row16[ek * 8 + (threadIdx.x & 7)], __ldg(gamma + ej), __ldg(beta + ej), mu, mc, rstd));
 }
 
 // ------------------------------------------------------------------ unaligned rows split over a cluster
@@ -682,9 +708,10 @@ layernorm_cluster_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* _
         t1 += box1[i].x;
         tq += box1[i].y;
     }
-    float mu, var;
+    float mu, mc = 0.0f, var;
     // every CTA adds the same values in the same order, so the whole cluster takes the same branch
-    if (!sweep_stats(t1, tq, inv_D, K, mu, var)) {
+    if (!sweep_stats<DT>(t1, tq, inv_D, K, mu, mc, var)) {
+        second_shift<DT>(mu, mc);   // the second sweep is shifted by the first estimate of the mean
         const float d1 = edge ? sub_h<DT>(xe, mu) : 0.0f;
         sp = pack2(d1, 0.0f);
         qp = pack2(d1 * d1, 0.0f);
@@ -698,7 +725,7 @@ layernorm_cluster_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* _
             t1 += box2[i].x;
             tq += box2[i].y;
         }
-        refine_stats(t1, tq, inv_D, mu, var);
+        refine_stats<DT>(t1, tq, inv_D, mu, mc, var);
     }
     const float rstd = rsqrtf(var + eps);
     if (!ok) return;
@@ -708,14 +735,14 @@ layernorm_cluster_stage_kernel(const uint16_t* __restrict__ x, const uint16_t* _
         const uint4* bt = tab + (size_t)(8 + phase) * nvp;
 #pragma unroll 2
         for (int k = i0 + threadIdx.x; k < i1; k += T)
-            st_stream(ya + k, ln_out_v<DT>(row[k - v0], gt[k], bt[k], mu, rstd));
+            st_stream(ya + k, ln_out_v<DT>(row[k - v0], gt[k], bt[k], mu, mc, rstd));
     } else {
         for (int k = i0 + threadIdx.x; k < i1; k += T) {
             const int64_t e0 = (int64_t)k * 8 - phase;
-            st_stream(ya + k, ln_out_v<DT>(row[k - v0], ln_load_shifted(gamma, e0), ln_load_shifted(beta, e0), mu, rstd));
+            st_stream(ya + k, ln_out_v<DT>(row[k - v0], ln_load_shifted(gamma, e0), ln_load_shifted(beta, e0), mu, mc, rstd));
         }
     }
-    if (edge) yr[ej] = Elem<DT>::from_float(ln_out1<DT>(xe, __ldg(gamma + ej), __ldg(beta + ej), mu, rstd));
+    if (edge) yr[ej] = Elem<DT>::from_float(ln_out1<DT>(xe, __ldg(gamma + ej), __ldg(beta + ej), mu, mc, rstd));
 }
 
 // ------------------------------------------------------------------ unaligned rows in registers
@@ -760,7 +787,7 @@ layernorm_regp_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict
     for (int i = 0; i < VPT; ++i)
         if (k_lo + (int)threadIdx.x + i * THREADS < k_hi) s1 += sumdev_v<DT>(xv[i], K);
     s1 = cta_sum<THREADS>(s1, slots, 0);
-    float mu = fmaf(s1, inv_D, K), var;
+    float mu = fmaf(s1, inv_D, K), mc = 0.0f, var;
     // the second pass also sums x - mu: what the first element as shift cost the mean (it may
     // be an outlier) is corrected, see refine_stats
     const float de = edge ? sub_h<DT>(xe, mu) : 0.0f;
@@ -770,7 +797,7 @@ layernorm_regp_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict
         if (k_lo + (int)threadIdx.x + i * THREADS < k_hi) moments_v<DT>(xv[i], mu, sp, qp);
     float s2, q2;
     cta_sum2<THREADS>(sp, qp, slots + kWarp, s2, q2);
-    refine_stats(s2, q2, inv_D, mu, var);
+    refine_stats<DT>(s2, q2, inv_D, mu, mc, var);
     const float rstd = rsqrtf(var + eps);
     if constexpr (TAB) {
         pdl_wait();   // the table is complete and visible; plain loads (cached in L1), not the read-only path
@@ -779,7 +806,7 @@ layernorm_regp_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict
 #pragma unroll
         for (int i = 0; i < VPT; ++i) {
             const int k = k_lo + threadIdx.x + i * THREADS;
-            if (k < k_hi) st_stream(ya + k, ln_out_v<DT>(xv[i], gt[k], bt[k], mu, rstd));
+            if (k < k_hi) st_stream(ya + k, ln_out_v<DT>(xv[i], gt[k], bt[k], mu, mc, rstd));
         }
     } else {
 #pragma unroll
@@ -787,11 +814,11 @@ layernorm_regp_kernel(const uint16_t* __restrict__ x, const uint16_t* __restrict
             const int k = k_lo + threadIdx.x + i * THREADS;
             if (k < k_hi) {
                 const int64_t j0 = (int64_t)k * 8 - phase;
-                st_stream(ya + k, ln_out_v<DT>(xv[i], ln_load_shifted(gamma, j0), ln_load_shifted(beta, j0), mu, rstd));
+                st_stream(ya + k, ln_out_v<DT>(xv[i], ln_load_shifted(gamma, j0), ln_load_shifted(beta, j0), mu, mc, rstd));
             }
         }
     }
-    if (edge) yr[ej] = Elem<DT>::from_float(ln_out1<DT>(xe, __ldg(gamma + ej), __ldg(beta + ej), mu, rstd));
+    if (edge) yr[ej] = Elem<DT>::from_float(ln_out1<DT>(xe, __ldg(gamma + ej), __ldg(beta + ej), mu, mc, rstd));
 }
 
 // ------------------------------------------------------------------ generic
@@ -814,7 +841,7 @@ layernorm_generic_kernel(const uint16_t* __restrict__ x, const uint16_t* __restr
         float s1 = 0.0f;
         for (int64_t j = threadIdx.x; j < D; j += T) s1 += sub_h<DT>(xr[j], K);
         s1 = cta_sum<T>(s1, slots, 0);
-        float mu = fmaf(s1, inv_D, K), var;
+        float mu = fmaf(s1, inv_D, K), mc = 0.0f, var;
         float r2 = 0.0f, s2 = 0.0f;   // the second pass also sums x - mu, see refine_stats
         for (int64_t j = threadIdx.x; j < D; j += T) {
             const float d = sub_h<DT>(xr[j], mu);
@@ -823,10 +850,10 @@ layernorm_generic_kernel(const uint16_t* __restrict__ x, const uint16_t* __restr
         }
         r2 = cta_sum<T>(r2, slots, 1);
         s2 = cta_sum<T>(s2, slots, 2);
-        refine_stats(r2, s2, inv_D, mu, var);
+        refine_stats<DT>(r2, s2, inv_D, mu, mc, var);
         const float rstd = rsqrtf(var + eps);
         for (int64_t j = threadIdx.x; j < D; j += T)
-            yr[j] = Elem<DT>::from_float(ln_out1<DT>(xr[j], __ldg(gamma + j), __ldg(beta + j), mu, rstd));
+            yr[j] = Elem<DT>::from_float(ln_out1<DT>(xr[j], __ldg(gamma + j), __ldg(beta + j), mu, mc, rstd));
     }
 }
 
@@ -843,7 +870,7 @@ layernorm_generic32_kernel(const float* __restrict__ x, const float* __restrict_
         float s1 = 0.0f;
         for (int64_t j = threadIdx.x; j < D; j += T) s1 += xr[j] - K;
         s1 = cta_sum<T>(s1, slots, 0);
-        float mu = fmaf(s1, inv_D, K), var;
+        float mu = fmaf(s1, inv_D, K), mc = 0.0f, var;
         float r2 = 0.0f, s2 = 0.0f;   // the second pass also sums x - mu, see refine_stats
         for (int64_t j = threadIdx.x; j < D; j += T) {
             const float d = xr[j] - mu;
@@ -852,9 +879,9 @@ layernorm_generic32_kernel(const float* __restrict__ x, const float* __restrict_
         }
         r2 = cta_sum<T>(r2, slots, 1);
         s2 = cta_sum<T>(s2, slots, 2);
-        refine_stats(r2, s2, inv_D, mu, var);
+        refine_stats<AK_DTYPE_F32>(r2, s2, inv_D, mu, mc, var);
         const float rstd = rsqrtf(var + eps);
-        for (int64_t j = threadIdx.x; j < D; j += T) yr[j] = fmaf((xr[j] - mu) * rstd, __ldg(gamma + j), __ldg(beta + j));
+        for (int64_t j = threadIdx.x; j < D; j += T) yr[j] = fmaf(((xr[j] - mu) - mc) * rstd, __ldg(gamma + j), __ldg(beta + j));
     }
 }
 

@@ -251,6 +251,28 @@ def test_layernorm_dt_parity_all_paths(rows, D, dtype):
 
 
 @pytest.mark.parametrize("dtype", DTS)
+@pytest.mark.parametrize("rows,D", [(72, 1024), (72, 4096), (70, 16384), (72, 65536), (66, 40008), (65, 131076), (66, 4099)])
+def test_layernorm_dt_far_shift_constant_and_offset_rows(rows, D, dtype):
+    """fp16 / fp32 counterpart of the bf16 test of the same name: rows whose first entry is an
+    outlier (the shift of the moments lands far from the mean, so the second sweep runs), constant
+    rows (output exactly beta) and rows at an offset of 1024 with a spread of 8, on every path."""
+    x, g, b = synth.layernorm_inputs(rows, D, synth.case_seed(29, rows * 131 + D), dtype=dtype)
+    x[1::4, 0] = 60000.0
+    x[2::8] = 3.5
+    x[3::8] = (1024.0 + 8.0 * torch.randint(0, 4, x[3::8].shape, generator=torch.Generator().manual_seed(5))).to(dtype)
+    ref = oracle.layernorm_dt(synth.to_elems(x), synth.to_elems(g), synth.to_elems(b), 1e-5, NAME[dtype])
+    xd, gd, bd = x.to(DEV), g.to(DEV), b.to(DEV)
+    for path in [ak.AK_PATH_AUTO] + _legal_paths(D, dtype):
+        y, check = guarded((rows, D), dtype, DEV)
+        ak.ak_layernorm_fwd_dt(xd, gd, bd, y, eps=1e-5, path=path)
+        torch.cuda.synchronize()
+        check()
+        _assert_ln_close_dt(y, ref, b, f"layernorm {NAME[dtype]} {rows}x{D} path {path}")
+        assert torch.equal(y[2::8].cpu(), b[None, :].expand(len(range(2, rows, 8)), D))
+    assert ak.ak_wait_timeouts() == 0
+
+
+@pytest.mark.parametrize("dtype", DTS)
 @pytest.mark.parametrize("rows,D", SHAPES + [(1000, 128), (300, 1025), (5, 4), (7, 13)])
 def test_rowsum_dt_parity_and_exact_integers(rows, D, dtype):
     x, _, _ = synth.layernorm_inputs(rows, D, synth.case_seed(20, rows * 131 + D), dtype=dtype)
