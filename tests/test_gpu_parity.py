@@ -1,5 +1,7 @@
 """GPU parity: every CUDA path against the fp64 CPU checker, element by element, on the
 same seeded bf16 bit patterns, through the C ABI (ctypes binding)."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -11,6 +13,15 @@ from parity import assert_bf16_close, assert_loss_close, guarded
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
+
+
+def _needs_clusters():
+    """Tests of what the dispatcher sends to thread-block clusters do not apply when the library's
+    diagnostic switch AK_DISABLE_CLUSTERS keeps every row on one CTA."""
+    if os.environ.get("AK_DISABLE_CLUSTERS", "0") not in ("", "0"):
+        pytest.skip("the cluster layouts are switched off in this environment")
+
+
 WARP, CTA, GEN, SMEM = ak.AK_PATH_WARP, ak.AK_PATH_CTA, ak.AK_PATH_GENERIC, ak.AK_PATH_SMEM
 CLUSTER = ak.AK_PATH_CLUSTER
 
@@ -400,6 +411,7 @@ def test_cluster_path_slices_and_limits(rows, D):
     the cluster size), the shortest legal rows (two vectors), rows far beyond one CTA's shared
     memory up to the 8 x 224 KiB limit, and both sides of the few-rows rule.  All three ops, forced
     and as the dispatcher's own choice; -inf and identical-value rows included."""
+    _needs_clusters()
     x, w = synth.rmsnorm_inputs(rows, D, synth.case_seed(9, rows * 131 + D))
     if rows > 1:
         x[0, : D // 2] = float("-inf")      # whole slices of -inf (softmax); replaced by -3 for the norms
@@ -531,6 +543,7 @@ def test_unaligned_rows_split_over_a_cluster(rows, D, xo):
 def test_layernorm_unaligned_cluster_with_the_shift_table():
     """Enough long unaligned rows for both the cluster layout and the table of shifted parameters
     (two launches: the table kernel, then the cluster kernel as its programmatic dependent)."""
+    _needs_clusters()
     rows, D = 300, 114700
     x, g, b = synth.layernorm_inputs(rows, D, synth.case_seed(14, D), device=DEV)
     n0 = ak.ak_launch_count()
