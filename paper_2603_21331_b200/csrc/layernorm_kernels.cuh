@@ -428,8 +428,11 @@ layernorm_smem_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gam
 // x - K (K = the row's first element, read by every CTA) and then of (x - mu)^2 meet through
 // distributed shared memory and are added in rank order in every CTA.  grid = rows * C,
 // cluster = C.  Dynamic shared memory = ceil(nvec / C) * 16 bytes.
+// Register cap: six CTAs of 256 threads per SM (40 registers; 32 KiB slices let shared memory hold
+// seven).  Occupancy is what this kernel lives on: five CTAs (48 registers, the compiler's choice
+// when asked for two) measured 1.5-3 % slower, seven (32 registers, spills) 9 % slower.
 template <int THREADS, int DT = AK_DTYPE_BF16>
-__global__ void __launch_bounds__(THREADS, 2)
+__global__ void __launch_bounds__(THREADS, THREADS <= 256 ? 6 : 2)
 layernorm_cluster_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamma, const uint4* __restrict__ beta,
                          uint4* __restrict__ y, int nvec, int C, float inv_D, float eps) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
