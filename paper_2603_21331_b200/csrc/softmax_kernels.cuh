@@ -52,6 +52,54 @@ __device__ __forceinline__ f32x2 exp_of_pair(f32x2 x2, f32x2 l2, f32x2 nm2) {
     unpack2(fma2(x2, l2, nm2), t0, t1);
     return pack2(fast_exp2(t0), fast_exp2(t1));
 }
+// The same on the FMA pipe: t = x*log2e - m2 <= 0 is clamped at -160, rounded to the nearest
+// integer n (the 1.5 * 2^23 trick), 2^(t - n) comes from a degree-4 minimax polynomial on
+// [-0.5, 0.5] (relative error 2.7e-6, far below the rounding of a 16-bit output), and n goes into
+// the exponent field.  Below the normal range the result is zero (the signed maximum with zero
+// catches the exponent field running negative: every t < -127.5) or, in the one binade under
+// 2^-126, a subnormal within 2^-126 of the true value; `ex2.approx.ftz` gives zero there.
+__device__ __forceinline__ f32x2 exp_of_pair_poly(f32x2 x2, f32x2 l2, f32x2 nm2) {
+    float t0, t1;
+    unpack2(fma2(x2, l2, nm2), t0, t1);
+    const f32x2 tc = pack2(fmaxf(t0, -160.0f), fmaxf(t1, -160.0f));
+    const f32x2 magic = pack2(12582912.0f, 12582912.0f);
+    const f32x2 z = add2(tc, magic);
+    const f32x2 n = sub2(z, magic);
+    const f32x2 f = sub2(tc, n);
+    f32x2 p = pack2(0.009570079855620861f, 0.009570079855620861f);
+    p = fma2(p, f, pack2(0.05591783672571182f, 0.05591783672571182f));
+    p = fma2(p, f, pack2(0.240247443318367f, 0.240247443318367f));
+    p = fma2(p, f, pack2(0.6931217908859253f, 0.6931217908859253f));
+    p = fma2(p, f, pack2(0.9999992847442627f, 0.9999992847442627f));
+    float p0, p1, z0, z1;
+    unpack2(p, p0, p1);
+    unpack2(z, z0, z1);
+    p0 = __int_as_float(max(__float_as_int(p0) + (__float_as_int(z0) << 23), 0));
+    p1 = __int_as_float(max(__float_as_int(p1) + (__float_as_int(z1) << 23), 0));
+    return pack2(p0, p1);
+}
+// pairs per recomputed vector that the aligned cluster kernel evaluates on the FMA pipe (the unaligned
+// one, which is not bound by the transcendental pipe, gained nothing from it)
+template <int DT> constexpr int kClusterPolyPairs = DT == AK_DTYPE_F32 ? 0 : 1;
+// exp_v with the first NP of the four pairs of a 16-bit vector on the FMA pipe (NP = 0: exp_v)
+template <int DT, int NP>
+__device__ __forceinline__ float exp_v_mix(const uint4& v, float m2, f32x2* e) {
+    static_assert(DT != AK_DTYPE_F32 || NP == 0, "the polynomial is for 16-bit outputs");
+    const f32x2 l2 = pack2(kLog2e, kLog2e), nm2 = pack2(-m2, -m2);
+    float lo, hi;
+    if constexpr (DT == AK_DTYPE_F32) {
+        e[0] = exp_of_pair(pack2(__uint_as_float(v.x), __uint_as_float(v.y)), l2, nm2);
+        e[1] = exp_of_pair(pack2(__uint_as_float(v.z), __uint_as_float(v.w)), l2, nm2);
+        unpack2(add2(e[0], e[1]), lo, hi);
+    } else {
+        e[0] = NP > 0 ? exp_of_pair_poly(widen2_t<DT>(v.x), l2, nm2) : exp_of_pair(widen2_t<DT>(v.x), l2, nm2);
+        e[1] = NP > 1 ? exp_of_pair_poly(widen2_t<DT>(v.y), l2, nm2) : exp_of_pair(widen2_t<DT>(v.y), l2, nm2);
+        e[2] = NP > 2 ? exp_of_pair_poly(widen2_t<DT>(v.z), l2, nm2) : exp_of_pair(widen2_t<DT>(v.z), l2, nm2);
+        e[3] = NP > 3 ? exp_of_pair_poly(widen2_t<DT>(v.w), l2, nm2) : exp_of_pair(widen2_t<DT>(v.w), l2, nm2);
+        unpack2(add2(add2(e[0], e[1]), add2(e[2], e[3])), lo, hi);
+    }
+    return lo + hi;
+}
 template <int DT>
 __device__ __forceinline__ float exp_v(const uint4& v, float m2, f32x2* e) {
     const f32x2 l2 = pack2(kLog2e, kLog2e), nm2 = pack2(-m2, -m2);
@@ -268,8 +316,12 @@ softmax_cluster_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int n
         const int i = threadIdx.x + k * THREADS;
         if (i < nn) sum += exp_v<DT>(row[i], m2, kept[k]);
     }
+    // The vectors that are not kept are evaluated twice, which makes the transcendental pipe the
+    // busiest unit of this kernel (63 % of its peak over the whole kernel); one of their four pairs
+    // goes to the FMA pipe instead (4096 x 65536: 168.6 -> 165.5 us; two pairs: 171.0 us).
+    constexpr int NP = kClusterPolyPairs<DT>;
 #pragma unroll 2
-    for (int i = threadIdx.x + KEEP * THREADS; i < nn; i += THREADS) sum += exp_v<DT>(row[i], m2, e);
+    for (int i = threadIdx.x + KEEP * THREADS; i < nn; i += THREADS) sum += exp_v_mix<DT, NP>(row[i], m2, e);
     sum = cta_sum<THREADS>(sum, slots, 1);
     if (!mailbox_exchange(sum, box_s, &xbar_s, C, c)) nn = 0;
     float tot = 0.0f;
@@ -284,7 +336,7 @@ softmax_cluster_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int n
     }
 #pragma unroll 2
     for (int i = threadIdx.x + KEEP * THREADS; i < nn; i += THREADS) {
-        exp_v<DT>(row[i], m2, e);
+        exp_v_mix<DT, NP>(row[i], m2, e);
         st_stream(yr + i, norm_v<DT>(e, inv));
     }
 }
