@@ -207,7 +207,7 @@ int ak_choose_path_dt(int op, int64_t rows, int64_t D, int aligned16, int dtype)
  * costs no accuracy either.  eps finite, >= 0.
  * Same path ids, size limits and alignment rules as RMSNorm (gamma and beta together play
  * the part of w).  Status codes as for RMSNorm.  One launch and no scratch, except for many
- * rows that are not 16-byte aligned (1024 or more of D <= about 32750, 256 or more longer ones
+ * rows that are not 16-byte aligned (1024 or more of D <= about 4090, 256 or more longer ones
  * up to 1792 KiB): then a small kernel first writes gamma and beta in all eight 2-byte shifts to
  * about 32 * D bytes of stream-ordered scratch obtained and released on `cuda_stream`, and
  * the row kernel runs as its programmatic dependent; if the scratch cannot be had the

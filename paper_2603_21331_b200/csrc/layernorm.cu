@@ -165,20 +165,16 @@ int launch_regp(const uint16_t* x, const uint16_t* g, const uint16_t* b, uint16_
     count_launch();
     return cudaGetLastError() == cudaSuccess ? AK_OK : AK_ERR_CUDA;
 }
-// unaligned rows held in registers: vectors per thread 1..8 for a CTA of THREADS threads
-// (register caps: M15 for 1..5 vectors, M68 for 6..8)
-template <int DT, int THREADS, int M15, int M68>
+// unaligned rows held in registers: one to four vectors per thread of a CTA of THREADS threads
+// (MINB: the minimum-CTAs-per-SM hint, a register cap)
+template <int DT, int THREADS, int MINB>
 int launch_regp_vpt(int vpt, const uint16_t* x, const uint16_t* g, const uint16_t* b, uint16_t* y, int64_t rows,
                     int64_t D, float inv_D, float eps, cudaStream_t st) {
     switch (vpt) {
-        case 1: return launch_regp<DT, THREADS, 1, M15>(x, g, b, y, rows, D, inv_D, eps, st);
-        case 2: return launch_regp<DT, THREADS, 2, M15>(x, g, b, y, rows, D, inv_D, eps, st);
-        case 3: return launch_regp<DT, THREADS, 3, M15>(x, g, b, y, rows, D, inv_D, eps, st);
-        case 4: return launch_regp<DT, THREADS, 4, M15>(x, g, b, y, rows, D, inv_D, eps, st);
-        case 5: return launch_regp<DT, THREADS, 5, M15>(x, g, b, y, rows, D, inv_D, eps, st);
-        case 6: return launch_regp<DT, THREADS, 6, M68>(x, g, b, y, rows, D, inv_D, eps, st);
-        case 7: return launch_regp<DT, THREADS, 7, M68>(x, g, b, y, rows, D, inv_D, eps, st);
-        case 8: return launch_regp<DT, THREADS, 8, M68>(x, g, b, y, rows, D, inv_D, eps, st);
+        case 1: return launch_regp<DT, THREADS, 1, MINB>(x, g, b, y, rows, D, inv_D, eps, st);
+        case 2: return launch_regp<DT, THREADS, 2, MINB>(x, g, b, y, rows, D, inv_D, eps, st);
+        case 3: return launch_regp<DT, THREADS, 3, MINB>(x, g, b, y, rows, D, inv_D, eps, st);
+        case 4: return launch_regp<DT, THREADS, 4, MINB>(x, g, b, y, rows, D, inv_D, eps, st);
         default: return AK_ERR_SHAPE;
     }
 }
@@ -267,7 +263,6 @@ int dispatch_t(const void* x, const void* gamma, const void* beta, void* y, int6
                 const uint16_t* gs = static_cast<const uint16_t*>(gamma);
                 const uint16_t* bs = static_cast<const uint16_t*>(beta);
                 uint16_t* ys = static_cast<uint16_t*>(y);
-                // rows of up to 1024 covering vectors stay in the registers of a 128-thread CTA ...
                 const int64_t max_nv = (D + 14) >> 3;   // vectors covering the row at the worst phase
                 // long rows (up to eight CTAs' shared memory), and a few rows (at most 64) of 32 KiB or
                 // more: the covering vectors split over a thread-block cluster;
@@ -278,12 +273,12 @@ int dispatch_t(const void* x, const void* gamma, const void* beta, void* y, int6
                     if (launch_cluster_stage<DT, 256>(xs, gs, bs, ys, rows, D, max_nv, Cu, inv_D, eps, st) == AK_OK) return AK_OK;
                     (void)cudaGetLastError();   // the cluster cannot be co-scheduled here: the kernels below
                 }
-                if (same_phase && params4 && max_nv <= 1024)
-                    return launch_regp_vpt<DT, 128, 10, 6>((int)((max_nv + 127) / 128), xs, gs, bs, ys, rows, D, inv_D, eps, st);
-                // ... and of a 512-thread CTA from 3073 to 4096 (in between, the staged kernel below
-                // measured 0-10 % faster than 256 or 512 threads holding the row)
-                if (same_phase && params4 && max_nv > 3072 && max_nv <= 4096)
-                    return launch_regp_vpt<DT, 512, 2, 2>((int)((max_nv + 511) / 512), xs, gs, bs, ys, rows, D, inv_D, eps, st);
+                // Rows of up to 512 covering vectors (D <= about 4090) stay in the registers of a 128-thread
+                // CTA; longer ones are staged in shared memory: with both moments taken in one pass over the
+                // staged row that kernel is the faster one from there on (8192 x 4099 28.3 -> 27.2 us, 8192 x 7001
+                // 48.3 -> 45.0 us, 4096 x 28001 96.7 -> 87.2 us against rows held by 128 or 512 threads).
+                if (same_phase && params4 && max_nv <= 512)
+                    return launch_regp_vpt<DT, 128, 10>((int)((max_nv + 127) / 128), xs, gs, bs, ys, rows, D, inv_D, eps, st);
                 if (same_phase && params4 && stage_bytes <= (size_t)kMaxRowSmemBytes) {
                     if (D <= 8192) return launch_stage<DT, 128>(xs, gs, bs, ys, rows, D, stage_bytes, inv_D, eps, st);
                     if (D <= 32768) return launch_stage<DT, 256>(xs, gs, bs, ys, rows, D, stage_bytes, inv_D, eps, st);

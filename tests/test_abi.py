@@ -213,22 +213,23 @@ def test_wait_timeout_flags_have_a_host_reader():
     assert ak.ak_wait_timeouts() in (-1, 0)
 
 
-def test_hot_kernels_compile_without_spills():
-    """The kernels the benchmark configurations run keep everything in registers: the compiler's
-    own report (written next to the library by its build) shows no spill stores or loads for
-    them.  Skipped when the library was built elsewhere and the report is not at hand."""
+def test_kernels_compile_without_spills():
+    """Every kernel of the library keeps everything in registers: the compiler's own report
+    (written next to the library by its build) shows no spill stores or loads for any entry
+    function.  Skipped when the library was built elsewhere and the report is not at hand."""
     log = os.path.join(ROOT, "paper_2603_21331_b200", "build", "ptxas.log")
     if not os.path.exists(log):
         pytest.skip("no compiler report beside the library")
     text = open(log).read()
     entries = re.findall(r"Compiling entry function '(\S+)' for 'sm_100a'\n.*?\n\s+(\d+) bytes stack frame, "
                          r"(\d+) bytes spill stores, (\d+) bytes spill loads", text)
-    hot = ("xent_row_kernel", "xent_split_kernel", "xent_finish_kernel", "xent_vp_partial_kernel",
-           "xent_vp_merge_kernel", "rmsnorm_reg_kernel", "softmax_reg_kernel", "softmax_smem_kernel",
-           "layernorm_reg_kernel", "rowsum_kernel", "rope_vec_kernel")
-    seen = 0
+    families = ("xent_row_kernel", "xent_split_kernel", "xent_finish_kernel", "xent_vp_partial_kernel",
+                "xent_vp_merge_kernel", "rmsnorm_reg_kernel", "softmax_reg_kernel", "softmax_smem_kernel",
+                "layernorm_reg_kernel", "rowsum_kernel", "rope_vec_kernel", "_cluster_kernel", "_stage_kernel",
+                "_regp_kernel")
+    seen = set()
     for name, _, stores, loads in entries:
-        if any(h in name for h in hot):
-            seen += 1
-            assert int(stores) == 0 and int(loads) == 0, f"{name} spills {stores} / {loads} bytes"
-    assert seen >= 100   # every instantiation of those families was looked at
+        assert int(stores) == 0 and int(loads) == 0, f"{name} spills {stores} / {loads} bytes"
+        seen.update(f for f in families if f in name)
+    assert seen == set(families), f"families missing from the report: {set(families) - seen}"
+    assert len(entries) >= 300   # every instantiation was looked at

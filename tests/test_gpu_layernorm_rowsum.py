@@ -117,11 +117,12 @@ def test_layernorm_misaligned_base_pointers():
             assert bool((ybuf[:yo] == 0).all()) and bool((ybuf[yo + rows * D:] == 0).all())
 
 
-@pytest.mark.parametrize("rows,D,xo,few", [(1024, 1027, 0, 1000), (1500, 4099, 0, 1000), (1100, 2051, 3, 1000),
-                                           (1024, 8190, 1, 200), (1030, 16379, 0, 255), (1025, 32754, 5, 1000),
-                                           (256, 32771, 0, 200), (300, 40001, 3, 255), (260, 65539, 1, 100)])
+@pytest.mark.parametrize("rows,D,xo,few", [(1024, 1027, 0, 1000), (1500, 4001, 0, 1000), (1100, 2051, 3, 1000),
+                                           (1500, 4099, 0, 200), (1024, 8190, 1, 200), (1030, 16379, 0, 255),
+                                           (1025, 32754, 5, 250), (256, 32771, 0, 200), (300, 40001, 3, 255),
+                                           (260, 65539, 1, 100)])
 def test_layernorm_unaligned_rows_with_the_shift_table(rows, D, xo, few):
-    """From 1024 rows on (256 for rows staged in shared memory), unaligned rows read gamma and beta
+    """From 1024 rows on (256 for rows staged in shared memory: D of about 4090 and more), unaligned rows read gamma and beta
     from a table of all eight shifts written by a small kernel in front.  Parity on such launches,
     and the same bits as the launch without the table (fewer rows) gives for the rows they share."""
     x, g, b = synth.layernorm_inputs(rows, D, synth.case_seed(8, rows + D))
