@@ -36,6 +36,10 @@ int launch_reg(const void* x, const void* w, void* y, int64_t rows, int nvec, fl
     constexpr int GROUPS = THREADS / GROUP;
     const int64_t grid = (rows + GROUPS - 1) / GROUPS;
     auto kernel = rmsnorm_reg_kernel<THREADS, GROUP, VPT, MINB, WE, DT>;
+    // every thread holds exactly VPT vectors of a live row: the form without bounds tests (the loads
+    // of x and w are then issued without waiting for predicates: 8192 x 2048 13.3 -> 11.7 us,
+    // 8192 x 8192 41.1 -> 40.6 us)
+    if (nvec == VPT * GROUP && rows % GROUPS == 0) kernel = rmsnorm_reg_kernel<THREADS, GROUP, VPT, MINB, WE, DT, true>;
     const cudaError_t e = launch_dependent(kernel, dim3((unsigned)grid), dim3(THREADS), 0, st,
                                            static_cast<const uint4*>(x), static_cast<const uint4*>(w),
                                            static_cast<uint4*>(y), rows, nvec, inv_D, eps,

@@ -75,8 +75,9 @@ __device__ __forceinline__ uint4 scale_v(const uint4& x, const uint4& w, float r
 // either before the reduction (W_EARLY: latency hidden behind the row loads, 4 * VPT more
 // live registers) or after it.  MINB is the launch-bounds occupancy hint that caps the
 // register count.  The grid may be smaller than the number of row slots: groups then walk
-// the rows with a grid stride.
-template <int THREADS, int GROUP, int VPT, int MINB, bool W_EARLY, int DT = AK_DTYPE_BF16>
+// the rows with a grid stride.  FULL: nvec == VPT * GROUP, the rows fill the CTAs' groups exactly
+// and the grid has one CTA per group of rows, so nothing tests a bound and the body runs once.
+template <int THREADS, int GROUP, int VPT, int MINB, bool W_EARLY, int DT = AK_DTYPE_BF16, bool FULL = false>
 __global__ void __launch_bounds__(THREADS, MINB)
 rmsnorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w, uint4* __restrict__ y,
                    int64_t rows, int nvec, float inv_D, float eps, int first_wave) {
@@ -99,21 +100,21 @@ rmsnorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w, uin
 #pragma unroll
         for (int k = 0; k < VPT; ++k) {
             const int i = t + k * GROUP;
-            wv[k] = (i < nvec) ? __ldg(w + i) : make_uint4(0, 0, 0, 0);
+            wv[k] = (FULL || i < nvec) ? __ldg(w + i) : make_uint4(0, 0, 0, 0);
         }
     }
     int phase = 0;
     // Whole CTAs iterate together (rows beyond the end are masked, not skipped) so the
     // barrier below is reached by every thread.
-    for (int64_t row0 = (int64_t)blockIdx.x * GROUPS; row0 < rows; row0 += (int64_t)gridDim.x * GROUPS) {
+    for (int64_t row0 = (int64_t)blockIdx.x * GROUPS; FULL || row0 < rows; row0 += (int64_t)gridDim.x * GROUPS) {
         const int64_t row = row0 + g;
-        const bool live = row < rows;
+        const bool live = FULL || row < rows;
         const uint4* xr = x + row * nvec;
         uint4 xv[VPT];
 #pragma unroll
         for (int k = 0; k < VPT; ++k) {
             const int i = t + k * GROUP;
-            xv[k] = (live && i < nvec) ? ld_stream(xr + i) : make_uint4(0, 0, 0, 0);
+            xv[k] = (FULL || (live && i < nvec)) ? ld_stream(xr + i) : make_uint4(0, 0, 0, 0);
         }
         float ss = 0.0f;
 #pragma unroll
@@ -132,11 +133,12 @@ rmsnorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ w, uin
 #pragma unroll
         for (int k = 0; k < VPT; ++k) {
             const int i = t + k * GROUP;
-            if (live && i < nvec) {
+            if (FULL || (live && i < nvec)) {
                 const uint4 wq = W_EARLY ? wv[k] : __ldg(w + i);
                 st_stream(yr + i, scale_v<DT>(xv[k], wq, rstd));
             }
         }
+        if constexpr (FULL) break;   // the grid has one CTA per group of rows
     }
 }
 

@@ -146,7 +146,7 @@ template <int DT> constexpr int kExpPairs = (DT == AK_DTYPE_F32) ? 2 : 4;
 // each is evaluated once; RECOMPUTE == true keeps only the packed inputs and evaluates the
 // exponentials a second time in the epilogue (half the registers, twice the SFU work) for
 // rows too long to hold in fp32.
-template <int THREADS, int GROUP, int VPT, int MINB, bool RECOMPUTE, int DT = AK_DTYPE_BF16>
+template <int THREADS, int GROUP, int VPT, int MINB, bool RECOMPUTE, int DT = AK_DTYPE_BF16, bool FULL = false>
 __global__ void __launch_bounds__(THREADS, MINB)
 softmax_reg_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t rows, int nvec, int first_wave) {
     constexpr int GROUPS = THREADS / GROUP;
@@ -163,15 +163,17 @@ softmax_reg_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t r
     const int lane = threadIdx.x & 31;
     const int warp_in_group = t >> 5;
 
-    for (int64_t row0 = (int64_t)blockIdx.x * GROUPS; row0 < rows; row0 += (int64_t)gridDim.x * GROUPS) {
+    // FULL: nvec == VPT * GROUP, the rows fill the groups exactly and the grid has one CTA per group of
+    // rows: nothing tests a bound and the body runs once
+    for (int64_t row0 = (int64_t)blockIdx.x * GROUPS; FULL || row0 < rows; row0 += (int64_t)gridDim.x * GROUPS) {
         const int64_t row = row0 + g;
-        const bool live = row < rows;
+        const bool live = FULL || row < rows;
         const uint4* xr = x + row * nvec;
         uint4 xv[VPT];
 #pragma unroll
         for (int k = 0; k < VPT; ++k) {
             const int i = t + k * GROUP;
-            xv[k] = (live && i < nvec) ? ld_stream(xr + i) : neg_inf_vec<DT>();
+            xv[k] = (FULL || (live && i < nvec)) ? ld_stream(xr + i) : neg_inf_vec<DT>();
         }
         uint32_t mx = neg_inf_word<DT>();
 #pragma unroll
@@ -201,8 +203,9 @@ softmax_reg_kernel(const uint4* __restrict__ x, uint4* __restrict__ y, int64_t r
         for (int k = 0; k < VPT; ++k) {
             const int i = t + k * GROUP;
             if constexpr (RECOMPUTE) exp_v<DT>(xv[k], m2, e[0]);
-            if (live && i < nvec) st_stream(yr + i, norm_v<DT>(e[RECOMPUTE ? 0 : k], inv));
+            if (FULL || (live && i < nvec)) st_stream(yr + i, norm_v<DT>(e[RECOMPUTE ? 0 : k], inv));
         }
+        if constexpr (FULL) break;
     }
 }
 
