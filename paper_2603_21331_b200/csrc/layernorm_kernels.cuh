@@ -222,8 +222,8 @@ __device__ __forceinline__ float first_elem(const void* row) {
 //
 // P_EARLY: gamma and beta are requested together with the row instead of after the reductions
 // (8 * VPT more live registers; for launches too small to fill the GPU, where latency counts).
-// FULL: every thread holds exactly VPT vectors of a live row (nvec == VPT * GROUP and one row
-// per CTA), so the loads and the sweep test no bounds; with AHEAD neither does the output phase,
+// FULL: every thread holds exactly VPT vectors of a live row (nvec == VPT * GROUP, the rows fill
+// the CTAs' groups, one CTA per group of rows), so the loads and the sweep test no bounds; with AHEAD neither does the output phase,
 // which lets the compiler fetch gamma and beta several vectors ahead (at the cost of registers).
 template <int THREADS, int GROUP, int VPT, int MINB, int DT = AK_DTYPE_BF16, bool P_EARLY = false, bool FULL = false,
           bool AHEAD = false>
@@ -234,7 +234,6 @@ layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamm
     constexpr int WARPS_PER_GROUP = GROUP / kWarp;
     constexpr bool SWEEP1 = GROUP >= 128;
     static_assert(GROUP % kWarp == 0 && THREADS % GROUP == 0, "groups are whole warps");
-    static_assert(!FULL || GROUPS == 1, "FULL is for one row per CTA");
     // SWEEP1 alternates between two sets of slots by row, so that one barrier per row is enough:
     // a warp can be at most one barrier ahead of the slowest reader
     __shared__ float slots2[2][4][THREADS / kWarp];
@@ -361,7 +360,7 @@ layernorm_reg_kernel(const uint4* __restrict__ x, const uint4* __restrict__ gamm
         }
         const float rstd = rsqrtf(var + eps);
         // FULL: the row index is read again rather than kept in registers across the reductions
-        uint4* yr = y + (FULL ? (int64_t)cta_id_x() : row) * nvec;
+        uint4* yr = y + (FULL ? (int64_t)cta_id_x() * GROUPS + g : row) * nvec;
 #pragma unroll
         for (int k = 0; k < VPT; ++k) {
             const int i = t + k * GROUP;
