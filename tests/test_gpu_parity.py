@@ -447,6 +447,45 @@ def test_cluster_path_slices_and_limits(rows, D):
         assert ak.ak_softmax_choose_path(rows, D, True) == want
 
 
+@pytest.mark.parametrize("rows,D", [(66, 65544), (70, 100000), (65, 131080), (68, 36872), (72, 262152),
+                                    (66, 65539), (65, 100001), (67, 128257), (66, 50001)])
+def test_many_long_rows_ragged_slices(rows, D):
+    """More than 64 long rows take the many-row shapes of the cluster kernels (128-thread CTAs that
+    keep exponentials in registers for softmax, one exchange for LayerNorm) and, unaligned, the
+    staged or cluster-staged kernels from their per-op lengths on.  Ragged slices (the vectors of a
+    row not a multiple of the cluster size, edge elements at both ends), rows with a -inf half, a
+    constant row and a row with one huge entry; every op against the oracle on the dispatcher's
+    own choice."""
+    x, w = synth.rmsnorm_inputs(rows, D, synth.case_seed(31, rows * 131 + D))
+    x[1, : D // 2] = float("-inf")
+    x[2] = -7.5
+    x[3, D - 1] = 65024.0
+    x[4, 0] = 65024.0
+    xs = x.clone()
+    xr = torch.nan_to_num(x, neginf=-3.0)
+    _, g, b = synth.layernorm_inputs(1, D, 79)
+    ref_r = oracle.rmsnorm(synth.to_bits(xr), synth.to_bits(w), 1e-6)
+    ref_s = oracle.softmax(synth.to_bits(xs))
+    ref_l = oracle.layernorm(synth.to_bits(xr), synth.to_bits(g), synth.to_bits(b), 1e-5)
+    y, check = guarded((rows, D), torch.bfloat16, DEV)
+    ak.ak_rmsnorm_fwd(xr.to(DEV), w.to(DEV), y, eps=1e-6)
+    torch.cuda.synchronize()
+    check()
+    assert_bf16_close(y, ref_r, f"rmsnorm {rows}x{D}")
+    y, check = guarded((rows, D), torch.bfloat16, DEV)
+    ak.ak_softmax_fwd(xs.to(DEV), y)
+    torch.cuda.synchronize()
+    check()
+    assert_bf16_close(y, ref_s, f"softmax {rows}x{D}")
+    y, check = guarded((rows, D), torch.bfloat16, DEV)
+    ak.ak_layernorm_fwd(xr.to(DEV), g.to(DEV), b.to(DEV), y, eps=1e-5)
+    torch.cuda.synchronize()
+    check()
+    assert_bf16_close(y, ref_l, f"layernorm {rows}x{D}", tight=False)
+    assert torch.equal(y[2].view(torch.int16).cpu(), b.view(torch.int16))   # constant row: beta exactly
+    assert ak.ak_wait_timeouts() == 0
+
+
 def test_cluster_path_rejects_rows_it_cannot_hold():
     x = torch.zeros((1, 8), dtype=torch.bfloat16, device=DEV)           # one vector: nothing to split
     w = torch.ones((8,), dtype=torch.bfloat16, device=DEV)
