@@ -65,6 +65,36 @@ def test_softmax_dt_parity_all_paths(rows, D, dtype):
 
 
 @pytest.mark.parametrize("dtype", DTS)
+@pytest.mark.parametrize("rows,D", [(66, 65544), (65, 131080), (68, 36872), (66, 65539), (65, 100001)])
+def test_softmax_rmsnorm_dt_many_long_rows(rows, D, dtype):
+    """More than 64 long rows in fp16 / fp32: the many-row shapes of the cluster kernels (for the
+    16-bit types the softmax kernel keeps some exponentials in registers and evaluates one pair in
+    four of the others by a polynomial) and, unaligned, the staged kernels; ragged slices, a -inf
+    half and a constant row."""
+    x = synth.softmax_inputs(rows, D, synth.case_seed(33, rows * 131 + D), mask_frac=0.0, dtype=dtype)
+    x[1, : D // 2] = float("-inf")
+    x[2] = -7.5
+    x[3, D - 1] = 60000.0
+    ref = oracle.softmax_dt(synth.to_elems(x), NAME[dtype])
+    xd = x.to(DEV)
+    y, check = guarded((rows, D), dtype, DEV)
+    ak.ak_softmax_fwd_dt(xd, y)
+    torch.cuda.synchronize()
+    check()
+    assert_close_dt(y, ref, f"softmax {NAME[dtype]} {rows}x{D}")
+    assert bool((y[xd == float("-inf")] == 0).all()), "-inf entries must give exactly 0"
+    xr = torch.nan_to_num(x, neginf=-3.0)
+    _, w = synth.rmsnorm_inputs(1, D, 81, dtype=dtype)
+    refr = oracle.rmsnorm_dt(synth.to_elems(xr), synth.to_elems(w), 1e-6, NAME[dtype])
+    y, check = guarded((rows, D), dtype, DEV)
+    ak.ak_rmsnorm_fwd_dt(xr.to(DEV), w.to(DEV), y, eps=1e-6)
+    torch.cuda.synchronize()
+    check()
+    assert_close_dt(y, refr, f"rmsnorm {NAME[dtype]} {rows}x{D}")
+    assert ak.ak_wait_timeouts() == 0
+
+
+@pytest.mark.parametrize("dtype", DTS)
 @pytest.mark.parametrize("rows,V", XENT_SHAPES)
 def test_xent_dt_parity_row_and_split(rows, V, dtype):
     lg, tg = synth.xent_inputs(rows, V, synth.case_seed(14, rows * 131 + V), dtype=dtype)
