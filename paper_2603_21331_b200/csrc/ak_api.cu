@@ -82,6 +82,9 @@ int cluster_ctas(int64_t rows, int64_t row_bytes, int64_t split_from) {
     return C;
 }
 
+// false when AK_DISABLE_CLUSTERS switches the cluster layouts off
+bool clusters_enabled() { return cluster_ctas(1, kClusterFrom, kClusterFrom) > 1; }
+
 int sm_count() {
     static std::mutex mu;
     static int cached[64] = {0};

@@ -375,6 +375,7 @@ int cluster_ctas(int64_t rows, int64_t row_bytes, int64_t split_from);
 // rows longer than 64 KiB are always split (at exactly 64 KiB the one-CTA kernels are as fast or
 // faster: softmax 16384 x 32768 317 us against 338 us in clusters of two)
 constexpr int64_t kClusterFrom = 65536 + 16;
+bool clusters_enabled();   // false when AK_DISABLE_CLUSTERS switches the cluster layouts off
 int sm_count();  // SMs of the current device (cached per device)
 // per translation unit: has a bounded mbarrier wait of its kernels ever given up on this device?
 int rmsnorm_wait_timeouts();

@@ -1,6 +1,8 @@
 """Vocabulary-parallel cross-entropy on one GPU: the ranks' shards are processed one after the
 other (no kernel waits on another), their partial buffers stacked as the all-gather would, and
 the merge compared with the fp64 CPU checker on the FULL logits."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -87,3 +89,41 @@ def test_vocab_parallel_adversarial_and_determinism():
         again, mean2 = _vp(x.to(DEV), t.to(DEV), world, 2)
         assert torch.equal(loss.view(torch.int32), again.view(torch.int32))
         assert torch.equal(mean.view(torch.int32), mean2.view(torch.int32))
+
+
+@pytest.mark.parametrize("rows,world,ignore", [(1, 2, 0.0), (127, 8, 0.1), (1024, 8, 0.1), (1025, 3, 0.3), (4096, 8, 0.05),
+                                               (8192, 2, 0.0), (300, 8, 1.0)])
+def test_vocab_parallel_merge_and_mean_in_one_launch(rows, world, ignore):
+    """Up to 8192 rows the merge and the fixed-order mean run as one cluster launch.  Its losses
+    are, bit for bit, those of the merge kernel alone (what `want_mean=False` runs), and its mean
+    is, bit for bit, the fixed-order mean of those losses (the row-shard kernels: fp64 sum and count
+    of the counted rows, then their quotient); larger batches take two kernels and agree too."""
+    if os.environ.get("AK_DISABLE_CLUSTERS", "0") not in ("", "0"):
+        pytest.skip("the cluster layouts are switched off in this environment")
+    V = 2048 * world
+    lg, tg = synth.xent_inputs(rows, V, synth.case_seed(41, rows * 7 + world), ignore_frac=min(ignore, 0.999))
+    if ignore >= 1.0:
+        tg[:] = -100
+    ld, td = lg.to(DEV), tg.to(DEV)
+    parts = []
+    for rank in range(world):
+        b, e = parallel.shard_vocab(V, rank, world)
+        parts.append(ak.ak_xent_vp_partial(ld[:, b:e].contiguous(), td, b, V, 1))
+    stack = torch.stack(parts).contiguous()
+    n0 = ak.ak_launch_count()
+    loss, mean = ak.ak_xent_vp_merge(stack, td, V)
+    torch.cuda.synchronize()
+    assert ak.ak_launch_count() - n0 == 1
+    loss_only, none = ak.ak_xent_vp_merge(stack, td, V, want_mean=False)
+    assert none is None
+    assert torch.equal(loss.view(torch.int32), loss_only.view(torch.int32))
+    want = ak.ak_xent_mean_merge(ak.ak_xent_sum_count(loss_only, td).view(1, 2))
+    torch.cuda.synchronize()
+    assert torch.equal(mean.view(torch.int32), want.view(torch.int32)) or (torch.isnan(mean).all() and torch.isnan(want).all())
+    ref_rows, ref_mean, n = oracle.xent(synth.to_bits(lg), tg.numpy())
+    assert_loss_close(loss, ref_rows, f"vp merge+mean {rows} rows world {world}")
+    if n > 0:
+        assert abs(float(mean) - ref_mean) <= 1e-5 * max(1.0, abs(ref_mean))
+    else:
+        assert torch.isnan(mean).all()
+    assert ak.ak_wait_timeouts() == 0
